@@ -1,0 +1,412 @@
+"""CPU oracle for the ZipCache quantize-and-attend path.  TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, step-by-step restatement of what the paper defines, in NumPy.
+It shares no code with the CUDA library and must never be imported by the
+product path: only the tests, the smoke check and the benchmark's CPU-baseline
+leg may use it.
+
+Arithmetic: everything is fp64 on inputs widened exactly from fp16/bf16, except
+the quantiser (CSTQuant), which follows one fixed fp32 sequence with
+round-to-nearest-even and no fused operations so that integer codes can be
+compared bit for bit.
+
+Passages followed (paper section / equation / algorithm):
+  probe selection ............ Sec. 4.3 "random+recent" strategy, Alg. 2 line 1
+  probe attention ............ Eq. 9 (with the causal mask of Eq. 2 / Sec. 4.2)
+  accumulated score .......... Eq. 7
+  normalised score ........... Eq. 8
+  split by saliency ratio .... Alg. 2 "Split"
+  uniform quantisation ....... Eq. 5 (dequantisation subtracts the zero point)
+  channel normalisation ...... Eq. 6
+  CSTQuant ................... Alg. 1
+  decode concat / attention .. Eq. 3, Eq. 4, Alg. 3
+  streaming re-compression ... Alg. 3 (every `window` = 100 generated tokens)
+  overhead accounting ........ Appendix A, Eq. (A)-(C)
+
+Pins (see tests/test_oracle_pins.py): brute-force l x l causal attention, the
+Q = 0 harmonic-number closed form, row-sum invariants, the half-step bound,
+textbook per-row affine quantisation when all channel factors are 1, exact
+attention at 16 bits, permutation and split invariance, Appendix A's printed
+ratios.  Conventions that no printed value or closed form fixes are marked
+"parity unpinned" where they are made:
+  * GQA aggregation of Eq. 8 over the query heads of one KV head and the
+    splitmix64 probe sampler                       -- parity unpinned
+  * floor() rounding of the salient / probe counts -- parity unpinned
+  * integer zero point (vs. a float offset)         -- parity unpinned
+  * streaming-flush semantics (which 100 tokens, the 100th step being a probe
+    step)                                           -- parity unpinned
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_M64 = (1 << 64) - 1
+
+
+# --------------------------------------------------------------------------
+# Probe selection (Sec. 4.3, "random+recent tokens")
+# --------------------------------------------------------------------------
+def _splitmix64(seed: int):
+    state = seed & _M64
+    while True:
+        state = (state + 0x9E3779B97F4A7C15) & _M64
+        z = state
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+        yield z ^ (z >> 31)
+
+
+def probe_counts(l: int, rho_recent: float, rho_random: float) -> Tuple[int, int]:
+    """(n_recent, n_random): floor of ratio*l in double; at least one recent
+    probe so that the last token is always a probe.  parity unpinned (rounding)."""
+    n_rec = min(l, max(1, int(math.floor(rho_recent * l))))
+    n_rnd = min(l - n_rec, int(math.floor(rho_random * l)))
+    return n_rec, n_rnd
+
+
+def probe_positions(l: int, rho_recent: float, rho_random: float, seed: int) -> np.ndarray:
+    """Ascending probe positions: the last n_recent tokens plus n_random tokens
+    drawn without replacement from the rest by a partial Fisher-Yates shuffle
+    driven by splitmix64(seed).  parity unpinned (sampler is a convention)."""
+    n_rec, n_rnd = probe_counts(l, rho_recent, rho_random)
+    pool = l - n_rec
+    perm = list(range(pool))
+    gen = _splitmix64(seed)
+    for i in range(n_rnd):
+        j = i + next(gen) % (pool - i)
+        perm[i], perm[j] = perm[j], perm[i]
+    chosen = sorted(perm[:n_rnd])
+    return np.asarray(chosen + list(range(pool, l)), dtype=np.int32)
+
+
+# --------------------------------------------------------------------------
+# Saliency (Eq. 7, 8, 9)
+# --------------------------------------------------------------------------
+def probe_attention(Qp: np.ndarray, K: np.ndarray, P: Sequence[int]) -> np.ndarray:
+    """Eq. 9 for one head: rows of Softmax(Q_probe K^T / sqrt(d_k)) under the
+    causal mask (row of position p sees columns j <= p).  Qp [n_p,d], K [l,d]."""
+    Qp = np.asarray(Qp, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    l, d = K.shape
+    S = (Qp @ K.T) / math.sqrt(d)
+    A = np.zeros_like(S)
+    for r, p in enumerate(P):
+        row = S[r, : p + 1]
+        e = np.exp(row - row.max())
+        A[r, : p + 1] = e / e.sum()
+    return A
+
+
+def accumulated_scores(A_list: Sequence[np.ndarray]) -> np.ndarray:
+    """Eq. 7: column sums of the attention matrix (summed over the given heads)."""
+    return sum(A.sum(axis=0) for A in A_list)
+
+
+def structural_nnz(P: Sequence[int], l: int) -> np.ndarray:
+    """Number of probe rows whose causal span contains column j: #{r : p_r >= j}."""
+    P = np.asarray(P)
+    return np.asarray([(P >= j).sum() for j in range(l)], dtype=np.int64)
+
+
+def normalized_scores(Q_heads: np.ndarray, K: np.ndarray, P: Sequence[int]) -> np.ndarray:
+    """Eq. 8 with A replaced by A_probe (Eq. 9), for one KV head.
+
+    Q_heads [G,l,d] are the G query heads that read this KV head (GQA: their
+    column sums are added and the count is G * nnz; reduces to Eq. 8 when G=1).
+    """
+    Q_heads = np.asarray(Q_heads, dtype=np.float64)
+    l = K.shape[0]
+    G = Q_heads.shape[0]
+    P = np.asarray(P, dtype=np.int64)
+    if len(P) == 0 or P[-1] != l - 1:
+        raise ValueError("probe list must end at the last token")
+    col = accumulated_scores([probe_attention(Q_heads[g][P], K, P) for g in range(G)])
+    return col / (G * structural_nnz(P, l))
+
+
+def split_salient(p_tilde: np.ndarray, n_s: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Alg. 2 Split: the n_s tokens with the largest score are salient (ties go
+    to the lower index); both index lists are returned ascending."""
+    order = np.argsort(-np.asarray(p_tilde, dtype=np.float64), kind="stable")
+    sal = np.sort(order[:n_s]).astype(np.int32)
+    reg = np.sort(order[n_s:]).astype(np.int32)
+    return sal, reg
+
+
+def salient_count(ratio: float, n: int) -> int:
+    """floor(ratio * n) in double.  parity unpinned (rounding convention)."""
+    return int(math.floor(ratio * n))
+
+
+# --------------------------------------------------------------------------
+# CSTQuant (Alg. 1, Eq. 5, Eq. 6) -- normative fp32 sequence
+# --------------------------------------------------------------------------
+def cst_quant(X: np.ndarray, bits: int) -> Dict[str, np.ndarray]:
+    """Channel-separable tokenwise quantisation of X [n_tokens, d] to `bits`.
+
+    Every operation below is a single IEEE fp32 operation rounded to nearest
+    even; nothing is fused.  Returns c [d], s [n], z [n] (integer-valued fp32)
+    and codes [n,d] (uint8, 0..2^bits-1).
+    """
+    f32 = np.float32
+    X = np.asarray(X, dtype=f32)
+    n, d = X.shape
+    L = f32((1 << bits) - 1)
+    # Eq. 6: c_i = sqrt(max |X_i|) over the tokens of this subset; all-zero channel -> 1
+    m = np.abs(X).max(axis=0) if n > 0 else np.zeros(d, dtype=f32)
+    c = np.sqrt(m, dtype=f32)
+    c = np.where(m == f32(0), f32(1), c).astype(f32)
+    # Alg. 1: normalise each channel
+    Y = (X / c[None, :]).astype(f32)
+    # TokenQuant = Eq. 5 with min/max over one token's channels
+    mn = Y.min(axis=1) if n > 0 else np.zeros(0, dtype=f32)
+    mx = Y.max(axis=1) if n > 0 else np.zeros(0, dtype=f32)
+    s = ((mx - mn).astype(f32) / L).astype(f32)
+    flat = mx == mn
+    s = np.where(flat, np.where(mn != f32(0), np.abs(mn), f32(1)), s).astype(f32)
+    z = (-np.rint((mn / s).astype(f32))).astype(f32)
+    q = (np.rint((Y / s[:, None]).astype(f32)).astype(f32) + z[:, None]).astype(f32)
+    codes = np.minimum(np.maximum(q, f32(0)), L).astype(np.uint8)
+    return {"c": c, "s": s, "z": z, "codes": codes, "bits": bits, "pre_round": (Y / s[:, None]).astype(f32)}
+
+
+def cst_dequant(qd: Dict[str, np.ndarray]) -> np.ndarray:
+    """x_hat = c * ((code - z) * s) in fp64 (Eq. 5 read with the zero point
+    subtracted, then Alg. 1's rescale)."""
+    c = qd["c"].astype(np.float64)
+    s = qd["s"].astype(np.float64)
+    z = qd["z"].astype(np.float64)
+    codes = qd["codes"].astype(np.float64)
+    return c[None, :] * ((codes - z[:, None]) * s[:, None])
+
+
+def token_quant_reference_fp64(Y: np.ndarray, bits: int) -> np.ndarray:
+    """Eq. 5 per row in fp64 (used only to cross-check fp32 codes away from
+    rounding boundaries).  Returns the pre-clipping real value y/s + z."""
+    Y = np.asarray(Y, dtype=np.float64)
+    L = (1 << bits) - 1
+    mn = Y.min(axis=1)
+    mx = Y.max(axis=1)
+    s = (mx - mn) / L
+    flat = mx == mn
+    s = np.where(flat, np.where(mn != 0, np.abs(mn), 1.0), s)
+    z = -np.rint(mn / s)
+    return Y / s[:, None] + z[:, None]
+
+
+def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
+    """Canonical packing of codes [n,d] -> bytes [n, d*bits/8]: 4-bit element
+    2m in the low nibble and 2m+1 in the high nibble of byte m; 2-bit element
+    4m+j in bits [2j, 2j+1] of byte m."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    n, d = codes.shape
+    if bits == 4:
+        return (codes[:, 0::2] | (codes[:, 1::2] << 4)).astype(np.uint8)
+    if bits == 2:
+        return (codes[:, 0::4] | (codes[:, 1::4] << 2) | (codes[:, 2::4] << 4)
+                | (codes[:, 3::4] << 6)).astype(np.uint8)
+    if bits == 8:
+        return codes.copy()
+    raise ValueError("bits must be 2, 4 or 8")
+
+
+def unpack_codes(packed: np.ndarray, bits: int, d: int) -> np.ndarray:
+    packed = np.asarray(packed, dtype=np.uint8)
+    n = packed.shape[0]
+    out = np.zeros((n, d), dtype=np.uint8)
+    per = 8 // bits
+    mask = (1 << bits) - 1
+    for j in range(per):
+        out[:, j::per] = (packed >> (bits * j)) & mask
+    return out
+
+
+# --------------------------------------------------------------------------
+# Appendix A: storage accounting
+# --------------------------------------------------------------------------
+def quant_param_count(granularity: str, b: int, hd: int, l: int, n: int = 32) -> float:
+    """Number of quantisation parameters for ONE tensor X in R^{b x h x l x d}
+    (hd = h*d), as counted in Sec. 4.1 and Table 1: tokenwise 2bl, groupwise
+    2bhld/n, channelwise 2hd, channel-separable tokenwise hd + 2bl."""
+    if granularity == "token":
+        return 2 * b * l
+    if granularity == "group":
+        return 2 * b * hd * l / n
+    if granularity == "channel":
+        return 2 * hd
+    if granularity == "cst":
+        return hd + 2 * b * l
+    raise ValueError(granularity)
+
+
+def compression_ratio(k_granularity: str, v_granularity: str, b: int, hd: int, l: int,
+                      bits: int = 4, n: int = 32, param_bits: int = 16) -> float:
+    """Appendix A, Eq. (A)-(C): bits of the 16-bit K and V over bits of the
+    quantised K and V plus their quantisation parameters."""
+    full = 2 * b * hd * l * 16
+    data = 2 * b * hd * l * bits
+    params = (quant_param_count(k_granularity, b, hd, l, n)
+              + quant_param_count(v_granularity, b, hd, l, n))
+    return full / (data + params * param_bits)
+
+
+# --------------------------------------------------------------------------
+# One (batch, KV head) unit of the mixed-precision cache (Alg. 2, Alg. 3)
+# --------------------------------------------------------------------------
+class _Subset:
+    """Tokens of one precision class inside one segment."""
+
+    def __init__(self, idx: np.ndarray, K: np.ndarray, V: np.ndarray, bits: int):
+        self.idx = idx.astype(np.int32)
+        self.bits = bits
+        self.n = len(idx)
+        if bits == 16:
+            self.qK = self.qV = None
+            self.K_hat = np.asarray(K, dtype=np.float64)[idx]
+            self.V_hat = np.asarray(V, dtype=np.float64)[idx]
+        else:
+            self.qK = cst_quant(np.asarray(K, dtype=np.float32)[idx], bits)
+            self.qV = cst_quant(np.asarray(V, dtype=np.float32)[idx], bits)
+            self.K_hat = cst_dequant(self.qK)
+            self.V_hat = cst_dequant(self.qV)
+
+
+class _Segment:
+    def __init__(self, K, V, p_tilde, ratio, bits_hi, bits_lo):
+        n = K.shape[0]
+        self.n = n
+        self.p_tilde = np.asarray(p_tilde, dtype=np.float64)
+        n_s = salient_count(ratio, n)
+        sal, reg = split_salient(self.p_tilde, n_s)
+        self.hi = _Subset(sal, K, V, bits_hi)
+        self.lo = _Subset(reg, K, V, bits_lo)
+
+
+class UnitCache:
+    """Mixed-precision cache of one (batch, KV head) with its G query heads."""
+
+    def __init__(self, G: int, d: int, ratio: float, bits_hi: int = 4, bits_lo: int = 2,
+                 window: int = 100):
+        self.G, self.d, self.ratio = G, d, ratio
+        self.bits_hi, self.bits_lo, self.window = bits_hi, bits_lo, window
+        self.segments: List[_Segment] = []
+        self.tail_K = np.zeros((0, d), dtype=np.float64)
+        self.tail_V = np.zeros((0, d), dtype=np.float64)
+        self.i = 0
+        self.tail_colsum = np.zeros(window, dtype=np.float64)
+        self.tail_nnz = np.zeros(window, dtype=np.int64)
+        self.last_attention: Optional[np.ndarray] = None
+
+    # ---- Alg. 2 (without its FlashAttention output line) ----
+    def prefill_compress(self, Q_heads: np.ndarray, K: np.ndarray, V: np.ndarray,
+                         P: Sequence[int], salient_idx: Optional[np.ndarray] = None) -> None:
+        K = np.asarray(K, dtype=np.float64)
+        V = np.asarray(V, dtype=np.float64)
+        p_tilde = normalized_scores(Q_heads, K, P)
+        seg = _Segment(K, V, p_tilde, self.ratio, self.bits_hi, self.bits_lo)
+        if salient_idx is not None:  # staged tests: impose a given split
+            sal = np.sort(np.asarray(salient_idx, dtype=np.int32))
+            reg = np.setdiff1d(np.arange(K.shape[0], dtype=np.int32), sal)
+            seg.hi = _Subset(sal, K, V, self.bits_hi)
+            seg.lo = _Subset(reg, K, V, self.bits_lo)
+        self.segments = [seg]
+        self.tail_K = np.zeros((0, self.d), dtype=np.float64)
+        self.tail_V = np.zeros((0, self.d), dtype=np.float64)
+        self.i = 0
+        self.tail_colsum[:] = 0
+        self.tail_nnz[:] = 0
+
+    # ---- Eq. 3 / Alg. 3: the new token joins the cache at full precision ----
+    def append(self, k: np.ndarray, v: np.ndarray) -> None:
+        if self.tail_K.shape[0] >= self.window:
+            raise RuntimeError("tail full: flush must have happened")
+        self.tail_K = np.vstack([self.tail_K, np.asarray(k, dtype=np.float64)[None, :]])
+        self.tail_V = np.vstack([self.tail_V, np.asarray(v, dtype=np.float64)[None, :]])
+
+    def _all_kv(self) -> Tuple[np.ndarray, np.ndarray]:
+        Ks = [sub.K_hat for seg in self.segments for sub in (seg.hi, seg.lo)]
+        Vs = [sub.V_hat for seg in self.segments for sub in (seg.hi, seg.lo)]
+        return np.vstack(Ks + [self.tail_K]), np.vstack(Vs + [self.tail_V])
+
+    # ---- Eq. 4 / Alg. 3: attention over every cached token, then bookkeeping ----
+    def decode_attention(self, q_heads: np.ndarray, is_probe_step: bool) -> np.ndarray:
+        q = np.asarray(q_heads, dtype=np.float64)             # [G,d]
+        K_all, V_all = self._all_kv()
+        logits = (q @ K_all.T) / math.sqrt(self.d)             # [G,n]
+        logits -= logits.max(axis=1, keepdims=True)
+        e = np.exp(logits)
+        a = e / e.sum(axis=1, keepdims=True)
+        o = a @ V_all
+        self.last_attention = a
+        n_tail = self.tail_K.shape[0]
+        self.i += 1
+        # the last five steps of a window are always probe steps (this includes
+        # the window's final step, taken before the re-compression)
+        if self.i > self.window - 5 or is_probe_step:
+            if n_tail > 0:
+                self.tail_colsum[:n_tail] += a[:, a.shape[1] - n_tail:].sum(axis=0)
+                self.tail_nnz[:n_tail] += 1
+        if self.i == self.window:
+            self._flush()
+        return o
+
+    def _flush(self) -> None:
+        n = self.tail_K.shape[0]
+        assert n == self.window
+        p_tilde = self.tail_colsum[:n] / (self.G * self.tail_nnz[:n])
+        self.segments.append(_Segment(self.tail_K, self.tail_V, p_tilde, self.ratio,
+                                      self.bits_hi, self.bits_lo))
+        self.tail_K = np.zeros((0, self.d), dtype=np.float64)
+        self.tail_V = np.zeros((0, self.d), dtype=np.float64)
+        self.i = 0
+        self.tail_colsum[:] = 0
+        self.tail_nnz[:] = 0
+
+
+def exact_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """Eq. 4 written out: softmax(q K^T / sqrt(d)) V for q [G,d]."""
+    q = np.asarray(q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    logits = (q @ K.T) / math.sqrt(K.shape[1])
+    logits -= logits.max(axis=1, keepdims=True)
+    e = np.exp(logits)
+    return (e / e.sum(axis=1, keepdims=True)) @ V
+
+
+# --------------------------------------------------------------------------
+# Whole-tensor convenience wrapper: [b, h, ...] tensors -> independent units
+# --------------------------------------------------------------------------
+class ZipCacheOracle:
+    """All (batch, KV head) units of one attention layer; units are independent."""
+
+    def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, ratio: float,
+                 bits_hi: int = 4, bits_lo: int = 2, window: int = 100,
+                 units: Optional[Sequence[Tuple[int, int]]] = None):
+        self.b, self.hq, self.hkv, self.d = batch, n_q_heads, n_kv_heads, head_dim
+        self.G = n_q_heads // n_kv_heads
+        self.unit_ids = list(units) if units is not None else [
+            (bi, kv) for bi in range(batch) for kv in range(n_kv_heads)]
+        self.units = {u: UnitCache(self.G, head_dim, ratio, bits_hi, bits_lo, window)
+                      for u in self.unit_ids}
+
+    def prefill_compress(self, Q, K, V, P, salient_idx=None) -> None:
+        """Q [b,h_q,l,d], K,V [b,h_kv,l,d] (float arrays); P ascending probe list."""
+        for (bi, kv) in self.unit_ids:
+            sal = None if salient_idx is None else salient_idx[bi][kv]
+            self.units[(bi, kv)].prefill_compress(
+                Q[bi, kv * self.G:(kv + 1) * self.G], K[bi, kv], V[bi, kv], P, sal)
+
+    def append(self, k, v) -> None:
+        for (bi, kv) in self.unit_ids:
+            self.units[(bi, kv)].append(k[bi, kv], v[bi, kv])
+
+    def decode_attention(self, q, is_probe_step: bool) -> Dict[Tuple[int, int], np.ndarray]:
+        out = {}
+        for (bi, kv) in self.unit_ids:
+            out[(bi, kv)] = self.units[(bi, kv)].decode_attention(
+                q[bi, kv * self.G:(kv + 1) * self.G], is_probe_step)
+        return out

@@ -1,0 +1,481 @@
+"""Pins for the CPU oracle: each test ties a part of it to something other than
+itself -- a value the paper prints, a closed form, brute force on tiny inputs,
+a library routine for a special case, or an invariant of the mathematics."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import zipcache_oracle as zo
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rng(seed):
+    return np.random.RandomState(seed)
+
+
+# ---------------------------------------------------------------- Eq. 8 / 9
+def _brute_force_causal_attention(Q, K):
+    """l x l causal softmax attention with pure Python loops (Eq. 2 + mask)."""
+    l, d = K.shape
+    A = [[0.0] * l for _ in range(l)]
+    for i in range(l):
+        logits = []
+        for j in range(i + 1):
+            acc = 0.0
+            for c in range(d):
+                acc += float(Q[i, c]) * float(K[j, c])
+            logits.append(acc / math.sqrt(d))
+        mx = max(logits)
+        es = [math.exp(v - mx) for v in logits]
+        tot = sum(es)
+        for j in range(i + 1):
+            A[i][j] = es[j] / tot
+    return A
+
+
+@pytest.mark.parametrize("l,d,seed", [(1, 4, 0), (2, 4, 1), (17, 8, 2), (24, 16, 3)])
+def test_normalized_score_matches_brute_force_full_matrix(l, d, seed):
+    """Eq. 8 on the explicit l x l lower-triangular matrix (all tokens probes)."""
+    rs = _rng(seed)
+    Q = rs.standard_normal((l, d))
+    K = rs.standard_normal((l, d))
+    A = _brute_force_causal_attention(Q, K)
+    expect = []
+    for j in range(l):
+        col = [A[i][j] for i in range(l)]
+        nnz = sum(1 for i in range(l) if i >= j)      # lower triangle incl. diagonal
+        expect.append(sum(col) / nnz)
+    got = zo.normalized_scores(Q[None], K, np.arange(l))
+    np.testing.assert_allclose(got, np.asarray(expect), rtol=1e-12, atol=0)
+
+
+def test_probe_subset_matches_brute_force_rows():
+    """Eq. 9 substituted into Eq. 8 with a strict subset of rows."""
+    l, d = 20, 8
+    rs = _rng(5)
+    Q = rs.standard_normal((l, d))
+    K = rs.standard_normal((l, d))
+    P = [3, 7, 8, 15, 19]
+    A = _brute_force_causal_attention(Q, K)
+    expect = np.zeros(l)
+    for j in range(l):
+        rows = [p for p in P if p >= j]
+        expect[j] = sum(A[p][j] for p in rows) / len(rows)
+    got = zo.normalized_scores(Q[None], K, P)
+    np.testing.assert_allclose(got, expect, rtol=1e-12)
+
+
+def test_zero_query_closed_form_harmonic():
+    """Q = 0 makes row r uniform over r+1 columns, so with all rows probes
+    p~_j = (H_l - H_j) / (l - j) and the accumulated score is H_l - H_j."""
+    l, d = 40, 8
+    K = _rng(7).standard_normal((l, d))
+    Q = np.zeros((1, l, d))
+    H = np.concatenate([[0.0], np.cumsum(1.0 / np.arange(1, l + 1))])
+    j = np.arange(l)
+    expect = (H[l] - H[j]) / (l - j)
+    got = zo.normalized_scores(Q, K, np.arange(l))
+    np.testing.assert_allclose(got, expect, rtol=1e-13)
+    acc = zo.accumulated_scores([zo.probe_attention(Q[0], K, np.arange(l))])
+    np.testing.assert_allclose(acc, H[l] - H[j], rtol=1e-13)
+    # the bias the paper describes (Sec. 4.2): first token's accumulated score
+    # exceeds 1 and always exceeds the last token's
+    assert acc[0] > 1.0 and acc[0] > acc[-1]
+    assert abs(acc[-1] - 1.0 / l) < 1e-15
+
+
+def test_probe_attention_invariants_and_gqa_reduction():
+    l, d, G = 33, 16, 4
+    rs = _rng(11)
+    Q = rs.standard_normal((G, l, d))
+    K = rs.standard_normal((l, d))
+    P = zo.probe_positions(l, 0.2, 0.2, 99)
+    assert P[-1] == l - 1
+    As = [zo.probe_attention(Q[g][P], K, P) for g in range(G)]
+    for A in As:
+        np.testing.assert_allclose(A.sum(axis=1), 1.0, rtol=1e-13)
+        for r, p in enumerate(P):
+            assert np.all(A[r, p + 1:] == 0.0)
+            assert np.all(A[r, : p + 1] > 0.0)
+    col = zo.accumulated_scores(As)
+    assert abs(col.sum() - G * len(P)) < 1e-10
+    # GQA aggregate = mean over heads of the single-head Eq. 8 score
+    per_head = np.stack([zo.normalized_scores(Q[g:g + 1], K, P) for g in range(G)])
+    np.testing.assert_allclose(zo.normalized_scores(Q, K, P), per_head.mean(axis=0), rtol=1e-12)
+    # l = 1
+    assert zo.normalized_scores(np.ones((1, 1, d)), np.ones((1, d)), [0])[0] == 1.0
+
+
+def test_normalized_scores_rejects_list_not_ending_at_last_token():
+    with pytest.raises(ValueError):
+        zo.normalized_scores(np.zeros((1, 8, 4)), np.zeros((8, 4)), [1, 2, 3])
+
+
+def test_structural_nnz_counts_unmasked_rows():
+    assert zo.structural_nnz([2, 5, 9], 10).tolist() == [3, 3, 3, 2, 2, 2, 1, 1, 1, 1]
+
+
+# ---------------------------------------------------------------- probe sampler
+@pytest.mark.parametrize("l", [1, 2, 17, 100, 512, 4096])
+def test_probe_positions_structure(l):
+    P = zo.probe_positions(l, 0.05, 0.05, 1234)
+    n_rec, n_rnd = zo.probe_counts(l, 0.05, 0.05)
+    assert n_rec == max(1, int(0.05 * l)) and n_rnd == min(l - n_rec, int(0.05 * l))
+    assert len(P) == n_rec + n_rnd
+    assert np.all(np.diff(P) > 0)                       # ascending, unique
+    assert P[-n_rec:].tolist() == list(range(l - n_rec, l))
+    assert np.all(P[:n_rnd] < l - n_rec)
+    # deterministic, seed-dependent
+    assert np.array_equal(P, zo.probe_positions(l, 0.05, 0.05, 1234))
+    if n_rnd > 4:
+        assert not np.array_equal(P, zo.probe_positions(l, 0.05, 0.05, 1235))
+
+
+def test_probe_counts_at_benchmark_lengths():
+    assert zo.probe_counts(512, 0.05, 0.05) == (25, 25)
+    assert zo.probe_counts(4096, 0.05, 0.05) == (204, 204)
+    assert zo.probe_counts(8192, 0.05, 0.05) == (409, 409)
+    assert zo.probe_counts(32768, 0.05, 0.05) == (1638, 1638)
+
+
+def test_probe_sampler_is_roughly_uniform():
+    hits = np.zeros(50)
+    for seed in range(400):
+        P = zo.probe_positions(60, 1 / 6, 0.2, seed)   # 10 recent, 12 random of 50
+        hits[P[:12]] += 1
+    assert hits.min() > 50 and hits.max() < 150          # expectation 96 each
+
+
+# ---------------------------------------------------------------- split
+def test_split_salient_brute_force_and_ties():
+    rs = _rng(3)
+    for trial in range(30):
+        n = int(rs.randint(1, 40))
+        p = rs.randint(0, 6, size=n).astype(np.float64) / 4.0   # many ties
+        n_s = int(rs.randint(0, n + 1))
+        keyed = sorted(range(n), key=lambda j: (-p[j], j))
+        sal, reg = zo.split_salient(p, n_s)
+        assert sal.tolist() == sorted(keyed[:n_s])
+        assert reg.tolist() == sorted(keyed[n_s:])
+        assert len(set(sal) & set(reg)) == 0 and len(sal) + len(reg) == n
+        if 0 < n_s < n:
+            assert p[sal].min() >= p[reg].max()
+
+
+def test_salient_counts_at_benchmark_lengths():
+    assert zo.salient_count(0.4, 512) == 204
+    assert zo.salient_count(0.4, 4096) == 1638
+    assert zo.salient_count(0.3, 8192) == 2457
+    assert zo.salient_count(0.4, 32768) == 13107
+    assert zo.salient_count(0.4, 100) == 40
+    assert zo.salient_count(0.0, 100) == 0 and zo.salient_count(1.0, 100) == 100
+
+
+# ---------------------------------------------------------------- CSTQuant
+def _outlier_matrix(n, d, seed, dtype=torch.float16):
+    rs = _rng(seed)
+    X = rs.standard_normal((n, d))
+    X[:, rs.choice(d, 3, replace=False)] *= 15.0
+    return torch.tensor(X).to(dtype).to(torch.float32).numpy()
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("n,d", [(1, 8), (5, 16), (64, 128), (201, 128)])
+def test_cst_quant_half_step_bound_and_code_range(bits, n, d):
+    X = _outlier_matrix(n, d, 17 + bits + n)
+    q = zo.cst_quant(X, bits)
+    L = (1 << bits) - 1
+    c, s, z, codes = (q[k].astype(np.float64) for k in ("c", "s", "z", "codes"))
+    assert codes.min() >= 0 and codes.max() <= L
+    Y = X.astype(np.float64) / c[None, :]
+    recon = (codes - z[:, None]) * s[:, None]
+    # |y - (code - z) s| <= s/2 (tiny slack for the fp32 division that formed y)
+    assert np.all(np.abs(Y - recon) <= s[:, None] * (0.5 + 1e-5))
+    # each token's smallest channel maps to code 0 and its largest to L
+    for t in range(n):
+        if Y[t].max() > Y[t].min():
+            assert codes[t, Y[t].argmin()] == 0 and codes[t, Y[t].argmax()] == L
+            order = np.argsort(Y[t], kind="stable")
+            assert np.all(np.diff(codes[t, order]) >= 0)        # monotone in y
+    # z is an integer; dequantised values restore each channel's magnitude
+    assert np.all(z == np.rint(z))
+    X_hat = zo.cst_dequant(q)
+    assert np.all(np.abs(X_hat - X) <= c[None, :] * s[:, None] * (0.5 + 1e-5))
+
+
+def test_channel_factor_is_sqrt_of_channel_absmax_and_roundtrips():
+    X = _outlier_matrix(50, 32, 23)
+    q = zo.cst_quant(X, 4)
+    np.testing.assert_array_equal(q["c"], np.sqrt(np.abs(X).max(axis=0)).astype(np.float32))
+    c = q["c"]
+    back = (X / c[None, :]).astype(np.float32) * c[None, :]
+    ulp = np.spacing(np.abs(X).astype(np.float32))
+    assert np.all(np.abs(back.astype(np.float64) - X) <= ulp)   # c * (x / c) = x to 1 ulp
+    # after normalisation every channel's magnitude is sqrt of what it was (Eq. 6)
+    Y = X / c[None, :]
+    np.testing.assert_allclose(np.abs(Y).max(axis=0), c, rtol=1e-6)
+
+
+def test_degenerate_rows_and_channels():
+    X = np.zeros((3, 8), dtype=np.float32)
+    X[1, :] = 2.5          # constant token
+    X[2, :] = -0.75        # constant negative token
+    q = zo.cst_quant(X, 2)
+    assert np.all(q["c"] == np.sqrt(np.float32(2.5)))
+    # constant rows (after normalisation) reconstruct exactly up to fp32 rounding of y
+    np.testing.assert_allclose(zo.cst_dequant(q), X, rtol=1e-6, atol=0)
+    assert np.all(q["codes"] == 0)
+    Z = np.zeros((3, 8), dtype=np.float32)
+    qz = zo.cst_quant(Z, 4)
+    assert np.all(qz["c"] == 1) and np.all(qz["s"] == 1) and np.all(qz["codes"] == 0)
+    assert np.all(zo.cst_dequant(qz) == 0)
+    # empty subset
+    qe = zo.cst_quant(np.zeros((0, 8), dtype=np.float32), 4)
+    assert qe["codes"].shape == (0, 8) and np.all(qe["c"] == 1)
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_unit_channel_factors_reduce_to_library_affine_quantiser(bits):
+    """With every |channel| max equal to 1 the factors are 1 and CSTQuant is
+    plain asymmetric per-row uniform quantisation; torch's per-channel fake
+    quantiser (axis = token) is the library statement of Eq. 5."""
+    rs = _rng(31)
+    n, d = 37, 24
+    X = rs.uniform(-1, 1, size=(n, d)).astype(np.float32)
+    X[rs.randint(0, n, size=d), np.arange(d)] = np.where(rs.rand(d) < 0.5, -1.0, 1.0)
+    q = zo.cst_quant(X, bits)
+    assert np.all(q["c"] == 1.0)
+    L = (1 << bits) - 1
+    xt = torch.tensor(X)
+    got = torch.fake_quantize_per_channel_affine(
+        xt, torch.tensor(q["s"]), torch.tensor(q["z"]).to(torch.int32), 0, 0, L).numpy()
+    np.testing.assert_allclose(zo.cst_dequant(q), got.astype(np.float64), rtol=0, atol=1e-6)
+    # and the parameters are Eq. 5's: s = (max - min) / (2^k - 1), z = -round(min / s)
+    for t in range(n):
+        assert abs(q["s"][t] - (X[t].max() - X[t].min()) / L) <= 1e-7
+        assert q["z"][t] == -round(float(np.float32(X[t].min()) / q["s"][t]))
+
+
+def test_fp32_codes_agree_with_fp64_away_from_rounding_boundaries():
+    X = _outlier_matrix(300, 128, 41, dtype=torch.bfloat16)
+    for bits in (2, 4):
+        q = zo.cst_quant(X, bits)
+        L = (1 << bits) - 1
+        Y = X.astype(np.float64) / q["c"].astype(np.float64)[None, :]
+        real = zo.token_quant_reference_fp64(Y, bits)
+        frac = np.abs(real - np.floor(real) - 0.5)
+        safe = frac > 1e-4
+        expect = np.clip(np.rint(real), 0, L)
+        assert safe.mean() > 0.99
+        assert np.array_equal(q["codes"][safe], expect[safe].astype(np.uint8))
+
+
+def test_round_half_to_even_is_used():
+    """A single token with x_i = y_i |y_i| has c_i = |y_i| and normalised values
+    y exactly; y = (0, .5, 1.5, 2.5, 3.5, 15) at 4 bits gives s = 1, z = 0 and
+    codes that sit on .5 boundaries: ties must go to the even integer."""
+    Y = np.array([[0.0, 0.5, 1.5, 2.5, 3.5, 15.0]], dtype=np.float32)
+    X = (Y * np.abs(Y)).astype(np.float32)
+    q = zo.cst_quant(X, 4)
+    assert q["s"][0] == 1.0 and q["z"][0] == 0.0
+    assert q["codes"][0].tolist() == [0, 0, 2, 2, 4, 15]
+
+
+def test_pack_unpack_canonical_layout():
+    codes = np.arange(16, dtype=np.uint8).reshape(1, 16) % 16
+    p4 = zo.pack_codes(codes, 4)
+    assert p4[0, 0] == (0 | (1 << 4)) and p4[0, 7] == (14 | (15 << 4))
+    c2 = (np.arange(16, dtype=np.uint8).reshape(1, 16)) % 4
+    p2 = zo.pack_codes(c2, 2)
+    assert p2[0, 0] == (0 | (1 << 2) | (2 << 4) | (3 << 6))
+    for bits, c in ((4, codes), (2, c2)):
+        assert np.array_equal(zo.unpack_codes(zo.pack_codes(c, bits), bits, 16), c)
+
+
+# ---------------------------------------------------------------- Appendix A
+def test_appendix_a_printed_ratios():
+    rows = {}
+    with open(os.path.join(GOLDEN, "appendix_a_ratios.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, v = line.split()
+                rows[k] = float(v)
+    got = {
+        "group": zo.compression_ratio("group", "group", 8, 4096, 4096, 4, 32, 16),
+        "token": zo.compression_ratio("token", "token", 8, 4096, 4096, 4, 32, 16),
+        "baseline": zo.compression_ratio("channel", "cst", 8, 4096, 4096, 4, 32, 16),
+    }
+    for k, v in rows.items():
+        assert round(got[k], 3) == v, (k, got[k], v)
+
+
+def test_table1_parameter_counts():
+    b, hd, l, n = 8, 4096, 4096, 32
+    want = {}
+    with open(os.path.join(GOLDEN, "table1_param_counts.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                name, _, val = line.split()
+                want[name] = int(val)
+    pc = zo.quant_param_count
+    assert pc("token", b, hd, l, n) == want["tokenwise_one_tensor"]
+    assert pc("group", b, hd, l, n) == want["groupwise_one_tensor"]
+    assert pc("cst", b, hd, l, n) == want["cst_one_tensor"]
+    assert pc("channel", b, hd, l, n) + pc("cst", b, hd, l, n) == want["channel_K_plus_cst_V"]
+    assert 2 * pc("token", b, hd, l, n) == want["tokenwise_K_and_V"]
+    assert 2 * pc("group", b, hd, l, n) == want["groupwise_K_and_V"]
+
+
+# ---------------------------------------------------------------- decode (Eq. 4, Alg. 3)
+def _small_unit(G=2, d=16, l=48, ratio=0.5, bits=(4, 2), window=100, seed=0):
+    rs = _rng(seed)
+    Q = rs.standard_normal((G, l, d))
+    K = _outlier_matrix(l, d, seed + 1).astype(np.float64)
+    V = rs.standard_normal((l, d)).astype(np.float32).astype(np.float64)
+    P = zo.probe_positions(l, 0.1, 0.1, seed)
+    u = zo.UnitCache(G, d, ratio, bits[0], bits[1], window)
+    u.prefill_compress(Q, K, V, P)
+    return u, Q, K, V, rs
+
+
+def test_all_tokens_16_bit_equals_library_attention():
+    """bits_hi = 16 with every token salient: decode must be exact attention."""
+    G, d, l = 4, 32, 70
+    u, Q, K, V, rs = _small_unit(G, d, l, ratio=1.0, bits=(16, 2), seed=3)
+    assert u.segments[0].lo.n == 0
+    ks, vs = [], []
+    for step in range(5):
+        k, v, q = rs.standard_normal(d), rs.standard_normal(d), rs.standard_normal((G, d))
+        ks.append(k), vs.append(v)
+        u.append(k, v)
+        o = u.decode_attention(q, False)
+        K_all = torch.tensor(np.vstack([K] + ks))
+        V_all = torch.tensor(np.vstack([V] + vs))
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.tensor(q)[None, :, None, :], K_all[None, None].expand(1, G, -1, -1),
+            V_all[None, None].expand(1, G, -1, -1))[0, :, 0, :].numpy()
+        np.testing.assert_allclose(o, ref, rtol=1e-10, atol=1e-12)
+        np.testing.assert_allclose(o, zo.exact_attention(q, K_all.numpy(), V_all.numpy()),
+                                   rtol=1e-12)
+
+
+def test_decode_equals_exact_attention_over_dequantised_cache_and_is_order_free():
+    u, Q, K, V, rs = _small_unit(seed=5)
+    seg = u.segments[0]
+    # rebuild the dequantised cache in ORIGINAL token order
+    K_hat = np.zeros_like(K)
+    V_hat = np.zeros_like(V)
+    for sub in (seg.hi, seg.lo):
+        K_hat[sub.idx] = sub.K_hat
+        V_hat[sub.idx] = sub.V_hat
+    k, v, q = rs.standard_normal(16), rs.standard_normal(16), rs.standard_normal((2, 16))
+    u.append(k, v)
+    o = u.decode_attention(q, False)
+    ref = zo.exact_attention(q, np.vstack([K_hat, k]), np.vstack([V_hat, v]))
+    np.testing.assert_allclose(o, ref, rtol=1e-11, atol=1e-13)
+    # any split of the tokens merged by (max, sum, weighted acc) gives the same result
+    Kc, Vc = np.vstack([K_hat, k]), np.vstack([V_hat, v])
+    parts = [(0, 10), (10, 11), (11, 49)]
+    m = np.full(2, -np.inf)
+    ssum = np.zeros(2)
+    acc = np.zeros((2, 16))
+    for a, b in parts:
+        lg = q @ Kc[a:b].T / math.sqrt(16)
+        m_new = np.maximum(m, lg.max(axis=1))
+        scale = np.exp(m - m_new)
+        e = np.exp(lg - m_new[:, None])
+        ssum = ssum * scale + e.sum(axis=1)
+        acc = acc * scale[:, None] + e @ Vc[a:b]
+        m = m_new
+    np.testing.assert_allclose(acc / ssum[:, None], o, rtol=1e-11)
+    # quantisation error is bounded through the half-step bound (sanity, not parity)
+    exact = zo.exact_attention(q, np.vstack([K, k]), np.vstack([V, v]))
+    assert np.abs(o - exact).max() < 1.0
+
+
+def test_folded_dequantisation_algebra():
+    """q . k_hat = s_t (q' . code - z_t sum q') with q' = q * c^K, and
+    o = c^V * (sum_t w_t code_t - sum_t w_t z_t) with w_t = a_t s_t."""
+    u, Q, K, V, rs = _small_unit(G=1, seed=9)
+    sub = u.segments[0].lo
+    q = rs.standard_normal(16)
+    qK, qV = sub.qK, sub.qV
+    qp = q * qK["c"].astype(np.float64)
+    dots = qK["codes"].astype(np.float64) @ qp
+    logits_folded = qK["s"].astype(np.float64) * (dots - qK["z"].astype(np.float64) * qp.sum())
+    np.testing.assert_allclose(logits_folded, sub.K_hat @ q, rtol=1e-9, atol=1e-11)
+    a = np.exp(logits_folded - logits_folded.max())
+    a /= a.sum()
+    w = a * qV["s"].astype(np.float64)
+    o_folded = qV["c"].astype(np.float64) * (w @ qV["codes"].astype(np.float64)
+                                             - (w * qV["z"].astype(np.float64)).sum())
+    np.testing.assert_allclose(o_folded, a @ sub.V_hat, rtol=1e-9, atol=1e-11)
+
+
+def test_streaming_flush_matches_window_submatrix():
+    """With every decode step a probe step, the flushed window's score is Eq. 8
+    on the window's columns of the decode-time attention rows (brute force here),
+    and the window becomes a new segment with floor(r * window) salient tokens."""
+    window, G, d = 8, 2, 16
+    u, Q, K, V, rs = _small_unit(G=G, d=d, l=30, ratio=0.5, window=window, seed=13)
+    rows = []
+    toks = []
+    for step in range(window):
+        k, v, q = rs.standard_normal(d), rs.standard_normal(d), rs.standard_normal((G, d))
+        toks.append((k, v))
+        u.append(k, v)
+        n_before = len(u.segments)
+        u.decode_attention(q, True)
+        rows.append(u.last_attention[:, -(step + 1):].copy())    # window columns so far
+    assert len(u.segments) == n_before + 1 and u.tail_K.shape[0] == 0 and u.i == 0
+    colsum = np.zeros(window)
+    nnz = np.zeros(window)
+    for step, a in enumerate(rows):
+        colsum[: step + 1] += a.sum(axis=0)
+        nnz[: step + 1] += 1
+    expect = colsum / (G * nnz)
+    seg = u.segments[-1]
+    np.testing.assert_allclose(seg.p_tilde, expect, rtol=1e-12)
+    assert nnz.tolist() == [window - j for j in range(window)]
+    assert seg.hi.n == 4 and seg.lo.n == 4
+    sal, reg = zo.split_salient(expect, 4)
+    assert np.array_equal(seg.hi.idx, sal) and np.array_equal(seg.lo.idx, reg)
+    Kw = np.stack([t[0] for t in toks]).astype(np.float32)
+    np.testing.assert_array_equal(seg.hi.qK["codes"], zo.cst_quant(Kw[sal], 4)["codes"])
+
+
+def test_probe_steps_without_flags_are_only_the_last_five():
+    window, G, d = 10, 1, 8
+    u, Q, K, V, rs = _small_unit(G=G, d=d, l=12, ratio=0.5, window=window, seed=17)
+    seen = []
+    for step in range(window - 1):
+        u.append(rs.standard_normal(d), rs.standard_normal(d))
+        u.decode_attention(rs.standard_normal((G, d)), False)
+        seen.append(u.tail_nnz.copy())
+    # steps 1..5 collect nothing; steps 6..9 (i > window-5) do
+    assert seen[4].sum() == 0
+    assert seen[5][:6].tolist() == [1] * 6 and seen[5][6:].sum() == 0
+    assert seen[8][:6].tolist() == [4] * 6 and seen[8][8] == 1
+
+
+def test_multi_unit_wrapper_keeps_units_independent():
+    b, hq, hkv, d, l = 2, 4, 2, 16, 40
+    rs = _rng(21)
+    Q = rs.standard_normal((b, hq, l, d))
+    K = rs.standard_normal((b, hkv, l, d)).astype(np.float32).astype(np.float64)
+    V = rs.standard_normal((b, hkv, l, d)).astype(np.float32).astype(np.float64)
+    P = zo.probe_positions(l, 0.1, 0.1, 5)
+    full = zo.ZipCacheOracle(b, hq, hkv, d, 0.4)
+    full.prefill_compress(Q, K, V, P)
+    one = zo.ZipCacheOracle(b, hq, hkv, d, 0.4, units=[(1, 0)])
+    one.prefill_compress(Q, K, V, P)
+    np.testing.assert_array_equal(full.units[(1, 0)].segments[0].hi.qK["codes"],
+                                  one.units[(1, 0)].segments[0].hi.qK["codes"])
+    single = zo.UnitCache(2, d, 0.4)
+    single.prefill_compress(Q[1, 0:2], K[1, 0], V[1, 0], P)
+    np.testing.assert_array_equal(single.segments[0].p_tilde,
+                                  full.units[(1, 0)].segments[0].p_tilde)
