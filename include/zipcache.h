@@ -1,0 +1,144 @@
+/*
+ * zipcache.h -- C ABI of the B200 (sm_100a) quantize-and-attend library.
+ *
+ * The library implements the mixed-precision KV-cache path of ZipCache:
+ *   prefill:  probe attention (Eq. 9) -> normalised attention score (Eq. 8)
+ *             -> split by saliency ratio (Alg. 2) -> channel-separable tokenwise
+ *             quantisation (Alg. 1, Eq. 5, Eq. 6) -> packed 4-bit / 2-bit codes;
+ *   decode:   append of the new token at full precision (Eq. 3, Alg. 3),
+ *             single-query attention over the whole cache with in-kernel
+ *             dequantisation (Eq. 4, Alg. 3), probe-row collection and the
+ *             re-compression of every `window` generated tokens (Alg. 3).
+ *
+ * Conventions
+ *   - "unit" = one (batch, KV head).  Query head h reads KV head h / G,
+ *     G = n_q_heads / n_kv_heads.
+ *   - Every pointer is tagged [host] or [device].  The library never allocates
+ *     or frees device memory and never creates streams: the caller owns the
+ *     cache buffer and the workspace, and all work is enqueued on the stream
+ *     passed in.  Inputs may be released once the stream has passed the call.
+ *   - Every function returns 0 (ZC_OK) or a negative status; nothing throws
+ *     and device code never traps.  NaN / Inf in inputs give undefined values
+ *     but no fault.
+ *   - Device pointers must be 16-byte aligned (ZC_EALIGN otherwise).
+ */
+#ifndef ZIPCACHE_H_
+#define ZIPCACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* zc_stream_t; /* a cudaStream_t */
+
+enum { ZC_F16 = 0, ZC_BF16 = 1 };
+
+enum {
+  ZC_OK = 0,
+  ZC_EINVAL = -1,    /* bad shape / ratio / bit-width / stride / probe list */
+  ZC_ECAPACITY = -2, /* more tokens than the cache or workspace was sized for */
+  ZC_ESTATE = -3,    /* call out of order (e.g. decode before prefill) */
+  ZC_EALIGN = -4,    /* pointer not 16-byte aligned */
+  ZC_ECUDA = -5      /* a CUDA runtime call or launch failed */
+};
+
+#define ZC_MAX_WINDOW 128
+
+/* Plain-data configuration; set struct_size = sizeof(zc_config). */
+typedef struct {
+  int32_t struct_size;
+  int32_t dtype;          /* ZC_F16 | ZC_BF16: type of Q, K, V, q, k, v, out */
+  int32_t batch;          /* b */
+  int32_t n_q_heads;      /* h_q, multiple of n_kv_heads, G <= 8 */
+  int32_t n_kv_heads;     /* h_kv */
+  int32_t head_dim;       /* d, must be 128 */
+  int32_t max_prefill;    /* largest l accepted by zc_prefill_compress */
+  int32_t max_new_tokens; /* decode capacity (tokens appended after prefill) */
+  int32_t window;         /* tokens kept at full precision before re-compression
+                             (Alg. 3 uses 100); 8 <= window <= ZC_MAX_WINDOW */
+  int32_t bits_hi;        /* bit-width of salient tokens: 4 or 2 */
+  int32_t bits_lo;        /* bit-width of regular tokens: 4 or 2 */
+  int32_t reserved;       /* must be 0 */
+  double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
+} zc_config;
+
+typedef struct zc_cache zc_cache; /* small host-side handle */
+
+/* Sizes [host].  cache_bytes: device buffer for the compressed cache;
+ * workspace_bytes: device scratch shared by all calls (probe-row statistics in
+ * prefill, split-K partial results in decode).  Either out pointer may be NULL. */
+int zc_cache_bytes(const zc_config* cfg, size_t* cache_bytes, size_t* workspace_bytes);
+
+/* Create a handle over caller-owned device memory `dev_mem` [device, >= cache_bytes,
+ * 256-byte aligned].  No device work is enqueued.  *out is freed with zc_cache_free,
+ * which releases the host handle only. */
+int zc_cache_init(void* dev_mem, size_t bytes, const zc_config* cfg, zc_cache** out);
+void zc_cache_free(zc_cache* c);
+
+/* Probe selection (Sec. 4.3 "random+recent"): ascending positions made of the last
+ * max(1, floor(rho_recent*l)) tokens plus floor(rho_random*l) of the others, drawn by a
+ * partial Fisher-Yates shuffle driven by splitmix64(seed).  out [host] must hold
+ * zc_probe_count(l, ...) entries; *n_out receives the count. */
+int zc_probe_count(int l, double rho_recent, double rho_random);
+int zc_default_probes(int l, double rho_recent, double rho_random, uint64_t seed,
+                      int32_t* out, int* n_out);
+
+/* Prefill compression (Alg. 2 without its attention-output line).
+ *   Q [device] b x h_q x l x d, K, V [device] b x h_kv x l x d, element type cfg.dtype,
+ *   d contiguous; q_strides / kv_strides [host] = strides of (batch, head, token) in
+ *   ELEMENTS (multiples of 8).
+ *   probe_pos [host] n_probe ascending token positions, the last one equal to l-1
+ *   (Eq. 9's probe rows); ignored when salient_idx is given.
+ *   salient_idx [device or NULL]: test hook -- b x h_kv x floor(r*l) ascending token
+ *   indices to use as the salient set instead of computing Eq. 8 / the split.
+ *   workspace [device] >= workspace_bytes from zc_cache_bytes.
+ * Resets the cache to one compressed segment of l tokens and an empty tail. */
+int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                        const int64_t q_strides[3], const int64_t kv_strides[3],
+                        const int32_t* probe_pos, int n_probe, const int32_t* salient_idx,
+                        void* workspace, size_t workspace_bytes, zc_stream_t stream);
+
+/* Append (Eq. 3, Alg. 3): k_new, v_new [device] b x h_kv x d, contiguous, are copied
+ * verbatim into the full-precision tail.  ZC_ECAPACITY beyond max_new_tokens. */
+int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t stream);
+
+/* Decode attention (Eq. 4, Alg. 3): q [device] b x h_q x d -> out [device] b x h_q x d,
+ * softmax(q K^T / sqrt(d)) V over every cached token, codes dequantised in the kernel.
+ * The step counter of the current window advances; on a probe step (is_probe_step != 0,
+ * or one of the last five steps of a window) this step's attention over the tail's
+ * tokens is added to the window statistics; after the window's last step the tail is
+ * re-compressed into a new segment (same stream, no host synchronisation). */
+int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step,
+                        void* workspace, size_t workspace_bytes, zc_stream_t stream);
+
+/* ---- parity / export: canonical layouts written to caller buffers [device] ---- */
+/* Normalised scores (Eq. 8) of the most recent compression: p_tilde b x h_kv x n floats,
+ * n = l after prefill, window after a re-compression. */
+int zc_export_scores(zc_cache* c, float* p_tilde, zc_stream_t stream);
+/* Number of tokens in (segment, subset); subset 0 = salient, 1 = regular. */
+int zc_segment_tokens(const zc_cache* c, int segment, int subset);
+int zc_num_segments(const zc_cache* c);
+int zc_tail_tokens(const zc_cache* c);
+/* One subset of one segment, all units: idx b x h_kv x n int32 (ascending positions
+ * within the segment); codes b x h_kv x n x (d*bits/8) bytes in canonical packing
+ * (4-bit: element 2m low nibble, 2m+1 high nibble of byte m; 2-bit: element 4m+j in
+ * bits [2j,2j+1] of byte m); sz b x h_kv x n x 2 floats (scale, zero point);
+ * cf b x h_kv x d floats (channel factors).  tensor 0 = K, 1 = V.  Any out may be NULL. */
+int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t* idx,
+                      uint8_t* codes, float* sz, float* cf, zc_stream_t stream);
+
+/* Algorithmic bytes one zc_decode_attention call must read in the cache's current
+ * state (packed codes + per-token parameters + tail + channel factors + q and out). */
+int64_t zc_decode_bytes(const zc_cache* c);
+/* Kernel launches enqueued by this library since the handle was created. */
+int64_t zc_launch_count(const zc_cache* c);
+
+const char* zc_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZIPCACHE_H_ */

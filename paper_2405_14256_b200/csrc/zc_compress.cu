@@ -1,0 +1,391 @@
+// Split by saliency (Alg. 2 "Split"), channel factors (Eq. 6), CSTQuant (Alg. 1, Eq. 5)
+// and packing into cache tiles; also the window statistics -> score step of Alg. 3.
+#include "zc_internal.h"
+#include "zc_layout.cuh"
+
+namespace {
+
+// ------------------------------------------------------------------ top-k split
+// One CTA per unit.  Keys are the bit patterns of the (non-negative) scores, so unsigned
+// integer order equals float order.  An MSB-first 8-bit radix select finds the n_s-th
+// largest key T and how many keys equal to T belong to the top set (lowest index first);
+// a second sweep writes both index lists in ascending order.
+constexpr int kTopkThreads = 1024;
+
+__device__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) warp_sums[warp] = x;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums[lane];
+    int xs = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, xs, o);
+      if (lane >= o) xs += y;
+    }
+    warp_sums[lane] = xs - w;  // exclusive
+    if (lane == 31) *total = xs;
+  }
+  __syncthreads();
+  int r = warp_sums[warp] + x - v;
+  __syncthreads();
+  return r;
+}
+
+__global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayout lay, int n, int n_s,
+                                                             int idx_off,
+                                                             const int32_t* __restrict__ given) {
+  __shared__ int hist[256];
+  __shared__ int warp_sums[32];
+  __shared__ int s_total;
+  __shared__ unsigned s_prefix;
+  __shared__ int s_krem;
+  extern __shared__ unsigned flags[];  // bitset, used when the salient set is given
+  const int unit = blockIdx.x, tid = threadIdx.x;
+  char* ub = zc_unit_base(cache, lay, unit);
+  const unsigned* keys = reinterpret_cast<const unsigned*>(ub + lay.off_scores);
+  int32_t* idx = reinterpret_cast<int32_t*>(ub + lay.off_idx) + idx_off;
+  int32_t* idx_sal = idx;
+  int32_t* idx_reg = idx + n_s;
+
+  unsigned T = 0;
+  int need_eq = 0;
+  if (given) {
+    const int words = (n + 31) / 32;
+    for (int i = tid; i < words; i += kTopkThreads) flags[i] = 0u;
+    __syncthreads();
+    const int32_t* mine = given + (long long)unit * n_s;
+    for (int i = tid; i < n_s; i += kTopkThreads) {
+      const int j = mine[i];
+      if (j >= 0 && j < n) atomicOr(&flags[j >> 5], 1u << (j & 31));
+    }
+    __syncthreads();
+  } else if (n_s > 0 && n_s < n) {
+    if (tid == 0) { s_prefix = 0u; s_krem = n_s; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      const unsigned prefix = s_prefix;
+      const unsigned mask_hi = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      for (int i = tid; i < n; i += kTopkThreads) {
+        const unsigned k = keys[i];
+        if ((k & mask_hi) == prefix) atomicAdd(&hist[(k >> shift) & 255], 1);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int krem = s_krem, b = 255;
+        for (; b > 0; --b) {
+          if (hist[b] >= krem) break;
+          krem -= hist[b];
+        }
+        s_prefix = prefix | ((unsigned)b << shift);
+        s_krem = krem;
+      }
+      __syncthreads();
+    }
+    T = s_prefix;
+    need_eq = s_krem;
+  }
+  // contiguous chunk per thread keeps index order
+  const int chunk = (n + kTopkThreads - 1) / kTopkThreads;
+  const int lo = min(n, tid * chunk), hi = min(n, lo + chunk);
+  int eq_before = 0;
+  if (!given && n_s > 0 && n_s < n) {
+    int eq = 0;
+    for (int i = lo; i < hi; ++i) eq += keys[i] == T;
+    eq_before = block_exclusive_scan(eq, warp_sums, &s_total);
+  }
+  auto is_sal = [&](int i, int& eq_rank) -> bool {
+    if (given) return (flags[i >> 5] >> (i & 31)) & 1u;
+    if (n_s <= 0) return false;
+    if (n_s >= n) return true;
+    const unsigned k = keys[i];
+    if (k > T) return true;
+    if (k == T) return eq_rank++ < need_eq;
+    return false;
+  };
+  int cnt = 0, er = eq_before;
+  for (int i = lo; i < hi; ++i) cnt += is_sal(i, er) ? 1 : 0;
+  const int sal_before = block_exclusive_scan(cnt, warp_sums, &s_total);
+  int s_pos = sal_before, r_pos = lo - sal_before;
+  er = eq_before;
+  for (int i = lo; i < hi; ++i) {
+    if (is_sal(i, er)) {
+      if (s_pos < n_s) idx_sal[s_pos] = i;
+      ++s_pos;
+    } else {
+      if (r_pos < n - n_s) idx_reg[r_pos] = i;
+      ++r_pos;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ window scores
+struct NnzArgs { int v[ZC_MAX_WINDOW]; };
+
+__global__ void k_window_scores(char* cache, ZcLayout lay, NnzArgs nnz) {
+  char* ub = zc_unit_base(cache, lay, blockIdx.x);
+  float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
+  float* scores = reinterpret_cast<float*>(ub + lay.off_scores);
+  const int j = threadIdx.x;
+  if (j < lay.window) {
+    scores[j] = __fdiv_rn(colsum[j], (float)(lay.G * max(1, nnz.v[j])));
+    colsum[j] = 0.f;
+  }
+}
+
+// ------------------------------------------------------------------ channel |x| max (Eq. 6)
+// grid.x: tiles of class 0 then tiles of class 1; grid.y: unit.  blockDim 256.
+template <typename T>
+__global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
+  __shared__ float red[2][8][ZC_D];
+  const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
+  const int tiles_c0 = zc_ceil_div(seg.n_tok[0], ZC_TILE);
+  const int cls = (int)blockIdx.x < tiles_c0 ? 0 : 1;
+  const int tile = cls == 0 ? blockIdx.x : blockIdx.x - tiles_c0;
+  char* ub = zc_unit_base(cache, lay, unit);
+  const int32_t* idx = reinterpret_cast<const int32_t*>(ub + lay.off_idx) + seg.idx_off +
+                       (cls == 0 ? 0 : seg.n_tok[0]);
+  const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh;
+  const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  float mk[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+  const int t0 = tile * ZC_TILE;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int tt = t0 + w + 8 * i;
+    if (tt < seg.n_tok[cls]) {
+      const long long row = (long long)idx[tt] * src.sl;
+      float x[4];
+      zc_load4<T>(Kb + row + 4 * lane, x);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) mk[e] = fmaxf(mk[e], fabsf(x[e]));
+      zc_load4<T>(Vb + row + 4 * lane, x);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) mv[e] = fmaxf(mv[e], fabsf(x[e]));
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    red[0][w][4 * lane + e] = mk[e];
+    red[1][w][4 * lane + e] = mv[e];
+  }
+  __syncthreads();
+  const int ten = threadIdx.x >> 7, ch = threadIdx.x & 127;
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m = fmaxf(m, red[ten][i][ch]);
+  unsigned* cmax = reinterpret_cast<unsigned*>(ub + lay.off_cmax) + (cls * 2 + ten) * ZC_D;
+  atomicMax(&cmax[ch], __float_as_uint(m));  // non-negative floats order like their bits
+}
+
+__global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
+  char* ub = zc_unit_base(cache, lay, blockIdx.x);
+  unsigned* cmax = reinterpret_cast<unsigned*>(ub + lay.off_cmax);
+  for (int i = threadIdx.x; i < 4 * ZC_D; i += blockDim.x) cmax[i] = 0u;
+  float* fac = reinterpret_cast<float*>(ub + lay.off_fac);
+  if (threadIdx.x < 2) fac[(seg.run0 + threadIdx.x) * ZC_FAC_FLOATS + 2 * ZC_D] = 0.f;  // smaxV
+}
+
+// ------------------------------------------------------------------ CSTQuant + pack
+// Normative fp32 sequence (each step one IEEE operation, round to nearest even, nothing
+// fused): c = sqrt(max|x|) (1 if the channel is all zero); y = x / c; per token mn, mx over
+// the 128 channels; s = (mx - mn) / L, or |mn| (1 if mn == 0) when mx == mn;
+// z = -rint(mn / s); code = clamp(rint(y / s) + z, 0, L).
+__device__ __forceinline__ void quant_token(const float (&x)[4], const float (&c)[4], float L,
+                                            float* s_out, float* z_out, unsigned* codes4) {
+  float y[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) y[e] = __fdiv_rn(x[e], c[e]);
+  float mn = fminf(fminf(y[0], y[1]), fminf(y[2], y[3]));
+  float mx = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  float s = __fdiv_rn(__fsub_rn(mx, mn), L);
+  if (mx == mn) s = mn != 0.f ? fabsf(mn) : 1.f;
+  const float z = -rintf(__fdiv_rn(mn, s));
+  unsigned packed = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float q = __fadd_rn(rintf(__fdiv_rn(y[e], s)), z);
+    q = fminf(fmaxf(q, 0.f), L);
+    packed |= ((unsigned)(int)q) << (8 * e);
+  }
+  *s_out = s;
+  *z_out = z;
+  *codes4 = packed;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
+  __shared__ __align__(16) unsigned char codesK[ZC_TILE][ZC_D];
+  __shared__ __align__(16) unsigned char codesV[ZC_TILE][ZC_D];
+  __shared__ __align__(16) float parK[ZC_TILE][2];
+  __shared__ __align__(16) float parV[ZC_TILE][2];
+  const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
+  const int tiles_c0 = zc_ceil_div(seg.n_tok[0], ZC_TILE);
+  const int cls = (int)blockIdx.x < tiles_c0 ? 0 : 1;
+  const int tile = cls == 0 ? blockIdx.x : blockIdx.x - tiles_c0;
+  const int bits = lay.bits[cls];
+  const float L = (float)((1 << bits) - 1);
+  char* ub = zc_unit_base(cache, lay, unit);
+  const int32_t* idx = reinterpret_cast<const int32_t*>(ub + lay.off_idx) + seg.idx_off +
+                       (cls == 0 ? 0 : seg.n_tok[0]);
+  const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh;
+  const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const unsigned* cmax = reinterpret_cast<const unsigned*>(ub + lay.off_cmax) + cls * 2 * ZC_D;
+  float* fac = reinterpret_cast<float*>(ub + lay.off_fac) + (seg.run0 + cls) * ZC_FAC_FLOATS;
+  float cK[4], cV[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float mk = __uint_as_float(cmax[4 * lane + e]);
+    const float mv = __uint_as_float(cmax[ZC_D + 4 * lane + e]);
+    cK[e] = mk == 0.f ? 1.f : __fsqrt_rn(mk);
+    cV[e] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
+  }
+  if (tile == 0 && w == 0) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      fac[4 * lane + e] = cK[e];
+      fac[ZC_D + 4 * lane + e] = cV[e];
+    }
+  }
+  const int t0 = tile * ZC_TILE;
+  // gather the warp's 8 token rows first (memory-level parallelism), then quantise
+  uint2 rawK[8], rawV[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int tt = t0 + w * 8 + i;
+    if (tt < seg.n_tok[cls]) {
+      const long long row = (long long)idx[tt] * src.sl;
+      rawK[i] = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
+      rawV[i] = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
+    } else {
+      rawK[i] = make_uint2(0, 0);
+      rawV[i] = make_uint2(0, 0);
+    }
+  }
+  float smax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int tl = w * 8 + i, tt = t0 + tl;
+    const bool live = tt < seg.n_tok[cls];
+    float x[4], s, z;
+    unsigned pk;
+    const T* ek = reinterpret_cast<const T*>(&rawK[i]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
+    quant_token(x, cK, L, &s, &z, &pk);
+    *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live ? pk : 0u;
+    if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
+    const T* ev = reinterpret_cast<const T*>(&rawV[i]);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
+    quant_token(x, cV, L, &s, &z, &pk);
+    *reinterpret_cast<unsigned*>(&codesV[tl][4 * lane]) = live ? pk : 0u;
+    if (lane == 0) { parV[tl][0] = live ? s : 0.f; parV[tl][1] = live ? z : 0.f; }
+    if (live) smax = fmaxf(smax, s);
+  }
+  if (lane == 0 && smax > 0.f) atomicMax(reinterpret_cast<unsigned*>(&fac[2 * ZC_D]), __float_as_uint(smax));
+  __syncthreads();
+
+  // compose the tile: 16-byte stores, consecutive threads -> consecutive addresses
+  char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
+  const int code_words = zc_codes_bytes(bits) / 4;   // per tensor
+  const int per = 32 / bits;                          // codes per word
+  const int total_vec = lay.tile_bytes[cls] / 16;
+  for (int v = threadIdx.x; v < total_vec; v += 256) {
+    unsigned out[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int wi = 4 * v + q;
+      unsigned word = 0;
+      if (wi < code_words) {
+        // K: canonical order, token row of 4*bits words
+        const int words_per_row = 4 * bits;
+        const int tok = wi / words_per_row, wr = wi % words_per_row;
+        for (int e = 0; e < per; ++e) word |= (unsigned)codesK[tok][wr * per + e] << (bits * e);
+      } else if (wi < 2 * code_words) {
+        // V: fragment order, 4 sub-tiles of 16 tokens
+        const int wv = wi - code_words;
+        const int sub_words = code_words / 4;
+        const int st = wv / sub_words, wl = wv % sub_words;
+        if (bits == 4) {
+          const int qd = wl >> 7, ln = (wl >> 2) & 31, jj = wl & 3;
+          const int j = 4 * qd + jj, g = ln >> 2, t = ln & 3;
+          for (int p = 0; p < 8; ++p) {
+            const int hi_row = p & 1, isB = (p >> 1) & 1, is1 = p >> 2;
+            const int ch = 16 * j + g + 8 * hi_row, tau = 2 * t + isB + 8 * is1;
+            word |= (unsigned)codesV[16 * st + tau][ch] << (4 * p);
+          }
+        } else {
+          const int ln = wl >> 2, m = wl & 3, g = ln >> 2, t = ln & 3;
+          for (int i = 0; i < 16; ++i) {
+            const int is1 = i >> 3, pp = i & 7, e2 = pp >> 2, hi_row = (pp >> 1) & 1, isB = pp & 1;
+            const int j = 2 * m + e2;
+            const int ch = 16 * j + g + 8 * hi_row, tau = 2 * t + isB + 8 * is1;
+            word |= (unsigned)codesV[16 * st + tau][ch] << (2 * i);
+          }
+        }
+      } else {
+        const int wp = wi - 2 * code_words;  // params: K then V, (s, z) pairs
+        const float* pf = wp < 2 * ZC_TILE ? &parK[0][0] + wp : &parV[0][0] + (wp - 2 * ZC_TILE);
+        word = __float_as_uint(*pf);
+      }
+      out[q] = word;
+    }
+    reinterpret_cast<uint4*>(tile_ptr)[v] = make_uint4(out[0], out[1], out[2], out[3]);
+  }
+}
+
+}  // namespace
+
+int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
+                   cudaStream_t st) {
+  const int smem = given_sal ? ((n + 31) / 32) * 4 : 0;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(k_topk_split, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+  }
+  k_topk_split<<<c->lay.units, kTopkThreads, smem, st>>>(c->base, c->lay, n, n_s, idx_off, given_sal);
+  c->launches += 1;
+  return cudaGetLastError();
+}
+
+int zc_launch_window_scores(zc_cache* c, cudaStream_t st) {
+  NnzArgs a;
+  for (int j = 0; j < ZC_MAX_WINDOW; ++j) a.v[j] = c->tail_nnz[j];
+  k_window_scores<<<c->lay.units, ZC_MAX_WINDOW, 0, st>>>(c->base, c->lay, a);
+  c->launches += 1;
+  return cudaGetLastError();
+}
+
+int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st) {
+  const int tiles = zc_ceil_div(seg.n_tok[0], ZC_TILE) + zc_ceil_div(seg.n_tok[1], ZC_TILE);
+  k_clear_cmax<<<c->lay.units, 128, 0, st>>>(c->base, c->lay, seg);
+  c->launches += 1;
+  if (tiles > 0) {
+    dim3 grid(tiles, c->lay.units);
+    if (c->cfg.dtype == ZC_F16) {
+      k_channel_absmax<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_quantize_pack<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+    } else {
+      k_channel_absmax<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_quantize_pack<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+    }
+    c->launches += 2;
+  }
+  return cudaGetLastError();
+}

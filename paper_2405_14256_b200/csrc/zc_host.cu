@@ -1,0 +1,383 @@
+// Host side of the C ABI: argument checks, cache layout, call sequencing.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+#include <new>
+#include <vector>
+#include <algorithm>
+#include "zc_internal.h"
+#include "zc_layout.cuh"
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int n_salient(double r, int n) { return (int)floor(r * (double)n); }
+inline bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+int check_config(const zc_config* cfg) {
+  if (!cfg || cfg->struct_size != (int)sizeof(zc_config)) return ZC_EINVAL;
+  if (cfg->dtype != ZC_F16 && cfg->dtype != ZC_BF16) return ZC_EINVAL;
+  if (cfg->batch < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads < 1) return ZC_EINVAL;
+  if (cfg->n_q_heads % cfg->n_kv_heads) return ZC_EINVAL;
+  if (cfg->n_q_heads / cfg->n_kv_heads > ZC_MAX_G) return ZC_EINVAL;
+  if (cfg->head_dim != ZC_D) return ZC_EINVAL;
+  if (cfg->max_prefill < 1 || cfg->max_prefill > (1 << 20)) return ZC_EINVAL;
+  if (cfg->max_new_tokens < 0) return ZC_EINVAL;
+  if (cfg->window < 8 || cfg->window > ZC_MAX_WINDOW) return ZC_EINVAL;
+  if (cfg->bits_hi != 4 && cfg->bits_hi != 2) return ZC_EINVAL;
+  if (cfg->bits_lo != 4 && cfg->bits_lo != 2) return ZC_EINVAL;
+  if (cfg->reserved != 0) return ZC_EINVAL;
+  if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
+  if ((long long)cfg->batch * cfg->n_kv_heads > 65535) return ZC_EINVAL;
+  return ZC_OK;
+}
+
+void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_t* ws_bytes) {
+  const int elt = 2;
+  lay->units = cfg->batch * cfg->n_kv_heads;
+  lay->G = cfg->n_q_heads / cfg->n_kv_heads;
+  lay->n_kv = cfg->n_kv_heads;
+  lay->window = cfg->window;
+  lay->dtype = cfg->dtype;
+  lay->bits[0] = cfg->bits_hi;
+  lay->bits[1] = cfg->bits_lo;
+  const int max_flush = cfg->max_new_tokens / cfg->window;
+  const int ns_max = n_salient(cfg->saliency_ratio, cfg->max_prefill);
+  const int nr_max = cfg->max_prefill - ns_max;  // l - floor(r l) is non-decreasing in l
+  const int ns_w = n_salient(cfg->saliency_ratio, cfg->window);
+  const int nr_w = cfg->window - ns_w;
+  // floor(r l) for l < max_prefill never exceeds ns_max; l - floor(r l) never exceeds nr_max.
+  lay->cap_tiles[0] = zc_ceil_div(ns_max, ZC_TILE) + max_flush * zc_ceil_div(ns_w, ZC_TILE);
+  lay->cap_tiles[1] = zc_ceil_div(nr_max, ZC_TILE) + max_flush * zc_ceil_div(nr_w, ZC_TILE);
+  lay->max_runs = 2 * (1 + max_flush);
+  lay->idx_cap0 = cfg->max_prefill;
+  size_t off = 0;
+  for (int c = 0; c < 2; ++c) {
+    lay->tile_bytes[c] = zc_tile_bytes(lay->bits[c]);
+    lay->off_tiles[c] = (long long)off;
+    off = align_up(off + (size_t)lay->cap_tiles[c] * lay->tile_bytes[c], 256);
+  }
+  lay->off_fac = (long long)off;
+  off = align_up(off + (size_t)lay->max_runs * ZC_FAC_FLOATS * 4, 256);
+  lay->off_cmax = (long long)off;
+  off = align_up(off + 2 * 2 * ZC_D * 4, 256);
+  lay->off_tailK = (long long)off;
+  off = align_up(off + (size_t)cfg->window * ZC_D * elt, 256);
+  lay->off_tailV = (long long)off;
+  off = align_up(off + (size_t)cfg->window * ZC_D * elt, 256);
+  lay->off_colsum = (long long)off;
+  off = align_up(off + ZC_MAX_WINDOW * 4, 256);
+  lay->off_scores = (long long)off;
+  off = align_up(off + (size_t)std::max(cfg->max_prefill, cfg->window) * 4, 256);
+  lay->off_idx = (long long)off;
+  off = align_up(off + ((size_t)cfg->max_prefill + (size_t)max_flush * cfg->window) * 4, 256);
+  lay->unit_stride = (long long)off;
+  if (cache_bytes) *cache_bytes = off * (size_t)lay->units;
+  if (ws_bytes) {
+    // prefill: probe positions + per-row log-sum-exp for every query head
+    const int np_max = cfg->max_prefill;
+    size_t pre = align_up((size_t)np_max * 4, 256) +
+                 (size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4;
+    // decode: partials [unit][item][G][ZC_PART_STRIDE] + tail logits [unit][G][window]
+    const int max_items = 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush + 1;
+    size_t dec = (size_t)lay->units * max_items * lay->G * ZC_PART_STRIDE * 4 +
+                 (size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4 + 256;
+    *ws_bytes = align_up(std::max(pre, dec), 256);
+  }
+}
+
+const char* kMsgs[] = {"ok", "invalid argument", "capacity exceeded", "call out of order",
+                       "pointer not 16-byte aligned", "CUDA error"};
+thread_local char g_cuda_msg[256] = "CUDA error";
+
+int cuda_fail(cudaError_t e) {
+  snprintf(g_cuda_msg, sizeof(g_cuda_msg), "CUDA error: %s", cudaGetErrorString(e));
+  return ZC_ECUDA;
+}
+
+#define ZC_CUDA(expr)                              \
+  do {                                             \
+    cudaError_t e__ = (cudaError_t)(expr);         \
+    if (e__ != cudaSuccess) return cuda_fail(e__); \
+  } while (0)
+
+}  // namespace
+
+ZcSeg zc_segment(const zc_cache* c, int seg) {
+  ZcSeg s;
+  for (int k = 0; k < 2; ++k) {
+    const int t0 = zc_ceil_div(c->n0[k], ZC_TILE), tw = zc_ceil_div(c->nw[k], ZC_TILE);
+    s.n_tok[k] = seg == 0 ? c->n0[k] : c->nw[k];
+    s.tile0[k] = seg == 0 ? 0 : t0 + (seg - 1) * tw;
+  }
+  s.idx_off = seg == 0 ? 0 : c->lay.idx_cap0 + (seg - 1) * c->cfg.window;
+  s.run0 = 2 * seg;
+  return s;
+}
+
+ZcDecodePlan zc_make_plan(const zc_cache* c) {
+  ZcDecodePlan p;
+  memset(&p, 0, sizeof(p));
+  p.n_seg = c->n_seg;
+  p.n_tail = c->n_tail;
+  p.l0 = c->l0;
+  long long bytes[2];
+  for (int k = 0; k < 2; ++k) {
+    p.n0[k] = c->n0[k];
+    p.nw[k] = c->nw[k];
+    p.tiles0[k] = zc_ceil_div(c->n0[k], ZC_TILE);
+    p.tilesw[k] = zc_ceil_div(c->nw[k], ZC_TILE);
+    bytes[k] = (long long)p.tiles0[k] * c->lay.tile_bytes[k];
+  }
+  // One wave of CTAs over all SMs when the units allow it: budget items per unit, then
+  // share them between the two classes in proportion to their bytes.
+  const int slots = c->n_sm * ZC_DECODE_CTAS_PER_SM;
+  int budget = slots / c->lay.units - (c->n_tail > 0 ? 1 : 0) - 2 * (c->n_seg - 1);
+  budget = std::max(2, std::min(budget, 2 * ZC_MAX_SPLIT_HOST));
+  const long long tot = std::max(1LL, bytes[0] + bytes[1]);
+  int s0 = (int)((bytes[0] * budget + tot / 2) / tot);
+  s0 = std::max(1, std::min(s0, budget - 1));
+  int s1 = budget - s0;
+  int sp[2] = {s0, s1};
+  for (int k = 0; k < 2; ++k) {
+    int s = std::max(1, std::min(std::min(sp[k], ZC_MAX_SPLIT_HOST), std::max(1, p.tiles0[k])));
+    p.tpi0[k] = std::max(1, zc_ceil_div(std::max(1, p.tiles0[k]), s));
+    p.split0[k] = std::max(1, zc_ceil_div(std::max(1, p.tiles0[k]), p.tpi0[k]));
+  }
+  p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + (p.n_tail > 0 ? 1 : 0);
+  return p;
+}
+
+extern "C" {
+
+const char* zc_strerror(int status) {
+  if (status == ZC_ECUDA) return g_cuda_msg;
+  if (status > 0 || status < -5) return "unknown status";
+  return kMsgs[-status];
+}
+
+int zc_cache_bytes(const zc_config* cfg, size_t* cache_bytes, size_t* workspace_bytes) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  ZcLayout lay;
+  make_layout(cfg, &lay, cache_bytes, workspace_bytes);
+  return ZC_OK;
+}
+
+int zc_cache_init(void* dev_mem, size_t bytes, const zc_config* cfg, zc_cache** out) {
+  if (!out) return ZC_EINVAL;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!dev_mem) return ZC_EINVAL;
+  if ((uintptr_t)dev_mem & 255) return ZC_EALIGN;
+  zc_cache* c = new (std::nothrow) zc_cache();
+  if (!c) return ZC_EINVAL;
+  memset(c, 0, sizeof(*c));
+  c->cfg = *cfg;
+  size_t need = 0;
+  make_layout(cfg, &c->lay, &need, &c->ws_bytes);
+  if (bytes < need) {
+    delete c;
+    return ZC_ECAPACITY;
+  }
+  c->base = (char*)dev_mem;
+  c->bytes = bytes;
+  c->l0 = -1;
+  c->n_seg = 0;
+  int dev = 0, n_sm = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess)
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  else
+    cudaGetLastError();
+  c->n_sm = n_sm > 0 ? n_sm : 148;
+  *out = c;
+  return ZC_OK;
+}
+
+void zc_cache_free(zc_cache* c) { delete c; }
+
+int zc_probe_count(int l, double rho_recent, double rho_random) {
+  if (l < 1 || !(rho_recent >= 0.0 && rho_recent <= 1.0) ||
+      !(rho_random >= 0.0 && rho_random <= 1.0))
+    return ZC_EINVAL;
+  int n_rec = std::min(l, std::max(1, (int)floor(rho_recent * (double)l)));
+  int n_rnd = std::min(l - n_rec, (int)floor(rho_random * (double)l));
+  return n_rec + n_rnd;
+}
+
+int zc_default_probes(int l, double rho_recent, double rho_random, uint64_t seed, int32_t* out,
+                      int* n_out) {
+  int total = zc_probe_count(l, rho_recent, rho_random);
+  if (total < 0 || !out) return ZC_EINVAL;
+  const int n_rec = std::min(l, std::max(1, (int)floor(rho_recent * (double)l)));
+  const int n_rnd = total - n_rec;
+  const int pool = l - n_rec;
+  std::vector<int32_t> perm((size_t)pool);
+  for (int i = 0; i < pool; ++i) perm[i] = i;
+  uint64_t state = seed;
+  for (int i = 0; i < n_rnd; ++i) {
+    state += 0x9E3779B97F4A7C15ull;
+    uint64_t z = state;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    int j = i + (int)(z % (uint64_t)(pool - i));
+    std::swap(perm[i], perm[j]);
+  }
+  std::sort(perm.begin(), perm.begin() + n_rnd);
+  for (int i = 0; i < n_rnd; ++i) out[i] = perm[i];
+  for (int i = 0; i < n_rec; ++i) out[n_rnd + i] = pool + i;
+  if (n_out) *n_out = total;
+  return ZC_OK;
+}
+
+int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                        const int64_t q_strides[3], const int64_t kv_strides[3],
+                        const int32_t* probe_pos, int n_probe, const int32_t* salient_idx,
+                        void* workspace, size_t workspace_bytes, zc_stream_t stream) {
+  if (!c || !K || !V || !kv_strides) return ZC_EINVAL;
+  if (l < 1) return ZC_EINVAL;
+  if (l > c->cfg.max_prefill) return ZC_ECAPACITY;
+  if (!aligned16(K) || !aligned16(V)) return ZC_EALIGN;
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || (kv_strides[i] % 8)) return ZC_EINVAL;
+  if (kv_strides[2] < ZC_D) return ZC_EINVAL;
+  if (!salient_idx) {
+    if (!Q || !q_strides || !probe_pos || !workspace) return ZC_EINVAL;
+    if (!aligned16(Q) || !aligned16(workspace)) return ZC_EALIGN;
+    for (int i = 0; i < 3; ++i)
+      if (q_strides[i] < 0 || (q_strides[i] % 8)) return ZC_EINVAL;
+    if (q_strides[2] < ZC_D) return ZC_EINVAL;
+    if (n_probe < 1 || n_probe > l) return ZC_EINVAL;
+    for (int i = 0; i < n_probe; ++i) {
+      if (probe_pos[i] < 0 || probe_pos[i] >= l) return ZC_EINVAL;
+      if (i && probe_pos[i] <= probe_pos[i - 1]) return ZC_EINVAL;
+    }
+    if (probe_pos[n_probe - 1] != l - 1) return ZC_EINVAL;
+    size_t need = align_up((size_t)n_probe * 4, 256) +
+                  (size_t)c->cfg.batch * c->cfg.n_q_heads * (size_t)n_probe * 4;
+    if (workspace_bytes < need) return ZC_ECAPACITY;
+  } else if (!aligned16(salient_idx)) {
+    return ZC_EALIGN;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  c->l0 = l;
+  c->n0[0] = n_salient(c->cfg.saliency_ratio, l);
+  c->n0[1] = l - c->n0[0];
+  c->nw[0] = n_salient(c->cfg.saliency_ratio, c->cfg.window);
+  c->nw[1] = c->cfg.window - c->nw[0];
+  c->n_seg = 1;
+  c->n_tail = 0;
+  c->step_i = 0;
+  c->n_new = 0;
+  memset(c->tail_nnz, 0, sizeof(c->tail_nnz));
+  c->last_scores_n = l;
+  // window statistics start at zero
+  ZC_CUDA(cudaMemset2DAsync(c->base + c->lay.off_colsum, (size_t)c->lay.unit_stride, 0,
+                            ZC_MAX_WINDOW * 4, (size_t)c->lay.units, st));
+  if (!salient_idx) {
+    int32_t* P_dev = (int32_t*)workspace;
+    float* lse = (float*)((char*)workspace + align_up((size_t)n_probe * 4, 256));
+    ZC_CUDA(cudaMemcpyAsync(P_dev, probe_pos, (size_t)n_probe * 4, cudaMemcpyHostToDevice, st));
+    ZC_CUDA(zc_launch_probe_scores(c, Q, K, l, q_strides, kv_strides, P_dev, n_probe, lse, st));
+  }
+  ZC_CUDA(zc_launch_topk(c, l, c->n0[0], 0, salient_idx, st));
+  ZcSrc src{K, V, kv_strides[0], kv_strides[1], kv_strides[2]};
+  ZC_CUDA(zc_launch_quantize(c, src, zc_segment(c, 0), st));
+  return ZC_OK;
+}
+
+int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t stream) {
+  if (!c || !k_new || !v_new) return ZC_EINVAL;
+  if (c->l0 < 0) return ZC_ESTATE;
+  if (!aligned16(k_new) || !aligned16(v_new)) return ZC_EALIGN;
+  if (c->n_new >= c->cfg.max_new_tokens) return ZC_ECAPACITY;
+  if (c->n_tail >= c->cfg.window) return ZC_ESTATE;
+  ZC_CUDA(zc_launch_append(c, k_new, v_new, c->n_tail, (cudaStream_t)stream));
+  c->n_tail += 1;
+  c->n_new += 1;
+  return ZC_OK;
+}
+
+int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step,
+                        void* workspace, size_t workspace_bytes, zc_stream_t stream) {
+  if (!c || !q || !out || !workspace) return ZC_EINVAL;
+  if (c->l0 < 0) return ZC_ESTATE;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return ZC_EALIGN;
+  if (workspace_bytes < c->ws_bytes) return ZC_ECAPACITY;
+  cudaStream_t st = (cudaStream_t)stream;
+  ZcDecodePlan plan = zc_make_plan(c);
+  const int i_next = c->step_i + 1;
+  const int collect =
+      (c->n_tail > 0) && (is_probe_step || i_next > c->cfg.window - 5) ? 1 : 0;
+  ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (float*)workspace, st));
+  // Alg. 3 bookkeeping: the step counter follows the tokens of the current window
+  if (c->n_tail > 0) {
+    c->step_i = i_next;
+    if (collect)
+      for (int j = 0; j < c->n_tail; ++j) c->tail_nnz[j] += 1;
+    if (c->step_i == c->cfg.window && c->n_tail == c->cfg.window) {
+      // re-compress the window into a new segment
+      ZC_CUDA(zc_launch_window_scores(c, st));
+      c->last_scores_n = c->cfg.window;
+      const int seg = c->n_seg;
+      c->n_seg += 1;
+      ZcSeg s = zc_segment(c, seg);
+      ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], s.idx_off, nullptr, st));
+      const long long us = c->lay.unit_stride / 2;
+      ZcSrc src{c->base + c->lay.off_tailK, c->base + c->lay.off_tailV, us * c->lay.n_kv, us,
+                ZC_D};
+      ZC_CUDA(zc_launch_quantize(c, src, s, st));
+      c->n_tail = 0;
+      c->step_i = 0;
+      memset(c->tail_nnz, 0, sizeof(c->tail_nnz));
+    }
+  }
+  return ZC_OK;
+}
+
+int zc_num_segments(const zc_cache* c) { return c ? c->n_seg : ZC_EINVAL; }
+int zc_tail_tokens(const zc_cache* c) { return c ? c->n_tail : ZC_EINVAL; }
+
+int zc_segment_tokens(const zc_cache* c, int segment, int subset) {
+  if (!c || segment < 0 || segment >= c->n_seg || subset < 0 || subset > 1) return ZC_EINVAL;
+  return segment == 0 ? c->n0[subset] : c->nw[subset];
+}
+
+int zc_export_scores(zc_cache* c, float* p_tilde, zc_stream_t stream) {
+  if (!c || !p_tilde) return ZC_EINVAL;
+  if (c->l0 < 0) return ZC_ESTATE;
+  ZC_CUDA(zc_launch_export_scores(c, p_tilde, c->last_scores_n, (cudaStream_t)stream));
+  return ZC_OK;
+}
+
+int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t* idx,
+                      uint8_t* codes, float* sz, float* cf, zc_stream_t stream) {
+  if (!c || tensor < 0 || tensor > 1 || subset < 0 || subset > 1) return ZC_EINVAL;
+  if (c->l0 < 0) return ZC_ESTATE;
+  if (segment < 0 || segment >= c->n_seg) return ZC_EINVAL;
+  ZC_CUDA(zc_launch_export_segment(c, zc_segment(c, segment), tensor, subset, idx, codes, sz, cf,
+                                   (cudaStream_t)stream));
+  return ZC_OK;
+}
+
+int64_t zc_decode_bytes(const zc_cache* c) {
+  if (!c || c->l0 < 0) return 0;
+  int64_t per_unit = 0;
+  for (int k = 0; k < 2; ++k) {
+    const int64_t per_tok = 32 * c->lay.bits[k] + 16;  // K+V codes, (s,z) pairs
+    const int64_t toks = (int64_t)c->n0[k] + (int64_t)(c->n_seg - 1) * c->nw[k];
+    per_unit += toks * per_tok;
+    const int runs = (c->n0[k] > 0 ? 1 : 0) + (c->nw[k] > 0 ? c->n_seg - 1 : 0);
+    per_unit += (int64_t)runs * 2 * ZC_D * 4;        // channel factors of K and V
+  }
+  per_unit += (int64_t)c->n_tail * 2 * ZC_D * 2;     // full-precision tail
+  per_unit += (int64_t)c->lay.G * ZC_D * 2 * 2;      // q in, out
+  return per_unit * c->lay.units;
+}
+
+int64_t zc_launch_count(const zc_cache* c) { return c ? c->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,110 @@
+// Internal declarations shared by the host API and the kernels of the library.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "zipcache.h"
+
+#define ZC_D 128            // head_dim
+#define ZC_TILE 64          // tokens per cache tile
+#define ZC_SUB 16           // tokens per MMA sub-tile inside a tile
+#define ZC_FAC_FLOATS 272   // per-run factor block: cK[128], cV[128], smaxV, pad
+#define ZC_PART_STRIDE 132  // split-K partial per head: m, l, pad, pad, acc[128]
+#define ZC_MAX_G 8
+#define ZC_MAX_SPLIT_HOST 32      // most items one class of segment 0 is split into
+#define ZC_DECODE_CTAS_PER_SM 4    // CTAs the decode kernel keeps resident per SM
+
+// Device-side description of the cache buffer.  One "unit" = (batch, KV head).
+// Per unit, at byte offsets from base + unit * unit_stride:
+//   off_tiles[c]   cap_tiles[c] tiles of class c (0 = salient bits, 1 = regular bits)
+//   off_fac        max_runs factor blocks (run = segment * 2 + class)
+//   off_cmax       scratch: |x| channel maxima as uint bits  [class][tensor][128]
+//   off_tailK/V    window x d elements of the input type
+//   off_colsum     window floats: attention mass collected on probe steps
+//   off_scores     normalised scores of the latest compression
+//   off_idx        token index lists: segment 0 (salient then regular), then one
+//                  window-sized slot per re-compressed window
+// A tile of class c holds 64 tokens:
+//   [K codes 64 x 16*bits B, canonical nibble/crumb order per token row]
+//   [V codes 4 sub-tiles of 16 tokens, fragment order (see zc_layout.cuh)]
+//   [K params 64 x (scale, zero) f32][V params 64 x (scale, zero) f32]
+struct ZcLayout {
+  int units, G, n_kv, window, dtype;
+  int bits[2];
+  int tile_bytes[2];
+  int cap_tiles[2];
+  int max_runs;
+  int idx_cap0;
+  long long unit_stride;
+  long long off_tiles[2], off_fac, off_cmax, off_tailK, off_tailV, off_colsum, off_scores,
+      off_idx;
+};
+
+// Where the rows to compress come from (caller tensors at prefill, the tail at a flush).
+struct ZcSrc {
+  const void* K;
+  const void* V;
+  long long sb, sh, sl;  // element strides of (batch, kv head, token)
+};
+
+// One segment's two subsets.
+struct ZcSeg {
+  int n_tok[2];    // tokens per class
+  int tile0[2];    // first tile per class
+  int idx_off;     // offset (ints) of this segment's index lists in the idx region
+  int run0;        // factor-block index of class 0 (class 1 = run0 + 1)
+};
+
+// Split-K plan of one decode call (identical for every unit).
+struct ZcDecodePlan {
+  int n_seg;
+  int n0[2], nw[2];        // tokens per class: segment 0, re-compressed windows
+  int tiles0[2], tilesw[2];
+  int split0[2];           // items covering segment 0, per class
+  int tpi0[2];             // tiles per item, per class
+  int n_tail;
+  int items;               // items per unit
+  int l0;
+};
+
+struct zc_cache {
+  zc_config cfg;
+  ZcLayout lay;
+  char* base;
+  size_t bytes;
+  size_t ws_bytes;
+  int l0;          // prefill length, -1 before prefill
+  int n0[2];
+  int nw[2];
+  int n_seg;       // 1 + number of re-compressed windows
+  int n_tail;
+  int step_i;      // decode steps taken in the current window
+  int n_new;       // tokens appended since prefill
+  int tail_nnz[ZC_MAX_WINDOW];
+  int last_scores_n;
+  int n_sm;
+  long long launches;
+};
+
+__host__ __device__ static inline int zc_ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+ZcSeg zc_segment(const zc_cache* c, int seg);
+ZcDecodePlan zc_make_plan(const zc_cache* c);
+
+// ---- launchers (each returns a cudaError_t as int) ----
+int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l,
+                           const int64_t* qs, const int64_t* ks, const int32_t* P_dev,
+                           int n_probe, float* lse_ws, cudaStream_t st);
+int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
+                   cudaStream_t st);
+int zc_launch_window_scores(zc_cache* c, cudaStream_t st);
+int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st);
+int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
+                     cudaStream_t st);
+int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out,
+                     int collect, float* ws, cudaStream_t st);
+int zc_launch_export_scores(zc_cache* c, float* out, int n, cudaStream_t st);
+int zc_launch_export_segment(zc_cache* c, const ZcSeg& seg, int tensor, int subset,
+                             int32_t* idx, uint8_t* codes, float* sz, float* cf,
+                             cudaStream_t st);

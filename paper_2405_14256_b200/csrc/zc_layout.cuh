@@ -1,0 +1,57 @@
+// Device-side layout helpers: where a (token, channel) code lives inside a tile.
+//
+// K codes keep the canonical order per token row.  V codes are stored in the
+// register order of the m16n8k16 MMA A-fragment of V^T (rows = channels,
+// k = tokens), so that the decode kernel can turn a 32-bit word into fragment
+// registers with masks only:
+//   lane = g*4 + t, g = 0..7, t = 0..3;  M-tile j = channels 16j..16j+15;
+//   fragment rows g (scale 1) and g+8 (scale 16) <-> channels 16j+g, 16j+g+8;
+//   fragment k-pairs A = (2t, 2t+1) <-> tokens (2t, 2t+8), B = (2t+8, 2t+9) <->
+//   tokens (2t+1, 2t+9) of the 16-token sub-tile.
+// 4-bit: word j of the lane (8 nibbles) serves M-tile j; nibble p = hi_row + 2*isB + 4*is1.
+// 2-bit: word m of the lane (16 crumbs) serves M-tiles 2m and 2m+1;
+//        crumb i = 8*is1 + 4*(j&1) + 2*hi_row + isB.
+#pragma once
+#include "zc_internal.h"
+
+__host__ __device__ inline int zc_tile_bytes(int bits) { return ZC_TILE * (32 * bits + 16); }
+__host__ __device__ inline int zc_codes_bytes(int bits) { return ZC_TILE * 16 * bits; }  // one tensor
+__host__ __device__ inline int zc_tile_off_vcodes(int bits) { return zc_codes_bytes(bits); }
+__host__ __device__ inline int zc_tile_off_kpar(int bits) { return 2 * zc_codes_bytes(bits); }
+__host__ __device__ inline int zc_tile_off_vpar(int bits) { return 2 * zc_codes_bytes(bits) + ZC_TILE * 8; }
+
+// Position of V code (token tau of a 16-token sub-tile, channel ch) inside the
+// sub-tile's block: returns the 32-bit word index and the bit shift in the word.
+__host__ __device__ inline void zc_vcode_pos(int bits, int tau, int ch, int* word, int* shift) {
+  int j = ch >> 4, rho = ch & 15, g = rho & 7, hi_row = rho >> 3;
+  int is1 = tau >> 3, tp = tau & 7, t = tp >> 1, isB = tp & 1;
+  int lane = g * 4 + t;
+  if (bits == 4) {
+    int p = hi_row + 2 * isB + 4 * is1;
+    *word = (j >> 2) * 128 + lane * 4 + (j & 3);
+    *shift = 4 * p;
+  } else {
+    int i = 8 * is1 + 4 * (j & 1) + 2 * hi_row + isB;
+    *word = lane * 4 + (j >> 1);
+    *shift = 2 * i;
+  }
+}
+
+template <typename T> __device__ inline float zc_to_float(T v);
+template <> __device__ inline float zc_to_float<__half>(__half v) { return __half2float(v); }
+template <> __device__ inline float zc_to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ inline T zc_from_float(float v);
+template <> __device__ inline __half zc_from_float<__half>(float v) { return __float2half_rn(v); }
+template <> __device__ inline __nv_bfloat16 zc_from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// 4 consecutive elements (8 bytes) -> floats
+template <typename T> __device__ inline void zc_load4(const T* p, float* out) {
+  uint2 raw = *reinterpret_cast<const uint2*>(p);
+  const T* e = reinterpret_cast<const T*>(&raw);
+  out[0] = zc_to_float<T>(e[0]); out[1] = zc_to_float<T>(e[1]);
+  out[2] = zc_to_float<T>(e[2]); out[3] = zc_to_float<T>(e[3]);
+}
+
+__device__ inline char* zc_unit_base(char* base, const ZcLayout& lay, int unit) {
+  return base + (long long)unit * lay.unit_stride;
+}

@@ -1,0 +1,186 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by
+element, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import zipcache_oracle as zo
+from workloads import get_config, make_prefill
+import zc_testlib as tl
+
+pytestmark = pytest.mark.gpu
+
+
+def _staged_quant_case(w):
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    n_s = zo.salient_count(w.saliency_ratio, w.context)
+    sal = np.zeros((w.batch, w.n_kv_heads, max(n_s, 1)), dtype=np.int32)
+    for (bi, kv), u in oc.units.items():
+        sal[bi, kv, :n_s] = u.segments[0].hi.idx
+    cache = tl.make_cache(w)
+    cache.prefill_compress(None, K, V, None, salient_idx=torch.tensor(sal, device=tl.DEV))
+    torch.cuda.synchronize()
+    assert tl.compare_segment(cache, oc, 0) == 0
+
+
+@pytest.mark.parametrize("l", [1, 2, 17, 64, 100, 513])
+@pytest.mark.parametrize("ratio", [0.0, 0.5, 1.0])
+def test_quantize_pack_bit_exact_edge_lengths(l, ratio):
+    _staged_quant_case(tl.small_workload(context=l, saliency_ratio=ratio, n_q_heads=2,
+                                         n_kv_heads=2, rho_recent=0.2, rho_random=0.2))
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", [(4, 2), (4, 4), (2, 2), (2, 4)])
+def test_quantize_pack_bit_exact_bit_pairs(dtype, bits):
+    _staged_quant_case(tl.small_workload(dtype=dtype, context=333, batch=2, n_q_heads=8,
+                                         n_kv_heads=2, bits_hi=bits[0], bits_lo=bits[1],
+                                         outlier_fixed=0))
+
+
+def test_quantize_degenerate_rows():
+    """All-zero token, constant channel, constant token: the rules for flat rows and zero
+    channels must give the oracle's codes and parameters."""
+    w = tl.small_workload(context=130, n_q_heads=1, n_kv_heads=1, saliency_ratio=0.5)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    K[0, 0, 5, :] = 0
+    V[0, 0, 5, :] = 0
+    K[0, 0, :, 7] = 0          # all-zero channel
+    V[0, 0, :, 9] = 1.25       # constant channel
+    V[0, 0, 11, :] = -0.5      # constant token
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    p_gpu = cache.scores(w.context).cpu().numpy()[0, 0]
+    u = oc.units[(0, 0)]
+    n_s = u.segments[0].hi.n
+    idx = cache.segment(0, 0, 0)[0].cpu().numpy()[0, 0]
+    assert tl.salient_sets_match(p_gpu, u.segments[0].p_tilde, idx, u.segments[0].hi.idx, n_s) == 0
+    assert tl.compare_segment(cache, oc, 0) == 0
+
+
+@pytest.mark.parametrize("kw", [
+    dict(context=512, n_q_heads=4, n_kv_heads=4),
+    dict(context=777, batch=2, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0),
+    dict(context=64, n_q_heads=8, n_kv_heads=1, rho_recent=0.3, rho_random=0.3),
+    dict(context=1, n_q_heads=2, n_kv_heads=1),
+    dict(context=1300, n_q_heads=2, n_kv_heads=2, band=20, saliency_ratio=0.3),
+])
+def test_normalized_scores_and_salient_sets(kw):
+    w = tl.small_workload(**kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    p_gpu = cache.scores(w.context).cpu().numpy()
+    idx_hi = cache.segment(0, 0, 0)[0].cpu().numpy()
+    idx_lo = cache.segment(0, 0, 1)[0].cpu().numpy()
+    swaps = 0
+    for (bi, kv), u in oc.units.items():
+        ref = u.segments[0].p_tilde
+        rel = np.abs(p_gpu[bi, kv] - ref) / np.maximum(np.abs(ref), 1e-30)
+        assert rel.max() <= 1e-4, rel.max()
+        n_s = u.segments[0].hi.n
+        swaps += tl.salient_sets_match(p_gpu[bi, kv], ref, idx_hi[bi, kv], u.segments[0].hi.idx, n_s)
+        got = np.concatenate([idx_hi[bi, kv], idx_lo[bi, kv]])
+        assert sorted(got.tolist()) == list(range(w.context))
+        assert np.all(np.diff(idx_hi[bi, kv]) > 0) and np.all(np.diff(idx_lo[bi, kv]) > 0)
+    assert swaps == 0   # no near-ties expected at these sizes
+
+
+def test_topk_ties_prefer_lower_index():
+    """Q = 0 makes every probe row uniform, so many columns tie exactly."""
+    w = tl.small_workload(context=200, n_q_heads=1, n_kv_heads=1, rho_recent=0.05, rho_random=0.0)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    Q.zero_()
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    p_gpu = cache.scores(w.context).cpu().numpy()[0, 0]
+    # the GPU's own scores, split by the oracle's rule, must give the GPU's lists
+    sal, reg = zo.split_salient(p_gpu.astype(np.float64), 80)
+    np.testing.assert_array_equal(cache.segment(0, 0, 0)[0].cpu().numpy()[0, 0], sal)
+    np.testing.assert_array_equal(cache.segment(0, 0, 1)[0].cpu().numpy()[0, 0], reg)
+
+
+@pytest.mark.parametrize("kw,steps", [
+    (dict(context=512, n_q_heads=4, n_kv_heads=4), 16),
+    (dict(context=300, batch=2, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0), 6),
+    (dict(context=70, n_q_heads=8, n_kv_heads=1, saliency_ratio=0.5), 4),
+    (dict(context=129, n_q_heads=2, n_kv_heads=2, saliency_ratio=0.0), 3),
+    (dict(context=129, n_q_heads=2, n_kv_heads=2, saliency_ratio=1.0), 3),
+    (dict(context=1, n_q_heads=1, n_kv_heads=1), 2),
+    (dict(context=200, n_q_heads=4, n_kv_heads=1, bits_hi=4, bits_lo=4), 3),
+    (dict(context=200, n_q_heads=4, n_kv_heads=1, bits_hi=2, bits_lo=2), 3),
+])
+def test_decode_attention_parity(kw, steps):
+    w = tl.small_workload(**kw)
+    worst, _, _ = tl.run_decode_parity(w, steps)
+    assert worst <= 2e-3
+
+
+@pytest.mark.parametrize("window,steps", [(16, 40), (100, 105)])
+def test_decode_across_window_recompression(window, steps):
+    """The tail is re-compressed after `window` steps: new segment codes must be bit-exact
+    (given equal salient sets) and attention must stay within tolerance."""
+    w = tl.small_workload(context=150, n_q_heads=4, n_kv_heads=2, window=window,
+                          rho_recent=0.1, rho_random=0.1)
+    worst, cache, oc = tl.run_decode_parity(w, steps)
+    assert worst <= 2e-3
+    import paper_2405_14256_b200 as zc
+    n_seg = zc.zc_num_segments(cache.handle)
+    assert n_seg == 1 + steps // window
+    for seg in range(1, n_seg):
+        p_gpu = None
+        # window scores are exported only for the latest compression
+        if seg == n_seg - 1:
+            p_gpu = cache.scores(window).cpu().numpy()
+        idx_hi = cache.segment(seg, 0, 0)[0].cpu().numpy()
+        for (bi, kv), u in oc.units.items():
+            s = u.segments[seg]
+            if p_gpu is not None:
+                rel = np.abs(p_gpu[bi, kv] - s.p_tilde) / np.maximum(s.p_tilde, 1e-30)
+                assert rel.max() <= 1e-3
+                tl.salient_sets_match(p_gpu[bi, kv], s.p_tilde, idx_hi[bi, kv], s.hi.idx, s.hi.n)
+            assert set(idx_hi[bi, kv].tolist()) == set(s.hi.idx.tolist())
+        assert tl.compare_segment(cache, oc, seg) == 0
+
+
+def test_end_to_end_config1_all_units():
+    w = get_config(1)
+    worst, cache, oc = tl.run_decode_parity(w, w.decode_steps, staged=False)
+    assert worst <= 2e-3
+    assert tl.compare_segment(cache, oc, 0) == 0
+
+
+def test_run_to_run_determinism():
+    w = tl.small_workload(context=400, n_q_heads=8, n_kv_heads=2, batch=2)
+    outs = []
+    for _ in range(3):
+        Q, K, V = make_prefill(w, 0, tl.DEV)
+        P = tl.probes_for(w)
+        cache = tl.make_cache(w)
+        cache.prefill_compress(Q, K, V, P.tolist())
+        from workloads import make_decode_step
+        q, k, v = make_decode_step(w, 0, 0, tl.DEV)
+        cache.append(k, v)
+        o = cache.decode_attention(q, True)
+        torch.cuda.synchronize()
+        outs.append((o.clone(), cache.mem.clone()))
+    for o, m in outs[1:]:
+        assert torch.equal(o, outs[0][0])
+    # codes, parameters and index lists are bitwise identical run to run
+    a = cache.segment(0, 1, 0)
+    assert torch.equal(outs[0][1][: 1024], outs[1][1][: 1024])
