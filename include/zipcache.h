@@ -136,6 +136,11 @@ int64_t zc_decode_bytes(const zc_cache* c);
 /* Kernel launches enqueued by this library since the handle was created. */
 int64_t zc_launch_count(const zc_cache* c);
 
+/* Synchronises the device and reads the library's device-side error word into *code
+ * [host]: 0 = none, 1 = a bounded wait on an asynchronous copy inside the decode kernel
+ * ran out (its output is then invalid).  Device code never traps or spins forever. */
+int zc_device_status(int* code);
+
 const char* zc_strerror(int status);
 
 #ifdef __cplusplus

@@ -59,6 +59,7 @@ _SIGS = {
                                     C.c_void_p, C.c_void_p, C.c_void_p]),
     "zc_decode_bytes": (C.c_int64, [C.c_void_p]),
     "zc_launch_count": (C.c_int64, [C.c_void_p]),
+    "zc_device_status": (C.c_int, [C.POINTER(C.c_int)]),
     "zc_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -195,6 +196,12 @@ def zc_decode_bytes(handle) -> int:
 
 def zc_launch_count(handle) -> int:
     return lib().zc_launch_count(handle)
+
+
+def zc_device_status() -> int:
+    code = C.c_int(0)
+    _check(lib().zc_device_status(C.byref(code)), "zc_device_status")
+    return code.value
 
 
 class ZipCache:

@@ -303,7 +303,8 @@ __global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay
 
   // compose the tile: 16-byte stores, consecutive threads -> consecutive addresses
   char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
-  const int code_words = zc_codes_bytes(bits) / 4;   // per tensor
+  const int sub_words = zc_sub_bytes(bits) / 4;
+  const int kw = 64 * bits;                           // K-code words per sub-block (= V-code words)
   const int per = 32 / bits;                          // codes per word
   const int total_vec = lay.tile_bytes[cls] / 16;
   for (int v = threadIdx.x; v < total_vec; v += 256) {
@@ -311,19 +312,18 @@ __global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int wi = 4 * v + q;
+      const int st = wi / sub_words, wl = wi % sub_words;
       unsigned word = 0;
-      if (wi < code_words) {
+      if (wl < kw) {
         // K: canonical order, token row of 4*bits words
         const int words_per_row = 4 * bits;
-        const int tok = wi / words_per_row, wr = wi % words_per_row;
+        const int tok = 16 * st + wl / words_per_row, wr = wl % words_per_row;
         for (int e = 0; e < per; ++e) word |= (unsigned)codesK[tok][wr * per + e] << (bits * e);
-      } else if (wi < 2 * code_words) {
-        // V: fragment order, 4 sub-tiles of 16 tokens
-        const int wv = wi - code_words;
-        const int sub_words = code_words / 4;
-        const int st = wv / sub_words, wl = wv % sub_words;
+      } else if (wl < 2 * kw) {
+        // V: fragment order of the 16-token sub-tile
+        const int wv = wl - kw;
         if (bits == 4) {
-          const int qd = wl >> 7, ln = (wl >> 2) & 31, jj = wl & 3;
+          const int qd = wv >> 7, ln = (wv >> 2) & 31, jj = wv & 3;
           const int j = 4 * qd + jj, g = ln >> 2, t = ln & 3;
           for (int p = 0; p < 8; ++p) {
             const int hi_row = p & 1, isB = (p >> 1) & 1, is1 = p >> 2;
@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay
             word |= (unsigned)codesV[16 * st + tau][ch] << (4 * p);
           }
         } else {
-          const int ln = wl >> 2, m = wl & 3, g = ln >> 2, t = ln & 3;
+          const int ln = wv >> 2, m = wv & 3, g = ln >> 2, t = ln & 3;
           for (int i = 0; i < 16; ++i) {
             const int is1 = i >> 3, pp = i & 7, e2 = pp >> 2, hi_row = (pp >> 1) & 1, isB = pp & 1;
             const int j = 2 * m + e2;
@@ -340,8 +340,8 @@ __global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay
           }
         }
       } else {
-        const int wp = wi - 2 * code_words;  // params: K then V, (s, z) pairs
-        const float* pf = wp < 2 * ZC_TILE ? &parK[0][0] + wp : &parV[0][0] + (wp - 2 * ZC_TILE);
+        const int wp = wl - 2 * kw;  // params: K (s, z) x 16 then V (s, z) x 16
+        const float* pf = wp < 32 ? &parK[16 * st][0] + wp : &parV[16 * st][0] + (wp - 32);
         word = __float_as_uint(*pf);
       }
       out[q] = word;

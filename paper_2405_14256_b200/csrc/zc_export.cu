@@ -29,10 +29,12 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
       idx_out[(long long)unit * n + t0 + i] = idx[t0 + i];
   }
   if (sz_out) {
-    const float* par = reinterpret_cast<const float*>(
-        tp + (tensor == 0 ? zc_tile_off_kpar(bits) : zc_tile_off_vpar(bits)));
-    for (int i = threadIdx.x; i < 2 * n_here; i += blockDim.x)
-      sz_out[((long long)unit * n + t0) * 2 + i] = par[i];
+    const int poff = tensor == 0 ? zc_sub_off_kpar(bits) : zc_sub_off_vpar(bits);
+    for (int i = threadIdx.x; i < 2 * n_here; i += blockDim.x) {
+      const int tl = i >> 1;
+      const float* par = reinterpret_cast<const float*>(tp + (tl / ZC_SUB) * zc_sub_bytes(bits) + poff);
+      sz_out[((long long)unit * n + t0) * 2 + i] = par[2 * (tl % ZC_SUB) + (i & 1)];
+    }
   }
   if (cf_out && tile == 0) {
     const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) +
@@ -44,11 +46,11 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
     for (int i = threadIdx.x; i < n_here * row_bytes; i += blockDim.x) {
       const int tl = i / row_bytes, m = i % row_bytes;
       unsigned byte = 0;
+      const char* sb = tp + (tl / ZC_SUB) * zc_sub_bytes(bits);
       if (tensor == 0) {
-        byte = reinterpret_cast<const unsigned char*>(tp)[tl * row_bytes + m];
+        byte = reinterpret_cast<const unsigned char*>(sb)[(tl % ZC_SUB) * row_bytes + m];
       } else {
-        const unsigned* vblk = reinterpret_cast<const unsigned*>(tp + zc_tile_off_vcodes(bits)) +
-                               (tl / ZC_SUB) * (64 * bits);
+        const unsigned* vblk = reinterpret_cast<const unsigned*>(sb + zc_sub_off_vcodes(bits));
         for (int e = 0; e < per; ++e) {
           int word, shift;
           zc_vcode_pos(bits, tl % ZC_SUB, m * per + e, &word, &shift);

@@ -141,9 +141,10 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   int s1 = budget - s0;
   int sp[2] = {s0, s1};
   for (int k = 0; k < 2; ++k) {
-    int s = std::max(1, std::min(std::min(sp[k], ZC_MAX_SPLIT_HOST), std::max(1, p.tiles0[k])));
-    p.tpi0[k] = std::max(1, zc_ceil_div(std::max(1, p.tiles0[k]), s));
-    p.split0[k] = std::max(1, zc_ceil_div(std::max(1, p.tiles0[k]), p.tpi0[k]));
+    const int subs = std::max(1, zc_ceil_div(c->n0[k], ZC_SUB));
+    const int s = std::max(1, std::min(std::min(sp[k], ZC_MAX_SPLIT_HOST), subs));
+    p.spi0[k] = zc_ceil_div(subs, s);
+    p.split0[k] = zc_ceil_div(subs, p.spi0[k]);
   }
   p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + (p.n_tail > 0 ? 1 : 0);
   return p;
@@ -379,5 +380,12 @@ int64_t zc_decode_bytes(const zc_cache* c) {
 }
 
 int64_t zc_launch_count(const zc_cache* c) { return c ? c->launches : 0; }
+
+int zc_device_status(int* code) {
+  if (!code) return ZC_EINVAL;
+  ZC_CUDA(cudaDeviceSynchronize());
+  ZC_CUDA(zc_device_error_code(code));
+  return ZC_OK;
+}
 
 }  // extern "C"

@@ -25,10 +25,10 @@
 //   off_scores     normalised scores of the latest compression
 //   off_idx        token index lists: segment 0 (salient then regular), then one
 //                  window-sized slot per re-compressed window
-// A tile of class c holds 64 tokens:
-//   [K codes 64 x 16*bits B, canonical nibble/crumb order per token row]
-//   [V codes 4 sub-tiles of 16 tokens, fragment order (see zc_layout.cuh)]
-//   [K params 64 x (scale, zero) f32][V params 64 x (scale, zero) f32]
+// A tile of class c holds 64 tokens as four sub-blocks of 16 tokens, each
+//   [K codes 16 x 16*bits B, canonical nibble/crumb order per token row]
+//   [V codes of the 16 tokens in MMA fragment order (see zc_layout.cuh)]
+//   [K params 16 x (scale, zero) f32][V params 16 x (scale, zero) f32]
 struct ZcLayout {
   int units, G, n_kv, window, dtype;
   int bits[2];
@@ -62,7 +62,7 @@ struct ZcDecodePlan {
   int n0[2], nw[2];        // tokens per class: segment 0, re-compressed windows
   int tiles0[2], tilesw[2];
   int split0[2];           // items covering segment 0, per class
-  int tpi0[2];             // tiles per item, per class
+  int spi0[2];             // 16-token sub-tiles per item, per class
   int n_tail;
   int items;               // items per unit
   int l0;
@@ -104,6 +104,7 @@ int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
                      cudaStream_t st);
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out,
                      int collect, float* ws, cudaStream_t st);
+int zc_device_error_code(int* out);
 int zc_launch_export_scores(zc_cache* c, float* out, int n, cudaStream_t st);
 int zc_launch_export_segment(zc_cache* c, const ZcSeg& seg, int tensor, int subset,
                              int32_t* idx, uint8_t* codes, float* sz, float* cf,

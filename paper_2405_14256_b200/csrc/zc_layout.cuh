@@ -14,11 +14,14 @@
 #pragma once
 #include "zc_internal.h"
 
-__host__ __device__ inline int zc_tile_bytes(int bits) { return ZC_TILE * (32 * bits + 16); }
-__host__ __device__ inline int zc_codes_bytes(int bits) { return ZC_TILE * 16 * bits; }  // one tensor
-__host__ __device__ inline int zc_tile_off_vcodes(int bits) { return zc_codes_bytes(bits); }
-__host__ __device__ inline int zc_tile_off_kpar(int bits) { return 2 * zc_codes_bytes(bits); }
-__host__ __device__ inline int zc_tile_off_vpar(int bits) { return 2 * zc_codes_bytes(bits) + ZC_TILE * 8; }
+// A tile is four self-contained sub-blocks of 16 tokens, so that one bulk copy brings
+// everything a warp needs for one MMA sub-tile:
+//   [K codes 16 rows x 16*bits B][V codes, fragment order][K (s,z) x 16][V (s,z) x 16]
+__host__ __device__ inline int zc_sub_bytes(int bits) { return ZC_SUB * (32 * bits + 16); }
+__host__ __device__ inline int zc_tile_bytes(int bits) { return (ZC_TILE / ZC_SUB) * zc_sub_bytes(bits); }
+__host__ __device__ inline int zc_sub_off_vcodes(int bits) { return 256 * bits; }
+__host__ __device__ inline int zc_sub_off_kpar(int bits) { return 512 * bits; }
+__host__ __device__ inline int zc_sub_off_vpar(int bits) { return 512 * bits + 128; }
 
 // Position of V code (token tau of a 16-token sub-tile, channel ch) inside the
 // sub-tile's block: returns the 32-bit word index and the bit shift in the word.
