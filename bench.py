@@ -197,6 +197,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--decode-steps", type=int, default=0,
+                    help="profiling only: fewer decode steps than the workload's own")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -221,7 +223,7 @@ def main():
     zc.load_library()
     w = get_config(args.config)
     R = args.layers
-    n_dec = w.decode_steps
+    n_dec = args.decode_steps or w.decode_steps
     # rank r owns layers r*R .. r*R+R-1 (independent units: no collective on the data path)
     layer_ids = [rank * R + i for i in range(R)]
     probes = [zc.zc_default_probes(w.context, w.rho_recent, w.rho_random, w.seed(ly))

@@ -340,9 +340,9 @@ __global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay
           }
         }
       } else {
-        const int wp = wl - 2 * kw;  // params: K (s, z) x 16 then V (s, z) x 16
-        const float* pf = wp < 32 ? &parK[16 * st][0] + wp : &parV[16 * st][0] + (wp - 32);
-        word = __float_as_uint(*pf);
+        const int wp = wl - 2 * kw;  // params: (sK, zK, sV, zV) per token
+        const int tk = 16 * st + (wp >> 2), f = wp & 3;
+        word = __float_as_uint(f < 2 ? parK[tk][f] : parV[tk][f - 2]);
       }
       out[q] = word;
     }

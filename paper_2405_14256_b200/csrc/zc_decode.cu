@@ -1,17 +1,18 @@
 // Append (Eq. 3) and single-query attention over the mixed-precision cache (Eq. 4, Alg. 3).
 //
-// Split-K: every unit's cache is cut into items (a range of 16-token sub-tiles of one
-// precision class of one segment, or the full-precision tail); one CTA per item produces a
-// partial (m, l, acc) per query head, and a combine kernel merges the partials in a fixed
+// Split-K in ONE launch: every unit's cache is cut into items (a range of 16-token
+// sub-tiles of one precision class of one segment, or up to 64 tokens of the
+// full-precision tail); one CTA per item produces a partial (m, l, acc) per query head,
+// and the CTA that arrives last at the unit's counter merges the partials in a fixed
 // order, writes the output and, on probe steps, adds the step's attention over the tail's
-// tokens to the window statistics.
+// tokens to the window statistics.  Nothing waits on another CTA.
 //
 // Dequantisation is folded so that it is never done per element:
 //   q . k_hat_t = s_t (q' . code_t - z_t sum(q')),  q' = q * c^K        (per run)
 //   o = c^V * (sum_t w_t code_t - sum_t w_t z_t),    w_t = a_t s_t
 // Both contractions run on tensor cores (warp-level m16n8k16, f16 operands, f32 accumulate)
-// with M = tokens for q'.code and M = channels for sum_t w_t code_t, N = the G query heads
-// of the KV head.  A masked 32-bit word of packed codes IS a pair of f16 subnormals
+// with M = tokens for q'.code and M = channels for sum_t w_t code_t, N = the query heads of
+// the KV head.  A masked 32-bit word of packed codes IS a pair of f16 subnormals
 // (code * 2^-24, times 16 / 4 / 64 for codes that sit higher in the word), which the
 // tensor cores multiply exactly; the power-of-two factors are folded into q' (per channel),
 // into the softmax weights (per token) and into the output rows.
@@ -29,16 +30,29 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kStages = 4;                 // ring depth per warp
 constexpr int kStageBytes = 2304;          // largest sub-block (4-bit)
 constexpr int kWarps = 4;
-constexpr int kRingBytes = kWarps * kStages * kStageBytes;   // 36864
+constexpr int kWarpRing = kStages * kStageBytes;             // 9216
+constexpr int kRingBytes = kWarps * kWarpRing;               // 36864
 constexpr int kWaitLimit = 1 << 22;
-constexpr float kPScale = 32768.f;         // 2^15: softmax weights are sent to f16 as p * s/smax * 2^15
+constexpr int kPExp = 12;      // softmax weights go to f16 as p * s^V * 2^kPExp / 2^ceil(log2 smax)
+constexpr float kTau = 3.5f;   // the running maximum is refreshed only when a logit exceeds it by this
+constexpr unsigned kFull = 0xffffffffu;
+
+// shared-memory map of k_decode
+constexpr int kOffBars = kRingBytes;                 // kWarps * kStages mbarriers
+constexpr int kOffQfrag = kOffBars + 128;            // q' B-fragments, 4 x 32 x uint4
+constexpr int kOffRed = kOffQfrag + 2048;            // [kWarps][4] |q'| maxima as bits
+constexpr int kOffWm = kOffRed + 64;                 // [kWarps][4] running maxima
+constexpr int kOffWl = kOffWm + 64;                  // [kWarps][4] sums
+constexpr int kOffWz = kOffWl + 64;                  // [kWarps][4] zero-point sums
+constexpr int kOffFlag = kOffWz + 64;
+constexpr int kDecodeSmem = kOffFlag + 64;
 
 __device__ int g_zc_error = 0;
 
 struct ItemDesc {
   int kind;      // 0 = compressed run, 1 = tail
   int cls, run;  // precision class, factor-block index
-  int sub_lo, sub_hi;  // absolute sub-tile range inside the class region
+  int sub_lo, sub_hi;  // absolute sub-tile range inside the class region (kind 1: sub_lo = tail item)
   int run_sub0;        // first sub-tile of the run
   int n_tok;           // tokens of the run (kind 0) or of the tail (kind 1)
 };
@@ -68,7 +82,7 @@ __device__ inline ItemDesc decode_item(const ZcDecodePlan& p, int it) {
     return d;
   }
   d.kind = 1; d.cls = 0; d.run = 0; d.run_sub0 = 0;
-  d.sub_lo = d.sub_hi = 0; d.n_tok = p.n_tail;
+  d.sub_lo = i2 - 2 * (p.n_seg - 1); d.sub_hi = d.sub_lo; d.n_tok = p.n_tail;
   return d;
 }
 
@@ -113,89 +127,46 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, int by
       "l"(src), "r"(bytes), "r"(zc_smem_u32(bar))
       : "memory");
 }
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;\n" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
+}
 
-// q' B-fragment geometry: channel offset (inside the lane's 32-channel slice) and the power
-// of two the matching A element carries, for MMA k-step ks and slot (0,1 -> b0; 2,3 -> b1).
-template <int BITS> __device__ __forceinline__ void qfrag_geom(int ks, int slot, int* ch, float* inv_sigma) {
+// Where channel `off` (0..31) of a lane's 32-channel slice of a K-code row sits in the MMA:
+// B-fragment register (2 * k-step + {0: k = 2t,2t+1; 1: k = 2t+8,2t+9}), half e of it, and the
+// inverse of the power of two that the matching masked code carries.
+template <int BITS> __device__ __forceinline__ void chan_slot(int off, int* reg, int* e, float* inv_sigma) {
   if (BITS == 4) {
-    const int jw = ks >> 1, hb = ks & 1;
-    const int odd = slot >> 1, hi = slot & 1;           // b1 <-> nibbles 2hb+1, 2hb+5 (x16)
-    *ch = 8 * jw + 2 * hb + odd + 4 * hi;
+    const int jw = off >> 3, hi = (off >> 2) & 1, hb = (off >> 1) & 1, odd = off & 1;
+    *reg = 2 * (2 * jw + hb) + odd;
+    *e = hi;
     *inv_sigma = odd ? (1.f / 16.f) : 1.f;
   } else {
-    const int jw = ks >> 2, e = ks & 3, hb = e >> 1, pr = e & 1;
-    const int odd = slot >> 1, hi = slot & 1;           // crumbs 4hb+2pr(+1), +8
-    *ch = 16 * jw + 4 * hb + 2 * pr + odd + 8 * hi;
-    const int pw = 2 * pr + odd;                         // sigma = 4^pw
+    const int jw = off >> 4, hi = (off >> 3) & 1, hb = (off >> 2) & 1, pr = (off >> 1) & 1, odd = off & 1;
+    *reg = 2 * (4 * jw + 2 * hb + pr) + odd;
+    *e = hi;
+    const int pw = 2 * pr + odd;   // sigma = 4^pw
     *inv_sigma = pw == 0 ? 1.f : (pw == 1 ? 0.25f : (pw == 2 ? (1.f / 16.f) : (1.f / 64.f)));
   }
 }
 
-// The compressed-run part of one item, for one warp.  A CTA serves up to four query heads
-// (h0 .. h0+Gl-1).  q' is split into two f16 numbers, q' = hi + lo, carried in MMA columns
-// n = head (hi) and n = 4 + head (lo): f16 alone would put ~1e-3 of rounding noise on the
-// logits of outlier key channels.
+// Compressed-run part of one item, one warp: prologue done by the CTA, stages primed.
+// Column n of the q' B-fragments is (head n >> 1, part n & 1) with q' = hi + lo in f16, so
+// that lane (g, t) receives both parts of head t for tokens g and g + 8 in its accumulator.
 template <int BITS>
-__device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* class_base, char* ring,
-                                             uint64_t* bars, const float* qp /*[G][128] smem*/,
-                                             const float* hscale /*[8] smem*/, float inv_smax, int h0,
-                                             int Gl, int warp, int lane, float (&oacc)[8][4],
-                                             float (&m)[2], float (&l)[2], float (&zacc)[2], int* err) {
+__device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* src0, char* my_ring,
+                                             uint64_t* my_bar, const uint32_t (&qb)[16], float qs,
+                                             float isc, float logK, int my_n, int warp, int lane,
+                                             float (&oacc)[8][4], float& m_out, float& l_out,
+                                             float& z_out, int* err) {
   constexpr int SB = ZC_SUB * (32 * BITS + 16);
   const int g = lane >> 2, t = lane & 3;
-  // ---- B fragments of q' for column n = g, and sum(q') consistent with the f16 rounding ----
-  uint32_t qb[8][2];
-  float qsum_mine = 0.f;
-  {
-    const int hl = g & 3, is_lo = g >> 2;
-    const bool live = hl < Gl;
-    const float hs = live ? hscale[h0 + hl] : 0.f;
-    const float* qrow = qp + (live ? h0 + hl : 0) * ZC_D + 32 * t;
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        __half hv[2];
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          int ch; float is;
-          qfrag_geom<BITS>(ks, 2 * r + e, &ch, &is);
-          const float x = live ? qrow[ch] * hs * is : 0.f;
-          const __half hi = __float2half_rn(x);
-          const __half lo = __float2half_rn(x - __half2float(hi));
-          hv[e] = is_lo ? lo : hi;
-          qsum_mine += __half2float(hv[e]) * (1.f / is);   // exact: is is a power of two
-        }
-        const __half2 h2 = __halves2half2(hv[0], hv[1]);
-        qb[ks][r] = *reinterpret_cast<const uint32_t*>(&h2);
-      }
-    }
-  }
-  qsum_mine += __shfl_xor_sync(0xffffffffu, qsum_mine, 1);
-  qsum_mine += __shfl_xor_sync(0xffffffffu, qsum_mine, 2);
-  // after the hi+lo columns are added, this thread holds local heads 2(t&1) and 2(t&1)+1
-  float zq[2], isc[2];
-#pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    const int hl = 2 * (t & 1) + e;
-    const float hs = hl < Gl ? hscale[h0 + hl] : 1.f;
-    const float qs = __shfl_sync(0xffffffffu, qsum_mine, hl * 4) +
-                     __shfl_sync(0xffffffffu, qsum_mine, (hl + 4) * 4);
-    isc[e] = 16777216.f / hs;           // D * 2^24 / head scale = q' . code
-    zq[e] = hl < Gl ? qs / hs : 0.f;    // sum(q')
-  }
-
-  const int n_sub = d.sub_hi - d.sub_lo;
-  const int my_n = (n_sub - warp + kWarps - 1) / kWarps;     // sub-tiles of this warp
-  char* my_ring = ring + warp * kStages * kStageBytes;
-  uint64_t* my_bar = bars + warp * kStages;
-  const char* src0 = class_base + (long long)(d.sub_lo + warp) * SB;
-  if (lane == 0) {
-    for (int s = 0; s < kStages && s < my_n; ++s) {
-      mbar_expect_tx(&my_bar[s], SB);
-      bulk_copy_g2s(my_ring + s * kStageBytes, src0 + (long long)s * kWarps * SB, SB, &my_bar[s]);
-    }
-  }
+  const bool odd_tok = BITS == 2 && (g & 1);
+  const float logKs = logK - (odd_tok ? 2.f : 0.f);      // weights of odd tokens carry 1/4 at 2 bits
+  const int srcA = 8 * t + g, srcB = 8 * t + 4 + g;
+  const int c0_src = (lane & ~3) | ((2 * t) & 3), c1_src = (lane & ~3) | ((2 * t + 1) & 3);
+  float m = -INFINITY, mo = 0.f, mthr = -INFINITY, l = 0.f, zacc = 0.f;
   bool dead = false;
   for (int i = 0; i < my_n; ++i) {
     const int s = i % kStages, parity = (i / kStages) & 1;
@@ -206,8 +177,7 @@ __device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* clas
       }
     }
     const char* st = my_ring + s * kStageBytes;
-    const int tok0 = (d.sub_lo - d.run_sub0 + warp + i * kWarps) * ZC_SUB;   // first token of the sub-tile
-    // ---- loads: K words of tokens g and g+8, V words, parameters ----
+    // ---- loads: K words of tokens g and g+8, V words, parameters (sK, zK, sV, zV) ----
     uint32_t kw[2][BITS];   // 4-bit: 4 words per token, 2-bit: 2 words per token
     uint32_t vw[2 * BITS];  // 4-bit: 8 words, 2-bit: 4 words
     if (BITS == 4) {
@@ -227,22 +197,20 @@ __device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* clas
       const uint4 c = *reinterpret_cast<const uint4*>(st + 512 + lane * 16);
       vw[0] = c.x; vw[1] = c.y; vw[2] = c.z; vw[3] = c.w;
     }
-    const float2 pk0 = *reinterpret_cast<const float2*>(st + 512 * BITS + g * 8);
-    const float2 pk1 = *reinterpret_cast<const float2*>(st + 512 * BITS + (g + 8) * 8);
-    const float2 pv0 = *reinterpret_cast<const float2*>(st + 512 * BITS + 128 + g * 8);
-    const float2 pv1 = *reinterpret_cast<const float2*>(st + 512 * BITS + 128 + (g + 8) * 8);
+    const float4 pa = *reinterpret_cast<const float4*>(st + 512 * BITS + g * 16);
+    const float4 pb = *reinterpret_cast<const float4*>(st + 512 * BITS + (g + 8) * 16);
 
-    // ---- S^T = codes(16 tokens x 128) . q'^T : 8 k-steps ----
-    float dacc[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- S^T = codes(16 tokens x 128) . q'^T : 8 k-steps, two accumulator chains ----
+    float dacc[4] = {0.f, 0.f, 0.f, 0.f}, dacc2[4] = {0.f, 0.f, 0.f, 0.f};
     if (BITS == 4) {
 #pragma unroll
       for (int jw = 0; jw < 4; ++jw) {
         const uint32_t w0 = kw[0][jw], w1 = kw[1][jw];
         const uint32_t a0[4] = {w0 & 0x000F000Fu, w1 & 0x000F000Fu, w0 & 0x00F000F0u, w1 & 0x00F000F0u};
-        zc_mma16816<__half>(dacc, a0, qb[2 * jw][0], qb[2 * jw][1]);
+        zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
         const uint32_t x0 = w0 >> 8, x1 = w1 >> 8;
         const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
-        zc_mma16816<__half>(dacc, a1, qb[2 * jw + 1][0], qb[2 * jw + 1][1]);
+        zc_mma16816<__half>(dacc2, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
       }
     } else {
 #pragma unroll
@@ -250,69 +218,52 @@ __device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* clas
 #pragma unroll
         for (int hb = 0; hb < 2; ++hb) {
           const uint32_t w0 = kw[0][jw] >> (8 * hb), w1 = kw[1][jw] >> (8 * hb);
+          const int ks = 4 * jw + 2 * hb;
           const uint32_t a0[4] = {w0 & 0x00030003u, w1 & 0x00030003u, w0 & 0x000C000Cu, w1 & 0x000C000Cu};
-          zc_mma16816<__half>(dacc, a0, qb[4 * jw + 2 * hb][0], qb[4 * jw + 2 * hb][1]);
+          zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
           const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
-          zc_mma16816<__half>(dacc, a1, qb[4 * jw + 2 * hb + 1][0], qb[4 * jw + 2 * hb + 1][1]);
+          zc_mma16816<__half>(dacc2, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
         }
       }
     }
-    // columns n and n+4 (hi and lo parts of q') live in lanes t and t^2: add them
-#pragma unroll
-    for (int e = 0; e < 4; ++e) dacc[e] += __shfl_xor_sync(0xffffffffu, dacc[e], 2);
-    // ---- logits (base 2), online softmax for local heads 2(t&1), +1 over tokens g, g+8 ----
-    const bool v0 = tok0 + g < d.n_tok, v1 = tok0 + g + 8 < d.n_tok;
-    float lg[2][2];  // [token slot][head]
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      lg[0][e] = v0 ? pk0.x * (dacc[e] * isc[e] - pk0.y * zq[e]) : -INFINITY;
-      lg[1][e] = v1 ? pk1.x * (dacc[2 + e] * isc[e] - pk1.y * zq[e]) : -INFINITY;
+    // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
+    const float D0 = (dacc[0] + dacc2[0]) + (dacc[1] + dacc2[1]);
+    const float D1 = (dacc[2] + dacc2[2]) + (dacc[3] + dacc2[3]);
+    // ---- logits (base 2) of head t for tokens g and g+8 ----
+    float lg0 = fmaf(-pa.y, qs, D0) * (pa.x * isc);
+    float lg1 = fmaf(-pb.y, qs, D1) * (pb.x * isc);
+    const int tok0 = (d.sub_lo - d.run_sub0 + warp + i * kWarps) * ZC_SUB;   // first token of the sub-tile
+    if (tok0 + ZC_SUB > d.n_tok) {
+      if (tok0 + g >= d.n_tok) lg0 = -INFINITY;
+      if (tok0 + g + 8 >= d.n_tok) lg1 = -INFINITY;
     }
-    float mx[2] = {fmaxf(lg[0][0], lg[1][0]), fmaxf(lg[0][1], lg[1][1])};
-#pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {
-      mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], o));
-      mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], o));
-    }
-    const float mn0 = fmaxf(m[0], mx[0]), mn1 = fmaxf(m[1], mx[1]);
-    if (mn0 > m[0] || mn1 > m[1]) {
-      const float c0 = zc_exp2(m[0] - mn0), c1 = zc_exp2(m[1] - mn1);
+    const float mx = fmaxf(lg0, lg1);
+    if (__any_sync(kFull, mx > mthr)) {
+      float mr = mx;
+      mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 4));
+      mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 8));
+      mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 16));
+      const float mn = fmaxf(m, mr);
+      const float corr = mn == -INFINITY ? 1.f : zc_exp2(m - mn);
+      l *= corr; zacc *= corr;
+      m = mn; mo = mn - logKs; mthr = mn + kTau;
+      const float c0 = __shfl_sync(kFull, corr, c0_src), c1 = __shfl_sync(kFull, corr, c1_src);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         oacc[j][0] *= c0; oacc[j][1] *= c1; oacc[j][2] *= c0; oacc[j][3] *= c1;
       }
-      l[0] *= c0; l[1] *= c1; zacc[0] *= c0; zacc[1] *= c1;
-      m[0] = mn0; m[1] = mn1;
     }
-    float p[2][2];
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      p[0][e] = zc_exp2(lg[0][e] - m[e]);
-      p[1][e] = zc_exp2(lg[1][e] - m[e]);
-      l[e] += p[0][e] + p[1][e];
-    }
-    // weights to f16: w' = p * s^V / smax * 2^15 (/4 for odd tokens at 2 bits)
-    const float sig = (BITS == 2 && (g & 1)) ? 0.25f : 1.f;
-    const float ws0 = pv0.x * inv_smax * kPScale * sig, ws1 = pv1.x * inv_smax * kPScale * sig;
-    const float zs0 = pv0.y / sig, zs1 = pv1.y / sig;   // zero points times sigma'
-    uint32_t X[2];
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const __half2 h2 = __floats2half2_rn(p[0][e] * ws0, p[1][e] * ws1);   // (token g, token g+8)
-      const float2 back = __half22float2(h2);
-      zacc[e] += back.x * zs0 + back.y * zs1;
-      X[e] = *reinterpret_cast<const uint32_t*>(&h2);
-    }
-    // B fragment of P^T for column n = g (local head g & 3, held by lanes t' = (g & 3) >> 1):
-    // (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
-    const uint32_t sendA = (g & 1) ? X[1] : X[0];
-    const uint32_t sendB = (g & 1) ? X[0] : X[1];
-    const int odd = g & 1;
-    const int srcA = ((2 * t + odd) << 2) | ((g & 3) >> 1);
-    const int srcB = ((2 * t + 1 - odd) << 2) | ((g & 3) >> 1);
-    const uint32_t rA = __shfl_sync(0xffffffffu, sendA, srcA);
-    const uint32_t rB = __shfl_sync(0xffffffffu, sendB, srcB);
-    const uint32_t pb0 = odd ? rB : rA, pb1 = odd ? rA : rB;
+    // p' = p * 2^logKs; weights w = p' * s^V go to f16, the same rounded values feed the z sum
+    const float p0 = zc_exp2(lg0 - mo), p1 = zc_exp2(lg1 - mo);
+    l += p0 + p1;
+    const __half2 h2 = __floats2half2_rn(p0 * pa.z, p1 * pb.z);   // (token g, token g+8)
+    const float2 back = __half22float2(h2);
+    zacc = fmaf(back.x, pa.w, zacc);
+    zacc = fmaf(back.y, pb.w, zacc);
+    const uint32_t X = *reinterpret_cast<const uint32_t*>(&h2);
+    // B fragment of P^T, column n = g = head g: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
+    uint32_t pb0 = __shfl_sync(kFull, X, srcA), pb1 = __shfl_sync(kFull, X, srcB);
+    if (g >= 4) { pb0 = 0u; pb1 = 0u; }
     // ---- O^T += V^T(128 channels x 16 tokens) . P^T : 8 M-tiles ----
     if (BITS == 4) {
 #pragma unroll
@@ -340,208 +291,389 @@ __device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* clas
                     &my_bar[s]);
     }
   }
+  // sums back to plain units: l' = sum p 2^logKs; zacc' = sum w z with w short by the odd-token 1/4
+  const float inv_sig = odd_tok ? 4.f : 1.f;
+  l_out = l * zc_exp2(-logKs);
+  z_out = zacc * inv_sig;
+  m_out = m;
+}
+
+// One compressed item, whole CTA.  On return every warp has put its (m, l, z-sum) and its
+// accumulators into shared memory; *chan_factor / *rowscale tell the merge how to bring a
+// channel's accumulator to true units.
+template <typename T, int BITS>
+__device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* class_base,
+                                                const float* fac, const T* qbase, int Gl, char* smem,
+                                                float* chan_factor, float* rowscale, int* err) {
+  constexpr int SB = ZC_SUB * (32 * BITS + 16);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  char* my_ring = smem + warp * kWarpRing;
+  uint64_t* my_bar = reinterpret_cast<uint64_t*>(smem + kOffBars) + warp * kStages;
+  uint4* qfrag = reinterpret_cast<uint4*>(smem + kOffQfrag);
+  unsigned* s_red = reinterpret_cast<unsigned*>(smem + kOffRed);
+  float* wm = reinterpret_cast<float*>(smem + kOffWm);
+  float* wl = reinterpret_cast<float*>(smem + kOffWl);
+  float* wz = reinterpret_cast<float*>(smem + kOffWz);
+  const int n_sub = d.sub_hi - d.sub_lo;
+  const int my_n = n_sub > warp ? (n_sub - warp + kWarps - 1) / kWarps : 0;
+  const char* src0 = class_base + (long long)(d.sub_lo + warp) * SB;
+  // ---- start the copies first: their latency covers the q' set-up ----
+  if (lane == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(&my_bar[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    for (int s = 0; s < kStages && s < my_n; ++s) {
+      mbar_expect_tx(&my_bar[s], SB);
+      bulk_copy_g2s(my_ring + s * kStageBytes, src0 + (long long)s * kWarps * SB, SB, &my_bar[s]);
+    }
+  }
+  // ---- q' = q * c^K * log2(e)/sqrt(d); thread = channel ----
+  const float scale = kLog2e * rsqrtf((float)ZC_D);
+  const float cK = fac[tid];
+  float x[4];
+#pragma unroll
+  for (int h = 0; h < 4; ++h)
+    x[h] = h < Gl ? zc_to_float<T>(qbase[h * ZC_D + tid]) * cK * scale : 0.f;
+#pragma unroll
+  for (int h = 0; h < 4; ++h) {
+    const unsigned mb = __reduce_max_sync(kFull, __float_as_uint(fabsf(x[h])));
+    if (lane == 0) s_red[warp * 4 + h] = mb;
+  }
+  __syncthreads();
+  // per-head power of two that brings max |q'| into [2^13, 2^14): keeps the lo parts normal in f16
+  {
+    int reg, e;
+    float is;
+    chan_slot<BITS>(tid & 31, &reg, &e, &is);
+    const int t_l = tid >> 5;
+    __half* qh = reinterpret_cast<__half*>(qfrag);
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      const unsigned mb = max(max(s_red[h], s_red[4 + h]), max(s_red[8 + h], s_red[12 + h]));
+      const unsigned ex = mb >> 23;
+      const float hs = (ex >= 14u && ex < 255u) ? __uint_as_float((267u - ex) << 23) : 1.f;
+      const float xs = x[h] * hs * is;
+      const __half hi = __float2half_rn(xs);
+      const __half lo = __float2half_rn(xs - __half2float(hi));
+      const int base = ((reg >> 2) * 32 + t_l) * 4 + (reg & 3);          // + 4 * (4 * column)
+      qh[(base + 16 * (2 * h)) * 2 + e] = hi;
+      qh[(base + 16 * (2 * h + 1)) * 2 + e] = lo;
+    }
+  }
+  __syncthreads();
+  uint32_t qb[16];
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) {
+    const uint4 v = qfrag[q4 * 32 + lane];
+    qb[4 * q4] = v.x; qb[4 * q4 + 1] = v.y; qb[4 * q4 + 2] = v.z; qb[4 * q4 + 3] = v.w;
+  }
+  // sum of q' exactly as the f16 operands represent it: one MMA pass against all-one codes
+  float ds[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int ks = 0; ks < 8; ++ks) {
+    uint32_t one_lo, one_hi;
+    if (BITS == 4) { one_lo = 0x00010001u; one_hi = 0x00100010u; }
+    else if ((ks & 1) == 0) { one_lo = 0x00010001u; one_hi = 0x00040004u; }
+    else { one_lo = 0x00100010u; one_hi = 0x00400040u; }
+    const uint32_t a[4] = {one_lo, one_lo, one_hi, one_hi};
+    zc_mma16816<__half>(ds, a, qb[2 * ks], qb[2 * ks + 1]);
+  }
+  const float qs = ds[0] + ds[1];
+  float isc;
+  {
+    const unsigned mb = max(max(s_red[t], s_red[4 + t]), max(s_red[8 + t], s_red[12 + t]));
+    const unsigned ex = mb >> 23;
+    const float ihs = (ex >= 14u && ex < 255u) ? __uint_as_float((ex - 13u) << 23) : 1.f;
+    isc = 16777216.f * ihs;   // accumulator * 2^24 / head scale = q' . code
+  }
+  // weights are scaled by 2^logK = 2^kPExp / 2^ceil(log2 smax) so that w <= 2^(kPExp + kTau)
+  const float smax = fac[2 * ZC_D];
+  const int es = (int)((__float_as_uint(smax) >> 23) & 255u) - 127;
+  const float logK = (float)(kPExp - es - 1);
+
+  float oacc[8][4];
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
+  float m, l, z;
+  run_subtiles<BITS>(d, src0, my_ring, my_bar, qb, qs, isc, logK, my_n, warp, lane, oacc, m, l, z, err);
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    l += __shfl_xor_sync(kFull, l, o);
+    z += __shfl_xor_sync(kFull, z, o);
+  }
+  if (g == 0) { wm[warp * 4 + t] = m; wl[warp * 4 + t] = l; wz[warp * 4 + t] = z; }
+  // the warp's own ring is free (all of its copies were consumed): accumulators go there
+  float* mbuf = reinterpret_cast<float*>(my_ring);   // [4 heads][128]
+  __syncwarp();
+  if (t < 2) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        mbuf[(2 * t + e) * ZC_D + 16 * j + g] = oacc[j][e];
+        mbuf[(2 * t + e) * ZC_D + 16 * j + g + 8] = oacc[j][2 + e];
+      }
+    }
+  }
+  // o[ch] = c^V[ch] 2^-logK (acc 2^24 / sigma(row) - z sum); rows g+8 of a tile carry sigma = 16
+  *chan_factor = fac[ZC_D + tid] * zc_exp2(-logK);
+  *rowscale = (tid & 8) ? 1048576.f : 16777216.f;
+}
+
+// Up to 64 tokens of the full-precision tail, 16 per warp, on tensor cores in the input
+// type: S^T = K_tail q^T with q exact in its own type, then O^T = V_tail^T P^T with
+// P = hi + lo in the input type (columns 0..3 and 4..7).
+template <typename T>
+__device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, const ZcLayout& lay,
+                                          const T* qbase, int Gl, int unit, int h0, char* smem,
+                                          float* __restrict__ tail_logits) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  float* wm = reinterpret_cast<float*>(smem + kOffWm);
+  float* wl = reinterpret_cast<float*>(smem + kOffWl);
+  float* wz = reinterpret_cast<float*>(smem + kOffWz);
+  float* mbuf = reinterpret_cast<float*>(smem + warp * kWarpRing);   // [4 heads][128]
+  const int base = d.sub_lo * (kWarps * ZC_SUB) + warp * ZC_SUB;
+  const int nv = min(ZC_SUB, d.n_tok - base);
+  if (nv <= 0) {
+    if (lane < 4) { wm[warp * 4 + lane] = -INFINITY; wl[warp * 4 + lane] = 0.f; wz[warp * 4 + lane] = 0.f; }
+    return;
+  }
+  const T* tK = reinterpret_cast<const T*>(ub + lay.off_tailK);
+  const T* tV = reinterpret_cast<const T*>(ub + lay.off_tailV);
+  const int last = d.n_tok - 1;
+  // rows past the end are read from the last valid row and masked
+  const int r0 = min(base + g, last), r1 = min(base + g + 8, last);
+  const int va_r = min(base + 2 * t, last), vb_r = min(base + 2 * t + 8, last);
+  const int vc_r = min(base + 2 * t + 1, last), vd_r = min(base + 2 * t + 9, last);
+  uint4 qv[4], ka[4], kb[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    qv[c] = g < Gl ? *reinterpret_cast<const uint4*>(qbase + g * ZC_D + 32 * c + 8 * t) : make_uint4(0, 0, 0, 0);
+    ka[c] = *reinterpret_cast<const uint4*>(tK + r0 * ZC_D + 32 * c + 8 * t);
+    kb[c] = *reinterpret_cast<const uint4*>(tK + r1 * ZC_D + 32 * c + 8 * t);
+  }
+  // V: this lane's 16 channels (16g .. 16g+15) of the four tokens its fragments pair up
+  uint4 va[2], vb[2], vc[2], vd[2];
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    va[u] = *reinterpret_cast<const uint4*>(tV + va_r * ZC_D + 16 * g + 8 * u);
+    vb[u] = *reinterpret_cast<const uint4*>(tV + vb_r * ZC_D + 16 * g + 8 * u);
+    vc[u] = *reinterpret_cast<const uint4*>(tV + vc_r * ZC_D + 16 * g + 8 * u);
+    vd[u] = *reinterpret_cast<const uint4*>(tV + vd_r * ZC_D + 16 * g + 8 * u);
+  }
+  // ---- S^T: k-step (c, pp) contracts channels 32c + 8t + 4pp + {0,1 | 2,3} ----
+  float dacc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const uint32_t a0[4] = {ka[c].x, kb[c].x, ka[c].y, kb[c].y};
+    zc_mma16816<T>(dacc, a0, qv[c].x, qv[c].y);
+    const uint32_t a1[4] = {ka[c].z, kb[c].z, ka[c].w, kb[c].w};
+    zc_mma16816<T>(dacc, a1, qv[c].z, qv[c].w);
+  }
+  const float scale = kLog2e * rsqrtf((float)ZC_D);
+  const bool v0 = g < nv, v1 = g + 8 < nv;
+  float lg[2][2];   // [token slot][head 2t + e]
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    lg[0][e] = dacc[e] * scale;
+    lg[1][e] = dacc[2 + e] * scale;
+    const int h = 2 * t + e;
+    if (t < 2 && h < Gl) {
+      float* tl = tail_logits + ((long long)unit * lay.G + h0 + h) * ZC_MAX_WINDOW + base;
+      if (v0) tl[g] = lg[0][e];
+      if (v1) tl[g + 8] = lg[1][e];
+    }
+    if (!v0) lg[0][e] = -INFINITY;
+    if (!v1) lg[1][e] = -INFINITY;
+  }
+  float mx[2] = {fmaxf(lg[0][0], lg[1][0]), fmaxf(lg[0][1], lg[1][1])};
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    mx[0] = fmaxf(mx[0], __shfl_xor_sync(kFull, mx[0], o));
+    mx[1] = fmaxf(mx[1], __shfl_xor_sync(kFull, mx[1], o));
+  }
+  float ls[2] = {0.f, 0.f};
+  uint32_t Xhi[2], Xlo[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const float pa = zc_exp2(lg[0][e] - mx[e]), pb = zc_exp2(lg[1][e] - mx[e]);
+    ls[e] = pa + pb;
+    const T ha = zc_from_float<T>(pa), hb = zc_from_float<T>(pb);
+    const T la = zc_from_float<T>(pa - zc_to_float<T>(ha)), lb = zc_from_float<T>(pb - zc_to_float<T>(hb));
+    Xhi[e] = (uint32_t)(*reinterpret_cast<const unsigned short*>(&ha)) |
+             ((uint32_t)(*reinterpret_cast<const unsigned short*>(&hb)) << 16);
+    Xlo[e] = (uint32_t)(*reinterpret_cast<const unsigned short*>(&la)) |
+             ((uint32_t)(*reinterpret_cast<const unsigned short*>(&lb)) << 16);
+  }
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    ls[0] += __shfl_xor_sync(kFull, ls[0], o);
+    ls[1] += __shfl_xor_sync(kFull, ls[1], o);
+  }
+  // B fragment of P^T: column n = g is head g & 3, part g >> 2; (tokens 2t, 2t+8) come from
+  // lane (2t, head >> 1), (tokens 2t+1, 2t+9) from lane (2t+1, head >> 1)
+  const int hh = g & 3, srcA = 8 * t + (hh >> 1), srcB = srcA + 4;
+  uint32_t pb0, pb1;
+  {
+    const uint32_t a_h0 = __shfl_sync(kFull, Xhi[0], srcA), a_h1 = __shfl_sync(kFull, Xhi[1], srcA);
+    const uint32_t a_l0 = __shfl_sync(kFull, Xlo[0], srcA), a_l1 = __shfl_sync(kFull, Xlo[1], srcA);
+    const uint32_t b_h0 = __shfl_sync(kFull, Xhi[0], srcB), b_h1 = __shfl_sync(kFull, Xhi[1], srcB);
+    const uint32_t b_l0 = __shfl_sync(kFull, Xlo[0], srcB), b_l1 = __shfl_sync(kFull, Xlo[1], srcB);
+    const bool lo_part = g >= 4, second = hh & 1;
+    pb0 = lo_part ? (second ? a_l1 : a_l0) : (second ? a_h1 : a_h0);
+    pb1 = lo_part ? (second ? b_l1 : b_l0) : (second ? b_h1 : b_h0);
+  }
+  // ---- O^T: M-tile i has rows g <-> channel 16g + 2i, g + 8 <-> channel 16g + 2i + 1 ----
+  float oacc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t ra = (&va[i >> 2].x)[i & 3], rb = (&vb[i >> 2].x)[i & 3];
+    const uint32_t rc = (&vc[i >> 2].x)[i & 3], rd = (&vd[i >> 2].x)[i & 3];
+    const uint32_t a[4] = {prmt(ra, rb, 0x5410u), prmt(ra, rb, 0x7632u), prmt(rc, rd, 0x5410u),
+                           prmt(rc, rd, 0x7632u)};
+    oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+    zc_mma16816<T>(oacc[i], a, pb0, pb1);
+  }
+  // columns 4..7 (lanes t >= 2) hold the lo-part products of heads 0..3: add them in
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) oacc[i][e] += __shfl_xor_sync(kFull, oacc[i][e], 2);
+  if (t < 2) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      if (g == 0) { wm[warp * 4 + 2 * t + e] = mx[e]; wl[warp * 4 + 2 * t + e] = ls[e]; wz[warp * 4 + 2 * t + e] = 0.f; }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        mbuf[(2 * t + e) * ZC_D + 16 * g + 2 * i] = oacc[i][e];
+        mbuf[(2 * t + e) * ZC_D + 16 * g + 2 * i + 1] = oacc[i][2 + e];
+      }
+    }
+  }
 }
 
 template <typename T>
-__global__ void __launch_bounds__(128, 4) k_decode_items(char* cache, ZcLayout lay, ZcDecodePlan plan,
-                                                         const T* __restrict__ q, float* __restrict__ part,
-                                                         float* __restrict__ tail_logits) {
+__global__ void __launch_bounds__(128, 4) k_decode(char* cache, ZcLayout lay, ZcDecodePlan plan,
+                                                   const T* __restrict__ q, T* __restrict__ out,
+                                                   float* part, float* tail_logits, int collect) {
   extern __shared__ __align__(128) char smem[];
-  char* ring = smem;                                               // kRingBytes, reused for the merge
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kRingBytes);  // kWarps * kStages
-  float* qp = reinterpret_cast<float*>(smem + kRingBytes + 128);    // [8][128]
-  float* hscale = qp + ZC_MAX_G * ZC_D;                             // [8]
-  float* wm = hscale + 8;                                           // [4 warps][4 heads] maxima
-  float* wl = wm + 32;                                              // [4 warps][4 heads] sums
+  float* wm = reinterpret_cast<float*>(smem + kOffWm);
+  float* wl = reinterpret_cast<float*>(smem + kOffWl);
+  float* wz = reinterpret_cast<float*>(smem + kOffWz);
+  int* s_flag = reinterpret_cast<int*>(smem + kOffFlag);
   const int unit = blockIdx.y, it = blockIdx.x;
   const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
   const int h0 = 4 * blockIdx.z, Gl = min(4, G - h0);              // this CTA's query heads
   const ItemDesc d = decode_item(plan, it);
   char* ub = zc_unit_base(cache, lay, unit);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, t = lane & 3;
-  const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
-  const float scale = kLog2e * rsqrtf((float)ZC_D);
-  const bool has = d.kind == 0 ? d.sub_hi > d.sub_lo : d.n_tok > 0;
-  float* my = part + (((long long)unit * plan.items + it) * G) * ZC_PART_STRIDE;
+  const T* qbase = q + ((long long)b * lay.n_kv * G + kv * G + h0) * ZC_D;
+  float* my = part + (((long long)unit * plan.items + it) * G + h0) * ZC_PART_STRIDE;
 
-  if (tid == 0) {
-    for (int i = 0; i < kWarps * kStages; ++i) mbar_init(&bars[i], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-  }
-  {
-    const float cK = (d.kind == 0 && has) ? fac[tid] : 1.f;
-    for (int h = 0; h < Gl; ++h)
-      qp[(h0 + h) * ZC_D + tid] =
-          zc_to_float<T>(q[((long long)b * lay.n_kv * G + kv * G + h0 + h) * ZC_D + tid]) * cK * scale;
-  }
-  __syncthreads();
-  // per-head power-of-two scale that brings max |q'| under 2^14
-  for (int h = h0 + warp; h < h0 + Gl; h += kWarps) {
-    float mxq = 0.f;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) mxq = fmaxf(mxq, fabsf(qp[h * ZC_D + lane + 32 * e]));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mxq = fmaxf(mxq, __shfl_xor_sync(0xffffffffu, mxq, o));
-    if (lane == 0) hscale[h] = mxq > 0.f ? exp2f(floorf(14.f - log2f(mxq)) - 1.f) : 1.f;
-  }
-  __syncthreads();
-
-  float* mbuf = reinterpret_cast<float*>(ring);   // [kWarps][4 heads][128], after the main loop
+  float chan_factor = 1.f, rowscale = 1.f;
+  bool has = true;
   if (d.kind == 0) {
-    float oacc[8][4];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-#pragma unroll
-      for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
-    float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f}, zacc[2] = {0.f, 0.f};
+    has = d.sub_hi > d.sub_lo;
     if (has) {
-      const float smax = fac[2 * ZC_D];
-      const float inv_smax = smax > 0.f ? 1.f / smax : 0.f;
+      const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
       const char* class_base = ub + lay.off_tiles[d.cls];
       if (lay.bits[d.cls] == 4)
-        run_subtiles<4>(d, class_base, ring, bars, qp, hscale, inv_smax, h0, Gl, warp, lane, oacc, m,
-                        l, zacc, &g_zc_error);
+        compressed_item<T, 4>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
       else
-        run_subtiles<2>(d, class_base, ring, bars, qp, hscale, inv_smax, h0, Gl, warp, lane, oacc, m,
-                        l, zacc, &g_zc_error);
-      // bring the accumulators to true units:
-      //   o[ch][h] = c^V[ch] * smax * 2^-15 * (oacc * 2^24 / sigma(row) - zacc)
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-#pragma unroll
-        for (int o = 4; o < 32; o <<= 1) {
-          l[e] += __shfl_xor_sync(0xffffffffu, l[e], o);
-          zacc[e] += __shfl_xor_sync(0xffffffffu, zacc[e], o);
-        }
-      }
-      const float k0 = smax / kPScale;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float c_lo = fac[ZC_D + 16 * j + g] * k0, c_hi = fac[ZC_D + 16 * j + g + 8] * k0;
-        oacc[j][0] = c_lo * (oacc[j][0] * 16777216.f - zacc[0]);
-        oacc[j][1] = c_lo * (oacc[j][1] * 16777216.f - zacc[1]);
-        oacc[j][2] = c_hi * (oacc[j][2] * 1048576.f - zacc[0]);
-        oacc[j][3] = c_hi * (oacc[j][3] * 1048576.f - zacc[1]);
-      }
-    }
-    __syncthreads();   // the ring is free: every warp consumed all of its copies
-    // lanes t = 0, 1 hold local heads 2t, 2t+1 in accumulator columns 2t, 2t+1
-    if (t < 2) {
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int hl = 2 * t + e;
-        if (hl < Gl) {
-          if (g == 0) { wm[warp * 4 + hl] = m[e]; wl[warp * 4 + hl] = l[e]; }
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            mbuf[(warp * 4 + hl) * ZC_D + 16 * j + g] = oacc[j][e];
-            mbuf[(warp * 4 + hl) * ZC_D + 16 * j + g + 8] = oacc[j][2 + e];
-          }
-        }
-      }
+        compressed_item<T, 2>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
     }
   } else {
-    // ---- full-precision tail: one warp per token, lanes over channels, scalar FMAs ----
-    float tm[4], tl_[4], tacc[4][4];
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      tm[h] = -INFINITY; tl_[h] = 0.f;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) tacc[h][e] = 0.f;
-    }
-    for (int tok = warp; tok < d.n_tok; tok += kWarps) {
-      float kc[4], vc[4];
-      zc_load4<T>(reinterpret_cast<const T*>(ub + lay.off_tailK) + tok * ZC_D + 4 * lane, kc);
-      zc_load4<T>(reinterpret_cast<const T*>(ub + lay.off_tailV) + tok * ZC_D + 4 * lane, vc);
-#pragma unroll
-      for (int h = 0; h < 4; ++h) {
-        if (h < Gl) {
-          float dot = 0.f;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) dot += qp[(h0 + h) * ZC_D + 4 * lane + e] * kc[e];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          if (lane == 0) tail_logits[((long long)unit * G + h0 + h) * ZC_MAX_WINDOW + tok] = dot;
-          const float mn = fmaxf(tm[h], dot);
-          const float corr = zc_exp2(tm[h] - mn), pp = zc_exp2(dot - mn);
-          tl_[h] = tl_[h] * corr + pp;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) tacc[h][e] = tacc[h][e] * corr + pp * vc[e];
-          tm[h] = mn;
-        }
-      }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      if (h < Gl) {
-        if (lane == 0) { wm[warp * 4 + h] = tm[h]; wl[warp * 4 + h] = tl_[h]; }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) mbuf[(warp * 4 + h) * ZC_D + 4 * lane + e] = tacc[h][e];
-      }
-    }
+    tail_item<T>(d, ub, lay, qbase, Gl, unit, h0, smem, tail_logits);
   }
   __syncthreads();
-  // merge the warps: thread = channel
+  // ---- merge the warps: thread = channel ----
   for (int h = 0; h < Gl; ++h) {
-    float ms = -INFINITY;
+    float ms = -INFINITY, ls = 0.f, o = 0.f;
+    if (has) {
 #pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) ms = fmaxf(ms, wm[w2 * 4 + h]);
-    float ls = 0.f, o = 0.f;
+      for (int w2 = 0; w2 < kWarps; ++w2) ms = fmaxf(ms, wm[w2 * 4 + h]);
 #pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) {
-      const float mw = wm[w2 * 4 + h];
-      const float cw = mw == -INFINITY ? 0.f : zc_exp2(mw - ms);
-      ls += wl[w2 * 4 + h] * cw;
-      o += mbuf[(w2 * 4 + h) * ZC_D + tid] * cw;
+      for (int w2 = 0; w2 < kWarps; ++w2) {
+        const float mw = wm[w2 * 4 + h];
+        if (mw != -INFINITY) {
+          const float cw = zc_exp2(mw - ms);
+          const float acc = reinterpret_cast<const float*>(smem + w2 * kWarpRing)[h * ZC_D + tid];
+          ls += wl[w2 * 4 + h] * cw;
+          o += cw * (acc * rowscale - wz[w2 * 4 + h]);
+        }
+      }
+      o *= chan_factor;
     }
-    float* dst = my + (h0 + h) * ZC_PART_STRIDE;
+    float* dst = my + h * ZC_PART_STRIDE;
     if (tid == 0) { dst[0] = ms; dst[1] = ls; }
     dst[4 + tid] = o;
   }
-}
-
-template <typename T>
-__global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout lay, int items, int n_tail,
-                                                        int collect, const float* __restrict__ part,
-                                                        const float* __restrict__ tail_logits,
-                                                        T* __restrict__ out) {
-  __shared__ float s_m[ZC_MAX_G], s_l[ZC_MAX_G];
-  const int unit = blockIdx.x, tid = threadIdx.x, G = lay.G;
-  const int b = unit / lay.n_kv, kv = unit % lay.n_kv;
-  const float* mine = part + (long long)unit * items * G * ZC_PART_STRIDE;
-  if (tid < G) {
-    float ms = -INFINITY;
-    for (int i = 0; i < items; ++i) ms = fmaxf(ms, mine[(i * G + tid) * ZC_PART_STRIDE]);
-    float ls = 0.f;
-    for (int i = 0; i < items; ++i) {
-      const float* p = mine + (i * G + tid) * ZC_PART_STRIDE;
-      ls += p[1] * zc_exp2(p[0] - ms);
-    }
-    s_m[tid] = ms;
-    s_l[tid] = ls;
+  // ---- the CTA that arrives last at the unit's counter combines all partials ----
+  __threadfence();
+  __syncthreads();
+  unsigned* counter = reinterpret_cast<unsigned*>(ub + lay.off_sync);
+  if (tid == 0) {
+    const unsigned total = gridDim.x * gridDim.z;
+    const unsigned prev = atomicAdd(counter, 1u);
+    *s_flag = prev == total - 1u;
   }
   __syncthreads();
-  for (int g = 0; g < G; ++g) {
-    float o = 0.f;
-    for (int i = 0; i < items; ++i) {
-      const float* p = mine + (i * G + g) * ZC_PART_STRIDE;
-      o += p[4 + tid] * zc_exp2(p[0] - s_m[g]);
+  if (!*s_flag) return;
+  __threadfence();
+  const int items = plan.items;
+  const float* mine = part + (long long)unit * items * G * ZC_PART_STRIDE;
+  float* s_M = wm;   // [ZC_MAX_G]
+  float* s_L = wl;
+  for (int h = warp; h < G; h += kWarps) {
+    float mxh = -INFINITY;
+    for (int i = lane; i < items; i += 32) mxh = fmaxf(mxh, __ldcg(mine + (long long)(i * G + h) * ZC_PART_STRIDE));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mxh = fmaxf(mxh, __shfl_xor_sync(kFull, mxh, o));
+    float lsum = 0.f;
+    for (int i = lane; i < items; i += 32) {
+      const float* p = mine + (long long)(i * G + h) * ZC_PART_STRIDE;
+      const float mi = __ldcg(p);
+      if (mi != -INFINITY) lsum += __ldcg(p + 1) * zc_exp2(mi - mxh);
     }
-    out[((long long)b * lay.n_kv * G + kv * G + g) * ZC_D + tid] = zc_from_float<T>(o / s_l[g]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(kFull, lsum, o);
+    if (lane == 0) { s_M[h] = mxh; s_L[h] = lsum; }
   }
-  if (collect && tid < n_tail) {
+  __syncthreads();
+  for (int h = 0; h < G; ++h) {
+    const float mh = s_M[h];
+    float o = 0.f;
+    int i = 0;
+    for (; i + 4 <= items; i += 4) {
+      float mi[4], ai[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float* p = mine + (long long)((i + u) * G + h) * ZC_PART_STRIDE;
+        mi[u] = __ldcg(p);
+        ai[u] = __ldcg(p + 4 + tid);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (mi[u] != -INFINITY) o += ai[u] * zc_exp2(mi[u] - mh);
+    }
+    for (; i < items; ++i) {
+      const float* p = mine + (long long)(i * G + h) * ZC_PART_STRIDE;
+      const float mi = __ldcg(p);
+      if (mi != -INFINITY) o += __ldcg(p + 4 + tid) * zc_exp2(mi - mh);
+    }
+    out[((long long)b * lay.n_kv * G + kv * G + h) * ZC_D + tid] = zc_from_float<T>(o / s_L[h]);
+  }
+  if (collect && tid < plan.n_tail) {
     float a = 0.f;
-    for (int g = 0; g < G; ++g)
-      a += zc_exp2(tail_logits[((long long)unit * G + g) * ZC_MAX_WINDOW + tid] - s_m[g]) / s_l[g];
-    float* colsum = reinterpret_cast<float*>(zc_unit_base(cache, lay, unit) + lay.off_colsum);
+    for (int h = 0; h < G; ++h)
+      a += zc_exp2(__ldcg(tail_logits + ((long long)unit * G + h) * ZC_MAX_WINDOW + tid) - s_M[h]) / s_L[h];
+    float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
     colsum[tid] += a;
   }
+  if (tid == 0) *counter = 0u;   // ready for the next call
 }
-
-constexpr int kDecodeSmem = kRingBytes + 128 + (ZC_MAX_G * ZC_D + 8 + 64) * 4;
 
 }  // namespace
 
@@ -564,23 +696,20 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   dim3 grid(plan.items, c->lay.units, (G + 3) / 4);
   cudaError_t e;
   if (c->cfg.dtype == ZC_F16) {
-    e = cudaFuncSetAttribute(k_decode_items<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(k_decode<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
+    if (e != cudaSuccess) return e;
+    k_decode<__half><<<grid, 128, kDecodeSmem, st>>>(c->base, c->lay, plan, (const __half*)q,
+                                                     (__half*)out, part, tail_logits, collect);
+  } else {
+    e = cudaFuncSetAttribute(k_decode<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kDecodeSmem);
     if (e != cudaSuccess) return e;
-    k_decode_items<__half><<<grid, 128, kDecodeSmem, st>>>(c->base, c->lay, plan, (const __half*)q,
-                                                           part, tail_logits);
-    k_decode_combine<__half><<<c->lay.units, 128, 0, st>>>(c->base, c->lay, plan.items, plan.n_tail,
-                                                           collect, part, tail_logits, (__half*)out);
-  } else {
-    e = cudaFuncSetAttribute(k_decode_items<__nv_bfloat16>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
-    if (e != cudaSuccess) return e;
-    k_decode_items<__nv_bfloat16><<<grid, 128, kDecodeSmem, st>>>(
-        c->base, c->lay, plan, (const __nv_bfloat16*)q, part, tail_logits);
-    k_decode_combine<__nv_bfloat16><<<c->lay.units, 128, 0, st>>>(
-        c->base, c->lay, plan.items, plan.n_tail, collect, part, tail_logits, (__nv_bfloat16*)out);
+    k_decode<__nv_bfloat16><<<grid, 128, kDecodeSmem, st>>>(c->base, c->lay, plan,
+                                                            (const __nv_bfloat16*)q,
+                                                            (__nv_bfloat16*)out, part, tail_logits,
+                                                            collect);
   }
-  c->launches += 2;
+  c->launches += 1;
   return cudaGetLastError();
 }
 

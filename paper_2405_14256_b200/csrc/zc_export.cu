@@ -29,11 +29,11 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
       idx_out[(long long)unit * n + t0 + i] = idx[t0 + i];
   }
   if (sz_out) {
-    const int poff = tensor == 0 ? zc_sub_off_kpar(bits) : zc_sub_off_vpar(bits);
+    const int poff = zc_sub_off_par(bits);
     for (int i = threadIdx.x; i < 2 * n_here; i += blockDim.x) {
       const int tl = i >> 1;
       const float* par = reinterpret_cast<const float*>(tp + (tl / ZC_SUB) * zc_sub_bytes(bits) + poff);
-      sz_out[((long long)unit * n + t0) * 2 + i] = par[2 * (tl % ZC_SUB) + (i & 1)];
+      sz_out[((long long)unit * n + t0) * 2 + i] = par[4 * (tl % ZC_SUB) + 2 * tensor + (i & 1)];
     }
   }
   if (cf_out && tile == 0) {

@@ -68,6 +68,8 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   off = align_up(off + (size_t)cfg->window * ZC_D * elt, 256);
   lay->off_colsum = (long long)off;
   off = align_up(off + ZC_MAX_WINDOW * 4, 256);
+  lay->off_sync = (long long)off;   // directly after colsum: both are cleared together
+  off = align_up(off + 256, 256);
   lay->off_scores = (long long)off;
   off = align_up(off + (size_t)std::max(cfg->max_prefill, cfg->window) * 4, 256);
   lay->off_idx = (long long)off;
@@ -80,7 +82,8 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
     size_t pre = align_up((size_t)np_max * 4, 256) +
                  (size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4;
     // decode: partials [unit][item][G][ZC_PART_STRIDE] + tail logits [unit][G][window]
-    const int max_items = 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush + 1;
+    const int max_items = 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush +
+                          zc_ceil_div(ZC_MAX_WINDOW, ZC_TAIL_ITEM_TOKENS);
     size_t dec = (size_t)lay->units * max_items * lay->G * ZC_PART_STRIDE * 4 +
                  (size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4 + 256;
     *ws_bytes = align_up(std::max(pre, dec), 256);
@@ -132,8 +135,9 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   }
   // One wave of CTAs over all SMs when the units allow it: budget items per unit, then
   // share them between the two classes in proportion to their bytes.
+  p.tail_items = zc_ceil_div(c->n_tail, ZC_TAIL_ITEM_TOKENS);
   const int slots = c->n_sm * ZC_DECODE_CTAS_PER_SM;
-  int budget = slots / c->lay.units - (c->n_tail > 0 ? 1 : 0) - 2 * (c->n_seg - 1);
+  int budget = slots / c->lay.units - p.tail_items - 2 * (c->n_seg - 1);
   budget = std::max(2, std::min(budget, 2 * ZC_MAX_SPLIT_HOST));
   const long long tot = std::max(1LL, bytes[0] + bytes[1]);
   int s0 = (int)((bytes[0] * budget + tot / 2) / tot);
@@ -146,7 +150,7 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
     p.spi0[k] = zc_ceil_div(subs, s);
     p.split0[k] = zc_ceil_div(subs, p.spi0[k]);
   }
-  p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + (p.n_tail > 0 ? 1 : 0);
+  p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + p.tail_items;
   return p;
 }
 
@@ -275,9 +279,10 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
   c->n_new = 0;
   memset(c->tail_nnz, 0, sizeof(c->tail_nnz));
   c->last_scores_n = l;
-  // window statistics start at zero
+  // window statistics and the decode kernel's arrival counter start at zero
   ZC_CUDA(cudaMemset2DAsync(c->base + c->lay.off_colsum, (size_t)c->lay.unit_stride, 0,
-                            ZC_MAX_WINDOW * 4, (size_t)c->lay.units, st));
+                            (size_t)(c->lay.off_sync + 256 - c->lay.off_colsum),
+                            (size_t)c->lay.units, st));
   if (!salient_idx) {
     int32_t* P_dev = (int32_t*)workspace;
     float* lse = (float*)((char*)workspace + align_up((size_t)n_probe * 4, 256));

@@ -22,13 +22,14 @@
 //   off_cmax       scratch: |x| channel maxima as uint bits  [class][tensor][128]
 //   off_tailK/V    window x d elements of the input type
 //   off_colsum     window floats: attention mass collected on probe steps
+//   off_sync       arrival counter of the decode kernel's split-K items (zero between calls)
 //   off_scores     normalised scores of the latest compression
 //   off_idx        token index lists: segment 0 (salient then regular), then one
 //                  window-sized slot per re-compressed window
 // A tile of class c holds 64 tokens as four sub-blocks of 16 tokens, each
 //   [K codes 16 x 16*bits B, canonical nibble/crumb order per token row]
 //   [V codes of the 16 tokens in MMA fragment order (see zc_layout.cuh)]
-//   [K params 16 x (scale, zero) f32][V params 16 x (scale, zero) f32]
+//   [params 16 x (K scale, K zero, V scale, V zero) f32]
 struct ZcLayout {
   int units, G, n_kv, window, dtype;
   int bits[2];
@@ -37,7 +38,7 @@ struct ZcLayout {
   int max_runs;
   int idx_cap0;
   long long unit_stride;
-  long long off_tiles[2], off_fac, off_cmax, off_tailK, off_tailV, off_colsum, off_scores,
+  long long off_tiles[2], off_fac, off_cmax, off_tailK, off_tailV, off_colsum, off_sync, off_scores,
       off_idx;
 };
 
@@ -64,6 +65,7 @@ struct ZcDecodePlan {
   int split0[2];           // items covering segment 0, per class
   int spi0[2];             // 16-token sub-tiles per item, per class
   int n_tail;
+  int tail_items;          // items covering the tail (64 tokens each)
   int items;               // items per unit
   int l0;
 };
@@ -104,6 +106,7 @@ int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
                      cudaStream_t st);
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out,
                      int collect, float* ws, cudaStream_t st);
+#define ZC_TAIL_ITEM_TOKENS 64
 int zc_device_error_code(int* out);
 int zc_launch_export_scores(zc_cache* c, float* out, int n, cudaStream_t st);
 int zc_launch_export_segment(zc_cache* c, const ZcSeg& seg, int tensor, int subset,

@@ -16,12 +16,11 @@
 
 // A tile is four self-contained sub-blocks of 16 tokens, so that one bulk copy brings
 // everything a warp needs for one MMA sub-tile:
-//   [K codes 16 rows x 16*bits B][V codes, fragment order][K (s,z) x 16][V (s,z) x 16]
+//   [K codes 16 rows x 16*bits B][V codes, fragment order][(sK, zK, sV, zV) x 16]
 __host__ __device__ inline int zc_sub_bytes(int bits) { return ZC_SUB * (32 * bits + 16); }
 __host__ __device__ inline int zc_tile_bytes(int bits) { return (ZC_TILE / ZC_SUB) * zc_sub_bytes(bits); }
 __host__ __device__ inline int zc_sub_off_vcodes(int bits) { return 256 * bits; }
-__host__ __device__ inline int zc_sub_off_kpar(int bits) { return 512 * bits; }
-__host__ __device__ inline int zc_sub_off_vpar(int bits) { return 512 * bits + 128; }
+__host__ __device__ inline int zc_sub_off_par(int bits) { return 512 * bits; }
 
 // Position of V code (token tau of a 16-token sub-tile, channel ch) inside the
 // sub-tile's block: returns the 32-bit word index and the bit shift in the word.
