@@ -40,12 +40,15 @@ constexpr unsigned kFull = 0xffffffffu;
 // shared-memory map of k_decode
 constexpr int kOffBars = kRingBytes;                 // kWarps * kStages mbarriers
 constexpr int kOffQfrag = kOffBars + 128;            // q' B-fragments, 4 x 32 x uint4
-constexpr int kOffRed = kOffQfrag + 2048;            // [kWarps][4] |q'| maxima as bits
+constexpr int kOffRed = kOffQfrag + 2048;            // [kWarps] |q'| maxima as bits
 constexpr int kOffWm = kOffRed + 64;                 // [kWarps][4] running maxima
 constexpr int kOffWl = kOffWm + 64;                  // [kWarps][4] sums
 constexpr int kOffWz = kOffWl + 64;                  // [kWarps][4] zero-point sums
-constexpr int kOffFlag = kOffWz + 64;
+constexpr int kOffCw = kOffWz + 64;                  // [4 heads][kWarps] merge weights
+constexpr int kOffHead = kOffCw + 64;                // [4 heads] x (M, L, Z, -)
+constexpr int kOffFlag = kOffHead + 64;
 constexpr int kDecodeSmem = kOffFlag + 64;
+constexpr int kMaxItems = ZC_MAX_ITEMS;              // partial (m, l) pairs staged in the ring
 
 __device__ int g_zc_error = 0;
 
@@ -86,9 +89,19 @@ __device__ inline ItemDesc decode_item(const ZcDecodePlan& p, int it) {
   return d;
 }
 
+// Programmatic dependent launch: the next kernel in the stream may start once every CTA has
+// passed launch_dependents; wait() returns when the previous kernel has completed and its
+// writes are visible.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+
 template <typename T>
 __global__ void k_append(char* cache, ZcLayout lay, const T* __restrict__ k_new,
                          const T* __restrict__ v_new, int pos) {
+  pdl_launch_dependents();
+  pdl_wait();   // k_new / v_new may come from the previous kernel; the tail may still be read by it
   const int unit = blockIdx.x;
   char* ub = zc_unit_base(cache, lay, unit);
   T* tk = reinterpret_cast<T*>(ub + lay.off_tailK) + pos * ZC_D;
@@ -164,7 +177,8 @@ __device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* src0
   const int g = lane >> 2, t = lane & 3;
   const bool odd_tok = BITS == 2 && (g & 1);
   const float logKs = logK - (odd_tok ? 2.f : 0.f);      // weights of odd tokens carry 1/4 at 2 bits
-  const int srcA = 8 * t + g, srcB = 8 * t + 4 + g;
+  // columns 4..7 of P^T repeat columns 0..3: their products land in accumulator columns no one reads
+  const int srcA = 8 * t + (g & 3), srcB = srcA + 4;
   const int c0_src = (lane & ~3) | ((2 * t) & 3), c1_src = (lane & ~3) | ((2 * t + 1) & 3);
   float m = -INFINITY, mo = 0.f, mthr = -INFINITY, l = 0.f, zacc = 0.f;
   bool dead = false;
@@ -261,9 +275,8 @@ __device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* src0
     zacc = fmaf(back.x, pa.w, zacc);
     zacc = fmaf(back.y, pb.w, zacc);
     const uint32_t X = *reinterpret_cast<const uint32_t*>(&h2);
-    // B fragment of P^T, column n = g = head g: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
-    uint32_t pb0 = __shfl_sync(kFull, X, srcA), pb1 = __shfl_sync(kFull, X, srcB);
-    if (g >= 4) { pb0 = 0u; pb1 = 0u; }
+    // B fragment of P^T, column n = g = head g & 3: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
+    const uint32_t pb0 = __shfl_sync(kFull, X, srcA), pb1 = __shfl_sync(kFull, X, srcB);
     // ---- O^T += V^T(128 channels x 16 tokens) . P^T : 8 M-tiles ----
     if (BITS == 4) {
 #pragma unroll
@@ -334,28 +347,28 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
 #pragma unroll
   for (int h = 0; h < 4; ++h)
     x[h] = h < Gl ? zc_to_float<T>(qbase[h * ZC_D + tid]) * cK * scale : 0.f;
-#pragma unroll
-  for (int h = 0; h < 4; ++h) {
-    const unsigned mb = __reduce_max_sync(kFull, __float_as_uint(fabsf(x[h])));
-    if (lane == 0) s_red[warp * 4 + h] = mb;
+  {
+    const float ax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
+    const unsigned mb = __reduce_max_sync(kFull, __float_as_uint(ax));
+    if (lane == 0) s_red[warp] = mb;
   }
   __syncthreads();
-  // per-head power of two that brings max |q'| into [2^13, 2^14): keeps the lo parts normal in f16
+  // one power of two per CTA that brings max |q'| into [2^13, 2^14): keeps the lo parts normal in f16
+  const unsigned ex_q = max(max(s_red[0], s_red[1]), max(s_red[2], s_red[3])) >> 23;
+  const bool scaled = ex_q >= 14u && ex_q < 255u;
   {
     int reg, e;
     float is;
     chan_slot<BITS>(tid & 31, &reg, &e, &is);
     const int t_l = tid >> 5;
     __half* qh = reinterpret_cast<__half*>(qfrag);
+    const float hs_is = (scaled ? __uint_as_float((267u - ex_q) << 23) : 1.f) * is;
+    const int base = ((reg >> 2) * 32 + t_l) * 4 + (reg & 3);          // + 4 * (4 * column)
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
-      const unsigned mb = max(max(s_red[h], s_red[4 + h]), max(s_red[8 + h], s_red[12 + h]));
-      const unsigned ex = mb >> 23;
-      const float hs = (ex >= 14u && ex < 255u) ? __uint_as_float((267u - ex) << 23) : 1.f;
-      const float xs = x[h] * hs * is;
+      const float xs = x[h] * hs_is;
       const __half hi = __float2half_rn(xs);
       const __half lo = __float2half_rn(xs - __half2float(hi));
-      const int base = ((reg >> 2) * 32 + t_l) * 4 + (reg & 3);          // + 4 * (4 * column)
       qh[(base + 16 * (2 * h)) * 2 + e] = hi;
       qh[(base + 16 * (2 * h + 1)) * 2 + e] = lo;
     }
@@ -379,13 +392,8 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
     zc_mma16816<__half>(ds, a, qb[2 * ks], qb[2 * ks + 1]);
   }
   const float qs = ds[0] + ds[1];
-  float isc;
-  {
-    const unsigned mb = max(max(s_red[t], s_red[4 + t]), max(s_red[8 + t], s_red[12 + t]));
-    const unsigned ex = mb >> 23;
-    const float ihs = (ex >= 14u && ex < 255u) ? __uint_as_float((ex - 13u) << 23) : 1.f;
-    isc = 16777216.f * ihs;   // accumulator * 2^24 / head scale = q' . code
-  }
+  // accumulator * 2^24 / CTA scale = q' . code
+  const float isc = 16777216.f * (scaled ? __uint_as_float((ex_q - 13u) << 23) : 1.f);
   // weights are scaled by 2^logK = 2^kPExp / 2^ceil(log2 smax) so that w <= 2^(kPExp + kTau)
   const float smax = fac[2 * ZC_D];
   const int es = (int)((__float_as_uint(smax) >> 23) & 255u) - 127;
@@ -438,6 +446,7 @@ __device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, con
   const int nv = min(ZC_SUB, d.n_tok - base);
   if (nv <= 0) {
     if (lane < 4) { wm[warp * 4 + lane] = -INFINITY; wl[warp * 4 + lane] = 0.f; wz[warp * 4 + lane] = 0.f; }
+    for (int i = lane; i < 4 * ZC_D; i += 32) mbuf[i] = 0.f;
     return;
   }
   const T* tK = reinterpret_cast<const T*>(ub + lay.off_tailK);
@@ -562,7 +571,10 @@ __global__ void __launch_bounds__(128, 4) k_decode(char* cache, ZcLayout lay, Zc
   float* wm = reinterpret_cast<float*>(smem + kOffWm);
   float* wl = reinterpret_cast<float*>(smem + kOffWl);
   float* wz = reinterpret_cast<float*>(smem + kOffWz);
+  float* s_cw = reinterpret_cast<float*>(smem + kOffCw);
+  float* s_head = reinterpret_cast<float*>(smem + kOffHead);
   int* s_flag = reinterpret_cast<int*>(smem + kOffFlag);
+  pdl_launch_dependents();
   const int unit = blockIdx.y, it = blockIdx.x;
   const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
   const int h0 = 4 * blockIdx.z, Gl = min(4, G - h0);              // this CTA's query heads
@@ -585,29 +597,43 @@ __global__ void __launch_bounds__(128, 4) k_decode(char* cache, ZcLayout lay, Zc
         compressed_item<T, 2>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
     }
   } else {
+    pdl_wait();   // the newest tail row is written by the append kernel just before this one
     tail_item<T>(d, ub, lay, qbase, Gl, unit, h0, smem, tail_logits);
   }
   __syncthreads();
-  // ---- merge the warps: thread = channel ----
+  // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
+  if (tid < 4) {
+    float ms = -INFINITY;
+#pragma unroll
+    for (int w2 = 0; w2 < kWarps; ++w2) ms = fmaxf(ms, wm[w2 * 4 + tid]);
+    float ls = 0.f, zs = 0.f;
+#pragma unroll
+    for (int w2 = 0; w2 < kWarps; ++w2) {
+      const float mw = wm[w2 * 4 + tid];
+      const float cw = (has && mw != -INFINITY) ? zc_exp2(mw - ms) : 0.f;
+      s_cw[tid * 4 + w2] = cw;
+      ls += wl[w2 * 4 + tid] * cw;
+      zs += wz[w2 * 4 + tid] * cw;
+    }
+    s_head[tid * 4] = has ? ms : -INFINITY;
+    s_head[tid * 4 + 1] = has ? ls : 0.f;
+    s_head[tid * 4 + 2] = has ? zs : 0.f;
+  }
+  __syncthreads();
+  // everything this CTA writes to global memory may still be in use by the previous kernel
+  pdl_wait();
   for (int h = 0; h < Gl; ++h) {
-    float ms = -INFINITY, ls = 0.f, o = 0.f;
+    float o = 0.f;
     if (has) {
-#pragma unroll
-      for (int w2 = 0; w2 < kWarps; ++w2) ms = fmaxf(ms, wm[w2 * 4 + h]);
-#pragma unroll
-      for (int w2 = 0; w2 < kWarps; ++w2) {
-        const float mw = wm[w2 * 4 + h];
-        if (mw != -INFINITY) {
-          const float cw = zc_exp2(mw - ms);
-          const float acc = reinterpret_cast<const float*>(smem + w2 * kWarpRing)[h * ZC_D + tid];
-          ls += wl[w2 * 4 + h] * cw;
-          o += cw * (acc * rowscale - wz[w2 * 4 + h]);
-        }
-      }
-      o *= chan_factor;
+      const float4 cw = *reinterpret_cast<const float4*>(s_cw + h * 4);
+      const float a0 = reinterpret_cast<const float*>(smem)[h * ZC_D + tid];
+      const float a1 = reinterpret_cast<const float*>(smem + kWarpRing)[h * ZC_D + tid];
+      const float a2 = reinterpret_cast<const float*>(smem + 2 * kWarpRing)[h * ZC_D + tid];
+      const float a3 = reinterpret_cast<const float*>(smem + 3 * kWarpRing)[h * ZC_D + tid];
+      o = (rowscale * (((cw.x * a0 + cw.y * a1) + cw.z * a2) + cw.w * a3) - s_head[h * 4 + 2]) * chan_factor;
     }
     float* dst = my + h * ZC_PART_STRIDE;
-    if (tid == 0) { dst[0] = ms; dst[1] = ls; }
+    if (tid == 0) { dst[0] = s_head[h * 4]; dst[1] = s_head[h * 4 + 1]; }
     dst[4 + tid] = o;
   }
   // ---- the CTA that arrives last at the unit's counter combines all partials ----
@@ -624,68 +650,119 @@ __global__ void __launch_bounds__(128, 4) k_decode(char* cache, ZcLayout lay, Zc
   __threadfence();
   const int items = plan.items;
   const float* mine = part + (long long)unit * items * G * ZC_PART_STRIDE;
-  float* s_M = wm;   // [ZC_MAX_G]
-  float* s_L = wl;
+  float* s_m = reinterpret_cast<float*>(smem);          // [items * G] maxima, then weights
+  float* s_l = s_m + kMaxItems * ZC_MAX_G;              // [items * G] sums
+  float* s_ML = s_l + kMaxItems * ZC_MAX_G;             // [G] x (M, L)
+  for (int e = tid; e < items * G; e += 128) {
+    const float2 ml = __ldcg(reinterpret_cast<const float2*>(mine + (long long)e * ZC_PART_STRIDE));
+    s_m[e] = ml.x;
+    s_l[e] = ml.y;
+  }
+  // each warp owns heads warp, warp + 4: its first rows are requested before the barrier
+  constexpr int kChunk = 12;
+  float4 acc4[kChunk];
+  const int n_first = min(items, kChunk);
+  if (warp < G) {
+#pragma unroll
+    for (int u = 0; u < kChunk; ++u)
+      if (u < n_first)
+        acc4[u] = __ldcg(reinterpret_cast<const float4*>(mine + (long long)(u * G + warp) * ZC_PART_STRIDE + 4) + lane);
+  }
+  __syncthreads();
   for (int h = warp; h < G; h += kWarps) {
+    if (h != warp) {
+#pragma unroll
+      for (int u = 0; u < kChunk; ++u)
+        if (u < n_first)
+          acc4[u] = __ldcg(reinterpret_cast<const float4*>(mine + (long long)(u * G + h) * ZC_PART_STRIDE + 4) + lane);
+    }
     float mxh = -INFINITY;
-    for (int i = lane; i < items; i += 32) mxh = fmaxf(mxh, __ldcg(mine + (long long)(i * G + h) * ZC_PART_STRIDE));
+    for (int i = lane; i < items; i += 32) mxh = fmaxf(mxh, s_m[i * G + h]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mxh = fmaxf(mxh, __shfl_xor_sync(kFull, mxh, o));
     float lsum = 0.f;
     for (int i = lane; i < items; i += 32) {
-      const float* p = mine + (long long)(i * G + h) * ZC_PART_STRIDE;
-      const float mi = __ldcg(p);
-      if (mi != -INFINITY) lsum += __ldcg(p + 1) * zc_exp2(mi - mxh);
+      const float mi = s_m[i * G + h];
+      const float sc = mi == -INFINITY ? 0.f : zc_exp2(mi - mxh);
+      s_m[i * G + h] = sc;
+      lsum += s_l[i * G + h] * sc;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(kFull, lsum, o);
-    if (lane == 0) { s_M[h] = mxh; s_L[h] = lsum; }
-  }
-  __syncthreads();
-  for (int h = 0; h < G; ++h) {
-    const float mh = s_M[h];
-    float o = 0.f;
-    int i = 0;
-    for (; i + 4 <= items; i += 4) {
-      float mi[4], ai[4];
+    __syncwarp();
+    if (lane == 0) { s_ML[2 * h] = mxh; s_ML[2 * h + 1] = lsum; }
+    float4 o4 = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float* p = mine + (long long)((i + u) * G + h) * ZC_PART_STRIDE;
-        mi[u] = __ldcg(p);
-        ai[u] = __ldcg(p + 4 + tid);
+    for (int u = 0; u < kChunk; ++u) {
+      if (u < n_first) {
+        const float sc = s_m[u * G + h];
+        o4.x += acc4[u].x * sc; o4.y += acc4[u].y * sc; o4.z += acc4[u].z * sc; o4.w += acc4[u].w * sc;
       }
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (mi[u] != -INFINITY) o += ai[u] * zc_exp2(mi[u] - mh);
     }
-    for (; i < items; ++i) {
-      const float* p = mine + (long long)(i * G + h) * ZC_PART_STRIDE;
-      const float mi = __ldcg(p);
-      if (mi != -INFINITY) o += __ldcg(p + 4 + tid) * zc_exp2(mi - mh);
+    for (int i = kChunk; i < items; ++i) {
+      const float4 a = __ldcg(reinterpret_cast<const float4*>(mine + (long long)(i * G + h) * ZC_PART_STRIDE + 4) + lane);
+      const float sc = s_m[i * G + h];
+      o4.x += a.x * sc; o4.y += a.y * sc; o4.z += a.z * sc; o4.w += a.w * sc;
     }
-    out[((long long)b * lay.n_kv * G + kv * G + h) * ZC_D + tid] = zc_from_float<T>(o / s_L[h]);
+    const float inv = 1.f / lsum;
+    T r[4] = {zc_from_float<T>(o4.x * inv), zc_from_float<T>(o4.y * inv), zc_from_float<T>(o4.z * inv),
+              zc_from_float<T>(o4.w * inv)};
+    *reinterpret_cast<uint2*>(out + ((long long)b * lay.n_kv * G + kv * G + h) * ZC_D + 4 * lane) =
+        *reinterpret_cast<const uint2*>(r);
   }
-  if (collect && tid < plan.n_tail) {
-    float a = 0.f;
-    for (int h = 0; h < G; ++h)
-      a += zc_exp2(__ldcg(tail_logits + ((long long)unit * G + h) * ZC_MAX_WINDOW + tid) - s_M[h]) / s_L[h];
-    float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
-    colsum[tid] += a;
+  if (collect) {
+    __syncthreads();
+    if (tid < plan.n_tail) {
+      float a = 0.f;
+      for (int h = 0; h < G; ++h)
+        a += zc_exp2(__ldcg(tail_logits + ((long long)unit * G + h) * ZC_MAX_WINDOW + tid) - s_ML[2 * h]) /
+             s_ML[2 * h + 1];
+      float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
+      colsum[tid] += a;
+    }
   }
   if (tid == 0) *counter = 0u;   // ready for the next call
 }
 
 }  // namespace
 
+namespace {
+
+// Launch with the programmatic-stream-serialisation attribute: the kernel may start while the
+// previous kernel of the stream is still running and orders itself with pdl_wait().
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       bool overlap, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = overlap ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// Output range of the latest decode launch: a decode call whose q lies inside it must not
+// start before that launch has finished, because q is read ahead of pdl_wait().
+const char* g_last_out_lo = nullptr;
+const char* g_last_out_hi = nullptr;
+
+}  // namespace
+
 int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos, cudaStream_t st) {
+  cudaError_t e;
   if (c->cfg.dtype == ZC_F16)
-    k_append<__half><<<c->lay.units, 32, 0, st>>>(c->base, c->lay, (const __half*)k_new,
-                                                  (const __half*)v_new, pos);
+    e = launch_pdl(k_append<__half>, dim3(c->lay.units), dim3(32), 0, st, true, c->base, c->lay,
+                   (const __half*)k_new, (const __half*)v_new, pos);
   else
-    k_append<__nv_bfloat16><<<c->lay.units, 32, 0, st>>>(c->base, c->lay, (const __nv_bfloat16*)k_new,
-                                                         (const __nv_bfloat16*)v_new, pos);
+    e = launch_pdl(k_append<__nv_bfloat16>, dim3(c->lay.units), dim3(32), 0, st, true, c->base, c->lay,
+                   (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new, pos);
   c->launches += 1;
-  return cudaGetLastError();
+  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
@@ -694,23 +771,26 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   float* part = ws;
   float* tail_logits = ws + (size_t)c->lay.units * plan.items * G * ZC_PART_STRIDE;
   dim3 grid(plan.items, c->lay.units, (G + 3) / 4);
+  const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
+  const char* q_lo = (const char*)q;
+  const bool overlap = !(g_last_out_lo && q_lo < g_last_out_hi && q_lo + io_bytes > g_last_out_lo);
   cudaError_t e;
   if (c->cfg.dtype == ZC_F16) {
     e = cudaFuncSetAttribute(k_decode<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
     if (e != cudaSuccess) return e;
-    k_decode<__half><<<grid, 128, kDecodeSmem, st>>>(c->base, c->lay, plan, (const __half*)q,
-                                                     (__half*)out, part, tail_logits, collect);
+    e = launch_pdl(k_decode<__half>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay, plan,
+                   (const __half*)q, (__half*)out, part, tail_logits, collect);
   } else {
     e = cudaFuncSetAttribute(k_decode<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kDecodeSmem);
     if (e != cudaSuccess) return e;
-    k_decode<__nv_bfloat16><<<grid, 128, kDecodeSmem, st>>>(c->base, c->lay, plan,
-                                                            (const __nv_bfloat16*)q,
-                                                            (__nv_bfloat16*)out, part, tail_logits,
-                                                            collect);
+    e = launch_pdl(k_decode<__nv_bfloat16>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay,
+                   plan, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, part, tail_logits, collect);
   }
+  g_last_out_lo = (const char*)out;
+  g_last_out_hi = (const char*)out + io_bytes;
   c->launches += 1;
-  return cudaGetLastError();
+  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 
 int zc_device_error_code(int* out) {

@@ -30,6 +30,8 @@ int check_config(const zc_config* cfg) {
   if (cfg->reserved != 0) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if ((long long)cfg->batch * cfg->n_kv_heads > 65535) return ZC_EINVAL;
+  // every re-compressed window adds two items to a decode call
+  if (2 * (cfg->max_new_tokens / cfg->window) + 2 + 2 > ZC_MAX_ITEMS) return ZC_EINVAL;
   return ZC_OK;
 }
 
@@ -82,8 +84,8 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
     size_t pre = align_up((size_t)np_max * 4, 256) +
                  (size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4;
     // decode: partials [unit][item][G][ZC_PART_STRIDE] + tail logits [unit][G][window]
-    const int max_items = 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush +
-                          zc_ceil_div(ZC_MAX_WINDOW, ZC_TAIL_ITEM_TOKENS);
+    const int max_items = std::min(ZC_MAX_ITEMS, 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush +
+                                                     zc_ceil_div(ZC_MAX_WINDOW, ZC_TAIL_ITEM_TOKENS));
     size_t dec = (size_t)lay->units * max_items * lay->G * ZC_PART_STRIDE * 4 +
                  (size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4 + 256;
     *ws_bytes = align_up(std::max(pre, dec), 256);
@@ -125,30 +127,34 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   p.n_seg = c->n_seg;
   p.n_tail = c->n_tail;
   p.l0 = c->l0;
-  long long bytes[2];
   for (int k = 0; k < 2; ++k) {
     p.n0[k] = c->n0[k];
     p.nw[k] = c->nw[k];
     p.tiles0[k] = zc_ceil_div(c->n0[k], ZC_TILE);
     p.tilesw[k] = zc_ceil_div(c->nw[k], ZC_TILE);
-    bytes[k] = (long long)p.tiles0[k] * c->lay.tile_bytes[k];
   }
-  // One wave of CTAs over all SMs when the units allow it: budget items per unit, then
-  // share them between the two classes in proportion to their bytes.
+  // Items of segment 0 aim at ZC_ITEM_SUBS sub-tiles: few enough CTAs that their set-up and
+  // merge stay small next to the streaming loop, which overlaps with the neighbouring calls
+  // of the stream; with few units the split grows until one wave of CTAs covers the SMs.
   p.tail_items = zc_ceil_div(c->n_tail, ZC_TAIL_ITEM_TOKENS);
+  const int extras = p.tail_items + 2 * (c->n_seg - 1);
   const int slots = c->n_sm * ZC_DECODE_CTAS_PER_SM;
-  int budget = slots / c->lay.units - p.tail_items - 2 * (c->n_seg - 1);
-  budget = std::max(2, std::min(budget, 2 * ZC_MAX_SPLIT_HOST));
-  const long long tot = std::max(1LL, bytes[0] + bytes[1]);
-  int s0 = (int)((bytes[0] * budget + tot / 2) / tot);
-  s0 = std::max(1, std::min(s0, budget - 1));
-  int s1 = budget - s0;
-  int sp[2] = {s0, s1};
+  int subs[2], want[2];
   for (int k = 0; k < 2; ++k) {
-    const int subs = std::max(1, zc_ceil_div(c->n0[k], ZC_SUB));
-    const int s = std::max(1, std::min(std::min(sp[k], ZC_MAX_SPLIT_HOST), subs));
-    p.spi0[k] = zc_ceil_div(subs, s);
-    p.split0[k] = zc_ceil_div(subs, p.spi0[k]);
+    subs[k] = zc_ceil_div(c->n0[k], ZC_SUB);
+    want[k] = std::max(1, zc_ceil_div(subs[k], ZC_ITEM_SUBS));
+  }
+  const int fill = slots / (2 * c->lay.units) - extras;   // half a wave from this call alone
+  if (want[0] + want[1] < fill) {
+    const int tot = std::max(1, subs[0] + subs[1]);
+    for (int k = 0; k < 2; ++k) want[k] = std::max(want[k], (int)((long long)subs[k] * fill / tot));
+  }
+  const int cap = std::max(1, (ZC_MAX_ITEMS - extras) / 2);
+  for (int k = 0; k < 2; ++k) {
+    const int s = std::max(1, std::min(std::min(want[k], std::min(ZC_MAX_SPLIT_HOST, cap)),
+                                       std::max(1, subs[k])));
+    p.spi0[k] = zc_ceil_div(std::max(1, subs[k]), s);
+    p.split0[k] = zc_ceil_div(std::max(1, subs[k]), p.spi0[k]);
   }
   p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + p.tail_items;
   return p;

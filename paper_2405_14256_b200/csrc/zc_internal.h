@@ -13,6 +13,10 @@
 #define ZC_PART_STRIDE 132  // split-K partial per head: m, l, pad, pad, acc[128]
 #define ZC_MAX_G 8
 #define ZC_MAX_SPLIT_HOST 32      // most items one class of segment 0 is split into
+#define ZC_MAX_ITEMS 128          // most items of one unit in one decode call
+#ifndef ZC_ITEM_SUBS
+#define ZC_ITEM_SUBS 64           // 16-token sub-tiles one item of segment 0 aims at
+#endif
 #define ZC_DECODE_CTAS_PER_SM 4    // CTAs the decode kernel keeps resident per SM
 
 // Device-side description of the cache buffer.  One "unit" = (batch, KV head).
