@@ -1,11 +1,12 @@
 // Append (Eq. 3) and single-query attention over the mixed-precision cache (Eq. 4, Alg. 3).
 //
-// Split-K in ONE launch: every unit's cache is cut into items (a range of 16-token
-// sub-tiles of one precision class of one segment, or up to 64 tokens of the
-// full-precision tail); one CTA per item produces a partial (m, l, acc) per query head,
-// and the CTA that arrives last at the unit's counter merges the partials in a fixed
-// order, writes the output and, on probe steps, adds the step's attention over the tail's
-// tokens to the window statistics.  Nothing waits on another CTA.
+// Split-K: every unit's cache is cut into items (a range of 16-token sub-tiles of one
+// precision class of one segment, or up to 64 tokens of the full-precision tail); one CTA per
+// item produces a partial (m, l, acc) per query head, and a small second kernel merges the
+// partials in a fixed order, writes the output and, on probe steps, adds the step's attention
+// over the tail's tokens to the window statistics.  The kernels of one step (append, items,
+// combine) are chained by programmatic dependent launch: each may start while its
+// predecessor drains and orders itself with griddepcontrol.wait.  Nothing spins on another CTA.
 //
 // Dequantisation is folded so that it is never done per element:
 //   q . k_hat_t = s_t (q' . code_t - z_t sum(q')),  q' = q * c^K        (per run)
@@ -27,27 +28,27 @@
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kStages = 4;                 // ring depth per warp
-constexpr int kStageBytes = 2304;          // largest sub-block (4-bit)
+constexpr int kMaxStages = 5;              // ring depth per warp: 3 pairs at 4 bits, 5 at 2 bits
 constexpr int kWarps = 4;
-constexpr int kWarpRing = kStages * kStageBytes;             // 9216
-constexpr int kRingBytes = kWarps * kWarpRing;               // 36864
+constexpr int kWarpRing = 13824;           // 3 x 4608 (4-bit pair) >= 5 x 2560 (2-bit pair)
+constexpr int kRingBytes = kWarps * kWarpRing;               // 55296
+constexpr int kCtasPerSm = ZC_DECODE_CTAS_PER_SM;
 constexpr int kWaitLimit = 1 << 22;
 constexpr int kPExp = 12;      // softmax weights go to f16 as p * s^V * 2^kPExp / 2^ceil(log2 smax)
 constexpr float kTau = 3.5f;   // the running maximum is refreshed only when a logit exceeds it by this
 constexpr unsigned kFull = 0xffffffffu;
 
 // shared-memory map of k_decode
-constexpr int kOffBars = kRingBytes;                 // kWarps * kStages mbarriers
-constexpr int kOffQfrag = kOffBars + 128;            // q' B-fragments, 4 x 32 x uint4
+constexpr int kOffBars = kRingBytes;                 // kWarps * kMaxStages mbarriers
+constexpr int kOffQfrag = kOffBars + 256;            // q' B-fragments, 4 x 32 x uint4
 constexpr int kOffRed = kOffQfrag + 2048;            // [kWarps] |q'| maxima as bits
 constexpr int kOffWm = kOffRed + 64;                 // [kWarps][4] running maxima
 constexpr int kOffWl = kOffWm + 64;                  // [kWarps][4] sums
 constexpr int kOffWz = kOffWl + 64;                  // [kWarps][4] zero-point sums
 constexpr int kOffCw = kOffWz + 64;                  // [4 heads][kWarps] merge weights
 constexpr int kOffHead = kOffCw + 64;                // [4 heads] x (M, L, Z, -)
-constexpr int kOffFlag = kOffHead + 64;
-constexpr int kDecodeSmem = kOffFlag + 64;
+constexpr int kDecodeSmem = kOffHead + 64;
+constexpr int kCombineSmem = (2 * ZC_MAX_ITEMS * ZC_MAX_G + 2 * ZC_MAX_G) * 4;
 constexpr int kMaxItems = ZC_MAX_ITEMS;              // partial (m, l) pairs staged in the ring
 
 __device__ int g_zc_error = 0;
@@ -165,102 +166,134 @@ template <int BITS> __device__ __forceinline__ void chan_slot(int off, int* reg,
 }
 
 // Compressed-run part of one item, one warp: prologue done by the CTA, stages primed.
+// One iteration handles a PAIR of 16-token sub-tiles (one ring stage): two independent
+// chains of work per warp keep the pipes busy between dependent instructions.
 // Column n of the q' B-fragments is (head n >> 1, part n & 1) with q' = hi + lo in f16, so
 // that lane (g, t) receives both parts of head t for tokens g and g + 8 in its accumulator.
 template <int BITS>
-__device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* src0, char* my_ring,
-                                             uint64_t* my_bar, const uint32_t (&qb)[16], float qs,
-                                             float isc, float logK, int my_n, int warp, int lane,
-                                             float (&oacc)[8][4], float& m_out, float& l_out,
-                                             float& z_out, int* err) {
+__device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_base, char* my_ring,
+                                          uint64_t* my_bar, const uint32_t (&qb)[16], float qs,
+                                          float isc, float logK, int my_np, int warp, int lane,
+                                          float (&oacc)[8][4], float& m_out, float& l_out,
+                                          float& z_out, int* err) {
   constexpr int SB = ZC_SUB * (32 * BITS + 16);
+  constexpr int PB = 2 * SB;
+  constexpr int NST = kWarpRing / PB;
   const int g = lane >> 2, t = lane & 3;
   const bool odd_tok = BITS == 2 && (g & 1);
   const float logKs = logK - (odd_tok ? 2.f : 0.f);      // weights of odd tokens carry 1/4 at 2 bits
   // columns 4..7 of P^T repeat columns 0..3: their products land in accumulator columns no one reads
   const int srcA = 8 * t + (g & 3), srcB = srcA + 4;
   const int c0_src = (lane & ~3) | ((2 * t) & 3), c1_src = (lane & ~3) | ((2 * t + 1) & 3);
-  float m = -INFINITY, mo = 0.f, mthr = -INFINITY, l = 0.f, zacc = 0.f;
-  bool dead = false;
-  for (int i = 0; i < my_n; ++i) {
-    const int s = i % kStages, parity = (i / kStages) & 1;
-    if (!dead) {
+  // Logits are kept divided by isc (u = lg / isc): u costs one multiply less per token.
+  float mu = -INFINITY;          // running maximum of u
+  float mo_neg = 0.f;            // logKs - mu * isc
+  float uthr = -INFINITY;        // mu + kTau / isc
+  const float tau_u = kTau / isc;
+  float l = 0.f, zacc = 0.f;
+  // loop state, advanced by additions only
+  const int s_first = d.sub_lo + 2 * warp;
+  int rem = d.n_tok - (s_first - d.run_sub0) * ZC_SUB;   // tokens from this pair's first token to the run's end
+  const char* src_refill = class_base + (long long)(s_first + 2 * kWarps * NST) * SB;
+  int rem_refill = rem - 2 * ZC_SUB * kWarps * NST;
+  int refills = my_np - NST;
+  int stage = 0;
+  uint32_t parity = 0;
+  const char* ring_lane = my_ring + lane * 16;
+  for (int i = 0; i < my_np; ++i) {
+    uint64_t* bar = &my_bar[stage];
+    if (!mbar_try_wait(bar, parity)) {
       int spins = 0;
-      while (!mbar_try_wait(&my_bar[s], parity)) {
-        if (++spins > kWaitLimit) { dead = true; atomicExch(err, 1); break; }
+      while (!mbar_try_wait(bar, parity)) {
+        if (++spins > kWaitLimit) { atomicExch(err, 1); break; }
       }
     }
-    const char* st = my_ring + s * kStageBytes;
-    // ---- loads: K words of tokens g and g+8, V words, parameters (sK, zK, sV, zV) ----
-    uint32_t kw[2][BITS];   // 4-bit: 4 words per token, 2-bit: 2 words per token
-    uint32_t vw[2 * BITS];  // 4-bit: 8 words, 2-bit: 4 words
-    if (BITS == 4) {
-      const uint4 a = *reinterpret_cast<const uint4*>(st + lane * 16);
-      const uint4 b = *reinterpret_cast<const uint4*>(st + 512 + lane * 16);
-      kw[0][0] = a.x; kw[0][1] = a.y; kw[0][2] = a.z; kw[0][3] = a.w;
-      kw[1][0] = b.x; kw[1][1] = b.y; kw[1][2] = b.z; kw[1][3] = b.w;
-      const uint4 c = *reinterpret_cast<const uint4*>(st + 1024 + lane * 16);
-      const uint4 e = *reinterpret_cast<const uint4*>(st + 1536 + lane * 16);
-      vw[0] = c.x; vw[1] = c.y; vw[2] = c.z; vw[3] = c.w;
-      vw[4] = e.x; vw[5] = e.y; vw[6] = e.z; vw[7] = e.w;
-    } else {
-      const uint2 a = *reinterpret_cast<const uint2*>(st + lane * 8);
-      const uint2 b = *reinterpret_cast<const uint2*>(st + 256 + lane * 8);
-      kw[0][0] = a.x; kw[0][1] = a.y;
-      kw[1][0] = b.x; kw[1][1] = b.y;
-      const uint4 c = *reinterpret_cast<const uint4*>(st + 512 + lane * 16);
-      vw[0] = c.x; vw[1] = c.y; vw[2] = c.z; vw[3] = c.w;
+    char* st = my_ring + stage * PB;
+    if (rem <= ZC_SUB) {
+      // the run ends inside the first half: the second half was not copied; its tokens are
+      // masked below, its parameters must not hold stale bits
+      if (lane < ZC_SUB) *reinterpret_cast<float4*>(st + SB + 512 * BITS + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+      __syncwarp();
     }
-    const float4 pa = *reinterpret_cast<const float4*>(st + 512 * BITS + g * 16);
-    const float4 pb = *reinterpret_cast<const float4*>(st + 512 * BITS + (g + 8) * 16);
-
-    // ---- S^T = codes(16 tokens x 128) . q'^T : 8 k-steps, two accumulator chains ----
-    float dacc[4] = {0.f, 0.f, 0.f, 0.f}, dacc2[4] = {0.f, 0.f, 0.f, 0.f};
-    if (BITS == 4) {
+    // ---- loads: K words of tokens g and g+8, V words, parameters (sK, zK, sV, zV), both halves ----
+    uint32_t kw[2][2][BITS];   // [half][token slot][word]
+    uint32_t vw[2][2 * BITS];
+    float4 pp[2][2];
 #pragma unroll
-      for (int jw = 0; jw < 4; ++jw) {
-        const uint32_t w0 = kw[0][jw], w1 = kw[1][jw];
-        const uint32_t a0[4] = {w0 & 0x000F000Fu, w1 & 0x000F000Fu, w0 & 0x00F000F0u, w1 & 0x00F000F0u};
-        zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
-        const uint32_t x0 = w0 >> 8, x1 = w1 >> 8;
-        const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
-        zc_mma16816<__half>(dacc2, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
+    for (int h = 0; h < 2; ++h) {
+      const char* sh = ring_lane + stage * PB + h * SB;
+      if (BITS == 4) {
+        const uint4 a = *reinterpret_cast<const uint4*>(sh);
+        const uint4 b = *reinterpret_cast<const uint4*>(sh + 512);
+        kw[h][0][0] = a.x; kw[h][0][1] = a.y; kw[h][0][2] = a.z; kw[h][0][3] = a.w;
+        kw[h][1][0] = b.x; kw[h][1][1] = b.y; kw[h][1][2] = b.z; kw[h][1][3] = b.w;
+        const uint4 c = *reinterpret_cast<const uint4*>(sh + 1024);
+        const uint4 e = *reinterpret_cast<const uint4*>(sh + 1536);
+        vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
+        vw[h][4] = e.x; vw[h][5] = e.y; vw[h][6] = e.z; vw[h][7] = e.w;
+      } else {
+        const uint2 a = *reinterpret_cast<const uint2*>(st + h * SB + lane * 8);
+        const uint2 b = *reinterpret_cast<const uint2*>(st + h * SB + 256 + lane * 8);
+        kw[h][0][0] = a.x; kw[h][0][1] = a.y;
+        kw[h][1][0] = b.x; kw[h][1][1] = b.y;
+        const uint4 c = *reinterpret_cast<const uint4*>(sh + 512);
+        vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
       }
-    } else {
+      pp[h][0] = *reinterpret_cast<const float4*>(st + h * SB + 512 * BITS + g * 16);
+      pp[h][1] = *reinterpret_cast<const float4*>(st + h * SB + 512 * BITS + (g + 8) * 16);
+    }
+    // ---- S^T = codes(16 tokens x 128) . q'^T per half: 8 k-steps; the halves are independent chains ----
+    float u[2][2];   // [half][token slot] logits (base 2) of head t, divided by isc
 #pragma unroll
-      for (int jw = 0; jw < 2; ++jw) {
+    for (int h = 0; h < 2; ++h) {
+      float dacc[4];
+      if (BITS == 4) {
 #pragma unroll
-        for (int hb = 0; hb < 2; ++hb) {
-          const uint32_t w0 = kw[0][jw] >> (8 * hb), w1 = kw[1][jw] >> (8 * hb);
-          const int ks = 4 * jw + 2 * hb;
-          const uint32_t a0[4] = {w0 & 0x00030003u, w1 & 0x00030003u, w0 & 0x000C000Cu, w1 & 0x000C000Cu};
-          zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
-          const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
-          zc_mma16816<__half>(dacc2, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
+        for (int jw = 0; jw < 4; ++jw) {
+          const uint32_t w0 = kw[h][0][jw], w1 = kw[h][1][jw];
+          const uint32_t a0[4] = {w0 & 0x000F000Fu, w1 & 0x000F000Fu, w0 & 0x00F000F0u, w1 & 0x00F000F0u};
+          if (jw == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
+          else zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
+          const uint32_t x0 = w0 >> 8, x1 = w1 >> 8;
+          const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
+          zc_mma16816<__half>(dacc, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
+        }
+      } else {
+#pragma unroll
+        for (int jw = 0; jw < 2; ++jw) {
+#pragma unroll
+          for (int hb = 0; hb < 2; ++hb) {
+            const uint32_t w0 = kw[h][0][jw] >> (8 * hb), w1 = kw[h][1][jw] >> (8 * hb);
+            const int ks = 4 * jw + 2 * hb;
+            const uint32_t a0[4] = {w0 & 0x00030003u, w1 & 0x00030003u, w0 & 0x000C000Cu, w1 & 0x000C000Cu};
+            if (ks == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
+            else zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
+            const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
+            zc_mma16816<__half>(dacc, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
+          }
         }
       }
+      // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
+      u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
+      u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;
     }
-    // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
-    const float D0 = (dacc[0] + dacc2[0]) + (dacc[1] + dacc2[1]);
-    const float D1 = (dacc[2] + dacc2[2]) + (dacc[3] + dacc2[3]);
-    // ---- logits (base 2) of head t for tokens g and g+8 ----
-    float lg0 = fmaf(-pa.y, qs, D0) * (pa.x * isc);
-    float lg1 = fmaf(-pb.y, qs, D1) * (pb.x * isc);
-    const int tok0 = (d.sub_lo - d.run_sub0 + warp + i * kWarps) * ZC_SUB;   // first token of the sub-tile
-    if (tok0 + ZC_SUB > d.n_tok) {
-      if (tok0 + g >= d.n_tok) lg0 = -INFINITY;
-      if (tok0 + g + 8 >= d.n_tok) lg1 = -INFINITY;
+    if (rem < 2 * ZC_SUB) {
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        if (16 * h + g >= rem) u[h][0] = -INFINITY;
+        if (16 * h + g + 8 >= rem) u[h][1] = -INFINITY;
+      }
     }
-    const float mx = fmaxf(lg0, lg1);
-    if (__any_sync(kFull, mx > mthr)) {
+    const float mx = fmaxf(fmaxf(u[0][0], u[0][1]), fmaxf(u[1][0], u[1][1]));
+    if (__any_sync(kFull, mx > uthr)) {
       float mr = mx;
       mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 4));
       mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 8));
       mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 16));
-      const float mn = fmaxf(m, mr);
-      const float corr = mn == -INFINITY ? 1.f : zc_exp2(m - mn);
+      const float mn = fmaxf(mu, mr);
+      const float corr = mn == -INFINITY ? 1.f : zc_exp2((mu - mn) * isc);
       l *= corr; zacc *= corr;
-      m = mn; mo = mn - logKs; mthr = mn + kTau;
+      mu = mn; mo_neg = fmaf(-mn, isc, logKs); uthr = mn + tau_u;
       const float c0 = __shfl_sync(kFull, corr, c0_src), c1 = __shfl_sync(kFull, corr, c1_src);
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -268,47 +301,62 @@ __device__ __forceinline__ void run_subtiles(const ItemDesc& d, const char* src0
       }
     }
     // p' = p * 2^logKs; weights w = p' * s^V go to f16, the same rounded values feed the z sum
-    const float p0 = zc_exp2(lg0 - mo), p1 = zc_exp2(lg1 - mo);
-    l += p0 + p1;
-    const __half2 h2 = __floats2half2_rn(p0 * pa.z, p1 * pb.z);   // (token g, token g+8)
-    const float2 back = __half22float2(h2);
-    zacc = fmaf(back.x, pa.w, zacc);
-    zacc = fmaf(back.y, pb.w, zacc);
-    const uint32_t X = *reinterpret_cast<const uint32_t*>(&h2);
-    // B fragment of P^T, column n = g = head g & 3: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
-    const uint32_t pb0 = __shfl_sync(kFull, X, srcA), pb1 = __shfl_sync(kFull, X, srcB);
-    // ---- O^T += V^T(128 channels x 16 tokens) . P^T : 8 M-tiles ----
-    if (BITS == 4) {
+    uint32_t pb[2][2];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const uint32_t w = vw[j], x = w >> 8;
-        const uint32_t a[4] = {w & 0x000F000Fu, w & 0x00F000F0u, x & 0x000F000Fu, x & 0x00F000F0u};
-        zc_mma16816<__half>(oacc[j], a, pb0, pb1);
-      }
-    } else {
+    for (int h = 0; h < 2; ++h) {
+      const float p0 = zc_exp2(fmaf(u[h][0], isc, mo_neg)), p1 = zc_exp2(fmaf(u[h][1], isc, mo_neg));
+      l += p0 + p1;
+      const __half2 h2 = __floats2half2_rn(p0 * pp[h][0].z, p1 * pp[h][1].z);   // (token g, token g+8)
+      const float2 back = __half22float2(h2);
+      zacc = fmaf(back.x, pp[h][0].w, zacc);
+      zacc = fmaf(back.y, pp[h][1].w, zacc);
+      const uint32_t X = *reinterpret_cast<const uint32_t*>(&h2);
+      // B fragment of P^T, column n = g = head g & 3: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
+      pb[h][0] = __shfl_sync(kFull, X, srcA);
+      pb[h][1] = __shfl_sync(kFull, X, srcB);
+    }
+    // ---- O^T += V^T(128 channels x 16 tokens) . P^T per half: 8 M-tiles ----
 #pragma unroll
-      for (int mw = 0; mw < 4; ++mw) {
+    for (int h = 0; h < 2; ++h) {
+      if (BITS == 4) {
 #pragma unroll
-        for (int e2 = 0; e2 < 2; ++e2) {
-          const uint32_t w = vw[mw] >> (8 * e2);
-          const uint32_t a[4] = {w & 0x00030003u, w & 0x00300030u, w & 0x000C000Cu, w & 0x00C000C0u};
-          zc_mma16816<__half>(oacc[2 * mw + e2], a, pb0, pb1);
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t w = vw[h][j], x = w >> 8;
+          const uint32_t a[4] = {w & 0x000F000Fu, w & 0x00F000F0u, x & 0x000F000Fu, x & 0x00F000F0u};
+          zc_mma16816<__half>(oacc[j], a, pb[h][0], pb[h][1]);
+        }
+      } else {
+#pragma unroll
+        for (int mw = 0; mw < 4; ++mw) {
+#pragma unroll
+          for (int e2 = 0; e2 < 2; ++e2) {
+            const uint32_t w = vw[h][mw] >> (8 * e2);
+            const uint32_t a[4] = {w & 0x00030003u, w & 0x00300030u, w & 0x000C000Cu, w & 0x00C000C0u};
+            zc_mma16816<__half>(oacc[2 * mw + e2], a, pb[h][0], pb[h][1]);
+          }
         }
       }
     }
     // ---- refill this stage ----
     __syncwarp();
-    if (lane == 0 && i + kStages < my_n) {
-      mbar_expect_tx(&my_bar[s], SB);
-      bulk_copy_g2s(my_ring + s * kStageBytes, src0 + (long long)(i + kStages) * kWarps * SB, SB,
-                    &my_bar[s]);
+    if (refills > 0) {
+      if (lane == 0) {
+        const int bytes = rem_refill > ZC_SUB ? PB : SB;
+        mbar_expect_tx(bar, bytes);
+        bulk_copy_g2s(st, src_refill, bytes, bar);
+      }
+      src_refill += kWarps * PB;
+      rem_refill -= 2 * ZC_SUB * kWarps;
     }
+    --refills;
+    rem -= 2 * ZC_SUB * kWarps;
+    if (++stage == NST) { stage = 0; parity ^= 1u; }
   }
   // sums back to plain units: l' = sum p 2^logKs; zacc' = sum w z with w short by the odd-token 1/4
   const float inv_sig = odd_tok ? 4.f : 1.f;
   l_out = l * zc_exp2(-logKs);
   z_out = zacc * inv_sig;
-  m_out = m;
+  m_out = mu == -INFINITY ? -INFINITY : mu * isc;
 }
 
 // One compressed item, whole CTA.  On return every warp has put its (m, l, z-sum) and its
@@ -320,26 +368,32 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
                                                 float* chan_factor, float* rowscale, int* err) {
   constexpr int SB = ZC_SUB * (32 * BITS + 16);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  constexpr int PB = 2 * SB;
+  constexpr int NST = kWarpRing / PB;
   char* my_ring = smem + warp * kWarpRing;
-  uint64_t* my_bar = reinterpret_cast<uint64_t*>(smem + kOffBars) + warp * kStages;
+  uint64_t* my_bar = reinterpret_cast<uint64_t*>(smem + kOffBars) + warp * kMaxStages;
   uint4* qfrag = reinterpret_cast<uint4*>(smem + kOffQfrag);
   unsigned* s_red = reinterpret_cast<unsigned*>(smem + kOffRed);
   float* wm = reinterpret_cast<float*>(smem + kOffWm);
   float* wl = reinterpret_cast<float*>(smem + kOffWl);
   float* wz = reinterpret_cast<float*>(smem + kOffWz);
-  const int n_sub = d.sub_hi - d.sub_lo;
-  const int my_n = n_sub > warp ? (n_sub - warp + kWarps - 1) / kWarps : 0;
-  const char* src0 = class_base + (long long)(d.sub_lo + warp) * SB;
+  const int n_pairs = (d.sub_hi - d.sub_lo + 1) >> 1;
+  const int my_np = n_pairs > warp ? (n_pairs - warp + kWarps - 1) / kWarps : 0;
   // ---- start the copies first: their latency covers the q' set-up ----
   if (lane == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(&my_bar[s], 1);
+    for (int s = 0; s < NST; ++s) mbar_init(&my_bar[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
-    for (int s = 0; s < kStages && s < my_n; ++s) {
-      mbar_expect_tx(&my_bar[s], SB);
-      bulk_copy_g2s(my_ring + s * kStageBytes, src0 + (long long)s * kWarps * SB, SB, &my_bar[s]);
+    for (int s = 0; s < NST && s < my_np; ++s) {
+      const int sn = d.sub_lo + 2 * (warp + s * kWarps);
+      const int bytes = sn + 1 < d.sub_hi ? PB : SB;
+      mbar_expect_tx(&my_bar[s], bytes);
+      bulk_copy_g2s(my_ring + s * PB, class_base + (long long)sn * SB, bytes, &my_bar[s]);
     }
   }
+  // everything this CTA needs from global memory besides the codes is requested now
+  const float cV = fac[ZC_D + tid];
+  const float smax = fac[2 * ZC_D];
   // ---- q' = q * c^K * log2(e)/sqrt(d); thread = channel ----
   const float scale = kLog2e * rsqrtf((float)ZC_D);
   const float cK = fac[tid];
@@ -395,7 +449,6 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
   // accumulator * 2^24 / CTA scale = q' . code
   const float isc = 16777216.f * (scaled ? __uint_as_float((ex_q - 13u) << 23) : 1.f);
   // weights are scaled by 2^logK = 2^kPExp / 2^ceil(log2 smax) so that w <= 2^(kPExp + kTau)
-  const float smax = fac[2 * ZC_D];
   const int es = (int)((__float_as_uint(smax) >> 23) & 255u) - 127;
   const float logK = (float)(kPExp - es - 1);
 
@@ -405,7 +458,7 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
 #pragma unroll
     for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
   float m, l, z;
-  run_subtiles<BITS>(d, src0, my_ring, my_bar, qb, qs, isc, logK, my_n, warp, lane, oacc, m, l, z, err);
+  run_pairs<BITS>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
 #pragma unroll
   for (int o = 4; o < 32; o <<= 1) {
     l += __shfl_xor_sync(kFull, l, o);
@@ -426,7 +479,7 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
     }
   }
   // o[ch] = c^V[ch] 2^-logK (acc 2^24 / sigma(row) - z sum); rows g+8 of a tile carry sigma = 16
-  *chan_factor = fac[ZC_D + tid] * zc_exp2(-logK);
+  *chan_factor = cV * zc_exp2(-logK);
   *rowscale = (tid & 8) ? 1048576.f : 16777216.f;
 }
 
@@ -564,16 +617,16 @@ __device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, con
 }
 
 template <typename T>
-__global__ void __launch_bounds__(128, 4) k_decode(char* cache, ZcLayout lay, ZcDecodePlan plan,
-                                                   const T* __restrict__ q, T* __restrict__ out,
-                                                   float* part, float* tail_logits, int collect) {
+__global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, ZcLayout lay,
+                                                                  ZcDecodePlan plan,
+                                                                  const T* __restrict__ q, float* part,
+                                                                  float* tail_logits) {
   extern __shared__ __align__(128) char smem[];
   float* wm = reinterpret_cast<float*>(smem + kOffWm);
   float* wl = reinterpret_cast<float*>(smem + kOffWl);
   float* wz = reinterpret_cast<float*>(smem + kOffWz);
   float* s_cw = reinterpret_cast<float*>(smem + kOffCw);
   float* s_head = reinterpret_cast<float*>(smem + kOffHead);
-  int* s_flag = reinterpret_cast<int*>(smem + kOffFlag);
   pdl_launch_dependents();
   const int unit = blockIdx.y, it = blockIdx.x;
   const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
@@ -636,18 +689,20 @@ __global__ void __launch_bounds__(128, 4) k_decode(char* cache, ZcLayout lay, Zc
     if (tid == 0) { dst[0] = s_head[h * 4]; dst[1] = s_head[h * 4 + 1]; }
     dst[4 + tid] = o;
   }
-  // ---- the CTA that arrives last at the unit's counter combines all partials ----
-  __threadfence();
-  __syncthreads();
-  unsigned* counter = reinterpret_cast<unsigned*>(ub + lay.off_sync);
-  if (tid == 0) {
-    const unsigned total = gridDim.x * gridDim.z;
-    const unsigned prev = atomicAdd(counter, 1u);
-    *s_flag = prev == total - 1u;
-  }
-  __syncthreads();
-  if (!*s_flag) return;
-  __threadfence();
+}
+
+// Merge of the split-K partials: one CTA per unit, warp w owns heads w, w + 4.
+template <typename T>
+__global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout lay, ZcDecodePlan plan,
+                                                        T* __restrict__ out, const float* part,
+                                                        const float* tail_logits, int collect) {
+  extern __shared__ __align__(128) char smem[];
+  pdl_launch_dependents();
+  const int unit = blockIdx.x;
+  const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  char* ub = zc_unit_base(cache, lay, unit);
+  pdl_wait();   // the partials come from the kernel just before this one
   const int items = plan.items;
   const float* mine = part + (long long)unit * items * G * ZC_PART_STRIDE;
   float* s_m = reinterpret_cast<float*>(smem);          // [items * G] maxima, then weights
@@ -721,7 +776,6 @@ __global__ void __launch_bounds__(128, 4) k_decode(char* cache, ZcLayout lay, Zc
       colsum[tid] += a;
     }
   }
-  if (tid == 0) *counter = 0u;   // ready for the next call
 }
 
 }  // namespace
@@ -774,22 +828,31 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
   const char* q_lo = (const char*)q;
   const bool overlap = !(g_last_out_lo && q_lo < g_last_out_hi && q_lo + io_bytes > g_last_out_lo);
+  const dim3 cgrid(c->lay.units);
   cudaError_t e;
   if (c->cfg.dtype == ZC_F16) {
-    e = cudaFuncSetAttribute(k_decode<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(k_decode<__half>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay, plan,
-                   (const __half*)q, (__half*)out, part, tail_logits, collect);
-  } else {
-    e = cudaFuncSetAttribute(k_decode<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(k_decode_items<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kDecodeSmem);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(k_decode<__nv_bfloat16>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay,
-                   plan, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, part, tail_logits, collect);
+    e = launch_pdl(k_decode_items<__half>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay,
+                   plan, (const __half*)q, part, tail_logits);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(k_decode_combine<__half>, cgrid, dim3(128), kCombineSmem, st, true, c->base, c->lay,
+                   plan, (__half*)out, (const float*)part, (const float*)tail_logits, collect);
+  } else {
+    e = cudaFuncSetAttribute(k_decode_items<__nv_bfloat16>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(k_decode_items<__nv_bfloat16>, grid, dim3(128), kDecodeSmem, st, overlap, c->base,
+                   c->lay, plan, (const __nv_bfloat16*)q, part, tail_logits);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(k_decode_combine<__nv_bfloat16>, cgrid, dim3(128), kCombineSmem, st, true, c->base,
+                   c->lay, plan, (__nv_bfloat16*)out, (const float*)part, (const float*)tail_logits,
+                   collect);
   }
   g_last_out_lo = (const char*)out;
   g_last_out_hi = (const char*)out + io_bytes;
-  c->launches += 1;
+  c->launches += 2;
   return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 

@@ -153,7 +153,8 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   for (int k = 0; k < 2; ++k) {
     const int s = std::max(1, std::min(std::min(want[k], std::min(ZC_MAX_SPLIT_HOST, cap)),
                                        std::max(1, subs[k])));
-    p.spi0[k] = zc_ceil_div(std::max(1, subs[k]), s);
+    // an even number of sub-tiles per item: the kernel consumes them in pairs
+    p.spi0[k] = (zc_ceil_div(std::max(1, subs[k]), s) + 1) & ~1;
     p.split0[k] = zc_ceil_div(std::max(1, subs[k]), p.spi0[k]);
   }
   p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + p.tail_items;

@@ -17,7 +17,7 @@
 #ifndef ZC_ITEM_SUBS
 #define ZC_ITEM_SUBS 64           // 16-token sub-tiles one item of segment 0 aims at
 #endif
-#define ZC_DECODE_CTAS_PER_SM 4    // CTAs the decode kernel keeps resident per SM
+#define ZC_DECODE_CTAS_PER_SM 3    // CTAs the decode kernel keeps resident per SM
 
 // Device-side description of the cache buffer.  One "unit" = (batch, KV head).
 // Per unit, at byte offsets from base + unit * unit_stride:
