@@ -30,12 +30,22 @@ namespace {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxStages = 5;              // ring depth per warp: 3 pairs at 4 bits, 5 at 2 bits
 constexpr int kWarps = 4;
-constexpr int kWarpRing = 13824;           // 3 x 4608 (4-bit pair) >= 5 x 2560 (2-bit pair)
+#ifndef ZC_WARP_RING
+#define ZC_WARP_RING 13824
+#endif
+constexpr int kWarpRing = ZC_WARP_RING;    // 13824 = 3 x 4608 (4-bit pair) >= 5 x 2560 (2-bit pair)
 constexpr int kRingBytes = kWarps * kWarpRing;               // 55296
 constexpr int kCtasPerSm = ZC_DECODE_CTAS_PER_SM;
 constexpr int kWaitLimit = 1 << 22;
-constexpr int kPExp = 12;      // softmax weights go to f16 as p * s^V * 2^kPExp / 2^ceil(log2 smax)
-constexpr float kTau = 3.5f;   // the running maximum is refreshed only when a logit exceeds it by this
+#ifndef ZC_KPEXP
+#define ZC_KPEXP 12
+#define ZC_TAU 3.5f
+#endif
+#ifndef ZC_QK_CHAINS
+#define ZC_QK_CHAINS 1
+#endif
+constexpr int kPExp = ZC_KPEXP;      // softmax weights go to f16 as p * s^V * 2^kPExp / 2^ceil(log2 smax)
+constexpr float kTau = ZC_TAU;   // the running maximum is refreshed only when a logit exceeds it by this
 constexpr unsigned kFull = 0xffffffffu;
 
 // shared-memory map of k_decode
@@ -246,7 +256,7 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
     float u[2][2];   // [half][token slot] logits (base 2) of head t, divided by isc
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      float dacc[4];
+      float dacc[4], dacc2[4] = {0.f, 0.f, 0.f, 0.f};
       if (BITS == 4) {
 #pragma unroll
         for (int jw = 0; jw < 4; ++jw) {
@@ -256,7 +266,8 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
           else zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
           const uint32_t x0 = w0 >> 8, x1 = w1 >> 8;
           const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
-          zc_mma16816<__half>(dacc, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
+          if (ZC_QK_CHAINS == 2 && jw == 0) zc_mma16816_z(dacc2, a1, qb[2], qb[3]);
+          else zc_mma16816<__half>(ZC_QK_CHAINS == 2 ? dacc2 : dacc, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
         }
       } else {
 #pragma unroll
@@ -269,11 +280,16 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
             if (ks == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
             else zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
             const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
-            zc_mma16816<__half>(dacc, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
+            if (ZC_QK_CHAINS == 2 && ks == 0) zc_mma16816_z(dacc2, a1, qb[2], qb[3]);
+            else zc_mma16816<__half>(ZC_QK_CHAINS == 2 ? dacc2 : dacc, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
           }
         }
       }
       // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
+      if (ZC_QK_CHAINS == 2) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dacc[e] += dacc2[e];
+      }
       u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
       u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;
     }

@@ -15,9 +15,11 @@
 #define ZC_MAX_SPLIT_HOST 32      // most items one class of segment 0 is split into
 #define ZC_MAX_ITEMS 128          // most items of one unit in one decode call
 #ifndef ZC_ITEM_SUBS
-#define ZC_ITEM_SUBS 64           // 16-token sub-tiles one item of segment 0 aims at
+#define ZC_ITEM_SUBS 128          // 16-token sub-tiles one item of segment 0 aims at
 #endif
-#define ZC_DECODE_CTAS_PER_SM 3    // CTAs the decode kernel keeps resident per SM
+#ifndef ZC_DECODE_CTAS_PER_SM
+#define ZC_DECODE_CTAS_PER_SM 3
+#endif    // CTAs the decode kernel keeps resident per SM
 
 // Device-side description of the cache buffer.  One "unit" = (batch, KV head).
 // Per unit, at byte offsets from base + unit * unit_stride:
