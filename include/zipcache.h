@@ -42,7 +42,9 @@ enum {
   ZC_ECAPACITY = -2, /* more tokens than the cache or workspace was sized for */
   ZC_ESTATE = -3,    /* call out of order (e.g. decode before prefill) */
   ZC_EALIGN = -4,    /* pointer not 16-byte aligned */
-  ZC_ECUDA = -5      /* a CUDA runtime call or launch failed */
+  ZC_ECUDA = -5,     /* a CUDA runtime call or launch failed */
+  ZC_ESCRATCH = -6   /* zc_decode_attention_noalloc: the call needs more scratch than the
+                        library's built-in buffer holds */
 };
 
 #define ZC_MAX_WINDOW 128
@@ -129,6 +131,32 @@ int zc_tail_tokens(const zc_cache* c);
  * cf b x h_kv x d floats (channel factors).  tensor 0 = K, 1 = V.  Any out may be NULL. */
 int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t* idx,
                       uint8_t* codes, float* sz, float* cf, zc_stream_t stream);
+
+/* Size of the scratch buffer built into the library for zc_decode_attention_noalloc. */
+#define ZC_NOALLOC_SCRATCH_BYTES (4u << 20)
+
+/* The paper has no counterpart for this entry point; it exists for integration reasons.
+ * Same operation, arguments and state changes as zc_decode_attention, for callers that have
+ * no way to hand the library a workspace: code that runs where device allocation is not
+ * allowed or not possible -- a plug-in inside a serving process whose memory pool owns the
+ * whole device and forbids further cudaMalloc calls, a latency-critical loop that must not
+ * enter the allocator, a caller that has already given away its memory budget.  The split-K
+ * partial results and the tail logits go to a fixed buffer of ZC_NOALLOC_SCRATCH_BYTES that is
+ * part of the library image (every GPU that loads the library carries it until the process
+ * ends); the caller still owns q [device] and out [device].  The call allocates and frees
+ * nothing.
+ *   - ZC_ESCRATCH, with nothing enqueued, when the cache's shape needs more than the
+ *     built-in buffer (about batch * n_q_heads * items * 528 bytes, items = split-K pieces
+ *     per KV head; use zc_decode_attention with a caller workspace then).
+ *   - The first call on each device looks up the buffer's device address (a synchronous
+ *     runtime query): make that first call outside any stream capture.
+ *   - All calls share the one buffer, whatever cache they work on.  Calls that follow one
+ *     another in ONE stream are ordered by the library; calls in different streams, or from
+ *     several host threads, that may run at the same time on the GPU overwrite each other's
+ *     partial results.  Nothing in the buffer has to survive between calls and nothing in it
+ *     has to be cleared: each call rewrites every word it later reads. */
+int zc_decode_attention_noalloc(zc_cache* c, const void* q, void* out, int is_probe_step,
+                                zc_stream_t stream);
 
 /* Algorithmic bytes one zc_decode_attention call must read in the cache's current
  * state (packed codes + per-token parameters + tail + channel factors + q and out). */

@@ -51,6 +51,7 @@ _SIGS = {
     "zc_append": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "zc_decode_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                       C.c_size_t, C.c_void_p]),
+    "zc_decode_attention_noalloc": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]),
     "zc_export_scores": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p]),
     "zc_segment_tokens": (C.c_int, [C.c_void_p, C.c_int, C.c_int]),
     "zc_num_segments": (C.c_int, [C.c_void_p]),
@@ -166,6 +167,13 @@ def zc_decode_attention(handle, q, out, is_probe_step: bool, workspace, stream=N
     _check(lib().zc_decode_attention(handle, _ptr(q), _ptr(out), int(bool(is_probe_step)),
                                      _ptr(workspace), ws_bytes, _stream(stream)),
            "zc_decode_attention")
+
+
+def zc_decode_attention_noalloc(handle, q, out, is_probe_step: bool, stream=None) -> None:
+    """zc_decode_attention with the library's built-in scratch buffer instead of a caller
+    workspace (for callers that cannot allocate device memory)."""
+    _check(lib().zc_decode_attention_noalloc(handle, _ptr(q), _ptr(out), int(bool(is_probe_step)),
+                                             _stream(stream)), "zc_decode_attention_noalloc")
 
 
 def zc_export_scores(handle, p_tilde, stream=None) -> None:

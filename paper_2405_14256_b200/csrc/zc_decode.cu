@@ -872,6 +872,28 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 
+// Scratch of zc_decode_attention_noalloc.  In host code the name below is only a handle for the
+// runtime, not a device address: kernels must be given the pointer cudaGetSymbolAddress returns
+// for the device that is current.
+static __device__ __align__(256) unsigned char g_zc_noalloc_scratch[ZC_NOALLOC_SCRATCH_BYTES];
+
+int zc_static_scratch(void** ptr) {
+  constexpr int kMaxDev = 64;
+  static void* addr[kMaxDev] = {nullptr};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return (int)e;
+  if (dev < 0 || dev >= kMaxDev) return (int)cudaErrorInvalidDevice;
+  if (!addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_zc_noalloc_scratch);
+    if (e != cudaSuccess) return (int)e;
+    addr[dev] = p;
+  }
+  *ptr = addr[dev];
+  return (int)cudaSuccess;
+}
+
 int zc_device_error_code(int* out) {
   return (int)cudaMemcpyFromSymbol(out, g_zc_error, sizeof(int));
 }

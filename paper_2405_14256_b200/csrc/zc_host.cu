@@ -93,7 +93,9 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
 }
 
 const char* kMsgs[] = {"ok", "invalid argument", "capacity exceeded", "call out of order",
-                       "pointer not 16-byte aligned", "CUDA error"};
+                       "pointer not 16-byte aligned", "CUDA error",
+                       "the call needs more scratch than the built-in buffer of "
+                       "zc_decode_attention_noalloc holds: pass a workspace to zc_decode_attention"};
 thread_local char g_cuda_msg[256] = "CUDA error";
 
 int cuda_fail(cudaError_t e) {
@@ -165,7 +167,7 @@ extern "C" {
 
 const char* zc_strerror(int status) {
   if (status == ZC_ECUDA) return g_cuda_msg;
-  if (status > 0 || status < -5) return "unknown status";
+  if (status > 0 || status < -6) return "unknown status";
   return kMsgs[-status];
 }
 
@@ -349,6 +351,22 @@ int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step
     }
   }
   return ZC_OK;
+}
+
+int zc_decode_attention_noalloc(zc_cache* c, const void* q, void* out, int is_probe_step,
+                                zc_stream_t stream) {
+  if (!c || !q || !out) return ZC_EINVAL;
+  if (c->l0 < 0) return ZC_ESTATE;
+  // what this call will really write: partials [unit][item][G][ZC_PART_STRIDE] + tail logits
+  const ZcDecodePlan plan = zc_make_plan(c);
+  const size_t need = ((size_t)c->lay.units * plan.items * c->lay.G * ZC_PART_STRIDE +
+                       (size_t)c->lay.units * c->lay.G * ZC_MAX_WINDOW) * 4;
+  if (need > (size_t)ZC_NOALLOC_SCRATCH_BYTES) return ZC_ESCRATCH;
+  void* scratch = nullptr;
+  ZC_CUDA(zc_static_scratch(&scratch));   // first call per device: a synchronous address query
+  // The ordinary entry point sizes its check for the worst case of the cache's whole life;
+  // the bytes above are the ones it touches in the cache's present state.
+  return zc_decode_attention(c, q, out, is_probe_step, scratch, c->ws_bytes, stream);
 }
 
 int zc_num_segments(const zc_cache* c) { return c ? c->n_seg : ZC_EINVAL; }

@@ -114,6 +114,8 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
                      int collect, float* ws, cudaStream_t st);
 #define ZC_TAIL_ITEM_TOKENS 64
 int zc_device_error_code(int* out);
+// Device address of the built-in scratch buffer on the current device (looked up once per device).
+int zc_static_scratch(void** ptr);
 int zc_launch_export_scores(zc_cache* c, float* out, int n, cudaStream_t st);
 int zc_launch_export_segment(zc_cache* c, const ZcSeg& seg, int tensor, int subset,
                              int32_t* idx, uint8_t* codes, float* sz, float* cf,

@@ -1,0 +1,67 @@
+"""zc_decode_attention_noalloc against zc_decode_attention.
+
+Some callers cannot give the library a workspace because they are not allowed to allocate
+device memory at that point (a plug-in inside a server whose pool owns the device, a loop
+that must stay out of the allocator).  For them the library carries a fixed scratch buffer
+and one extra entry point that uses it.  Here two caches are filled with the same seeded
+input; one is driven through the ordinary call with a caller workspace, the other through the
+no-allocation call, for two decode steps in a row.  The second step re-uses the shared
+buffer with the first step's contents still in it, which is the case a stale-scratch bug
+would show up in.  This file sorts last on purpose: it runs after every other GPU test and
+must also pass alone in a fresh process.
+"""
+import pytest
+import torch
+
+import zc_testlib as tl
+from workloads import make_prefill, make_decode_step
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("kw", [
+    dict(context=300, batch=2, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0),
+    dict(context=512, n_q_heads=4, n_kv_heads=4),
+])
+def test_noalloc_entry_matches_workspace_entry_two_calls_in_a_row(kw):
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(**kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w).tolist()
+    ref_cache, new_cache = tl.make_cache(w), tl.make_cache(w)
+    ref_cache.mem.zero_()
+    new_cache.mem.zero_()
+    ref_cache.prefill_compress(Q, K, V, P)
+    new_cache.prefill_compress(Q, K, V, P)
+    for step in range(2):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        ref_cache.append(k, v)
+        new_cache.append(k, v)
+        want = ref_cache.decode_attention(q, step == 1)
+        got = torch.empty_like(q)
+        zc.zc_decode_attention_noalloc(new_cache.handle, q, got, step == 1)
+        torch.cuda.synchronize()
+        err = float((got.double() - want.double()).abs().max())
+        assert err <= 2e-3, (step, err)   # the tolerance of the decode parity tests
+        assert torch.equal(got, want)      # same kernels, same order of operations
+    assert zc.zc_device_status() == 0
+    # the window statistics collected on the probe step went through the built-in buffer too
+    assert torch.equal(ref_cache.mem, new_cache.mem)
+
+
+def test_noalloc_entry_rejects_shapes_beyond_its_buffer():
+    import paper_2405_14256_b200 as zc
+    # 64 x 32 heads: the split-K partials of one call alone exceed the 4 MiB buffer
+    w = tl.small_workload(context=64, batch=64, n_q_heads=32, n_kv_heads=32, window=8)
+    big = tl.make_cache(w, max_new=64)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    big.prefill_compress(Q, K, V, tl.probes_for(w).tolist())
+    q, k, v = make_decode_step(w, 0, 0, tl.DEV)
+    big.append(k, v)
+    out = torch.empty_like(q)
+    with pytest.raises(zc.ZipCacheError, match="built-in buffer"):
+        zc.zc_decode_attention_noalloc(big.handle, q, out, False)
+    # the ordinary entry point still serves the same cache
+    big.decode_attention(q, False, out=out)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out.float()).all()
