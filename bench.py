@@ -161,6 +161,25 @@ def oracle_sample(w, n_units: int, n_steps: int, layer: int = 0):
             f"{n_steps} decode steps")
 
 
+def rank_layers(rank: int, layers_per_rank: int):
+    """Layers (independent units of work) owned by one rank: the path shards over units with
+    no exchange step, so ranks never share a layer."""
+    return [rank * layers_per_rank + i for i in range(layers_per_rank)]
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of per-rank timings (the slowest rank sets the job's time)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def aggregate_throughput(bytes_per_rank: int, world: int, ms: float) -> float:
+    """Whole-job GB/s: every rank moves `bytes_per_rank` in the slowest rank's time."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 def run_reference(args):
     """The oracle as the reference arm: same metric, same workload, bounded sample."""
     from workloads import get_config
@@ -225,7 +244,7 @@ def main():
     R = args.layers
     n_dec = args.decode_steps or w.decode_steps
     # rank r owns layers r*R .. r*R+R-1 (independent units: no collective on the data path)
-    layer_ids = [rank * R + i for i in range(R)]
+    layer_ids = rank_layers(rank, R)
     probes = [zc.zc_default_probes(w.context, w.rho_recent, w.rho_random, w.seed(ly))
               for ly in layer_ids]
     inputs = [make_prefill(w, ly, dev) for ly in layer_ids]
@@ -301,10 +320,7 @@ def main():
     t_pre = sum(ev[0].elapsed_time(ev[1]) for ev in evs) / args.steps      # ms per step
     t_dec = sum(ev[1].elapsed_time(ev[2]) for ev in evs) / args.steps
     t_step = evs[0][0].elapsed_time(evs[-1][2]) / args.steps
-    times = torch.tensor([t_step, t_pre, t_dec], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    t_step, t_pre, t_dec = (float(x) for x in times.cpu())
+    t_step, t_pre, t_dec = max_over_ranks([t_step, t_pre, t_dec], dist, dev)
 
     # ---- end to end through the C ABI with host buffers ----
     e2e = None
@@ -340,12 +356,8 @@ def main():
                     d2h += outs[i].numel() * outs[i].element_size()
             e2_.record(stream)
         sync_all()
-        te = torch.tensor([e1.elapsed_time(e2_), e0.elapsed_time(e1)], dtype=torch.float64,
-                          device=dev)
-        if dist is not None:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        te_dec, te_pre = (float(x) for x in te.cpu())
-        e2e = {"value": world * eb / (te_dec * 1e-3) / 1e9, "unit": UNIT,
+        te_dec, te_pre = max_over_ranks([e1.elapsed_time(e2_), e0.elapsed_time(e1)], dist, dev)
+        e2e = {"value": aggregate_throughput(eb, world, te_dec), "unit": UNIT,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                "prefill_tokens_per_s": world * R * w.batch * w.context / (te_pre * 1e-3),
                "note": "eager C-ABI calls, pinned host buffers, copies inside the timed region"}
@@ -355,7 +367,7 @@ def main():
             dist.destroy_process_group()
         return
     peak, peak_kind = _peaks()
-    value = world * dec_bytes / (t_dec * 1e-3) / 1e9
+    value = aggregate_throughput(dec_bytes, world, t_dec)
     per_call_us = t_dec * 1e3 / n_decode_calls
     achieved = dec_bytes / (t_dec * 1e-3) / 1e9          # per GPU
     traffic = PROFILED_DRAM_BYTES_PER_DECODE_CALL.get(w.cfg_id)
