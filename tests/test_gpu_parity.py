@@ -184,3 +184,29 @@ def test_run_to_run_determinism():
     # codes, parameters and index lists are bitwise identical run to run
     a = cache.segment(0, 1, 0)
     assert torch.equal(outs[0][1][: 1024], outs[1][1][: 1024])
+
+
+@pytest.mark.parametrize("cfg_id,units,steps", [
+    (2, [(0, 0), (5, 3), (7, 7)], 3),
+    (3, [(0, 0), (11, 5)], 2),
+    (4, [(0, 0), (17, 13), (31, 31)], 3),
+    (5, [(2, 6)], 2),
+])
+def test_full_size_configs_on_sampled_units(cfg_id, units, steps):
+    """The benchmark's shapes at full size (one layer), end to end through the C ABI in the
+    launch configuration the benchmark times; the oracle follows a seeded sample of units:
+    normalised scores, salient sets, packed codes, parameters and decode outputs."""
+    w = get_config(cfg_id)
+    worst, cache, oc = tl.run_decode_parity(w, steps, units=units, staged=False)
+    assert worst <= 2e-3
+    p_gpu = cache.scores(w.context).cpu().numpy()
+    idx_hi = cache.segment(0, 0, 0)[0].cpu().numpy()
+    swaps = 0
+    for (bi, kv) in units:
+        s0 = oc.units[(bi, kv)].segments[0]
+        rel = np.abs(p_gpu[bi, kv] - s0.p_tilde) / np.maximum(np.abs(s0.p_tilde), 1e-30)
+        assert rel.max() <= 1e-4, rel.max()
+        swaps += tl.salient_sets_match(p_gpu[bi, kv], s0.p_tilde, idx_hi[bi, kv], s0.hi.idx, s0.hi.n)
+    print(f"config {cfg_id}: near-tie swaps {swaps}, worst decode error {worst:.2e}")
+    if swaps == 0:
+        assert tl.compare_segment(cache, oc, 0, units=units) == 0
