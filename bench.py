@@ -218,6 +218,9 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--decode-steps", type=int, default=0,
                     help="profiling only: fewer decode steps than the workload's own")
+    ap.add_argument("--append", default="deferred", choices=["deferred", "kernel"],
+                    help="deferred: zc_append hands the new row to the next zc_decode_attention "
+                         "(ZC_FLAG_DEFER_APPEND); kernel: zc_append copies with its own launch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -254,7 +257,8 @@ def main():
     workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)   # shared by all layers
     caches = [zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context, n_dec,
                           w.saliency_ratio, w.bits_hi, w.bits_lo, w.window, device=dev,
-                          workspace=workspace) for _ in range(R)]
+                          workspace=workspace, defer_append=args.append == "deferred")
+              for _ in range(R)]
     flags = [decode_probe_flags(w, ly, n_dec) for ly in layer_ids]
     # decode inputs: 4 distinct seeded sets per step, cycled over layers (fresh N(0,1) each)
     dec_in = [[make_decode_step(w, v, s, dev) for v in range(4)] for s in range(n_dec)]
@@ -380,7 +384,10 @@ def main():
                          f"({R * dec_bytes / n_decode_calls / 1e6:.0f} MB) cycled every decode step",
                    "batch": w.batch, "context": w.context, "n_q_heads": w.n_q_heads,
                    "n_kv_heads": w.n_kv_heads, "decode_steps": n_dec, "bits": "4/2",
-                   "saliency_ratio": w.saliency_ratio, "decode_phase": "CUDA graph replay"},
+                   "saliency_ratio": w.saliency_ratio, "decode_phase": "CUDA graph replay",
+                   "append": ("zc_append defers the copy into the next zc_decode_attention "
+                              "(ZC_FLAG_DEFER_APPEND)" if args.append == "deferred"
+                              else "zc_append launches its own copy kernel")},
         "prefill_tokens_per_s": world * R * w.batch * w.context / (t_pre * 1e-3),
         "prefill_ms": t_pre, "decode_ms": t_dec, "decode_us_per_call": per_call_us,
         "pct_of_hbm_peak": 100.0 * achieved / peak,

@@ -49,6 +49,14 @@ enum {
 
 #define ZC_MAX_WINDOW 128
 
+/* zc_config.flags.  With ZC_FLAG_DEFER_APPEND, zc_append enqueues nothing: the new row is
+ * taken straight from k_new / v_new by the next zc_decode_attention on the same cache and
+ * stream, which also stores it into the tail (Alg. 3's concat and attention as one step: one
+ * launch less and no wait between the two).  The caller then promises that k_new and v_new
+ * stay valid and unchanged until the stream has passed that zc_decode_attention call.  Any
+ * other call on the cache first performs the pending append as its own launch. */
+#define ZC_FLAG_DEFER_APPEND 1
+
 /* Plain-data configuration; set struct_size = sizeof(zc_config). */
 typedef struct {
   int32_t struct_size;
@@ -63,7 +71,7 @@ typedef struct {
                              (Alg. 3 uses 100); 8 <= window <= ZC_MAX_WINDOW */
   int32_t bits_hi;        /* bit-width of salient tokens: 4 or 2 */
   int32_t bits_lo;        /* bit-width of regular tokens: 4 or 2 */
-  int32_t reserved;       /* must be 0 */
+  int32_t flags;          /* 0 or ZC_FLAG_DEFER_APPEND */
   double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
 } zc_config;
 
@@ -104,7 +112,8 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
                         void* workspace, size_t workspace_bytes, zc_stream_t stream);
 
 /* Append (Eq. 3, Alg. 3): k_new, v_new [device] b x h_kv x d, contiguous, are copied
- * verbatim into the full-precision tail.  ZC_ECAPACITY beyond max_new_tokens. */
+ * verbatim into the full-precision tail.  ZC_ECAPACITY beyond max_new_tokens.  With
+ * ZC_FLAG_DEFER_APPEND the copy happens inside the next zc_decode_attention (see the flag). */
 int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t stream);
 
 /* Decode attention (Eq. 4, Alg. 3): q [device] b x h_q x d -> out [device] b x h_q x d,

@@ -12,6 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libzipcache.so")
 
 ZC_F16, ZC_BF16 = 0, 1
+ZC_FLAG_DEFER_APPEND = 1
 
 
 class ZipCacheError(RuntimeError):
@@ -23,16 +24,17 @@ class ZcConfig(C.Structure):
         ("struct_size", C.c_int32), ("dtype", C.c_int32), ("batch", C.c_int32),
         ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
         ("max_prefill", C.c_int32), ("max_new_tokens", C.c_int32), ("window", C.c_int32),
-        ("bits_hi", C.c_int32), ("bits_lo", C.c_int32), ("reserved", C.c_int32),
+        ("bits_hi", C.c_int32), ("bits_lo", C.c_int32), ("flags", C.c_int32),
         ("saliency_ratio", C.c_double),
     ]
 
     @classmethod
     def make(cls, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
-             saliency_ratio, bits_hi=4, bits_lo=2, window=100, head_dim=128) -> "ZcConfig":
+             saliency_ratio, bits_hi=4, bits_lo=2, window=100, head_dim=128,
+             flags=0) -> "ZcConfig":
         code = {torch.float16: ZC_F16, torch.bfloat16: ZC_BF16}.get(dtype, dtype)
         return cls(C.sizeof(cls), code, batch, n_q_heads, n_kv_heads, head_dim, max_prefill,
-                   max_new_tokens, window, bits_hi, bits_lo, 0, float(saliency_ratio))
+                   max_new_tokens, window, bits_hi, bits_lo, flags, float(saliency_ratio))
 
 
 _lib = None
@@ -218,11 +220,12 @@ class ZipCache:
 
     def __init__(self, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
-                 workspace: Optional[torch.Tensor] = None):
+                 workspace: Optional[torch.Tensor] = None, defer_append: bool = False):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
-                                 saliency_ratio, bits_hi, bits_lo, window)
+                                 saliency_ratio, bits_hi, bits_lo, window,
+                                 flags=ZC_FLAG_DEFER_APPEND if defer_append else 0)
         self.dtype, self.device = dtype, torch.device(device)
         self.batch, self.n_q_heads, self.n_kv_heads = batch, n_q_heads, n_kv_heads
         self.cache_bytes, self.workspace_bytes = zc_cache_bytes(self.cfg)

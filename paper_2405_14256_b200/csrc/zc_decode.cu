@@ -505,7 +505,7 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
 template <typename T>
 __device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, const ZcLayout& lay,
                                           const T* qbase, int Gl, int unit, int h0, char* smem,
-                                          float* __restrict__ tail_logits) {
+                                          const T* k_new, const T* v_new) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   float* wm = reinterpret_cast<float*>(smem + kOffWm);
   float* wl = reinterpret_cast<float*>(smem + kOffWl);
@@ -518,28 +518,46 @@ __device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, con
     for (int i = lane; i < 4 * ZC_D; i += 32) mbuf[i] = 0.f;
     return;
   }
-  const T* tK = reinterpret_cast<const T*>(ub + lay.off_tailK);
-  const T* tV = reinterpret_cast<const T*>(ub + lay.off_tailV);
+  T* tK = reinterpret_cast<T*>(const_cast<char*>(ub) + lay.off_tailK);
+  T* tV = reinterpret_cast<T*>(const_cast<char*>(ub) + lay.off_tailV);
   const int last = d.n_tok - 1;
+  // Deferred append: the newest row still lives in the caller's k_new / v_new [unit][128].
+  // It is read from there, and the warp whose 16 tokens include it stores it into the tail.
+  const T* newK = k_new ? k_new + (long long)unit * ZC_D : nullptr;
+  const T* newV = v_new ? v_new + (long long)unit * ZC_D : nullptr;
+  if (newK && last >= base && last < base + ZC_SUB) {
+    if (lane < 16)
+      reinterpret_cast<uint4*>(tK + last * ZC_D)[lane] = reinterpret_cast<const uint4*>(newK)[lane];
+    else
+      reinterpret_cast<uint4*>(tV + last * ZC_D)[lane - 16] = reinterpret_cast<const uint4*>(newV)[lane - 16];
+  }
   // rows past the end are read from the last valid row and masked
   const int r0 = min(base + g, last), r1 = min(base + g + 8, last);
   const int va_r = min(base + 2 * t, last), vb_r = min(base + 2 * t + 8, last);
   const int vc_r = min(base + 2 * t + 1, last), vd_r = min(base + 2 * t + 9, last);
+  auto krow = [&](int r) -> const T* { return (newK && r == last) ? newK : tK + r * ZC_D; };
+  auto vrow = [&](int r) -> const T* { return (newV && r == last) ? newV : tV + r * ZC_D; };
+  const T* k0p = krow(r0);
+  const T* k1p = krow(r1);
   uint4 qv[4], ka[4], kb[4];
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     qv[c] = g < Gl ? *reinterpret_cast<const uint4*>(qbase + g * ZC_D + 32 * c + 8 * t) : make_uint4(0, 0, 0, 0);
-    ka[c] = *reinterpret_cast<const uint4*>(tK + r0 * ZC_D + 32 * c + 8 * t);
-    kb[c] = *reinterpret_cast<const uint4*>(tK + r1 * ZC_D + 32 * c + 8 * t);
+    ka[c] = *reinterpret_cast<const uint4*>(k0p + 32 * c + 8 * t);
+    kb[c] = *reinterpret_cast<const uint4*>(k1p + 32 * c + 8 * t);
   }
   // V: this lane's 16 channels (16g .. 16g+15) of the four tokens its fragments pair up
+  const T* vap = vrow(va_r);
+  const T* vbp = vrow(vb_r);
+  const T* vcp = vrow(vc_r);
+  const T* vdp = vrow(vd_r);
   uint4 va[2], vb[2], vc[2], vd[2];
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
-    va[u] = *reinterpret_cast<const uint4*>(tV + va_r * ZC_D + 16 * g + 8 * u);
-    vb[u] = *reinterpret_cast<const uint4*>(tV + vb_r * ZC_D + 16 * g + 8 * u);
-    vc[u] = *reinterpret_cast<const uint4*>(tV + vc_r * ZC_D + 16 * g + 8 * u);
-    vd[u] = *reinterpret_cast<const uint4*>(tV + vd_r * ZC_D + 16 * g + 8 * u);
+    va[u] = *reinterpret_cast<const uint4*>(vap + 16 * g + 8 * u);
+    vb[u] = *reinterpret_cast<const uint4*>(vbp + 16 * g + 8 * u);
+    vc[u] = *reinterpret_cast<const uint4*>(vcp + 16 * g + 8 * u);
+    vd[u] = *reinterpret_cast<const uint4*>(vdp + 16 * g + 8 * u);
   }
   // ---- S^T: k-step (c, pp) contracts channels 32c + 8t + 4pp + {0,1 | 2,3} ----
   float dacc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -559,9 +577,11 @@ __device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, con
     lg[1][e] = dacc[2 + e] * scale;
     const int h = 2 * t + e;
     if (t < 2 && h < Gl) {
-      float* tl = tail_logits + ((long long)unit * lay.G + h0 + h) * ZC_MAX_WINDOW + base;
-      if (v0) tl[g] = lg[0][e];
-      if (v1) tl[g + 8] = lg[1][e];
+      // kept in shared memory: the scratch in global memory may still be read by the previous
+      // call's combine kernel until this kernel has passed its wait
+      float* stash = mbuf + 4 * ZC_D + h * ZC_SUB;
+      if (v0) stash[g] = lg[0][e];
+      if (v1) stash[g + 8] = lg[1][e];
     }
     if (!v0) lg[0][e] = -INFINITY;
     if (!v1) lg[1][e] = -INFINITY;
@@ -636,7 +656,8 @@ template <typename T>
 __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, ZcLayout lay,
                                                                   ZcDecodePlan plan,
                                                                   const T* __restrict__ q, float* part,
-                                                                  float* tail_logits) {
+                                                                  float* tail_logits, const T* k_new,
+                                                                  const T* v_new) {
   extern __shared__ __align__(128) char smem[];
   float* wm = reinterpret_cast<float*>(smem + kOffWm);
   float* wl = reinterpret_cast<float*>(smem + kOffWl);
@@ -666,8 +687,10 @@ __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, Z
         compressed_item<T, 2>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
     }
   } else {
-    pdl_wait();   // the newest tail row is written by the append kernel just before this one
-    tail_item<T>(d, ub, lay, qbase, Gl, unit, h0, smem, tail_logits);
+    // the newest tail row comes from the append kernel just before this one, unless the
+    // append was deferred into this kernel
+    if (!k_new) pdl_wait();
+    tail_item<T>(d, ub, lay, qbase, Gl, unit, h0, smem, k_new, v_new);
   }
   __syncthreads();
   // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
@@ -691,6 +714,16 @@ __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, Z
   __syncthreads();
   // everything this CTA writes to global memory may still be in use by the previous kernel
   pdl_wait();
+  if (d.kind == 1) {
+    const int base = d.sub_lo * (kWarps * ZC_SUB) + warp * ZC_SUB;
+    const int nv = min(ZC_SUB, d.n_tok - base);
+    const float* stash = reinterpret_cast<const float*>(smem + warp * kWarpRing) + 4 * ZC_D;
+    for (int e = lane; e < Gl * ZC_SUB; e += 32) {
+      const int h = e / ZC_SUB, tok = e % ZC_SUB;
+      if (tok < nv)
+        tail_logits[((long long)unit * G + h0 + h) * ZC_MAX_WINDOW + base + tok] = stash[h * ZC_SUB + tok];
+    }
+  }
   for (int h = 0; h < Gl; ++h) {
     float o = 0.f;
     if (has) {
@@ -836,14 +869,23 @@ int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
 }
 
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
-                     float* ws, cudaStream_t st) {
+                     float* ws, const void* k_new, const void* v_new, cudaStream_t st) {
   const int G = c->lay.G;
   float* part = ws;
   float* tail_logits = ws + (size_t)c->lay.units * plan.items * G * ZC_PART_STRIDE;
   dim3 grid(plan.items, c->lay.units, (G + 3) / 4);
   const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
   const char* q_lo = (const char*)q;
-  const bool overlap = !(g_last_out_lo && q_lo < g_last_out_hi && q_lo + io_bytes > g_last_out_lo);
+  bool overlap = !(g_last_out_lo && q_lo < g_last_out_hi && q_lo + io_bytes > g_last_out_lo);
+  if (k_new && g_last_out_lo) {
+    // a deferred append is read ahead of the wait as well
+    const size_t kv_bytes = (size_t)c->lay.units * ZC_D * 2;
+    const char* kl = (const char*)k_new;
+    const char* vl = (const char*)v_new;
+    if ((kl < g_last_out_hi && kl + kv_bytes > g_last_out_lo) ||
+        (vl < g_last_out_hi && vl + kv_bytes > g_last_out_lo))
+      overlap = false;
+  }
   const dim3 cgrid(c->lay.units);
   cudaError_t e;
   if (c->cfg.dtype == ZC_F16) {
@@ -851,7 +893,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
                              kDecodeSmem);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_items<__half>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay,
-                   plan, (const __half*)q, part, tail_logits);
+                   plan, (const __half*)q, part, tail_logits, (const __half*)k_new, (const __half*)v_new);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_combine<__half>, cgrid, dim3(128), kCombineSmem, st, true, c->base, c->lay,
                    plan, (__half*)out, (const float*)part, (const float*)tail_logits, collect);
@@ -860,7 +902,8 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_items<__nv_bfloat16>, grid, dim3(128), kDecodeSmem, st, overlap, c->base,
-                   c->lay, plan, (const __nv_bfloat16*)q, part, tail_logits);
+                   c->lay, plan, (const __nv_bfloat16*)q, part, tail_logits, (const __nv_bfloat16*)k_new,
+                   (const __nv_bfloat16*)v_new);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_combine<__nv_bfloat16>, cgrid, dim3(128), kCombineSmem, st, true, c->base,
                    c->lay, plan, (__nv_bfloat16*)out, (const float*)part, (const float*)tail_logits,

@@ -27,7 +27,7 @@ int check_config(const zc_config* cfg) {
   if (cfg->window < 8 || cfg->window > ZC_MAX_WINDOW) return ZC_EINVAL;
   if (cfg->bits_hi != 4 && cfg->bits_hi != 2) return ZC_EINVAL;
   if (cfg->bits_lo != 4 && cfg->bits_lo != 2) return ZC_EINVAL;
-  if (cfg->reserved != 0) return ZC_EINVAL;
+  if (cfg->flags & ~ZC_FLAG_DEFER_APPEND) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if ((long long)cfg->batch * cfg->n_kv_heads > 65535) return ZC_EINVAL;
   // every re-compressed window adds two items to a decode call
@@ -110,6 +110,16 @@ int cuda_fail(cudaError_t e) {
   } while (0)
 
 }  // namespace
+
+// Performs a deferred append as its own launch (a call other than decode attention came first).
+static int flush_pending(zc_cache* c) {
+  if (!c->pend_k) return ZC_OK;
+  const void* k = c->pend_k;
+  const void* v = c->pend_v;
+  c->pend_k = c->pend_v = nullptr;
+  ZC_CUDA(zc_launch_append(c, k, v, c->n_tail - 1, c->pend_stream));
+  return ZC_OK;
+}
 
 ZcSeg zc_segment(const zc_cache* c, int seg) {
   ZcSeg s;
@@ -277,6 +287,7 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
     return ZC_EALIGN;
   }
   cudaStream_t st = (cudaStream_t)stream;
+  c->pend_k = c->pend_v = nullptr;   // a prefill starts the cache over
   c->l0 = l;
   c->n0[0] = n_salient(c->cfg.saliency_ratio, l);
   c->n0[1] = l - c->n0[0];
@@ -310,7 +321,15 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
   if (!aligned16(k_new) || !aligned16(v_new)) return ZC_EALIGN;
   if (c->n_new >= c->cfg.max_new_tokens) return ZC_ECAPACITY;
   if (c->n_tail >= c->cfg.window) return ZC_ESTATE;
-  ZC_CUDA(zc_launch_append(c, k_new, v_new, c->n_tail, (cudaStream_t)stream));
+  int rc = flush_pending(c);
+  if (rc) return rc;
+  if (c->cfg.flags & ZC_FLAG_DEFER_APPEND) {
+    c->pend_k = k_new;
+    c->pend_v = v_new;
+    c->pend_stream = (cudaStream_t)stream;
+  } else {
+    ZC_CUDA(zc_launch_append(c, k_new, v_new, c->n_tail, (cudaStream_t)stream));
+  }
   c->n_tail += 1;
   c->n_new += 1;
   return ZC_OK;
@@ -323,11 +342,18 @@ int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return ZC_EALIGN;
   if (workspace_bytes < c->ws_bytes) return ZC_ECAPACITY;
   cudaStream_t st = (cudaStream_t)stream;
+  if (c->pend_k && c->pend_stream != st) {
+    int rc = flush_pending(c);
+    if (rc) return rc;
+  }
   ZcDecodePlan plan = zc_make_plan(c);
   const int i_next = c->step_i + 1;
   const int collect =
       (c->n_tail > 0) && (is_probe_step || i_next > c->cfg.window - 5) ? 1 : 0;
-  ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (float*)workspace, st));
+  const void* pk = c->pend_k;
+  const void* pv = c->pend_v;
+  c->pend_k = c->pend_v = nullptr;
+  ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (float*)workspace, pk, pv, st));
   // Alg. 3 bookkeeping: the step counter follows the tokens of the current window
   if (c->n_tail > 0) {
     c->step_i = i_next;
@@ -380,6 +406,7 @@ int zc_segment_tokens(const zc_cache* c, int segment, int subset) {
 int zc_export_scores(zc_cache* c, float* p_tilde, zc_stream_t stream) {
   if (!c || !p_tilde) return ZC_EINVAL;
   if (c->l0 < 0) return ZC_ESTATE;
+  { int rc = flush_pending(c); if (rc) return rc; }
   ZC_CUDA(zc_launch_export_scores(c, p_tilde, c->last_scores_n, (cudaStream_t)stream));
   return ZC_OK;
 }
@@ -389,6 +416,7 @@ int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t*
   if (!c || tensor < 0 || tensor > 1 || subset < 0 || subset > 1) return ZC_EINVAL;
   if (c->l0 < 0) return ZC_ESTATE;
   if (segment < 0 || segment >= c->n_seg) return ZC_EINVAL;
+  { int rc = flush_pending(c); if (rc) return rc; }
   ZC_CUDA(zc_launch_export_segment(c, zc_segment(c, segment), tensor, subset, idx, codes, sz, cf,
                                    (cudaStream_t)stream));
   return ZC_OK;

@@ -93,6 +93,10 @@ struct zc_cache {
   int last_scores_n;
   int n_sm;
   long long launches;
+  // deferred append: the row at tail index n_tail - 1 still lives in the caller's buffers
+  const void* pend_k;
+  const void* pend_v;
+  cudaStream_t pend_stream;
 };
 
 __host__ __device__ static inline int zc_ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -110,8 +114,10 @@ int zc_launch_window_scores(zc_cache* c, cudaStream_t st);
 int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st);
 int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
                      cudaStream_t st);
+// k_new / v_new non-null: the newest tail row is read from them and stored into the tail.
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out,
-                     int collect, float* ws, cudaStream_t st);
+                     int collect, float* ws, const void* k_new, const void* v_new,
+                     cudaStream_t st);
 #define ZC_TAIL_ITEM_TOKENS 64
 int zc_device_error_code(int* out);
 // Device address of the built-in scratch buffer on the current device (looked up once per device).

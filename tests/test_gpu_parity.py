@@ -210,3 +210,51 @@ def test_full_size_configs_on_sampled_units(cfg_id, units, steps):
     print(f"config {cfg_id}: near-tie swaps {swaps}, worst decode error {worst:.2e}")
     if swaps == 0:
         assert tl.compare_segment(cache, oc, 0, units=units) == 0
+
+
+@pytest.mark.parametrize("kw,steps", [
+    (dict(context=512, n_q_heads=4, n_kv_heads=4), 16),
+    (dict(context=300, batch=2, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0), 6),
+    (dict(context=70, n_q_heads=8, n_kv_heads=1, saliency_ratio=0.5), 4),
+    (dict(context=150, n_q_heads=4, n_kv_heads=2, window=16, rho_recent=0.1, rho_random=0.1), 40),
+    (dict(context=150, n_q_heads=4, n_kv_heads=2, window=100, rho_recent=0.1, rho_random=0.1), 105),
+])
+def test_deferred_append_gives_the_same_results(kw, steps):
+    """With ZC_FLAG_DEFER_APPEND the new row is consumed from the caller's buffers by the
+    decode kernel and stored into the tail there: outputs, re-compressed windows and the
+    tail must match the oracle exactly as with the separate append launch."""
+    w = tl.small_workload(**kw)
+    worst, cache, oc = tl.run_decode_parity(w, steps, defer_append=True)
+    assert worst <= 2e-3
+    import paper_2405_14256_b200 as zc
+    for seg in range(1, zc.zc_num_segments(cache.handle)):
+        assert tl.compare_segment(cache, oc, seg) == 0
+    assert zc.zc_device_status() == 0
+
+
+def test_deferred_append_is_performed_by_any_other_call():
+    """Two appends in a row, and an export between append and decode: the pending row must
+    reach the tail through its own launch, and the result must equal the undeferred path."""
+    from workloads import make_decode_step
+    w = tl.small_workload(context=200, n_q_heads=4, n_kv_heads=2, batch=2)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w).tolist()
+    outs = []
+    for defer in (False, True):
+        cache = tl.make_cache(w, max_new=8, defer_append=defer)
+        cache.mem.zero_()
+        cache.prefill_compress(Q, K, V, P)
+        q0, k0, v0 = make_decode_step(w, 0, 0, tl.DEV)
+        q1, k1, v1 = make_decode_step(w, 0, 1, tl.DEV)
+        q2, k2, v2 = make_decode_step(w, 0, 2, tl.DEV)
+        cache.append(k0, v0)
+        cache.append(k1, v1)            # performs the first one
+        o1 = cache.decode_attention(q1, True)
+        cache.append(k2, v2)
+        cache.scores(w.context)         # an export performs the pending append
+        o2 = cache.decode_attention(q2, False)
+        torch.cuda.synchronize()
+        outs.append((o1.clone(), o2.clone(), cache.mem.clone()))
+    assert torch.equal(outs[0][0], outs[1][0])
+    assert torch.equal(outs[0][1], outs[1][1])
+    assert torch.equal(outs[0][2], outs[1][2])

@@ -24,11 +24,11 @@ def to64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu", torch.float64).numpy()
 
 
-def make_cache(w: Workload, max_new=None):
+def make_cache(w: Workload, max_new=None, defer_append: bool = False):
     import paper_2405_14256_b200 as zc
     return zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context,
                        w.decode_steps if max_new is None else max_new, w.saliency_ratio,
-                       w.bits_hi, w.bits_lo, w.window, device=DEV)
+                       w.bits_hi, w.bits_lo, w.window, device=DEV, defer_append=defer_append)
 
 
 def make_oracle(w: Workload, units=None) -> zo.ZipCacheOracle:
@@ -88,14 +88,14 @@ def output_error(got: np.ndarray, ref: np.ndarray, dtype) -> float:
 
 
 def run_decode_parity(w: Workload, n_steps: int, tol: float = 2e-3, units=None, layer: int = 0,
-                      staged: bool = True, check_segments: bool = True):
+                      staged: bool = True, check_segments: bool = True, defer_append: bool = False):
     """Prefill + n_steps of append/decode on GPU and oracle; returns max abs output error."""
     Q, K, V = make_prefill(w, layer, DEV)
     P = probes_for(w, layer)
     oc = make_oracle(w, units)
     Qh, Kh, Vh = to64(Q), to64(K), to64(V)
     oc.prefill_compress(Qh, Kh, Vh, P)
-    cache = make_cache(w, max_new=max(n_steps, 1))
+    cache = make_cache(w, max_new=max(n_steps, 1), defer_append=defer_append)
     if staged:
         n_s = zo.salient_count(w.saliency_ratio, w.context)
         sal = np.zeros((w.batch, w.n_kv_heads, max(n_s, 1)), dtype=np.int32)
