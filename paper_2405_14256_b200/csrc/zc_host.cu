@@ -145,29 +145,37 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
     p.tiles0[k] = zc_ceil_div(c->n0[k], ZC_TILE);
     p.tilesw[k] = zc_ceil_div(c->nw[k], ZC_TILE);
   }
-  // Items of segment 0 aim at ZC_ITEM_SUBS sub-tiles: few enough CTAs that their set-up and
-  // merge stay small next to the streaming loop, which overlaps with the neighbouring calls
-  // of the stream; with few units the split grows until one wave of CTAs covers the SMs.
+  // How finely to cut segment 0.  Two things cost time: CTAs that do not fill a whole wave of
+  // the GPU (slots = SMs x resident CTAs), and the fixed set-up and merge of every CTA, worth
+  // about ZC_ITEM_OVERHEAD sub-tiles of streaming.  Each candidate item size is scored by
+  // (share of the slot-time its waves use) x (share of a CTA's life spent streaming).
   p.tail_items = zc_ceil_div(c->n_tail, ZC_TAIL_ITEM_TOKENS);
   const int extras = p.tail_items + 2 * (c->n_seg - 1);
   const int slots = c->n_sm * ZC_DECODE_CTAS_PER_SM;
-  int subs[2], want[2];
-  for (int k = 0; k < 2; ++k) {
-    subs[k] = zc_ceil_div(c->n0[k], ZC_SUB);
-    want[k] = std::max(1, zc_ceil_div(subs[k], ZC_ITEM_SUBS));
-  }
-  const int fill = slots / (2 * c->lay.units) - extras;   // half a wave from this call alone
-  if (want[0] + want[1] < fill) {
-    const int tot = std::max(1, subs[0] + subs[1]);
-    for (int k = 0; k < 2; ++k) want[k] = std::max(want[k], (int)((long long)subs[k] * fill / tot));
-  }
+  const int zs = zc_ceil_div(c->lay.G, 4);
   const int cap = std::max(1, (ZC_MAX_ITEMS - extras) / 2);
-  for (int k = 0; k < 2; ++k) {
-    const int s = std::max(1, std::min(std::min(want[k], std::min(ZC_MAX_SPLIT_HOST, cap)),
-                                       std::max(1, subs[k])));
-    // an even number of sub-tiles per item: the kernel consumes them in pairs
-    p.spi0[k] = (zc_ceil_div(std::max(1, subs[k]), s) + 1) & ~1;
-    p.split0[k] = zc_ceil_div(std::max(1, subs[k]), p.spi0[k]);
+  int subs[2];
+  for (int k = 0; k < 2; ++k) subs[k] = std::max(1, zc_ceil_div(c->n0[k], ZC_SUB));
+  static const int kCand[] = {256, 192, 128, 96, 64, 48, 32};
+  double best = -1.0;
+  for (int target : kCand) {
+    int spi[2], split[2];
+    for (int k = 0; k < 2; ++k) {
+      const int want = std::min(std::min(zc_ceil_div(subs[k], target), std::min(ZC_MAX_SPLIT_HOST, cap)),
+                                subs[k]);
+      // an even number of sub-tiles per item: the kernel consumes them in pairs
+      spi[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;
+      split[k] = zc_ceil_div(subs[k], spi[k]);
+    }
+    const double n_ctas = (double)(split[0] + split[1] + extras) * c->lay.units * zs;
+    const double waves = n_ctas / slots;
+    const double fill = n_ctas / (ceil(waves) * slots);
+    const double per_item = (double)(subs[0] + subs[1]) / (split[0] + split[1]);
+    const double score = fill * per_item / (per_item + ZC_ITEM_OVERHEAD);
+    if (score > best) {
+      best = score;
+      for (int k = 0; k < 2; ++k) { p.spi0[k] = spi[k]; p.split0[k] = split[k]; }
+    }
   }
   p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + p.tail_items;
   return p;

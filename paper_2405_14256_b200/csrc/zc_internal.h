@@ -14,8 +14,8 @@
 #define ZC_MAX_G 8
 #define ZC_MAX_SPLIT_HOST 32      // most items one class of segment 0 is split into
 #define ZC_MAX_ITEMS 128          // most items of one unit in one decode call
-#ifndef ZC_ITEM_SUBS
-#define ZC_ITEM_SUBS 128          // 16-token sub-tiles one item of segment 0 aims at
+#ifndef ZC_ITEM_OVERHEAD
+#define ZC_ITEM_OVERHEAD 24       // fixed cost of one split-K item, in 16-token sub-tiles of streaming
 #endif
 #ifndef ZC_DECODE_CTAS_PER_SM
 #define ZC_DECODE_CTAS_PER_SM 3
