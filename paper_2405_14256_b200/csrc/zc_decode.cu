@@ -41,8 +41,8 @@ constexpr int kWaitLimit = 1 << 22;
 #define ZC_KPEXP 12
 #define ZC_TAU 3.5f
 #endif
-#ifndef ZC_QK_CHAINS
-#define ZC_QK_CHAINS 1
+#ifndef ZC_SHIFT_ON_FMA
+#define ZC_SHIFT_ON_FMA 0
 #endif
 constexpr int kPExp = ZC_KPEXP;      // softmax weights go to f16 as p * s^V * 2^kPExp / 2^ceil(log2 smax)
 constexpr float kTau = ZC_TAU;   // the running maximum is refreshed only when a logit exceeds it by this
@@ -175,11 +175,182 @@ template <int BITS> __device__ __forceinline__ void chan_slot(int off, int* reg,
   }
 }
 
-// Compressed-run part of one item, one warp: prologue done by the CTA, stages primed.
-// One iteration handles a PAIR of 16-token sub-tiles (one ring stage): two independent
-// chains of work per warp keep the pipes busy between dependent instructions.
-// Column n of the q' B-fragments is (head n >> 1, part n & 1) with q' = hi + lo in f16, so
-// that lane (g, t) receives both parts of head t for tokens g and g + 8 in its accumulator.
+// w >> 8 on the multiply pipe: the integer pipe is the busiest unit of the loop (one mask per
+// tensor-core operand register), every shift moved off it is a net gain.
+__device__ __forceinline__ uint32_t shr8(uint32_t w) {
+#if ZC_SHIFT_ON_FMA
+  uint32_t r;
+  asm("mul.hi.u32 %0, %1, 16777216;\n" : "=r"(r) : "r"(w));
+  return r;
+#else
+  return w >> 8;
+#endif
+}
+
+// expect_tx + bulk copy by one lane without a divergent branch
+__device__ __forceinline__ void refill_if(bool pred, uint64_t* bar, void* dst, const void* src, int bytes) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %0, 0;\n"
+      " @p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n"
+      " @p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%3], [%4], %2, [%1];\n}\n" ::"r"(
+          (int)pred),
+      "r"(zc_smem_u32(bar)), "r"(bytes), "r"(zc_smem_u32(dst)), "l"(src)
+      : "memory");
+}
+
+struct PairState {
+  float mu;       // running maximum of u = logit / isc
+  float mo_neg;   // logKs - mu * isc
+  float uthr;     // mu + kTau / isc
+  float l, zacc;
+};
+
+// One PAIR of 16-token sub-tiles (one ring stage) for one warp: two independent chains of work
+// keep the pipes busy between dependent instructions.  Column n of the q' B-fragments is
+// (head n >> 1, part n & 1) with q' = hi + lo in f16, so that lane (g, t) receives both parts
+// of head t for tokens g and g + 8 in its accumulator.  LAST: the pair may reach past the end
+// of the run (`rem` tokens left from its first token); otherwise it is complete.
+template <int BITS, bool LAST>
+__device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uint32_t (&qb)[16],
+                                          float qs, float isc, float logKs, float tau_u, int srcA,
+                                          int srcB, int c0_src, int c1_src, float (&oacc)[8][4],
+                                          PairState& S) {
+  constexpr int SB = ZC_SUB * (32 * BITS + 16);
+  const int g = lane >> 2;
+  if (LAST && rem <= ZC_SUB) {
+    // the run ends inside the first half: the second half was not copied; its tokens are
+    // masked below, its parameters must not hold stale bits
+    if (lane < ZC_SUB) *reinterpret_cast<float4*>(st + SB + 512 * BITS + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncwarp();
+  }
+  // ---- loads: K words of tokens g and g+8, V words, parameters (sK, zK, sV, zV), both halves ----
+  uint32_t kw[2][2][BITS];   // [half][token slot][word]
+  uint32_t vw[2][2 * BITS];
+  float4 pp[2][2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const char* sh = st + h * SB;
+    if (BITS == 4) {
+      const uint4 a = *reinterpret_cast<const uint4*>(sh + lane * 16);
+      const uint4 b = *reinterpret_cast<const uint4*>(sh + 512 + lane * 16);
+      kw[h][0][0] = a.x; kw[h][0][1] = a.y; kw[h][0][2] = a.z; kw[h][0][3] = a.w;
+      kw[h][1][0] = b.x; kw[h][1][1] = b.y; kw[h][1][2] = b.z; kw[h][1][3] = b.w;
+      const uint4 c = *reinterpret_cast<const uint4*>(sh + 1024 + lane * 16);
+      const uint4 e = *reinterpret_cast<const uint4*>(sh + 1536 + lane * 16);
+      vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
+      vw[h][4] = e.x; vw[h][5] = e.y; vw[h][6] = e.z; vw[h][7] = e.w;
+    } else {
+      const uint2 a = *reinterpret_cast<const uint2*>(sh + lane * 8);
+      const uint2 b = *reinterpret_cast<const uint2*>(sh + 256 + lane * 8);
+      kw[h][0][0] = a.x; kw[h][0][1] = a.y;
+      kw[h][1][0] = b.x; kw[h][1][1] = b.y;
+      const uint4 c = *reinterpret_cast<const uint4*>(sh + 512 + lane * 16);
+      vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
+    }
+    pp[h][0] = *reinterpret_cast<const float4*>(sh + 512 * BITS + g * 16);
+    pp[h][1] = *reinterpret_cast<const float4*>(sh + 512 * BITS + (g + 8) * 16);
+  }
+  // ---- S^T = codes(16 tokens x 128) . q'^T per half: 8 k-steps; the halves are independent chains ----
+  float u[2][2];   // [half][token slot] logits (base 2) of head t, divided by isc
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float dacc[4];
+    if (BITS == 4) {
+#pragma unroll
+      for (int jw = 0; jw < 4; ++jw) {
+        const uint32_t w0 = kw[h][0][jw], w1 = kw[h][1][jw];
+        const uint32_t a0[4] = {w0 & 0x000F000Fu, w1 & 0x000F000Fu, w0 & 0x00F000F0u, w1 & 0x00F000F0u};
+        if (jw == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
+        else zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
+        const uint32_t x0 = shr8(w0), x1 = shr8(w1);
+        const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
+        zc_mma16816<__half>(dacc, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
+      }
+    } else {
+#pragma unroll
+      for (int jw = 0; jw < 2; ++jw) {
+#pragma unroll
+        for (int hb = 0; hb < 2; ++hb) {
+          const uint32_t w0 = hb ? shr8(kw[h][0][jw]) : kw[h][0][jw];
+          const uint32_t w1 = hb ? shr8(kw[h][1][jw]) : kw[h][1][jw];
+          const int ks = 4 * jw + 2 * hb;
+          const uint32_t a0[4] = {w0 & 0x00030003u, w1 & 0x00030003u, w0 & 0x000C000Cu, w1 & 0x000C000Cu};
+          if (ks == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
+          else zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
+          const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
+          zc_mma16816<__half>(dacc, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
+        }
+      }
+    }
+    // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
+    u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
+    u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;
+  }
+  if (LAST && rem < 2 * ZC_SUB) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (16 * h + g >= rem) u[h][0] = -INFINITY;
+      if (16 * h + g + 8 >= rem) u[h][1] = -INFINITY;
+    }
+  }
+  const float mx = fmaxf(fmaxf(u[0][0], u[0][1]), fmaxf(u[1][0], u[1][1]));
+  if (__any_sync(kFull, mx > S.uthr)) {
+    float mr = mx;
+    mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 4));
+    mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 8));
+    mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 16));
+    const float mn = fmaxf(S.mu, mr);
+    const float corr = mn == -INFINITY ? 1.f : zc_exp2((S.mu - mn) * isc);
+    S.l *= corr; S.zacc *= corr;
+    S.mu = mn; S.mo_neg = fmaf(-mn, isc, logKs); S.uthr = mn + tau_u;
+    const float c0 = __shfl_sync(kFull, corr, c0_src), c1 = __shfl_sync(kFull, corr, c1_src);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      oacc[j][0] *= c0; oacc[j][1] *= c1; oacc[j][2] *= c0; oacc[j][3] *= c1;
+    }
+  }
+  // p' = p * 2^logKs; weights w = p' * s^V go to f16, the same rounded values feed the z sum
+  uint32_t pb[2][2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const float p0 = zc_exp2(fmaf(u[h][0], isc, S.mo_neg)), p1 = zc_exp2(fmaf(u[h][1], isc, S.mo_neg));
+    S.l += p0 + p1;
+    const __half2 h2 = __floats2half2_rn(p0 * pp[h][0].z, p1 * pp[h][1].z);   // (token g, token g+8)
+    const float2 back = __half22float2(h2);
+    S.zacc = fmaf(back.x, pp[h][0].w, S.zacc);
+    S.zacc = fmaf(back.y, pp[h][1].w, S.zacc);
+    const uint32_t X = *reinterpret_cast<const uint32_t*>(&h2);
+    // B fragment of P^T, column n = g = head g & 3: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
+    pb[h][0] = __shfl_sync(kFull, X, srcA);
+    pb[h][1] = __shfl_sync(kFull, X, srcB);
+  }
+  // ---- O^T += V^T(128 channels x 16 tokens) . P^T per half: 8 M-tiles ----
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    if (BITS == 4) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint32_t w = vw[h][j], x = shr8(w);
+        const uint32_t a[4] = {w & 0x000F000Fu, w & 0x00F000F0u, x & 0x000F000Fu, x & 0x00F000F0u};
+        zc_mma16816<__half>(oacc[j], a, pb[h][0], pb[h][1]);
+      }
+    } else {
+#pragma unroll
+      for (int mw = 0; mw < 4; ++mw) {
+#pragma unroll
+        for (int e2 = 0; e2 < 2; ++e2) {
+          const uint32_t w = e2 ? shr8(vw[h][mw]) : vw[h][mw];
+          const uint32_t a[4] = {w & 0x00030003u, w & 0x00300030u, w & 0x000C000Cu, w & 0x00C000C0u};
+          zc_mma16816<__half>(oacc[2 * mw + e2], a, pb[h][0], pb[h][1]);
+        }
+      }
+    }
+  }
+}
+
+// Compressed-run part of one item, one warp: prologue done by the CTA, stages primed.  The
+// first my_np - NST iterations refill their stage and need no end-of-run handling; the last
+// NST do not refill and the very last pair may be cut short by the end of the run.
 template <int BITS>
 __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_base, char* my_ring,
                                           uint64_t* my_bar, const uint32_t (&qb)[16], float qs,
@@ -196,183 +367,46 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
   const int srcA = 8 * t + (g & 3), srcB = srcA + 4;
   const int c0_src = (lane & ~3) | ((2 * t) & 3), c1_src = (lane & ~3) | ((2 * t + 1) & 3);
   // Logits are kept divided by isc (u = lg / isc): u costs one multiply less per token.
-  float mu = -INFINITY;          // running maximum of u
-  float mo_neg = 0.f;            // logKs - mu * isc
-  float uthr = -INFINITY;        // mu + kTau / isc
+  PairState S;
+  S.mu = -INFINITY; S.mo_neg = 0.f; S.uthr = -INFINITY; S.l = 0.f; S.zacc = 0.f;
   const float tau_u = kTau / isc;
-  float l = 0.f, zacc = 0.f;
-  // loop state, advanced by additions only
   const int s_first = d.sub_lo + 2 * warp;
-  int rem = d.n_tok - (s_first - d.run_sub0) * ZC_SUB;   // tokens from this pair's first token to the run's end
+  const int rem0 = d.n_tok - (s_first - d.run_sub0) * ZC_SUB;   // tokens from the first pair's first token to the run's end
   const char* src_refill = class_base + (long long)(s_first + 2 * kWarps * NST) * SB;
-  int rem_refill = rem - 2 * ZC_SUB * kWarps * NST;
-  int refills = my_np - NST;
+  int rem_refill = rem0 - 2 * ZC_SUB * kWarps * NST;
   int stage = 0;
   uint32_t parity = 0;
-  const char* ring_lane = my_ring + lane * 16;
-  for (int i = 0; i < my_np; ++i) {
-    uint64_t* bar = &my_bar[stage];
+  auto wait_stage = [&](uint64_t* bar) {
     if (!mbar_try_wait(bar, parity)) {
       int spins = 0;
       while (!mbar_try_wait(bar, parity)) {
         if (++spins > kWaitLimit) { atomicExch(err, 1); break; }
       }
     }
+  };
+  const int n_refill = my_np - NST;
+  for (int i = 0; i < n_refill; ++i) {
+    uint64_t* bar = &my_bar[stage];
+    wait_stage(bar);
     char* st = my_ring + stage * PB;
-    if (rem <= ZC_SUB) {
-      // the run ends inside the first half: the second half was not copied; its tokens are
-      // masked below, its parameters must not hold stale bits
-      if (lane < ZC_SUB) *reinterpret_cast<float4*>(st + SB + 512 * BITS + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
-      __syncwarp();
-    }
-    // ---- loads: K words of tokens g and g+8, V words, parameters (sK, zK, sV, zV), both halves ----
-    uint32_t kw[2][2][BITS];   // [half][token slot][word]
-    uint32_t vw[2][2 * BITS];
-    float4 pp[2][2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const char* sh = ring_lane + stage * PB + h * SB;
-      if (BITS == 4) {
-        const uint4 a = *reinterpret_cast<const uint4*>(sh);
-        const uint4 b = *reinterpret_cast<const uint4*>(sh + 512);
-        kw[h][0][0] = a.x; kw[h][0][1] = a.y; kw[h][0][2] = a.z; kw[h][0][3] = a.w;
-        kw[h][1][0] = b.x; kw[h][1][1] = b.y; kw[h][1][2] = b.z; kw[h][1][3] = b.w;
-        const uint4 c = *reinterpret_cast<const uint4*>(sh + 1024);
-        const uint4 e = *reinterpret_cast<const uint4*>(sh + 1536);
-        vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
-        vw[h][4] = e.x; vw[h][5] = e.y; vw[h][6] = e.z; vw[h][7] = e.w;
-      } else {
-        const uint2 a = *reinterpret_cast<const uint2*>(st + h * SB + lane * 8);
-        const uint2 b = *reinterpret_cast<const uint2*>(st + h * SB + 256 + lane * 8);
-        kw[h][0][0] = a.x; kw[h][0][1] = a.y;
-        kw[h][1][0] = b.x; kw[h][1][1] = b.y;
-        const uint4 c = *reinterpret_cast<const uint4*>(sh + 512);
-        vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
-      }
-      pp[h][0] = *reinterpret_cast<const float4*>(st + h * SB + 512 * BITS + g * 16);
-      pp[h][1] = *reinterpret_cast<const float4*>(st + h * SB + 512 * BITS + (g + 8) * 16);
-    }
-    // ---- S^T = codes(16 tokens x 128) . q'^T per half: 8 k-steps; the halves are independent chains ----
-    float u[2][2];   // [half][token slot] logits (base 2) of head t, divided by isc
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      float dacc[4], dacc2[4] = {0.f, 0.f, 0.f, 0.f};
-      if (BITS == 4) {
-#pragma unroll
-        for (int jw = 0; jw < 4; ++jw) {
-          const uint32_t w0 = kw[h][0][jw], w1 = kw[h][1][jw];
-          const uint32_t a0[4] = {w0 & 0x000F000Fu, w1 & 0x000F000Fu, w0 & 0x00F000F0u, w1 & 0x00F000F0u};
-          if (jw == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
-          else zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
-          const uint32_t x0 = w0 >> 8, x1 = w1 >> 8;
-          const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
-          if (ZC_QK_CHAINS == 2 && jw == 0) zc_mma16816_z(dacc2, a1, qb[2], qb[3]);
-          else zc_mma16816<__half>(ZC_QK_CHAINS == 2 ? dacc2 : dacc, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
-        }
-      } else {
-#pragma unroll
-        for (int jw = 0; jw < 2; ++jw) {
-#pragma unroll
-          for (int hb = 0; hb < 2; ++hb) {
-            const uint32_t w0 = kw[h][0][jw] >> (8 * hb), w1 = kw[h][1][jw] >> (8 * hb);
-            const int ks = 4 * jw + 2 * hb;
-            const uint32_t a0[4] = {w0 & 0x00030003u, w1 & 0x00030003u, w0 & 0x000C000Cu, w1 & 0x000C000Cu};
-            if (ks == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
-            else zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
-            const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
-            if (ZC_QK_CHAINS == 2 && ks == 0) zc_mma16816_z(dacc2, a1, qb[2], qb[3]);
-            else zc_mma16816<__half>(ZC_QK_CHAINS == 2 ? dacc2 : dacc, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
-          }
-        }
-      }
-      // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
-      if (ZC_QK_CHAINS == 2) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) dacc[e] += dacc2[e];
-      }
-      u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
-      u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;
-    }
-    if (rem < 2 * ZC_SUB) {
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        if (16 * h + g >= rem) u[h][0] = -INFINITY;
-        if (16 * h + g + 8 >= rem) u[h][1] = -INFINITY;
-      }
-    }
-    const float mx = fmaxf(fmaxf(u[0][0], u[0][1]), fmaxf(u[1][0], u[1][1]));
-    if (__any_sync(kFull, mx > uthr)) {
-      float mr = mx;
-      mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 4));
-      mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 8));
-      mr = fmaxf(mr, __shfl_xor_sync(kFull, mr, 16));
-      const float mn = fmaxf(mu, mr);
-      const float corr = mn == -INFINITY ? 1.f : zc_exp2((mu - mn) * isc);
-      l *= corr; zacc *= corr;
-      mu = mn; mo_neg = fmaf(-mn, isc, logKs); uthr = mn + tau_u;
-      const float c0 = __shfl_sync(kFull, corr, c0_src), c1 = __shfl_sync(kFull, corr, c1_src);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        oacc[j][0] *= c0; oacc[j][1] *= c1; oacc[j][2] *= c0; oacc[j][3] *= c1;
-      }
-    }
-    // p' = p * 2^logKs; weights w = p' * s^V go to f16, the same rounded values feed the z sum
-    uint32_t pb[2][2];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const float p0 = zc_exp2(fmaf(u[h][0], isc, mo_neg)), p1 = zc_exp2(fmaf(u[h][1], isc, mo_neg));
-      l += p0 + p1;
-      const __half2 h2 = __floats2half2_rn(p0 * pp[h][0].z, p1 * pp[h][1].z);   // (token g, token g+8)
-      const float2 back = __half22float2(h2);
-      zacc = fmaf(back.x, pp[h][0].w, zacc);
-      zacc = fmaf(back.y, pp[h][1].w, zacc);
-      const uint32_t X = *reinterpret_cast<const uint32_t*>(&h2);
-      // B fragment of P^T, column n = g = head g & 3: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
-      pb[h][0] = __shfl_sync(kFull, X, srcA);
-      pb[h][1] = __shfl_sync(kFull, X, srcB);
-    }
-    // ---- O^T += V^T(128 channels x 16 tokens) . P^T per half: 8 M-tiles ----
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      if (BITS == 4) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t w = vw[h][j], x = w >> 8;
-          const uint32_t a[4] = {w & 0x000F000Fu, w & 0x00F000F0u, x & 0x000F000Fu, x & 0x00F000F0u};
-          zc_mma16816<__half>(oacc[j], a, pb[h][0], pb[h][1]);
-        }
-      } else {
-#pragma unroll
-        for (int mw = 0; mw < 4; ++mw) {
-#pragma unroll
-          for (int e2 = 0; e2 < 2; ++e2) {
-            const uint32_t w = vw[h][mw] >> (8 * e2);
-            const uint32_t a[4] = {w & 0x00030003u, w & 0x00300030u, w & 0x000C000Cu, w & 0x00C000C0u};
-            zc_mma16816<__half>(oacc[2 * mw + e2], a, pb[h][0], pb[h][1]);
-          }
-        }
-      }
-    }
-    // ---- refill this stage ----
+    pair_step<BITS, false>(st, lane, 0, qb, qs, isc, logKs, tau_u, srcA, srcB, c0_src, c1_src, oacc, S);
     __syncwarp();
-    if (refills > 0) {
-      if (lane == 0) {
-        const int bytes = rem_refill > ZC_SUB ? PB : SB;
-        mbar_expect_tx(bar, bytes);
-        bulk_copy_g2s(st, src_refill, bytes, bar);
-      }
-      src_refill += kWarps * PB;
-      rem_refill -= 2 * ZC_SUB * kWarps;
-    }
-    --refills;
-    rem -= 2 * ZC_SUB * kWarps;
+    refill_if(lane == 0, bar, st, src_refill, rem_refill > ZC_SUB ? PB : SB);
+    src_refill += kWarps * PB;
+    rem_refill -= 2 * ZC_SUB * kWarps;
+    if (++stage == NST) { stage = 0; parity ^= 1u; }
+  }
+  for (int i = max(n_refill, 0); i < my_np; ++i) {
+    wait_stage(&my_bar[stage]);
+    pair_step<BITS, true>(my_ring + stage * PB, lane, rem0 - i * (2 * ZC_SUB * kWarps), qb, qs, isc, logKs,
+                          tau_u, srcA, srcB, c0_src, c1_src, oacc, S);
     if (++stage == NST) { stage = 0; parity ^= 1u; }
   }
   // sums back to plain units: l' = sum p 2^logKs; zacc' = sum w z with w short by the odd-token 1/4
   const float inv_sig = odd_tok ? 4.f : 1.f;
-  l_out = l * zc_exp2(-logKs);
-  z_out = zacc * inv_sig;
-  m_out = mu == -INFINITY ? -INFINITY : mu * isc;
+  l_out = S.l * zc_exp2(-logKs);
+  z_out = S.zacc * inv_sig;
+  m_out = S.mu * isc;
 }
 
 // One compressed item, whole CTA.  On return every warp has put its (m, l, z-sum) and its
