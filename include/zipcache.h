@@ -150,7 +150,7 @@ int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t*
  * allowed or not possible -- a plug-in inside a serving process whose memory pool owns the
  * whole device and forbids further cudaMalloc calls, a latency-critical loop that must not
  * enter the allocator, a caller that has already given away its memory budget.  The split-K
- * partial results and the tail logits go to a fixed buffer of ZC_NOALLOC_SCRATCH_BYTES that is
+ * partial results go to a fixed buffer of ZC_NOALLOC_SCRATCH_BYTES that is
  * part of the library image (every GPU that loads the library carries it until the process
  * ends); the caller still owns q [device] and out [device].  The call allocates and frees
  * nothing.

@@ -1,12 +1,13 @@
 // Append (Eq. 3) and single-query attention over the mixed-precision cache (Eq. 4, Alg. 3).
 //
-// Split-K: every unit's cache is cut into items (a range of 16-token sub-tiles of one
-// precision class of one segment, or up to 64 tokens of the full-precision tail); one CTA per
-// item produces a partial (m, l, acc) per query head, and a small second kernel merges the
-// partials in a fixed order, writes the output and, on probe steps, adds the step's attention
+// Split-K: every unit's compressed cache is cut into items (a range of 16-token sub-tiles of
+// one precision class of one segment); one CTA per item produces a partial (m, l, acc) per
+// query head.  A small second kernel, one CTA per unit, computes the attention over the
+// full-precision tail on tensor cores while the items kernel is still streaming, then merges
+// everything in a fixed order, writes the output and, on probe steps, adds the step's attention
 // over the tail's tokens to the window statistics.  The kernels of one step (append, items,
-// combine) are chained by programmatic dependent launch: each may start while its
-// predecessor drains and orders itself with griddepcontrol.wait.  Nothing spins on another CTA.
+// combine) are chained by programmatic dependent launch: each may start while its predecessor
+// drains and orders itself with griddepcontrol.wait.  Nothing spins on another CTA.
 //
 // Dequantisation is folded so that it is never done per element:
 //   q . k_hat_t = s_t (q' . code_t - z_t sum(q')),  q' = q * c^K        (per run)
@@ -58,17 +59,15 @@ constexpr int kOffWz = kOffWl + 64;                  // [kWarps][4] zero-point s
 constexpr int kOffCw = kOffWz + 64;                  // [4 heads][kWarps] merge weights
 constexpr int kOffHead = kOffCw + 64;                // [4 heads] x (M, L, Z, -)
 constexpr int kDecodeSmem = kOffHead + 64;
-constexpr int kCombineSmem = (2 * ZC_MAX_ITEMS * ZC_MAX_G + 2 * ZC_MAX_G) * 4;
-constexpr int kMaxItems = ZC_MAX_ITEMS;              // partial (m, l) pairs staged in the ring
 
 __device__ int g_zc_error = 0;
 
 struct ItemDesc {
-  int kind;      // 0 = compressed run, 1 = tail
+  int kind;      // 0 = compressed run
   int cls, run;  // precision class, factor-block index
-  int sub_lo, sub_hi;  // absolute sub-tile range inside the class region (kind 1: sub_lo = tail item)
+  int sub_lo, sub_hi;  // absolute sub-tile range inside the class region
   int run_sub0;        // first sub-tile of the run
-  int n_tok;           // tokens of the run (kind 0) or of the tail (kind 1)
+  int n_tok;           // tokens of the run
 };
 
 __device__ inline ItemDesc decode_item(const ZcDecodePlan& p, int it) {
@@ -95,8 +94,8 @@ __device__ inline ItemDesc decode_item(const ZcDecodePlan& p, int it) {
     d.sub_hi = d.run_sub0 + (p.nw[k] + ZC_SUB - 1) / ZC_SUB;
     return d;
   }
-  d.kind = 1; d.cls = 0; d.run = 0; d.run_sub0 = 0;
-  d.sub_lo = i2 - 2 * (p.n_seg - 1); d.sub_hi = d.sub_lo; d.n_tok = p.n_tail;
+  // not reached for it < plan.items
+  d.kind = 1; d.cls = 0; d.run = 0; d.run_sub0 = 0; d.sub_lo = d.sub_hi = 0; d.n_tok = 0;
   return d;
 }
 
@@ -429,7 +428,15 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
   float* wz = reinterpret_cast<float*>(smem + kOffWz);
   const int n_pairs = (d.sub_hi - d.sub_lo + 1) >> 1;
   const int my_np = n_pairs > warp ? (n_pairs - warp + kWarps - 1) / kWarps : 0;
-  // ---- start the copies first: their latency covers the q' set-up ----
+  // ---- the few words the set-up needs go out first, ahead of this CTA's own 55 KB of copies ----
+  const float scale = kLog2e * rsqrtf((float)ZC_D);
+  const float cK = fac[tid];
+  const float cV = fac[ZC_D + tid];
+  const float smax = fac[2 * ZC_D];
+  float x[4];
+#pragma unroll
+  for (int h = 0; h < 4; ++h) x[h] = h < Gl ? zc_to_float<T>(qbase[h * ZC_D + tid]) : 0.f;
+  // ---- then the code copies: their latency covers the q' set-up ----
   if (lane == 0) {
     for (int s = 0; s < NST; ++s) mbar_init(&my_bar[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -441,16 +448,9 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
       bulk_copy_g2s(my_ring + s * PB, class_base + (long long)sn * SB, bytes, &my_bar[s]);
     }
   }
-  // everything this CTA needs from global memory besides the codes is requested now
-  const float cV = fac[ZC_D + tid];
-  const float smax = fac[2 * ZC_D];
   // ---- q' = q * c^K * log2(e)/sqrt(d); thread = channel ----
-  const float scale = kLog2e * rsqrtf((float)ZC_D);
-  const float cK = fac[tid];
-  float x[4];
 #pragma unroll
-  for (int h = 0; h < 4; ++h)
-    x[h] = h < Gl ? zc_to_float<T>(qbase[h * ZC_D + tid]) * cK * scale : 0.f;
+  for (int h = 0; h < 4; ++h) x[h] *= cK * scale;
   {
     const float ax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
     const unsigned mb = __reduce_max_sync(kFull, __float_as_uint(ax));
@@ -533,38 +533,29 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
   *rowscale = (tid & 8) ? 1048576.f : 16777216.f;
 }
 
-// Up to 64 tokens of the full-precision tail, 16 per warp, on tensor cores in the input
-// type: S^T = K_tail q^T with q exact in its own type, then O^T = V_tail^T P^T with
-// P = hi + lo in the input type (columns 0..3 and 4..7).
+// Sixteen tokens of the full-precision tail for one warp and up to four query heads, on tensor
+// cores in the input type: S^T = K_tail q^T with q exact in its own type, then
+// O^T = V_tail^T P^T with P = hi + lo in the input type (columns 0..3 and 4..7).
+// Results: wm / wl [warp][4] (row maximum, sum), mbuf [4 heads][128] for this warp, and the
+// logits (base 2) of the tokens into stash [4 heads][ZC_MAX_WINDOW].
 template <typename T>
-__device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, const ZcLayout& lay,
-                                          const T* qbase, int Gl, int unit, int h0, char* smem,
-                                          const T* k_new, const T* v_new) {
+__device__ __forceinline__ void tail_tile(const char* ub, const ZcLayout& lay, int n_tail, int base,
+                                          const T* qbase, int Gl, int unit, float* wm, float* wl,
+                                          float* mbuf, float* stash, const T* k_new, const T* v_new) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  float* wm = reinterpret_cast<float*>(smem + kOffWm);
-  float* wl = reinterpret_cast<float*>(smem + kOffWl);
-  float* wz = reinterpret_cast<float*>(smem + kOffWz);
-  float* mbuf = reinterpret_cast<float*>(smem + warp * kWarpRing);   // [4 heads][128]
-  const int base = d.sub_lo * (kWarps * ZC_SUB) + warp * ZC_SUB;
-  const int nv = min(ZC_SUB, d.n_tok - base);
+  const int nv = min(ZC_SUB, n_tail - base);
   if (nv <= 0) {
-    if (lane < 4) { wm[warp * 4 + lane] = -INFINITY; wl[warp * 4 + lane] = 0.f; wz[warp * 4 + lane] = 0.f; }
+    if (lane < 4) { wm[warp * 4 + lane] = -INFINITY; wl[warp * 4 + lane] = 0.f; }
     for (int i = lane; i < 4 * ZC_D; i += 32) mbuf[i] = 0.f;
     return;
   }
-  T* tK = reinterpret_cast<T*>(const_cast<char*>(ub) + lay.off_tailK);
-  T* tV = reinterpret_cast<T*>(const_cast<char*>(ub) + lay.off_tailV);
-  const int last = d.n_tok - 1;
-  // Deferred append: the newest row still lives in the caller's k_new / v_new [unit][128].
-  // It is read from there, and the warp whose 16 tokens include it stores it into the tail.
+  const T* tK = reinterpret_cast<const T*>(ub + lay.off_tailK);
+  const T* tV = reinterpret_cast<const T*>(ub + lay.off_tailV);
+  const int last = n_tail - 1;
+  // Deferred append: the newest row is read from the caller's k_new / v_new [unit][128] (the
+  // items kernel stores it into the tail).
   const T* newK = k_new ? k_new + (long long)unit * ZC_D : nullptr;
   const T* newV = v_new ? v_new + (long long)unit * ZC_D : nullptr;
-  if (newK && last >= base && last < base + ZC_SUB) {
-    if (lane < 16)
-      reinterpret_cast<uint4*>(tK + last * ZC_D)[lane] = reinterpret_cast<const uint4*>(newK)[lane];
-    else
-      reinterpret_cast<uint4*>(tV + last * ZC_D)[lane - 16] = reinterpret_cast<const uint4*>(newV)[lane - 16];
-  }
   // rows past the end are read from the last valid row and masked
   const int r0 = min(base + g, last), r1 = min(base + g + 8, last);
   const int va_r = min(base + 2 * t, last), vb_r = min(base + 2 * t + 8, last);
@@ -611,11 +602,8 @@ __device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, con
     lg[1][e] = dacc[2 + e] * scale;
     const int h = 2 * t + e;
     if (t < 2 && h < Gl) {
-      // kept in shared memory: the scratch in global memory may still be read by the previous
-      // call's combine kernel until this kernel has passed its wait
-      float* stash = mbuf + 4 * ZC_D + h * ZC_SUB;
-      if (v0) stash[g] = lg[0][e];
-      if (v1) stash[g + 8] = lg[1][e];
+      if (v0) stash[h * ZC_MAX_WINDOW + base + g] = lg[0][e];
+      if (v1) stash[h * ZC_MAX_WINDOW + base + g + 8] = lg[1][e];
     }
     if (!v0) lg[0][e] = -INFINITY;
     if (!v1) lg[1][e] = -INFINITY;
@@ -676,7 +664,7 @@ __device__ __forceinline__ void tail_item(const ItemDesc& d, const char* ub, con
   if (t < 2) {
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      if (g == 0) { wm[warp * 4 + 2 * t + e] = mx[e]; wl[warp * 4 + 2 * t + e] = ls[e]; wz[warp * 4 + 2 * t + e] = 0.f; }
+      if (g == 0) { wm[warp * 4 + 2 * t + e] = mx[e]; wl[warp * 4 + 2 * t + e] = ls[e]; }
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         mbuf[(2 * t + e) * ZC_D + 16 * g + 2 * i] = oacc[i][e];
@@ -690,41 +678,49 @@ template <typename T>
 __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, ZcLayout lay,
                                                                   ZcDecodePlan plan,
                                                                   const T* __restrict__ q, float* part,
-                                                                  float* tail_logits, const T* k_new,
-                                                                  const T* v_new) {
+                                                                  const T* k_new, const T* v_new) {
   extern __shared__ __align__(128) char smem[];
   float* wm = reinterpret_cast<float*>(smem + kOffWm);
   float* wl = reinterpret_cast<float*>(smem + kOffWl);
   float* wz = reinterpret_cast<float*>(smem + kOffWz);
   float* s_cw = reinterpret_cast<float*>(smem + kOffCw);
   float* s_head = reinterpret_cast<float*>(smem + kOffHead);
-  pdl_launch_dependents();
   const int unit = blockIdx.y, it = blockIdx.x;
+  char* ub = zc_unit_base(cache, lay, unit);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (k_new && it == 0 && blockIdx.z == 0) {
+    // Deferred append: the first item of every unit stores the newest row into the tail and
+    // makes it visible BEFORE it lets the next kernels start: later steps read that row ahead
+    // of their own wait.  Nothing reads row n_tail - 1 of the tail buffer during this step.
+    if (warp == 0) {
+      const int pos = plan.n_tail - 1;
+      T* tk = reinterpret_cast<T*>(ub + lay.off_tailK) + pos * ZC_D;
+      T* tv = reinterpret_cast<T*>(ub + lay.off_tailV) + pos * ZC_D;
+      if (lane < 16)
+        reinterpret_cast<uint4*>(tk)[lane] = reinterpret_cast<const uint4*>(k_new + (long long)unit * ZC_D)[lane];
+      else
+        reinterpret_cast<uint4*>(tv)[lane - 16] =
+            reinterpret_cast<const uint4*>(v_new + (long long)unit * ZC_D)[lane - 16];
+      __threadfence();
+    }
+    __syncthreads();
+  }
+  pdl_launch_dependents();
   const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
   const int h0 = 4 * blockIdx.z, Gl = min(4, G - h0);              // this CTA's query heads
   const ItemDesc d = decode_item(plan, it);
-  char* ub = zc_unit_base(cache, lay, unit);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const T* qbase = q + ((long long)b * lay.n_kv * G + kv * G + h0) * ZC_D;
   float* my = part + (((long long)unit * plan.items + it) * G + h0) * ZC_PART_STRIDE;
 
   float chan_factor = 1.f, rowscale = 1.f;
-  bool has = true;
-  if (d.kind == 0) {
-    has = d.sub_hi > d.sub_lo;
-    if (has) {
-      const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
-      const char* class_base = ub + lay.off_tiles[d.cls];
-      if (lay.bits[d.cls] == 4)
-        compressed_item<T, 4>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
-      else
-        compressed_item<T, 2>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
-    }
-  } else {
-    // the newest tail row comes from the append kernel just before this one, unless the
-    // append was deferred into this kernel
-    if (!k_new) pdl_wait();
-    tail_item<T>(d, ub, lay, qbase, Gl, unit, h0, smem, k_new, v_new);
+  const bool has = d.sub_hi > d.sub_lo;
+  if (has) {
+    const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
+    const char* class_base = ub + lay.off_tiles[d.cls];
+    if (lay.bits[d.cls] == 4)
+      compressed_item<T, 4>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
+    else
+      compressed_item<T, 2>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
   }
   __syncthreads();
   // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
@@ -746,18 +742,8 @@ __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, Z
     s_head[tid * 4 + 2] = has ? zs : 0.f;
   }
   __syncthreads();
-  // everything this CTA writes to global memory may still be in use by the previous kernel
+  // the partials go to scratch the previous call's combine kernel may still be reading
   pdl_wait();
-  if (d.kind == 1) {
-    const int base = d.sub_lo * (kWarps * ZC_SUB) + warp * ZC_SUB;
-    const int nv = min(ZC_SUB, d.n_tok - base);
-    const float* stash = reinterpret_cast<const float*>(smem + warp * kWarpRing) + 4 * ZC_D;
-    for (int e = lane; e < Gl * ZC_SUB; e += 32) {
-      const int h = e / ZC_SUB, tok = e % ZC_SUB;
-      if (tok < nv)
-        tail_logits[((long long)unit * G + h0 + h) * ZC_MAX_WINDOW + base + tok] = stash[h * ZC_SUB + tok];
-    }
-  }
   for (int h = 0; h < Gl; ++h) {
     float o = 0.f;
     if (has) {
@@ -774,23 +760,89 @@ __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, Z
   }
 }
 
-// Merge of the split-K partials: one CTA per unit, warp w owns heads w, w + 4.
+// shared-memory map of k_decode_combine
+constexpr int kCmbEntries = (ZC_MAX_ITEMS + 1) * ZC_MAX_G;       // items + the tail, per head
+constexpr int kCmbOffM = 0;                                       // [entries] maxima, then weights
+constexpr int kCmbOffL = kCmbOffM + kCmbEntries * 4;              // [entries] sums
+constexpr int kCmbOffML = kCmbOffL + kCmbEntries * 4;             // [G] x (M, L)
+constexpr int kCmbOffTail = kCmbOffML + 2 * ZC_MAX_G * 4;         // [G][ZC_PART_STRIDE] tail partial
+constexpr int kCmbOffStash = kCmbOffTail + ZC_MAX_G * ZC_PART_STRIDE * 4;   // [G][ZC_MAX_WINDOW] tail logits
+constexpr int kCmbOffWm = kCmbOffStash + ZC_MAX_G * ZC_MAX_WINDOW * 4;      // [kWarps][4] x (m, l)
+constexpr int kCmbOffMbuf = kCmbOffWm + 2 * kWarps * 4 * 4;       // [kWarps][4 heads][128]
+constexpr int kCombineSmem = kCmbOffMbuf + kWarps * 4 * ZC_D * 4;
+
+// Tail attention + merge of the split-K partials: one CTA per unit.  The tail (full-precision
+// rows, 16 tokens per warp and pass) needs nothing from the items kernel, so with a deferred
+// append it runs before the wait, while the items kernel streams the codes.
 template <typename T>
 __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout lay, ZcDecodePlan plan,
-                                                        T* __restrict__ out, const float* part,
-                                                        const float* tail_logits, int collect) {
+                                                        const T* __restrict__ q, T* __restrict__ out,
+                                                        const float* part, int collect,
+                                                        const T* k_new, const T* v_new) {
   extern __shared__ __align__(128) char smem[];
+  float* s_m = reinterpret_cast<float*>(smem + kCmbOffM);
+  float* s_l = reinterpret_cast<float*>(smem + kCmbOffL);
+  float* s_ML = reinterpret_cast<float*>(smem + kCmbOffML);
+  float* tailp = reinterpret_cast<float*>(smem + kCmbOffTail);
+  float* stash = reinterpret_cast<float*>(smem + kCmbOffStash);
+  float* twm = reinterpret_cast<float*>(smem + kCmbOffWm);
+  float* twl = twm + kWarps * 4;
   pdl_launch_dependents();
   const int unit = blockIdx.x;
   const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   char* ub = zc_unit_base(cache, lay, unit);
-  pdl_wait();   // the partials come from the kernel just before this one
+  const T* qunit = q + ((long long)b * lay.n_kv * G + kv * G) * ZC_D;
+  // without a deferred append the newest tail row comes from the append kernel, which is
+  // complete once the items kernel is
+  if (!k_new) pdl_wait();
+  // ---- tail: per group of four heads, passes of 64 tokens; thread = channel keeps the running
+  //      (M, L, O) of its heads in registers across passes ----
+  const int n_tail = plan.n_tail;
+  for (int hg = 0; hg * 4 < G; ++hg) {
+    const int Gl = min(4, G - 4 * hg);
+    float Mr[4], Lr[4], Or[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) { Mr[h] = -INFINITY; Lr[h] = 0.f; Or[h] = 0.f; }
+    for (int base0 = 0; base0 < n_tail; base0 += kWarps * ZC_SUB) {
+      float* mbuf = reinterpret_cast<float*>(smem + kCmbOffMbuf) + warp * 4 * ZC_D;
+      tail_tile<T>(ub, lay, n_tail, base0 + warp * ZC_SUB, qunit + 4 * hg * ZC_D, Gl, unit, twm, twl, mbuf,
+                   stash + 4 * hg * ZC_MAX_WINDOW, k_new, v_new);
+      __syncthreads();
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        if (h < Gl) {
+          float mn = Mr[h];
+#pragma unroll
+          for (int w2 = 0; w2 < kWarps; ++w2) mn = fmaxf(mn, twm[w2 * 4 + h]);
+          const float c_old = Mr[h] == -INFINITY ? 0.f : zc_exp2(Mr[h] - mn);
+          float o = Or[h] * c_old, l = Lr[h] * c_old;
+#pragma unroll
+          for (int w2 = 0; w2 < kWarps; ++w2) {
+            const float mw = twm[w2 * 4 + h];
+            if (mw != -INFINITY) {
+              const float cw = zc_exp2(mw - mn);
+              l += twl[w2 * 4 + h] * cw;
+              o += reinterpret_cast<const float*>(smem + kCmbOffMbuf)[(w2 * 4 + h) * ZC_D + tid] * cw;
+            }
+          }
+          Mr[h] = mn; Lr[h] = l; Or[h] = o;
+        }
+      }
+      __syncthreads();
+    }
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+      if (h < Gl) {
+        float* tp = tailp + (4 * hg + h) * ZC_PART_STRIDE;
+        if (tid == 0) { tp[0] = Mr[h]; tp[1] = Lr[h]; }
+        tp[4 + tid] = Or[h];
+      }
+    }
+  }
+  if (k_new) pdl_wait();   // the partials come from the items kernel just before this one
   const int items = plan.items;
   const float* mine = part + (long long)unit * items * G * ZC_PART_STRIDE;
-  float* s_m = reinterpret_cast<float*>(smem);          // [items * G] maxima, then weights
-  float* s_l = s_m + kMaxItems * ZC_MAX_G;              // [items * G] sums
-  float* s_ML = s_l + kMaxItems * ZC_MAX_G;             // [G] x (M, L)
   for (int e = tid; e < items * G; e += 128) {
     const float2 ml = __ldcg(reinterpret_cast<const float2*>(mine + (long long)e * ZC_PART_STRIDE));
     s_m[e] = ml.x;
@@ -806,7 +858,13 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
       if (u < n_first)
         acc4[u] = __ldcg(reinterpret_cast<const float4*>(mine + (long long)(u * G + warp) * ZC_PART_STRIDE + 4) + lane);
   }
+  __syncthreads();   // s_m / s_l and the tail partial are in place
+  if (tid < G) {     // the tail is one more entry, merged last
+    s_m[items * G + tid] = tailp[tid * ZC_PART_STRIDE];
+    s_l[items * G + tid] = tailp[tid * ZC_PART_STRIDE + 1];
+  }
   __syncthreads();
+  const int entries = items + 1;
   for (int h = warp; h < G; h += kWarps) {
     if (h != warp) {
 #pragma unroll
@@ -815,11 +873,11 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
           acc4[u] = __ldcg(reinterpret_cast<const float4*>(mine + (long long)(u * G + h) * ZC_PART_STRIDE + 4) + lane);
     }
     float mxh = -INFINITY;
-    for (int i = lane; i < items; i += 32) mxh = fmaxf(mxh, s_m[i * G + h]);
+    for (int i = lane; i < entries; i += 32) mxh = fmaxf(mxh, s_m[i * G + h]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mxh = fmaxf(mxh, __shfl_xor_sync(kFull, mxh, o));
     float lsum = 0.f;
-    for (int i = lane; i < items; i += 32) {
+    for (int i = lane; i < entries; i += 32) {
       const float mi = s_m[i * G + h];
       const float sc = mi == -INFINITY ? 0.f : zc_exp2(mi - mxh);
       s_m[i * G + h] = sc;
@@ -842,6 +900,11 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
       const float sc = s_m[i * G + h];
       o4.x += a.x * sc; o4.y += a.y * sc; o4.z += a.z * sc; o4.w += a.w * sc;
     }
+    {
+      const float4 a = *reinterpret_cast<const float4*>(tailp + h * ZC_PART_STRIDE + 4 + 4 * lane);
+      const float sc = s_m[items * G + h];
+      o4.x += a.x * sc; o4.y += a.y * sc; o4.z += a.z * sc; o4.w += a.w * sc;
+    }
     const float inv = 1.f / lsum;
     T r[4] = {zc_from_float<T>(o4.x * inv), zc_from_float<T>(o4.y * inv), zc_from_float<T>(o4.z * inv),
               zc_from_float<T>(o4.w * inv)};
@@ -850,11 +913,9 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
   }
   if (collect) {
     __syncthreads();
-    if (tid < plan.n_tail) {
+    if (tid < n_tail) {
       float a = 0.f;
-      for (int h = 0; h < G; ++h)
-        a += zc_exp2(__ldcg(tail_logits + ((long long)unit * G + h) * ZC_MAX_WINDOW + tid) - s_ML[2 * h]) /
-             s_ML[2 * h + 1];
+      for (int h = 0; h < G; ++h) a += zc_exp2(stash[h * ZC_MAX_WINDOW + tid] - s_ML[2 * h]) / s_ML[2 * h + 1];
       float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
       colsum[tid] += a;
     }
@@ -906,7 +967,6 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
                      float* ws, const void* k_new, const void* v_new, cudaStream_t st) {
   const int G = c->lay.G;
   float* part = ws;
-  float* tail_logits = ws + (size_t)c->lay.units * plan.items * G * ZC_PART_STRIDE;
   dim3 grid(plan.items, c->lay.units, (G + 3) / 4);
   const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
   const char* q_lo = (const char*)q;
@@ -927,21 +987,22 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
                              kDecodeSmem);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_items<__half>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay,
-                   plan, (const __half*)q, part, tail_logits, (const __half*)k_new, (const __half*)v_new);
+                   plan, (const __half*)q, part, (const __half*)k_new, (const __half*)v_new);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_combine<__half>, cgrid, dim3(128), kCombineSmem, st, true, c->base, c->lay,
-                   plan, (__half*)out, (const float*)part, (const float*)tail_logits, collect);
+                   plan, (const __half*)q, (__half*)out, (const float*)part, collect,
+                   (const __half*)k_new, (const __half*)v_new);
   } else {
     e = cudaFuncSetAttribute(k_decode_items<__nv_bfloat16>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_items<__nv_bfloat16>, grid, dim3(128), kDecodeSmem, st, overlap, c->base,
-                   c->lay, plan, (const __nv_bfloat16*)q, part, tail_logits, (const __nv_bfloat16*)k_new,
+                   c->lay, plan, (const __nv_bfloat16*)q, part, (const __nv_bfloat16*)k_new,
                    (const __nv_bfloat16*)v_new);
     if (e != cudaSuccess) return e;
     e = launch_pdl(k_decode_combine<__nv_bfloat16>, cgrid, dim3(128), kCombineSmem, st, true, c->base,
-                   c->lay, plan, (__nv_bfloat16*)out, (const float*)part, (const float*)tail_logits,
-                   collect);
+                   c->lay, plan, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, (const float*)part, collect,
+                   (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new);
   }
   g_last_out_lo = (const char*)out;
   g_last_out_hi = (const char*)out + io_bytes;

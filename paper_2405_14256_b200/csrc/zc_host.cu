@@ -149,8 +149,8 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   // the GPU (slots = SMs x resident CTAs), and the fixed set-up and merge of every CTA, worth
   // about ZC_ITEM_OVERHEAD sub-tiles of streaming.  Each candidate item size is scored by
   // (share of the slot-time its waves use) x (share of a CTA's life spent streaming).
-  p.tail_items = zc_ceil_div(c->n_tail, ZC_TAIL_ITEM_TOKENS);
-  const int extras = p.tail_items + 2 * (c->n_seg - 1);
+  p.tail_items = 0;   // the tail is handled by the combine kernel
+  const int extras = 2 * (c->n_seg - 1);
   const int slots = c->n_sm * ZC_DECODE_CTAS_PER_SM;
   const int zs = zc_ceil_div(c->lay.G, 4);
   const int cap = std::max(1, (ZC_MAX_ITEMS - extras) / 2);
@@ -177,7 +177,7 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
       for (int k = 0; k < 2; ++k) { p.spi0[k] = spi[k]; p.split0[k] = split[k]; }
     }
   }
-  p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1) + p.tail_items;
+  p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1);
   return p;
 }
 
@@ -391,10 +391,9 @@ int zc_decode_attention_noalloc(zc_cache* c, const void* q, void* out, int is_pr
                                 zc_stream_t stream) {
   if (!c || !q || !out) return ZC_EINVAL;
   if (c->l0 < 0) return ZC_ESTATE;
-  // what this call will really write: partials [unit][item][G][ZC_PART_STRIDE] + tail logits
+  // what this call will really write: partials [unit][item][G][ZC_PART_STRIDE]
   const ZcDecodePlan plan = zc_make_plan(c);
-  const size_t need = ((size_t)c->lay.units * plan.items * c->lay.G * ZC_PART_STRIDE +
-                       (size_t)c->lay.units * c->lay.G * ZC_MAX_WINDOW) * 4;
+  const size_t need = (size_t)c->lay.units * plan.items * c->lay.G * ZC_PART_STRIDE * 4;
   if (need > (size_t)ZC_NOALLOC_SCRATCH_BYTES) return ZC_ESCRATCH;
   void* scratch = nullptr;
   ZC_CUDA(zc_static_scratch(&scratch));   // first call per device: a synchronous address query

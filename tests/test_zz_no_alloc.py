@@ -51,8 +51,8 @@ def test_noalloc_entry_matches_workspace_entry_two_calls_in_a_row(kw):
 
 def test_noalloc_entry_rejects_shapes_beyond_its_buffer():
     import paper_2405_14256_b200 as zc
-    # 64 x 32 heads: the split-K partials of one call alone exceed the 4 MiB buffer
-    w = tl.small_workload(context=64, batch=64, n_q_heads=32, n_kv_heads=32, window=8)
+    # 128 x 32 heads: the split-K partials of one call alone exceed the 4 MiB buffer
+    w = tl.small_workload(context=64, batch=128, n_q_heads=32, n_kv_heads=32, window=8)
     big = tl.make_cache(w, max_new=64)
     Q, K, V = make_prefill(w, 0, tl.DEV)
     big.prefill_compress(Q, K, V, tl.probes_for(w).tolist())
