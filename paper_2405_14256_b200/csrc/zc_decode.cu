@@ -31,12 +31,11 @@ namespace {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxStages = 5;              // ring depth per warp: 3 pairs at 4 bits, 5 at 2 bits
 constexpr int kWarps = 4;
-#ifndef ZC_WARP_RING
-#define ZC_WARP_RING 13824
-#endif
-constexpr int kWarpRing = ZC_WARP_RING;    // 13824 = 3 x 4608 (4-bit pair) >= 5 x 2560 (2-bit pair)
-constexpr int kRingBytes = kWarps * kWarpRing;               // 55296
-constexpr int kCtasPerSm = ZC_DECODE_CTAS_PER_SM;
+// Two builds of the items kernel: 3 CTAs per SM with a 13824-byte ring per warp (3 pairs in
+// flight at 4 bits, 5 at 2 bits) for calls whose CTAs fit one or two waves, and 4 CTAs per SM
+// with a 9216-byte ring (2 / 3 pairs) for calls of many waves, where more resident warps hide
+// the set-up and merge of their neighbours.
+constexpr int kRingWide = 13824, kRingNarrow = 9216;
 constexpr int kWaitLimit = 1 << 22;
 #ifndef ZC_KPEXP
 #define ZC_KPEXP 12
@@ -49,8 +48,8 @@ constexpr int kPExp = ZC_KPEXP;      // softmax weights go to f16 as p * s^V * 2
 constexpr float kTau = ZC_TAU;   // the running maximum is refreshed only when a logit exceeds it by this
 constexpr unsigned kFull = 0xffffffffu;
 
-// shared-memory map of k_decode
-constexpr int kOffBars = kRingBytes;                 // kWarps * kMaxStages mbarriers
+// shared-memory map of k_decode_items: small arrays first, then the warps' rings
+constexpr int kOffBars = 0;                          // kWarps * kMaxStages mbarriers
 constexpr int kOffQfrag = kOffBars + 256;            // q' B-fragments, 4 x 32 x uint4
 constexpr int kOffRed = kOffQfrag + 2048;            // [kWarps] |q'| maxima as bits
 constexpr int kOffWm = kOffRed + 64;                 // [kWarps][4] running maxima
@@ -58,7 +57,8 @@ constexpr int kOffWl = kOffWm + 64;                  // [kWarps][4] sums
 constexpr int kOffWz = kOffWl + 64;                  // [kWarps][4] zero-point sums
 constexpr int kOffCw = kOffWz + 64;                  // [4 heads][kWarps] merge weights
 constexpr int kOffHead = kOffCw + 64;                // [4 heads] x (M, L, Z, -)
-constexpr int kDecodeSmem = kOffHead + 64;
+constexpr int kOffRing = kOffHead + 128;             // kWarps rings
+constexpr int decode_smem(int ring) { return kOffRing + kWarps * ring; }
 
 __device__ int g_zc_error = 0;
 
@@ -350,7 +350,7 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
 // Compressed-run part of one item, one warp: prologue done by the CTA, stages primed.  The
 // first my_np - NST iterations refill their stage and need no end-of-run handling; the last
 // NST do not refill and the very last pair may be cut short by the end of the run.
-template <int BITS>
+template <int BITS, int RING>
 __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_base, char* my_ring,
                                           uint64_t* my_bar, const uint32_t (&qb)[16], float qs,
                                           float isc, float logK, int my_np, int warp, int lane,
@@ -358,7 +358,7 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
                                           float& z_out, int* err) {
   constexpr int SB = ZC_SUB * (32 * BITS + 16);
   constexpr int PB = 2 * SB;
-  constexpr int NST = kWarpRing / PB;
+  constexpr int NST = RING / PB;
   const int g = lane >> 2, t = lane & 3;
   const bool odd_tok = BITS == 2 && (g & 1);
   const float logKs = logK - (odd_tok ? 2.f : 0.f);      // weights of odd tokens carry 1/4 at 2 bits
@@ -411,15 +411,15 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
 // One compressed item, whole CTA.  On return every warp has put its (m, l, z-sum) and its
 // accumulators into shared memory; *chan_factor / *rowscale tell the merge how to bring a
 // channel's accumulator to true units.
-template <typename T, int BITS>
+template <typename T, int BITS, int RING>
 __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* class_base,
                                                 const float* fac, const T* qbase, int Gl, char* smem,
                                                 float* chan_factor, float* rowscale, int* err) {
   constexpr int SB = ZC_SUB * (32 * BITS + 16);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   constexpr int PB = 2 * SB;
-  constexpr int NST = kWarpRing / PB;
-  char* my_ring = smem + warp * kWarpRing;
+  constexpr int NST = RING / PB;
+  char* my_ring = smem + kOffRing + warp * RING;
   uint64_t* my_bar = reinterpret_cast<uint64_t*>(smem + kOffBars) + warp * kMaxStages;
   uint4* qfrag = reinterpret_cast<uint4*>(smem + kOffQfrag);
   unsigned* s_red = reinterpret_cast<unsigned*>(smem + kOffRed);
@@ -508,7 +508,7 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
 #pragma unroll
     for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
   float m, l, z;
-  run_pairs<BITS>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
+  run_pairs<BITS, RING>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
 #pragma unroll
   for (int o = 4; o < 32; o <<= 1) {
     l += __shfl_xor_sync(kFull, l, o);
@@ -674,8 +674,8 @@ __device__ __forceinline__ void tail_tile(const char* ub, const ZcLayout& lay, i
   }
 }
 
-template <typename T>
-__global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, ZcLayout lay,
+template <typename T, int RING, int NCTA>
+__global__ void __launch_bounds__(128, NCTA) k_decode_items(char* cache, ZcLayout lay,
                                                                   ZcDecodePlan plan,
                                                                   const T* __restrict__ q, float* part,
                                                                   const T* k_new, const T* v_new) {
@@ -718,9 +718,9 @@ __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, Z
     const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
     const char* class_base = ub + lay.off_tiles[d.cls];
     if (lay.bits[d.cls] == 4)
-      compressed_item<T, 4>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
+      compressed_item<T, 4, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
     else
-      compressed_item<T, 2>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
+      compressed_item<T, 2, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
   }
   __syncthreads();
   // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
@@ -748,10 +748,10 @@ __global__ void __launch_bounds__(128, kCtasPerSm) k_decode_items(char* cache, Z
     float o = 0.f;
     if (has) {
       const float4 cw = *reinterpret_cast<const float4*>(s_cw + h * 4);
-      const float a0 = reinterpret_cast<const float*>(smem)[h * ZC_D + tid];
-      const float a1 = reinterpret_cast<const float*>(smem + kWarpRing)[h * ZC_D + tid];
-      const float a2 = reinterpret_cast<const float*>(smem + 2 * kWarpRing)[h * ZC_D + tid];
-      const float a3 = reinterpret_cast<const float*>(smem + 3 * kWarpRing)[h * ZC_D + tid];
+      const float a0 = reinterpret_cast<const float*>(smem + kOffRing)[h * ZC_D + tid];
+      const float a1 = reinterpret_cast<const float*>(smem + kOffRing + RING)[h * ZC_D + tid];
+      const float a2 = reinterpret_cast<const float*>(smem + kOffRing + 2 * RING)[h * ZC_D + tid];
+      const float a3 = reinterpret_cast<const float*>(smem + kOffRing + 3 * RING)[h * ZC_D + tid];
       o = (rowscale * (((cw.x * a0 + cw.y * a1) + cw.z * a2) + cw.w * a3) - s_head[h * 4 + 2]) * chan_factor;
     }
     float* dst = my + h * ZC_PART_STRIDE;
@@ -982,28 +982,26 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   }
   const dim3 cgrid(c->lay.units);
   cudaError_t e;
+#define ZC_LAUNCH_STEP(T, RING, NCTA)                                                              \
+  do {                                                                                             \
+    e = cudaFuncSetAttribute(k_decode_items<T, RING, NCTA>,                                        \
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));      \
+    if (e != cudaSuccess) return e;                                                                \
+    e = launch_pdl(k_decode_items<T, RING, NCTA>, grid, dim3(128), decode_smem(RING), st, overlap, \
+                   c->base, c->lay, plan, (const T*)q, part, (const T*)k_new, (const T*)v_new);    \
+    if (e != cudaSuccess) return e;                                                                \
+    e = launch_pdl(k_decode_combine<T>, cgrid, dim3(128), kCombineSmem, st, true, c->base, c->lay, \
+                   plan, (const T*)q, (T*)out, (const float*)part, collect, (const T*)k_new,       \
+                   (const T*)v_new);                                                               \
+  } while (0)
   if (c->cfg.dtype == ZC_F16) {
-    e = cudaFuncSetAttribute(k_decode_items<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kDecodeSmem);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(k_decode_items<__half>, grid, dim3(128), kDecodeSmem, st, overlap, c->base, c->lay,
-                   plan, (const __half*)q, part, (const __half*)k_new, (const __half*)v_new);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(k_decode_combine<__half>, cgrid, dim3(128), kCombineSmem, st, true, c->base, c->lay,
-                   plan, (const __half*)q, (__half*)out, (const float*)part, collect,
-                   (const __half*)k_new, (const __half*)v_new);
+    if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(__half, kRingNarrow, 4);
+    else ZC_LAUNCH_STEP(__half, kRingWide, 3);
   } else {
-    e = cudaFuncSetAttribute(k_decode_items<__nv_bfloat16>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(k_decode_items<__nv_bfloat16>, grid, dim3(128), kDecodeSmem, st, overlap, c->base,
-                   c->lay, plan, (const __nv_bfloat16*)q, part, (const __nv_bfloat16*)k_new,
-                   (const __nv_bfloat16*)v_new);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(k_decode_combine<__nv_bfloat16>, cgrid, dim3(128), kCombineSmem, st, true, c->base,
-                   c->lay, plan, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, (const float*)part, collect,
-                   (const __nv_bfloat16*)k_new, (const __nv_bfloat16*)v_new);
+    if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(__nv_bfloat16, kRingNarrow, 4);
+    else ZC_LAUNCH_STEP(__nv_bfloat16, kRingWide, 3);
   }
+#undef ZC_LAUNCH_STEP
   g_last_out_lo = (const char*)out;
   g_last_out_hi = (const char*)out + io_bytes;
   c->launches += 2;

@@ -84,8 +84,7 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
     size_t pre = align_up((size_t)np_max * 4, 256) +
                  (size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4;
     // decode: partials [unit][item][G][ZC_PART_STRIDE] + tail logits [unit][G][window]
-    const int max_items = std::min(ZC_MAX_ITEMS, 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush +
-                                                     zc_ceil_div(ZC_MAX_WINDOW, ZC_TAIL_ITEM_TOKENS));
+    const int max_items = std::min(ZC_MAX_ITEMS, 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush);
     size_t dec = (size_t)lay->units * max_items * lay->G * ZC_PART_STRIDE * 4 +
                  (size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4 + 256;
     *ws_bytes = align_up(std::max(pre, dec), 256);
@@ -148,35 +147,42 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   // How finely to cut segment 0.  Two things cost time: CTAs that do not fill a whole wave of
   // the GPU (slots = SMs x resident CTAs), and the fixed set-up and merge of every CTA, worth
   // about ZC_ITEM_OVERHEAD sub-tiles of streaming.  Each candidate item size is scored by
-  // (share of the slot-time its waves use) x (share of a CTA's life spent streaming).
-  p.tail_items = 0;   // the tail is handled by the combine kernel
+  // (share of the slot-time its waves use) x (share of a CTA's life spent streaming).  Calls
+  // of many waves use the build with 4 CTAs per SM.
   const int extras = 2 * (c->n_seg - 1);
-  const int slots = c->n_sm * ZC_DECODE_CTAS_PER_SM;
   const int zs = zc_ceil_div(c->lay.G, 4);
   const int cap = std::max(1, (ZC_MAX_ITEMS - extras) / 2);
   int subs[2];
   for (int k = 0; k < 2; ++k) subs[k] = std::max(1, zc_ceil_div(c->n0[k], ZC_SUB));
   static const int kCand[] = {256, 192, 128, 96, 64, 48, 32};
-  double best = -1.0;
-  for (int target : kCand) {
-    int spi[2], split[2];
-    for (int k = 0; k < 2; ++k) {
-      const int want = std::min(std::min(zc_ceil_div(subs[k], target), std::min(ZC_MAX_SPLIT_HOST, cap)),
-                                subs[k]);
-      // an even number of sub-tiles per item: the kernel consumes them in pairs
-      spi[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;
-      split[k] = zc_ceil_div(subs[k], spi[k]);
+  auto choose = [&](int per_sm) -> double {
+    const int slots = c->n_sm * per_sm;
+    double best = -1.0, best_ctas = 0.0;
+    for (int target : kCand) {
+      int spi[2], split[2];
+      for (int k = 0; k < 2; ++k) {
+        const int want = std::min(std::min(zc_ceil_div(subs[k], target), std::min(ZC_MAX_SPLIT_HOST, cap)),
+                                  subs[k]);
+        // an even number of sub-tiles per item: the kernel consumes them in pairs
+        spi[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;
+        split[k] = zc_ceil_div(subs[k], spi[k]);
+      }
+      const double n_ctas = (double)(split[0] + split[1] + extras) * c->lay.units * zs;
+      const double waves = n_ctas / slots;
+      const double fill = n_ctas / (ceil(waves) * slots);
+      const double per_item = (double)(subs[0] + subs[1]) / (split[0] + split[1]);
+      const double score = fill * per_item / (per_item + ZC_ITEM_OVERHEAD);
+      if (score > best) {
+        best = score;
+        best_ctas = n_ctas;
+        for (int k = 0; k < 2; ++k) { p.spi0[k] = spi[k]; p.split0[k] = split[k]; }
+      }
     }
-    const double n_ctas = (double)(split[0] + split[1] + extras) * c->lay.units * zs;
-    const double waves = n_ctas / slots;
-    const double fill = n_ctas / (ceil(waves) * slots);
-    const double per_item = (double)(subs[0] + subs[1]) / (split[0] + split[1]);
-    const double score = fill * per_item / (per_item + ZC_ITEM_OVERHEAD);
-    if (score > best) {
-      best = score;
-      for (int k = 0; k < 2; ++k) { p.spi0[k] = spi[k]; p.split0[k] = split[k]; }
-    }
-  }
+    return best_ctas;
+  };
+  p.ctas_per_sm = 3;
+  if (choose(4) >= ZC_MANY_WAVES * c->n_sm * 4) p.ctas_per_sm = 4;
+  else choose(3);
   p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1);
   return p;
 }

@@ -17,8 +17,8 @@
 #ifndef ZC_ITEM_OVERHEAD
 #define ZC_ITEM_OVERHEAD 24       // fixed cost of one split-K item, in 16-token sub-tiles of streaming
 #endif
-#ifndef ZC_DECODE_CTAS_PER_SM
-#define ZC_DECODE_CTAS_PER_SM 3
+#ifndef ZC_MANY_WAVES
+#define ZC_MANY_WAVES 1.2          // from this many waves of 4-per-SM CTAs on, the narrow build is used
 #endif    // CTAs the decode kernel keeps resident per SM
 
 // Device-side description of the cache buffer.  One "unit" = (batch, KV head).
@@ -71,7 +71,7 @@ struct ZcDecodePlan {
   int split0[2];           // items covering segment 0, per class
   int spi0[2];             // 16-token sub-tiles per item, per class
   int n_tail;
-  int tail_items;          // items covering the tail (64 tokens each)
+  int ctas_per_sm;         // build of the items kernel: 3 (wide rings) or 4 (narrow rings)
   int items;               // items per unit
   int l0;
 };
@@ -118,7 +118,6 @@ int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out,
                      int collect, float* ws, const void* k_new, const void* v_new,
                      cudaStream_t st);
-#define ZC_TAIL_ITEM_TOKENS 64
 int zc_device_error_code(int* out);
 // Device address of the built-in scratch buffer on the current device (looked up once per device).
 int zc_static_scratch(void** ptr);
