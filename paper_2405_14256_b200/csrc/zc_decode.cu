@@ -41,6 +41,9 @@ constexpr int kWaitLimit = 1 << 22;
 #define ZC_KPEXP 12
 #define ZC_TAU 3.5f
 #endif
+#ifndef ZC_QK_CHAINS
+#define ZC_QK_CHAINS 1
+#endif
 #ifndef ZC_SHIFT_ON_FMA
 #define ZC_SHIFT_ON_FMA 0
 #endif
@@ -254,6 +257,12 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     float dacc[4];
+#if ZC_QK_CHAINS == 2
+    float dacc2[4];
+#define ZC_SECOND dacc2
+#else
+#define ZC_SECOND dacc
+#endif
     if (BITS == 4) {
 #pragma unroll
       for (int jw = 0; jw < 4; ++jw) {
@@ -263,7 +272,8 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
         else zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
         const uint32_t x0 = shr8(w0), x1 = shr8(w1);
         const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
-        zc_mma16816<__half>(dacc, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
+        if (ZC_QK_CHAINS == 2 && jw == 0) zc_mma16816_z(ZC_SECOND, a1, qb[2], qb[3]);
+        else zc_mma16816<__half>(ZC_SECOND, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
       }
     } else {
 #pragma unroll
@@ -277,10 +287,16 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
           if (ks == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
           else zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
           const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
-          zc_mma16816<__half>(dacc, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
+          if (ZC_QK_CHAINS == 2 && ks == 0) zc_mma16816_z(ZC_SECOND, a1, qb[2], qb[3]);
+          else zc_mma16816<__half>(ZC_SECOND, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
         }
       }
     }
+#if ZC_QK_CHAINS == 2
+#pragma unroll
+    for (int e = 0; e < 4; ++e) dacc[e] += dacc2[e];
+#endif
+#undef ZC_SECOND
     // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
     u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
     u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;

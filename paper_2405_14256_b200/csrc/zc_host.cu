@@ -154,7 +154,7 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   const int cap = std::max(1, (ZC_MAX_ITEMS - extras) / 2);
   int subs[2];
   for (int k = 0; k < 2; ++k) subs[k] = std::max(1, zc_ceil_div(c->n0[k], ZC_SUB));
-  static const int kCand[] = {256, 192, 128, 96, 64, 48, 32};
+  static const int kCand[] = {256, 192, 128, 96, 80, 64, 56, 48, 40, 32};
   auto choose = [&](int per_sm) -> double {
     const int slots = c->n_sm * per_sm;
     double best = -1.0, best_ctas = 0.0;
@@ -169,7 +169,9 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
       }
       const double n_ctas = (double)(split[0] + split[1] + extras) * c->lay.units * zs;
       const double waves = n_ctas / slots;
-      const double fill = n_ctas / (ceil(waves) * slots);
+      // a handful of CTAs beyond a whole wave start as soon as the first ones retire
+      const double whole = std::max(1.0, (waves - floor(waves) <= ZC_WAVE_SLACK) ? floor(waves) : ceil(waves));
+      const double fill = std::min(1.0, n_ctas / (whole * slots));
       const double per_item = (double)(subs[0] + subs[1]) / (split[0] + split[1]);
       const double score = fill * per_item / (per_item + ZC_ITEM_OVERHEAD);
       if (score > best) {

@@ -17,6 +17,9 @@
 #ifndef ZC_ITEM_OVERHEAD
 #define ZC_ITEM_OVERHEAD 24       // fixed cost of one split-K item, in 16-token sub-tiles of streaming
 #endif
+#ifndef ZC_WAVE_SLACK
+#define ZC_WAVE_SLACK 0.0         // share of a wave that may spill over without counting as one more
+#endif
 #ifndef ZC_MANY_WAVES
 #define ZC_MANY_WAVES 1.2          // from this many waves of 4-per-SM CTAs on, the narrow build is used
 #endif    // CTAs the decode kernel keeps resident per SM
