@@ -449,14 +449,13 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
   const float cK = fac[tid];
   const float cV = fac[ZC_D + tid];
   const float smax = fac[2 * ZC_D];
-  float x[4];
+  T qraw[4];   // used only after the copies below are on their way
 #pragma unroll
-  for (int h = 0; h < 4; ++h) x[h] = h < Gl ? zc_to_float<T>(qbase[h * ZC_D + tid]) : 0.f;
+  for (int h = 0; h < 4; ++h) qraw[h] = qbase[(h < Gl ? h : 0) * ZC_D + tid];
   // ---- then the code copies: their latency covers the q' set-up ----
   if (lane == 0) {
     for (int s = 0; s < NST; ++s) mbar_init(&my_bar[s], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");   // init visible to the copy engine
     for (int s = 0; s < NST && s < my_np; ++s) {
       const int sn = d.sub_lo + 2 * (warp + s * kWarps);
       const int bytes = sn + 1 < d.sub_hi ? PB : SB;
@@ -465,8 +464,9 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
     }
   }
   // ---- q' = q * c^K * log2(e)/sqrt(d); thread = channel ----
+  float x[4];
 #pragma unroll
-  for (int h = 0; h < 4; ++h) x[h] *= cK * scale;
+  for (int h = 0; h < 4; ++h) x[h] = h < Gl ? zc_to_float<T>(qraw[h]) * cK * scale : 0.f;
   {
     const float ax = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
     const unsigned mb = __reduce_max_sync(kFull, __float_as_uint(ax));
@@ -501,7 +501,7 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
     qb[4 * q4] = v.x; qb[4 * q4 + 1] = v.y; qb[4 * q4 + 2] = v.z; qb[4 * q4 + 3] = v.w;
   }
   // sum of q' exactly as the f16 operands represent it: one MMA pass against all-one codes
-  float ds[4] = {0.f, 0.f, 0.f, 0.f};
+  float ds[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) {
     uint32_t one_lo, one_hi;
@@ -509,9 +509,9 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
     else if ((ks & 1) == 0) { one_lo = 0x00010001u; one_hi = 0x00040004u; }
     else { one_lo = 0x00100010u; one_hi = 0x00400040u; }
     const uint32_t a[4] = {one_lo, one_lo, one_hi, one_hi};
-    zc_mma16816<__half>(ds, a, qb[2 * ks], qb[2 * ks + 1]);
+    zc_mma16816<__half>(ds[ks & 1], a, qb[2 * ks], qb[2 * ks + 1]);
   }
-  const float qs = ds[0] + ds[1];
+  const float qs = (ds[0][0] + ds[1][0]) + (ds[0][1] + ds[1][1]);
   // accumulator * 2^24 / CTA scale = q' . code
   const float isc = 16777216.f * (scaled ? __uint_as_float((ex_q - 13u) << 23) : 1.f);
   // weights are scaled by 2^logK = 2^kPExp / 2^ceil(log2 smax) so that w <= 2^(kPExp + kTau)
