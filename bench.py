@@ -106,8 +106,9 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# DRAM bytes per decode call measured once with ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload id; the summaries are under profiles/.
+# DRAM bytes of one k_decode_items launch measured with ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum), keyed by workload id; the capture and its conditions are in
+# profiles/k_decode_items_config2.md.
 PROFILED_DRAM_BYTES_PER_DECODE_CALL = {}
 
 
@@ -133,7 +134,9 @@ def oracle_sample(w, n_units: int, n_steps: int, layer: int = 0):
     from oracle import zipcache_oracle as zo
     from workloads import make_prefill, make_decode_step, decode_probe_flags
     Q, K, V = make_prefill(w, layer, "cpu")
-    units = [(i % w.batch, (i * 3) % w.n_kv_heads) for i in range(n_units)]
+    every = [(b, kv) for b in range(w.batch) for kv in range(w.n_kv_heads)]
+    order = np.random.RandomState(1234).permutation(len(every))
+    units = [every[j] for j in order[: min(n_units, len(every))]]
     f64 = lambda t: t.to(torch.float64).numpy()
     Qh, Kh, Vh = f64(Q), f64(K), f64(V)
     P = zo.probe_positions(w.context, w.rho_recent, w.rho_random, w.seed(layer))
@@ -191,7 +194,7 @@ def run_reference(args):
     sample = ""
     for i in range(args.warmup + args.steps):
         t0 = time.perf_counter()
-        gbs, tps, secs, threads, sample = oracle_sample(w, 2, 4)
+        gbs, tps, secs, threads, sample = oracle_sample(w, 16, 32)
         if i >= args.warmup:
             vals.append(gbs)
             times.append(time.perf_counter() - t0)
@@ -393,7 +396,8 @@ def main():
         "pct_of_hbm_peak": 100.0 * achieved / peak,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                     "kernel": "decode attention (items + combine) incl. append",
+                     "kernel": "k_decode_items (+ k_decode_combine of the same call: decode phase "
+                               "time / decode calls; consecutive calls overlap)",
                      "bytes_per_launch": dec_bytes / n_decode_calls,
                      "us_per_launch": per_call_us},
         "clocks": clocks,
@@ -403,7 +407,7 @@ def main():
     if e2e is not None:
         line["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
-        gbs, tps, secs, threads, sample = oracle_sample(w, 4, 8)
+        gbs, tps, secs, threads, sample = oracle_sample(w, 64, 96)
         line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": sample, "prefill_tokens_per_s": tps, "seconds": secs}
     print(json.dumps(line))

@@ -1000,9 +1000,15 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   cudaError_t e;
 #define ZC_LAUNCH_STEP(T, RING, NCTA)                                                              \
   do {                                                                                             \
-    e = cudaFuncSetAttribute(k_decode_items<T, RING, NCTA>,                                        \
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));      \
-    if (e != cudaSuccess) return e;                                                                \
+    static int attr_dev = -1; /* the opt-in to large shared memory is per device */                \
+    int dev_now = 0;                                                                               \
+    cudaGetDevice(&dev_now);                                                                       \
+    if (attr_dev != dev_now) {                                                                     \
+      e = cudaFuncSetAttribute(k_decode_items<T, RING, NCTA>,                                      \
+                               cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));    \
+      if (e != cudaSuccess) return e;                                                              \
+      attr_dev = dev_now;                                                                          \
+    }                                                                                              \
     e = launch_pdl(k_decode_items<T, RING, NCTA>, grid, dim3(128), decode_smem(RING), st, overlap, \
                    c->base, c->lay, plan, (const T*)q, part, (const T*)k_new, (const T*)v_new);    \
     if (e != cudaSuccess) return e;                                                                \
