@@ -106,10 +106,12 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# DRAM bytes of one k_decode_items launch measured with ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum), keyed by workload id; the capture and its conditions are in
-# profiles/k_decode_items_config2.md.
-PROFILED_DRAM_BYTES_PER_DECODE_CALL = {}
+# DRAM bytes of one decode-attention call measured with ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum of its k_decode_items launch plus its k_decode_combine launch where
+# that was captured), keyed by workload id. Captured with few tail tokens (the first decode
+# steps after a prefill); the commands are in profiles/k_decode_items_config2.md and
+# profiles/k_decode_items_config4.md.
+PROFILED_DRAM_BYTES_PER_DECODE_CALL = {2: 28.09e6 + 0.91e6, 4: 447.97e6 + 21.0e6}
 
 
 def algorithmic_decode_bytes(w, n_windows: int, n_tail: int) -> int:
