@@ -106,12 +106,10 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# DRAM bytes of one decode-attention call measured with ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum of its k_decode_items launch plus its k_decode_combine launch where
-# that was captured), keyed by workload id. Captured with few tail tokens (the first decode
-# steps after a prefill); the commands are in profiles/k_decode_items_config2.md and
-# profiles/k_decode_items_config4.md.
-PROFILED_DRAM_BYTES_PER_DECODE_CALL = {2: 28.09e6 + 0.91e6, 4: 447.97e6 + 21.0e6}
+# DRAM bytes of one k_decode launch (= one decode-attention call) measured with ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload id; the captures and their
+# conditions are in profiles/.  Empty entries: the kernel changed since the last capture.
+PROFILED_DRAM_BYTES_PER_DECODE_CALL = {}
 
 
 def algorithmic_decode_bytes(w, n_windows: int, n_tail: int) -> int:
@@ -223,6 +221,9 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--decode-steps", type=int, default=0,
                     help="profiling only: fewer decode steps than the workload's own")
+    ap.add_argument("--items", default="overlap", choices=["overlap", "single"],
+                    help="overlap: ZC_FLAG_OVERLAP_CALLS (the layers' calls share the GPU: few large "
+                         "work items); single: items sized for a call that has the GPU to itself")
     ap.add_argument("--append", default="deferred", choices=["deferred", "kernel"],
                     help="deferred: zc_append hands the new row to the next zc_decode_attention "
                          "(ZC_FLAG_DEFER_APPEND); kernel: zc_append copies with its own launch")
@@ -262,7 +263,8 @@ def main():
     workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)   # shared by all layers
     caches = [zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context, n_dec,
                           w.saliency_ratio, w.bits_hi, w.bits_lo, w.window, device=dev,
-                          workspace=workspace, defer_append=args.append == "deferred")
+                          workspace=workspace, defer_append=args.append == "deferred",
+                          overlap_calls=args.items == "overlap")
               for _ in range(R)]
     flags = [decode_probe_flags(w, ly, n_dec) for ly in layer_ids]
     # decode inputs: 4 distinct seeded sets per step, cycled over layers (fresh N(0,1) each)
@@ -390,6 +392,8 @@ def main():
                    "batch": w.batch, "context": w.context, "n_q_heads": w.n_q_heads,
                    "n_kv_heads": w.n_kv_heads, "decode_steps": n_dec, "bits": "4/2",
                    "saliency_ratio": w.saliency_ratio, "decode_phase": "CUDA graph replay",
+                   "items": ("ZC_FLAG_OVERLAP_CALLS: consecutive layers' calls run side by side"
+                             if args.items == "overlap" else "sized for one call at a time"),
                    "append": ("zc_append defers the copy into the next zc_decode_attention "
                               "(ZC_FLAG_DEFER_APPEND)" if args.append == "deferred"
                               else "zc_append launches its own copy kernel")},
@@ -398,8 +402,8 @@ def main():
         "pct_of_hbm_peak": 100.0 * achieved / peak,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                     "kernel": "k_decode_items (+ k_decode_combine of the same call: decode phase "
-                               "time / decode calls; consecutive calls overlap)",
+                     "kernel": "k_decode (one launch per call: decode phase time / decode calls; "
+                               "consecutive calls run side by side)",
                      "bytes_per_launch": dec_bytes / n_decode_calls,
                      "us_per_launch": per_call_us},
         "clocks": clocks,

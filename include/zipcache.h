@@ -56,6 +56,13 @@ enum {
  * stay valid and unchanged until the stream has passed that zc_decode_attention call.  Any
  * other call on the cache first performs the pending append as its own launch. */
 #define ZC_FLAG_DEFER_APPEND 1
+/* With ZC_FLAG_OVERLAP_CALLS the caller tells the library that decode calls on independent
+ * caches follow one another on the stream with nothing else between them (the layers of a
+ * benchmark, caches of different requests).  Consecutive zc_decode_attention calls always run
+ * side by side on the GPU where their buffers allow it; the flag only changes how a call is
+ * cut into work items: few large ones, which is best when several calls share the GPU and
+ * worst for a single call that has the GPU to itself. */
+#define ZC_FLAG_OVERLAP_CALLS 2
 
 /* Plain-data configuration; set struct_size = sizeof(zc_config). */
 typedef struct {
@@ -71,7 +78,7 @@ typedef struct {
                              (Alg. 3 uses 100); 8 <= window <= ZC_MAX_WINDOW */
   int32_t bits_hi;        /* bit-width of salient tokens: 4 or 2 */
   int32_t bits_lo;        /* bit-width of regular tokens: 4 or 2 */
-  int32_t flags;          /* 0 or ZC_FLAG_DEFER_APPEND */
+  int32_t flags;          /* 0 or an OR of ZC_FLAG_DEFER_APPEND, ZC_FLAG_OVERLAP_CALLS */
   double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
 } zc_config;
 
@@ -121,7 +128,14 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
  * The step counter of the current window advances; on a probe step (is_probe_step != 0,
  * or one of the last five steps of a window) this step's attention over the tail's
  * tokens is added to the window statistics; after the window's last step the tail is
- * re-compressed into a new segment (same stream, no host synchronisation). */
+ * re-compressed into a new segment (same stream, no host synchronisation).
+ * Ordering: consecutive calls on one stream may run at the same time on the GPU.  The library
+ * orders a call after the earlier ones whenever it reads or overwrites one of their outputs,
+ * overwrites one of their inputs, or updates the same cache's window statistics; it cannot see
+ * other aliasing, so q, k_new, v_new and out of calls issued back to back must not overlap
+ * buffers that an earlier call of the stream still uses in any other way.  Kernels of other
+ * libraries on the stream are ordered as usual.  The workspace must not be used by calls on
+ * another stream at the same time. */
 int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step,
                         void* workspace, size_t workspace_bytes, zc_stream_t stream);
 
@@ -160,9 +174,9 @@ int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t*
  *   - The first call on each device looks up the buffer's device address (a synchronous
  *     runtime query): make that first call outside any stream capture.
  *   - All calls share the one buffer, whatever cache they work on.  Calls that follow one
- *     another in ONE stream are ordered by the library; calls in different streams, or from
- *     several host threads, that may run at the same time on the GPU overwrite each other's
- *     partial results.  Nothing in the buffer has to survive between calls and nothing in it
+ *     another in ONE stream get separate parts of it or are ordered by the library; calls in
+ *     different streams, or from several host threads, that may run at the same time on the
+ *     GPU overwrite each other's partial results.  Nothing in the buffer has to survive between calls and nothing in it
  *     has to be cleared: each call rewrites every word it later reads. */
 int zc_decode_attention_noalloc(zc_cache* c, const void* q, void* out, int is_probe_step,
                                 zc_stream_t stream);

@@ -13,6 +13,7 @@ LIB_PATH = os.path.join(HERE, "libzipcache.so")
 
 ZC_F16, ZC_BF16 = 0, 1
 ZC_FLAG_DEFER_APPEND = 1
+ZC_FLAG_OVERLAP_CALLS = 2
 
 
 class ZipCacheError(RuntimeError):
@@ -220,12 +221,14 @@ class ZipCache:
 
     def __init__(self, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
-                 workspace: Optional[torch.Tensor] = None, defer_append: bool = False):
+                 workspace: Optional[torch.Tensor] = None, defer_append: bool = False,
+                 overlap_calls: bool = False):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                                  saliency_ratio, bits_hi, bits_lo, window,
-                                 flags=ZC_FLAG_DEFER_APPEND if defer_append else 0)
+                                 flags=(ZC_FLAG_DEFER_APPEND if defer_append else 0) |
+                                 (ZC_FLAG_OVERLAP_CALLS if overlap_calls else 0))
         self.dtype, self.device = dtype, torch.device(device)
         self.batch, self.n_q_heads, self.n_kv_heads = batch, n_q_heads, n_kv_heads
         self.cache_bytes, self.workspace_bytes = zc_cache_bytes(self.cfg)

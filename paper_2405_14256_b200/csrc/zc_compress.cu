@@ -5,6 +5,32 @@
 
 namespace {
 
+// The kernels of a re-compression can be launched as links of the decode calls' chain
+// (programmatic dependent launch): each lets its successor start at once and itself waits for
+// its predecessor to complete, so the decode calls of other caches that follow on the stream
+// are not held up.  In an ordinary launch both instructions do nothing.
+__device__ __forceinline__ void chain_link() {
+  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+  asm volatile("griddepcontrol.wait;\n" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_link(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                        bool chained, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = chained ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+
 // ------------------------------------------------------------------ top-k split
 // One CTA per unit.  Keys are the bit patterns of the (non-negative) scores, so unsigned
 // integer order equals float order.  An MSB-first 8-bit radix select finds the n_s-th
@@ -42,6 +68,7 @@ __device__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
 __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayout lay, int n, int n_s,
                                                              int idx_off,
                                                              const int32_t* __restrict__ given) {
+  chain_link();
   __shared__ int hist[256];
   __shared__ int warp_sums[32];
   __shared__ int s_total;
@@ -132,6 +159,7 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayo
 struct NnzArgs { int v[ZC_MAX_WINDOW]; };
 
 __global__ void k_window_scores(char* cache, ZcLayout lay, NnzArgs nnz) {
+  chain_link();
   char* ub = zc_unit_base(cache, lay, blockIdx.x);
   float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
   float* scores = reinterpret_cast<float*>(ub + lay.off_scores);
@@ -146,6 +174,7 @@ __global__ void k_window_scores(char* cache, ZcLayout lay, NnzArgs nnz) {
 // grid.x: tiles of class 0 then tiles of class 1; grid.y: unit.  blockDim 256.
 template <typename T>
 __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
+  chain_link();
   __shared__ float red[2][8][ZC_D];
   const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
   const int tiles_c0 = zc_ceil_div(seg.n_tok[0], ZC_TILE);
@@ -188,6 +217,7 @@ __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout la
 }
 
 __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
+  chain_link();
   char* ub = zc_unit_base(cache, lay, blockIdx.x);
   unsigned* cmax = reinterpret_cast<unsigned*>(ub + lay.off_cmax);
   for (int i = threadIdx.x; i < 4 * ZC_D; i += blockDim.x) cmax[i] = 0u;
@@ -229,6 +259,7 @@ __device__ __forceinline__ void quant_token(const float (&x)[4], const float (&c
 
 template <typename T>
 __global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
+  chain_link();
   __shared__ __align__(16) unsigned char codesK[ZC_TILE][ZC_D];
   __shared__ __align__(16) unsigned char codesV[ZC_TILE][ZC_D];
   __shared__ __align__(16) float parK[ZC_TILE][2];
@@ -353,39 +384,43 @@ __global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay
 }  // namespace
 
 int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
-                   cudaStream_t st) {
+                   cudaStream_t st, bool chained) {
   const int smem = given_sal ? ((n + 31) / 32) * 4 : 0;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k_topk_split, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
-  k_topk_split<<<c->lay.units, kTopkThreads, smem, st>>>(c->base, c->lay, n, n_s, idx_off, given_sal);
+  cudaError_t e = launch_link(k_topk_split, dim3(c->lay.units), dim3(kTopkThreads), (size_t)smem, st, chained,
+                              c->base, c->lay, n, n_s, idx_off, given_sal);
   c->launches += 1;
-  return cudaGetLastError();
+  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 
-int zc_launch_window_scores(zc_cache* c, cudaStream_t st) {
+int zc_launch_window_scores(zc_cache* c, cudaStream_t st, bool chained) {
   NnzArgs a;
   for (int j = 0; j < ZC_MAX_WINDOW; ++j) a.v[j] = c->tail_nnz[j];
-  k_window_scores<<<c->lay.units, ZC_MAX_WINDOW, 0, st>>>(c->base, c->lay, a);
+  cudaError_t e = launch_link(k_window_scores, dim3(c->lay.units), dim3(ZC_MAX_WINDOW), 0, st, chained,
+                              c->base, c->lay, a);
   c->launches += 1;
-  return cudaGetLastError();
+  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 
-int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st) {
+int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st, bool chained) {
   const int tiles = zc_ceil_div(seg.n_tok[0], ZC_TILE) + zc_ceil_div(seg.n_tok[1], ZC_TILE);
-  k_clear_cmax<<<c->lay.units, 128, 0, st>>>(c->base, c->lay, seg);
+  cudaError_t e = launch_link(k_clear_cmax, dim3(c->lay.units), dim3(128), 0, st, chained, c->base, c->lay, seg);
   c->launches += 1;
-  if (tiles > 0) {
+  if (e == cudaSuccess && tiles > 0) {
     dim3 grid(tiles, c->lay.units);
     if (c->cfg.dtype == ZC_F16) {
-      k_channel_absmax<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
-      k_quantize_pack<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      e = launch_link(k_channel_absmax<__half>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
+      if (e == cudaSuccess)
+        e = launch_link(k_quantize_pack<__half>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
     } else {
-      k_channel_absmax<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
-      k_quantize_pack<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      e = launch_link(k_channel_absmax<__nv_bfloat16>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
+      if (e == cudaSuccess)
+        e = launch_link(k_quantize_pack<__nv_bfloat16>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
     }
     c->launches += 2;
   }
-  return cudaGetLastError();
+  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }

@@ -1,13 +1,15 @@
 // Append (Eq. 3) and single-query attention over the mixed-precision cache (Eq. 4, Alg. 3).
 //
 // Split-K: every unit's compressed cache is cut into items (a range of 16-token sub-tiles of
-// one precision class of one segment); one CTA per item produces a partial (m, l, acc) per
-// query head.  A small second kernel, one CTA per unit, computes the attention over the
-// full-precision tail on tensor cores while the items kernel is still streaming, then merges
-// everything in a fixed order, writes the output and, on probe steps, adds the step's attention
-// over the tail's tokens to the window statistics.  The kernels of one step (append, items,
-// combine) are chained by programmatic dependent launch: each may start while its predecessor
-// drains and orders itself with griddepcontrol.wait.  Nothing spins on another CTA.
+// one precision class of one segment); a CTA works through one or more items and stores a
+// partial (m, l, acc) per item and query head.  The attention over the full-precision tail runs
+// on tensor cores in the input type, in a CTA of its own or in the unit's first item CTA.  The
+// CTA of a unit that finishes last (an arrival counter tells) merges the unit's partials in a
+// fixed order, writes the output and, on probe steps, adds the step's attention over the
+// tail's tokens to the window statistics: one kernel per call, nothing spins on another CTA.
+// Consecutive calls on a stream are chained by programmatic dependent launch and run side by
+// side; what orders them where they touch the same memory is described at ZcOrder and at
+// zc_launch_decode.
 //
 // Dequantisation is folded so that it is never done per element:
 //   q . k_hat_t = s_t (q' . code_t - z_t sum(q')),  q' = q * c^K        (per run)
@@ -22,6 +24,7 @@
 // Each warp owns a ring of shared-memory stages filled by bulk asynchronous copies (one per
 // 16-token sub-block, completion on an mbarrier), so a CTA needs no block-wide barrier in
 // its main loop.  Every wait is bounded; a wait that runs out records an error code.
+#include <mutex>
 #include "zc_internal.h"
 #include "zc_layout.cuh"
 #include "zc_mma.cuh"
@@ -31,10 +34,10 @@ namespace {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kMaxStages = 5;              // ring depth per warp: 3 pairs at 4 bits, 5 at 2 bits
 constexpr int kWarps = 4;
-// Two builds of the items kernel: 3 CTAs per SM with a 13824-byte ring per warp (3 pairs in
-// flight at 4 bits, 5 at 2 bits) for calls whose CTAs fit one or two waves, and 4 CTAs per SM
-// with a 9216-byte ring (2 / 3 pairs) for calls of many waves, where more resident warps hide
-// the set-up and merge of their neighbours.
+// Two builds of the kernel: 3 CTAs per SM with a 13824-byte ring per warp (3 pairs in flight
+// at 4 bits, 5 at 2 bits) for calls whose CTAs fit one or two waves, and 4 CTAs per SM with a
+// 9216-byte ring (2 / 3 pairs) for calls of many waves and for calls that share the GPU with
+// their neighbours, where more resident warps hide the set-up and merge of the others.
 constexpr int kRingWide = 13824, kRingNarrow = 9216;
 constexpr int kWaitLimit = 1 << 22;
 #ifndef ZC_KPEXP
@@ -51,7 +54,7 @@ constexpr int kPExp = ZC_KPEXP;      // softmax weights go to f16 as p * s^V * 2
 constexpr float kTau = ZC_TAU;   // the running maximum is refreshed only when a logit exceeds it by this
 constexpr unsigned kFull = 0xffffffffu;
 
-// shared-memory map of k_decode_items: small arrays first, then the warps' rings
+// shared-memory map of an item CTA: small arrays first, then the warps' rings
 constexpr int kOffBars = 0;                          // kWarps * kMaxStages mbarriers
 constexpr int kOffQfrag = kOffBars + 256;            // q' B-fragments, 4 x 32 x uint4
 constexpr int kOffRed = kOffQfrag + 2048;            // [kWarps] |q'| maxima as bits
@@ -110,6 +113,47 @@ __device__ __forceinline__ void pdl_launch_dependents() {
 }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 
+// Ordering between decode calls that run side by side on a stream.  One word per stream,
+// (epoch tag << 20) | n, says that the first n calls of the epoch have completed; it is written
+// by one CTA per kernel after that kernel's predecessor has completed.  A call that must not
+// touch something before an earlier call of its epoch is done waits for the word to reach that
+// call's number.  The calls waited for are always resident or finished (a kernel starts only
+// after every CTA of its predecessor has started), so the wait ends; it is bounded all the same.
+struct ZcOrder {
+  unsigned* done;     // the stream's word
+  unsigned tag;       // epoch tag
+  int e;              // number of this call within its epoch
+  int need_start;     // calls that must have completed before this call reads its inputs
+  int need_end;       // ... before it writes partials, the output and the window statistics
+  int epoch_start;    // launched without early start: everything before it has completed
+};
+__device__ __forceinline__ unsigned ld_order(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.volatile.global.u32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ bool order_ok(unsigned v, unsigned tag, int need) {
+  return (v >> 20) == tag && (int)(v & 0xFFFFFu) >= need;
+}
+__device__ __noinline__ void order_wait_slow(const unsigned* p, unsigned tag, int need, int* err) {
+  if (*reinterpret_cast<volatile int*>(err) == 2) return;   // a wait already ran out: do not add to it
+  for (int spins = 0; spins < (1 << 20); ++spins) {
+    if (order_ok(ld_order(p), tag, need)) { __threadfence(); return; }
+    __nanosleep(256);
+  }
+  atomicExch(err, 2);
+}
+// acquire: the caller goes on to READ what the earlier call wrote (a fence orders those loads
+// behind the observation); stores and read-modify-writes issued afterwards need none.
+__device__ __forceinline__ void order_wait(const ZcOrder& o, unsigned first, int need, bool acquire, int* err) {
+  if (need <= 0) return;
+  if (order_ok(first, o.tag, need)) {
+    if (acquire) __threadfence();
+    return;
+  }
+  order_wait_slow(o.done, o.tag, need, err);
+}
+
 template <typename T>
 __global__ void k_append(char* cache, ZcLayout lay, const T* __restrict__ k_new,
                          const T* __restrict__ v_new, int pos) {
@@ -130,6 +174,9 @@ __global__ void k_append(char* cache, ZcLayout lay, const T* __restrict__ k_new,
 // ---- mbarrier / bulk-copy primitives ----
 __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(zc_smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_inval(uint64_t* bar) {
+  asm volatile("mbarrier.inval.shared::cta.b64 [%0];\n" ::"r"(zc_smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, int bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(zc_smem_u32(bar)),
@@ -525,6 +572,9 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
     for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
   float m, l, z;
   run_pairs<BITS, RING>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
+  __syncwarp();
+  if (lane == 0)   // every copy has landed and been consumed: retire the barriers
+    for (int s = 0; s < NST; ++s) mbar_inval(&my_bar[s]);
 #pragma unroll
   for (int o = 4; o < 32; o <<= 1) {
     l += __shfl_xor_sync(kFull, l, o);
@@ -555,7 +605,7 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
 // Results: wm / wl [warp][4] (row maximum, sum), mbuf [4 heads][128] for this warp, and the
 // logits (base 2) of the tokens into stash [4 heads][ZC_MAX_WINDOW].
 template <typename T>
-__device__ __forceinline__ void tail_tile(const char* ub, const ZcLayout& lay, int n_tail, int base,
+__device__ __forceinline__ void tail_tile(const T* tK, const T* tV, int n_tail, int base,
                                           const T* qbase, int Gl, int unit, float* wm, float* wl,
                                           float* mbuf, float* stash, const T* k_new, const T* v_new) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
@@ -565,11 +615,9 @@ __device__ __forceinline__ void tail_tile(const char* ub, const ZcLayout& lay, i
     for (int i = lane; i < 4 * ZC_D; i += 32) mbuf[i] = 0.f;
     return;
   }
-  const T* tK = reinterpret_cast<const T*>(ub + lay.off_tailK);
-  const T* tV = reinterpret_cast<const T*>(ub + lay.off_tailV);
   const int last = n_tail - 1;
   // Deferred append: the newest row is read from the caller's k_new / v_new [unit][128] (the
-  // items kernel stores it into the tail).
+  // unit's first item CTA stores it into the tail).
   const T* newK = k_new ? k_new + (long long)unit * ZC_D : nullptr;
   const T* newV = v_new ? v_new + (long long)unit * ZC_D : nullptr;
   // rows past the end are read from the last valid row and masked
@@ -584,8 +632,8 @@ __device__ __forceinline__ void tail_tile(const char* ub, const ZcLayout& lay, i
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     qv[c] = g < Gl ? *reinterpret_cast<const uint4*>(qbase + g * ZC_D + 32 * c + 8 * t) : make_uint4(0, 0, 0, 0);
-    ka[c] = *reinterpret_cast<const uint4*>(k0p + 32 * c + 8 * t);
-    kb[c] = *reinterpret_cast<const uint4*>(k1p + 32 * c + 8 * t);
+    ka[c] = __ldcg(reinterpret_cast<const uint4*>(k0p + 32 * c + 8 * t));
+    kb[c] = __ldcg(reinterpret_cast<const uint4*>(k1p + 32 * c + 8 * t));
   }
   // V: this lane's 16 channels (16g .. 16g+15) of the four tokens its fragments pair up
   const T* vap = vrow(va_r);
@@ -595,10 +643,10 @@ __device__ __forceinline__ void tail_tile(const char* ub, const ZcLayout& lay, i
   uint4 va[2], vb[2], vc[2], vd[2];
 #pragma unroll
   for (int u = 0; u < 2; ++u) {
-    va[u] = *reinterpret_cast<const uint4*>(vap + 16 * g + 8 * u);
-    vb[u] = *reinterpret_cast<const uint4*>(vbp + 16 * g + 8 * u);
-    vc[u] = *reinterpret_cast<const uint4*>(vcp + 16 * g + 8 * u);
-    vd[u] = *reinterpret_cast<const uint4*>(vdp + 16 * g + 8 * u);
+    va[u] = __ldcg(reinterpret_cast<const uint4*>(vap + 16 * g + 8 * u));
+    vb[u] = __ldcg(reinterpret_cast<const uint4*>(vbp + 16 * g + 8 * u));
+    vc[u] = __ldcg(reinterpret_cast<const uint4*>(vcp + 16 * g + 8 * u));
+    vd[u] = __ldcg(reinterpret_cast<const uint4*>(vdp + 16 * g + 8 * u));
   }
   // ---- S^T: k-step (c, pp) contracts channels 32c + 8t + 4pp + {0,1 | 2,3} ----
   float dacc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -690,131 +738,32 @@ __device__ __forceinline__ void tail_tile(const char* ub, const ZcLayout& lay, i
   }
 }
 
-template <typename T, int RING, int NCTA>
-__global__ void __launch_bounds__(128, NCTA) k_decode_items(char* cache, ZcLayout lay,
-                                                                  ZcDecodePlan plan,
-                                                                  const T* __restrict__ q, float* part,
-                                                                  const T* k_new, const T* v_new) {
-  extern __shared__ __align__(128) char smem[];
-  float* wm = reinterpret_cast<float*>(smem + kOffWm);
-  float* wl = reinterpret_cast<float*>(smem + kOffWl);
-  float* wz = reinterpret_cast<float*>(smem + kOffWz);
-  float* s_cw = reinterpret_cast<float*>(smem + kOffCw);
-  float* s_head = reinterpret_cast<float*>(smem + kOffHead);
-  const int unit = blockIdx.y, it = blockIdx.x;
-  char* ub = zc_unit_base(cache, lay, unit);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  if (k_new && it == 0 && blockIdx.z == 0) {
-    // Deferred append: the first item of every unit stores the newest row into the tail and
-    // makes it visible BEFORE it lets the next kernels start: later steps read that row ahead
-    // of their own wait.  Nothing reads row n_tail - 1 of the tail buffer during this step.
-    if (warp == 0) {
-      const int pos = plan.n_tail - 1;
-      T* tk = reinterpret_cast<T*>(ub + lay.off_tailK) + pos * ZC_D;
-      T* tv = reinterpret_cast<T*>(ub + lay.off_tailV) + pos * ZC_D;
-      if (lane < 16)
-        reinterpret_cast<uint4*>(tk)[lane] = reinterpret_cast<const uint4*>(k_new + (long long)unit * ZC_D)[lane];
-      else
-        reinterpret_cast<uint4*>(tv)[lane - 16] =
-            reinterpret_cast<const uint4*>(v_new + (long long)unit * ZC_D)[lane - 16];
-      __threadfence();
-    }
-    __syncthreads();
-  }
-  pdl_launch_dependents();
-  const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
-  const int h0 = 4 * blockIdx.z, Gl = min(4, G - h0);              // this CTA's query heads
-  const ItemDesc d = decode_item(plan, it);
-  const T* qbase = q + ((long long)b * lay.n_kv * G + kv * G + h0) * ZC_D;
-  float* my = part + (((long long)unit * plan.items + it) * G + h0) * ZC_PART_STRIDE;
-
-  float chan_factor = 1.f, rowscale = 1.f;
-  const bool has = d.sub_hi > d.sub_lo;
-  if (has) {
-    const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
-    const char* class_base = ub + lay.off_tiles[d.cls];
-    if (lay.bits[d.cls] == 4)
-      compressed_item<T, 4, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
-    else
-      compressed_item<T, 2, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
-  }
-  __syncthreads();
-  // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
-  if (tid < 4) {
-    float ms = -INFINITY;
-#pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) ms = fmaxf(ms, wm[w2 * 4 + tid]);
-    float ls = 0.f, zs = 0.f;
-#pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) {
-      const float mw = wm[w2 * 4 + tid];
-      const float cw = (has && mw != -INFINITY) ? zc_exp2(mw - ms) : 0.f;
-      s_cw[tid * 4 + w2] = cw;
-      ls += wl[w2 * 4 + tid] * cw;
-      zs += wz[w2 * 4 + tid] * cw;
-    }
-    s_head[tid * 4] = has ? ms : -INFINITY;
-    s_head[tid * 4 + 1] = has ? ls : 0.f;
-    s_head[tid * 4 + 2] = has ? zs : 0.f;
-  }
-  __syncthreads();
-  // the partials go to scratch the previous call's combine kernel may still be reading
-  pdl_wait();
-  for (int h = 0; h < Gl; ++h) {
-    float o = 0.f;
-    if (has) {
-      const float4 cw = *reinterpret_cast<const float4*>(s_cw + h * 4);
-      const float a0 = reinterpret_cast<const float*>(smem + kOffRing)[h * ZC_D + tid];
-      const float a1 = reinterpret_cast<const float*>(smem + kOffRing + RING)[h * ZC_D + tid];
-      const float a2 = reinterpret_cast<const float*>(smem + kOffRing + 2 * RING)[h * ZC_D + tid];
-      const float a3 = reinterpret_cast<const float*>(smem + kOffRing + 3 * RING)[h * ZC_D + tid];
-      o = (rowscale * (((cw.x * a0 + cw.y * a1) + cw.z * a2) + cw.w * a3) - s_head[h * 4 + 2]) * chan_factor;
-    }
-    float* dst = my + h * ZC_PART_STRIDE;
-    if (tid == 0) { dst[0] = s_head[h * 4]; dst[1] = s_head[h * 4 + 1]; }
-    dst[4 + tid] = o;
-  }
-}
-
-// shared-memory map of k_decode_combine
+// shared-memory map of the tail and merge phases (they reuse the memory of the item phase)
 constexpr int kCmbEntries = (ZC_MAX_ITEMS + 1) * ZC_MAX_G;       // items + the tail, per head
-constexpr int kCmbOffM = 0;                                       // [entries] maxima, then weights
+// The map starts behind the mbarriers: memory that holds mbarrier objects is never reused as
+// data (plain stores over a used barrier were observed to be replaced by barrier state).
+constexpr int kCmbOffM = kOffQfrag;                               // [entries] maxima, then weights
 constexpr int kCmbOffL = kCmbOffM + kCmbEntries * 4;              // [entries] sums
 constexpr int kCmbOffML = kCmbOffL + kCmbEntries * 4;             // [G] x (M, L)
-constexpr int kCmbOffTail = kCmbOffML + 2 * ZC_MAX_G * 4;         // [G][ZC_PART_STRIDE] tail partial
-constexpr int kCmbOffStash = kCmbOffTail + ZC_MAX_G * ZC_PART_STRIDE * 4;   // [G][ZC_MAX_WINDOW] tail logits
+constexpr int kCmbOffStash = kCmbOffML + 2 * ZC_MAX_G * 4;        // [G][ZC_MAX_WINDOW] tail logits
 constexpr int kCmbOffWm = kCmbOffStash + ZC_MAX_G * ZC_MAX_WINDOW * 4;      // [kWarps][4] x (m, l)
 constexpr int kCmbOffMbuf = kCmbOffWm + 2 * kWarps * 4 * 4;       // [kWarps][4 heads][128]
-constexpr int kCombineSmem = kCmbOffMbuf + kWarps * 4 * ZC_D * 4;
+constexpr int kCmbOffFlag = kCmbOffMbuf + kWarps * 4 * ZC_D * 4;  // "this CTA arrived last"
+constexpr int kCombineSmem = kCmbOffFlag + 16;
+static_assert(kCombineSmem <= decode_smem(kRingNarrow), "tail and merge phases must fit the item phase's memory");
 
-// Tail attention + merge of the split-K partials: one CTA per unit.  The tail (full-precision
-// rows, 16 tokens per warp and pass) needs nothing from the items kernel, so with a deferred
-// append it runs before the wait, while the items kernel streams the codes.
+// Attention over the full-precision tail, whole CTA, all query heads of the unit: passes of 64
+// tokens (16 per warp); thread = channel keeps the running (M, L, O) of its heads in registers
+// across passes.  The result goes out as one more split-K partial, the logits (base 2) to
+// stash_g [G][ZC_MAX_WINDOW] when the step collects probe statistics.
 template <typename T>
-__global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout lay, ZcDecodePlan plan,
-                                                        const T* __restrict__ q, T* __restrict__ out,
-                                                        const float* part, int collect,
-                                                        const T* k_new, const T* v_new) {
-  extern __shared__ __align__(128) char smem[];
-  float* s_m = reinterpret_cast<float*>(smem + kCmbOffM);
-  float* s_l = reinterpret_cast<float*>(smem + kCmbOffL);
-  float* s_ML = reinterpret_cast<float*>(smem + kCmbOffML);
-  float* tailp = reinterpret_cast<float*>(smem + kCmbOffTail);
+__device__ __noinline__ void tail_phase(const T* tK, const T* tV, int G, int n_tail, const T* qunit, int unit,
+                                        char* smem, float* part_tail, float* stash_g, const T* k_new,
+                                        const T* v_new, ZcOrder ord, unsigned ord_first, int* err) {
   float* stash = reinterpret_cast<float*>(smem + kCmbOffStash);
   float* twm = reinterpret_cast<float*>(smem + kCmbOffWm);
   float* twl = twm + kWarps * 4;
-  pdl_launch_dependents();
-  const int unit = blockIdx.x;
-  const int b = unit / lay.n_kv, kv = unit % lay.n_kv, G = lay.G;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  char* ub = zc_unit_base(cache, lay, unit);
-  const T* qunit = q + ((long long)b * lay.n_kv * G + kv * G) * ZC_D;
-  // without a deferred append the newest tail row comes from the append kernel, which is
-  // complete once the items kernel is
-  if (!k_new) pdl_wait();
-  // ---- tail: per group of four heads, passes of 64 tokens; thread = channel keeps the running
-  //      (M, L, O) of its heads in registers across passes ----
-  const int n_tail = plan.n_tail;
+  const int tid = threadIdx.x, warp = tid >> 5;
   for (int hg = 0; hg * 4 < G; ++hg) {
     const int Gl = min(4, G - 4 * hg);
     float Mr[4], Lr[4], Or[4];
@@ -822,7 +771,7 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
     for (int h = 0; h < 4; ++h) { Mr[h] = -INFINITY; Lr[h] = 0.f; Or[h] = 0.f; }
     for (int base0 = 0; base0 < n_tail; base0 += kWarps * ZC_SUB) {
       float* mbuf = reinterpret_cast<float*>(smem + kCmbOffMbuf) + warp * 4 * ZC_D;
-      tail_tile<T>(ub, lay, n_tail, base0 + warp * ZC_SUB, qunit + 4 * hg * ZC_D, Gl, unit, twm, twl, mbuf,
+      tail_tile<T>(tK, tV, n_tail, base0 + warp * ZC_SUB, qunit + 4 * hg * ZC_D, Gl, unit, twm, twl, mbuf,
                    stash + 4 * hg * ZC_MAX_WINDOW, k_new, v_new);
       __syncthreads();
 #pragma unroll
@@ -847,19 +796,34 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
       }
       __syncthreads();
     }
+    if (hg == 0) order_wait(ord, ord_first, ord.need_end, false, err);   // the workspace region is free
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
       if (h < Gl) {
-        float* tp = tailp + (4 * hg + h) * ZC_PART_STRIDE;
+        float* tp = part_tail + (4 * hg + h) * ZC_PART_STRIDE;
         if (tid == 0) { tp[0] = Mr[h]; tp[1] = Lr[h]; }
         tp[4 + tid] = Or[h];
       }
     }
   }
-  if (k_new) pdl_wait();   // the partials come from the items kernel just before this one
-  const int items = plan.items;
-  const float* mine = part + (long long)unit * items * G * ZC_PART_STRIDE;
-  for (int e = tid; e < items * G; e += 128) {
+  if (stash_g) {
+    for (int i = tid; i < G * ZC_MAX_WINDOW; i += 128)
+      if ((i & (ZC_MAX_WINDOW - 1)) < n_tail) stash_g[i] = stash[i];
+  }
+}
+
+// Merge of a unit's split-K partials (items, then the tail as the last entry) in a fixed order,
+// the output row of every query head and, on probe steps, this step's attention over the
+// tail's tokens added to the window statistics.  Run by the CTA of the unit that finished last.
+template <typename T>
+__device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_tail, T* __restrict__ out_unit,
+                                        const float* mine, const float* stash_g, int collect, char* smem) {
+  float* s_m = reinterpret_cast<float*>(smem + kCmbOffM);
+  float* s_l = reinterpret_cast<float*>(smem + kCmbOffL);
+  float* s_ML = reinterpret_cast<float*>(smem + kCmbOffML);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int entries = items + 1;
+  for (int e = tid; e < entries * G; e += 128) {
     const float2 ml = __ldcg(reinterpret_cast<const float2*>(mine + (long long)e * ZC_PART_STRIDE));
     s_m[e] = ml.x;
     s_l[e] = ml.y;
@@ -867,20 +831,14 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
   // each warp owns heads warp, warp + 4: its first rows are requested before the barrier
   constexpr int kChunk = 12;
   float4 acc4[kChunk];
-  const int n_first = min(items, kChunk);
+  const int n_first = min(entries, kChunk);
   if (warp < G) {
 #pragma unroll
     for (int u = 0; u < kChunk; ++u)
       if (u < n_first)
         acc4[u] = __ldcg(reinterpret_cast<const float4*>(mine + (long long)(u * G + warp) * ZC_PART_STRIDE + 4) + lane);
   }
-  __syncthreads();   // s_m / s_l and the tail partial are in place
-  if (tid < G) {     // the tail is one more entry, merged last
-    s_m[items * G + tid] = tailp[tid * ZC_PART_STRIDE];
-    s_l[items * G + tid] = tailp[tid * ZC_PART_STRIDE + 1];
-  }
   __syncthreads();
-  const int entries = items + 1;
   for (int h = warp; h < G; h += kWarps) {
     if (h != warp) {
 #pragma unroll
@@ -911,31 +869,189 @@ __global__ void __launch_bounds__(128) k_decode_combine(char* cache, ZcLayout la
         o4.x += acc4[u].x * sc; o4.y += acc4[u].y * sc; o4.z += acc4[u].z * sc; o4.w += acc4[u].w * sc;
       }
     }
-    for (int i = kChunk; i < items; ++i) {
+    for (int i = kChunk; i < entries; ++i) {
       const float4 a = __ldcg(reinterpret_cast<const float4*>(mine + (long long)(i * G + h) * ZC_PART_STRIDE + 4) + lane);
       const float sc = s_m[i * G + h];
-      o4.x += a.x * sc; o4.y += a.y * sc; o4.z += a.z * sc; o4.w += a.w * sc;
-    }
-    {
-      const float4 a = *reinterpret_cast<const float4*>(tailp + h * ZC_PART_STRIDE + 4 + 4 * lane);
-      const float sc = s_m[items * G + h];
       o4.x += a.x * sc; o4.y += a.y * sc; o4.z += a.z * sc; o4.w += a.w * sc;
     }
     const float inv = 1.f / lsum;
     T r[4] = {zc_from_float<T>(o4.x * inv), zc_from_float<T>(o4.y * inv), zc_from_float<T>(o4.z * inv),
               zc_from_float<T>(o4.w * inv)};
-    *reinterpret_cast<uint2*>(out + ((long long)b * lay.n_kv * G + kv * G + h) * ZC_D + 4 * lane) =
-        *reinterpret_cast<const uint2*>(r);
+    *reinterpret_cast<uint2*>(out_unit + h * ZC_D + 4 * lane) = *reinterpret_cast<const uint2*>(r);
   }
   if (collect) {
     __syncthreads();
     if (tid < n_tail) {
       float a = 0.f;
-      for (int h = 0; h < G; ++h) a += zc_exp2(stash[h * ZC_MAX_WINDOW + tid] - s_ML[2 * h]) / s_ML[2 * h + 1];
-      float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
+      for (int h = 0; h < G; ++h)
+        a += zc_exp2(__ldcg(stash_g + h * ZC_MAX_WINDOW + tid) - s_ML[2 * h]) / s_ML[2 * h + 1];
       colsum[tid] += a;
     }
   }
+}
+
+// One decode-attention call as ONE grid.  CTA roles, by linear index: for every unit
+// block 0 only waits; then for every unit (items x head groups) item CTAs and one tail CTA.
+//   item     streams its range of sub-tiles and stores a partial per query head
+//   tail     attention over the full-precision tail, stored as the unit's last partial (with
+//            plan.fold_tail there is no such CTA: the unit's first item CTA does it first)
+//   either   counts itself in at the unit's arrival counter; the CTA that arrives last merges
+//            the unit's partials and writes the output.  Nothing spins on another CTA.
+// Every CTA lets the next kernel of the stream start at once and none of the working CTAs
+// waits for the previous kernel, so calls on independent caches stream through the GPU like
+// one grid; block 0 does nothing but wait for the previous kernel, which
+// makes kernels complete in stream order (a launch made without early start then finds every
+// earlier call finished) at the price of one idle CTA.  What calls in flight together may
+// share is kept apart by the host: each call of an epoch (the launches between two launches
+// made without early start) gets its own `slot`, which selects its region of the workspace
+// and its arrival counter.
+template <typename T, int RING, int NCTA>
+__global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay, ZcDecodePlan plan,
+                                                      const T* __restrict__ q, T* __restrict__ out,
+                                                      float* part, float* stash_all, int slot,
+                                                      int collect, const T* k_new, const T* v_new,
+                                                      ZcOrder ord) {
+  extern __shared__ __align__(128) char smem[];
+  const int G = lay.G, zs = (G + 3) >> 2;
+  const int groups = (plan.items + plan.cta_items - 1) / plan.cta_items;   // item CTAs per head group
+  const int per_unit = groups * zs + (plan.fold_tail ? 0 : 1);
+  // Block 0 is the CTA that only waits: it is dispatched first, so it holds a slot even when
+  // the rest of a large grid is waiting for what it is going to publish.
+  const int idx = (int)blockIdx.x - 1;
+  if (idx < 0) {
+    // The one CTA that ties this kernel's completion to its predecessor's and publishes it.
+    // The first kernel of an epoch resets the word before any later kernel can start.
+    if (ord.epoch_start && threadIdx.x == 0) {
+      *reinterpret_cast<volatile unsigned*>(ord.done) = ord.tag << 20;
+      __threadfence();
+    }
+    __syncthreads();
+    pdl_launch_dependents();
+    pdl_wait();
+    if (!ord.epoch_start && threadIdx.x == 0)
+      *reinterpret_cast<volatile unsigned*>(ord.done) = (ord.tag << 20) | (unsigned)ord.e;
+    return;
+  }
+  const int unit = idx / per_unit, j = idx - unit * per_unit;
+  const bool is_tail = !plan.fold_tail && j == per_unit - 1;
+  char* ub = zc_unit_base(cache, lay, unit);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // the stream's word is requested first and looked at when it is needed
+  const unsigned ord_first = (ord.need_start > 0 || ord.need_end > 0) ? ld_order(ord.done) : 0u;
+  order_wait(ord, ord_first, ord.need_start, true, &g_zc_error);   // inputs written by an earlier call
+  if (k_new && j == 0) {
+    // Deferred append: the first item of every unit stores the newest row into the tail and
+    // makes it visible BEFORE it lets the next kernel start: later steps read that row without
+    // waiting for this kernel.  Nothing reads row n_tail - 1 of the tail buffer during this step.
+    if (warp == 0) {
+      const int pos = plan.n_tail - 1;
+      T* tk = reinterpret_cast<T*>(ub + lay.off_tailK) + pos * ZC_D;
+      T* tv = reinterpret_cast<T*>(ub + lay.off_tailV) + pos * ZC_D;
+      if (lane < 16)
+        reinterpret_cast<uint4*>(tk)[lane] = reinterpret_cast<const uint4*>(k_new + (long long)unit * ZC_D)[lane];
+      else
+        reinterpret_cast<uint4*>(tv)[lane - 16] =
+            reinterpret_cast<const uint4*>(v_new + (long long)unit * ZC_D)[lane - 16];
+      __threadfence();
+    }
+    __syncthreads();
+  }
+  pdl_launch_dependents();
+  const int b = unit / lay.n_kv, kv = unit % lay.n_kv;
+  const T* qunit = q + ((long long)b * lay.n_kv * G + kv * G) * ZC_D;
+  float* mine = part + (long long)unit * (plan.items + 1) * G * ZC_PART_STRIDE;
+  float* stash_g = collect ? stash_all + (long long)unit * G * ZC_MAX_WINDOW : nullptr;
+
+  if (is_tail || (plan.fold_tail && j == 0)) {
+    // The tail is the work of a CTA of its own, or (calls that share the GPU with their
+    // neighbours) of the unit's first item CTA before it turns to its codes.
+    // without a deferred append the newest tail row comes from the append kernel just before
+    if (!k_new) pdl_wait();
+    tail_phase<T>(reinterpret_cast<const T*>(ub + lay.off_tailK), reinterpret_cast<const T*>(ub + lay.off_tailV), G,
+                  plan.n_tail, qunit, unit, smem, mine + (long long)plan.items * G * ZC_PART_STRIDE, stash_g,
+                  k_new, v_new, ord, ord_first, &g_zc_error);
+    __syncthreads();   // the item phase reuses the shared memory
+  }
+  if (!is_tail) {
+    float* wm = reinterpret_cast<float*>(smem + kOffWm);
+    float* wl = reinterpret_cast<float*>(smem + kOffWl);
+    float* wz = reinterpret_cast<float*>(smem + kOffWz);
+    float* s_cw = reinterpret_cast<float*>(smem + kOffCw);
+    float* s_head = reinterpret_cast<float*>(smem + kOffHead);
+    const int z = j / groups, gi = j - z * groups;
+    const int h0 = 4 * z, Gl = min(4, G - h0);              // this CTA's query heads
+    const T* qbase = qunit + h0 * ZC_D;
+    const int it_end = min(plan.items, (gi + 1) * plan.cta_items);
+    for (int it = gi * plan.cta_items; it < it_end; ++it) {   // usually one item; all of them when calls overlap
+    const ItemDesc d = decode_item(plan, it);
+    float* my = mine + ((long long)it * G + h0) * ZC_PART_STRIDE;
+    float chan_factor = 1.f, rowscale = 1.f;
+    const bool has = d.sub_hi > d.sub_lo;
+    if (has) {
+      const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
+      const char* class_base = ub + lay.off_tiles[d.cls];
+      if (lay.bits[d.cls] == 4)
+        compressed_item<T, 4, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
+      else
+        compressed_item<T, 2, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
+    }
+    __syncthreads();
+    // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
+    if (tid < 4) {
+      float ms = -INFINITY;
+#pragma unroll
+      for (int w2 = 0; w2 < kWarps; ++w2) ms = fmaxf(ms, wm[w2 * 4 + tid]);
+      float ls = 0.f, zsum = 0.f;
+#pragma unroll
+      for (int w2 = 0; w2 < kWarps; ++w2) {
+        const float mw = wm[w2 * 4 + tid];
+        const float cw = (has && mw != -INFINITY) ? zc_exp2(mw - ms) : 0.f;
+        s_cw[tid * 4 + w2] = cw;
+        ls += wl[w2 * 4 + tid] * cw;
+        zsum += wz[w2 * 4 + tid] * cw;
+      }
+      s_head[tid * 4] = has ? ms : -INFINITY;
+      s_head[tid * 4 + 1] = has ? ls : 0.f;
+      s_head[tid * 4 + 2] = has ? zsum : 0.f;
+    }
+    __syncthreads();
+    order_wait(ord, ord_first, ord.need_end, false, &g_zc_error);   // the workspace region is free
+    for (int h = 0; h < Gl; ++h) {
+      float o = 0.f;
+      if (has) {
+        const float4 cw = *reinterpret_cast<const float4*>(s_cw + h * 4);
+        const float a0 = reinterpret_cast<const float*>(smem + kOffRing)[h * ZC_D + tid];
+        const float a1 = reinterpret_cast<const float*>(smem + kOffRing + RING)[h * ZC_D + tid];
+        const float a2 = reinterpret_cast<const float*>(smem + kOffRing + 2 * RING)[h * ZC_D + tid];
+        const float a3 = reinterpret_cast<const float*>(smem + kOffRing + 3 * RING)[h * ZC_D + tid];
+        o = (rowscale * (((cw.x * a0 + cw.y * a1) + cw.z * a2) + cw.w * a3) - s_head[h * 4 + 2]) * chan_factor;
+      }
+      float* dst = my + h * ZC_PART_STRIDE;
+      if (tid == 0) { dst[0] = s_head[h * 4]; dst[1] = s_head[h * 4 + 1]; }
+      dst[4 + tid] = o;
+    }
+    if (it + 1 < it_end) __syncthreads();   // the next item reuses the rings and the small arrays
+    }
+  }
+  // ---- count in: the barrier orders every thread's stores before thread 0's fence, the fence
+  //      before the count; the CTA that finds all others counted reads their partials from L2 ----
+  __syncthreads();
+  int* s_last = reinterpret_cast<int*>(smem + kCmbOffFlag);
+  if (tid == 0) {
+    unsigned* cnt = reinterpret_cast<unsigned*>(ub + lay.off_sync) + slot;
+    __threadfence();
+    const unsigned old = atomicAdd(cnt, 1u);
+    const int last = old == (unsigned)(per_unit - 1);
+    if (last) {
+      *cnt = 0u;          // next used in a later epoch, after this kernel has completed
+      __threadfence();
+    }
+    *s_last = last;
+  }
+  __syncthreads();
+  if (*s_last)
+    merge_unit<T>(reinterpret_cast<float*>(ub + lay.off_colsum), G, plan.items, plan.n_tail,
+                out + ((long long)b * lay.n_kv * G + kv * G) * ZC_D, mine, stash_g, collect, smem);
 }
 
 }  // namespace
@@ -960,10 +1076,41 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-// Output range of the latest decode launch: a decode call whose q lies inside it must not
-// start before that launch has finished, because q is read ahead of pdl_wait().
-const char* g_last_out_lo = nullptr;
-const char* g_last_out_hi = nullptr;
+// What the host remembers about a stream: the decode calls launched on it since the last
+// launch made without early start (an epoch).  Calls of an epoch may be in flight together.
+// Call e uses region e mod K of the workspace and arrival counter e mod K; the kernel itself
+// waits (see ZcOrder) until call e - K has completed before it writes there, until every
+// earlier call whose output it reads has completed before it reads, and until every earlier
+// call whose output or inputs it overwrites, or whose window statistics it adds to, has
+// completed before it writes.  The host finds those calls by comparing address ranges with
+// the last kRing calls; anything older is covered by waiting for call e - kRing.
+struct Range { const char* lo; const char* hi; };
+constexpr int kRing = ZC_EPOCH_CALLS;
+struct CallRec {
+  Range in[3];                      // q, k_new, v_new
+  Range out;
+  const zc_cache* collected;        // cache whose window statistics the call updates
+};
+struct StreamRec {
+  cudaStream_t st;
+  bool used;
+  int dev;
+  unsigned tag;                     // epoch tag, 12 bits
+  int e;                            // calls launched in the current epoch
+  int K;                            // workspace regions / arrival counters in use
+  const char* ws;
+  size_t ws_bytes, slot_bytes;
+  int capturing;
+  unsigned long long capture_id;
+  CallRec ring[kRing];
+  unsigned long long age;
+};
+constexpr int kStreamRecs = 16;
+StreamRec g_rec[kStreamRecs];
+unsigned long long g_rec_clock = 0;
+std::mutex g_rec_mutex;
+
+bool meet(const Range& a, const Range& b) { return a.lo && b.lo && a.lo < b.hi && b.lo < a.hi; }
 
 }  // namespace
 
@@ -979,24 +1126,149 @@ int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
   return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 
-int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
-                     float* ws, const void* k_new, const void* v_new, cudaStream_t st) {
-  const int G = c->lay.G;
-  float* part = ws;
-  dim3 grid(plan.items, c->lay.units, (G + 3) / 4);
-  const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
-  const char* q_lo = (const char*)q;
-  bool overlap = !(g_last_out_lo && q_lo < g_last_out_hi && q_lo + io_bytes > g_last_out_lo);
-  if (k_new && g_last_out_lo) {
-    // a deferred append is read ahead of the wait as well
-    const size_t kv_bytes = (size_t)c->lay.units * ZC_D * 2;
-    const char* kl = (const char*)k_new;
-    const char* vl = (const char*)v_new;
-    if ((kl < g_last_out_hi && kl + kv_bytes > g_last_out_lo) ||
-        (vl < g_last_out_hi && vl + kv_bytes > g_last_out_lo))
-      overlap = false;
+size_t zc_decode_scratch_bytes(const zc_cache* c, int items) {
+  const size_t part = (size_t)c->lay.units * (items + 1) * c->lay.G * ZC_PART_STRIDE * 4;
+  const size_t stash = (size_t)c->lay.units * c->lay.G * ZC_MAX_WINDOW * 4;
+  return ((part + 255) & ~(size_t)255) + ((stash + 255) & ~(size_t)255);
+}
+
+void zc_order_fence(zc_cache* c, cudaStream_t st) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::lock_guard<std::mutex> lock(g_rec_mutex);
+  c->fence_rec = -1;
+  for (int i = 0; i < kStreamRecs; ++i) {
+    const StreamRec& r = g_rec[i];
+    if (r.used && r.st == st && r.dev == dev) {
+      c->fence_rec = i;
+      c->fence_tag = r.tag;
+      c->fence_e = r.e;            // the next call of the epoch publishes their completion
+      c->fence_capturing = r.capturing;
+    }
   }
-  const dim3 cgrid(c->lay.units);
+}
+
+// One word per stream record, in the library image (like the built-in scratch below).
+// Two per record: calls issued under stream capture use the second, so that replaying a
+// captured graph never disturbs the word of the calls issued directly.
+static __device__ unsigned g_zc_order_words[32];
+
+int zc_order_words(unsigned** ptr) {
+  constexpr int kMaxDev = 64;
+  static unsigned* addr[kMaxDev] = {nullptr};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return (int)e;
+  if (dev < 0 || dev >= kMaxDev) return (int)cudaErrorInvalidDevice;
+  if (!addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_zc_order_words);
+    if (e != cudaSuccess) return (int)e;
+    addr[dev] = (unsigned*)p;
+  }
+  if (ptr) *ptr = addr[dev];
+  return (int)cudaSuccess;
+}
+
+int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
+                     char* ws, size_t ws_bytes, const void* k_new, const void* v_new, cudaStream_t st) {
+  static_assert(kStreamRecs == 16, "one order word per stream record");
+  const int G = c->lay.G, zs = (G + 3) / 4;
+  const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
+  const size_t kv_bytes = (size_t)c->lay.units * ZC_D * 2;
+  const size_t part_bytes = ((size_t)c->lay.units * (plan.items + 1) * G * ZC_PART_STRIDE * 4 + 255) & ~(size_t)255;
+  const size_t need = zc_decode_scratch_bytes(c, plan.items);
+  if (need > ws_bytes) return (int)cudaErrorInvalidValue;
+  unsigned* words = nullptr;
+  {
+    const int rc = zc_order_words(&words);
+    if (rc != (int)cudaSuccess) return rc;
+  }
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaStreamCaptureStatus cap_status = cudaStreamCaptureStatusNone;
+  unsigned long long cap_id = 0;
+  if (cudaStreamGetCaptureInfo(st, &cap_status, &cap_id) != cudaSuccess) {
+    cudaGetLastError();
+    cap_status = cudaStreamCaptureStatusNone;
+    cap_id = 0;
+  }
+  const int capturing = cap_status == cudaStreamCaptureStatusActive ? 1 : 0;
+  auto range = [](const void* p, size_t n) { return Range{(const char*)p, p ? (const char*)p + n : nullptr}; };
+  CallRec me;
+  me.in[0] = range(q, io_bytes);
+  me.in[1] = range(k_new, kv_bytes);
+  me.in[2] = range(v_new, kv_bytes);
+  me.out = range(out, io_bytes);
+  me.collected = collect ? c : nullptr;
+  ZcOrder ord;
+  int slot = 0;
+  size_t ws_off = 0;
+  {
+    std::lock_guard<std::mutex> lock(g_rec_mutex);
+    StreamRec* r = nullptr;
+    StreamRec* victim = nullptr;   // an unused record, else the one touched longest ago
+    for (int i = 0; i < kStreamRecs; ++i) {
+      StreamRec* x = &g_rec[i];
+      if (x->used && x->st == st && x->dev == dev) r = x;
+      if (!victim || (victim->used && (!x->used || x->age < victim->age))) victim = x;
+    }
+    bool fresh = false;
+    if (!r) {
+      r = victim;
+      if (r->used && !capturing) cudaStreamSynchronize(r->st);   // its word changes hands
+      cudaGetLastError();
+      r->used = true;
+      r->st = st;
+      r->dev = dev;
+      r->e = 0;
+      fresh = true;
+    }
+    // a new epoch: this launch is made without early start and so finds the stream drained
+    if (fresh || r->e == 0 || r->e >= (1 << 20) - 1 || r->ws != ws || r->ws_bytes != ws_bytes ||
+        need > r->slot_bytes || r->capturing != capturing || r->capture_id != cap_id) {
+      r->tag = (r->tag + 1) & 0xFFFu;
+      r->e = 0;
+      r->ws = ws;
+      r->ws_bytes = ws_bytes;
+      r->K = (int)std::min<size_t>((size_t)kRing, ws_bytes / need);
+      r->slot_bytes = (ws_bytes / (size_t)r->K) & ~(size_t)255;
+      if (r->slot_bytes < need) {   // alignment took the room: fewer, larger regions
+        r->K = std::max(1, r->K - 1);
+        r->slot_bytes = r->K == 1 ? ws_bytes : (ws_bytes / (size_t)r->K) & ~(size_t)255;
+      }
+      r->capturing = capturing;
+      r->capture_id = cap_id;
+    }
+    const int e = r->e;
+    ord.done = words + 2 * (r - g_rec) + capturing;
+    ord.tag = r->tag;
+    ord.e = e;
+    ord.epoch_start = e == 0;
+    ord.need_end = e - r->K + 1;
+    ord.need_start = e - kRing + 1;
+    for (int i = std::max(0, e - kRing + 1); i < e; ++i) {
+      const CallRec& o = r->ring[i % kRing];
+      for (int k = 0; k < 3; ++k) {
+        if (meet(me.in[k], o.out)) ord.need_start = std::max(ord.need_start, i + 1);
+        if (meet(me.out, o.in[k])) ord.need_end = std::max(ord.need_end, i + 1);
+      }
+      if (meet(me.out, o.out) || (collect && o.collected == c)) ord.need_end = std::max(ord.need_end, i + 1);
+    }
+    // kernels chained behind an earlier call changed this cache (a re-compressed window)
+    if (e > 0 && c->fence_rec == (int)(r - g_rec) && c->fence_tag == r->tag && c->fence_capturing == capturing)
+      ord.need_start = std::max(ord.need_start, c->fence_e);
+    slot = e % r->K;
+    ws_off = (size_t)slot * r->slot_bytes;
+    r->ring[e % kRing] = me;
+    r->e = e + 1;
+    r->age = ++g_rec_clock;
+  }
+  const bool overlap = !ord.epoch_start;
+  float* part = reinterpret_cast<float*>(ws + ws_off);
+  float* stash = reinterpret_cast<float*>(ws + ws_off + part_bytes);
+  const int groups = (plan.items + plan.cta_items - 1) / plan.cta_items;
+  const dim3 grid((unsigned)(c->lay.units * (groups * zs + (plan.fold_tail ? 0 : 1)) + 1));
   cudaError_t e;
 #define ZC_LAUNCH_STEP(T, RING, NCTA)                                                              \
   do {                                                                                             \
@@ -1004,17 +1276,14 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
     int dev_now = 0;                                                                               \
     cudaGetDevice(&dev_now);                                                                       \
     if (attr_dev != dev_now) {                                                                     \
-      e = cudaFuncSetAttribute(k_decode_items<T, RING, NCTA>,                                      \
+      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA>,                                            \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));    \
       if (e != cudaSuccess) return e;                                                              \
       attr_dev = dev_now;                                                                          \
     }                                                                                              \
-    e = launch_pdl(k_decode_items<T, RING, NCTA>, grid, dim3(128), decode_smem(RING), st, overlap, \
-                   c->base, c->lay, plan, (const T*)q, part, (const T*)k_new, (const T*)v_new);    \
-    if (e != cudaSuccess) return e;                                                                \
-    e = launch_pdl(k_decode_combine<T>, cgrid, dim3(128), kCombineSmem, st, true, c->base, c->lay, \
-                   plan, (const T*)q, (T*)out, (const float*)part, collect, (const T*)k_new,       \
-                   (const T*)v_new);                                                               \
+    e = launch_pdl(k_decode<T, RING, NCTA>, grid, dim3(128), decode_smem(RING), st, overlap,       \
+                   c->base, c->lay, plan, (const T*)q, (T*)out, part, stash, slot, collect,        \
+                   (const T*)k_new, (const T*)v_new, ord);                                         \
   } while (0)
   if (c->cfg.dtype == ZC_F16) {
     if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(__half, kRingNarrow, 4);
@@ -1024,9 +1293,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
     else ZC_LAUNCH_STEP(__nv_bfloat16, kRingWide, 3);
   }
 #undef ZC_LAUNCH_STEP
-  g_last_out_lo = (const char*)out;
-  g_last_out_hi = (const char*)out + io_bytes;
-  c->launches += 2;
+  c->launches += 1;
   return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }
 

@@ -6,6 +6,7 @@
 #include <new>
 #include <vector>
 #include <algorithm>
+#include <cstdlib>
 #include "zc_internal.h"
 #include "zc_layout.cuh"
 
@@ -27,7 +28,7 @@ int check_config(const zc_config* cfg) {
   if (cfg->window < 8 || cfg->window > ZC_MAX_WINDOW) return ZC_EINVAL;
   if (cfg->bits_hi != 4 && cfg->bits_hi != 2) return ZC_EINVAL;
   if (cfg->bits_lo != 4 && cfg->bits_lo != 2) return ZC_EINVAL;
-  if (cfg->flags & ~ZC_FLAG_DEFER_APPEND) return ZC_EINVAL;
+  if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS)) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if ((long long)cfg->batch * cfg->n_kv_heads > 65535) return ZC_EINVAL;
   // every re-compressed window adds two items to a decode call
@@ -71,7 +72,7 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   lay->off_colsum = (long long)off;
   off = align_up(off + ZC_MAX_WINDOW * 4, 256);
   lay->off_sync = (long long)off;   // directly after colsum: both are cleared together
-  off = align_up(off + 256, 256);
+  off = align_up(off + ZC_EPOCH_CALLS * 4, 256);
   lay->off_scores = (long long)off;
   off = align_up(off + (size_t)std::max(cfg->max_prefill, cfg->window) * 4, 256);
   lay->off_idx = (long long)off;
@@ -83,11 +84,13 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
     const int np_max = cfg->max_prefill;
     size_t pre = align_up((size_t)np_max * 4, 256) +
                  (size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4;
-    // decode: partials [unit][item][G][ZC_PART_STRIDE] + tail logits [unit][G][window]
+    // decode: partials [unit][item + tail][G][ZC_PART_STRIDE] + tail logits
+    // [unit][G][ZC_MAX_WINDOW]; twice the worst case, so that calls in flight together (each
+    // takes what its present number of items needs) find room
     const int max_items = std::min(ZC_MAX_ITEMS, 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush);
-    size_t dec = (size_t)lay->units * max_items * lay->G * ZC_PART_STRIDE * 4 +
-                 (size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4 + 256;
-    *ws_bytes = align_up(std::max(pre, dec), 256);
+    size_t dec = align_up((size_t)lay->units * (max_items + 1) * lay->G * ZC_PART_STRIDE * 4, 256) +
+                 align_up((size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4, 256);
+    *ws_bytes = align_up(std::max(pre, 2 * dec), 512);
   }
 }
 
@@ -167,7 +170,8 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
         spi[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;
         split[k] = zc_ceil_div(subs[k], spi[k]);
       }
-      const double n_ctas = (double)(split[0] + split[1] + extras) * c->lay.units * zs;
+      // items of every head group, one tail CTA per unit, one sentinel
+      const double n_ctas = ((double)(split[0] + split[1] + extras) * zs + 1) * c->lay.units + 1;
       const double waves = n_ctas / slots;
       // a handful of CTAs beyond a whole wave start as soon as the first ones retire
       const double whole = std::max(1.0, (waves - floor(waves) <= ZC_WAVE_SLACK) ? floor(waves) : ceil(waves));
@@ -185,7 +189,24 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   p.ctas_per_sm = 3;
   if (choose(4) >= ZC_MANY_WAVES * c->n_sm * 4) p.ctas_per_sm = 4;
   else choose(3);
+  if (c->cfg.flags & ZC_FLAG_OVERLAP_CALLS) {
+    // Calls of independent caches follow one another on the stream and run side by side:
+    // wave fill is then no concern, only the fixed cost per CTA, so items are as large as
+    // they get and the build with more resident warps is used.
+    p.ctas_per_sm = 4;
+    p.fold_tail = 1;
+    for (int k = 0; k < 2; ++k) {
+      const int want = std::min(std::min(zc_ceil_div(subs[k], kCand[0]), std::min(ZC_MAX_SPLIT_HOST, cap)), subs[k]);
+      p.spi0[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;
+      p.split0[k] = zc_ceil_div(subs[k], p.spi0[k]);
+    }
+  }
   p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1);
+  p.cta_items = 1;
+  if (c->cfg.flags & ZC_FLAG_OVERLAP_CALLS) {
+    static const char* e_ci = getenv("ZIPCACHE_CTA_ITEMS");   // tuning override (experiments)
+    p.cta_items = e_ci ? std::max(1, atoi(e_ci)) : p.items;
+  }
   return p;
 }
 
@@ -226,12 +247,15 @@ int zc_cache_init(void* dev_mem, size_t bytes, const zc_config* cfg, zc_cache** 
   c->bytes = bytes;
   c->l0 = -1;
   c->n_seg = 0;
+  c->fence_rec = -1;
   int dev = 0, n_sm = 148;
   if (cudaGetDevice(&dev) == cudaSuccess)
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
   else
     cudaGetLastError();
   c->n_sm = n_sm > 0 ? n_sm : 148;
+  // the address look-ups the decode launches need are done here, outside any stream capture
+  if (zc_order_words(nullptr) != (int)cudaSuccess) cudaGetLastError();
   *out = c;
   return ZC_OK;
 }
@@ -317,7 +341,7 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
   c->last_scores_n = l;
   // window statistics and the decode kernel's arrival counter start at zero
   ZC_CUDA(cudaMemset2DAsync(c->base + c->lay.off_colsum, (size_t)c->lay.unit_stride, 0,
-                            (size_t)(c->lay.off_sync + 256 - c->lay.off_colsum),
+                            (size_t)(c->lay.off_sync + ZC_EPOCH_CALLS * 4 - c->lay.off_colsum),
                             (size_t)c->lay.units, st));
   if (!salient_idx) {
     int32_t* P_dev = (int32_t*)workspace;
@@ -351,12 +375,14 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
   return ZC_OK;
 }
 
-int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step,
-                        void* workspace, size_t workspace_bytes, zc_stream_t stream) {
+// need_worst: check the workspace against the worst case of the cache's whole life (the public
+// contract) rather than against what this call touches.
+static int decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step, void* workspace,
+                            size_t workspace_bytes, bool need_worst, zc_stream_t stream) {
   if (!c || !q || !out || !workspace) return ZC_EINVAL;
   if (c->l0 < 0) return ZC_ESTATE;
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return ZC_EALIGN;
-  if (workspace_bytes < c->ws_bytes) return ZC_ECAPACITY;
+  if (need_worst && workspace_bytes < c->ws_bytes) return ZC_ECAPACITY;
   cudaStream_t st = (cudaStream_t)stream;
   if (c->pend_k && c->pend_stream != st) {
     int rc = flush_pending(c);
@@ -369,7 +395,7 @@ int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step
   const void* pk = c->pend_k;
   const void* pv = c->pend_v;
   c->pend_k = c->pend_v = nullptr;
-  ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (float*)workspace, pk, pv, st));
+  ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (char*)workspace, workspace_bytes, pk, pv, st));
   // Alg. 3 bookkeeping: the step counter follows the tokens of the current window
   if (c->n_tail > 0) {
     c->step_i = i_next;
@@ -377,16 +403,19 @@ int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step
       for (int j = 0; j < c->n_tail; ++j) c->tail_nnz[j] += 1;
     if (c->step_i == c->cfg.window && c->n_tail == c->cfg.window) {
       // re-compress the window into a new segment
-      ZC_CUDA(zc_launch_window_scores(c, st));
+      // the re-compression runs as links of the decode calls' chain: calls on other caches
+      // that follow on the stream start without waiting for it
+      ZC_CUDA(zc_launch_window_scores(c, st, true));
       c->last_scores_n = c->cfg.window;
       const int seg = c->n_seg;
       c->n_seg += 1;
       ZcSeg s = zc_segment(c, seg);
-      ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], s.idx_off, nullptr, st));
+      ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], s.idx_off, nullptr, st, true));
       const long long us = c->lay.unit_stride / 2;
       ZcSrc src{c->base + c->lay.off_tailK, c->base + c->lay.off_tailV, us * c->lay.n_kv, us,
                 ZC_D};
-      ZC_CUDA(zc_launch_quantize(c, src, s, st));
+      ZC_CUDA(zc_launch_quantize(c, src, s, st, true));
+      zc_order_fence(c, st);
       c->n_tail = 0;
       c->step_i = 0;
       memset(c->tail_nnz, 0, sizeof(c->tail_nnz));
@@ -395,19 +424,23 @@ int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step
   return ZC_OK;
 }
 
+int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step,
+                        void* workspace, size_t workspace_bytes, zc_stream_t stream) {
+  return decode_attention(c, q, out, is_probe_step, workspace, workspace_bytes, true, stream);
+}
+
 int zc_decode_attention_noalloc(zc_cache* c, const void* q, void* out, int is_probe_step,
                                 zc_stream_t stream) {
   if (!c || !q || !out) return ZC_EINVAL;
   if (c->l0 < 0) return ZC_ESTATE;
-  // what this call will really write: partials [unit][item][G][ZC_PART_STRIDE]
+  // what this call really writes: partials and tail logits for the cache's present number of
+  // items (calls that follow take further room in the buffer, or wait for this one)
   const ZcDecodePlan plan = zc_make_plan(c);
-  const size_t need = (size_t)c->lay.units * plan.items * c->lay.G * ZC_PART_STRIDE * 4;
+  const size_t need = zc_decode_scratch_bytes(c, plan.items);
   if (need > (size_t)ZC_NOALLOC_SCRATCH_BYTES) return ZC_ESCRATCH;
   void* scratch = nullptr;
   ZC_CUDA(zc_static_scratch(&scratch));   // first call per device: a synchronous address query
-  // The ordinary entry point sizes its check for the worst case of the cache's whole life;
-  // the bytes above are the ones it touches in the cache's present state.
-  return zc_decode_attention(c, q, out, is_probe_step, scratch, c->ws_bytes, stream);
+  return decode_attention(c, q, out, is_probe_step, scratch, (size_t)ZC_NOALLOC_SCRATCH_BYTES, false, stream);
 }
 
 int zc_num_segments(const zc_cache* c) { return c ? c->n_seg : ZC_EINVAL; }

@@ -14,6 +14,7 @@
 #define ZC_MAX_G 8
 #define ZC_MAX_SPLIT_HOST 32      // most items one class of segment 0 is split into
 #define ZC_MAX_ITEMS 128          // most items of one unit in one decode call
+#define ZC_EPOCH_CALLS 64          // most decode calls in flight together on a stream (arrival counters per unit)
 #ifndef ZC_ITEM_OVERHEAD
 #define ZC_ITEM_OVERHEAD 24       // fixed cost of one split-K item, in 16-token sub-tiles of streaming
 #endif
@@ -31,7 +32,7 @@
 //   off_cmax       scratch: |x| channel maxima as uint bits  [class][tensor][128]
 //   off_tailK/V    window x d elements of the input type
 //   off_colsum     window floats: attention mass collected on probe steps
-//   off_sync       arrival counter of the decode kernel's split-K items (zero between calls)
+//   off_sync       ZC_EPOCH_CALLS arrival counters of the decode kernel's CTAs (zero between calls)
 //   off_scores     normalised scores of the latest compression
 //   off_idx        token index lists: segment 0 (salient then regular), then one
 //                  window-sized slot per re-compressed window
@@ -74,8 +75,10 @@ struct ZcDecodePlan {
   int split0[2];           // items covering segment 0, per class
   int spi0[2];             // 16-token sub-tiles per item, per class
   int n_tail;
-  int ctas_per_sm;         // build of the items kernel: 3 (wide rings) or 4 (narrow rings)
+  int ctas_per_sm;         // build of the decode kernel: 3 (wide rings) or 4 (narrow rings)
   int items;               // items per unit
+  int cta_items;           // consecutive items one CTA works through
+  int fold_tail;           // the tail is attended by the unit's first item CTA, not by a CTA of its own
   int l0;
 };
 
@@ -100,6 +103,11 @@ struct zc_cache {
   const void* pend_k;
   const void* pend_v;
   cudaStream_t pend_stream;
+  // ordering of decode calls behind chained kernels that changed this cache (zc_order_fence)
+  int fence_rec;
+  unsigned fence_tag;
+  int fence_e;
+  int fence_capturing;
 };
 
 __host__ __device__ static inline int zc_ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -111,17 +119,29 @@ ZcDecodePlan zc_make_plan(const zc_cache* c);
 int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l,
                            const int64_t* qs, const int64_t* ks, const int32_t* P_dev,
                            int n_probe, float* lse_ws, cudaStream_t st);
+// chained: launched as a link of the decode calls' chain on the stream (see zc_compress.cu);
+// the caller then fences the cache with zc_order_fence.
 int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
-                   cudaStream_t st);
-int zc_launch_window_scores(zc_cache* c, cudaStream_t st);
-int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st);
+                   cudaStream_t st, bool chained = false);
+int zc_launch_window_scores(zc_cache* c, cudaStream_t st, bool chained = false);
+int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st,
+                       bool chained = false);
+// Marks the cache as changed by kernels just launched on st: decode calls on this cache
+// that follow within the same epoch wait for them before they read anything.
+void zc_order_fence(zc_cache* c, cudaStream_t st);
 int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
                      cudaStream_t st);
 // k_new / v_new non-null: the newest tail row is read from them and stored into the tail.
+// Calls that may be in flight together on a stream take consecutive regions of ws.
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out,
-                     int collect, float* ws, const void* k_new, const void* v_new,
+                     int collect, char* ws, size_t ws_bytes, const void* k_new, const void* v_new,
                      cudaStream_t st);
+// Bytes of ws one call of `items` items per unit takes.
+size_t zc_decode_scratch_bytes(const zc_cache* c, int items);
 int zc_device_error_code(int* out);
+// Device address of the per-stream ordering words on the current device (looked up once per
+// device; pass nullptr to only perform the look-up).
+int zc_order_words(unsigned** ptr);
 // Device address of the built-in scratch buffer on the current device (looked up once per device).
 int zc_static_scratch(void** ptr);
 int zc_launch_export_scores(zc_cache* c, float* out, int n, cudaStream_t st);

@@ -24,11 +24,12 @@ def to64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu", torch.float64).numpy()
 
 
-def make_cache(w: Workload, max_new=None, defer_append: bool = False):
+def make_cache(w: Workload, max_new=None, defer_append: bool = False, overlap_calls: bool = False):
     import paper_2405_14256_b200 as zc
     return zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context,
                        w.decode_steps if max_new is None else max_new, w.saliency_ratio,
-                       w.bits_hi, w.bits_lo, w.window, device=DEV, defer_append=defer_append)
+                       w.bits_hi, w.bits_lo, w.window, device=DEV, defer_append=defer_append,
+                       overlap_calls=overlap_calls)
 
 
 def make_oracle(w: Workload, units=None) -> zo.ZipCacheOracle:
