@@ -474,10 +474,12 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
 // One compressed item, whole CTA.  On return every warp has put its (m, l, z-sum) and its
 // accumulators into shared memory; *chan_factor / *rowscale tell the merge how to bring a
 // channel's accumulator to true units.
+// Not inlined: the loop inside gets the whole register budget to itself, whatever the caller
+// keeps alive around the call.
+struct ItemScale { float chan_factor, rowscale; };
 template <typename T, int BITS, int RING>
-__device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* class_base,
-                                                const float* fac, const T* qbase, int Gl, char* smem,
-                                                float* chan_factor, float* rowscale, int* err) {
+__device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_base, const float* fac,
+                                                  const T* qbase, int Gl, char* smem, int* err) {
   constexpr int SB = ZC_SUB * (32 * BITS + 16);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   constexpr int PB = 2 * SB;
@@ -595,26 +597,26 @@ __device__ __forceinline__ void compressed_item(const ItemDesc& d, const char* c
     }
   }
   // o[ch] = c^V[ch] 2^-logK (acc 2^24 / sigma(row) - z sum); rows g+8 of a tile carry sigma = 16
-  *chan_factor = cV * zc_exp2(-logK);
-  *rowscale = (tid & 8) ? 1048576.f : 16777216.f;
+  ItemScale r;
+  r.chan_factor = cV * zc_exp2(-logK);
+  r.rowscale = (tid & 8) ? 1048576.f : 16777216.f;
+  return r;
 }
 
 // Sixteen tokens of the full-precision tail for one warp and up to four query heads, on tensor
 // cores in the input type: S^T = K_tail q^T with q exact in its own type, then
 // O^T = V_tail^T P^T with P = hi + lo in the input type (columns 0..3 and 4..7).
-// Results: wm / wl [warp][4] (row maximum, sum), mbuf [4 heads][128] for this warp, and the
-// logits (base 2) of the tokens into stash [4 heads][ZC_MAX_WINDOW].
+// The tile is a split-K partial of its own: (row maximum, sum) and the accumulators of head h
+// go to dst + h * ZC_PART_STRIDE, the logits (base 2) of the tokens, when the step collects
+// probe statistics, to stash [4 heads][ZC_MAX_WINDOW] (global memory).  One warp, no shared
+// memory, no barrier: the warps of a CTA take tiles independently.
 template <typename T>
 __device__ __forceinline__ void tail_tile(const T* tK, const T* tV, int n_tail, int base,
-                                          const T* qbase, int Gl, int unit, float* wm, float* wl,
-                                          float* mbuf, float* stash, const T* k_new, const T* v_new) {
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+                                          const T* qbase, int Gl, int unit, float* dst, float* stash,
+                                          const T* k_new, const T* v_new) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int nv = min(ZC_SUB, n_tail - base);
-  if (nv <= 0) {
-    if (lane < 4) { wm[warp * 4 + lane] = -INFINITY; wl[warp * 4 + lane] = 0.f; }
-    for (int i = lane; i < 4 * ZC_D; i += 32) mbuf[i] = 0.f;
-    return;
-  }
+  if (nv <= 0) return;
   const int last = n_tail - 1;
   // Deferred append: the newest row is read from the caller's k_new / v_new [unit][128] (the
   // unit's first item CTA stores it into the tail).
@@ -665,7 +667,7 @@ __device__ __forceinline__ void tail_tile(const T* tK, const T* tV, int n_tail, 
     lg[0][e] = dacc[e] * scale;
     lg[1][e] = dacc[2 + e] * scale;
     const int h = 2 * t + e;
-    if (t < 2 && h < Gl) {
+    if (stash && t < 2 && h < Gl) {
       if (v0) stash[h * ZC_MAX_WINDOW + base + g] = lg[0][e];
       if (v1) stash[h * ZC_MAX_WINDOW + base + g + 8] = lg[1][e];
     }
@@ -728,91 +730,48 @@ __device__ __forceinline__ void tail_tile(const T* tK, const T* tV, int n_tail, 
   if (t < 2) {
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
-      if (g == 0) { wm[warp * 4 + 2 * t + e] = mx[e]; wl[warp * 4 + 2 * t + e] = ls[e]; }
+      if (2 * t + e < Gl) {
+        float* d = dst + (2 * t + e) * ZC_PART_STRIDE;
+        if (g == 0) *reinterpret_cast<float2*>(d) = make_float2(mx[e], ls[e]);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        mbuf[(2 * t + e) * ZC_D + 16 * g + 2 * i] = oacc[i][e];
-        mbuf[(2 * t + e) * ZC_D + 16 * g + 2 * i + 1] = oacc[i][2 + e];
+        for (int i = 0; i < 8; ++i)
+          *reinterpret_cast<float2*>(d + 4 + 16 * g + 2 * i) = make_float2(oacc[i][e], oacc[i][2 + e]);
       }
     }
   }
 }
 
-// shared-memory map of the tail and merge phases (they reuse the memory of the item phase)
-constexpr int kCmbEntries = (ZC_MAX_ITEMS + 1) * ZC_MAX_G;       // items + the tail, per head
-// The map starts behind the mbarriers: memory that holds mbarrier objects is never reused as
-// data (plain stores over a used barrier were observed to be replaced by barrier state).
+// shared-memory map of the merge phase (it reuses the memory of the item phase, but not the
+// mbarriers': memory that holds mbarrier objects is never reused as data -- plain stores
+// over a used barrier were observed to be replaced by barrier state)
+constexpr int kMaxTailTiles = ZC_MAX_WINDOW / ZC_SUB;
+constexpr int kCmbEntries = (ZC_MAX_ITEMS + kMaxTailTiles) * ZC_MAX_G;   // items + tail tiles, per head
 constexpr int kCmbOffM = kOffQfrag;                               // [entries] maxima, then weights
 constexpr int kCmbOffL = kCmbOffM + kCmbEntries * 4;              // [entries] sums
 constexpr int kCmbOffML = kCmbOffL + kCmbEntries * 4;             // [G] x (M, L)
-constexpr int kCmbOffStash = kCmbOffML + 2 * ZC_MAX_G * 4;        // [G][ZC_MAX_WINDOW] tail logits
-constexpr int kCmbOffWm = kCmbOffStash + ZC_MAX_G * ZC_MAX_WINDOW * 4;      // [kWarps][4] x (m, l)
-constexpr int kCmbOffMbuf = kCmbOffWm + 2 * kWarps * 4 * 4;       // [kWarps][4 heads][128]
-constexpr int kCmbOffFlag = kCmbOffMbuf + kWarps * 4 * ZC_D * 4;  // "this CTA arrived last"
+constexpr int kCmbOffFlag = kCmbOffML + 2 * ZC_MAX_G * 4;         // "this CTA arrived last"
 constexpr int kCombineSmem = kCmbOffFlag + 16;
-static_assert(kCombineSmem <= decode_smem(kRingNarrow), "tail and merge phases must fit the item phase's memory");
+static_assert(kCombineSmem <= decode_smem(kRingNarrow), "the merge phase must fit the item phase's memory");
 
-// Attention over the full-precision tail, whole CTA, all query heads of the unit: passes of 64
-// tokens (16 per warp); thread = channel keeps the running (M, L, O) of its heads in registers
-// across passes.  The result goes out as one more split-K partial, the logits (base 2) to
-// stash_g [G][ZC_MAX_WINDOW] when the step collects probe statistics.
+// Attention over the full-precision tail, all query heads of the unit: tile i (16 tokens) is
+// taken by warp i mod 4 and becomes split-K partial `first_entry + i`.  Nothing here touches
+// shared memory or a barrier.
 template <typename T>
 __device__ __noinline__ void tail_phase(const T* tK, const T* tV, int G, int n_tail, const T* qunit, int unit,
-                                        char* smem, float* part_tail, float* stash_g, const T* k_new,
+                                        float* part_unit, int first_entry, float* stash_g, const T* k_new,
                                         const T* v_new, ZcOrder ord, unsigned ord_first, int* err) {
-  float* stash = reinterpret_cast<float*>(smem + kCmbOffStash);
-  float* twm = reinterpret_cast<float*>(smem + kCmbOffWm);
-  float* twl = twm + kWarps * 4;
-  const int tid = threadIdx.x, warp = tid >> 5;
-  for (int hg = 0; hg * 4 < G; ++hg) {
-    const int Gl = min(4, G - 4 * hg);
-    float Mr[4], Lr[4], Or[4];
-#pragma unroll
-    for (int h = 0; h < 4; ++h) { Mr[h] = -INFINITY; Lr[h] = 0.f; Or[h] = 0.f; }
-    for (int base0 = 0; base0 < n_tail; base0 += kWarps * ZC_SUB) {
-      float* mbuf = reinterpret_cast<float*>(smem + kCmbOffMbuf) + warp * 4 * ZC_D;
-      tail_tile<T>(tK, tV, n_tail, base0 + warp * ZC_SUB, qunit + 4 * hg * ZC_D, Gl, unit, twm, twl, mbuf,
-                   stash + 4 * hg * ZC_MAX_WINDOW, k_new, v_new);
-      __syncthreads();
-#pragma unroll
-      for (int h = 0; h < 4; ++h) {
-        if (h < Gl) {
-          float mn = Mr[h];
-#pragma unroll
-          for (int w2 = 0; w2 < kWarps; ++w2) mn = fmaxf(mn, twm[w2 * 4 + h]);
-          const float c_old = Mr[h] == -INFINITY ? 0.f : zc_exp2(Mr[h] - mn);
-          float o = Or[h] * c_old, l = Lr[h] * c_old;
-#pragma unroll
-          for (int w2 = 0; w2 < kWarps; ++w2) {
-            const float mw = twm[w2 * 4 + h];
-            if (mw != -INFINITY) {
-              const float cw = zc_exp2(mw - mn);
-              l += twl[w2 * 4 + h] * cw;
-              o += reinterpret_cast<const float*>(smem + kCmbOffMbuf)[(w2 * 4 + h) * ZC_D + tid] * cw;
-            }
-          }
-          Mr[h] = mn; Lr[h] = l; Or[h] = o;
-        }
-      }
-      __syncthreads();
-    }
-    if (hg == 0) order_wait(ord, ord_first, ord.need_end, false, err);   // the workspace region is free
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-      if (h < Gl) {
-        float* tp = part_tail + (4 * hg + h) * ZC_PART_STRIDE;
-        if (tid == 0) { tp[0] = Mr[h]; tp[1] = Lr[h]; }
-        tp[4 + tid] = Or[h];
-      }
-    }
-  }
-  if (stash_g) {
-    for (int i = tid; i < G * ZC_MAX_WINDOW; i += 128)
-      if ((i & (ZC_MAX_WINDOW - 1)) < n_tail) stash_g[i] = stash[i];
+  const int warp = threadIdx.x >> 5;
+  order_wait(ord, ord_first, ord.need_end, false, err);   // the workspace region is free
+  for (int base = warp * ZC_SUB; base < n_tail; base += kWarps * ZC_SUB) {
+    float* entry = part_unit + (long long)(first_entry + base / ZC_SUB) * G * ZC_PART_STRIDE;
+    for (int hg = 0; hg * 4 < G; ++hg)
+      tail_tile<T>(tK, tV, n_tail, base, qunit + 4 * hg * ZC_D, min(4, G - 4 * hg), unit,
+                   entry + 4 * hg * ZC_PART_STRIDE, stash_g ? stash_g + 4 * hg * ZC_MAX_WINDOW : nullptr, k_new,
+                   v_new);
   }
 }
 
-// Merge of a unit's split-K partials (items, then the tail as the last entry) in a fixed order,
+// Merge of a unit's split-K partials (items, then the tail's tiles) in a fixed order,
 // the output row of every query head and, on probe steps, this step's attention over the
 // tail's tokens added to the window statistics.  Run by the CTA of the unit that finished last.
 template <typename T>
@@ -822,7 +781,7 @@ __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_t
   float* s_l = reinterpret_cast<float*>(smem + kCmbOffL);
   float* s_ML = reinterpret_cast<float*>(smem + kCmbOffML);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int entries = items + 1;
+  const int entries = items + (n_tail + ZC_SUB - 1) / ZC_SUB;
   for (int e = tid; e < entries * G; e += 128) {
     const float2 ml = __ldcg(reinterpret_cast<const float2*>(mine + (long long)e * ZC_PART_STRIDE));
     s_m[e] = ml.x;
@@ -938,39 +897,34 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // the stream's word is requested first and looked at when it is needed
   const unsigned ord_first = (ord.need_start > 0 || ord.need_end > 0) ? ld_order(ord.done) : 0u;
-  order_wait(ord, ord_first, ord.need_start, true, &g_zc_error);   // inputs written by an earlier call
-  if (k_new && j == 0) {
-    // Deferred append: the first item of every unit stores the newest row into the tail and
-    // makes it visible BEFORE it lets the next kernel start: later steps read that row without
-    // waiting for this kernel.  Nothing reads row n_tail - 1 of the tail buffer during this step.
-    if (warp == 0) {
-      const int pos = plan.n_tail - 1;
-      T* tk = reinterpret_cast<T*>(ub + lay.off_tailK) + pos * ZC_D;
-      T* tv = reinterpret_cast<T*>(ub + lay.off_tailV) + pos * ZC_D;
-      if (lane < 16)
-        reinterpret_cast<uint4*>(tk)[lane] = reinterpret_cast<const uint4*>(k_new + (long long)unit * ZC_D)[lane];
-      else
-        reinterpret_cast<uint4*>(tv)[lane - 16] =
-            reinterpret_cast<const uint4*>(v_new + (long long)unit * ZC_D)[lane - 16];
-      __threadfence();
-    }
-    __syncthreads();
-  }
   pdl_launch_dependents();
+  // inputs written by an earlier call, a re-compressed window, the previous call's tail row
+  order_wait(ord, ord_first, ord.need_start, true, &g_zc_error);
+  if (k_new && j == 0 && warp == kWarps - 1) {
+    // Deferred append: the newest row goes into the tail for the steps to come (this step reads
+    // it from k_new / v_new).  The next call on this cache is told to wait for this one.
+    const int pos = plan.n_tail - 1;
+    T* tk = reinterpret_cast<T*>(ub + lay.off_tailK) + pos * ZC_D;
+    T* tv = reinterpret_cast<T*>(ub + lay.off_tailV) + pos * ZC_D;
+    if (lane < 16)
+      reinterpret_cast<uint4*>(tk)[lane] = reinterpret_cast<const uint4*>(k_new + (long long)unit * ZC_D)[lane];
+    else
+      reinterpret_cast<uint4*>(tv)[lane - 16] =
+          reinterpret_cast<const uint4*>(v_new + (long long)unit * ZC_D)[lane - 16];
+  }
   const int b = unit / lay.n_kv, kv = unit % lay.n_kv;
   const T* qunit = q + ((long long)b * lay.n_kv * G + kv * G) * ZC_D;
-  float* mine = part + (long long)unit * (plan.items + 1) * G * ZC_PART_STRIDE;
+  const int n_tiles = (plan.n_tail + ZC_SUB - 1) / ZC_SUB;
+  float* mine = part + (long long)unit * (plan.items + kMaxTailTiles) * G * ZC_PART_STRIDE;
   float* stash_g = collect ? stash_all + (long long)unit * G * ZC_MAX_WINDOW : nullptr;
 
-  if (is_tail || (plan.fold_tail && j == 0)) {
+  if (n_tiles > 0 && (is_tail || (plan.fold_tail && j == 0))) {
     // The tail is the work of a CTA of its own, or (calls that share the GPU with their
     // neighbours) of the unit's first item CTA before it turns to its codes.
     // without a deferred append the newest tail row comes from the append kernel just before
     if (!k_new) pdl_wait();
     tail_phase<T>(reinterpret_cast<const T*>(ub + lay.off_tailK), reinterpret_cast<const T*>(ub + lay.off_tailV), G,
-                  plan.n_tail, qunit, unit, smem, mine + (long long)plan.items * G * ZC_PART_STRIDE, stash_g,
-                  k_new, v_new, ord, ord_first, &g_zc_error);
-    __syncthreads();   // the item phase reuses the shared memory
+                  plan.n_tail, qunit, unit, mine, plan.items, stash_g, k_new, v_new, ord, ord_first, &g_zc_error);
   }
   if (!is_tail) {
     float* wm = reinterpret_cast<float*>(smem + kOffWm);
@@ -985,15 +939,17 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     for (int it = gi * plan.cta_items; it < it_end; ++it) {   // usually one item; all of them when calls overlap
     const ItemDesc d = decode_item(plan, it);
     float* my = mine + ((long long)it * G + h0) * ZC_PART_STRIDE;
-    float chan_factor = 1.f, rowscale = 1.f;
+    ItemScale sc;
+    sc.chan_factor = 1.f;
+    sc.rowscale = 1.f;
     const bool has = d.sub_hi > d.sub_lo;
     if (has) {
       const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
       const char* class_base = ub + lay.off_tiles[d.cls];
       if (lay.bits[d.cls] == 4)
-        compressed_item<T, 4, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
+        sc = compressed_item<T, 4, RING>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
       else
-        compressed_item<T, 2, RING>(d, class_base, fac, qbase, Gl, smem, &chan_factor, &rowscale, &g_zc_error);
+        sc = compressed_item<T, 2, RING>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
     }
     __syncthreads();
     // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
@@ -1024,7 +980,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
         const float a1 = reinterpret_cast<const float*>(smem + kOffRing + RING)[h * ZC_D + tid];
         const float a2 = reinterpret_cast<const float*>(smem + kOffRing + 2 * RING)[h * ZC_D + tid];
         const float a3 = reinterpret_cast<const float*>(smem + kOffRing + 3 * RING)[h * ZC_D + tid];
-        o = (rowscale * (((cw.x * a0 + cw.y * a1) + cw.z * a2) + cw.w * a3) - s_head[h * 4 + 2]) * chan_factor;
+        o = (sc.rowscale * (((cw.x * a0 + cw.y * a1) + cw.z * a2) + cw.w * a3) - s_head[h * 4 + 2]) * sc.chan_factor;
       }
       float* dst = my + h * ZC_PART_STRIDE;
       if (tid == 0) { dst[0] = s_head[h * 4]; dst[1] = s_head[h * 4 + 1]; }
@@ -1037,7 +993,10 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
   //      before the count; the CTA that finds all others counted reads their partials from L2 ----
   __syncthreads();
   int* s_last = reinterpret_cast<int*>(smem + kCmbOffFlag);
-  if (tid == 0) {
+  if (per_unit == 1) {
+    // the unit's only CTA: its own stores are visible to it after the barrier
+    if (tid == 0) *s_last = 1;
+  } else if (tid == 0) {
     unsigned* cnt = reinterpret_cast<unsigned*>(ub + lay.off_sync) + slot;
     __threadfence();
     const unsigned old = atomicAdd(cnt, 1u);
@@ -1127,7 +1086,7 @@ int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
 }
 
 size_t zc_decode_scratch_bytes(const zc_cache* c, int items) {
-  const size_t part = (size_t)c->lay.units * (items + 1) * c->lay.G * ZC_PART_STRIDE * 4;
+  const size_t part = (size_t)c->lay.units * (items + kMaxTailTiles) * c->lay.G * ZC_PART_STRIDE * 4;
   const size_t stash = (size_t)c->lay.units * c->lay.G * ZC_MAX_WINDOW * 4;
   return ((part + 255) & ~(size_t)255) + ((stash + 255) & ~(size_t)255);
 }
@@ -1176,7 +1135,8 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   const int G = c->lay.G, zs = (G + 3) / 4;
   const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
   const size_t kv_bytes = (size_t)c->lay.units * ZC_D * 2;
-  const size_t part_bytes = ((size_t)c->lay.units * (plan.items + 1) * G * ZC_PART_STRIDE * 4 + 255) & ~(size_t)255;
+  const size_t part_bytes =
+      ((size_t)c->lay.units * (plan.items + kMaxTailTiles) * G * ZC_PART_STRIDE * 4 + 255) & ~(size_t)255;
   const size_t need = zc_decode_scratch_bytes(c, plan.items);
   if (need > ws_bytes) return (int)cudaErrorInvalidValue;
   unsigned* words = nullptr;
@@ -1260,6 +1220,13 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
       ord.need_start = std::max(ord.need_start, c->fence_e);
     slot = e % r->K;
     ws_off = (size_t)slot * r->slot_bytes;
+    if (k_new) {
+      // this call stores a tail row that the cache's next call reads from the tail buffer
+      c->fence_rec = (int)(r - g_rec);
+      c->fence_tag = r->tag;
+      c->fence_e = e + 1;
+      c->fence_capturing = capturing;
+    }
     r->ring[e % kRing] = me;
     r->e = e + 1;
     r->age = ++g_rec_clock;

@@ -84,13 +84,29 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
     const int np_max = cfg->max_prefill;
     size_t pre = align_up((size_t)np_max * 4, 256) +
                  (size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4;
-    // decode: partials [unit][item + tail][G][ZC_PART_STRIDE] + tail logits
-    // [unit][G][ZC_MAX_WINDOW]; twice the worst case, so that calls in flight together (each
-    // takes what its present number of items needs) find room
+    // decode: partials [unit][items + tail tiles][G][ZC_PART_STRIDE] + tail logits
+    // [unit][G][ZC_MAX_WINDOW] per call.  Calls in flight together take separate regions: room
+    // for kCallsInFlight calls of the largest plan this configuration produces, and never less
+    // than twice the worst case of any plan.
     const int max_items = std::min(ZC_MAX_ITEMS, 2 * ZC_MAX_SPLIT_HOST + 2 * max_flush);
-    size_t dec = align_up((size_t)lay->units * (max_items + 1) * lay->G * ZC_PART_STRIDE * 4, 256) +
-                 align_up((size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4, 256);
-    *ws_bytes = align_up(std::max(pre, 2 * dec), 512);
+    auto per_call = [&](int items) {
+      return align_up((size_t)lay->units * (items + ZC_MAX_WINDOW / ZC_SUB) * lay->G * ZC_PART_STRIDE * 4, 256) +
+             align_up((size_t)lay->units * lay->G * ZC_MAX_WINDOW * 4, 256);
+    };
+    zc_cache probe;   // the cache at its fullest, for the planner
+    memset(&probe, 0, sizeof(probe));
+    probe.cfg = *cfg;
+    probe.lay = *lay;
+    probe.l0 = cfg->max_prefill;
+    probe.n0[0] = ns_max;
+    probe.n0[1] = cfg->max_prefill - n_salient(cfg->saliency_ratio, cfg->max_prefill);
+    probe.nw[0] = ns_w;
+    probe.nw[1] = nr_w;
+    probe.n_seg = 1 + max_flush;
+    probe.n_sm = 148;
+    constexpr int kCallsInFlight = 16;
+    const size_t dec = std::max(2 * per_call(max_items), kCallsInFlight * per_call(zc_make_plan(&probe).items));
+    *ws_bytes = align_up(std::max(pre, dec), 512);
   }
 }
 
