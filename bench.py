@@ -108,8 +108,9 @@ class ClockSampler:
 
 # DRAM bytes of one k_decode launch (= one decode-attention call) measured with ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload id; the captures and their
-# conditions are in profiles/.  Empty entries: the kernel changed since the last capture.
-PROFILED_DRAM_BYTES_PER_DECODE_CALL = {}
+# conditions are in profiles/k_decode_config2.md and profiles/k_decode_config4.md (the first
+# decode steps after a prefill, when the tail holds a few tokens).
+PROFILED_DRAM_BYTES_PER_DECODE_CALL = {2: 28.18e6, 4: 449.2e6 + 17.3e6}
 
 
 def algorithmic_decode_bytes(w, n_windows: int, n_tail: int) -> int:
