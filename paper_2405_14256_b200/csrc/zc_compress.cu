@@ -258,7 +258,7 @@ __device__ __forceinline__ void quant_token(const float (&x)[4], const float (&c
 }
 
 template <typename T>
-__global__ void __launch_bounds__(256) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
+__global__ void __launch_bounds__(256, 3) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
   chain_link();
   __shared__ __align__(16) unsigned char codesK[ZC_TILE][ZC_D];
   __shared__ __align__(16) unsigned char codesV[ZC_TILE][ZC_D];
