@@ -135,7 +135,9 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
  * other aliasing, so q, k_new, v_new and out of calls issued back to back must not overlap
  * buffers that an earlier call of the stream still uses in any other way.  Kernels of other
  * libraries on the stream are ordered as usual.  The workspace must not be used by calls on
- * another stream at the same time. */
+ * another stream at the same time, and CUDA graphs captured from one stream must not be
+ * replayed at the same time on several streams (the calls of a capture share one ordering
+ * word per captured stream). */
 int zc_decode_attention(zc_cache* c, const void* q, void* out, int is_probe_step,
                         void* workspace, size_t workspace_bytes, zc_stream_t stream);
 
@@ -189,7 +191,8 @@ int64_t zc_launch_count(const zc_cache* c);
 
 /* Synchronises the device and reads the library's device-side error word into *code
  * [host]: 0 = none, 1 = a bounded wait on an asynchronous copy inside the decode kernel
- * ran out (its output is then invalid).  Device code never traps or spins forever. */
+ * ran out, 2 = a bounded wait for an earlier decode call of the stream ran out (outputs
+ * are then invalid).  Device code never traps or spins forever. */
 int zc_device_status(int* code);
 
 const char* zc_strerror(int status);
