@@ -191,8 +191,8 @@ int64_t zc_launch_count(const zc_cache* c);
 
 /* Synchronises the device and reads the library's device-side error word into *code
  * [host]: 0 = none, 1 = a bounded wait on an asynchronous copy inside the decode kernel
- * ran out, 2 = a bounded wait for an earlier decode call of the stream ran out (outputs
- * are then invalid).  Device code never traps or spins forever. */
+ * ran out, 2 = a bounded wait for an earlier decode call of the stream ran out, 3 = a bounded wait
+ * on the tensor cores inside a probe-score kernel ran out (outputs are then invalid).  Device code never traps or spins forever. */
 int zc_device_status(int* code);
 
 const char* zc_strerror(int status);

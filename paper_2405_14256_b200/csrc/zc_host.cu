@@ -507,6 +507,9 @@ int zc_device_status(int* code) {
   if (!code) return ZC_EINVAL;
   ZC_CUDA(cudaDeviceSynchronize());
   ZC_CUDA(zc_device_error_code(code));
+  int probe = 0;
+  ZC_CUDA(zc_probe_error_code(&probe));
+  if (*code == 0 && probe) *code = 3;
   return ZC_OK;
 }
 

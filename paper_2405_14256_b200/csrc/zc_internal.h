@@ -139,6 +139,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
 // Bytes of ws one call of `items` items per unit takes.
 size_t zc_decode_scratch_bytes(const zc_cache* c, int items);
 int zc_device_error_code(int* out);
+int zc_probe_error_code(int* out);   // 0 or 1: a bounded wait in a probe-score kernel ran out
 // Device address of the per-stream ordering words on the current device (looked up once per
 // device; pass nullptr to only perform the look-up).
 int zc_order_words(unsigned** ptr);

@@ -1,261 +1,382 @@
-// Probe attention (Eq. 9) and the normalised attention score (Eq. 8).
+// Probe attention (Eq. 9) and the normalised attention score (Eq. 8) on the 5th-generation
+// tensor cores: tcgen05.mma with both operands in shared memory and the 128 x 128 fp32
+// score tile in tensor memory (TMEM).
 //
 // Two passes over the probe rows, neither of which stores the n_probe x l matrix:
-//   pass 1  per (query head, 64 probe rows): log-sum-exp of each causal row;
-//   pass 2  per (KV head, 64 keys): column sums of exp(s - lse) over the G query heads
-//           and all probe rows that see the column, divided by G * nnz_j, where
-//           nnz_j = #{r : p_r >= j} is the structural count of unmasked rows.
-// Both passes are the same tensor-core contraction (warp-level m16n8k16 MMA, fp32
-// accumulate): a resident 64 x 128 A tile against streamed 64 x 128 B tiles.
+//   pass 1  per (group of query heads of one KV head, block of probe rows): log-sum-exp of
+//           each causal row.  A tile = 128 rows = Gt heads x 128/Gt probe rows, B tiles = 128
+//           keys each, streamed.
+//   pass 2  per (KV head, 128 keys): column sums of exp(s - lse) over the G query heads and
+//           all probe rows that see the column, divided by G * nnz_j (nnz_j = #{r : p_r >= j},
+//           the structural count of unmasked rows).  A tile = 128 keys, B tiles = 128 probe
+//           rows of one query head, streamed.
+// In both, D[m][n] = A[m] . B[n] lands in TMEM with row m in TMEM lane m, so after
+// tcgen05.ld every thread holds one row of the tile: row maxima, row sums (pass 1) and the
+// column sums of pass 2 (columns of the score matrix are the rows of its tile) need no
+// shuffle.  The MMA of tile i + 1 runs while the threads work on tile i (two TMEM buffers, two
+// B buffers).  Operand tiles are [2 k-blocks][128 rows][128 bytes] with the 128-byte swizzle
+// of the shared-memory matrix descriptor, written by cp.async.  Every wait is bounded; a wait
+// that runs out records an error code and the kernel still frees its TMEM.
+#include <type_traits>
 #include "zc_internal.h"
 #include "zc_layout.cuh"
 #include "zc_mma.cuh"
 
+__device__ int g_zc_probe_error = 0;
+
 namespace {
 
-constexpr int kRows = 64;                       // rows per tile
-constexpr int kTileBytes = kRows * ZC_D * 2;    // 16 KB
+constexpr int kM = 128;                          // rows of a tile (TMEM lanes)
+constexpr int kTile = kM * ZC_D * 2;             // 32 KB: [2][128][128 B]
+constexpr int kKBlock = kM * 128;                // bytes of one k-block of a tile
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kSpinLimit = 1 << 22;
+constexpr uint32_t kTmemCols = 256;              // two 128-column accumulators
 
-// 16-byte chunk `chunk` of row `row` inside a swizzled [64][128] 16-bit tile
-__device__ __forceinline__ char* tile_ptr(char* tile, int row, int chunk) {
-  return tile + row * 256 + ((chunk ^ (row & 7)) << 4);
+// 16-byte chunk `chunk` (0..15) of row `row` inside a tile
+__device__ __forceinline__ char* tile_chunk(char* tile, int row, int chunk) {
+  return tile + (chunk >> 3) * kKBlock + row * 128 + (((chunk & 7) ^ (row & 7)) << 4);
 }
-
-// Copy one 256-byte row (or zeros) into a tile; 16 threads per row.
-__device__ __forceinline__ void load_row_async(char* tile, int row, int chunk, const char* src) {
-  if (src) {
-    zc_cp_async16(tile_ptr(tile, row, chunk), src + chunk * 16);
-  } else {
-    *reinterpret_cast<uint4*>(tile_ptr(tile, row, chunk)) = make_uint4(0, 0, 0, 0);
+__device__ __forceinline__ void load_row(char* tile, int row, int chunk, const char* src) {
+  if (src) zc_cp_async16(tile_chunk(tile, row, chunk), src + chunk * 16);
+  else {
+    *reinterpret_cast<uint4*>(tile_chunk(tile, row, chunk)) = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");   // a plain store the tensor core will read
   }
 }
 
-__device__ __forceinline__ void load_a_frags(uint32_t (&a)[8][4], char* tile, int warp, int lane) {
-#pragma unroll
-  for (int ks = 0; ks < 8; ++ks)
-    zc_ldmatrix_x4(a[ks], tile_ptr(tile, warp * 16 + (lane & 15), 2 * ks + (lane >> 4)));
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes
+// apart; `addr` = shared address of the tile + k-block * kKBlock + (k16 step within it) * 32.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Instruction descriptor: fp32 accumulate, A and B of type T (0 = f16, 1 = bf16), both K-major,
+// N = 128, M = 128.
+template <typename T> __device__ __forceinline__ uint32_t instr_desc() {
+  const uint32_t fmt = std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// acc[nt][.] (16 x 64 per warp) = A(16 x 128) * B(64 x 128)^T
-template <typename T>
-__device__ __forceinline__ void block_mma(float (&acc)[8][4], const uint32_t (&a)[8][4],
-                                          char* btile, int lane) {
-#pragma unroll
-  for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+__device__ __forceinline__ void mma_tile(uint32_t tmem_d, uint32_t a_addr, uint32_t b_addr, uint32_t idesc) {
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) {
-#pragma unroll
-    for (int np = 0; np < 4; ++np) {
-      uint32_t b[4];
-      const int row = np * 16 + (lane & 7) + ((lane >> 4) << 3);
-      zc_ldmatrix_x4(b, tile_ptr(btile, row, 2 * ks + ((lane >> 3) & 1)));
-      zc_mma16816<T>(acc[2 * np], a[ks], b[0], b[1]);
-      zc_mma16816<T>(acc[2 * np + 1], a[ks], b[2], b[3]);
-    }
+    const uint32_t off = (ks >> 2) * kKBlock + (ks & 3) * 32;
+    const uint64_t da = smem_desc(a_addr + off), db = smem_desc(b_addr + off);
+    const uint32_t acc = ks > 0 ? 1u : 0u;
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n}\n" ::"r"(tmem_d),
+        "l"(da), "l"(db), "r"(idesc), "r"(acc), "r"(0u)
+        : "memory");
   }
+}
+__device__ __forceinline__ void mma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(
+                   zc_smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void bar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(zc_smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ bool bar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(zc_smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void bar_wait(uint64_t* bar, uint32_t parity) {
+  for (int spins = 0; !bar_try(bar, parity); ++spins) {
+    if (spins > kSpinLimit) { atomicExch(&g_zc_probe_error, 1); break; }
+    // once a wait has run out somewhere the results are void: do not add to the delay
+    if ((spins & 1023) == 1023 && *reinterpret_cast<volatile int*>(&g_zc_probe_error)) break;
+  }
+}
+__device__ __forceinline__ void tmem_ld32_nowait(float* v, uint32_t taddr) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+// one thread's whole row of a 128-column accumulator: four loads in flight, one wait
+__device__ __forceinline__ void tmem_ld128(float (&v)[128], uint32_t taddr) {
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) tmem_ld32_nowait(v + 32 * q4, taddr + 32 * q4);
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void async_proxy_fence() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
+// What both kernels share: shared memory carved at a 1024-byte boundary, TMEM, barriers.
+// 160 threads: lane 0 of warp 0 issues the MMAs, warps 1..4 are the row workers (they also
+// copy the tiles into shared memory, 16 bytes per thread and row); worker warp w may touch
+// TMEM lanes 32 (w mod 4) .. +31, so together they cover the 128 rows of a tile.
+//   b_full[b]     all 128 workers' copies into B buffer b have landed (cp.async.mbarrier.arrive)
+//   mma_done[b]   the MMA into accumulator b has completed (tcgen05.commit): the workers may
+//                 read it, and the B buffer it read may be refilled
+//   tmem_free[b]  the four worker warps have read accumulator b: the next MMA may overwrite it
+constexpr int kThreads = 160;
+struct TcCtx {
+  char* As;
+  char* Bs;          // two tiles
+  uint64_t* mma_done;
+  uint64_t* tmem_free;
+  uint64_t* b_full;
+  uint32_t* tmem_slot;
+  char* extra;       // pass 2: probe positions and lse of the last kSide B tiles
+  uint32_t a_addr, b_addr, tmem;
+};
+constexpr int kSide = 8;           // per-column data of pass 2 is kept for 8 tiles (see k_probe_colsum)
+constexpr int kTcSmem = 3 * kTile + 1024 /* alignment */ + 128 /* barriers, tmem slot */ + kSide * kM * 8;
+
+__device__ __forceinline__ void bar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];\n" ::"r"(zc_smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ TcCtx tc_setup(char* raw) {
+  TcCtx c;
+  const uint32_t raw_u = zc_smem_u32(raw);
+  const uint32_t base_u = (raw_u + 1023u) & ~1023u;
+  char* base = raw + (base_u - raw_u);
+  c.As = base;
+  c.Bs = base + kTile;
+  c.mma_done = reinterpret_cast<uint64_t*>(base + 3 * kTile);
+  c.tmem_free = c.mma_done + 2;
+  c.b_full = c.mma_done + 4;
+  c.tmem_slot = reinterpret_cast<uint32_t*>(base + 3 * kTile + 96);
+  c.extra = base + 3 * kTile + 128;
+  c.a_addr = base_u;
+  c.b_addr = base_u + kTile;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      bar_init(&c.mma_done[i], 1);
+      bar_init(&c.tmem_free[i], 4);
+      bar_init(&c.b_full[i], kM);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+  }
+  if (threadIdx.x < 32) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(
+                     zc_smem_u32(c.tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  c.tmem = *reinterpret_cast<volatile uint32_t*>(c.tmem_slot);
+  return c;
+}
+__device__ __forceinline__ void tc_teardown(const TcCtx& c) {
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x < 32)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(c.tmem), "r"(kTmemCols) : "memory");
+}
+
+// Tile `cb` goes into B buffer cb & 1 and accumulator cb & 1.
+// The issuing thread: for every tile, wait until its operands are in shared memory and its
+// accumulator has been read, then issue its MMAs.
+__device__ __forceinline__ void issue_loop(const TcCtx& c, int n, uint32_t idesc) {
+  for (int cb = 0; cb < n; ++cb) {
+    const int buf = cb & 1;
+    bar_wait(&c.b_full[buf], (uint32_t)(cb >> 1) & 1u);
+    async_proxy_fence();
+    if (cb >= 2) bar_wait(&c.tmem_free[buf], (uint32_t)((cb - 2) >> 1) & 1u);
+    tc_fence_after();
+    mma_tile(c.tmem + (uint32_t)buf * kM, c.a_addr, c.b_addr + buf * kTile, idesc);
+    mma_commit(&c.mma_done[buf]);
+  }
+}
+// A worker has issued its copies of a tile: the barrier gets this thread's arrival when they land.
+__device__ __forceinline__ void copies_arrive(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(zc_smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
+
+// Worker: waits for tile cb's accumulator and fetches this thread's row of it.
+__device__ __forceinline__ void worker_fetch(const TcCtx& c, int cb, int quarter, float (&v)[kM]) {
+  const int buf = cb & 1;
+  bar_wait(&c.mma_done[buf], (uint32_t)(cb >> 1) & 1u);
+  tc_fence_after();
+  tmem_ld128(v, c.tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kM);
+  tc_fence_before();
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) bar_arrive(&c.tmem_free[buf]);
 }
 
 // ---- pass 1: row log-sum-exp (base 2) of the causal probe rows ----
+// grid.x: blocks of rph = 128 / Gt probe rows, longest first; grid.y: (batch, group of Gt query heads).
 template <typename T>
-__global__ void __launch_bounds__(128) k_probe_lse(const T* __restrict__ Q, const T* __restrict__ K,
-                                                   const int32_t* __restrict__ P, int n_probe, int l,
-                                                   int h_q, int G, long long qsb, long long qsh,
-                                                   long long qsl, long long ksb, long long ksh,
-                                                   long long ksl, float* __restrict__ lse) {
-  extern __shared__ __align__(128) char smem[];
-  char* As = smem;
-  char* Bs = smem + kTileBytes;  // two buffers
+__global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__ Q, const T* __restrict__ K,
+                                                             const int32_t* __restrict__ P, int n_probe, int l,
+                                                             int h_q, int G, int Gt, long long qsb,
+                                                             long long qsh, long long qsl, long long ksb,
+                                                             long long ksh, long long ksl,
+                                                             float* __restrict__ lse) {
+  extern __shared__ char smem_raw[];
+  TcCtx c = tc_setup(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int r0 = blockIdx.x * kRows;
-  const int bh = blockIdx.y, b = bh / h_q, h = bh % h_q, kv = h / G;
-  const char* Qb = reinterpret_cast<const char*>(Q + b * qsb + h * qsh);
-  const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
-  const int row_ld = tid >> 4, chunk = tid & 15;  // 8 rows per pass of 128 threads
-
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int row = row_ld + 8 * i, r = r0 + row;
-    load_row_async(As, row, chunk, r < n_probe ? Qb + (long long)P[r] * qsl * 2 : nullptr);
-  }
-  const int p_last = P[min(r0 + kRows - 1, n_probe - 1)];
-  const int n_cb = p_last / kRows + 1;
-  auto load_b = [&](int cb, int buf) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int row = row_ld + 8 * i, j = cb * kRows + row;
-      load_row_async(Bs + buf * kTileBytes, row, chunk, j < l ? Kb + (long long)j * ksl * 2 : nullptr);
+  const int rph = kM / Gt;
+  const int r0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * rph;   // rows ascend in position: long blocks first
+  const int groups = h_q / Gt;
+  const int b = blockIdx.y / groups, hg = blockIdx.y % groups, h0 = hg * Gt, kv = h0 / G;
+  const int p_last = P[min(r0 + rph - 1, n_probe - 1)];
+  const int n_cb = p_last / kM + 1;
+  if (warp == 0) {
+    if (lane == 0) issue_loop(c, n_cb, instr_desc<T>());
+  } else {
+    const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
+    const int quarter = warp & 3, row = quarter * 32 + lane;
+    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the 128 workers
+    auto load_b = [&](int cb) {   // tile cb's keys into B buffer cb & 1
+#pragma unroll 4
+      for (int i = 0; i < 16; ++i) {
+        const int rw = row_ld + 8 * i, j = cb * kM + rw;
+        load_row(c.Bs + (cb & 1) * kTile, rw, chunk, j < l ? Kb + (long long)j * ksl * 2 : nullptr);
+      }
+      copies_arrive(&c.b_full[cb & 1]);
+    };
+    // A: the block's probe rows of the Gt heads (it lands with tile 0)
+#pragma unroll 4
+    for (int i = 0; i < 16; ++i) {
+      const int rw = row_ld + 8 * i, hl = rw / rph, r = r0 + rw % rph;
+      const char* src = nullptr;
+      if (r < n_probe) src = reinterpret_cast<const char*>(Q + b * qsb + (h0 + hl) * qsh) + (long long)P[r] * qsl * 2;
+      load_row(c.As, rw, chunk, src);
     }
-  };
-  load_b(0, 0);
-  zc_cp_async_commit();
-
-  const int g = lane >> 2, t = lane & 3;
-  const int ra = r0 + warp * 16 + g, rb = ra + 8;
-  const int pa = ra < n_probe ? P[ra] : -1, pb = rb < n_probe ? P[rb] : -1;
-  float m_a = -INFINITY, m_b = -INFINITY, s_a = 0.f, s_b = 0.f;
-  const float scale = kLog2e * rsqrtf((float)ZC_D);
-  uint32_t a[8][4];
-  float acc[8][4];
-  for (int cb = 0; cb < n_cb; ++cb) {
-    if (cb + 1 < n_cb) load_b(cb + 1, (cb + 1) & 1);
-    zc_cp_async_commit();
-    zc_cp_async_wait<1>();
-    __syncthreads();
-    if (cb == 0) load_a_frags(a, As, warp, lane);
-    block_mma<T>(acc, a, Bs + (cb & 1) * kTileBytes, lane);
-    float mx_a = -INFINITY, mx_b = -INFINITY;
+    load_b(0);
+    if (n_cb > 1) load_b(1);
+    const int my_r = r0 + row % rph;
+    const int my_p = my_r < n_probe ? P[my_r] : -1;
+    const float scale = kLog2e * rsqrtf((float)ZC_D);
+    float m_run = -INFINITY, s_run = 0.f;
+    for (int cb = 0; cb < n_cb; ++cb) {
+      float v[kM];
+      worker_fetch(c, cb, quarter, v);
+      if (cb + 2 < n_cb) load_b(cb + 2);   // its buffer was read by the MMA that has just completed
+      const int j_base = cb * kM;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (j_base + kM - 1 <= my_p) {
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
+        for (int e = 0; e < kM; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
+      } else {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int j = cb * kRows + nt * 8 + 2 * t + e;
-        acc[nt][e] = j <= pa ? acc[nt][e] * scale : -INFINITY;
-        acc[nt][2 + e] = j <= pb ? acc[nt][2 + e] * scale : -INFINITY;
-        mx_a = fmaxf(mx_a, acc[nt][e]);
-        mx_b = fmaxf(mx_b, acc[nt][2 + e]);
+        for (int e = 0; e < kM; ++e) {
+          if (j_base + e > my_p) v[e] = -INFINITY;
+          mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
+        }
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      const float mn = fmaxf(m_run, mx * scale);
+      if (mn != -INFINITY) {
+        float add[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int e = 0; e < kM; ++e) add[e & 3] += zc_exp2(fmaf(v[e], scale, -mn));
+        s_run = s_run * zc_exp2(m_run - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
+        m_run = mn;
       }
     }
-    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 1));
-    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, 2));
-    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 1));
-    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, 2));
-    const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
-    // a row with no visible column yet keeps (m, s) = (-inf, 0)
-    const float ca = mn_a == -INFINITY ? 0.f : zc_exp2(m_a - mn_a);
-    const float cbf = mn_b == -INFINITY ? 0.f : zc_exp2(m_b - mn_b);
-    const float ba = mn_a == -INFINITY ? 0.f : mn_a, bb = mn_b == -INFINITY ? 0.f : mn_b;
-    float add_a = 0.f, add_b = 0.f;
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        add_a += zc_exp2(acc[nt][e] - ba);
-        add_b += zc_exp2(acc[nt][2 + e] - bb);
-      }
-    }
-    s_a = s_a * ca + add_a;
-    s_b = s_b * cbf + add_b;
-    m_a = mn_a;
-    m_b = mn_b;
-    __syncthreads();
+    if (my_r < n_probe) lse[((long long)b * h_q + h0 + row / rph) * n_probe + my_r] = m_run + log2f(s_run);
   }
-  s_a += __shfl_xor_sync(0xffffffffu, s_a, 1);
-  s_a += __shfl_xor_sync(0xffffffffu, s_a, 2);
-  s_b += __shfl_xor_sync(0xffffffffu, s_b, 1);
-  s_b += __shfl_xor_sync(0xffffffffu, s_b, 2);
-  if (t == 0) {
-    if (ra < n_probe) lse[(long long)bh * n_probe + ra] = m_a + log2f(s_a);
-    if (rb < n_probe) lse[(long long)bh * n_probe + rb] = m_b + log2f(s_b);
-  }
+  tc_teardown(c);
 }
 
 // ---- pass 2: column sums of the normalised probe rows -> p_tilde ----
+// grid.x: blocks of 128 keys; grid.y: unit (batch, KV head).  B tiles: for every query head of
+// the KV head, the probe rows from the first one that sees key j0 on, 128 at a time.
 template <typename T>
-__global__ void __launch_bounds__(128) k_probe_colsum(const T* __restrict__ Q, const T* __restrict__ K,
-                                                      const int32_t* __restrict__ P, int n_probe, int l,
-                                                      int h_q, int n_kv, int G, long long qsb,
-                                                      long long qsh, long long qsl, long long ksb,
-                                                      long long ksh, long long ksl,
-                                                      const float* __restrict__ lse, char* cache,
-                                                      long long unit_stride, long long off_scores) {
-  extern __shared__ __align__(128) char smem[];
-  char* As = smem;
-  char* Bs = smem + kTileBytes;
-  int* Pp = reinterpret_cast<int*>(smem + 3 * kTileBytes);          // [2][64]
-  float* Ll = reinterpret_cast<float*>(smem + 3 * kTileBytes + 512);  // [2][64]
-  __shared__ int s_rstart;
+__global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
+    const T* __restrict__ Q, const T* __restrict__ K, const int32_t* __restrict__ P, int n_probe, int l,
+    int h_q, int n_kv, int G, long long qsb, long long qsh, long long qsl, long long ksb, long long ksh,
+    long long ksl, const float* __restrict__ lse, char* cache, long long unit_stride, long long off_scores) {
+  extern __shared__ char smem_raw[];
+  TcCtx c = tc_setup(smem_raw);
+  // Per-column data of a B tile (probe position and lse of each of its rows), slot = tile mod 8,
+  // written by the workers two tiles ahead of its use; they meet at a barrier of their own once
+  // per tile, so no warp is more than one tile ahead of another.
+  int* Pp = reinterpret_cast<int*>(c.extra);                      // [kSide][128]
+  float* Ll = reinterpret_cast<float*>(c.extra + kSide * kM * 4);  // [kSide][128]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int j0 = blockIdx.x * kRows;
+  const int j0 = blockIdx.x * kM;
   const int unit = blockIdx.y, b = unit / n_kv, kv = unit % n_kv;
-  const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
-  const int row_ld = tid >> 4, chunk = tid & 15;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int row = row_ld + 8 * i, j = j0 + row;
-    load_row_async(As, row, chunk, j < l ? Kb + (long long)j * ksl * 2 : nullptr);
+  int lo = 0, hi = n_probe;   // first probe row that sees column j0
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (P[mid] < j0) lo = mid + 1; else hi = mid;
   }
-  if (tid == 0) {  // first probe row that sees column j0
-    int lo = 0, hi = n_probe;
-    while (lo < hi) {
-      int mid = (lo + hi) >> 1;
-      if (P[mid] < j0) lo = mid + 1; else hi = mid;
-    }
-    s_rstart = lo;
-  }
-  __syncthreads();
-  const int r_start = s_rstart;
-  const int n_rb = (n_probe - r_start + kRows - 1) / kRows;
+  const int r_start = lo;
+  const int n_rb = (n_probe - r_start + kM - 1) / kM;
   const int n_tiles = n_rb * G;
-  auto load_b = [&](int tile, int buf) {
-    const int gq = tile / n_rb, rb = tile % n_rb;
-    const char* Qb = reinterpret_cast<const char*>(Q + b * qsb + (kv * G + gq) * qsh);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int row = row_ld + 8 * i, r = r_start + rb * kRows + row;
-      load_row_async(Bs + buf * kTileBytes, row, chunk,
-                     r < n_probe ? Qb + (long long)P[r] * qsl * 2 : nullptr);
+  if (warp == 0) {
+    if (lane == 0) issue_loop(c, n_tiles, instr_desc<T>());
+  } else {
+    const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
+    const int quarter = warp & 3, row = quarter * 32 + lane;
+    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the 128 workers
+    auto load_b = [&](int tile) {   // tile's probe rows into B buffer tile & 1, its per-column data into its slot
+      const int gq = tile / n_rb, rb = tile % n_rb;
+      const char* Qb = reinterpret_cast<const char*>(Q + b * qsb + (kv * G + gq) * qsh);
+#pragma unroll 4
+      for (int i = 0; i < 16; ++i) {
+        const int rw = row_ld + 8 * i, r = r_start + rb * kM + rw;
+        load_row(c.Bs + (tile & 1) * kTile, rw, chunk, r < n_probe ? Qb + (long long)P[r] * qsl * 2 : nullptr);
+      }
+      copies_arrive(&c.b_full[tile & 1]);
+      const int slot = tile & (kSide - 1), r = r_start + rb * kM + wt;
+      Pp[slot * kM + wt] = r < n_probe ? P[r] : -1;
+      Ll[slot * kM + wt] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
+    };
+#pragma unroll 4
+    for (int i = 0; i < 16; ++i) {
+      const int rw = row_ld + 8 * i, jj = j0 + rw;
+      load_row(c.As, rw, chunk, jj < l ? Kb + (long long)jj * ksl * 2 : nullptr);
     }
-    if (tid < kRows) {
-      const int r = r_start + rb * kRows + tid;
-      Pp[buf * kRows + tid] = r < n_probe ? P[r] : -1;
-      Ll[buf * kRows + tid] =
-          r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
-    }
-  };
-  if (n_tiles > 0) load_b(0, 0);
-  zc_cp_async_commit();
-  const int g = lane >> 2, t = lane & 3;
-  const int ja = j0 + warp * 16 + g, jb = ja + 8;
-  const float scale = kLog2e * rsqrtf((float)ZC_D);
-  float sum_a = 0.f, sum_b = 0.f;
-  uint32_t a[8][4];
-  float acc[8][4];
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    if (tile + 1 < n_tiles) load_b(tile + 1, (tile + 1) & 1);
-    zc_cp_async_commit();
-    zc_cp_async_wait<1>();
-    __syncthreads();
-    if (tile == 0) load_a_frags(a, As, warp, lane);
-    const int buf = tile & 1;
-    block_mma<T>(acc, a, Bs + buf * kTileBytes, lane);
+    load_b(0);
+    if (n_tiles > 1) load_b(1);
+    workers_sync();   // per-column data of tiles 0 and 1 is visible to all workers
+    const int j = j0 + row;
+    const float scale = kLog2e * rsqrtf((float)ZC_D);
+    float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int slot = tile & (kSide - 1);
+      float v[kM];
+      worker_fetch(c, tile, quarter, v);
+      if (tile + 2 < n_tiles) load_b(tile + 2);   // its buffer was read by the MMA that has just completed
+      workers_sync();   // per-column data written here is read two iterations on; the warps stay in step
+      const int* pp = Pp + slot * kM;
+      const float* ll = Ll + slot * kM;
+      if (j <= pp[0]) {   // probe rows ascend in position: every row of the tile sees column j
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
+        for (int e = 0; e < kM; ++e) sum4[e & 3] += zc_exp2(fmaf(v[e], scale, -ll[e]));
+      } else {
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int col = nt * 8 + 2 * t + e;
-        const int p = Pp[buf * kRows + col];
-        const float ls = Ll[buf * kRows + col];
-        sum_a += ja <= p ? zc_exp2(acc[nt][e] * scale - ls) : 0.f;
-        sum_b += jb <= p ? zc_exp2(acc[nt][2 + e] * scale - ls) : 0.f;
+        for (int e = 0; e < kM; ++e) sum4[e & 3] += j <= pp[e] ? zc_exp2(fmaf(v[e], scale, -ll[e])) : 0.f;
       }
     }
-    __syncthreads();
-  }
-  sum_a += __shfl_xor_sync(0xffffffffu, sum_a, 1);
-  sum_a += __shfl_xor_sync(0xffffffffu, sum_a, 2);
-  sum_b += __shfl_xor_sync(0xffffffffu, sum_b, 1);
-  sum_b += __shfl_xor_sync(0xffffffffu, sum_b, 2);
-  if (t == 0) {
-    float* scores = reinterpret_cast<float*>(cache + unit * unit_stride + off_scores);
-    const int js[2] = {ja, jb};
-    const float sums[2] = {sum_a, sum_b};
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const int j = js[k];
-      if (j < l) {
-        int lo = r_start, hi = n_probe;  // rows with p_r >= j
-        while (lo < hi) {
-          int mid = (lo + hi) >> 1;
-          if (P[mid] < j) lo = mid + 1; else hi = mid;
-        }
-        const int nnz = n_probe - lo;
-        scores[j] = __fdiv_rn(sums[k], (float)(G * nnz));
+    if (j < l) {
+      int lo2 = r_start, hi2 = n_probe;   // rows with p_r >= j
+      while (lo2 < hi2) {
+        const int mid = (lo2 + hi2) >> 1;
+        if (P[mid] < j) lo2 = mid + 1; else hi2 = mid;
       }
+      float* scores = reinterpret_cast<float*>(cache + unit * unit_stride + off_scores);
+      scores[j] = __fdiv_rn((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]), (float)(G * (n_probe - lo2)));
     }
   }
+  tc_teardown(c);
 }
 
 }  // namespace
@@ -265,27 +386,31 @@ int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, con
                            cudaStream_t st) {
   const zc_config& cfg = c->cfg;
   const int G = c->lay.G;
-  const int smem1 = 3 * kTileBytes, smem2 = 3 * kTileBytes + 1024;
-  dim3 g1(zc_ceil_div(n_probe, kRows), cfg.batch * cfg.n_q_heads);
-  dim3 g2(zc_ceil_div(l, kRows), c->lay.units);
+  const int Gt = (G % 4 == 0) ? 4 : ((G % 2 == 0) ? 2 : 1);
+  const int rph = kM / Gt;
+  dim3 g1(zc_ceil_div(n_probe, rph), cfg.batch * (cfg.n_q_heads / Gt));
+  dim3 g2(zc_ceil_div(l, kM), c->lay.units);
   cudaError_t e;
-#define ZC_GO(T)                                                                                   \
-  do {                                                                                             \
-    e = cudaFuncSetAttribute(k_probe_lse<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem1);   \
-    if (e != cudaSuccess) return e;                                                                \
-    e = cudaFuncSetAttribute(k_probe_colsum<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,        \
-                             smem2);                                                               \
-    if (e != cudaSuccess) return e;                                                                \
-    k_probe_lse<T><<<g1, 128, smem1, st>>>((const T*)Q, (const T*)K, P_dev, n_probe, l,            \
-                                           cfg.n_q_heads, G, qs[0], qs[1], qs[2], ks[0], ks[1],    \
-                                           ks[2], lse_ws);                                         \
-    k_probe_colsum<T><<<g2, 128, smem2, st>>>((const T*)Q, (const T*)K, P_dev, n_probe, l,         \
-                                              cfg.n_q_heads, cfg.n_kv_heads, G, qs[0], qs[1],      \
-                                              qs[2], ks[0], ks[1], ks[2], lse_ws, c->base,         \
-                                              c->lay.unit_stride, c->lay.off_scores);              \
+#define ZC_GO(T)                                                                                       \
+  do {                                                                                                 \
+    e = cudaFuncSetAttribute(k_probe_lse<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);  \
+    if (e != cudaSuccess) return e;                                                                    \
+    e = cudaFuncSetAttribute(k_probe_colsum<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem); \
+    if (e != cudaSuccess) return e;                                                                    \
+    k_probe_lse<T><<<g1, kThreads, kTcSmem, st>>>((const T*)Q, (const T*)K, P_dev, n_probe, l,      \
+                                                     cfg.n_q_heads, G, Gt, qs[0], qs[1], qs[2], ks[0], \
+                                                     ks[1], ks[2], lse_ws);                            \
+    k_probe_colsum<T><<<g2, kThreads, kTcSmem, st>>>((const T*)Q, (const T*)K, P_dev, n_probe, l,   \
+                                                        cfg.n_q_heads, cfg.n_kv_heads, G, qs[0], qs[1], \
+                                                        qs[2], ks[0], ks[1], ks[2], lse_ws, c->base,   \
+                                                        c->lay.unit_stride, c->lay.off_scores);        \
   } while (0)
   if (cfg.dtype == ZC_F16) ZC_GO(__half); else ZC_GO(__nv_bfloat16);
 #undef ZC_GO
   c->launches += 2;
   return cudaGetLastError();
+}
+
+int zc_probe_error_code(int* out) {
+  return (int)cudaMemcpyFromSymbol(out, g_zc_probe_error, sizeof(int));
 }
