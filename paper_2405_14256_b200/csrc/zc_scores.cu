@@ -15,8 +15,12 @@
 // column sums of pass 2 (columns of the score matrix are the rows of its tile) need no
 // shuffle.  The MMA of tile i + 1 runs while the threads work on tile i (two TMEM buffers, two
 // B buffers).  Operand tiles are [2 k-blocks][128 rows][128 bytes] with the 128-byte swizzle
-// of the shared-memory matrix descriptor, written by cp.async.  Every wait is bounded; a wait
-// that runs out records an error code and the kernel still frees its TMEM.
+// of the shared-memory matrix descriptor.  Tiles of consecutive keys come in by tensor-map bulk
+// copies (TMA, hardware swizzle) issued by the MMA thread; tiles of gathered probe rows are
+// written by the workers with cp.async.  Every wait is bounded; a wait that runs out records
+// an error code and the kernel still frees its TMEM.
+#include <cuda.h>
+#include <cstring>
 #include <type_traits>
 #include "zc_internal.h"
 #include "zc_layout.cuh"
@@ -121,7 +125,9 @@ __device__ __forceinline__ void async_proxy_fence() { asm volatile("fence.proxy.
 // 160 threads: lane 0 of warp 0 issues the MMAs, warps 1..4 are the row workers (they also
 // copy the tiles into shared memory, 16 bytes per thread and row); worker warp w may touch
 // TMEM lanes 32 (w mod 4) .. +31, so together they cover the 128 rows of a tile.
-//   b_full[b]     all 128 workers' copies into B buffer b have landed (cp.async.mbarrier.arrive)
+//   a_full        the A tile has landed
+//   b_full[b]     B buffer b has been filled: by all 128 workers' copies
+//                 (cp.async.mbarrier.arrive) or by the bulk copies (complete_tx)
 //   mma_done[b]   the MMA into accumulator b has completed (tcgen05.commit): the workers may
 //                 read it, and the B buffer it read may be refilled
 //   tmem_free[b]  the four worker warps have read accumulator b: the next MMA may overwrite it
@@ -132,6 +138,7 @@ struct TcCtx {
   uint64_t* mma_done;
   uint64_t* tmem_free;
   uint64_t* b_full;
+  uint64_t* a_full;
   uint32_t* tmem_slot;
   char* extra;       // pass 2: probe positions and lse of the last kSide B tiles
   uint32_t a_addr, b_addr, tmem;
@@ -143,7 +150,7 @@ __device__ __forceinline__ void bar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];\n" ::"r"(zc_smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ TcCtx tc_setup(char* raw) {
+__device__ __forceinline__ TcCtx tc_setup(char* raw, int a_count, int b_count) {
   TcCtx c;
   const uint32_t raw_u = zc_smem_u32(raw);
   const uint32_t base_u = (raw_u + 1023u) & ~1023u;
@@ -153,6 +160,7 @@ __device__ __forceinline__ TcCtx tc_setup(char* raw) {
   c.mma_done = reinterpret_cast<uint64_t*>(base + 3 * kTile);
   c.tmem_free = c.mma_done + 2;
   c.b_full = c.mma_done + 4;
+  c.a_full = c.mma_done + 6;
   c.tmem_slot = reinterpret_cast<uint32_t*>(base + 3 * kTile + 96);
   c.extra = base + 3 * kTile + 128;
   c.a_addr = base_u;
@@ -161,8 +169,9 @@ __device__ __forceinline__ TcCtx tc_setup(char* raw) {
     for (int i = 0; i < 2; ++i) {
       bar_init(&c.mma_done[i], 1);
       bar_init(&c.tmem_free[i], 4);
-      bar_init(&c.b_full[i], kM);
+      bar_init(&c.b_full[i], b_count);
     }
+    bar_init(c.a_full, a_count);
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
   if (threadIdx.x < 32) {
@@ -186,10 +195,28 @@ __device__ __forceinline__ void tc_teardown(const TcCtx& c) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(c.tmem), "r"(kTmemCols) : "memory");
 }
 
+// One 128-row tile of consecutive keys (rows j0 .. j0 + 127 of K[b][kv]) by two bulk tensor
+// copies (one per k-block); rows past the end of the tensor arrive as zeros.
+__device__ __forceinline__ void tma_key_tile(const CUtensorMap* map, uint32_t dst, uint64_t* bar, int j0,
+                                             int kv, int b) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(zc_smem_u32(bar)), "r"(kTile)
+               : "memory");
+#pragma unroll
+  for (int kb = 0; kb < 2; ++kb)
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], "
+        "[%6];\n" ::"r"(dst + kb * kKBlock),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(kb * 64), "r"(j0), "r"(kv), "r"(b), "r"(zc_smem_u32(bar))
+        : "memory");
+}
+
 // Tile `cb` goes into B buffer cb & 1 and accumulator cb & 1.
 // The issuing thread: for every tile, wait until its operands are in shared memory and its
-// accumulator has been read, then issue its MMAs.
-__device__ __forceinline__ void issue_loop(const TcCtx& c, int n, uint32_t idesc) {
+// accumulator has been read, then issue its MMAs.  refill(tile, buffer): called once the MMA
+// that read `buffer` has completed, for kernels whose B tiles this thread fetches itself.
+template <typename Refill>
+__device__ __forceinline__ void issue_loop(const TcCtx& c, int n, uint32_t idesc, bool refills, Refill refill) {
+  bar_wait(c.a_full, 0u);
   for (int cb = 0; cb < n; ++cb) {
     const int buf = cb & 1;
     bar_wait(&c.b_full[buf], (uint32_t)(cb >> 1) & 1u);
@@ -198,6 +225,10 @@ __device__ __forceinline__ void issue_loop(const TcCtx& c, int n, uint32_t idesc
     tc_fence_after();
     mma_tile(c.tmem + (uint32_t)buf * kM, c.a_addr, c.b_addr + buf * kTile, idesc);
     mma_commit(&c.mma_done[buf]);
+    if (refills && cb + 2 < n) {
+      bar_wait(&c.mma_done[buf], (uint32_t)(cb >> 1) & 1u);
+      refill(cb + 2, buf);
+    }
   }
 }
 // A worker has issued its copies of a tile: the barrier gets this thread's arrival when they land.
@@ -225,9 +256,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
                                                              int h_q, int G, int Gt, long long qsb,
                                                              long long qsh, long long qsl, long long ksb,
                                                              long long ksh, long long ksl,
-                                                             float* __restrict__ lse) {
+                                                             float* __restrict__ lse,
+                                                             const __grid_constant__ CUtensorMap kmap,
+                                                             int use_tma) {
   extern __shared__ char smem_raw[];
-  TcCtx c = tc_setup(smem_raw);
+  // A (gathered probe rows): the 128 workers' copies; B (key tiles): bulk copies, or the workers
+  TcCtx c = tc_setup(smem_raw, kM, use_tma ? 1 : kM);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rph = kM / Gt;
   const int r0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * rph;   // rows ascend in position: long blocks first
@@ -236,7 +270,14 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
   const int p_last = P[min(r0 + rph - 1, n_probe - 1)];
   const int n_cb = p_last / kM + 1;
   if (warp == 0) {
-    if (lane == 0) issue_loop(c, n_cb, instr_desc<T>());
+    if (lane == 0) {
+      auto fetch = [&](int cb, int buf) { tma_key_tile(&kmap, c.b_addr + buf * kTile, &c.b_full[buf], cb * kM, kv, b); };
+      if (use_tma) {
+        fetch(0, 0);
+        if (n_cb > 1) fetch(1, 1);
+      }
+      issue_loop(c, n_cb, instr_desc<T>(), use_tma != 0, fetch);
+    }
   } else {
     const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
     const int quarter = warp & 3, row = quarter * 32 + lane;
@@ -257,8 +298,11 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
       if (r < n_probe) src = reinterpret_cast<const char*>(Q + b * qsb + (h0 + hl) * qsh) + (long long)P[r] * qsl * 2;
       load_row(c.As, rw, chunk, src);
     }
-    load_b(0);
-    if (n_cb > 1) load_b(1);
+    copies_arrive(c.a_full);
+    if (!use_tma) {
+      load_b(0);
+      if (n_cb > 1) load_b(1);
+    }
     const int my_r = r0 + row % rph;
     const int my_p = my_r < n_probe ? P[my_r] : -1;
     const float scale = kLog2e * rsqrtf((float)ZC_D);
@@ -266,7 +310,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
     for (int cb = 0; cb < n_cb; ++cb) {
       float v[kM];
       worker_fetch(c, cb, quarter, v);
-      if (cb + 2 < n_cb) load_b(cb + 2);   // its buffer was read by the MMA that has just completed
+      if (!use_tma && cb + 2 < n_cb) load_b(cb + 2);   // its buffer was read by the MMA that has just completed
       const int j_base = cb * kM;
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       if (j_base + kM - 1 <= my_p) {
@@ -301,9 +345,11 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     const T* __restrict__ Q, const T* __restrict__ K, const int32_t* __restrict__ P, int n_probe, int l,
     int h_q, int n_kv, int G, long long qsb, long long qsh, long long qsl, long long ksb, long long ksh,
-    long long ksl, const float* __restrict__ lse, char* cache, long long unit_stride, long long off_scores) {
+    long long ksl, const float* __restrict__ lse, char* cache, long long unit_stride, long long off_scores,
+    const __grid_constant__ CUtensorMap kmap, int use_tma) {
   extern __shared__ char smem_raw[];
-  TcCtx c = tc_setup(smem_raw);
+  // A (the key block): one bulk copy, or the workers; B (gathered probe rows): the workers
+  TcCtx c = tc_setup(smem_raw, use_tma ? 1 : kM, kM);
   // Per-column data of a B tile (probe position and lse of each of its rows), slot = tile mod 8,
   // written by the workers two tiles ahead of its use; they meet at a barrier of their own once
   // per tile, so no warp is more than one tile ahead of another.
@@ -321,7 +367,10 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
   const int n_rb = (n_probe - r_start + kM - 1) / kM;
   const int n_tiles = n_rb * G;
   if (warp == 0) {
-    if (lane == 0) issue_loop(c, n_tiles, instr_desc<T>());
+    if (lane == 0) {
+      if (use_tma) tma_key_tile(&kmap, c.a_addr, c.a_full, j0, kv, b);
+      issue_loop(c, n_tiles, instr_desc<T>(), false, [](int, int) {});
+    }
   } else {
     const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
     const int quarter = warp & 3, row = quarter * 32 + lane;
@@ -339,10 +388,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
       Pp[slot * kM + wt] = r < n_probe ? P[r] : -1;
       Ll[slot * kM + wt] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
     };
+    if (!use_tma) {
 #pragma unroll 4
-    for (int i = 0; i < 16; ++i) {
-      const int rw = row_ld + 8 * i, jj = j0 + rw;
-      load_row(c.As, rw, chunk, jj < l ? Kb + (long long)jj * ksl * 2 : nullptr);
+      for (int i = 0; i < 16; ++i) {
+        const int rw = row_ld + 8 * i, jj = j0 + rw;
+        load_row(c.As, rw, chunk, jj < l ? Kb + (long long)jj * ksl * 2 : nullptr);
+      }
+      copies_arrive(c.a_full);
     }
     load_b(0);
     if (n_tiles > 1) load_b(1);
@@ -381,6 +433,46 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
 
 }  // namespace
 
+namespace {
+
+// Tensor map of K as (d, l, h_kv, b) with boxes of 64 elements x 128 rows in the 128-byte
+// swizzle; false when the driver entry point is missing or refuses the tensor (the kernels
+// then copy the key tiles themselves).
+bool make_key_map(CUtensorMap* map, const void* K, int dtype, int l, int n_kv, int batch, const int64_t* ks) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = nullptr;
+  static bool looked = false;
+  if (!looked) {
+    looked = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      encode = (EncodeFn)p;
+    else
+      cudaGetLastError();
+  }
+  if (!encode) return false;
+  const cuuint64_t dims[4] = {(cuuint64_t)ZC_D, (cuuint64_t)l, (cuuint64_t)n_kv, (cuuint64_t)batch};
+  // byte strides of dimensions 1..3; a dimension of extent 1 may come with any stride
+  cuuint64_t strides[3] = {(cuuint64_t)ks[2] * 2, (cuuint64_t)ks[1] * 2, (cuuint64_t)ks[0] * 2};
+  if (n_kv == 1 && strides[1] == 0) strides[1] = strides[0] * (cuuint64_t)l;
+  if (batch == 1 && strides[2] == 0) strides[2] = strides[1] * (cuuint64_t)n_kv;
+  for (int i = 0; i < 3; ++i)
+    if (strides[i] == 0 || (strides[i] & 15) || strides[i] >= ((cuuint64_t)1 << 40)) return false;
+  const cuuint32_t box[4] = {64, (cuuint32_t)kM, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  const CUresult r = encode(map, dtype == ZC_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                            4, const_cast<void*>(K), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, const int64_t* qs,
                            const int64_t* ks, const int32_t* P_dev, int n_probe, float* lse_ws,
                            cudaStream_t st) {
@@ -390,6 +482,9 @@ int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, con
   const int rph = kM / Gt;
   dim3 g1(zc_ceil_div(n_probe, rph), cfg.batch * (cfg.n_q_heads / Gt));
   dim3 g2(zc_ceil_div(l, kM), c->lay.units);
+  CUtensorMap kmap;
+  memset(&kmap, 0, sizeof(kmap));
+  const int use_tma = make_key_map(&kmap, K, cfg.dtype, l, cfg.n_kv_heads, cfg.batch, ks) ? 1 : 0;
   cudaError_t e;
 #define ZC_GO(T)                                                                                       \
   do {                                                                                                 \
@@ -399,11 +494,12 @@ int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, con
     if (e != cudaSuccess) return e;                                                                    \
     k_probe_lse<T><<<g1, kThreads, kTcSmem, st>>>((const T*)Q, (const T*)K, P_dev, n_probe, l,      \
                                                      cfg.n_q_heads, G, Gt, qs[0], qs[1], qs[2], ks[0], \
-                                                     ks[1], ks[2], lse_ws);                            \
+                                                     ks[1], ks[2], lse_ws, kmap, use_tma);             \
     k_probe_colsum<T><<<g2, kThreads, kTcSmem, st>>>((const T*)Q, (const T*)K, P_dev, n_probe, l,   \
                                                         cfg.n_q_heads, cfg.n_kv_heads, G, qs[0], qs[1], \
                                                         qs[2], ks[0], ks[1], ks[2], lse_ws, c->base,   \
-                                                        c->lay.unit_stride, c->lay.off_scores);        \
+                                                        c->lay.unit_stride, c->lay.off_scores, kmap,   \
+                                                        use_tma);                                      \
   } while (0)
   if (cfg.dtype == ZC_F16) ZC_GO(__half); else ZC_GO(__nv_bfloat16);
 #undef ZC_GO
