@@ -83,7 +83,10 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
     // prefill: probe positions + per-row log-sum-exp for every query head
     const int np_max = cfg->max_prefill;
     size_t pre = align_up((size_t)np_max * 4, 256) +
-                 (size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4;
+                 align_up((size_t)cfg->batch * cfg->n_q_heads * (size_t)np_max * 4, 256);
+    // ... and a dense copy of the probe rows for probe sets of up to an eighth of the context
+    // (larger sets are gathered tile by tile instead)
+    pre += (size_t)cfg->batch * cfg->n_q_heads * (size_t)std::max(512, cfg->max_prefill / 8) * ZC_D * 2;
     // decode: partials [unit][items + tail tiles][G][ZC_PART_STRIDE] + tail logits
     // [unit][G][ZC_MAX_WINDOW] per call.  Calls in flight together take separate regions: room
     // for kCallsInFlight calls of the largest plan this configuration produces, and never less
@@ -363,7 +366,11 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
     int32_t* P_dev = (int32_t*)workspace;
     float* lse = (float*)((char*)workspace + align_up((size_t)n_probe * 4, 256));
     ZC_CUDA(cudaMemcpyAsync(P_dev, probe_pos, (size_t)n_probe * 4, cudaMemcpyHostToDevice, st));
-    ZC_CUDA(zc_launch_probe_scores(c, Q, K, l, q_strides, kv_strides, P_dev, n_probe, lse, st));
+    const size_t used = align_up((size_t)n_probe * 4, 256) +
+                        align_up((size_t)c->cfg.batch * c->cfg.n_q_heads * (size_t)n_probe * 4, 256);
+    void* qp = used < workspace_bytes ? (char*)workspace + used : nullptr;
+    ZC_CUDA(zc_launch_probe_scores(c, Q, K, l, q_strides, kv_strides, P_dev, n_probe, lse, qp,
+                                   qp ? workspace_bytes - used : 0, st));
   }
   ZC_CUDA(zc_launch_topk(c, l, c->n0[0], 0, salient_idx, st));
   ZcSrc src{K, V, kv_strides[0], kv_strides[1], kv_strides[2]};

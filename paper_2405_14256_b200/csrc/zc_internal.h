@@ -116,9 +116,11 @@ ZcSeg zc_segment(const zc_cache* c, int seg);
 ZcDecodePlan zc_make_plan(const zc_cache* c);
 
 // ---- launchers (each returns a cudaError_t as int) ----
+// qp_ws / qp_bytes: room for a dense copy of the probe rows (batch * n_q_heads * n_probe rows of
+// 256 bytes, 16-byte aligned); used when large enough.
 int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l,
                            const int64_t* qs, const int64_t* ks, const int32_t* P_dev,
-                           int n_probe, float* lse_ws, cudaStream_t st);
+                           int n_probe, float* lse_ws, void* qp_ws, size_t qp_bytes, cudaStream_t st);
 // chained: launched as a link of the decode calls' chain on the stream (see zc_compress.cu);
 // the caller then fences the cache with zc_order_fence.
 int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,

@@ -195,8 +195,9 @@ __device__ __forceinline__ void tc_teardown(const TcCtx& c) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(c.tmem), "r"(kTmemCols) : "memory");
 }
 
-// One 128-row tile of consecutive keys (rows j0 .. j0 + 127 of K[b][kv]) by two bulk tensor
-// copies (one per k-block); rows past the end of the tensor arrive as zeros.
+// One 128-row tile of consecutive rows (rows j0 .. j0 + 127 of tensor[b][h]: keys, or the
+// gathered probe rows) by two bulk tensor copies (one per k-block); rows past the end of the
+// tensor arrive as zeros.
 __device__ __forceinline__ void tma_key_tile(const CUtensorMap* map, uint32_t dst, uint64_t* bar, int j0,
                                              int kv, int b) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(zc_smem_u32(bar)), "r"(kTile)
@@ -346,10 +347,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     const T* __restrict__ Q, const T* __restrict__ K, const int32_t* __restrict__ P, int n_probe, int l,
     int h_q, int n_kv, int G, long long qsb, long long qsh, long long qsl, long long ksb, long long ksh,
     long long ksl, const float* __restrict__ lse, char* cache, long long unit_stride, long long off_scores,
-    const __grid_constant__ CUtensorMap kmap, int use_tma) {
+    const __grid_constant__ CUtensorMap kmap, int use_tma, const __grid_constant__ CUtensorMap qmap,
+    int use_qp) {
   extern __shared__ char smem_raw[];
-  // A (the key block): one bulk copy, or the workers; B (gathered probe rows): the workers
-  TcCtx c = tc_setup(smem_raw, use_tma ? 1 : kM, kM);
+  // A (the key block): one bulk copy, or the workers; B (probe rows): bulk copies from the
+  // gathered copy of the probe rows when there is one (qmap), else the workers gather them
+  TcCtx c = tc_setup(smem_raw, use_tma ? 1 : kM, use_qp ? 1 : kM);
   // Per-column data of a B tile (probe position and lse of each of its rows), slot = tile mod 8,
   // written by the workers two tiles ahead of its use; they meet at a barrier of their own once
   // per tile, so no warp is more than one tile ahead of another.
@@ -369,7 +372,15 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
   if (warp == 0) {
     if (lane == 0) {
       if (use_tma) tma_key_tile(&kmap, c.a_addr, c.a_full, j0, kv, b);
-      issue_loop(c, n_tiles, instr_desc<T>(), false, [](int, int) {});
+      auto fetch = [&](int tile, int buf) {
+        const int gq = tile / n_rb, rb = tile % n_rb;
+        tma_key_tile(&qmap, c.b_addr + buf * kTile, &c.b_full[buf], r_start + rb * kM, kv * G + gq, b);
+      };
+      if (use_qp) {
+        fetch(0, 0);
+        if (n_tiles > 1) fetch(1, 1);
+      }
+      issue_loop(c, n_tiles, instr_desc<T>(), use_qp != 0, fetch);
     }
   } else {
     const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
@@ -377,13 +388,15 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the 128 workers
     auto load_b = [&](int tile) {   // tile's probe rows into B buffer tile & 1, its per-column data into its slot
       const int gq = tile / n_rb, rb = tile % n_rb;
-      const char* Qb = reinterpret_cast<const char*>(Q + b * qsb + (kv * G + gq) * qsh);
+      if (!use_qp) {
+        const char* Qb = reinterpret_cast<const char*>(Q + b * qsb + (kv * G + gq) * qsh);
 #pragma unroll 4
-      for (int i = 0; i < 16; ++i) {
-        const int rw = row_ld + 8 * i, r = r_start + rb * kM + rw;
-        load_row(c.Bs + (tile & 1) * kTile, rw, chunk, r < n_probe ? Qb + (long long)P[r] * qsl * 2 : nullptr);
+        for (int i = 0; i < 16; ++i) {
+          const int rw = row_ld + 8 * i, r = r_start + rb * kM + rw;
+          load_row(c.Bs + (tile & 1) * kTile, rw, chunk, r < n_probe ? Qb + (long long)P[r] * qsl * 2 : nullptr);
+        }
+        copies_arrive(&c.b_full[tile & 1]);
       }
-      copies_arrive(&c.b_full[tile & 1]);
       const int slot = tile & (kSide - 1), r = r_start + rb * kM + wt;
       Pp[slot * kM + wt] = r < n_probe ? P[r] : -1;
       Ll[slot * kM + wt] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
@@ -435,6 +448,19 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
 
 namespace {
 
+// Dense copy of the probe rows, Qp[b][h][r] = Q[b][h][P[r]]: pass 2 streams its tiles from it
+// with bulk copies.  8 rows per CTA, 16 threads x 16 bytes per row.
+template <typename T>
+__global__ void k_gather_probe_rows(const T* __restrict__ Q, const int32_t* __restrict__ P, int n_probe,
+                                    int h_q, long long qsb, long long qsh, long long qsl,
+                                    T* __restrict__ Qp) {
+  const int r = blockIdx.x * 8 + (threadIdx.x >> 4), ch = threadIdx.x & 15;
+  if (r >= n_probe) return;
+  const int b = blockIdx.y / h_q, h = blockIdx.y % h_q;
+  const uint4 v = *(reinterpret_cast<const uint4*>(Q + b * qsb + h * qsh + (long long)P[r] * qsl) + ch);
+  *(reinterpret_cast<uint4*>(Qp + ((long long)blockIdx.y * n_probe + r) * ZC_D) + ch) = v;
+}
+
 // Tensor map of K as (d, l, h_kv, b) with boxes of 64 elements x 128 rows in the 128-byte
 // swizzle; false when the driver entry point is missing or refuses the tensor (the kernels
 // then copy the key tiles themselves).
@@ -475,7 +501,7 @@ bool make_key_map(CUtensorMap* map, const void* K, int dtype, int l, int n_kv, i
 
 int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, const int64_t* qs,
                            const int64_t* ks, const int32_t* P_dev, int n_probe, float* lse_ws,
-                           cudaStream_t st) {
+                           void* qp_ws, size_t qp_bytes, cudaStream_t st) {
   const zc_config& cfg = c->cfg;
   const int G = c->lay.G;
   const int Gt = (G % 4 == 0) ? 4 : ((G % 2 == 0) ? 2 : 1);
@@ -485,6 +511,15 @@ int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, con
   CUtensorMap kmap;
   memset(&kmap, 0, sizeof(kmap));
   const int use_tma = make_key_map(&kmap, K, cfg.dtype, l, cfg.n_kv_heads, cfg.batch, ks) ? 1 : 0;
+  // the gathered copy of the probe rows, when the workspace has room for it
+  CUtensorMap qmap;
+  memset(&qmap, 0, sizeof(qmap));
+  const size_t qp_need = (size_t)cfg.batch * cfg.n_q_heads * (size_t)n_probe * ZC_D * 2;
+  int use_qp = 0;
+  if (use_tma && qp_ws && qp_bytes >= qp_need) {
+    const int64_t qps[3] = {(int64_t)cfg.n_q_heads * n_probe * ZC_D, (int64_t)n_probe * ZC_D, ZC_D};
+    use_qp = make_key_map(&qmap, qp_ws, cfg.dtype, n_probe, cfg.n_q_heads, cfg.batch, qps) ? 1 : 0;
+  }
   cudaError_t e;
 #define ZC_GO(T)                                                                                       \
   do {                                                                                                 \
@@ -492,6 +527,9 @@ int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, con
     if (e != cudaSuccess) return e;                                                                    \
     e = cudaFuncSetAttribute(k_probe_colsum<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem); \
     if (e != cudaSuccess) return e;                                                                    \
+    if (use_qp)                                                                                        \
+      k_gather_probe_rows<T><<<dim3(zc_ceil_div(n_probe, 8), cfg.batch * cfg.n_q_heads), 128, 0, st>>>( \
+          (const T*)Q, P_dev, n_probe, cfg.n_q_heads, qs[0], qs[1], qs[2], (T*)qp_ws);                 \
     k_probe_lse<T><<<g1, kThreads, kTcSmem, st>>>((const T*)Q, (const T*)K, P_dev, n_probe, l,      \
                                                      cfg.n_q_heads, G, Gt, qs[0], qs[1], qs[2], ks[0], \
                                                      ks[1], ks[2], lse_ws, kmap, use_tma);             \
@@ -499,11 +537,11 @@ int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l, con
                                                         cfg.n_q_heads, cfg.n_kv_heads, G, qs[0], qs[1], \
                                                         qs[2], ks[0], ks[1], ks[2], lse_ws, c->base,   \
                                                         c->lay.unit_stride, c->lay.off_scores, kmap,   \
-                                                        use_tma);                                      \
+                                                        use_tma, qmap, use_qp);                        \
   } while (0)
   if (cfg.dtype == ZC_F16) ZC_GO(__half); else ZC_GO(__nv_bfloat16);
 #undef ZC_GO
-  c->launches += 2;
+  c->launches += 2 + use_qp;
   return cudaGetLastError();
 }
 
