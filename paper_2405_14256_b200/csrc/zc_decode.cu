@@ -40,18 +40,8 @@ constexpr int kWarps = 4;
 // their neighbours, where more resident warps hide the set-up and merge of the others.
 constexpr int kRingWide = 13824, kRingNarrow = 9216;
 constexpr int kWaitLimit = 1 << 22;
-#ifndef ZC_KPEXP
-#define ZC_KPEXP 12
-#define ZC_TAU 3.5f
-#endif
-#ifndef ZC_QK_CHAINS
-#define ZC_QK_CHAINS 1
-#endif
-#ifndef ZC_SHIFT_ON_FMA
-#define ZC_SHIFT_ON_FMA 0
-#endif
-constexpr int kPExp = ZC_KPEXP;      // softmax weights go to f16 as p * s^V * 2^kPExp / 2^ceil(log2 smax)
-constexpr float kTau = ZC_TAU;   // the running maximum is refreshed only when a logit exceeds it by this
+constexpr int kPExp = 12;      // softmax weights go to f16 as p * s^V * 2^kPExp / 2^ceil(log2 smax)
+constexpr float kTau = 3.5f;   // the running maximum is refreshed only when a logit exceeds it by this
 constexpr unsigned kFull = 0xffffffffu;
 
 // shared-memory map of an item CTA: small arrays first, then the warps' rings
@@ -224,17 +214,7 @@ template <int BITS> __device__ __forceinline__ void chan_slot(int off, int* reg,
   }
 }
 
-// w >> 8 on the multiply pipe: the integer pipe is the busiest unit of the loop (one mask per
-// tensor-core operand register), every shift moved off it is a net gain.
-__device__ __forceinline__ uint32_t shr8(uint32_t w) {
-#if ZC_SHIFT_ON_FMA
-  uint32_t r;
-  asm("mul.hi.u32 %0, %1, 16777216;\n" : "=r"(r) : "r"(w));
-  return r;
-#else
-  return w >> 8;
-#endif
-}
+__device__ __forceinline__ uint32_t shr8(uint32_t w) { return w >> 8; }
 
 // expect_tx + bulk copy by one lane without a divergent branch
 __device__ __forceinline__ void refill_if(bool pred, uint64_t* bar, void* dst, const void* src, int bytes) {
@@ -304,12 +284,6 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     float dacc[4];
-#if ZC_QK_CHAINS == 2
-    float dacc2[4];
-#define ZC_SECOND dacc2
-#else
-#define ZC_SECOND dacc
-#endif
     if (BITS == 4) {
 #pragma unroll
       for (int jw = 0; jw < 4; ++jw) {
@@ -319,8 +293,7 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
         else zc_mma16816<__half>(dacc, a0, qb[4 * jw], qb[4 * jw + 1]);
         const uint32_t x0 = shr8(w0), x1 = shr8(w1);
         const uint32_t a1[4] = {x0 & 0x000F000Fu, x1 & 0x000F000Fu, x0 & 0x00F000F0u, x1 & 0x00F000F0u};
-        if (ZC_QK_CHAINS == 2 && jw == 0) zc_mma16816_z(ZC_SECOND, a1, qb[2], qb[3]);
-        else zc_mma16816<__half>(ZC_SECOND, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
+        zc_mma16816<__half>(dacc, a1, qb[4 * jw + 2], qb[4 * jw + 3]);
       }
     } else {
 #pragma unroll
@@ -334,16 +307,10 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
           if (ks == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
           else zc_mma16816<__half>(dacc, a0, qb[2 * ks], qb[2 * ks + 1]);
           const uint32_t a1[4] = {w0 & 0x00300030u, w1 & 0x00300030u, w0 & 0x00C000C0u, w1 & 0x00C000C0u};
-          if (ZC_QK_CHAINS == 2 && ks == 0) zc_mma16816_z(ZC_SECOND, a1, qb[2], qb[3]);
-          else zc_mma16816<__half>(ZC_SECOND, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
+          zc_mma16816<__half>(dacc, a1, qb[2 * ks + 2], qb[2 * ks + 3]);
         }
       }
     }
-#if ZC_QK_CHAINS == 2
-#pragma unroll
-    for (int e = 0; e < 4; ++e) dacc[e] += dacc2[e];
-#endif
-#undef ZC_SECOND
     // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
     u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
     u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;

@@ -6,7 +6,6 @@
 #include <new>
 #include <vector>
 #include <algorithm>
-#include <cstdlib>
 #include "zc_internal.h"
 #include "zc_layout.cuh"
 
@@ -222,10 +221,7 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   }
   p.items = p.split0[0] + p.split0[1] + 2 * (p.n_seg - 1);
   p.cta_items = 1;
-  if (c->cfg.flags & ZC_FLAG_OVERLAP_CALLS) {
-    static const char* e_ci = getenv("ZIPCACHE_CTA_ITEMS");   // tuning override (experiments)
-    p.cta_items = e_ci ? std::max(1, atoi(e_ci)) : p.items;
-  }
+  if (c->cfg.flags & ZC_FLAG_OVERLAP_CALLS) p.cta_items = p.items;   // one CTA per unit and head group
   return p;
 }
 
