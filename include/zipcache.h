@@ -85,8 +85,9 @@ typedef struct {
 typedef struct zc_cache zc_cache; /* small host-side handle */
 
 /* Sizes [host].  cache_bytes: device buffer for the compressed cache;
- * workspace_bytes: device scratch shared by all calls (probe-row statistics in
- * prefill, split-K partial results in decode).  Either out pointer may be NULL. */
+ * workspace_bytes: device scratch shared by all calls (in prefill: probe positions, probe-row
+ * statistics and a dense copy of the probe rows; in decode: split-K partial results, with room
+ * for 16 calls in flight together).  Either out pointer may be NULL. */
 int zc_cache_bytes(const zc_config* cfg, size_t* cache_bytes, size_t* workspace_bytes);
 
 /* Create a handle over caller-owned device memory `dev_mem` [device, >= cache_bytes,
@@ -171,8 +172,9 @@ int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t*
  * ends); the caller still owns q [device] and out [device].  The call allocates and frees
  * nothing.
  *   - ZC_ESCRATCH, with nothing enqueued, when the cache's shape needs more than the
- *     built-in buffer (about batch * n_q_heads * items * 528 bytes, items = split-K pieces
- *     per KV head; use zc_decode_attention with a caller workspace then).
+ *     built-in buffer (about batch * n_q_heads * (items + 8) * 528 bytes, items = split-K
+ *     pieces per KV head, 8 = tiles of the full-precision tail; use zc_decode_attention with a
+ *     caller workspace then).
  *   - The first call on each device looks up the buffer's device address (a synchronous
  *     runtime query): make that first call outside any stream capture.
  *   - All calls share the one buffer, whatever cache they work on.  Calls that follow one

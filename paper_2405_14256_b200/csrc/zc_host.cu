@@ -188,7 +188,7 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
         spi[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;
         split[k] = zc_ceil_div(subs[k], spi[k]);
       }
-      // items of every head group, one tail CTA per unit, one sentinel
+      // items of every head group, one tail CTA per unit, the one CTA that only waits
       const double n_ctas = ((double)(split[0] + split[1] + extras) * zs + 1) * c->lay.units + 1;
       const double waves = n_ctas / slots;
       // a handful of CTAs beyond a whole wave start as soon as the first ones retire
