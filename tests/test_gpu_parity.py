@@ -258,3 +258,30 @@ def test_deferred_append_is_performed_by_any_other_call():
     assert torch.equal(outs[0][0], outs[1][0])
     assert torch.equal(outs[0][1], outs[1][1])
     assert torch.equal(outs[0][2], outs[1][2])
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_prefill_accepts_token_major_inputs(dtype):
+    """Q, K, V handed over as views of [batch, token, head, d] buffers (the layout projection
+    kernels usually write): strides instead of copies.  Scores, salient sets and packed codes
+    must equal those of the contiguous [batch, head, token, d] call bit for bit, and match the
+    oracle."""
+    w = tl.small_workload(dtype=dtype, context=700, batch=2, n_q_heads=8, n_kv_heads=2)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    views = [t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for t in (Q, K, V)]
+    assert not views[1].is_contiguous() and torch.equal(views[1], K)
+    results = []
+    for q_, k_, v_ in ((Q, K, V), views):
+        cache = tl.make_cache(w)
+        cache.mem.zero_()
+        cache.prefill_compress(q_, k_, v_, P.tolist())
+        torch.cuda.synchronize()
+        results.append((cache.scores(w.context).clone(), cache.mem.clone(), cache))
+    assert torch.equal(results[0][0], results[1][0])
+    assert torch.equal(results[0][1], results[1][1])
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    assert tl.compare_segment(results[1][2], oc, 0) == 0
+    import paper_2405_14256_b200 as zc
+    assert zc.zc_device_status() == 0
