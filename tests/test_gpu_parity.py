@@ -71,6 +71,9 @@ def test_quantize_degenerate_rows():
     dict(context=64, n_q_heads=8, n_kv_heads=1, rho_recent=0.3, rho_random=0.3),
     dict(context=1, n_q_heads=2, n_kv_heads=1),
     dict(context=1300, n_q_heads=2, n_kv_heads=2, band=20, saliency_ratio=0.3),
+    # every row a probe row: more than the workspace keeps a dense copy of, so the column-sum
+    # kernel gathers its probe tiles itself
+    dict(context=1100, n_q_heads=4, n_kv_heads=2, rho_recent=0.5, rho_random=0.5),
 ])
 def test_normalized_scores_and_salient_sets(kw):
     w = tl.small_workload(**kw)
