@@ -140,11 +140,11 @@ struct TcCtx {
   uint64_t* b_full;
   uint64_t* a_full;
   uint32_t* tmem_slot;
-  char* extra;       // pass 2: probe positions and lse of the last kSide B tiles
+  char* extra;       // pass 2: per worker warp, probe positions and lse of kSide B tiles
   uint32_t a_addr, b_addr, tmem;
 };
-constexpr int kSide = 8;           // per-column data of pass 2 is kept for 8 tiles (see k_probe_colsum)
-constexpr int kTcSmem = 3 * kTile + 1024 /* alignment */ + 128 /* barriers, tmem slot */ + kSide * kM * 8;
+constexpr int kSide = 3;           // per-column data of pass 2: three tiles per worker warp (see k_probe_colsum)
+constexpr int kTcSmem = 3 * kTile + 1024 /* alignment */ + 128 /* barriers, tmem slot */ + 4 * kSide * kM * 8;
 
 __device__ __forceinline__ void bar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];\n" ::"r"(zc_smem_u32(bar)) : "memory");
@@ -236,7 +236,6 @@ __device__ __forceinline__ void issue_loop(const TcCtx& c, int n, uint32_t idesc
 __device__ __forceinline__ void copies_arrive(uint64_t* bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(zc_smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, 128;\n" ::: "memory"); }
 
 // Worker: waits for tile cb's accumulator and fetches this thread's row of it.
 __device__ __forceinline__ void worker_fetch(const TcCtx& c, int cb, int quarter, float (&v)[kM]) {
@@ -353,11 +352,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
   // A (the key block): one bulk copy, or the workers; B (probe rows): bulk copies from the
   // gathered copy of the probe rows when there is one (qmap), else the workers gather them
   TcCtx c = tc_setup(smem_raw, use_tma ? 1 : kM, use_qp ? 1 : kM);
-  // Per-column data of a B tile (probe position and lse of each of its rows), slot = tile mod 8,
-  // written by the workers two tiles ahead of its use; they meet at a barrier of their own once
-  // per tile, so no warp is more than one tile ahead of another.
-  int* Pp = reinterpret_cast<int*>(c.extra);                      // [kSide][128]
-  float* Ll = reinterpret_cast<float*>(c.extra + kSide * kM * 4);  // [kSide][128]
+  // Per-column data of a B tile (probe position and lse of each of its 128 rows): every worker
+  // warp keeps its own copy, slot = tile mod 3, written two tiles ahead of its use, so the
+  // warps need no barrier among themselves.
+  const int wq = (threadIdx.x >> 5) > 0 ? (threadIdx.x >> 5) - 1 : 0;
+  int* Pp = reinterpret_cast<int*>(c.extra + wq * (kSide * kM * 8));   // [kSide][128]
+  float* Ll = reinterpret_cast<float*>(Pp + kSide * kM);                // [kSide][128]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int j0 = blockIdx.x * kM;
   const int unit = blockIdx.y, b = unit / n_kv, kv = unit % n_kv;
@@ -397,9 +397,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
         }
         copies_arrive(&c.b_full[tile & 1]);
       }
-      const int slot = tile & (kSide - 1), r = r_start + rb * kM + wt;
-      Pp[slot * kM + wt] = r < n_probe ? P[r] : -1;
-      Ll[slot * kM + wt] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
+      const int slot = tile % kSide;
+#pragma unroll
+      for (int k = 0; k < kM / 32; ++k) {
+        const int i = lane + 32 * k, r = r_start + rb * kM + i;
+        Pp[slot * kM + i] = r < n_probe ? P[r] : -1;
+        Ll[slot * kM + i] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
+      }
     };
     if (!use_tma) {
 #pragma unroll 4
@@ -411,16 +415,16 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     }
     load_b(0);
     if (n_tiles > 1) load_b(1);
-    workers_sync();   // per-column data of tiles 0 and 1 is visible to all workers
+    __syncwarp();   // per-column data of tiles 0 and 1 is visible to the warp
     const int j = j0 + row;
     const float scale = kLog2e * rsqrtf((float)ZC_D);
     float sum4[4] = {0.f, 0.f, 0.f, 0.f};
     for (int tile = 0; tile < n_tiles; ++tile) {
-      const int slot = tile & (kSide - 1);
+      const int slot = tile % kSide;
       float v[kM];
       worker_fetch(c, tile, quarter, v);
       if (tile + 2 < n_tiles) load_b(tile + 2);   // its buffer was read by the MMA that has just completed
-      workers_sync();   // per-column data written here is read two iterations on; the warps stay in step
+      __syncwarp();   // per-column data written here is read two iterations on
       const int* pp = Pp + slot * kM;
       const float* ll = Ll + slot * kM;
       if (j <= pp[0]) {   // probe rows ascend in position: every row of the tile sees column j
