@@ -64,6 +64,11 @@ _SIGS = {
     "zc_decode_bytes": (C.c_int64, [C.c_void_p]),
     "zc_launch_count": (C.c_int64, [C.c_void_p]),
     "zc_device_status": (C.c_int, [C.POINTER(C.c_int)]),
+    "zc_order_model_reset": (None, []),
+    "zc_order_model_call": (C.c_int, [C.c_uint64, C.c_int, C.POINTER(C.c_uint64), C.c_uint64, C.c_uint64,
+                                      C.c_int, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64,
+                                      C.POINTER(C.c_int)]),
+    "zc_order_model_fence": (C.c_int, [C.c_uint64, C.c_int]),
     "zc_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -213,6 +218,27 @@ def zc_device_status() -> int:
     code = C.c_int(0)
     _check(lib().zc_device_status(C.byref(code)), "zc_device_status")
     return code.value
+
+
+ORDER_FIELDS = ("epoch_start", "e", "need_start", "need_end", "slot", "tag", "record", "drain")
+
+
+def zc_order_model_reset() -> None:
+    lib().zc_order_model_reset()
+
+
+def zc_order_model_call(stream_id, cache_id, q, k_new, v_new, out, io_bytes, kv_bytes, collect,
+                        ws_addr, ws_bytes, need, capture_id=0) -> dict:
+    """Books one call in the host-only model of the call ordering; addresses are integers."""
+    addr = (C.c_uint64 * 4)(q, k_new, v_new, out)
+    res = (C.c_int * 8)()
+    _check(lib().zc_order_model_call(stream_id, cache_id, addr, io_bytes, kv_bytes, int(collect),
+                                     ws_addr, ws_bytes, need, capture_id, res), "zc_order_model_call")
+    return dict(zip(ORDER_FIELDS, list(res)))
+
+
+def zc_order_model_fence(stream_id, cache_id) -> None:
+    _check(lib().zc_order_model_fence(stream_id, cache_id), "zc_order_model_fence")
 
 
 class ZipCache:

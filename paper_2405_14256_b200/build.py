@@ -11,8 +11,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzipcache.so")
-SOURCES = ["zc_host.cu", "zc_scores.cu", "zc_compress.cu", "zc_decode.cu", "zc_export.cu"]
-HEADERS = ["zc_internal.h", "zc_layout.cuh", "zc_mma.cuh"]
+SOURCES = ["zc_host.cu", "zc_scores.cu", "zc_compress.cu", "zc_decode.cu", "zc_order.cu",
+           "zc_export.cu"]
+HEADERS = ["zc_internal.h", "zc_layout.cuh", "zc_mma.cuh", "zc_order.h"]
 
 
 def _nvcc() -> str:

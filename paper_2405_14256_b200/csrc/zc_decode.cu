@@ -28,6 +28,7 @@
 #include "zc_internal.h"
 #include "zc_layout.cuh"
 #include "zc_mma.cuh"
+#include "zc_order.h"
 
 namespace {
 
@@ -1002,41 +1003,9 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-// What the host remembers about a stream: the decode calls launched on it since the last
-// launch made without early start (an epoch).  Calls of an epoch may be in flight together.
-// Call e uses region e mod K of the workspace and arrival counter e mod K; the kernel itself
-// waits (see ZcOrder) until call e - K has completed before it writes there, until every
-// earlier call whose output it reads has completed before it reads, and until every earlier
-// call whose output or inputs it overwrites, or whose window statistics it adds to, has
-// completed before it writes.  The host finds those calls by comparing address ranges with
-// the last kRing calls; anything older is covered by waiting for call e - kRing.
-struct Range { const char* lo; const char* hi; };
-constexpr int kRing = ZC_EPOCH_CALLS;
-struct CallRec {
-  Range in[3];                      // q, k_new, v_new
-  Range out;
-  const zc_cache* collected;        // cache whose window statistics the call updates
-};
-struct StreamRec {
-  cudaStream_t st;
-  bool used;
-  int dev;
-  unsigned tag;                     // epoch tag, 12 bits
-  int e;                            // calls launched in the current epoch
-  int K;                            // workspace regions / arrival counters in use
-  const char* ws;
-  size_t ws_bytes, slot_bytes;
-  int capturing;
-  unsigned long long capture_id;
-  CallRec ring[kRing];
-  unsigned long long age;
-};
-constexpr int kStreamRecs = 16;
-StreamRec g_rec[kStreamRecs];
-unsigned long long g_rec_clock = 0;
-std::mutex g_rec_mutex;
-
-bool meet(const Range& a, const Range& b) { return a.lo && b.lo && a.lo < b.hi && b.lo < a.hi; }
+// The calls issued so far, per stream (the rules are in zc_order.h / zc_order.cu).
+ZcOrderTable g_table;
+std::mutex g_table_mutex;
 
 }  // namespace
 
@@ -1061,23 +1030,14 @@ size_t zc_decode_scratch_bytes(const zc_cache* c, int items) {
 void zc_order_fence(zc_cache* c, cudaStream_t st) {
   int dev = 0;
   cudaGetDevice(&dev);
-  std::lock_guard<std::mutex> lock(g_rec_mutex);
-  c->fence_rec = -1;
-  for (int i = 0; i < kStreamRecs; ++i) {
-    const StreamRec& r = g_rec[i];
-    if (r.used && r.st == st && r.dev == dev) {
-      c->fence_rec = i;
-      c->fence_tag = r.tag;
-      c->fence_e = r.e;            // the next call of the epoch publishes their completion
-      c->fence_capturing = r.capturing;
-    }
-  }
+  std::lock_guard<std::mutex> lock(g_table_mutex);
+  zc_order_fence_at(&g_table, &c->fence, (const void*)st, dev);
 }
 
 // One word per stream record, in the library image (like the built-in scratch below).
 // Two per record: calls issued under stream capture use the second, so that replaying a
 // captured graph never disturbs the word of the calls issued directly.
-static __device__ unsigned g_zc_order_words[32];
+static __device__ unsigned g_zc_order_words[2 * kZcStreamRecs];
 
 int zc_order_words(unsigned** ptr) {
   constexpr int kMaxDev = 64;
@@ -1098,7 +1058,7 @@ int zc_order_words(unsigned** ptr) {
 
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
                      char* ws, size_t ws_bytes, const void* k_new, const void* v_new, cudaStream_t st) {
-  static_assert(kStreamRecs == 16, "one order word per stream record");
+  static_assert(2 * kZcStreamRecs == 32, "two order words per stream record");
   const int G = c->lay.G, zs = (G + 3) / 4;
   const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
   const size_t kv_bytes = (size_t)c->lay.units * ZC_D * 2;
@@ -1121,82 +1081,39 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
     cap_id = 0;
   }
   const int capturing = cap_status == cudaStreamCaptureStatusActive ? 1 : 0;
-  auto range = [](const void* p, size_t n) { return Range{(const char*)p, p ? (const char*)p + n : nullptr}; };
-  CallRec me;
-  me.in[0] = range(q, io_bytes);
-  me.in[1] = range(k_new, kv_bytes);
-  me.in[2] = range(v_new, kv_bytes);
-  me.out = range(out, io_bytes);
-  me.collected = collect ? c : nullptr;
+  ZcOrderCall call{};
+  call.st = (const void*)st;
+  call.dev = dev;
+  call.me.in[0] = zc_range(q, io_bytes);
+  call.me.in[1] = zc_range(k_new, kv_bytes);
+  call.me.in[2] = zc_range(v_new, kv_bytes);
+  call.me.out = zc_range(out, io_bytes);
+  call.cache = c;
+  call.collect = collect;
+  call.stores_tail_row = k_new != nullptr;
+  call.ws = ws;
+  call.ws_bytes = ws_bytes;
+  call.need = need;
+  call.capturing = capturing;
+  call.capture_id = cap_id;
   ZcOrder ord;
   int slot = 0;
   size_t ws_off = 0;
   {
-    std::lock_guard<std::mutex> lock(g_rec_mutex);
-    StreamRec* r = nullptr;
-    StreamRec* victim = nullptr;   // an unused record, else the one touched longest ago
-    for (int i = 0; i < kStreamRecs; ++i) {
-      StreamRec* x = &g_rec[i];
-      if (x->used && x->st == st && x->dev == dev) r = x;
-      if (!victim || (victim->used && (!x->used || x->age < victim->age))) victim = x;
-    }
-    bool fresh = false;
-    if (!r) {
-      r = victim;
-      if (r->used && !capturing) cudaStreamSynchronize(r->st);   // its word changes hands
+    std::lock_guard<std::mutex> lock(g_table_mutex);
+    const ZcOrderSlot s = zc_order_next(&g_table, &c->fence, call);
+    if (s.drain && !capturing) {
+      cudaStreamSynchronize((cudaStream_t)s.drain);
       cudaGetLastError();
-      r->used = true;
-      r->st = st;
-      r->dev = dev;
-      r->e = 0;
-      fresh = true;
     }
-    // a new epoch: this launch is made without early start and so finds the stream drained
-    if (fresh || r->e == 0 || r->e >= (1 << 20) - 1 || r->ws != ws || r->ws_bytes != ws_bytes ||
-        need > r->slot_bytes || r->capturing != capturing || r->capture_id != cap_id) {
-      r->tag = (r->tag + 1) & 0xFFFu;
-      r->e = 0;
-      r->ws = ws;
-      r->ws_bytes = ws_bytes;
-      r->K = (int)std::min<size_t>((size_t)kRing, ws_bytes / need);
-      r->slot_bytes = (ws_bytes / (size_t)r->K) & ~(size_t)255;
-      if (r->slot_bytes < need) {   // alignment took the room: fewer, larger regions
-        r->K = std::max(1, r->K - 1);
-        r->slot_bytes = r->K == 1 ? ws_bytes : (ws_bytes / (size_t)r->K) & ~(size_t)255;
-      }
-      r->capturing = capturing;
-      r->capture_id = cap_id;
-    }
-    const int e = r->e;
-    ord.done = words + 2 * (r - g_rec) + capturing;
-    ord.tag = r->tag;
-    ord.e = e;
-    ord.epoch_start = e == 0;
-    ord.need_end = e - r->K + 1;
-    ord.need_start = e - kRing + 1;
-    for (int i = std::max(0, e - kRing + 1); i < e; ++i) {
-      const CallRec& o = r->ring[i % kRing];
-      for (int k = 0; k < 3; ++k) {
-        if (meet(me.in[k], o.out)) ord.need_start = std::max(ord.need_start, i + 1);
-        if (meet(me.out, o.in[k])) ord.need_end = std::max(ord.need_end, i + 1);
-      }
-      if (meet(me.out, o.out) || (collect && o.collected == c)) ord.need_end = std::max(ord.need_end, i + 1);
-    }
-    // kernels chained behind an earlier call changed this cache (a re-compressed window)
-    if (e > 0 && c->fence_rec == (int)(r - g_rec) && c->fence_tag == r->tag && c->fence_capturing == capturing)
-      ord.need_start = std::max(ord.need_start, c->fence_e);
-    slot = e % r->K;
-    ws_off = (size_t)slot * r->slot_bytes;
-    if (k_new) {
-      // this call stores a tail row that the cache's next call reads from the tail buffer
-      c->fence_rec = (int)(r - g_rec);
-      c->fence_tag = r->tag;
-      c->fence_e = e + 1;
-      c->fence_capturing = capturing;
-    }
-    r->ring[e % kRing] = me;
-    r->e = e + 1;
-    r->age = ++g_rec_clock;
+    ord.done = words + 2 * s.rec + capturing;
+    ord.tag = s.tag;
+    ord.e = s.e;
+    ord.epoch_start = s.epoch_start;
+    ord.need_start = s.need_start;
+    ord.need_end = s.need_end;
+    slot = s.slot;
+    ws_off = s.ws_off;
   }
   const bool overlap = !ord.epoch_start;
   float* part = reinterpret_cast<float*>(ws + ws_off);

@@ -262,7 +262,7 @@ int zc_cache_init(void* dev_mem, size_t bytes, const zc_config* cfg, zc_cache** 
   c->bytes = bytes;
   c->l0 = -1;
   c->n_seg = 0;
-  c->fence_rec = -1;
+  c->fence.rec = -1;
   int dev = 0, n_sm = 148;
   if (cudaGetDevice(&dev) == cudaSuccess)
     cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);

@@ -82,6 +82,15 @@ struct ZcDecodePlan {
   int l0;
 };
 
+// Where in a stream's sequence of decode calls a cache was last changed by something other
+// than a decode call's own output (see zc_order.h).
+struct ZcFence {
+  int rec;          // stream record, -1: none
+  unsigned tag;     // epoch
+  int e;            // calls of that epoch that must have completed
+  int capturing;
+};
+
 struct zc_cache {
   zc_config cfg;
   ZcLayout lay;
@@ -104,10 +113,7 @@ struct zc_cache {
   const void* pend_v;
   cudaStream_t pend_stream;
   // ordering of decode calls behind chained kernels that changed this cache (zc_order_fence)
-  int fence_rec;
-  unsigned fence_tag;
-  int fence_e;
-  int fence_capturing;
+  ZcFence fence;
 };
 
 __host__ __device__ static inline int zc_ceil_div(int a, int b) { return (a + b - 1) / b; }
