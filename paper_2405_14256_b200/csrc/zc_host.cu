@@ -424,16 +424,20 @@ static int decode_attention(zc_cache* c, const void* q, void* out, int is_probe_
       // re-compress the window into a new segment
       // the re-compression runs as links of the decode calls' chain: calls on other caches
       // that follow on the stream start without waiting for it
-      ZC_CUDA(zc_launch_window_scores(c, st, true));
       c->last_scores_n = c->cfg.window;
       const int seg = c->n_seg;
       c->n_seg += 1;
       ZcSeg s = zc_segment(c, seg);
-      ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], s.idx_off, nullptr, st, true));
       const long long us = c->lay.unit_stride / 2;
       ZcSrc src{c->base + c->lay.off_tailK, c->base + c->lay.off_tailV, us * c->lay.n_kv, us,
                 ZC_D};
-      ZC_CUDA(zc_launch_quantize(c, src, s, st, true));
+      if (zc_window_flush_fits(c, s)) {
+        ZC_CUDA(zc_launch_window_flush(c, src, s, st, true));
+      } else {
+        ZC_CUDA(zc_launch_window_scores(c, st, true));
+        ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], s.idx_off, nullptr, st, true));
+        ZC_CUDA(zc_launch_quantize(c, src, s, st, true));
+      }
       zc_order_fence(c, st);
       c->n_tail = 0;
       c->step_i = 0;

@@ -134,6 +134,11 @@ int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* give
 int zc_launch_window_scores(zc_cache* c, cudaStream_t st, bool chained = false);
 int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st,
                        bool chained = false);
+// The whole re-compression of a window (scores, split, factors, quantise, pack) as one kernel,
+// for windows whose two classes fit one tile each (zc_window_flush_fits).
+bool zc_window_flush_fits(const zc_cache* c, const ZcSeg& seg);
+int zc_launch_window_flush(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st,
+                           bool chained = false);
 // Marks the cache as changed by kernels just launched on st: decode calls on this cache
 // that follow within the same epoch wait for them before they read anything.
 void zc_order_fence(zc_cache* c, cudaStream_t st);

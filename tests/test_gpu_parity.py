@@ -134,12 +134,17 @@ def test_decode_attention_parity(kw, steps):
     assert worst <= 2e-3
 
 
-@pytest.mark.parametrize("window,steps", [(16, 40), (100, 105)])
-def test_decode_across_window_recompression(window, steps):
+@pytest.mark.parametrize("window,steps,ratio", [
+    (16, 40, 0.4), (100, 105, 0.4),
+    (100, 105, 0.8),                  # 80 salient tokens: more than one tile in a class
+    (16, 20, 0.0), (16, 20, 1.0),     # an empty class
+    (128, 130, 0.5),                  # the largest window, both tiles full
+])
+def test_decode_across_window_recompression(window, steps, ratio):
     """The tail is re-compressed after `window` steps: new segment codes must be bit-exact
     (given equal salient sets) and attention must stay within tolerance."""
     w = tl.small_workload(context=150, n_q_heads=4, n_kv_heads=2, window=window,
-                          rho_recent=0.1, rho_random=0.1)
+                          rho_recent=0.1, rho_random=0.1, saliency_ratio=ratio)
     worst, cache, oc = tl.run_decode_parity(w, steps)
     assert worst <= 2e-3
     import paper_2405_14256_b200 as zc
