@@ -2,6 +2,7 @@
 // and packing into cache tiles; also the window statistics -> score step of Alg. 3.
 #include "zc_internal.h"
 #include "zc_layout.cuh"
+#include "zc_quant.cuh"
 
 namespace {
 
@@ -225,88 +226,7 @@ __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
   if (threadIdx.x < 2) fac[(seg.run0 + threadIdx.x) * ZC_FAC_FLOATS + 2 * ZC_D] = 0.f;  // smaxV
 }
 
-// ------------------------------------------------------------------ CSTQuant + pack
-// Normative fp32 sequence (each step one IEEE operation, round to nearest even, nothing
-// fused): c = sqrt(max|x|) (1 if the channel is all zero); y = x / c; per token mn, mx over
-// the 128 channels; s = (mx - mn) / L, or |mn| (1 if mn == 0) when mx == mn;
-// z = -rint(mn / s); code = clamp(rint(y / s) + z, 0, L).
-__device__ __forceinline__ void quant_token(const float (&x)[4], const float (&c)[4], float L,
-                                            float* s_out, float* z_out, unsigned* codes4) {
-  float y[4];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) y[e] = __fdiv_rn(x[e], c[e]);
-  float mn = fminf(fminf(y[0], y[1]), fminf(y[2], y[3]));
-  float mx = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  }
-  float s = __fdiv_rn(__fsub_rn(mx, mn), L);
-  if (mx == mn) s = mn != 0.f ? fabsf(mn) : 1.f;
-  const float z = -rintf(__fdiv_rn(mn, s));
-  unsigned packed = 0;
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    float q = __fadd_rn(rintf(__fdiv_rn(y[e], s)), z);
-    q = fminf(fmaxf(q, 0.f), L);
-    packed |= ((unsigned)(int)q) << (8 * e);
-  }
-  *s_out = s;
-  *z_out = z;
-  *codes4 = packed;
-}
-
-// One 16-byte vector v of a cache tile from the tile's 64 x 128 byte codes and its per-token
-// (s, z): K codes in canonical order, V codes in fragment order, then the parameters, per
-// 16-token sub-block.
-__device__ __forceinline__ uint4 compose_vec(int bits, int v, const unsigned char (*codesK)[ZC_D],
-                                             const unsigned char (*codesV)[ZC_D], const float (*parK)[2],
-                                             const float (*parV)[2]) {
-  const int sub_words = zc_sub_bytes(bits) / 4;
-  const int kw = 64 * bits;                           // K-code words per sub-block (= V-code words)
-  const int per = 32 / bits;                          // codes per word
-  unsigned out[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int wi = 4 * v + q;
-    const int st = wi / sub_words, wl = wi % sub_words;
-    unsigned word = 0;
-    if (wl < kw) {
-      // K: canonical order, token row of 4*bits words
-      const int words_per_row = 4 * bits;
-      const int tok = 16 * st + wl / words_per_row, wr = wl % words_per_row;
-      for (int e = 0; e < per; ++e) word |= (unsigned)codesK[tok][wr * per + e] << (bits * e);
-    } else if (wl < 2 * kw) {
-      // V: fragment order of the 16-token sub-tile
-      const int wv = wl - kw;
-      if (bits == 4) {
-        const int qd = wv >> 7, ln = (wv >> 2) & 31, jj = wv & 3;
-        const int j = 4 * qd + jj, g = ln >> 2, t = ln & 3;
-        for (int p = 0; p < 8; ++p) {
-          const int hi_row = p & 1, isB = (p >> 1) & 1, is1 = p >> 2;
-          const int ch = 16 * j + g + 8 * hi_row, tau = 2 * t + isB + 8 * is1;
-          word |= (unsigned)codesV[16 * st + tau][ch] << (4 * p);
-        }
-      } else {
-        const int ln = wv >> 2, m = wv & 3, g = ln >> 2, t = ln & 3;
-        for (int i = 0; i < 16; ++i) {
-          const int is1 = i >> 3, pp = i & 7, e2 = pp >> 2, hi_row = (pp >> 1) & 1, isB = pp & 1;
-          const int j = 2 * m + e2;
-          const int ch = 16 * j + g + 8 * hi_row, tau = 2 * t + isB + 8 * is1;
-          word |= (unsigned)codesV[16 * st + tau][ch] << (2 * i);
-        }
-      }
-    } else {
-      const int wp = wl - 2 * kw;  // params: (sK, zK, sV, zV) per token
-      const int tk = 16 * st + (wp >> 2), f = wp & 3;
-      word = __float_as_uint(f < 2 ? parK[tk][f] : parV[tk][f - 2]);
-    }
-    out[q] = word;
-  }
-  return make_uint4(out[0], out[1], out[2], out[3]);
-}
-
+// ------------------------------------------------------------------ CSTQuant + pack (arithmetic in zc_quant.cuh)
 template <typename T>
 __global__ void __launch_bounds__(256, 3) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
   chain_link();
@@ -386,178 +306,7 @@ __global__ void __launch_bounds__(256, 3) k_quantize_pack(char* cache, ZcLayout 
   char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
   const int total_vec = lay.tile_bytes[cls] / 16;
   for (int v = threadIdx.x; v < total_vec; v += 256)
-    reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(bits, v, codesK, codesV, parK, parV);
-}
-
-// ------------------------------------------------------------------ window re-compression, fused
-// Alg. 3's re-compression of one window (at most 128 tokens, at most 64 per class) in one
-// kernel and so one link of the chain: scores from the window statistics, split, channel
-// factors, CSTQuant and packing, with the same arithmetic as the separate kernels above.
-// One CTA of 1024 threads per unit; warp w owns slots 4w .. 4w+3, slots 0..63 being the
-// salient tile and 64..127 the regular tile.
-constexpr int kFlushThreads = 1024;
-
-template <typename T>
-__global__ void __launch_bounds__(kFlushThreads) k_window_flush(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg,
-                                                                NnzArgs nnz) {
-  chain_link();
-  __shared__ __align__(16) unsigned char codesK[2 * ZC_TILE][ZC_D];
-  __shared__ __align__(16) unsigned char codesV[2 * ZC_TILE][ZC_D];
-  __shared__ __align__(16) float parK[2 * ZC_TILE][2];
-  __shared__ __align__(16) float parV[2 * ZC_TILE][2];
-  __shared__ unsigned s_key[ZC_MAX_WINDOW];
-  __shared__ int s_tok[2 * ZC_TILE];
-  __shared__ unsigned s_cmax[2][2][ZC_D];
-  __shared__ unsigned s_smax[2];
-  __shared__ unsigned s_mask[ZC_MAX_WINDOW / 32];
-  const int unit = blockIdx.x, b = unit / lay.n_kv, kv = unit % lay.n_kv;
-  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-  const int n = lay.window, n_s = seg.n_tok[0];
-  char* ub = zc_unit_base(cache, lay, unit);
-
-  // ---- scores of the window's tokens (Alg. 3), statistics cleared for the next window ----
-  if (tid < ZC_MAX_WINDOW) {
-    unsigned key = 0u;
-    if (tid < n) {
-      float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
-      const float sc = __fdiv_rn(colsum[tid], (float)(lay.G * max(1, nnz.v[tid])));
-      reinterpret_cast<float*>(ub + lay.off_scores)[tid] = sc;
-      colsum[tid] = 0.f;
-      key = __float_as_uint(sc);   // scores are non-negative: unsigned order is float order
-    }
-    s_key[tid] = key;
-  }
-  for (int i = tid; i < 2 * 2 * ZC_D; i += kFlushThreads) (&s_cmax[0][0][0])[i] = 0u;
-  if (tid < 2 * ZC_TILE) s_tok[tid] = -1;
-  if (tid < 2) s_smax[tid] = 0u;
-  __syncthreads();
-
-  // ---- split: the n_s largest scores, equal scores by lowest index; both lists ascending ----
-  if (tid < ZC_MAX_WINDOW) {
-    bool sal = false;
-    if (tid < n) {
-      const unsigned mine = s_key[tid];
-      int rank = 0;
-      for (int i = 0; i < n; ++i) {
-        const unsigned k = s_key[i];
-        rank += (k > mine || (k == mine && i < tid)) ? 1 : 0;
-      }
-      sal = rank < n_s;
-    }
-    const unsigned m = __ballot_sync(0xffffffffu, sal);
-    if (lane == 0) s_mask[w] = m;
-  }
-  __syncthreads();
-  if (tid < n) {
-    int before = __popc(s_mask[w] & ((1u << lane) - 1u));
-    for (int i = 0; i < w; ++i) before += __popc(s_mask[i]);
-    const bool sal = (s_mask[w] >> lane) & 1u;
-    int32_t* idx = reinterpret_cast<int32_t*>(ub + lay.off_idx) + seg.idx_off;
-    if (sal) {
-      idx[before] = tid;
-      s_tok[before] = tid;
-    } else {
-      idx[n_s + tid - before] = tid;
-      s_tok[ZC_TILE + tid - before] = tid;
-    }
-  }
-  __syncthreads();
-
-  // ---- this warp's four token rows; channel |x| maxima of the class (Eq. 6) ----
-  const int cls = w >> 4;
-  const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh;
-  const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
-  uint2 rawK[4], rawV[4];
-  bool live[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int tok = s_tok[4 * w + i];
-    live[i] = tok >= 0;
-    if (live[i]) {
-      const long long row = (long long)tok * src.sl;
-      rawK[i] = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
-      rawV[i] = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
-    } else {
-      rawK[i] = make_uint2(0, 0);
-      rawV[i] = make_uint2(0, 0);
-    }
-  }
-  {
-    float mk[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const T* ek = reinterpret_cast<const T*>(&rawK[i]);
-      const T* ev = reinterpret_cast<const T*>(&rawV[i]);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        mk[e] = fmaxf(mk[e], fabsf(zc_to_float<T>(ek[e])));
-        mv[e] = fmaxf(mv[e], fabsf(zc_to_float<T>(ev[e])));
-      }
-    }
-    if (live[0]) {   // slots fill from the front: a warp without a first token has none
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        atomicMax(&s_cmax[cls][0][4 * lane + e], __float_as_uint(mk[e]));
-        atomicMax(&s_cmax[cls][1][4 * lane + e], __float_as_uint(mv[e]));
-      }
-    }
-  }
-  __syncthreads();
-
-  // ---- CSTQuant of the warp's tokens ----
-  const int bits = lay.bits[cls];
-  const float L = (float)((1 << bits) - 1);
-  float cK[4], cV[4];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const float mk = __uint_as_float(s_cmax[cls][0][4 * lane + e]);
-    const float mv = __uint_as_float(s_cmax[cls][1][4 * lane + e]);
-    cK[e] = mk == 0.f ? 1.f : __fsqrt_rn(mk);
-    cV[e] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
-  }
-  float* fac = reinterpret_cast<float*>(ub + lay.off_fac) + (seg.run0 + cls) * ZC_FAC_FLOATS;
-  if ((w & 15) == 0 && seg.n_tok[cls] > 0) {
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      fac[4 * lane + e] = cK[e];
-      fac[ZC_D + 4 * lane + e] = cV[e];
-    }
-  }
-  float smax = 0.f;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int slot = 4 * w + i;
-    float x[4], sc, z;
-    unsigned pk;
-    const T* ek = reinterpret_cast<const T*>(&rawK[i]);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
-    quant_token(x, cK, L, &sc, &z, &pk);
-    *reinterpret_cast<unsigned*>(&codesK[slot][4 * lane]) = live[i] ? pk : 0u;
-    if (lane == 0) { parK[slot][0] = live[i] ? sc : 0.f; parK[slot][1] = live[i] ? z : 0.f; }
-    const T* ev = reinterpret_cast<const T*>(&rawV[i]);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
-    quant_token(x, cV, L, &sc, &z, &pk);
-    *reinterpret_cast<unsigned*>(&codesV[slot][4 * lane]) = live[i] ? pk : 0u;
-    if (lane == 0) { parV[slot][0] = live[i] ? sc : 0.f; parV[slot][1] = live[i] ? z : 0.f; }
-    if (live[i]) smax = fmaxf(smax, sc);
-  }
-  if (lane == 0 && smax > 0.f) atomicMax(&s_smax[cls], __float_as_uint(smax));
-  __syncthreads();
-
-  // ---- both tiles ----
-  if (tid < 2)
-    reinterpret_cast<unsigned*>(ub + lay.off_fac)[(seg.run0 + tid) * ZC_FAC_FLOATS + 2 * ZC_D] = s_smax[tid];
-  const int vec0 = seg.n_tok[0] > 0 ? lay.tile_bytes[0] / 16 : 0;
-  const int vec1 = seg.n_tok[1] > 0 ? lay.tile_bytes[1] / 16 : 0;
-  for (int v = tid; v < vec0 + vec1; v += kFlushThreads) {
-    const int c2 = v < vec0 ? 0 : 1, vl = c2 == 0 ? v : v - vec0;
-    char* tile_ptr = ub + lay.off_tiles[c2] + (long long)seg.tile0[c2] * lay.tile_bytes[c2];
-    reinterpret_cast<uint4*>(tile_ptr)[vl] =
-        compose_vec(lay.bits[c2], vl, codesK + ZC_TILE * c2, codesV + ZC_TILE * c2, parK + ZC_TILE * c2,
-                    parV + ZC_TILE * c2);
-  }
+    reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(bits, v, 0, codesK, codesV, parK, parV);
 }
 
 }  // namespace
@@ -601,24 +350,5 @@ int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStre
     }
     c->launches += 2;
   }
-  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
-}
-
-bool zc_window_flush_fits(const zc_cache* c, const ZcSeg& seg) {
-  return c->cfg.window <= ZC_MAX_WINDOW && ZC_MAX_WINDOW <= 2 * ZC_TILE && seg.n_tok[0] <= ZC_TILE &&
-         seg.n_tok[1] <= ZC_TILE && seg.n_tok[0] + seg.n_tok[1] == c->cfg.window;
-}
-
-int zc_launch_window_flush(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st, bool chained) {
-  NnzArgs a;
-  for (int j = 0; j < ZC_MAX_WINDOW; ++j) a.v[j] = c->tail_nnz[j];
-  cudaError_t e;
-  if (c->cfg.dtype == ZC_F16)
-    e = launch_link(k_window_flush<__half>, dim3(c->lay.units), dim3(kFlushThreads), 0, st, chained, c->base,
-                    c->lay, src, seg, a);
-  else
-    e = launch_link(k_window_flush<__nv_bfloat16>, dim3(c->lay.units), dim3(kFlushThreads), 0, st, chained,
-                    c->base, c->lay, src, seg, a);
-  c->launches += 1;
   return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
 }

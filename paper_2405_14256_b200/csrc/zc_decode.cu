@@ -29,6 +29,7 @@
 #include "zc_layout.cuh"
 #include "zc_mma.cuh"
 #include "zc_order.h"
+#include "zc_quant.cuh"
 
 namespace {
 
@@ -742,6 +743,189 @@ __device__ __noinline__ void tail_phase(const T* tK, const T* tV, int G, int n_t
 // Merge of a unit's split-K partials (items, then the tail's tiles) in a fixed order,
 // the output row of every query head and, on probe steps, this step's attention over the
 // tail's tokens added to the window statistics.  Run by the CTA of the unit that finished last.
+// ------------------------------------------------------------------ window re-compression
+// Alg. 3: when a call completes the window, the CTA that merged a unit's partials turns the
+// unit's tail into a new segment: scores from the window statistics (which this call was the
+// last to add to), split, channel factors (Eq. 6), CSTQuant and packing, sub-block by
+// sub-block, with the arithmetic of the prefill kernels.  Everything it touches belongs to
+// the unit, so no other CTA is involved; the cache's next call waits for this one.
+constexpr int kFlOffCodesK = kOffQfrag;                                  // [16][128] bytes
+constexpr int kFlOffCodesV = kFlOffCodesK + ZC_SUB * ZC_D;
+constexpr int kFlOffParK = kFlOffCodesV + ZC_SUB * ZC_D;                 // [16][2] floats
+constexpr int kFlOffParV = kFlOffParK + ZC_SUB * 2 * 4;
+constexpr int kFlOffKey = kFlOffParV + ZC_SUB * 2 * 4;                   // [128] score bits
+constexpr int kFlOffTok = kFlOffKey + ZC_MAX_WINDOW * 4;                 // [2][128] token of each class slot
+constexpr int kFlOffRed = kFlOffTok + 2 * ZC_MAX_WINDOW * 4;             // [4 warps][2][128] floats
+constexpr int kFlOffC = kFlOffRed + kWarps * 2 * ZC_D * 4;               // [2][128] channel factors
+constexpr int kFlOffMask = kFlOffC + 2 * ZC_D * 4;                       // [4] ballots
+constexpr int kFlOffSmax = kFlOffMask + 16;                              // [2] V scale maxima as bits
+constexpr int kFlushSmem = kFlOffSmax + 16;
+static_assert(kFlushSmem <= decode_smem(kRingNarrow), "the re-compression must fit the item phase's memory");
+static_assert(ZC_MAX_WINDOW == 32 * kWarps, "one thread per window token");
+
+template <typename T>
+__device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay, const ZcFlushArgs& fl, char* smem) {
+  auto codesK = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesK);
+  auto codesV = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesV);
+  auto parK = reinterpret_cast<float (*)[2]>(smem + kFlOffParK);
+  auto parV = reinterpret_cast<float (*)[2]>(smem + kFlOffParV);
+  unsigned* s_key = reinterpret_cast<unsigned*>(smem + kFlOffKey);
+  auto s_tok = reinterpret_cast<int (*)[ZC_MAX_WINDOW]>(smem + kFlOffTok);
+  auto red = reinterpret_cast<float (*)[2][ZC_D]>(smem + kFlOffRed);
+  auto s_c = reinterpret_cast<float (*)[ZC_D]>(smem + kFlOffC);
+  unsigned* s_mask = reinterpret_cast<unsigned*>(smem + kFlOffMask);
+  unsigned* s_smax = reinterpret_cast<unsigned*>(smem + kFlOffSmax);
+  const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+  const int n = lay.window, n_s = fl.seg.n_tok[0];
+
+  // ---- scores of the window's tokens; the statistics start from zero for the next window ----
+  {
+    unsigned key = 0u;
+    if (tid < n) {
+      float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
+      const float sc = __fdiv_rn(colsum[tid], (float)(lay.G * max(1, (int)fl.nnz[tid])));
+      reinterpret_cast<float*>(ub + lay.off_scores)[tid] = sc;
+      colsum[tid] = 0.f;
+      key = __float_as_uint(sc);   // scores are non-negative: unsigned order is float order
+    }
+    s_key[tid] = key;
+    if (tid < 2) s_smax[tid] = 0u;
+  }
+  __syncthreads();
+  // ---- split: the n_s largest scores, equal scores by lowest index; both lists ascending ----
+  {
+    bool sal = false;
+    if (tid < n) {
+      const unsigned mine = s_key[tid];
+      int rank = 0;
+      for (int i = 0; i < n; ++i) {
+        const unsigned k = s_key[i];
+        rank += (k > mine || (k == mine && i < tid)) ? 1 : 0;
+      }
+      sal = rank < n_s;
+    }
+    const unsigned m = __ballot_sync(kFull, sal);
+    if (lane == 0) s_mask[w] = m;
+  }
+  __syncthreads();
+  if (tid < n) {
+    int before = __popc(s_mask[w] & ((1u << lane) - 1u));
+    for (int i = 0; i < w; ++i) before += __popc(s_mask[i]);
+    const bool sal = (s_mask[w] >> lane) & 1u;
+    int32_t* idx = reinterpret_cast<int32_t*>(ub + lay.off_idx) + fl.seg.idx_off;
+    if (sal) {
+      s_tok[0][before] = tid;
+      idx[before] = tid;
+    } else {
+      s_tok[1][tid - before] = tid;
+      idx[n_s + tid - before] = tid;
+    }
+  }
+  __syncthreads();
+
+  const T* tK = reinterpret_cast<const T*>(ub + lay.off_tailK);
+  const T* tV = reinterpret_cast<const T*>(ub + lay.off_tailV);
+  for (int cls = 0; cls < 2; ++cls) {
+    const int n_c = fl.seg.n_tok[cls];
+    if (n_c == 0) continue;
+    // ---- channel |x| maxima over the class (Eq. 6) ----
+    {
+      float mk[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int r = w; r < n_c; r += kWarps) {
+        const int row = s_tok[cls][r] * ZC_D;
+        float x[4];
+        zc_load4<T>(tK + row + 4 * lane, x);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mk[e] = fmaxf(mk[e], fabsf(x[e]));
+        zc_load4<T>(tV + row + 4 * lane, x);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) mv[e] = fmaxf(mv[e], fabsf(x[e]));
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        red[w][0][4 * lane + e] = mk[e];
+        red[w][1][4 * lane + e] = mv[e];
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int ten = 0; ten < 2; ++ten) {
+      float m = 0.f;
+#pragma unroll
+      for (int i = 0; i < kWarps; ++i) m = fmaxf(m, red[i][ten][tid]);
+      s_c[ten][tid] = m == 0.f ? 1.f : __fsqrt_rn(m);
+    }
+    __syncthreads();
+    const int bits = lay.bits[cls];
+    const float L = (float)((1 << bits) - 1);
+    float cK[4], cV[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      cK[e] = s_c[0][4 * lane + e];
+      cV[e] = s_c[1][4 * lane + e];
+    }
+    float* fac = reinterpret_cast<float*>(ub + lay.off_fac) + (fl.seg.run0 + cls) * ZC_FAC_FLOATS;
+    if (w == 0) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        fac[4 * lane + e] = cK[e];
+        fac[ZC_D + 4 * lane + e] = cV[e];
+      }
+    }
+    // ---- CSTQuant and packing, one 16-token sub-block at a time: four tokens per warp ----
+    float smax = 0.f;
+    const int subs = (n_c + ZC_SUB - 1) / ZC_SUB;
+    const int vecs = zc_sub_bytes(bits) / 16;
+    for (int sb = 0; sb < subs; ++sb) {
+      uint2 rawK[4], rawV[4];
+      bool live[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int tt = ZC_SUB * sb + 4 * w + i;
+        live[i] = tt < n_c;
+        rawK[i] = make_uint2(0, 0);
+        rawV[i] = make_uint2(0, 0);
+        if (live[i]) {
+          const int row = s_tok[cls][tt] * ZC_D;
+          rawK[i] = *reinterpret_cast<const uint2*>(tK + row + 4 * lane);
+          rawV[i] = *reinterpret_cast<const uint2*>(tV + row + 4 * lane);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int tl = 4 * w + i;
+        float x[4], sc, z;
+        unsigned pk;
+        const T* ek = reinterpret_cast<const T*>(&rawK[i]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
+        quant_token(x, cK, L, &sc, &z, &pk);
+        *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live[i] ? pk : 0u;
+        if (lane == 0) { parK[tl][0] = live[i] ? sc : 0.f; parK[tl][1] = live[i] ? z : 0.f; }
+        const T* ev = reinterpret_cast<const T*>(&rawV[i]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
+        quant_token(x, cV, L, &sc, &z, &pk);
+        *reinterpret_cast<unsigned*>(&codesV[tl][4 * lane]) = live[i] ? pk : 0u;
+        if (lane == 0) { parV[tl][0] = live[i] ? sc : 0.f; parV[tl][1] = live[i] ? z : 0.f; }
+        if (live[i]) smax = fmaxf(smax, sc);
+      }
+      __syncthreads();
+      const int sub_in_tile = sb % (ZC_TILE / ZC_SUB);
+      char* tile_ptr = ub + lay.off_tiles[cls] +
+                       (long long)(fl.seg.tile0[cls] + sb / (ZC_TILE / ZC_SUB)) * lay.tile_bytes[cls];
+      for (int v = tid; v < vecs; v += 128)
+        reinterpret_cast<uint4*>(tile_ptr)[sub_in_tile * vecs + v] =
+            compose_vec(bits, sub_in_tile * vecs + v, ZC_SUB * sub_in_tile, codesK, codesV, parK, parV);
+      __syncthreads();   // the next sub-block reuses the code arrays
+    }
+    if (lane == 0 && smax > 0.f) atomicMax(&s_smax[cls], __float_as_uint(smax));
+  }
+  __syncthreads();
+  if (tid < 2)
+    reinterpret_cast<unsigned*>(ub + lay.off_fac)[(fl.seg.run0 + tid) * ZC_FAC_FLOATS + 2 * ZC_D] = s_smax[tid];
+}
+
 template <typename T>
 __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_tail, T* __restrict__ out_unit,
                                         const float* mine, const float* stash_g, int collect, char* smem) {
@@ -837,7 +1021,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
                                                       const T* __restrict__ q, T* __restrict__ out,
                                                       float* part, float* stash_all, int slot,
                                                       int collect, const T* k_new, const T* v_new,
-                                                      ZcOrder ord) {
+                                                      ZcOrder ord, ZcFlushArgs fl) {
   extern __shared__ __align__(128) char smem[];
   const int G = lay.G, zs = (G + 3) >> 2;
   const int groups = (plan.items + plan.cta_items - 1) / plan.cta_items;   // item CTAs per head group
@@ -976,9 +1160,14 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     *s_last = last;
   }
   __syncthreads();
-  if (*s_last)
+  if (*s_last) {
     merge_unit<T>(reinterpret_cast<float*>(ub + lay.off_colsum), G, plan.items, plan.n_tail,
                 out + ((long long)b * lay.n_kv * G + kv * G) * ZC_D, mine, stash_g, collect, smem);
+    if (fl.on) {
+      __syncthreads();   // the merge is done with the shared arrays; its additions to the statistics are visible
+      window_flush_unit<T>(ub, lay, fl, smem);
+    }
+  }
 }
 
 }  // namespace
@@ -1057,7 +1246,11 @@ int zc_order_words(unsigned** ptr) {
 }
 
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
-                     char* ws, size_t ws_bytes, const void* k_new, const void* v_new, cudaStream_t st) {
+                     char* ws, size_t ws_bytes, const void* k_new, const void* v_new,
+                     const ZcFlushArgs* flush, cudaStream_t st) {
+  ZcFlushArgs fl;
+  if (flush) fl = *flush;
+  else memset(&fl, 0, sizeof(fl));
   static_assert(2 * kZcStreamRecs == 32, "two order words per stream record");
   const int G = c->lay.G, zs = (G + 3) / 4;
   const size_t io_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * ZC_D * 2;
@@ -1090,7 +1283,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   call.me.out = zc_range(out, io_bytes);
   call.cache = c;
   call.collect = collect;
-  call.stores_tail_row = k_new != nullptr;
+  call.changes_cache = k_new != nullptr || fl.on;
   call.ws = ws;
   call.ws_bytes = ws_bytes;
   call.need = need;
@@ -1134,7 +1327,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
     }                                                                                              \
     e = launch_pdl(k_decode<T, RING, NCTA>, grid, dim3(128), decode_smem(RING), st, overlap,       \
                    c->base, c->lay, plan, (const T*)q, (T*)out, part, stash, slot, collect,        \
-                   (const T*)k_new, (const T*)v_new, ord);                                         \
+                   (const T*)k_new, (const T*)v_new, ord, fl);                                     \
   } while (0)
   if (c->cfg.dtype == ZC_F16) {
     if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(__half, kRingNarrow, 4);

@@ -414,31 +414,25 @@ static int decode_attention(zc_cache* c, const void* q, void* out, int is_probe_
   const void* pk = c->pend_k;
   const void* pv = c->pend_v;
   c->pend_k = c->pend_v = nullptr;
-  ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (char*)workspace, workspace_bytes, pk, pv, st));
+  // Alg. 3: the call that completes the window also re-compresses it (inside its kernel)
+  const bool completes = c->n_tail > 0 && i_next == c->cfg.window && c->n_tail == c->cfg.window;
+  ZcFlushArgs fl;
+  memset(&fl, 0, sizeof(fl));
+  if (completes) {
+    fl.on = 1;
+    fl.seg = zc_segment(c, c->n_seg);
+    for (int j = 0; j < c->n_tail; ++j) fl.nnz[j] = (unsigned char)(c->tail_nnz[j] + (collect ? 1 : 0));
+  }
+  ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (char*)workspace, workspace_bytes, pk, pv,
+                           completes ? &fl : nullptr, st));
   // Alg. 3 bookkeeping: the step counter follows the tokens of the current window
   if (c->n_tail > 0) {
     c->step_i = i_next;
     if (collect)
       for (int j = 0; j < c->n_tail; ++j) c->tail_nnz[j] += 1;
-    if (c->step_i == c->cfg.window && c->n_tail == c->cfg.window) {
-      // re-compress the window into a new segment
-      // the re-compression runs as links of the decode calls' chain: calls on other caches
-      // that follow on the stream start without waiting for it
+    if (completes) {
       c->last_scores_n = c->cfg.window;
-      const int seg = c->n_seg;
       c->n_seg += 1;
-      ZcSeg s = zc_segment(c, seg);
-      const long long us = c->lay.unit_stride / 2;
-      ZcSrc src{c->base + c->lay.off_tailK, c->base + c->lay.off_tailV, us * c->lay.n_kv, us,
-                ZC_D};
-      if (zc_window_flush_fits(c, s)) {
-        ZC_CUDA(zc_launch_window_flush(c, src, s, st, true));
-      } else {
-        ZC_CUDA(zc_launch_window_scores(c, st, true));
-        ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], s.idx_off, nullptr, st, true));
-        ZC_CUDA(zc_launch_quantize(c, src, s, st, true));
-      }
-      zc_order_fence(c, st);
       c->n_tail = 0;
       c->step_i = 0;
       memset(c->tail_nnz, 0, sizeof(c->tail_nnz));

@@ -67,6 +67,14 @@ struct ZcSeg {
   int run0;        // factor-block index of class 0 (class 1 = run0 + 1)
 };
 
+// Re-compression of the window by the decode call that completes it (Alg. 3).
+struct ZcFlushArgs {
+  int on;
+  ZcSeg seg;                             // the segment the window becomes
+  unsigned char nnz[ZC_MAX_WINDOW];      // per tail token: probe steps that saw it
+};
+static_assert(ZC_MAX_WINDOW <= 255, "probe-step counts are kept in bytes");
+
 // Split-K plan of one decode call (identical for every unit).
 struct ZcDecodePlan {
   int n_seg;
@@ -146,9 +154,9 @@ int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
                      cudaStream_t st);
 // k_new / v_new non-null: the newest tail row is read from them and stored into the tail.
 // Calls that may be in flight together on a stream take consecutive regions of ws.
-int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out,
-                     int collect, char* ws, size_t ws_bytes, const void* k_new, const void* v_new,
-                     cudaStream_t st);
+int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
+                     char* ws, size_t ws_bytes, const void* k_new, const void* v_new,
+                     const ZcFlushArgs* flush, cudaStream_t st);
 // Bytes of ws one call of `items` items per unit takes.
 size_t zc_decode_scratch_bytes(const zc_cache* c, int items);
 int zc_device_error_code(int* out);

@@ -70,8 +70,8 @@ ZcOrderSlot zc_order_next(ZcOrderTable* t, ZcFence* fence, const ZcOrderCall& ca
     s.need_start = std::max(s.need_start, fence->e);
   s.slot = e % r->K;
   s.ws_off = (size_t)s.slot * r->slot_bytes;
-  if (call.stores_tail_row) {
-    // this call stores a tail row that the cache's next call reads from the tail buffer
+  if (call.changes_cache) {
+    // what this call stores in the cache, the cache's next call reads
     fence->rec = rec;
     fence->tag = r->tag;
     fence->e = e + 1;
@@ -134,7 +134,7 @@ extern "C" int zc_order_model_call(uint64_t stream_id, int cache_id, const uint6
   call.me.out = zc_range((const void*)(uintptr_t)addr[3], (size_t)io_bytes);
   call.cache = &g_model_fence[cache_id];
   call.collect = collect;
-  call.stores_tail_row = addr[1] != 0;
+  call.changes_cache = addr[1] != 0;
   call.ws = (const char*)(uintptr_t)ws_addr;
   call.ws_bytes = (size_t)ws_bytes;
   call.need = (size_t)need;

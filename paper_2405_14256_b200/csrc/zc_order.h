@@ -53,7 +53,7 @@ struct ZcOrderCall {
   ZcCallRec me;
   const void* cache;
   int collect;
-  int stores_tail_row;              // the call copies k_new / v_new into the cache's tail
+  int changes_cache;                // the call stores a tail row or re-compresses the window
   const char* ws;
   size_t ws_bytes;
   size_t need;                      // workspace bytes of this call

@@ -1,0 +1,88 @@
+// CSTQuant (Alg. 1, Eq. 5) of one token row and the composition of packed cache tiles: shared
+// by the prefill compression kernels and the window re-compression inside the decode kernel.
+#pragma once
+
+#include "zc_internal.h"
+#include "zc_layout.cuh"
+
+// Normative fp32 sequence (each step one IEEE operation, round to nearest even, nothing
+// fused): c = sqrt(max|x|) (1 if the channel is all zero); y = x / c; per token mn, mx over
+// the 128 channels; s = (mx - mn) / L, or |mn| (1 if mn == 0) when mx == mn;
+// z = -rint(mn / s); code = clamp(rint(y / s) + z, 0, L).
+static __device__ __forceinline__ void quant_token(const float (&x)[4], const float (&c)[4], float L,
+                                            float* s_out, float* z_out, unsigned* codes4) {
+  float y[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) y[e] = __fdiv_rn(x[e], c[e]);
+  float mn = fminf(fminf(y[0], y[1]), fminf(y[2], y[3]));
+  float mx = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  }
+  float s = __fdiv_rn(__fsub_rn(mx, mn), L);
+  if (mx == mn) s = mn != 0.f ? fabsf(mn) : 1.f;
+  const float z = -rintf(__fdiv_rn(mn, s));
+  unsigned packed = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float q = __fadd_rn(rintf(__fdiv_rn(y[e], s)), z);
+    q = fminf(fmaxf(q, 0.f), L);
+    packed |= ((unsigned)(int)q) << (8 * e);
+  }
+  *s_out = s;
+  *z_out = z;
+  *codes4 = packed;
+}
+
+// One 16-byte vector v of a cache tile from byte codes and per-token (s, z), the arrays holding
+// the tile's tokens from token row0 on: K codes in canonical order, V codes in fragment order, then the parameters, per
+// 16-token sub-block.
+static __device__ __forceinline__ uint4 compose_vec(int bits, int v, int row0, const unsigned char (*codesK)[ZC_D],
+                                             const unsigned char (*codesV)[ZC_D], const float (*parK)[2],
+                                             const float (*parV)[2]) {
+  const int sub_words = zc_sub_bytes(bits) / 4;
+  const int kw = 64 * bits;                           // K-code words per sub-block (= V-code words)
+  const int per = 32 / bits;                          // codes per word
+  unsigned out[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int wi = 4 * v + q;
+    const int st = wi / sub_words, wl = wi % sub_words;
+    unsigned word = 0;
+    if (wl < kw) {
+      // K: canonical order, token row of 4*bits words
+      const int words_per_row = 4 * bits;
+      const int tok = 16 * st - row0 + wl / words_per_row, wr = wl % words_per_row;
+      for (int e = 0; e < per; ++e) word |= (unsigned)codesK[tok][wr * per + e] << (bits * e);
+    } else if (wl < 2 * kw) {
+      // V: fragment order of the 16-token sub-tile
+      const int wv = wl - kw;
+      if (bits == 4) {
+        const int qd = wv >> 7, ln = (wv >> 2) & 31, jj = wv & 3;
+        const int j = 4 * qd + jj, g = ln >> 2, t = ln & 3;
+        for (int p = 0; p < 8; ++p) {
+          const int hi_row = p & 1, isB = (p >> 1) & 1, is1 = p >> 2;
+          const int ch = 16 * j + g + 8 * hi_row, tau = 2 * t + isB + 8 * is1;
+          word |= (unsigned)codesV[16 * st - row0 + tau][ch] << (4 * p);
+        }
+      } else {
+        const int ln = wv >> 2, m = wv & 3, g = ln >> 2, t = ln & 3;
+        for (int i = 0; i < 16; ++i) {
+          const int is1 = i >> 3, pp = i & 7, e2 = pp >> 2, hi_row = (pp >> 1) & 1, isB = pp & 1;
+          const int j = 2 * m + e2;
+          const int ch = 16 * j + g + 8 * hi_row, tau = 2 * t + isB + 8 * is1;
+          word |= (unsigned)codesV[16 * st - row0 + tau][ch] << (2 * i);
+        }
+      }
+    } else {
+      const int wp = wl - 2 * kw;  // params: (sK, zK, sV, zV) per token
+      const int tk = 16 * st - row0 + (wp >> 2), f = wp & 3;
+      word = __float_as_uint(f < 2 ? parK[tk][f] : parV[tk][f - 2]);
+    }
+    out[q] = word;
+  }
+  return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
