@@ -199,7 +199,7 @@ int zc_device_status(int* code);
 
 /* Host-only model of the ordering the library applies to zc_decode_attention calls issued on
  * one stream (the contract stated at zc_decode_attention): what each call's kernel waits for
- * before it reads its inputs and before it writes.  These three functions make no CUDA call,
+ * before it reads its inputs and before it writes.  These two functions make no CUDA call,
  * need no device and keep a table of their own, apart from the one real calls use; they exist
  * so that the rules can be checked on any machine.  Not thread-safe.
  *
@@ -207,7 +207,7 @@ int zc_device_status(int* code);
  *
  * zc_order_model_call books one call.  stream_id: any integer naming the stream; cache_id in
  * [0, 16) names the cache; addr [host] = the addresses of q, k_new, v_new, out as integers
- * (k_new = v_new = 0: the call stores no tail row), of io_bytes (q, out) and kv_bytes (k_new,
+ * (k_new = v_new = 0: the call changes nothing in the cache), of io_bytes (q, out) and kv_bytes (k_new,
  * v_new); collect = is_probe_step; ws_addr / ws_bytes = the workspace, need = the bytes one
  * call uses of it; capture_id = 0 outside stream capture, else the capture's id.
  * result [host, 8 ints] = {epoch_start (1: launched without early start, everything issued
@@ -217,14 +217,11 @@ int zc_device_status(int* code);
  * arrival counter), tag (12-bit epoch number), record (stream record used), drain (1: the
  * record was taken from another stream, which a real call drains first)}.
  * Returns ZC_OK, or ZC_EINVAL (null pointer, cache_id out of range, need = 0 or > ws_bytes).
- *
- * zc_order_model_fence notes that kernels chained behind the calls issued so far on the
- * stream change the cache (what the library does after re-compressing a window). */
+ */
 void zc_order_model_reset(void);
 int zc_order_model_call(uint64_t stream_id, int cache_id, const uint64_t addr[4], uint64_t io_bytes,
                         uint64_t kv_bytes, int collect, uint64_t ws_addr, uint64_t ws_bytes,
                         uint64_t need, uint64_t capture_id, int result[8]);
-int zc_order_model_fence(uint64_t stream_id, int cache_id);
 
 const char* zc_strerror(int status);
 

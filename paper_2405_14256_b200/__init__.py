@@ -13,5 +13,5 @@ from .binding import (  # noqa: F401
     zc_export_scores,
     zc_export_segment, zc_segment_tokens, zc_num_segments, zc_tail_tokens,
     zc_decode_bytes, zc_launch_count, zc_strerror, zc_device_status, ZipCache,
-    zc_order_model_reset, zc_order_model_call, zc_order_model_fence,
+    zc_order_model_reset, zc_order_model_call,
 )

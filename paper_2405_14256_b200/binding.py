@@ -68,7 +68,6 @@ _SIGS = {
     "zc_order_model_call": (C.c_int, [C.c_uint64, C.c_int, C.POINTER(C.c_uint64), C.c_uint64, C.c_uint64,
                                       C.c_int, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint64,
                                       C.POINTER(C.c_int)]),
-    "zc_order_model_fence": (C.c_int, [C.c_uint64, C.c_int]),
     "zc_strerror": (C.c_char_p, [C.c_int]),
 }
 
@@ -235,10 +234,6 @@ def zc_order_model_call(stream_id, cache_id, q, k_new, v_new, out, io_bytes, kv_
     _check(lib().zc_order_model_call(stream_id, cache_id, addr, io_bytes, kv_bytes, int(collect),
                                      ws_addr, ws_bytes, need, capture_id, res), "zc_order_model_call")
     return dict(zip(ORDER_FIELDS, list(res)))
-
-
-def zc_order_model_fence(stream_id, cache_id) -> None:
-    _check(lib().zc_order_model_fence(stream_id, cache_id), "zc_order_model_fence")
 
 
 class ZipCache:

@@ -1,36 +1,10 @@
 // Split by saliency (Alg. 2 "Split"), channel factors (Eq. 6), CSTQuant (Alg. 1, Eq. 5)
-// and packing into cache tiles; also the window statistics -> score step of Alg. 3.
+// and packing into cache tiles, for the prefill compression.
 #include "zc_internal.h"
 #include "zc_layout.cuh"
 #include "zc_quant.cuh"
 
 namespace {
-
-// The kernels of a re-compression can be launched as links of the decode calls' chain
-// (programmatic dependent launch): each lets its successor start at once and itself waits for
-// its predecessor to complete, so the decode calls of other caches that follow on the stream
-// are not held up.  In an ordinary launch both instructions do nothing.
-__device__ __forceinline__ void chain_link() {
-  asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
-  asm volatile("griddepcontrol.wait;\n" ::: "memory");
-}
-
-template <typename... KArgs, typename... Args>
-cudaError_t launch_link(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                        bool chained, Args... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = chained ? 1 : 0;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
-}
-
 
 // ------------------------------------------------------------------ top-k split
 // One CTA per unit.  Keys are the bit patterns of the (non-negative) scores, so unsigned
@@ -69,7 +43,6 @@ __device__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
 __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayout lay, int n, int n_s,
                                                              int idx_off,
                                                              const int32_t* __restrict__ given) {
-  chain_link();
   __shared__ int hist[256];
   __shared__ int warp_sums[32];
   __shared__ int s_total;
@@ -156,26 +129,10 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayo
   }
 }
 
-// ------------------------------------------------------------------ window scores
-struct NnzArgs { int v[ZC_MAX_WINDOW]; };
-
-__global__ void k_window_scores(char* cache, ZcLayout lay, NnzArgs nnz) {
-  chain_link();
-  char* ub = zc_unit_base(cache, lay, blockIdx.x);
-  float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
-  float* scores = reinterpret_cast<float*>(ub + lay.off_scores);
-  const int j = threadIdx.x;
-  if (j < lay.window) {
-    scores[j] = __fdiv_rn(colsum[j], (float)(lay.G * max(1, nnz.v[j])));
-    colsum[j] = 0.f;
-  }
-}
-
 // ------------------------------------------------------------------ channel |x| max (Eq. 6)
 // grid.x: tiles of class 0 then tiles of class 1; grid.y: unit.  blockDim 256.
 template <typename T>
 __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
-  chain_link();
   __shared__ float red[2][8][ZC_D];
   const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
   const int tiles_c0 = zc_ceil_div(seg.n_tok[0], ZC_TILE);
@@ -218,7 +175,6 @@ __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout la
 }
 
 __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
-  chain_link();
   char* ub = zc_unit_base(cache, lay, blockIdx.x);
   unsigned* cmax = reinterpret_cast<unsigned*>(ub + lay.off_cmax);
   for (int i = threadIdx.x; i < 4 * ZC_D; i += blockDim.x) cmax[i] = 0u;
@@ -229,7 +185,6 @@ __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
 // ------------------------------------------------------------------ CSTQuant + pack (arithmetic in zc_quant.cuh)
 template <typename T>
 __global__ void __launch_bounds__(256, 3) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
-  chain_link();
   __shared__ __align__(16) unsigned char codesK[ZC_TILE][ZC_D];
   __shared__ __align__(16) unsigned char codesV[ZC_TILE][ZC_D];
   __shared__ __align__(16) float parK[ZC_TILE][2];
@@ -312,43 +267,31 @@ __global__ void __launch_bounds__(256, 3) k_quantize_pack(char* cache, ZcLayout 
 }  // namespace
 
 int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
-                   cudaStream_t st, bool chained) {
+                   cudaStream_t st) {
   const int smem = given_sal ? ((n + 31) / 32) * 4 : 0;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(k_topk_split, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
   }
-  cudaError_t e = launch_link(k_topk_split, dim3(c->lay.units), dim3(kTopkThreads), (size_t)smem, st, chained,
-                              c->base, c->lay, n, n_s, idx_off, given_sal);
+  k_topk_split<<<c->lay.units, kTopkThreads, (size_t)smem, st>>>(c->base, c->lay, n, n_s, idx_off, given_sal);
   c->launches += 1;
-  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
+  return (int)cudaGetLastError();
 }
 
-int zc_launch_window_scores(zc_cache* c, cudaStream_t st, bool chained) {
-  NnzArgs a;
-  for (int j = 0; j < ZC_MAX_WINDOW; ++j) a.v[j] = c->tail_nnz[j];
-  cudaError_t e = launch_link(k_window_scores, dim3(c->lay.units), dim3(ZC_MAX_WINDOW), 0, st, chained,
-                              c->base, c->lay, a);
-  c->launches += 1;
-  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
-}
-
-int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st, bool chained) {
+int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st) {
   const int tiles = zc_ceil_div(seg.n_tok[0], ZC_TILE) + zc_ceil_div(seg.n_tok[1], ZC_TILE);
-  cudaError_t e = launch_link(k_clear_cmax, dim3(c->lay.units), dim3(128), 0, st, chained, c->base, c->lay, seg);
+  k_clear_cmax<<<c->lay.units, 128, 0, st>>>(c->base, c->lay, seg);
   c->launches += 1;
-  if (e == cudaSuccess && tiles > 0) {
+  if (tiles > 0) {
     dim3 grid(tiles, c->lay.units);
     if (c->cfg.dtype == ZC_F16) {
-      e = launch_link(k_channel_absmax<__half>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
-      if (e == cudaSuccess)
-        e = launch_link(k_quantize_pack<__half>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
+      k_channel_absmax<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_quantize_pack<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
     } else {
-      e = launch_link(k_channel_absmax<__nv_bfloat16>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
-      if (e == cudaSuccess)
-        e = launch_link(k_quantize_pack<__nv_bfloat16>, grid, dim3(256), 0, st, chained, c->base, c->lay, src, seg);
+      k_channel_absmax<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_quantize_pack<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
     }
     c->launches += 2;
   }
-  return e != cudaSuccess ? (int)e : (int)cudaGetLastError();
+  return (int)cudaGetLastError();
 }

@@ -1216,13 +1216,6 @@ size_t zc_decode_scratch_bytes(const zc_cache* c, int items) {
   return ((part + 255) & ~(size_t)255) + ((stash + 255) & ~(size_t)255);
 }
 
-void zc_order_fence(zc_cache* c, cudaStream_t st) {
-  int dev = 0;
-  cudaGetDevice(&dev);
-  std::lock_guard<std::mutex> lock(g_table_mutex);
-  zc_order_fence_at(&g_table, &c->fence, (const void*)st, dev);
-}
-
 // One word per stream record, in the library image (like the built-in scratch below).
 // Two per record: calls issued under stream capture use the second, so that replaying a
 // captured graph never disturbs the word of the calls issued directly.

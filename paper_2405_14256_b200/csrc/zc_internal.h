@@ -90,8 +90,8 @@ struct ZcDecodePlan {
   int l0;
 };
 
-// Where in a stream's sequence of decode calls a cache was last changed by something other
-// than a decode call's own output (see zc_order.h).
+// Where in a stream's sequence of decode calls a cache was last changed (a stored tail row,
+// a re-compressed window); see zc_order.h.
 struct ZcFence {
   int rec;          // stream record, -1: none
   unsigned tag;     // epoch
@@ -135,21 +135,9 @@ ZcDecodePlan zc_make_plan(const zc_cache* c);
 int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l,
                            const int64_t* qs, const int64_t* ks, const int32_t* P_dev,
                            int n_probe, float* lse_ws, void* qp_ws, size_t qp_bytes, cudaStream_t st);
-// chained: launched as a link of the decode calls' chain on the stream (see zc_compress.cu);
-// the caller then fences the cache with zc_order_fence.
 int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
-                   cudaStream_t st, bool chained = false);
-int zc_launch_window_scores(zc_cache* c, cudaStream_t st, bool chained = false);
-int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st,
-                       bool chained = false);
-// The whole re-compression of a window (scores, split, factors, quantise, pack) as one kernel,
-// for windows whose two classes fit one tile each (zc_window_flush_fits).
-bool zc_window_flush_fits(const zc_cache* c, const ZcSeg& seg);
-int zc_launch_window_flush(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st,
-                           bool chained = false);
-// Marks the cache as changed by kernels just launched on st: decode calls on this cache
-// that follow within the same epoch wait for them before they read anything.
-void zc_order_fence(zc_cache* c, cudaStream_t st);
+                   cudaStream_t st);
+int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st);
 int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
                      cudaStream_t st);
 // k_new / v_new non-null: the newest tail row is read from them and stored into the tail.

@@ -64,8 +64,7 @@ ZcOrderSlot zc_order_next(ZcOrderTable* t, ZcFence* fence, const ZcOrderCall& ca
     if (meet(call.me.out, o.out) || (call.collect && o.collected == call.cache))
       s.need_end = std::max(s.need_end, i + 1);
   }
-  // kernels chained behind an earlier call changed this cache (a re-compressed window), or an
-  // earlier call stored a tail row
+  // an earlier call stored a tail row of this cache or re-compressed its window
   if (e > 0 && fence->rec == rec && fence->tag == r->tag && fence->capturing == call.capturing)
     s.need_start = std::max(s.need_start, fence->e);
   s.slot = e % r->K;
@@ -82,19 +81,6 @@ ZcOrderSlot zc_order_next(ZcOrderTable* t, ZcFence* fence, const ZcOrderCall& ca
   r->e = e + 1;
   r->age = ++t->clock;
   return s;
-}
-
-void zc_order_fence_at(ZcOrderTable* t, ZcFence* fence, const void* st, int dev) {
-  fence->rec = -1;
-  for (int i = 0; i < kZcStreamRecs; ++i) {
-    const ZcStreamRec& r = t->rec[i];
-    if (r.used && r.st == st && r.dev == dev) {
-      fence->rec = i;
-      fence->tag = r.tag;
-      fence->e = r.e;              // the next call of the epoch publishes their completion
-      fence->capturing = r.capturing;
-    }
-  }
 }
 
 // ---- the model behind zc_order_model_*: the same rules on a table of its own ----
@@ -149,12 +135,5 @@ extern "C" int zc_order_model_call(uint64_t stream_id, int cache_id, const uint6
   result[5] = (int)s.tag;
   result[6] = s.rec;
   result[7] = s.drain ? 1 : 0;
-  return ZC_OK;
-}
-
-extern "C" int zc_order_model_fence(uint64_t stream_id, int cache_id) {
-  if (cache_id < 0 || cache_id >= kModelCaches) return ZC_EINVAL;
-  model_init();
-  zc_order_fence_at(&g_model, &g_model_fence[cache_id], (const void*)(uintptr_t)stream_id, 0);
   return ZC_OK;
 }

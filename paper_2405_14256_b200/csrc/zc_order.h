@@ -77,7 +77,3 @@ static inline ZcRange zc_range(const void* p, size_t n) {
 
 // Books the next call of a stream and returns what its kernel has to wait for.
 ZcOrderSlot zc_order_next(ZcOrderTable* t, ZcFence* fence, const ZcOrderCall& call);
-
-// Kernels chained behind the calls issued so far on (st, dev) change the cache: its next call
-// of the same epoch reads nothing before those calls, and with them the chain, have completed.
-void zc_order_fence_at(ZcOrderTable* t, ZcFence* fence, const void* st, int dev);

@@ -99,20 +99,11 @@ def test_a_stored_tail_row_is_complete_before_the_caches_next_call_reads_it(zc):
     assert r["need_start"] == 2
 
 
-def test_fence_after_chained_kernels(zc):
-    for i in range(5):
-        call(zc, cache=i % 2, q=0x1000_0000 + i * IO, out=0x2000_0000 + i * IO)
-    zc.zc_order_model_fence(1, 0)        # cache 0 re-compressed behind calls 0..4
-    r = call(zc, cache=1, q=0x1100_0000, out=0x2100_0000)
-    assert r["need_start"] <= 0
-    r = call(zc, cache=0, q=0x1200_0000, out=0x2200_0000)
-    assert r["need_start"] == 5
-    # a fence taken on another stream, or in an earlier epoch, means nothing: those kernels
-    # completed before this epoch's first launch
-    zc.zc_order_model_fence(1, 2)
+def test_a_change_in_an_earlier_epoch_needs_no_wait(zc):
+    call(zc, cache=2, q=0x1000_0000, k=0x3000_0000, v=0x3100_0000, out=0x2000_0000)
     call(zc, cache=3, q=0x1300_0000, out=0x2300_0000, ws_bytes=8 * NEED)   # new workspace: new epoch
     r = call(zc, cache=2, q=0x1400_0000, out=0x2400_0000, ws_bytes=8 * NEED)
-    assert r["e"] == 1 and r["need_start"] <= 0
+    assert r["e"] == 1 and r["need_start"] <= 0              # that kernel completed before the epoch began
 
 
 def test_epoch_restarts(zc):
