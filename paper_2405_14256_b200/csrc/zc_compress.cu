@@ -81,14 +81,32 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayo
         if ((k & mask_hi) == prefix) atomicAdd(&hist[(k >> shift) & 255], 1);
       }
       __syncthreads();
-      if (tid == 0) {
-        int krem = s_krem, b = 255;
-        for (; b > 0; --b) {
-          if (hist[b] >= krem) break;
-          krem -= hist[b];
+      // the bin, from the top, at which the count reaches the krem keys still wanted: lane l
+      // of warp 0 owns bins 255 - 8l down to 248 - 8l
+      if (tid < 32) {
+        const int krem = s_krem, top = 255 - 8 * tid;
+        int cnt[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { cnt[j] = hist[top - j]; sum += cnt[j]; }
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, incl, o);
+          if (tid >= o) incl += y;
         }
-        s_prefix = prefix | ((unsigned)b << shift);
-        s_krem = krem;
+        const int excl = incl - sum;
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        if ((excl < krem && krem <= incl) || (tid == 31 && total < krem)) {
+          int r = krem - excl, b = top;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            b = top - j;
+            if (b == 0 || cnt[j] >= r) break;
+            r -= cnt[j];
+          }
+          s_prefix = prefix | ((unsigned)b << shift);
+          s_krem = r;
+        }
       }
       __syncthreads();
     }
