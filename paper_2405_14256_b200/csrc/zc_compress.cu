@@ -148,14 +148,18 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayo
 }
 
 // ------------------------------------------------------------------ channel |x| max (Eq. 6)
-// grid.x: tiles of class 0 then tiles of class 1; grid.y: unit.  blockDim 256.
+// grid.x: groups of kAbsTiles tiles of class 0, then of class 1; grid.y: unit.  blockDim 256.
+// A CTA folds several tiles before it touches the unit's shared maxima: one atomic per
+// channel and CTA.
+constexpr int kAbsTiles = 4;
+
 template <typename T>
 __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
   __shared__ float red[2][8][ZC_D];
   const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
-  const int tiles_c0 = zc_ceil_div(seg.n_tok[0], ZC_TILE);
-  const int cls = (int)blockIdx.x < tiles_c0 ? 0 : 1;
-  const int tile = cls == 0 ? blockIdx.x : blockIdx.x - tiles_c0;
+  const int groups_c0 = zc_ceil_div(zc_ceil_div(seg.n_tok[0], ZC_TILE), kAbsTiles);
+  const int cls = (int)blockIdx.x < groups_c0 ? 0 : 1;
+  const int grp = cls == 0 ? blockIdx.x : blockIdx.x - groups_c0;
   char* ub = zc_unit_base(cache, lay, unit);
   const int32_t* idx = reinterpret_cast<const int32_t*>(ub + lay.off_idx) + seg.idx_off +
                        (cls == 0 ? 0 : seg.n_tok[0]);
@@ -163,20 +167,18 @@ __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout la
   const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   float mk[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
-  const int t0 = tile * ZC_TILE;
+  const int t_lo = grp * kAbsTiles * ZC_TILE;
+  const int t_hi = min(seg.n_tok[cls], t_lo + kAbsTiles * ZC_TILE);
+#pragma unroll 4
+  for (int tt = t_lo + w; tt < t_hi; tt += 8) {
+    const long long row = (long long)idx[tt] * src.sl;
+    float x[4];
+    zc_load4<T>(Kb + row + 4 * lane, x);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int tt = t0 + w + 8 * i;
-    if (tt < seg.n_tok[cls]) {
-      const long long row = (long long)idx[tt] * src.sl;
-      float x[4];
-      zc_load4<T>(Kb + row + 4 * lane, x);
+    for (int e = 0; e < 4; ++e) mk[e] = fmaxf(mk[e], fabsf(x[e]));
+    zc_load4<T>(Vb + row + 4 * lane, x);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) mk[e] = fmaxf(mk[e], fabsf(x[e]));
-      zc_load4<T>(Vb + row + 4 * lane, x);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) mv[e] = fmaxf(mv[e], fabsf(x[e]));
-    }
+    for (int e = 0; e < 4; ++e) mv[e] = fmaxf(mv[e], fabsf(x[e]));
   }
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
@@ -202,7 +204,7 @@ __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
 
 // ------------------------------------------------------------------ CSTQuant + pack (arithmetic in zc_quant.cuh)
 template <typename T>
-__global__ void __launch_bounds__(256, 3) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
+__global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
   __shared__ __align__(16) unsigned char codesK[ZC_TILE][ZC_D];
   __shared__ __align__(16) unsigned char codesV[ZC_TILE][ZC_D];
   __shared__ __align__(16) float parK[ZC_TILE][2];
@@ -237,40 +239,44 @@ __global__ void __launch_bounds__(256, 3) k_quantize_pack(char* cache, ZcLayout 
     }
   }
   const int t0 = tile * ZC_TILE;
-  // gather the warp's 8 token rows first (memory-level parallelism), then quantise
-  uint2 rawK[8], rawV[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int tt = t0 + w * 8 + i;
-    if (tt < seg.n_tok[cls]) {
-      const long long row = (long long)idx[tt] * src.sl;
-      rawK[i] = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
-      rawV[i] = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
-    } else {
-      rawK[i] = make_uint2(0, 0);
-      rawV[i] = make_uint2(0, 0);
-    }
-  }
+  // the warp's 8 token rows in two batches of four: gather a batch (memory-level parallelism),
+  // then quantise it
   float smax = 0.f;
+#pragma unroll 1
+  for (int half = 0; half < 2; ++half) {
+    uint2 rawK[4], rawV[4];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int tl = w * 8 + i, tt = t0 + tl;
-    const bool live = tt < seg.n_tok[cls];
-    float x[4], s, z;
-    unsigned pk;
-    const T* ek = reinterpret_cast<const T*>(&rawK[i]);
+    for (int i = 0; i < 4; ++i) {
+      const int tt = t0 + w * 8 + 4 * half + i;
+      if (tt < seg.n_tok[cls]) {
+        const long long row = (long long)idx[tt] * src.sl;
+        rawK[i] = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
+        rawV[i] = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
+      } else {
+        rawK[i] = make_uint2(0, 0);
+        rawV[i] = make_uint2(0, 0);
+      }
+    }
 #pragma unroll
-    for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
-    quant_token(x, cK, L, &s, &z, &pk);
-    *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live ? pk : 0u;
-    if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
-    const T* ev = reinterpret_cast<const T*>(&rawV[i]);
+    for (int i = 0; i < 4; ++i) {
+      const int tl = w * 8 + 4 * half + i, tt = t0 + tl;
+      const bool live = tt < seg.n_tok[cls];
+      float x[4], s, z;
+      unsigned pk;
+      const T* ek = reinterpret_cast<const T*>(&rawK[i]);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
-    quant_token(x, cV, L, &s, &z, &pk);
-    *reinterpret_cast<unsigned*>(&codesV[tl][4 * lane]) = live ? pk : 0u;
-    if (lane == 0) { parV[tl][0] = live ? s : 0.f; parV[tl][1] = live ? z : 0.f; }
-    if (live) smax = fmaxf(smax, s);
+      for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
+      quant_token(x, cK, L, &s, &z, &pk);
+      *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live ? pk : 0u;
+      if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
+      const T* ev = reinterpret_cast<const T*>(&rawV[i]);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
+      quant_token(x, cV, L, &s, &z, &pk);
+      *reinterpret_cast<unsigned*>(&codesV[tl][4 * lane]) = live ? pk : 0u;
+      if (lane == 0) { parV[tl][0] = live ? s : 0.f; parV[tl][1] = live ? z : 0.f; }
+      if (live) smax = fmaxf(smax, s);
+    }
   }
   if (lane == 0 && smax > 0.f) atomicMax(reinterpret_cast<unsigned*>(&fac[2 * ZC_D]), __float_as_uint(smax));
   __syncthreads();
@@ -302,11 +308,14 @@ int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStre
   c->launches += 1;
   if (tiles > 0) {
     dim3 grid(tiles, c->lay.units);
+    dim3 grid_max(zc_ceil_div(zc_ceil_div(seg.n_tok[0], ZC_TILE), kAbsTiles) +
+                      zc_ceil_div(zc_ceil_div(seg.n_tok[1], ZC_TILE), kAbsTiles),
+                  c->lay.units);
     if (c->cfg.dtype == ZC_F16) {
-      k_channel_absmax<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_channel_absmax<__half><<<grid_max, 256, 0, st>>>(c->base, c->lay, src, seg);
       k_quantize_pack<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
     } else {
-      k_channel_absmax<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_channel_absmax<__nv_bfloat16><<<grid_max, 256, 0, st>>>(c->base, c->lay, src, seg);
       k_quantize_pack<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
     }
     c->launches += 2;
