@@ -6,7 +6,9 @@
 // on tensor cores in the input type, in a CTA of its own or in the unit's first item CTA.  The
 // CTA of a unit that finishes last (an arrival counter tells) merges the unit's partials in a
 // fixed order, writes the output and, on probe steps, adds the step's attention over the
-// tail's tokens to the window statistics: one kernel per call, nothing spins on another CTA.
+// tail's tokens to the window statistics; when the call completes a window, the same CTA then
+// re-compresses the unit's tail into a new segment (Alg. 3).  One kernel per call, nothing
+// spins on another CTA.
 // Consecutive calls on a stream are chained by programmatic dependent launch and run side by
 // side; what orders them where they touch the same memory is described at ZcOrder and at
 // zc_launch_decode.

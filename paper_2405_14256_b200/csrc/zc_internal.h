@@ -120,7 +120,7 @@ struct zc_cache {
   const void* pend_k;
   const void* pend_v;
   cudaStream_t pend_stream;
-  // ordering of decode calls behind chained kernels that changed this cache (zc_order_fence)
+  // the cache's last change by a decode call (a stored tail row, a re-compressed window): its next call waits for it
   ZcFence fence;
 };
 
