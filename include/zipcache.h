@@ -128,8 +128,9 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
  * softmax(q K^T / sqrt(d)) V over every cached token, codes dequantised in the kernel.
  * The step counter of the current window advances; on a probe step (is_probe_step != 0,
  * or one of the last five steps of a window) this step's attention over the tail's
- * tokens is added to the window statistics; after the window's last step the tail is
- * re-compressed into a new segment (same stream, no host synchronisation).
+ * tokens is added to the window statistics; the call that takes the window's last step
+ * also re-compresses the tail into a new segment, inside the same kernel (no further launch,
+ * no host synchronisation).
  * Ordering: consecutive calls on one stream may run at the same time on the GPU.  The library
  * orders a call after the earlier ones whenever it reads or overwrites one of their outputs,
  * overwrites one of their inputs, or updates the same cache's window statistics; it cannot see
