@@ -45,6 +45,7 @@ def _check(w, got, ref_units):
 @pytest.mark.parametrize("layers,steps,kw", [
     (4, 40, dict(context=300, batch=2, n_q_heads=8, n_kv_heads=2, window=16)),      # 160 calls, 2 flushes per layer
     (1, 90, dict(context=200, batch=1, n_q_heads=4, n_kv_heads=4, window=100)),     # one cache, call after call
+    (2, 100, dict(context=150, batch=1, n_q_heads=4, n_kv_heads=2, window=16)),     # 6 windows: 14 items per unit
     (3, 30, dict(context=260, batch=2, n_q_heads=16, n_kv_heads=2, dtype="bf16")),  # two head groups per unit
 ])
 @pytest.mark.parametrize("overlap_items", [False, True])

@@ -136,6 +136,7 @@ def test_decode_attention_parity(kw, steps):
 
 @pytest.mark.parametrize("window,steps,ratio", [
     (16, 40, 0.4), (100, 105, 0.4),
+    (16, 100, 0.4),                   # six windows: more partials per unit than the merge keeps in registers
     (100, 105, 0.8),                  # 80 salient tokens: more than one tile in a class
     (16, 20, 0.0), (16, 20, 1.0),     # an empty class
     (128, 130, 0.5),                  # the largest window, both tiles full
