@@ -49,6 +49,32 @@ def test_noalloc_entry_matches_workspace_entry_two_calls_in_a_row(kw):
     assert torch.equal(ref_cache.mem, new_cache.mem)
 
 
+def test_noalloc_entry_across_a_recompressed_window():
+    """The call that completes a window re-compresses it inside the same kernel: through the
+    built-in buffer the cache must end up byte for byte as through a caller workspace."""
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(context=200, batch=2, n_q_heads=8, n_kv_heads=2, window=8)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w).tolist()
+    ref_cache, new_cache = tl.make_cache(w, max_new=32), tl.make_cache(w, max_new=32)
+    ref_cache.mem.zero_()
+    new_cache.mem.zero_()
+    ref_cache.prefill_compress(Q, K, V, P)
+    new_cache.prefill_compress(Q, K, V, P)
+    for step in range(19):                       # two windows and three steps of the third
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        ref_cache.append(k, v)
+        new_cache.append(k, v)
+        want = ref_cache.decode_attention(q, step % 3 == 0)
+        got = torch.empty_like(q)
+        zc.zc_decode_attention_noalloc(new_cache.handle, q, got, step % 3 == 0)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want), step
+    assert zc.zc_device_status() == 0
+    assert zc.zc_num_segments(new_cache.handle) == 3
+    assert torch.equal(ref_cache.mem, new_cache.mem)
+
+
 def test_noalloc_entry_rejects_shapes_beyond_its_buffer():
     import paper_2405_14256_b200 as zc
     # 128 x 32 heads: the split-K partials of one call alone exceed the 4 MiB buffer
