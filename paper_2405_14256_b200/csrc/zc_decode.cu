@@ -126,6 +126,13 @@ __device__ __forceinline__ unsigned ld_order(const unsigned* p) {
   asm volatile("ld.volatile.global.u32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+// The same read as an acquire: what the thread loads afterwards is ordered behind it, without
+// the cost of a fence.
+__device__ __forceinline__ unsigned ld_order_acquire(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ bool order_ok(unsigned v, unsigned tag, int need) {
   return (v >> 20) == tag && (int)(v & 0xFFFFFu) >= need;
 }
@@ -137,14 +144,11 @@ __device__ __noinline__ void order_wait_slow(const unsigned* p, unsigned tag, in
   }
   atomicExch(err, 2);
 }
-// acquire: the caller goes on to READ what the earlier call wrote (a fence orders those loads
-// behind the observation); stores and read-modify-writes issued afterwards need none.
-__device__ __forceinline__ void order_wait(const ZcOrder& o, unsigned first, int need, bool acquire, int* err) {
-  if (need <= 0) return;
-  if (order_ok(first, o.tag, need)) {
-    if (acquire) __threadfence();
-    return;
-  }
+// `first` is the value the thread read when it started: with ld_order_acquire if it goes on to
+// READ what the earlier call wrote (need_start), so those loads are ordered behind the
+// observation; stores and read-modify-writes issued after a wait need no such ordering.
+__device__ __forceinline__ void order_wait(const ZcOrder& o, unsigned first, int need, int* err) {
+  if (need <= 0 || order_ok(first, o.tag, need)) return;
   order_wait_slow(o.done, o.tag, need, err);
 }
 
@@ -732,7 +736,7 @@ __device__ __noinline__ void tail_phase(const T* tK, const T* tV, int G, int n_t
                                         float* part_unit, int first_entry, float* stash_g, const T* k_new,
                                         const T* v_new, ZcOrder ord, unsigned ord_first, int* err) {
   const int warp = threadIdx.x >> 5;
-  order_wait(ord, ord_first, ord.need_end, false, err);   // the workspace region is free
+  order_wait(ord, ord_first, ord.need_end, err);   // the workspace region is free
   for (int base = warp * ZC_SUB; base < n_tail; base += kWarps * ZC_SUB) {
     float* entry = part_unit + (long long)(first_entry + base / ZC_SUB) * G * ZC_PART_STRIDE;
     for (int hg = 0; hg * 4 < G; ++hg)
@@ -1050,10 +1054,10 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
   char* ub = zc_unit_base(cache, lay, unit);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // the stream's word is requested first and looked at when it is needed
-  const unsigned ord_first = (ord.need_start > 0 || ord.need_end > 0) ? ld_order(ord.done) : 0u;
+  const unsigned ord_first = ord.need_start > 0 ? ld_order_acquire(ord.done) : ord.need_end > 0 ? ld_order(ord.done) : 0u;
   pdl_launch_dependents();
   // inputs written by an earlier call, a re-compressed window, the previous call's tail row
-  order_wait(ord, ord_first, ord.need_start, true, &g_zc_error);
+  order_wait(ord, ord_first, ord.need_start, &g_zc_error);
   if (k_new && j == 0 && warp == kWarps - 1) {
     // Deferred append: the newest row goes into the tail for the steps to come (this step reads
     // it from k_new / v_new).  The next call on this cache is told to wait for this one.
@@ -1125,7 +1129,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
       s_head[tid * 4 + 2] = has ? zsum : 0.f;
     }
     __syncthreads();
-    order_wait(ord, ord_first, ord.need_end, false, &g_zc_error);   // the workspace region is free
+    order_wait(ord, ord_first, ord.need_end, &g_zc_error);   // the workspace region is free
     for (int h = 0; h < Gl; ++h) {
       float o = 0.f;
       if (has) {
