@@ -1147,8 +1147,8 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     if (it + 1 < it_end) __syncthreads();   // the next item reuses the rings and the small arrays
     }
   }
-  // ---- count in: the barrier orders every thread's stores before thread 0's fence, the fence
-  //      before the count; the CTA that finds all others counted reads their partials from L2 ----
+  // ---- count in: the barrier orders every thread's stores before thread 0's count; the CTA
+  //      that finds all others counted reads their partials from L2 ----
   __syncthreads();
   int* s_last = reinterpret_cast<int*>(smem + kCmbOffFlag);
   if (per_unit == 1) {
@@ -1156,13 +1156,12 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     if (tid == 0) *s_last = 1;
   } else if (tid == 0) {
     unsigned* cnt = reinterpret_cast<unsigned*>(ub + lay.off_sync) + slot;
-    __threadfence();
-    const unsigned old = atomicAdd(cnt, 1u);
+    // release: this CTA's stores (the barrier put them before this thread) are visible to whoever
+    // sees the count; acquire: the CTA that counts last sees the others' stores
+    unsigned old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(old) : "l"(cnt) : "memory");
     const int last = old == (unsigned)(per_unit - 1);
-    if (last) {
-      *cnt = 0u;          // next used in a later epoch, after this kernel has completed
-      __threadfence();
-    }
+    if (last) *cnt = 0u;  // next used by a later call, after this kernel has completed
     *s_last = last;
   }
   __syncthreads();
