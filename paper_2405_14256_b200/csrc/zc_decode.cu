@@ -1053,6 +1053,12 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
   const bool is_tail = !plan.fold_tail && j == per_unit - 1;
   char* ub = zc_unit_base(cache, lay, unit);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (plan.n_tail > 0 && tid < 2 && plan.fold_tail && j == 0) {
+    // the tail's rows start their way from DRAM to L2 while the CTA sets up (a CTA that has
+    // only the tail to do loads them at once anyway)
+    const char* rows = ub + (tid == 0 ? lay.off_tailK : lay.off_tailV);
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(rows), "r"(plan.n_tail * ZC_D * 2) : "memory");
+  }
   // the stream's word is requested first and looked at when it is needed
   const unsigned ord_first = ord.need_start > 0 ? ld_order_acquire(ord.done) : ord.need_end > 0 ? ld_order(ord.done) : 0u;
   pdl_launch_dependents();
