@@ -110,7 +110,7 @@ class ClockSampler:
 # (dram__bytes_read.sum + dram__bytes_write.sum), keyed by workload id; the captures and their
 # conditions are in profiles/k_decode_config2.md and profiles/k_decode_config4.md (the first
 # decode steps after a prefill, when the tail holds a few tokens).
-PROFILED_DRAM_BYTES_PER_DECODE_CALL = {2: 28.22e6, 4: 449.1e6 + 19.0e6}
+PROFILED_DRAM_BYTES_PER_DECODE_CALL = {2: 28.26e6, 4: 449.6e6 + 19.0e6}
 
 
 def algorithmic_decode_bytes(w, n_windows: int, n_tail: int) -> int:
