@@ -63,6 +63,12 @@ enum {
  * cut into work items: few large ones, which is best when several calls share the GPU and
  * worst for a single call that has the GPU to itself. */
 #define ZC_FLAG_OVERLAP_CALLS 2
+/* With ZC_FLAG_OUT_F32 zc_decode_attention stores its result as fp32 (out [device]
+ * b x h_q x d floats) instead of rounding it to cfg.dtype.  A 16-bit output cannot be closer
+ * to the exact result than half a unit in its last place (bf16: 2e-3 from |o| = 0.25 on), so
+ * this is the form in which the kernel's own arithmetic (Eq. 4 over the dequantised cache)
+ * can be compared with a reference at a tolerance below that. */
+#define ZC_FLAG_OUT_F32 4
 
 /* Plain-data configuration; set struct_size = sizeof(zc_config). */
 typedef struct {
@@ -78,7 +84,7 @@ typedef struct {
                              (Alg. 3 uses 100); 8 <= window <= ZC_MAX_WINDOW */
   int32_t bits_hi;        /* bit-width of salient tokens: 4 or 2 */
   int32_t bits_lo;        /* bit-width of regular tokens: 4 or 2 */
-  int32_t flags;          /* 0 or an OR of ZC_FLAG_DEFER_APPEND, ZC_FLAG_OVERLAP_CALLS */
+  int32_t flags;          /* 0 or an OR of the ZC_FLAG_* values above */
   double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
 } zc_config;
 

@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(HERE, "libzipcache.so")
 ZC_F16, ZC_BF16 = 0, 1
 ZC_FLAG_DEFER_APPEND = 1
 ZC_FLAG_OVERLAP_CALLS = 2
+ZC_FLAG_OUT_F32 = 4
 
 
 class ZipCacheError(RuntimeError):
@@ -243,13 +244,15 @@ class ZipCache:
     def __init__(self, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
                  workspace: Optional[torch.Tensor] = None, defer_append: bool = False,
-                 overlap_calls: bool = False):
+                 overlap_calls: bool = False, out_f32: bool = False):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                                  saliency_ratio, bits_hi, bits_lo, window,
                                  flags=(ZC_FLAG_DEFER_APPEND if defer_append else 0) |
-                                 (ZC_FLAG_OVERLAP_CALLS if overlap_calls else 0))
+                                 (ZC_FLAG_OVERLAP_CALLS if overlap_calls else 0) |
+                                 (ZC_FLAG_OUT_F32 if out_f32 else 0))
+        self.out_dtype = torch.float32 if out_f32 else dtype
         self.dtype, self.device = dtype, torch.device(device)
         self.batch, self.n_q_heads, self.n_kv_heads = batch, n_q_heads, n_kv_heads
         self.cache_bytes, self.workspace_bytes = zc_cache_bytes(self.cfg)
@@ -280,7 +283,7 @@ class ZipCache:
 
     def decode_attention(self, q, is_probe_step=False, out=None, stream=None):
         if out is None:
-            out = torch.empty_like(q)
+            out = torch.empty(q.shape, dtype=self.out_dtype, device=q.device)
         zc_decode_attention(self.handle, q, out, is_probe_step, self.workspace, stream)
         return out
 

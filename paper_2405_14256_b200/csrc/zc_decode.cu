@@ -346,20 +346,28 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
       oacc[j][0] *= c0; oacc[j][1] *= c1; oacc[j][2] *= c0; oacc[j][3] *= c1;
     }
   }
-  // p' = p * 2^logKs; weights w = p' * s^V go to f16, the same rounded values feed the z sum
+  // p' = p * 2^logKs; weights w = p' * s^V go to the tensor cores as hi + lo in f16 (columns
+  // 0..3 and 4..7 of P^T: a single f16 would put a relative error of 2^-11 on every weight,
+  // which a few dominant tokens turn into an output error above 1e-3)
   uint32_t pb[2][2];
+  const bool lo_col = g >= 4;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const float p0 = zc_exp2(fmaf(u[h][0], isc, S.mo_neg)), p1 = zc_exp2(fmaf(u[h][1], isc, S.mo_neg));
     S.l += p0 + p1;
-    const __half2 h2 = __floats2half2_rn(p0 * pp[h][0].z, p1 * pp[h][1].z);   // (token g, token g+8)
+    const float w0 = p0 * pp[h][0].z, w1 = p1 * pp[h][1].z;
+    S.zacc = fmaf(w0, pp[h][0].w, S.zacc);
+    S.zacc = fmaf(w1, pp[h][1].w, S.zacc);
+    const __half2 h2 = __floats2half2_rn(w0, w1);   // (token g, token g+8)
     const float2 back = __half22float2(h2);
-    S.zacc = fmaf(back.x, pp[h][0].w, S.zacc);
-    S.zacc = fmaf(back.y, pp[h][1].w, S.zacc);
-    const uint32_t X = *reinterpret_cast<const uint32_t*>(&h2);
-    // B fragment of P^T, column n = g = head g & 3: (tokens 2t, 2t+8) and (tokens 2t+1, 2t+9)
-    pb[h][0] = __shfl_sync(kFull, X, srcA);
-    pb[h][1] = __shfl_sync(kFull, X, srcB);
+    const __half2 l2 = __floats2half2_rn(w0 - back.x, w1 - back.y);
+    const uint32_t Xh = *reinterpret_cast<const uint32_t*>(&h2);
+    const uint32_t Xl = *reinterpret_cast<const uint32_t*>(&l2);
+    // B fragment of P^T, column n = g: head g & 3, part g >> 2; (tokens 2t, 2t+8) and (2t+1, 2t+9)
+    const uint32_t ah = __shfl_sync(kFull, Xh, srcA), al = __shfl_sync(kFull, Xl, srcA);
+    const uint32_t bh = __shfl_sync(kFull, Xh, srcB), bl = __shfl_sync(kFull, Xl, srcB);
+    pb[h][0] = lo_col ? al : ah;
+    pb[h][1] = lo_col ? bl : bh;
   }
   // ---- O^T += V^T(128 channels x 16 tokens) . P^T per half: 8 M-tiles ----
 #pragma unroll
@@ -400,7 +408,7 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
   const int g = lane >> 2, t = lane & 3;
   const bool odd_tok = BITS == 2 && (g & 1);
   const float logKs = logK - (odd_tok ? 2.f : 0.f);      // weights of odd tokens carry 1/4 at 2 bits
-  // columns 4..7 of P^T repeat columns 0..3: their products land in accumulator columns no one reads
+  // columns 4..7 of P^T carry the lo parts of the weights of heads 0..3
   const int srcA = 8 * t + (g & 3), srcB = srcA + 4;
   const int c0_src = (lane & ~3) | ((2 * t) & 3), c1_src = (lane & ~3) | ((2 * t + 1) & 3);
   // Logits are kept divided by isc (u = lg / isc): u costs one multiply less per token.
@@ -558,6 +566,11 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
     z += __shfl_xor_sync(kFull, z, o);
   }
   if (g == 0) { wm[warp * 4 + t] = m; wl[warp * 4 + t] = l; wz[warp * 4 + t] = z; }
+  // columns 4..7 (lanes t >= 2) hold the products of the weights' lo parts for heads 0..3
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) oacc[j][e] += __shfl_xor_sync(kFull, oacc[j][e], 2);
   // the warp's own ring is free (all of its copies were consumed): accumulators go there
   float* mbuf = reinterpret_cast<float*>(my_ring);   // [4 heads][128]
   __syncwarp();
@@ -734,9 +747,9 @@ static_assert(kCombineSmem <= decode_smem(kRingNarrow), "the merge phase must fi
 template <typename T>
 __device__ __noinline__ void tail_phase(const T* tK, const T* tV, int G, int n_tail, const T* qunit, int unit,
                                         float* part_unit, int first_entry, float* stash_g, const T* k_new,
-                                        const T* v_new, ZcOrder ord, unsigned ord_first, int* err) {
+                                        const T* v_new, ZcOrder ord, unsigned ord_first, bool free_run, int* err) {
   const int warp = threadIdx.x >> 5;
-  order_wait(ord, ord_first, ord.need_end, err);   // the workspace region is free
+  if (free_run) order_wait(ord, ord_first, ord.need_end, err);   // the workspace region is free
   for (int base = warp * ZC_SUB; base < n_tail; base += kWarps * ZC_SUB) {
     float* entry = part_unit + (long long)(first_entry + base / ZC_SUB) * G * ZC_PART_STRIDE;
     for (int hg = 0; hg * 4 < G; ++hg)
@@ -934,7 +947,8 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
 
 template <typename T>
 __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_tail, T* __restrict__ out_unit,
-                                        const float* mine, const float* stash_g, int collect, char* smem) {
+                                        float* __restrict__ out_unit_f32, const float* mine,
+                                        const float* stash_g, int collect, char* smem) {
   float* s_m = reinterpret_cast<float*>(smem + kCmbOffM);
   float* s_l = reinterpret_cast<float*>(smem + kCmbOffL);
   float* s_ML = reinterpret_cast<float*>(smem + kCmbOffML);
@@ -992,9 +1006,14 @@ __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_t
       o4.x += a.x * sc; o4.y += a.y * sc; o4.z += a.z * sc; o4.w += a.w * sc;
     }
     const float inv = 1.f / lsum;
-    T r[4] = {zc_from_float<T>(o4.x * inv), zc_from_float<T>(o4.y * inv), zc_from_float<T>(o4.z * inv),
-              zc_from_float<T>(o4.w * inv)};
-    *reinterpret_cast<uint2*>(out_unit + h * ZC_D + 4 * lane) = *reinterpret_cast<const uint2*>(r);
+    if (out_unit_f32) {   // ZC_FLAG_OUT_F32: the result before its rounding to the 16-bit type
+      *reinterpret_cast<float4*>(out_unit_f32 + h * ZC_D + 4 * lane) =
+          make_float4(o4.x * inv, o4.y * inv, o4.z * inv, o4.w * inv);
+    } else {
+      T r[4] = {zc_from_float<T>(o4.x * inv), zc_from_float<T>(o4.y * inv), zc_from_float<T>(o4.z * inv),
+                zc_from_float<T>(o4.w * inv)};
+      *reinterpret_cast<uint2*>(out_unit + h * ZC_D + 4 * lane) = *reinterpret_cast<const uint2*>(r);
+    }
   }
   if (collect) {
     __syncthreads();
@@ -1060,10 +1079,22 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(rows), "r"(plan.n_tail * ZC_D * 2) : "memory");
   }
   // the stream's word is requested first and looked at when it is needed
-  const unsigned ord_first = ord.need_start > 0 ? ld_order_acquire(ord.done) : ord.need_end > 0 ? ld_order(ord.done) : 0u;
+  const bool free_run = plan.chain_free != 0;
+  const unsigned ord_first =
+      !free_run ? 0u : ord.need_start > 0 ? ld_order_acquire(ord.done) : ord.need_end > 0 ? ld_order(ord.done) : 0u;
   pdl_launch_dependents();
-  // inputs written by an earlier call, a re-compressed window, the previous call's tail row
-  order_wait(ord, ord_first, ord.need_start, &g_zc_error);
+  if (free_run) {
+    // The caller promised (ZC_FLAG_OVERLAP_CALLS) that only calls of this library precede this
+    // one on the stream: the working CTAs do not wait for the previous kernel, only for what
+    // the host found them to depend on (inputs written by an earlier call, a re-compressed
+    // window, the previous call's tail row).
+    order_wait(ord, ord_first, ord.need_start, &g_zc_error);
+  } else {
+    // Anything may precede this call on the stream, e.g. the kernel that produces q, and it
+    // may have let this kernel start early: everything the stream holds before this launch
+    // must have completed before q, k_new, v_new or the cache are read.
+    pdl_wait();
+  }
   if (k_new && j == 0 && warp == kWarps - 1) {
     // Deferred append: the newest row goes into the tail for the steps to come (this step reads
     // it from k_new / v_new).  The next call on this cache is told to wait for this one.
@@ -1086,9 +1117,10 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     // The tail is the work of a CTA of its own, or (calls that share the GPU with their
     // neighbours) of the unit's first item CTA before it turns to its codes.
     // without a deferred append the newest tail row comes from the append kernel just before
-    if (!k_new) pdl_wait();
+    if (!k_new && free_run) pdl_wait();
     tail_phase<T>(reinterpret_cast<const T*>(ub + lay.off_tailK), reinterpret_cast<const T*>(ub + lay.off_tailV), G,
-                  plan.n_tail, qunit, unit, mine, plan.items, stash_g, k_new, v_new, ord, ord_first, &g_zc_error);
+                  plan.n_tail, qunit, unit, mine, plan.items, stash_g, k_new, v_new, ord, ord_first, free_run,
+                  &g_zc_error);
   }
   if (!is_tail) {
     float* wm = reinterpret_cast<float*>(smem + kOffWm);
@@ -1135,7 +1167,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
       s_head[tid * 4 + 2] = has ? zsum : 0.f;
     }
     __syncthreads();
-    order_wait(ord, ord_first, ord.need_end, &g_zc_error);   // the workspace region is free
+    if (free_run) order_wait(ord, ord_first, ord.need_end, &g_zc_error);   // the workspace region is free
     for (int h = 0; h < Gl; ++h) {
       float o = 0.f;
       if (has) {
@@ -1172,8 +1204,9 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
   }
   __syncthreads();
   if (*s_last) {
-    merge_unit<T>(reinterpret_cast<float*>(ub + lay.off_colsum), G, plan.items, plan.n_tail,
-                out + ((long long)b * lay.n_kv * G + kv * G) * ZC_D, mine, stash_g, collect, smem);
+    const long long out_off = ((long long)b * lay.n_kv * G + kv * G) * ZC_D;
+    merge_unit<T>(reinterpret_cast<float*>(ub + lay.off_colsum), G, plan.items, plan.n_tail, out + out_off,
+                  lay.out_f32 ? reinterpret_cast<float*>(out) + out_off : nullptr, mine, stash_g, collect, smem);
     if (fl.on) {
       __syncthreads();   // the merge is done with the shared arrays; its additions to the statistics are visible
       window_flush_unit<T>(ub, lay, fl, smem);
@@ -1284,7 +1317,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   call.me.in[0] = zc_range(q, io_bytes);
   call.me.in[1] = zc_range(k_new, kv_bytes);
   call.me.in[2] = zc_range(v_new, kv_bytes);
-  call.me.out = zc_range(out, io_bytes);
+  call.me.out = zc_range(out, c->lay.out_f32 ? 2 * io_bytes : io_bytes);
   call.cache = c;
   call.collect = collect;
   call.changes_cache = k_new != nullptr || fl.on;

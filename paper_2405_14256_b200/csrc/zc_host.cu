@@ -27,7 +27,7 @@ int check_config(const zc_config* cfg) {
   if (cfg->window < 8 || cfg->window > ZC_MAX_WINDOW) return ZC_EINVAL;
   if (cfg->bits_hi != 4 && cfg->bits_hi != 2) return ZC_EINVAL;
   if (cfg->bits_lo != 4 && cfg->bits_lo != 2) return ZC_EINVAL;
-  if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS)) return ZC_EINVAL;
+  if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32)) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if ((long long)cfg->batch * cfg->n_kv_heads > 65535) return ZC_EINVAL;
   // every re-compressed window adds two items to a decode call
@@ -42,6 +42,7 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   lay->n_kv = cfg->n_kv_heads;
   lay->window = cfg->window;
   lay->dtype = cfg->dtype;
+  lay->out_f32 = (cfg->flags & ZC_FLAG_OUT_F32) ? 1 : 0;
   lay->bits[0] = cfg->bits_hi;
   lay->bits[1] = cfg->bits_lo;
   const int max_flush = cfg->max_new_tokens / cfg->window;
@@ -213,6 +214,7 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
     // they get and the build with more resident warps is used.
     p.ctas_per_sm = 4;
     p.fold_tail = 1;
+    p.chain_free = 1;
     for (int k = 0; k < 2; ++k) {
       const int want = std::min(std::min(zc_ceil_div(subs[k], kCand[0]), std::min(ZC_MAX_SPLIT_HOST, cap)), subs[k]);
       p.spi0[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;

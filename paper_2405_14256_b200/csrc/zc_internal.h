@@ -42,6 +42,7 @@
 //   [params 16 x (K scale, K zero, V scale, V zero) f32]
 struct ZcLayout {
   int units, G, n_kv, window, dtype;
+  int out_f32;            // decode outputs are stored as fp32 (ZC_FLAG_OUT_F32)
   int bits[2];
   int tile_bytes[2];
   int cap_tiles[2];
@@ -87,6 +88,7 @@ struct ZcDecodePlan {
   int items;               // items per unit
   int cta_items;           // consecutive items one CTA works through
   int fold_tail;           // the tail is attended by the unit's first item CTA, not by a CTA of its own
+  int chain_free;          // ZC_FLAG_OVERLAP_CALLS: working CTAs do not wait for the previous kernel
   int l0;
 };
 

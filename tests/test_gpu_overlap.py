@@ -34,11 +34,12 @@ def _prefilled(w, layers, shared_ws=True, **kw):
 
 
 def _check(w, got, ref_units):
+    """Worst excess over the bound of the edge-size tests (see zc_testlib.output_excess)."""
     G = w.group
-    worst = 0.0
+    worst = -1.0
     g = tl.to64(got)
     for (bi, kv), o in ref_units.items():
-        worst = max(worst, tl.output_error(g[bi, kv * G:(kv + 1) * G], o, w.torch_dtype))
+        worst = max(worst, tl.output_excess(g[bi, kv * G:(kv + 1) * G], o, w.torch_dtype))
     return worst
 
 
@@ -66,14 +67,14 @@ def test_calls_in_flight_together_match_the_oracle(layers, steps, kw, overlap_it
             c.decode_attention(q, bool(flags[ly][s]), out=outs[s][ly])
     torch.cuda.synchronize()
     assert zc.zc_device_status() == 0
-    worst = 0.0
+    worst = -1.0
     for s in range(steps):
         for ly, oc in enumerate(oracles):
             q, k, v = ins[s][ly]
             oc.append(tl.to64(k), tl.to64(v))
             ref = oc.decode_attention(tl.to64(q), bool(flags[ly][s]))
             worst = max(worst, _check(w, outs[s][ly], ref))
-    assert worst <= 2e-3, worst
+    assert worst <= 0.0, worst
     # the re-compressed windows depend on the statistics every probe step added, in order
     for ly, (c, oc) in enumerate(zip(caches, oracles)):
         n_seg = zc.zc_num_segments(c.handle)
@@ -98,12 +99,12 @@ def test_a_call_that_reads_the_previous_output_waits_for_it():
         c.decode_attention(bufs[s], False, out=bufs[s + 1])
     torch.cuda.synchronize()
     assert zc.zc_device_status() == 0
-    worst = 0.0
+    worst = -1.0
     for s in range(steps):
         oc.append(tl.to64(kv[s][1]), tl.to64(kv[s][2]))
         ref = oc.decode_attention(tl.to64(bufs[s]), False)
         worst = max(worst, _check(w, bufs[s + 1], ref))
-    assert worst <= 2e-3, worst
+    assert worst <= 0.0, worst
 
 
 def test_calls_that_write_the_same_output_land_in_order():
@@ -130,7 +131,7 @@ def test_calls_that_write_the_same_output_land_in_order():
             q, k, v = ins[s][ly]
             oc.append(tl.to64(k), tl.to64(v))
             ref = oc.decode_attention(tl.to64(q), False)
-    assert _check(w, out, ref) <= 2e-3
+    assert _check(w, out, ref) <= 0.0
 
 
 @pytest.mark.parametrize("window", [100, 16])   # 16: a window is re-compressed inside the graph
@@ -182,3 +183,44 @@ def test_captured_calls_replay_to_the_same_results(window):
     for a, b in zip(outs_all[0], outs_all[1]):
         for x, y in zip(a, b):
             assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("promise", [False])
+def test_a_producer_that_lets_us_start_early_is_waited_for(promise):
+    """q of the second call is written, between the two calls, by a kernel of "another library"
+    that triggers programmatic launch completion at its very start and stores q 100 us later
+    (tests/helpers/zc_test_kernels.cu).  Without ZC_FLAG_OVERLAP_CALLS the decode kernel must
+    not read q before that kernel has completed."""
+    import ctypes as C
+    import os
+    import sys
+    sys.path.insert(0, os.path.join(os.path.dirname(os.path.abspath(__file__)), "helpers"))
+    import build_helpers
+    helper = C.CDLL(build_helpers.build())
+    helper.zct_late_copy.restype = C.c_int
+    helper.zct_late_copy.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_longlong, C.c_void_p]
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(context=400, batch=2, n_q_heads=8, n_kv_heads=2)
+    for defer in (False, True):
+        (c,), (oc,) = _prefilled(w, 1, defer_append=defer, overlap_calls=promise)
+        q0, k0, v0 = make_decode_step(w, 0, 0, tl.DEV)
+        q1, k1, v1 = make_decode_step(w, 0, 1, tl.DEV)
+        q_buf = torch.zeros_like(q1)             # stale contents: zeros
+        k_buf, v_buf = torch.zeros_like(k1), torch.zeros_like(v1)
+        st = torch.cuda.current_stream().cuda_stream
+        torch.cuda.synchronize()
+        c.append(k0, v0)
+        o0 = c.decode_attention(q0, False)
+        for dst, src in ((q_buf, q1), (k_buf, k1), (v_buf, v1)):
+            rc = helper.zct_late_copy(dst.data_ptr(), src.data_ptr(), dst.numel() * dst.element_size(),
+                                      200000, st)
+            assert rc == 0
+        c.append(k_buf, v_buf)
+        o1 = c.decode_attention(q_buf, True)
+        torch.cuda.synchronize()
+        assert zc.zc_device_status() == 0
+        assert torch.equal(q_buf, q1)
+        for (q, k, v, o, fl) in ((q0, k0, v0, o0, False), (q1, k1, v1, o1, True)):
+            oc.append(tl.to64(k), tl.to64(v))
+            ref = oc.decode_attention(tl.to64(q), fl)
+            assert _check(w, o, ref) <= 0.0
