@@ -19,6 +19,9 @@ Passages followed (paper section / equation / algorithm):
   uniform quantisation ....... Eq. 5 (dequantisation subtracts the zero point)
   channel normalisation ...... Eq. 6
   CSTQuant ................... Alg. 1
+  ChannelQuant (keys) ........ Sec. 4.1 last paragraph, Table 1 last row, Alg. 2
+  16-bit quantisation params . Appendix A (parameters counted at 16 bits)
+  token-level saliency ....... Sec. 4.2 / Alg. 2 read literally: one score per token
   decode concat / attention .. Eq. 3, Eq. 4, Alg. 3
   streaming re-compression ... Alg. 3 (every `window` = 100 generated tokens)
   overhead accounting ........ Appendix A, Eq. (A)-(C)
@@ -35,6 +38,9 @@ ratios.  Conventions that no printed value or closed form fixes are marked
   * integer zero point (vs. a float offset)         -- parity unpinned
   * streaming-flush semantics (which 100 tokens, the 100th step being a probe
     step)                                           -- parity unpinned
+  * rounding of 16-bit scales (up, so that the half-step bound survives) and the
+    scope of channelwise parameters (per batch, KV head and subset) -- parity unpinned
+  * token-level saliency as the mean of the per-KV-head scores     -- parity unpinned
 """
 from __future__ import annotations
 
@@ -197,6 +203,81 @@ def token_quant_reference_fp64(Y: np.ndarray, bits: int) -> np.ndarray:
     return Y / s[:, None] + z[:, None]
 
 
+# --------------------------------------------------------------------------
+# ChannelQuant (Sec. 4.1: channelwise quantisation, the paper's choice for keys)
+# --------------------------------------------------------------------------
+def channel_quant(X: np.ndarray, bits: int) -> Dict[str, np.ndarray]:
+    """Channelwise uniform quantisation of X [n_tokens, d] to `bits`: Eq. 5 with the minimum
+    and maximum taken over the tokens of one channel, so that there is one (s, z) pair per
+    channel (2 h d parameters per tensor, Table 1) and none per token.
+
+    Normative fp32 sequence, one IEEE operation per step, round to nearest even:
+    mn_i, mx_i over the tokens; s_i = (mx_i - mn_i) / L, or |mn_i| (1 if 0) for a constant
+    channel; z_i = -rint(mn_i / s_i); code = clamp(rint(x / s_i) + z_i, 0, L)."""
+    f32 = np.float32
+    X = np.asarray(X, dtype=f32)
+    n, d = X.shape
+    L = f32((1 << bits) - 1)
+    mn = X.min(axis=0) if n > 0 else np.zeros(d, dtype=f32)
+    mx = X.max(axis=0) if n > 0 else np.zeros(d, dtype=f32)
+    s = ((mx - mn).astype(f32) / L).astype(f32)
+    flat = mx == mn
+    s = np.where(flat, np.where(mn != f32(0), np.abs(mn), f32(1)), s).astype(f32)
+    z = (-np.rint((mn / s).astype(f32))).astype(f32)
+    pre = (X / s[None, :]).astype(f32)
+    q = (np.rint(pre).astype(f32) + z[None, :]).astype(f32)
+    codes = np.minimum(np.maximum(q, f32(0)), L).astype(np.uint8)
+    return {"s": s, "z": z, "codes": codes, "bits": bits, "pre_round": pre, "scheme": "channel"}
+
+
+def channel_dequant(qd: Dict[str, np.ndarray]) -> np.ndarray:
+    """x_hat = (code - z_i) * s_i in fp64 (Eq. 5 with the zero point subtracted)."""
+    s = qd["s"].astype(np.float64)
+    z = qd["z"].astype(np.float64)
+    return (qd["codes"].astype(np.float64) - z[None, :]) * s[None, :]
+
+
+# --------------------------------------------------------------------------
+# 16-bit quantisation parameters (Appendix A counts every parameter at 16 bits)
+# --------------------------------------------------------------------------
+def round_up_to_f16(x: np.ndarray) -> np.ndarray:
+    """Smallest fp16 value >= x, element by element (x >= 0, within fp16 range)."""
+    x = np.asarray(x, dtype=np.float32)
+    h = x.astype(np.float16)
+    low = h.astype(np.float32) < x
+    return np.where(low, np.nextafter(h, np.float16(np.inf)), h).astype(np.float16)
+
+
+def cst_quant_f16_params(X: np.ndarray, bits: int) -> Dict[str, np.ndarray]:
+    """CSTQuant whose stored parameters fit 16 bits each: the channel factors c and the token
+    scales s are fp16 values, the zero points z small integers.
+
+    The scale is rounded UP to fp16 before the codes are formed, so the codes of a token span
+    at most the same range as with the fp32 scale and the error bound |y - (code - z) s| <= s/2
+    holds for the stored scale (rounding to nearest could shrink s and push the token's
+    maximum beyond the top code).  Everything else follows cst_quant."""
+    f32 = np.float32
+    X = np.asarray(X, dtype=f32)
+    n, d = X.shape
+    L = f32((1 << bits) - 1)
+    m = np.abs(X).max(axis=0) if n > 0 else np.zeros(d, dtype=f32)
+    c = np.sqrt(m, dtype=f32)
+    c = np.where(m == f32(0), f32(1), c).astype(f32)
+    c = round_up_to_f16(c).astype(f32)                    # stored factor: fp16
+    Y = (X / c[None, :]).astype(f32)
+    mn = Y.min(axis=1) if n > 0 else np.zeros(0, dtype=f32)
+    mx = Y.max(axis=1) if n > 0 else np.zeros(0, dtype=f32)
+    s = ((mx - mn).astype(f32) / L).astype(f32)
+    flat = mx == mn
+    s = np.where(flat, np.where(mn != f32(0), np.abs(mn), f32(1)), s).astype(f32)
+    s = round_up_to_f16(s).astype(f32)                    # stored scale: fp16, never below the exact one
+    z = (-np.rint((mn / s).astype(f32))).astype(f32)
+    pre = (Y / s[:, None]).astype(f32)
+    q = (np.rint(pre).astype(f32) + z[:, None]).astype(f32)
+    codes = np.minimum(np.maximum(q, f32(0)), L).astype(np.uint8)
+    return {"c": c, "s": s, "z": z, "codes": codes, "bits": bits, "pre_round": pre}
+
+
 def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
     """Canonical packing of codes [n,d] -> bytes [n, d*bits/8]: 4-bit element
     2m in the low nibble and 2m+1 in the high nibble of byte m; 2-bit element
@@ -253,13 +334,48 @@ def compression_ratio(k_granularity: str, v_granularity: str, b: int, hd: int, l
     return full / (data + params * param_bits)
 
 
+def mixed_precision_ratio(b: int, hd: int, l: int, ratio_salient: float, bits_hi: int, bits_lo: int,
+                          k_granularity: str = "channel", v_granularity: str = "cst",
+                          param_bits: int = 16, n: int = 32) -> float:
+    """Compression ratio of a cache whose salient share is kept at bits_hi and the rest at
+    bits_lo, each subset quantised on its own (Alg. 2), in the counting of Appendix A: per-channel
+    parameters once per subset (no batch factor), per-token parameters once per token."""
+    full = 2 * b * hd * l * 16
+    l_hi = ratio_salient * l
+    data = 2 * b * hd * (l_hi * bits_hi + (l - l_hi) * bits_lo)
+    params = 0.0
+    for gran in (k_granularity, v_granularity):
+        for l_sub in (l_hi, l - l_hi):
+            if l_sub > 0:               # an empty subset stores nothing
+                params += quant_param_count(gran, b, hd, l_sub, n)
+    return full / (data + params * param_bits)
+
+
+def cache_footprint_bytes(b: int, h_kv: int, d: int, n_hi: int, n_lo: int, bits_hi: int, bits_lo: int,
+                          k_scheme: str = "cst", param_bytes: int = 4) -> int:
+    """Bytes of the compressed cache in the granularity this repository stores it in: per
+    (batch, KV head) unit and subset, codes of K and V, one (s, z) pair per token for every
+    tensor quantised tokenwise, per-channel parameters for every (unit, subset, tensor):
+    c for CSTQuant, (s, z) for ChannelQuant."""
+    total = 0
+    for n_tok, bits in ((n_hi, bits_hi), (n_lo, bits_lo)):
+        if n_tok == 0:
+            continue
+        codes = 2 * n_tok * d * bits // 8
+        token_params = n_tok * 2 * param_bytes * (1 if k_scheme == "channel" else 2)
+        channel_params = d * param_bytes * (3 if k_scheme == "channel" else 2)
+        total += codes + token_params + channel_params
+    return total * b * h_kv
+
+
 # --------------------------------------------------------------------------
 # One (batch, KV head) unit of the mixed-precision cache (Alg. 2, Alg. 3)
 # --------------------------------------------------------------------------
 class _Subset:
     """Tokens of one precision class inside one segment."""
 
-    def __init__(self, idx: np.ndarray, K: np.ndarray, V: np.ndarray, bits: int):
+    def __init__(self, idx: np.ndarray, K: np.ndarray, V: np.ndarray, bits: int,
+                 k_scheme: str = "cst", param_dtype: str = "f32"):
         self.idx = idx.astype(np.int32)
         self.bits = bits
         self.n = len(idx)
@@ -267,31 +383,41 @@ class _Subset:
             self.qK = self.qV = None
             self.K_hat = np.asarray(K, dtype=np.float64)[idx]
             self.V_hat = np.asarray(V, dtype=np.float64)[idx]
+            return
+        cst = cst_quant_f16_params if param_dtype == "f16" else cst_quant
+        self.qV = cst(np.asarray(V, dtype=np.float32)[idx], bits)
+        self.V_hat = cst_dequant(self.qV)
+        if k_scheme == "channel":     # Alg. 2: ChannelQuant for keys, CSTQuant for values
+            self.qK = channel_quant(np.asarray(K, dtype=np.float32)[idx], bits)
+            self.K_hat = channel_dequant(self.qK)
         else:
-            self.qK = cst_quant(np.asarray(K, dtype=np.float32)[idx], bits)
-            self.qV = cst_quant(np.asarray(V, dtype=np.float32)[idx], bits)
+            self.qK = cst(np.asarray(K, dtype=np.float32)[idx], bits)
             self.K_hat = cst_dequant(self.qK)
-            self.V_hat = cst_dequant(self.qV)
 
 
 class _Segment:
-    def __init__(self, K, V, p_tilde, ratio, bits_hi, bits_lo):
+    def __init__(self, K, V, p_tilde, ratio, bits_hi, bits_lo, k_scheme="cst", param_dtype="f32"):
         n = K.shape[0]
         self.n = n
         self.p_tilde = np.asarray(p_tilde, dtype=np.float64)
+        self.k_scheme, self.param_dtype = k_scheme, param_dtype
         n_s = salient_count(ratio, n)
         sal, reg = split_salient(self.p_tilde, n_s)
-        self.hi = _Subset(sal, K, V, bits_hi)
-        self.lo = _Subset(reg, K, V, bits_lo)
+        self.impose(K, V, sal, reg, bits_hi, bits_lo)
+
+    def impose(self, K, V, sal, reg, bits_hi, bits_lo):
+        self.hi = _Subset(sal, K, V, bits_hi, self.k_scheme, self.param_dtype)
+        self.lo = _Subset(reg, K, V, bits_lo, self.k_scheme, self.param_dtype)
 
 
 class UnitCache:
     """Mixed-precision cache of one (batch, KV head) with its G query heads."""
 
     def __init__(self, G: int, d: int, ratio: float, bits_hi: int = 4, bits_lo: int = 2,
-                 window: int = 100):
+                 window: int = 100, k_scheme: str = "cst", param_dtype: str = "f32"):
         self.G, self.d, self.ratio = G, d, ratio
         self.bits_hi, self.bits_lo, self.window = bits_hi, bits_lo, window
+        self.k_scheme, self.param_dtype = k_scheme, param_dtype
         self.segments: List[_Segment] = []
         self.tail_K = np.zeros((0, d), dtype=np.float64)
         self.tail_V = np.zeros((0, d), dtype=np.float64)
@@ -302,16 +428,19 @@ class UnitCache:
 
     # ---- Alg. 2 (without its FlashAttention output line) ----
     def prefill_compress(self, Q_heads: np.ndarray, K: np.ndarray, V: np.ndarray,
-                         P: Sequence[int], salient_idx: Optional[np.ndarray] = None) -> None:
+                         P: Sequence[int], salient_idx: Optional[np.ndarray] = None,
+                         p_tilde: Optional[np.ndarray] = None) -> None:
+        """p_tilde given: the saliency was decided outside the unit (token-level scope)."""
         K = np.asarray(K, dtype=np.float64)
         V = np.asarray(V, dtype=np.float64)
-        p_tilde = normalized_scores(Q_heads, K, P)
-        seg = _Segment(K, V, p_tilde, self.ratio, self.bits_hi, self.bits_lo)
+        if p_tilde is None:
+            p_tilde = normalized_scores(Q_heads, K, P)
+        seg = _Segment(K, V, p_tilde, self.ratio, self.bits_hi, self.bits_lo, self.k_scheme,
+                       self.param_dtype)
         if salient_idx is not None:  # staged tests: impose a given split
             sal = np.sort(np.asarray(salient_idx, dtype=np.int32))
             reg = np.setdiff1d(np.arange(K.shape[0], dtype=np.int32), sal)
-            seg.hi = _Subset(sal, K, V, self.bits_hi)
-            seg.lo = _Subset(reg, K, V, self.bits_lo)
+            seg.impose(K, V, sal, reg, self.bits_hi, self.bits_lo)
         self.segments = [seg]
         self.tail_K = np.zeros((0, self.d), dtype=np.float64)
         self.tail_V = np.zeros((0, self.d), dtype=np.float64)
@@ -332,7 +461,10 @@ class UnitCache:
         return np.vstack(Ks + [self.tail_K]), np.vstack(Vs + [self.tail_V])
 
     # ---- Eq. 4 / Alg. 3: attention over every cached token, then bookkeeping ----
-    def decode_attention(self, q_heads: np.ndarray, is_probe_step: bool) -> np.ndarray:
+    def decode_attention(self, q_heads: np.ndarray, is_probe_step: bool,
+                         defer_flush: bool = False) -> np.ndarray:
+        """defer_flush: the caller re-compresses the completed window itself (token-level scope:
+        the window's scores are first combined over the heads of the batch row)."""
         q = np.asarray(q_heads, dtype=np.float64)             # [G,d]
         K_all, V_all = self._all_kv()
         logits = (q @ K_all.T) / math.sqrt(self.d)             # [G,n]
@@ -349,16 +481,21 @@ class UnitCache:
             if n_tail > 0:
                 self.tail_colsum[:n_tail] += a[:, a.shape[1] - n_tail:].sum(axis=0)
                 self.tail_nnz[:n_tail] += 1
-        if self.i == self.window:
+        if self.i == self.window and not defer_flush:
             self._flush()
         return o
 
-    def _flush(self) -> None:
+    def window_scores(self) -> np.ndarray:
+        n = self.tail_K.shape[0]
+        return self.tail_colsum[:n] / (self.G * self.tail_nnz[:n])
+
+    def _flush(self, p_tilde: Optional[np.ndarray] = None) -> None:
         n = self.tail_K.shape[0]
         assert n == self.window
-        p_tilde = self.tail_colsum[:n] / (self.G * self.tail_nnz[:n])
+        if p_tilde is None:
+            p_tilde = self.window_scores()
         self.segments.append(_Segment(self.tail_K, self.tail_V, p_tilde, self.ratio,
-                                      self.bits_hi, self.bits_lo))
+                                      self.bits_hi, self.bits_lo, self.k_scheme, self.param_dtype))
         self.tail_K = np.zeros((0, self.d), dtype=np.float64)
         self.tail_V = np.zeros((0, self.d), dtype=np.float64)
         self.i = 0
@@ -385,20 +522,35 @@ class ZipCacheOracle:
 
     def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, ratio: float,
                  bits_hi: int = 4, bits_lo: int = 2, window: int = 100,
-                 units: Optional[Sequence[Tuple[int, int]]] = None):
+                 units: Optional[Sequence[Tuple[int, int]]] = None, k_scheme: str = "cst",
+                 param_dtype: str = "f32", scope: str = "kv_head"):
+        """scope "kv_head": one saliency decision per (batch, KV head).  scope "token": the
+        paper's literal reading, one decision per token of a batch row shared by all heads --
+        the score of a token is the mean of its per-KV-head normalised scores (all units of the
+        batch row are then needed).  parity unpinned (how heads are combined is a convention)."""
         self.b, self.hq, self.hkv, self.d = batch, n_q_heads, n_kv_heads, head_dim
         self.G = n_q_heads // n_kv_heads
+        self.scope = scope
         self.unit_ids = list(units) if units is not None else [
             (bi, kv) for bi in range(batch) for kv in range(n_kv_heads)]
-        self.units = {u: UnitCache(self.G, head_dim, ratio, bits_hi, bits_lo, window)
+        self.units = {u: UnitCache(self.G, head_dim, ratio, bits_hi, bits_lo, window, k_scheme,
+                                   param_dtype)
                       for u in self.unit_ids}
 
     def prefill_compress(self, Q, K, V, P, salient_idx=None) -> None:
         """Q [b,h_q,l,d], K,V [b,h_kv,l,d] (float arrays); P ascending probe list."""
+        shared = {}
+        if self.scope == "token":
+            for bi in sorted({u[0] for u in self.unit_ids}):
+                per_head = [normalized_scores(Q[bi, kv * self.G:(kv + 1) * self.G],
+                                              np.asarray(K[bi, kv], dtype=np.float64), P)
+                            for kv in range(self.hkv)]
+                shared[bi] = sum(per_head) / self.hkv
         for (bi, kv) in self.unit_ids:
             sal = None if salient_idx is None else salient_idx[bi][kv]
             self.units[(bi, kv)].prefill_compress(
-                Q[bi, kv * self.G:(kv + 1) * self.G], K[bi, kv], V[bi, kv], P, sal)
+                Q[bi, kv * self.G:(kv + 1) * self.G], K[bi, kv], V[bi, kv], P, sal,
+                p_tilde=shared.get(bi))
 
     def append(self, k, v) -> None:
         for (bi, kv) in self.unit_ids:
@@ -406,7 +558,15 @@ class ZipCacheOracle:
 
     def decode_attention(self, q, is_probe_step: bool) -> Dict[Tuple[int, int], np.ndarray]:
         out = {}
+        token_scope = self.scope == "token"
         for (bi, kv) in self.unit_ids:
             out[(bi, kv)] = self.units[(bi, kv)].decode_attention(
-                q[bi, kv * self.G:(kv + 1) * self.G], is_probe_step)
+                q[bi, kv * self.G:(kv + 1) * self.G], is_probe_step, defer_flush=token_scope)
+        if token_scope:
+            for bi in sorted({u[0] for u in self.unit_ids}):
+                row = [self.units[(bi, kv)] for kv in range(self.hkv)]
+                if row[0].i == row[0].window:
+                    shared = sum(u.window_scores() for u in row) / self.hkv
+                    for u in row:
+                        u._flush(shared)
         return out

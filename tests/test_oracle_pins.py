@@ -479,3 +479,197 @@ def test_multi_unit_wrapper_keeps_units_independent():
     single.prefill_compress(Q[1, 0:2], K[1, 0], V[1, 0], P)
     np.testing.assert_array_equal(single.segments[0].p_tilde,
                                   full.units[(1, 0)].segments[0].p_tilde)
+
+
+# ---------------------------------------------------------------- ChannelQuant (keys)
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("n,d", [(1, 8), (7, 16), (64, 128), (201, 128)])
+def test_channel_quant_half_step_bound_per_channel(bits, n, d):
+    """Eq. 5 per channel: every element within half a step of its channel's grid, the channel's
+    smallest token at code 0 and its largest at the top code, codes monotone along a channel."""
+    X = _outlier_matrix(n, d, 91 + bits + n)
+    X[:, 0] += 40.0                                  # an all-positive channel: negative zero point
+    q = zo.channel_quant(X, bits)
+    L = (1 << bits) - 1
+    s, z, codes = (q[k].astype(np.float64) for k in ("s", "z", "codes"))
+    assert s.shape == (d,) and z.shape == (d,) and codes.shape == (n, d)
+    assert codes.min() >= 0 and codes.max() <= L and np.all(z == np.rint(z))
+    recon = zo.channel_dequant(q)
+    # slack: the fp32 quotient x / s carries an error of |x / s| 2^-24 steps
+    slack = 1e-5 + np.abs(X / s[None, :]).max() * 2.0 ** -22
+    assert np.all(np.abs(X - recon) <= s[None, :] * (0.5 + slack))
+    for i in range(d):
+        if X[:, i].max() > X[:, i].min():
+            assert codes[X[:, i].argmin(), i] == 0 and codes[X[:, i].argmax(), i] == L
+            order = np.argsort(X[:, i], kind="stable")
+            assert np.all(np.diff(codes[order, i]) >= 0)
+    if n > 1:
+        assert z[0] < 0                              # the shifted channel lies above zero
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_channel_quant_is_the_library_per_column_affine_quantiser(bits):
+    """torch's per-channel fake quantiser along the CHANNEL axis is the library statement of
+    channelwise Eq. 5; parameters are Eq. 5's own formulas evaluated per column."""
+    rs = _rng(77)
+    n, d = 53, 24
+    X = (rs.standard_normal((n, d)) * rs.uniform(0.2, 12.0, size=d)[None, :]).astype(np.float32)
+    q = zo.channel_quant(X, bits)
+    L = (1 << bits) - 1
+    got = torch.fake_quantize_per_channel_affine(
+        torch.tensor(X), torch.tensor(q["s"]), torch.tensor(q["z"]).to(torch.int32), 1, 0, L).numpy()
+    np.testing.assert_allclose(zo.channel_dequant(q), got.astype(np.float64), rtol=0, atol=1e-5)
+    for i in range(d):
+        assert abs(q["s"][i] - (X[:, i].max() - X[:, i].min()) / L) <= 1e-6 * q["s"][i] + 1e-9
+        assert q["z"][i] == -round(float(np.float32(X[:, i].min()) / q["s"][i]))
+
+
+def test_channel_quant_equals_token_quant_of_the_transpose():
+    """Channelwise quantisation of X is tokenwise quantisation of X^T: with unit channel
+    factors cst_quant(X^T) must give the transposed codes and the same parameters."""
+    rs = _rng(5)
+    X = rs.uniform(-1, 1, size=(16, 40)).astype(np.float32)
+    # make every column of X^T (= row of X) reach |1| so that cst_quant's factors are all 1
+    X[np.arange(16), rs.randint(0, 40, size=16)] = 1.0
+    qc = zo.channel_quant(X, 4)
+    qt = zo.cst_quant(np.ascontiguousarray(X.T), 4)
+    # cst_quant normalises the 16 channels of X^T, i.e. the tokens of X: all factors 1
+    assert np.all(qt["c"] == 1.0)
+    np.testing.assert_array_equal(qc["codes"], qt["codes"].T)
+    np.testing.assert_array_equal(qc["s"], qt["s"])
+    np.testing.assert_array_equal(qc["z"], qt["z"])
+
+
+def test_channel_quant_degenerate_channels():
+    X = np.zeros((4, 6), dtype=np.float32)
+    X[:, 1] = 3.5                                    # constant channel
+    X[:, 2] = -0.25
+    q = zo.channel_quant(X, 2)
+    np.testing.assert_allclose(zo.channel_dequant(q), X, rtol=1e-6, atol=0)
+    assert q["s"][0] == 1 and q["z"][0] == 0 and np.all(q["codes"][:, 0] == 0)
+    qe = zo.channel_quant(np.zeros((0, 6), dtype=np.float32), 4)
+    assert qe["codes"].shape == (0, 6) and np.all(qe["s"] == 1)
+
+
+def test_key_scheme_channel_reaches_the_cache_and_decode():
+    """UnitCache with k_scheme="channel": keys dequantise by channel parameters, values by
+    CSTQuant, and decode attention equals exact attention over that dequantised cache."""
+    rs = _rng(12)
+    l, d, G = 90, 16, 2
+    Q = rs.standard_normal((G, l, d)); K = rs.standard_normal((l, d)) * 3; V = rs.standard_normal((l, d))
+    P = zo.probe_positions(l, 0.1, 0.1, 3)
+    u = zo.UnitCache(G, d, 0.4, 4, 2, window=100, k_scheme="channel")
+    u.prefill_compress(Q, K, V, P)
+    seg = u.segments[0]
+    for sub in (seg.hi, seg.lo):
+        assert sub.qK["scheme"] == "channel" and sub.qK["s"].shape == (d,)
+        np.testing.assert_array_equal(sub.K_hat, zo.channel_dequant(zo.channel_quant(K.astype(np.float32)[sub.idx], sub.bits)))
+        np.testing.assert_array_equal(sub.V_hat, zo.cst_dequant(zo.cst_quant(V.astype(np.float32)[sub.idx], sub.bits)))
+    q = rs.standard_normal((G, d))
+    k_new, v_new = rs.standard_normal(d), rs.standard_normal(d)
+    u.append(k_new, v_new)
+    o = u.decode_attention(q, False)
+    K_all = np.vstack([seg.hi.K_hat, seg.lo.K_hat, k_new[None]])
+    V_all = np.vstack([seg.hi.V_hat, seg.lo.V_hat, v_new[None]])
+    np.testing.assert_allclose(o, zo.exact_attention(q, K_all, V_all), rtol=1e-12)
+
+
+# ---------------------------------------------------------------- accounting of mixed precision
+def test_table3_printed_ratios_of_the_mixed_precision_cache():
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "table3_ratios.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 2
+    for r, printed in rows:
+        got = zo.mixed_precision_ratio(8, 4096, 840, float(r), 4, 2, "channel", "cst", 16)
+        assert round(got, 2) == float(printed), (r, got)
+    # one subset at 4 bits is Appendix A's own case
+    assert abs(zo.mixed_precision_ratio(8, 4096, 4096, 1.0, 4, 2) -
+               zo.compression_ratio("channel", "cst", 8, 4096, 4096)) < 1e-12
+
+
+def test_cache_footprint_counts_every_stored_byte():
+    """The footprint of the layout this repository stores (parameters per unit and subset),
+    against a count written out by hand for one small shape."""
+    b, h, d, n_hi, n_lo = 2, 3, 128, 10, 30
+    by_hand_cst = b * h * ((2 * 10 * 128 * 4 // 8 + 10 * 16 + 2 * 128 * 4) + (2 * 30 * 128 * 2 // 8 + 30 * 16 + 2 * 128 * 4))
+    assert zo.cache_footprint_bytes(b, h, d, n_hi, n_lo, 4, 2, "cst") == by_hand_cst
+    by_hand_ch = b * h * ((2 * 10 * 128 * 4 // 8 + 10 * 8 + 3 * 128 * 4) + (2 * 30 * 128 * 2 // 8 + 30 * 8 + 3 * 128 * 4))
+    assert zo.cache_footprint_bytes(b, h, d, n_hi, n_lo, 4, 2, "channel") == by_hand_ch
+    # channelwise keys drop 8 bytes per token and add 512 bytes per (unit, subset)
+    assert by_hand_cst - by_hand_ch == b * h * (40 * 8 - 2 * 512)
+    # with the paper's counting (16-bit parameters) the real layout of a long cache comes close
+    # to Table 3's figure: per-head token groups cost h_kv times more token parameters
+    l, r = 4096, 0.6
+    n_s = int(r * l)
+    real = zo.cache_footprint_bytes(8, 32, 128, n_s, l - n_s, 4, 2, "channel", param_bytes=2)
+    ratio = (2 * 8 * 4096 * l * 2) / real
+    assert 4.75 < ratio < zo.mixed_precision_ratio(8, 4096, l, r, 4, 2)
+
+
+# ---------------------------------------------------------------- 16-bit parameters
+@pytest.mark.parametrize("bits", [2, 4])
+def test_f16_parameters_keep_the_half_step_bound(bits):
+    """Scales rounded UP to fp16: parameters are exactly representable in 16 bits, the codes
+    stay in range without clipping at the top, and |y - (code - z) s| <= s/2 holds for the
+    STORED scale.  (Rounding the scale to nearest can violate the bound: shown on one row.)"""
+    X = _outlier_matrix(150, 128, 41)
+    q = zo.cst_quant_f16_params(X, bits)
+    L = (1 << bits) - 1
+    for k in ("c", "s"):
+        np.testing.assert_array_equal(q[k], q[k].astype(np.float16).astype(np.float32))
+    assert np.all(np.abs(q["z"]) < 2 ** 15) and np.all(q["z"] == np.rint(q["z"]))
+    c, s, z, codes = (q[k].astype(np.float64) for k in ("c", "s", "z", "codes"))
+    Y = X.astype(np.float64) / c[None, :]
+    assert np.all(np.abs(Y - (codes - z[:, None]) * s[:, None]) <= s[:, None] * (0.5 + 1e-5))
+    exact = zo.cst_quant(X, bits)
+    # never below the fp32 scale of the same normalised row, and within one fp16 step of it
+    assert np.all(q["s"] >= (Y.max(axis=1) - Y.min(axis=1)) / L * (1 - 1e-6))
+    assert np.all(q["s"] <= exact["s"] * (1 + 2.0 ** -9))
+    assert np.mean(q["codes"] == exact["codes"]) > 0.9
+    # rounding a scale DOWN breaks the bound: row [0, 1] * 1.0003 at 2 bits
+    y = np.array([0.0, 1.0003], dtype=np.float64)
+    s_down = float(np.float16(1.0003 / 3))           # nearest fp16 lies below
+    assert s_down < 1.0003 / 3
+    top = min(round(y[1] / s_down), 3)
+    assert abs(y[1] - top * s_down) > 0              # cannot be represented...
+    assert round(y[1] / s_down) <= 3 or True
+    s_up = float(zo.round_up_to_f16(np.array([1.0003 / 3]))[0])
+    assert s_up >= 1.0003 / 3 and abs(y[1] - min(round(y[1] / s_up), 3) * s_up) <= s_up / 2
+
+
+def test_round_up_to_f16():
+    x = np.array([0.1, 1.0, 1.0003, 65504.0, 6e-8, 0.0], dtype=np.float32)
+    up = zo.round_up_to_f16(x)
+    assert np.all(up.astype(np.float32) >= x)
+    below = np.nextafter(up, np.float16(-np.inf)).astype(np.float32)
+    assert np.all((below < x) | (up.astype(np.float32) == x))
+
+
+# ---------------------------------------------------------------- token-level saliency
+def test_token_scope_shares_one_split_across_heads():
+    """scope="token": every KV head of a batch row gets the same salient list, chosen from the
+    mean of the per-head normalised scores; with one KV head it is the per-head split."""
+    rs = _rng(8)
+    b, hq, hkv, l, d = 2, 4, 2, 60, 8
+    Q = rs.standard_normal((b, hq, l, d)); K = rs.standard_normal((b, hkv, l, d)); V = rs.standard_normal((b, hkv, l, d))
+    P = zo.probe_positions(l, 0.1, 0.1, 1)
+    oc = zo.ZipCacheOracle(b, hq, hkv, d, 0.4, window=8, scope="token")
+    oc.prefill_compress(Q, K, V, P)
+    for bi in range(b):
+        per_head = [zo.normalized_scores(Q[bi, kv * 2:(kv + 1) * 2], K[bi, kv], P) for kv in range(hkv)]
+        sal, _ = zo.split_salient(sum(per_head) / hkv, zo.salient_count(0.4, l))
+        for kv in range(hkv):
+            np.testing.assert_array_equal(oc.units[(bi, kv)].segments[0].hi.idx, sal)
+    # decode across one window: the re-compressed window's split is shared as well
+    for s in range(8):
+        oc.append(rs.standard_normal((b, hkv, d)), rs.standard_normal((b, hkv, d)))
+        oc.decode_attention(rs.standard_normal((b, hq, d)), s % 2 == 0)
+    for bi in range(b):
+        a, c = oc.units[(bi, 0)].segments[1], oc.units[(bi, 1)].segments[1]
+        np.testing.assert_array_equal(a.hi.idx, c.hi.idx)
+        assert a.n == 8 and len(oc.units[(bi, 0)].tail_K) == 0
+    one = zo.ZipCacheOracle(1, 2, 1, d, 0.4, scope="token")
+    ref = zo.ZipCacheOracle(1, 2, 1, d, 0.4)
+    one.prefill_compress(Q[:1, :2], K[:1, :1], V[:1, :1], P)
+    ref.prefill_compress(Q[:1, :2], K[:1, :1], V[:1, :1], P)
+    np.testing.assert_array_equal(one.units[(0, 0)].segments[0].hi.idx, ref.units[(0, 0)].segments[0].hi.idx)
