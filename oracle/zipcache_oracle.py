@@ -254,8 +254,8 @@ def cst_quant_f16_params(X: np.ndarray, bits: int) -> Dict[str, np.ndarray]:
 
     The scale is rounded UP to fp16 before the codes are formed, so the codes of a token span
     at most the same range as with the fp32 scale and the error bound |y - (code - z) s| <= s/2
-    holds for the stored scale (rounding to nearest could shrink s and push the token's
-    maximum beyond the top code).  Everything else follows cst_quant."""
+    holds for the stored scale (a scale rounded down no longer covers the row: the token's
+    maximum then lies beyond the top code).  Everything else follows cst_quant."""
     f32 = np.float32
     X = np.asarray(X, dtype=f32)
     n, d = X.shape
