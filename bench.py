@@ -370,6 +370,8 @@ def run_reference(args):
 MODES = {
     "overlap": dict(overlap_calls=True, defer_append=True),
     "dependent": dict(overlap_calls=False, defer_append=True),
+    # the paper's own key quantiser (channelwise keys: 8 bytes per token less to read)
+    "overlap_channelwise_keys": dict(overlap_calls=True, defer_append=True, k_channel=True),
 }
 
 
@@ -595,7 +597,7 @@ def main():
     ap.add_argument("--config", type=int, default=0, help="one workload only (default: 2, 3, 4 and 5)")
     ap.add_argument("--decode-steps", type=int, default=0,
                     help="profiling only: fewer decode steps than the workload's own")
-    ap.add_argument("--mode", default="both", choices=["both", "overlap", "dependent"],
+    ap.add_argument("--mode", default="both", choices=["both", "overlap", "dependent", "overlap_channelwise_keys"],
                     help="overlap: ZC_FLAG_OVERLAP_CALLS (independent caches, calls side by side); "
                          "dependent: every call waits for the kernel before it")
     ap.add_argument("--append", default="deferred", choices=["deferred", "kernel"],
@@ -625,7 +627,7 @@ def main():
     zc.load_library()
     configs = [args.config] if args.config else list(DEFAULT_CONFIGS)
     head_cfg = args.config or HEADLINE_CONFIG
-    modes = ["overlap", "dependent"] if args.mode == "both" else [args.mode]
+    modes = ["overlap", "dependent", "overlap_channelwise_keys"] if args.mode == "both" else [args.mode]
     head_mode = modes[0]
     per_config, head = {}, None
     e2e = None

@@ -35,6 +35,11 @@ extern "C" {
 typedef struct CUstream_st* zc_stream_t; /* a cudaStream_t */
 
 enum { ZC_F16 = 0, ZC_BF16 = 1 };
+/* How keys are quantised (values always by CSTQuant, Alg. 1).  ZC_K_CHANNEL is the paper's own
+ * setting (Sec. 4.1, Table 1 last row, Alg. 2 "ChannelQuant"): Eq. 5 with minimum and maximum
+ * taken over the tokens of a subset, one (s, z) pair per channel and none per token, which
+ * saves 8 bytes per cached token. */
+enum { ZC_K_CST = 0, ZC_K_CHANNEL = 1 };
 
 enum {
   ZC_OK = 0,
@@ -86,6 +91,9 @@ typedef struct {
   int32_t bits_lo;        /* bit-width of regular tokens: 4 or 2 */
   int32_t flags;          /* 0 or an OR of the ZC_FLAG_* values above */
   double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
+  int32_t k_scheme;       /* quantiser of the keys: ZC_K_CST (Alg. 1 on K and V) or ZC_K_CHANNEL
+                             (channelwise keys, Sec. 4.1 last paragraph / Alg. 2; values stay CST) */
+  int32_t reserved;       /* must be 0 */
 } zc_config;
 
 typedef struct zc_cache zc_cache; /* small host-side handle */
@@ -161,7 +169,10 @@ int zc_tail_tokens(const zc_cache* c);
  * within the segment); codes b x h_kv x n x (d*bits/8) bytes in canonical packing
  * (4-bit: element 2m low nibble, 2m+1 high nibble of byte m; 2-bit: element 4m+j in
  * bits [2j,2j+1] of byte m); sz b x h_kv x n x 2 floats (scale, zero point);
- * cf b x h_kv x d floats (channel factors).  tensor 0 = K, 1 = V.  Any out may be NULL. */
+ * cf b x h_kv x d floats (channel factors).  tensor 0 = K, 1 = V.  Any out may be NULL.
+ * Keys under ZC_K_CHANNEL have no per-token parameters and no channel factors: for tensor 0,
+ * sz then receives b x h_kv x d x 2 floats, the (scale, zero point) of every channel, and cf
+ * is left untouched. */
 int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t* idx,
                       uint8_t* codes, float* sz, float* cf, zc_stream_t stream);
 

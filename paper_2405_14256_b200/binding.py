@@ -15,6 +15,7 @@ ZC_F16, ZC_BF16 = 0, 1
 ZC_FLAG_DEFER_APPEND = 1
 ZC_FLAG_OVERLAP_CALLS = 2
 ZC_FLAG_OUT_F32 = 4
+ZC_K_CST, ZC_K_CHANNEL = 0, 1
 
 
 class ZipCacheError(RuntimeError):
@@ -27,16 +28,17 @@ class ZcConfig(C.Structure):
         ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
         ("max_prefill", C.c_int32), ("max_new_tokens", C.c_int32), ("window", C.c_int32),
         ("bits_hi", C.c_int32), ("bits_lo", C.c_int32), ("flags", C.c_int32),
-        ("saliency_ratio", C.c_double),
+        ("saliency_ratio", C.c_double), ("k_scheme", C.c_int32), ("reserved", C.c_int32),
     ]
 
     @classmethod
     def make(cls, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
              saliency_ratio, bits_hi=4, bits_lo=2, window=100, head_dim=128,
-             flags=0) -> "ZcConfig":
+             flags=0, k_scheme=0) -> "ZcConfig":
         code = {torch.float16: ZC_F16, torch.bfloat16: ZC_BF16}.get(dtype, dtype)
         return cls(C.sizeof(cls), code, batch, n_q_heads, n_kv_heads, head_dim, max_prefill,
-                   max_new_tokens, window, bits_hi, bits_lo, flags, float(saliency_ratio))
+                   max_new_tokens, window, bits_hi, bits_lo, flags, float(saliency_ratio),
+                   int(k_scheme), 0)
 
 
 _lib = None
@@ -244,14 +246,16 @@ class ZipCache:
     def __init__(self, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
                  workspace: Optional[torch.Tensor] = None, defer_append: bool = False,
-                 overlap_calls: bool = False, out_f32: bool = False):
+                 overlap_calls: bool = False, out_f32: bool = False, k_channel: bool = False):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                                  saliency_ratio, bits_hi, bits_lo, window,
                                  flags=(ZC_FLAG_DEFER_APPEND if defer_append else 0) |
                                  (ZC_FLAG_OVERLAP_CALLS if overlap_calls else 0) |
-                                 (ZC_FLAG_OUT_F32 if out_f32 else 0))
+                                 (ZC_FLAG_OUT_F32 if out_f32 else 0),
+                                 k_scheme=ZC_K_CHANNEL if k_channel else ZC_K_CST)
+        self.k_channel = bool(k_channel)
         self.out_dtype = torch.float32 if out_f32 else dtype
         self.dtype, self.device = dtype, torch.device(device)
         self.batch, self.n_q_heads, self.n_kv_heads = batch, n_q_heads, n_kv_heads
@@ -300,7 +304,9 @@ class ZipCache:
         dev = self.device
         idx = torch.zeros((b, h, n), dtype=torch.int32, device=dev)
         codes = torch.zeros((b, h, n, 16 * bits), dtype=torch.uint8, device=dev)
-        sz = torch.zeros((b, h, n, 2), dtype=torch.float32, device=dev)
+        # channelwise keys: (scale, zero point) per channel instead of per token
+        sz = torch.zeros((b, h, 128 if (self.k_channel and tensor == 0) else n, 2), dtype=torch.float32,
+                         device=dev)
         cf = torch.zeros((b, h, 128), dtype=torch.float32, device=dev)
         if n > 0:
             zc_export_segment(self.handle, segment, tensor, subset, idx, codes, sz, cf)

@@ -153,9 +153,11 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayo
 // channel and CTA.
 constexpr int kAbsTiles = 4;
 
+// Channelwise keys (lay.kch): the same pass takes the signed minimum and maximum of every key
+// channel instead of the maximum of its magnitude.
 template <typename T>
 __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
-  __shared__ float red[2][8][ZC_D];
+  __shared__ float red[3][8][ZC_D];
   const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
   const int groups_c0 = zc_ceil_div(zc_ceil_div(seg.n_tok[0], ZC_TILE), kAbsTiles);
   const int cls = (int)blockIdx.x < groups_c0 ? 0 : 1;
@@ -166,7 +168,10 @@ __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout la
   const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh;
   const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  float mk[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+  const bool kch = lay.kch != 0;
+  const float k0 = kch ? -INFINITY : 0.f;
+  float mk[4] = {k0, k0, k0, k0}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+  float nk[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
   const int t_lo = grp * kAbsTiles * ZC_TILE;
   const int t_hi = min(seg.n_tok[cls], t_lo + kAbsTiles * ZC_TILE);
 #pragma unroll 4
@@ -175,7 +180,10 @@ __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout la
     float x[4];
     zc_load4<T>(Kb + row + 4 * lane, x);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) mk[e] = fmaxf(mk[e], fabsf(x[e]));
+    for (int e = 0; e < 4; ++e) {
+      mk[e] = fmaxf(mk[e], kch ? x[e] : fabsf(x[e]));
+      nk[e] = fminf(nk[e], x[e]);
+    }
     zc_load4<T>(Vb + row + 4 * lane, x);
 #pragma unroll
     for (int e = 0; e < 4; ++e) mv[e] = fmaxf(mv[e], fabsf(x[e]));
@@ -184,20 +192,26 @@ __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout la
   for (int e = 0; e < 4; ++e) {
     red[0][w][4 * lane + e] = mk[e];
     red[1][w][4 * lane + e] = mv[e];
+    red[2][w][4 * lane + e] = nk[e];
   }
   __syncthreads();
-  const int ten = threadIdx.x >> 7, ch = threadIdx.x & 127;
-  float m = 0.f;
+  unsigned* cmax = reinterpret_cast<unsigned*>(ub + lay.off_cmax) + cls * 3 * ZC_D;
+  for (int a = threadIdx.x; a < (kch ? 3 : 2) * ZC_D; a += 256) {
+    const int ten = a >> 7, ch = a & 127;
+    float m = red[ten][0][ch];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) m = fmaxf(m, red[ten][i][ch]);
-  unsigned* cmax = reinterpret_cast<unsigned*>(ub + lay.off_cmax) + (cls * 2 + ten) * ZC_D;
-  atomicMax(&cmax[ch], __float_as_uint(m));  // non-negative floats order like their bits
+    for (int i = 1; i < 8; ++i) m = ten == 2 ? fminf(m, red[ten][i][ch]) : fmaxf(m, red[ten][i][ch]);
+    // ordered keys: integer order is float order for signed values too
+    if (ten == 2) atomicMin(&cmax[ten * ZC_D + ch], zc_float_key(m));
+    else atomicMax(&cmax[ten * ZC_D + ch], zc_float_key(m));
+  }
 }
 
 __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
   char* ub = zc_unit_base(cache, lay, blockIdx.x);
   unsigned* cmax = reinterpret_cast<unsigned*>(ub + lay.off_cmax);
-  for (int i = threadIdx.x; i < 4 * ZC_D; i += blockDim.x) cmax[i] = 0u;
+  // maxima start below every key, minima above (per class: K max, V max, K min)
+  for (int i = threadIdx.x; i < 6 * ZC_D; i += blockDim.x) cmax[i] = ((i / ZC_D) % 3 == 2) ? 0xffffffffu : 0u;
   float* fac = reinterpret_cast<float*>(ub + lay.off_fac);
   if (threadIdx.x < 2) fac[(seg.run0 + threadIdx.x) * ZC_FAC_FLOATS + 2 * ZC_D] = 0.f;  // smaxV
 }
@@ -221,14 +235,20 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh;
   const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const unsigned* cmax = reinterpret_cast<const unsigned*>(ub + lay.off_cmax) + cls * 2 * ZC_D;
+  const unsigned* cmax = reinterpret_cast<const unsigned*>(ub + lay.off_cmax) + cls * 3 * ZC_D;
   float* fac = reinterpret_cast<float*>(ub + lay.off_fac) + (seg.run0 + cls) * ZC_FAC_FLOATS;
-  float cK[4], cV[4];
+  const bool kch = lay.kch != 0;
+  float cK[4], cV[4], zK[4];   // channelwise keys: cK holds the channel scales, zK the zero points
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
-    const float mk = __uint_as_float(cmax[4 * lane + e]);
-    const float mv = __uint_as_float(cmax[ZC_D + 4 * lane + e]);
-    cK[e] = mk == 0.f ? 1.f : __fsqrt_rn(mk);
+    const float mk = zc_key_float(cmax[4 * lane + e]);
+    const float mv = zc_key_float(cmax[ZC_D + 4 * lane + e]);
+    if (kch) {
+      channel_params(zc_key_float(cmax[2 * ZC_D + 4 * lane + e]), mk, L, &cK[e], &zK[e]);
+    } else {
+      cK[e] = mk == 0.f ? 1.f : __fsqrt_rn(mk);
+      zK[e] = 0.f;
+    }
     cV[e] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
   }
   if (tile == 0 && w == 0) {
@@ -236,6 +256,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     for (int e = 0; e < 4; ++e) {
       fac[4 * lane + e] = cK[e];
       fac[ZC_D + 4 * lane + e] = cV[e];
+      if (kch) fac[ZC_FAC_ZK + 4 * lane + e] = zK[e];
     }
   }
   const int t0 = tile * ZC_TILE;
@@ -266,9 +287,13 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
       const T* ek = reinterpret_cast<const T*>(&rawK[i]);
 #pragma unroll
       for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
-      quant_token(x, cK, L, &s, &z, &pk);
+      if (kch) {
+        pk = quant_channel4(x, cK, zK, L);
+      } else {
+        quant_token(x, cK, L, &s, &z, &pk);
+        if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
+      }
       *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live ? pk : 0u;
-      if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
       const T* ev = reinterpret_cast<const T*>(&rawV[i]);
 #pragma unroll
       for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
@@ -285,7 +310,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
   const int total_vec = lay.tile_bytes[cls] / 16;
   for (int v = threadIdx.x; v < total_vec; v += 256)
-    reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(bits, v, 0, codesK, codesV, parK, parV);
+    reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(bits, lay.kch, v, 0, codesK, codesV, parK, parV);
 }
 
 }  // namespace

@@ -26,6 +26,7 @@
 // Each warp owns a ring of shared-memory stages filled by bulk asynchronous copies (one per
 // 16-token sub-block, completion on an mbarrier), so a CTA needs no block-wide barrier in
 // its main loop.  Every wait is bounded; a wait that runs out records an error code.
+#include <atomic>
 #include <mutex>
 #include "zc_internal.h"
 #include "zc_layout.cuh"
@@ -57,7 +58,8 @@ constexpr int kOffWl = kOffWm + 64;                  // [kWarps][4] sums
 constexpr int kOffWz = kOffWl + 64;                  // [kWarps][4] zero-point sums
 constexpr int kOffCw = kOffWz + 64;                  // [4 heads][kWarps] merge weights
 constexpr int kOffHead = kOffCw + 64;                // [4 heads] x (M, L, Z, -)
-constexpr int kOffRing = kOffHead + 128;             // kWarps rings
+constexpr int kOffZq = kOffHead + 128;               // [kWarps][4 heads] partial sums of q' . z (channelwise keys)
+constexpr int kOffRing = kOffZq + 128;               // kWarps rings
 constexpr int decode_smem(int ring) { return kOffRing + kWarps * ring; }
 
 __device__ int g_zc_error = 0;
@@ -247,17 +249,24 @@ struct PairState {
 // (head n >> 1, part n & 1) with q' = hi + lo in f16, so that lane (g, t) receives both parts
 // of head t for tokens g and g + 8 in its accumulator.  LAST: the pair may reach past the end
 // of the run (`rem` tokens left from its first token); otherwise it is complete.
-template <int BITS, bool LAST>
+// KCH: channelwise keys -- a token has no key parameters (the channel scales are folded into
+// q', qs is then sum_i q'_i z_i), its parameter slot holds (sV, zV) only.
+template <int BITS, bool LAST, bool KCH>
 __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uint32_t (&qb)[16],
                                           float qs, float isc, float logKs, float tau_u, int srcA,
                                           int srcB, int c0_src, int c1_src, float (&oacc)[8][4],
                                           PairState& S) {
-  constexpr int SB = ZC_SUB * (32 * BITS + 16);
+  constexpr int PARB = KCH ? 8 : 16;
+  constexpr int SB = ZC_SUB * (32 * BITS + PARB);
   const int g = lane >> 2;
   if (LAST && rem <= ZC_SUB) {
     // the run ends inside the first half: the second half was not copied; its tokens are
     // masked below, its parameters must not hold stale bits
-    if (lane < ZC_SUB) *reinterpret_cast<float4*>(st + SB + 512 * BITS + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (KCH) {
+      if (lane < ZC_SUB) *reinterpret_cast<float2*>(st + SB + 512 * BITS + lane * 8) = make_float2(0.f, 0.f);
+    } else {
+      if (lane < ZC_SUB) *reinterpret_cast<float4*>(st + SB + 512 * BITS + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     __syncwarp();
   }
   // ---- loads: K words of tokens g and g+8, V words, parameters (sK, zK, sV, zV), both halves ----
@@ -284,8 +293,15 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
       const uint4 c = *reinterpret_cast<const uint4*>(sh + 512 + lane * 16);
       vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
     }
-    pp[h][0] = *reinterpret_cast<const float4*>(sh + 512 * BITS + g * 16);
-    pp[h][1] = *reinterpret_cast<const float4*>(sh + 512 * BITS + (g + 8) * 16);
+    if (KCH) {
+      const float2 a = *reinterpret_cast<const float2*>(sh + 512 * BITS + g * 8);
+      const float2 b = *reinterpret_cast<const float2*>(sh + 512 * BITS + (g + 8) * 8);
+      pp[h][0] = make_float4(1.f, 1.f, a.x, a.y);
+      pp[h][1] = make_float4(1.f, 1.f, b.x, b.y);
+    } else {
+      pp[h][0] = *reinterpret_cast<const float4*>(sh + 512 * BITS + g * 16);
+      pp[h][1] = *reinterpret_cast<const float4*>(sh + 512 * BITS + (g + 8) * 16);
+    }
   }
   // ---- S^T = codes(16 tokens x 128) . q'^T per half: 8 k-steps; the halves are independent chains ----
   float u[2][2];   // [half][token slot] logits (base 2) of head t, divided by isc
@@ -320,8 +336,13 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
       }
     }
     // hi and lo parts of q' sit in columns 2t and 2t+1 of this lane
-    u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
-    u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;
+    if (KCH) {
+      u[h][0] = (dacc[0] + dacc[1]) - qs;
+      u[h][1] = (dacc[2] + dacc[3]) - qs;
+    } else {
+      u[h][0] = fmaf(-pp[h][0].y, qs, dacc[0] + dacc[1]) * pp[h][0].x;
+      u[h][1] = fmaf(-pp[h][1].y, qs, dacc[2] + dacc[3]) * pp[h][1].x;
+    }
   }
   if (LAST && rem < 2 * ZC_SUB) {
 #pragma unroll
@@ -396,15 +417,15 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
 // Compressed-run part of one item, one warp: prologue done by the CTA, stages primed.  The
 // first my_np - NST iterations refill their stage and need no end-of-run handling; the last
 // NST do not refill and the very last pair may be cut short by the end of the run.
-template <int BITS, int RING>
+template <int BITS, int RING, bool KCH>
 __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_base, char* my_ring,
                                           uint64_t* my_bar, const uint32_t (&qb)[16], float qs,
                                           float isc, float logK, int my_np, int warp, int lane,
                                           float (&oacc)[8][4], float& m_out, float& l_out,
                                           float& z_out, int* err) {
-  constexpr int SB = ZC_SUB * (32 * BITS + 16);
+  constexpr int SB = ZC_SUB * (32 * BITS + (KCH ? 8 : 16));
   constexpr int PB = 2 * SB;
-  constexpr int NST = RING / PB;
+  constexpr int NST = (RING / PB) < kMaxStages ? (RING / PB) : kMaxStages;
   const int g = lane >> 2, t = lane & 3;
   const bool odd_tok = BITS == 2 && (g & 1);
   const float logKs = logK - (odd_tok ? 2.f : 0.f);      // weights of odd tokens carry 1/4 at 2 bits
@@ -434,7 +455,7 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
     uint64_t* bar = &my_bar[stage];
     wait_stage(bar);
     char* st = my_ring + stage * PB;
-    pair_step<BITS, false>(st, lane, 0, qb, qs, isc, logKs, tau_u, srcA, srcB, c0_src, c1_src, oacc, S);
+    pair_step<BITS, false, KCH>(st, lane, 0, qb, qs, isc, logKs, tau_u, srcA, srcB, c0_src, c1_src, oacc, S);
     __syncwarp();
     refill_if(lane == 0, bar, st, src_refill, rem_refill > ZC_SUB ? PB : SB);
     src_refill += kWarps * PB;
@@ -443,7 +464,7 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
   }
   for (int i = max(n_refill, 0); i < my_np; ++i) {
     wait_stage(&my_bar[stage]);
-    pair_step<BITS, true>(my_ring + stage * PB, lane, rem0 - i * (2 * ZC_SUB * kWarps), qb, qs, isc, logKs,
+    pair_step<BITS, true, KCH>(my_ring + stage * PB, lane, rem0 - i * (2 * ZC_SUB * kWarps), qb, qs, isc, logKs,
                           tau_u, srcA, srcB, c0_src, c1_src, oacc, S);
     if (++stage == NST) { stage = 0; parity ^= 1u; }
   }
@@ -460,13 +481,13 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
 // Not inlined: the loop inside gets the whole register budget to itself, whatever the caller
 // keeps alive around the call.
 struct ItemScale { float chan_factor, rowscale; };
-template <typename T, int BITS, int RING>
+template <typename T, int BITS, int RING, bool KCH>
 __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_base, const float* fac,
                                                   const T* qbase, int Gl, char* smem, int* err) {
-  constexpr int SB = ZC_SUB * (32 * BITS + 16);
+  constexpr int SB = ZC_SUB * (32 * BITS + (KCH ? 8 : 16));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   constexpr int PB = 2 * SB;
-  constexpr int NST = RING / PB;
+  constexpr int NST = (RING / PB) < kMaxStages ? (RING / PB) : kMaxStages;
   char* my_ring = smem + kOffRing + warp * RING;
   uint64_t* my_bar = reinterpret_cast<uint64_t*>(smem + kOffBars) + warp * kMaxStages;
   uint4* qfrag = reinterpret_cast<uint4*>(smem + kOffQfrag);
@@ -478,9 +499,10 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
   const int my_np = n_pairs > warp ? (n_pairs - warp + kWarps - 1) / kWarps : 0;
   // ---- the few words the set-up needs go out first, ahead of this CTA's own 55 KB of copies ----
   const float scale = kLog2e * rsqrtf((float)ZC_D);
-  const float cK = fac[tid];
+  const float cK = fac[tid];              // channelwise keys: the channel's scale
   const float cV = fac[ZC_D + tid];
   const float smax = fac[2 * ZC_D];
+  const float zK = KCH ? fac[ZC_FAC_ZK + tid] : 0.f;
   T qraw[4];   // used only after the copies below are on their way
 #pragma unroll
   for (int h = 0; h < 4; ++h) qraw[h] = qbase[(h < Gl ? h : 0) * ZC_D + tid];
@@ -516,6 +538,7 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
     __half* qh = reinterpret_cast<__half*>(qfrag);
     const float hs_is = (scaled ? __uint_as_float((267u - ex_q) << 23) : 1.f) * is;
     const int base = ((reg >> 2) * 32 + t_l) * 4 + (reg & 3);          // + 4 * (4 * column)
+    float zq[4];   // channelwise keys: this channel's share of sum_i q'_i z_i, in the accumulator's units
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
       const float xs = x[h] * hs_is;
@@ -523,6 +546,20 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
       const __half lo = __float2half_rn(xs - __half2float(hi));
       qh[(base + 16 * (2 * h)) * 2 + e] = hi;
       qh[(base + 16 * (2 * h + 1)) * 2 + e] = lo;
+      // the operands as the tensor cores see them, times the code's power of two (1 / is), 2^-24
+      if (KCH) zq[h] = (__half2float(hi) + __half2float(lo)) * (zK * (5.9604644775390625e-8f / is));
+    }
+    if (KCH) {
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) zq[h] += __shfl_xor_sync(kFull, zq[h], o);
+      }
+      if (lane == 0) {
+        float* zred = reinterpret_cast<float*>(smem + kOffZq);
+#pragma unroll
+        for (int h = 0; h < 4; ++h) zred[warp * 4 + h] = zq[h];
+      }
     }
   }
   __syncthreads();
@@ -543,7 +580,11 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
     const uint32_t a[4] = {one_lo, one_lo, one_hi, one_hi};
     zc_mma16816<__half>(ds[ks & 1], a, qb[2 * ks], qb[2 * ks + 1]);
   }
-  const float qs = (ds[0][0] + ds[1][0]) + (ds[0][1] + ds[1][1]);
+  float qs = (ds[0][0] + ds[1][0]) + (ds[0][1] + ds[1][1]);
+  if (KCH) {
+    const float* zred = reinterpret_cast<const float*>(smem + kOffZq);
+    qs = (zred[t] + zred[4 + t]) + (zred[8 + t] + zred[12 + t]);   // sum_i q'_i z_i of head t
+  }
   // accumulator * 2^24 / CTA scale = q' . code
   const float isc = 16777216.f * (scaled ? __uint_as_float((ex_q - 13u) << 23) : 1.f);
   // weights are scaled by 2^logK = 2^kPExp / 2^ceil(log2 smax) so that w <= 2^(kPExp + kTau)
@@ -556,7 +597,7 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
 #pragma unroll
     for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
   float m, l, z;
-  run_pairs<BITS, RING>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
+  run_pairs<BITS, RING, KCH>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
   __syncwarp();
   if (lane == 0)   // every copy has landed and been consumed: retire the barriers
     for (int s = 0; s < NST; ++s) mbar_inval(&my_bar[s]);
@@ -774,15 +815,15 @@ constexpr int kFlOffParK = kFlOffCodesV + ZC_SUB * ZC_D;                 // [16]
 constexpr int kFlOffParV = kFlOffParK + ZC_SUB * 2 * 4;
 constexpr int kFlOffKey = kFlOffParV + ZC_SUB * 2 * 4;                   // [128] score bits
 constexpr int kFlOffTok = kFlOffKey + ZC_MAX_WINDOW * 4;                 // [2][128] token of each class slot
-constexpr int kFlOffRed = kFlOffTok + 2 * ZC_MAX_WINDOW * 4;             // [4 warps][2][128] floats
-constexpr int kFlOffC = kFlOffRed + kWarps * 2 * ZC_D * 4;               // [2][128] channel factors
-constexpr int kFlOffMask = kFlOffC + 2 * ZC_D * 4;                       // [4] ballots
+constexpr int kFlOffRed = kFlOffTok + 2 * ZC_MAX_WINDOW * 4;             // [4 warps][3][128] floats
+constexpr int kFlOffC = kFlOffRed + kWarps * 3 * ZC_D * 4;               // [3][128] channel factors (cK | sK, cV, zK)
+constexpr int kFlOffMask = kFlOffC + 3 * ZC_D * 4;                       // [4] ballots
 constexpr int kFlOffSmax = kFlOffMask + 16;                              // [2] V scale maxima as bits
 constexpr int kFlushSmem = kFlOffSmax + 16;
 static_assert(kFlushSmem <= decode_smem(kRingNarrow), "the re-compression must fit the item phase's memory");
 static_assert(ZC_MAX_WINDOW == 32 * kWarps, "one thread per window token");
 
-template <typename T>
+template <typename T, bool KCH>
 __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay, const ZcFlushArgs& fl, char* smem) {
   auto codesK = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesK);
   auto codesV = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesV);
@@ -790,8 +831,9 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
   auto parV = reinterpret_cast<float (*)[2]>(smem + kFlOffParV);
   unsigned* s_key = reinterpret_cast<unsigned*>(smem + kFlOffKey);
   auto s_tok = reinterpret_cast<int (*)[ZC_MAX_WINDOW]>(smem + kFlOffTok);
-  auto red = reinterpret_cast<float (*)[2][ZC_D]>(smem + kFlOffRed);
-  auto s_c = reinterpret_cast<float (*)[ZC_D]>(smem + kFlOffC);
+  auto red = reinterpret_cast<float (*)[3][ZC_D]>(smem + kFlOffRed);
+  constexpr bool kch = KCH;
+  auto s_c = reinterpret_cast<float (*)[ZC_D]>(smem + kFlOffC);   // [3][128]
   unsigned* s_mask = reinterpret_cast<unsigned*>(smem + kFlOffMask);
   unsigned* s_smax = reinterpret_cast<unsigned*>(smem + kFlOffSmax);
   const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -847,15 +889,22 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
   for (int cls = 0; cls < 2; ++cls) {
     const int n_c = fl.seg.n_tok[cls];
     if (n_c == 0) continue;
-    // ---- channel |x| maxima over the class (Eq. 6) ----
+    // ---- channel |x| maxima over the class (Eq. 6); channelwise keys: their signed min and max ----
+    const int bits = lay.bits[cls];
+    const float L = (float)((1 << bits) - 1);
     {
-      float mk[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+      const float k0 = kch ? -INFINITY : 0.f;
+      float mk[4] = {k0, k0, k0, k0}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+      float nk[4] = {INFINITY, INFINITY, INFINITY, INFINITY};
       for (int r = w; r < n_c; r += kWarps) {
         const int row = s_tok[cls][r] * ZC_D;
         float x[4];
         zc_load4<T>(tK + row + 4 * lane, x);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) mk[e] = fmaxf(mk[e], fabsf(x[e]));
+        for (int e = 0; e < 4; ++e) {
+          mk[e] = fmaxf(mk[e], kch ? x[e] : fabsf(x[e]));
+          nk[e] = fminf(nk[e], x[e]);
+        }
         zc_load4<T>(tV + row + 4 * lane, x);
 #pragma unroll
         for (int e = 0; e < 4; ++e) mv[e] = fmaxf(mv[e], fabsf(x[e]));
@@ -864,24 +913,35 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
       for (int e = 0; e < 4; ++e) {
         red[w][0][4 * lane + e] = mk[e];
         red[w][1][4 * lane + e] = mv[e];
+        red[w][2][4 * lane + e] = nk[e];
       }
     }
     __syncthreads();
+    {
+      float mk = red[0][0][tid], mv = red[0][1][tid], nk = red[0][2][tid];
 #pragma unroll
-    for (int ten = 0; ten < 2; ++ten) {
-      float m = 0.f;
-#pragma unroll
-      for (int i = 0; i < kWarps; ++i) m = fmaxf(m, red[i][ten][tid]);
-      s_c[ten][tid] = m == 0.f ? 1.f : __fsqrt_rn(m);
+      for (int i = 1; i < kWarps; ++i) {
+        mk = fmaxf(mk, red[i][0][tid]);
+        mv = fmaxf(mv, red[i][1][tid]);
+        nk = fminf(nk, red[i][2][tid]);
+      }
+      if (kch) {
+        float sk, zk;
+        channel_params(nk, mk, L, &sk, &zk);
+        s_c[0][tid] = sk;
+        s_c[2][tid] = zk;
+      } else {
+        s_c[0][tid] = mk == 0.f ? 1.f : __fsqrt_rn(mk);
+      }
+      s_c[1][tid] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
     }
     __syncthreads();
-    const int bits = lay.bits[cls];
-    const float L = (float)((1 << bits) - 1);
-    float cK[4], cV[4];
+    float cK[4], cV[4], zK[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       cK[e] = s_c[0][4 * lane + e];
       cV[e] = s_c[1][4 * lane + e];
+      zK[e] = kch ? s_c[2][4 * lane + e] : 0.f;
     }
     float* fac = reinterpret_cast<float*>(ub + lay.off_fac) + (fl.seg.run0 + cls) * ZC_FAC_FLOATS;
     if (w == 0) {
@@ -889,12 +949,13 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
       for (int e = 0; e < 4; ++e) {
         fac[4 * lane + e] = cK[e];
         fac[ZC_D + 4 * lane + e] = cV[e];
+        if (kch) fac[ZC_FAC_ZK + 4 * lane + e] = zK[e];
       }
     }
     // ---- CSTQuant and packing, one 16-token sub-block at a time: four tokens per warp ----
     float smax = 0.f;
     const int subs = (n_c + ZC_SUB - 1) / ZC_SUB;
-    const int vecs = zc_sub_bytes(bits) / 16;
+    const int vecs = zc_sub_bytes(bits, kch) / 16;
     for (int sb = 0; sb < subs; ++sb) {
       uint2 rawK[4], rawV[4];
       bool live[4];
@@ -918,9 +979,13 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
         const T* ek = reinterpret_cast<const T*>(&rawK[i]);
 #pragma unroll
         for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
-        quant_token(x, cK, L, &sc, &z, &pk);
+        if (kch) {
+          pk = quant_channel4(x, cK, zK, L);
+        } else {
+          quant_token(x, cK, L, &sc, &z, &pk);
+          if (lane == 0) { parK[tl][0] = live[i] ? sc : 0.f; parK[tl][1] = live[i] ? z : 0.f; }
+        }
         *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live[i] ? pk : 0u;
-        if (lane == 0) { parK[tl][0] = live[i] ? sc : 0.f; parK[tl][1] = live[i] ? z : 0.f; }
         const T* ev = reinterpret_cast<const T*>(&rawV[i]);
 #pragma unroll
         for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
@@ -935,7 +1000,7 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
                        (long long)(fl.seg.tile0[cls] + sb / (ZC_TILE / ZC_SUB)) * lay.tile_bytes[cls];
       for (int v = tid; v < vecs; v += 128)
         reinterpret_cast<uint4*>(tile_ptr)[sub_in_tile * vecs + v] =
-            compose_vec(bits, sub_in_tile * vecs + v, ZC_SUB * sub_in_tile, codesK, codesV, parK, parV);
+            compose_vec(bits, kch, sub_in_tile * vecs + v, ZC_SUB * sub_in_tile, codesK, codesV, parK, parV);
       __syncthreads();   // the next sub-block reuses the code arrays
     }
     if (lane == 0 && smax > 0.f) atomicMax(&s_smax[cls], __float_as_uint(smax));
@@ -1041,7 +1106,7 @@ __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_t
 // share is kept apart by the host: each call of an epoch (the launches between two launches
 // made without early start) gets its own `slot`, which selects its region of the workspace
 // and its arrival counter.
-template <typename T, int RING, int NCTA>
+template <typename T, int RING, int NCTA, bool KCH>
 __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay, ZcDecodePlan plan,
                                                       const T* __restrict__ q, T* __restrict__ out,
                                                       float* part, float* stash_all, int slot,
@@ -1143,9 +1208,9 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
       const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
       const char* class_base = ub + lay.off_tiles[d.cls];
       if (lay.bits[d.cls] == 4)
-        sc = compressed_item<T, 4, RING>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
+        sc = compressed_item<T, 4, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
       else
-        sc = compressed_item<T, 2, RING>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
+        sc = compressed_item<T, 2, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
     }
     __syncthreads();
     // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
@@ -1209,7 +1274,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
                   lay.out_f32 ? reinterpret_cast<float*>(out) + out_off : nullptr, mine, stash_g, collect, smem);
     if (fl.on) {
       __syncthreads();   // the merge is done with the shared arrays; its additions to the statistics are visible
-      window_flush_unit<T>(ub, lay, fl, smem);
+      window_flush_unit<T, KCH>(ub, lay, fl, smem);
     }
   }
 }
@@ -1351,28 +1416,36 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   const int groups = (plan.items + plan.cta_items - 1) / plan.cta_items;
   const dim3 grid((unsigned)(c->lay.units * (groups * zs + (plan.fold_tail ? 0 : 1)) + 1));
   cudaError_t e;
-#define ZC_LAUNCH_STEP(T, RING, NCTA)                                                              \
+#define ZC_LAUNCH_STEP(T, RING, NCTA, KCH)                                                         \
   do {                                                                                             \
-    static int attr_dev = -1; /* the opt-in to large shared memory is per device */                \
+    /* the opt-in to large shared memory is per device and per kernel: one bit per device */       \
+    static std::atomic<unsigned long long> attr_done{0};                                           \
     int dev_now = 0;                                                                               \
     cudaGetDevice(&dev_now);                                                                       \
-    if (attr_dev != dev_now) {                                                                     \
-      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA>,                                            \
+    const unsigned long long bit = 1ull << (dev_now & 63);                                         \
+    if (!(attr_done.load(std::memory_order_acquire) & bit)) {                                      \
+      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA, KCH>,                                       \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));    \
       if (e != cudaSuccess) return e;                                                              \
-      attr_dev = dev_now;                                                                          \
+      attr_done.fetch_or(bit, std::memory_order_release);                                          \
     }                                                                                              \
-    e = launch_pdl(k_decode<T, RING, NCTA>, grid, dim3(128), decode_smem(RING), st, overlap,       \
+    e = launch_pdl(k_decode<T, RING, NCTA, KCH>, grid, dim3(128), decode_smem(RING), st, overlap,  \
                    c->base, c->lay, plan, (const T*)q, (T*)out, part, stash, slot, collect,        \
                    (const T*)k_new, (const T*)v_new, ord, fl);                                     \
   } while (0)
-  if (c->cfg.dtype == ZC_F16) {
-    if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(__half, kRingNarrow, 4);
-    else ZC_LAUNCH_STEP(__half, kRingWide, 3);
-  } else {
-    if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(__nv_bfloat16, kRingNarrow, 4);
-    else ZC_LAUNCH_STEP(__nv_bfloat16, kRingWide, 3);
-  }
+#define ZC_LAUNCH_T(T)                                                                             \
+  do {                                                                                             \
+    if (c->lay.kch) {                                                                              \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true);                          \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, true);                                                  \
+    } else {                                                                                       \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false);                         \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, false);                                                 \
+    }                                                                                              \
+  } while (0)
+  if (c->cfg.dtype == ZC_F16) ZC_LAUNCH_T(__half);
+  else ZC_LAUNCH_T(__nv_bfloat16);
+#undef ZC_LAUNCH_T
 #undef ZC_LAUNCH_STEP
   c->launches += 1;
   return e != cudaSuccess ? (int)e : (int)cudaGetLastError();

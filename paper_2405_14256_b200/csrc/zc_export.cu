@@ -28,15 +28,24 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
     for (int i = threadIdx.x; i < n_here; i += blockDim.x)
       idx_out[(long long)unit * n + t0 + i] = idx[t0 + i];
   }
-  if (sz_out) {
+  const int kch = lay.kch;
+  if (sz_out && kch && tensor == 0) {
+    // channelwise keys: (scale, zero point) of every channel, from the run's factor block
+    if (tile == 0) {
+      const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + (seg.run0 + subset) * ZC_FAC_FLOATS;
+      for (int i = threadIdx.x; i < 2 * ZC_D; i += blockDim.x)
+        sz_out[(long long)unit * 2 * ZC_D + i] = (i & 1) ? fac[ZC_FAC_ZK + (i >> 1)] : fac[i >> 1];
+    }
+  } else if (sz_out) {
     const int poff = zc_sub_off_par(bits);
     for (int i = threadIdx.x; i < 2 * n_here; i += blockDim.x) {
       const int tl = i >> 1;
-      const float* par = reinterpret_cast<const float*>(tp + (tl / ZC_SUB) * zc_sub_bytes(bits) + poff);
-      sz_out[((long long)unit * n + t0) * 2 + i] = par[4 * (tl % ZC_SUB) + 2 * tensor + (i & 1)];
+      const float* par = reinterpret_cast<const float*>(tp + (tl / ZC_SUB) * zc_sub_bytes(bits, kch) + poff);
+      sz_out[((long long)unit * n + t0) * 2 + i] =
+          kch ? par[2 * (tl % ZC_SUB) + (i & 1)] : par[4 * (tl % ZC_SUB) + 2 * tensor + (i & 1)];
     }
   }
-  if (cf_out && tile == 0) {
+  if (cf_out && tile == 0 && !(kch && tensor == 0)) {
     const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) +
                        (seg.run0 + subset) * ZC_FAC_FLOATS + (tensor == 0 ? 0 : ZC_D);
     for (int i = threadIdx.x; i < ZC_D; i += blockDim.x) cf_out[(long long)unit * ZC_D + i] = fac[i];
@@ -46,7 +55,7 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
     for (int i = threadIdx.x; i < n_here * row_bytes; i += blockDim.x) {
       const int tl = i / row_bytes, m = i % row_bytes;
       unsigned byte = 0;
-      const char* sb = tp + (tl / ZC_SUB) * zc_sub_bytes(bits);
+      const char* sb = tp + (tl / ZC_SUB) * zc_sub_bytes(bits, kch);
       if (tensor == 0) {
         byte = reinterpret_cast<const unsigned char*>(sb)[(tl % ZC_SUB) * row_bytes + m];
       } else {

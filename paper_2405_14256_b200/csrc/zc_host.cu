@@ -29,6 +29,8 @@ int check_config(const zc_config* cfg) {
   if (cfg->bits_lo != 4 && cfg->bits_lo != 2) return ZC_EINVAL;
   if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32)) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
+  if (cfg->k_scheme != ZC_K_CST && cfg->k_scheme != ZC_K_CHANNEL) return ZC_EINVAL;
+  if (cfg->reserved != 0) return ZC_EINVAL;
   if ((long long)cfg->batch * cfg->n_kv_heads > 65535) return ZC_EINVAL;
   // every re-compressed window adds two items to a decode call
   if (2 * (cfg->max_new_tokens / cfg->window) + 2 + 2 > ZC_MAX_ITEMS) return ZC_EINVAL;
@@ -43,6 +45,7 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   lay->window = cfg->window;
   lay->dtype = cfg->dtype;
   lay->out_f32 = (cfg->flags & ZC_FLAG_OUT_F32) ? 1 : 0;
+  lay->kch = cfg->k_scheme == ZC_K_CHANNEL ? 1 : 0;
   lay->bits[0] = cfg->bits_hi;
   lay->bits[1] = cfg->bits_lo;
   const int max_flush = cfg->max_new_tokens / cfg->window;
@@ -57,14 +60,14 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   lay->idx_cap0 = cfg->max_prefill;
   size_t off = 0;
   for (int c = 0; c < 2; ++c) {
-    lay->tile_bytes[c] = zc_tile_bytes(lay->bits[c]);
+    lay->tile_bytes[c] = zc_tile_bytes(lay->bits[c], lay->kch);
     lay->off_tiles[c] = (long long)off;
     off = align_up(off + (size_t)lay->cap_tiles[c] * lay->tile_bytes[c], 256);
   }
   lay->off_fac = (long long)off;
   off = align_up(off + (size_t)lay->max_runs * ZC_FAC_FLOATS * 4, 256);
   lay->off_cmax = (long long)off;
-  off = align_up(off + 2 * 2 * ZC_D * 4, 256);
+  off = align_up(off + 2 * 3 * ZC_D * 4, 256);
   lay->off_tailK = (long long)off;
   off = align_up(off + (size_t)cfg->window * ZC_D * elt, 256);
   lay->off_tailV = (long long)off;
@@ -493,11 +496,11 @@ int64_t zc_decode_bytes(const zc_cache* c) {
   if (!c || c->l0 < 0) return 0;
   int64_t per_unit = 0;
   for (int k = 0; k < 2; ++k) {
-    const int64_t per_tok = 32 * c->lay.bits[k] + 16;  // K+V codes, (s,z) pairs
+    const int64_t per_tok = 32 * c->lay.bits[k] + (c->lay.kch ? 8 : 16);  // K+V codes, (s,z) pairs
     const int64_t toks = (int64_t)c->n0[k] + (int64_t)(c->n_seg - 1) * c->nw[k];
     per_unit += toks * per_tok;
     const int runs = (c->n0[k] > 0 ? 1 : 0) + (c->nw[k] > 0 ? c->n_seg - 1 : 0);
-    per_unit += (int64_t)runs * 2 * ZC_D * 4;        // channel factors of K and V
+    per_unit += (int64_t)runs * (c->lay.kch ? 3 : 2) * ZC_D * 4;   // channel factors of V; of K, or its (s, z) per channel
   }
   per_unit += (int64_t)c->n_tail * 2 * ZC_D * 2;     // full-precision tail
   per_unit += (int64_t)c->lay.G * ZC_D * 2 * 2;      // q in, out

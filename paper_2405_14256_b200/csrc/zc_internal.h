@@ -9,7 +9,9 @@
 #define ZC_D 128            // head_dim
 #define ZC_TILE 64          // tokens per cache tile
 #define ZC_SUB 16           // tokens per MMA sub-tile inside a tile
-#define ZC_FAC_FLOATS 272   // per-run factor block: cK[128], cV[128], smaxV, pad
+#define ZC_FAC_FLOATS 400   // per-run factor block: cK[128] (channelwise keys: their scales), cV[128],
+                            // smaxV, pad to 272, then the zero points of channelwise keys [128]
+#define ZC_FAC_ZK 272
 #define ZC_PART_STRIDE 132  // split-K partial per head: m, l, pad, pad, acc[128]
 #define ZC_MAX_G 8
 #define ZC_MAX_SPLIT_HOST 32      // most items one class of segment 0 is split into
@@ -29,7 +31,8 @@
 // Per unit, at byte offsets from base + unit * unit_stride:
 //   off_tiles[c]   cap_tiles[c] tiles of class c (0 = salient bits, 1 = regular bits)
 //   off_fac        max_runs factor blocks (run = segment * 2 + class)
-//   off_cmax       scratch: |x| channel maxima as uint bits  [class][tensor][128]
+//   off_cmax       scratch of the quantiser, as ordered uint keys  [class][3][128]: channel maxima of
+//                  |K| (channelwise keys: of K), of |V|, and channel minima of K (channelwise keys)
 //   off_tailK/V    window x d elements of the input type
 //   off_colsum     window floats: attention mass collected on probe steps
 //   off_sync       ZC_EPOCH_CALLS arrival counters of the decode kernel's CTAs (zero between calls)
@@ -39,10 +42,11 @@
 // A tile of class c holds 64 tokens as four sub-blocks of 16 tokens, each
 //   [K codes 16 x 16*bits B, canonical nibble/crumb order per token row]
 //   [V codes of the 16 tokens in MMA fragment order (see zc_layout.cuh)]
-//   [params 16 x (K scale, K zero, V scale, V zero) f32]
+//   [params 16 x (K scale, K zero, V scale, V zero) f32; channelwise keys: 16 x (V scale, V zero)]
 struct ZcLayout {
   int units, G, n_kv, window, dtype;
   int out_f32;            // decode outputs are stored as fp32 (ZC_FLAG_OUT_F32)
+  int kch;                // keys are quantised channelwise (ZC_K_CHANNEL): no per-token key parameters
   int bits[2];
   int tile_bytes[2];
   int cap_tiles[2];

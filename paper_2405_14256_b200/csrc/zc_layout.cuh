@@ -17,8 +17,9 @@
 // A tile is four self-contained sub-blocks of 16 tokens, so that one bulk copy brings
 // everything a warp needs for one MMA sub-tile:
 //   [K codes 16 rows x 16*bits B][V codes, fragment order][(sK, zK, sV, zV) x 16]
-__host__ __device__ inline int zc_sub_bytes(int bits) { return ZC_SUB * (32 * bits + 16); }
-__host__ __device__ inline int zc_tile_bytes(int bits) { return (ZC_TILE / ZC_SUB) * zc_sub_bytes(bits); }
+// kch: keys quantised channelwise, the parameter block is [(sV, zV) x 16].
+__host__ __device__ inline int zc_sub_bytes(int bits, int kch) { return ZC_SUB * (32 * bits + (kch ? 8 : 16)); }
+__host__ __device__ inline int zc_tile_bytes(int bits, int kch) { return (ZC_TILE / ZC_SUB) * zc_sub_bytes(bits, kch); }
 __host__ __device__ inline int zc_sub_off_vcodes(int bits) { return 256 * bits; }
 __host__ __device__ inline int zc_sub_off_par(int bits) { return 512 * bits; }
 
@@ -52,6 +53,16 @@ template <typename T> __device__ inline void zc_load4(const T* p, float* out) {
   const T* e = reinterpret_cast<const T*>(&raw);
   out[0] = zc_to_float<T>(e[0]); out[1] = zc_to_float<T>(e[1]);
   out[2] = zc_to_float<T>(e[2]); out[3] = zc_to_float<T>(e[3]);
+}
+
+// Order-preserving map of floats onto unsigned keys (and back), for minima and maxima by
+// integer atomics: key(a) < key(b) exactly when a < b.
+__device__ inline unsigned zc_float_key(float x) {
+  const unsigned b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ inline float zc_key_float(unsigned k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
 __device__ inline char* zc_unit_base(char* base, const ZcLayout& lay, int unit) {

@@ -36,13 +36,37 @@ static __device__ __forceinline__ void quant_token(const float (&x)[4], const fl
   *codes4 = packed;
 }
 
+// ChannelQuant (Eq. 5 per channel, Sec. 4.1) of one token's four channels, whose (s, z) the
+// caller holds: code = clamp(rint(x / s_i) + z_i, 0, L), each step one IEEE operation.
+static __device__ __forceinline__ unsigned quant_channel4(const float (&x)[4], const float (&s)[4],
+                                                          const float (&z)[4], float L) {
+  unsigned packed = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float q = __fadd_rn(rintf(__fdiv_rn(x[e], s[e])), z[e]);
+    q = fminf(fmaxf(q, 0.f), L);
+    packed |= ((unsigned)(int)q) << (8 * e);
+  }
+  return packed;
+}
+// Channel parameters from the channel's minimum and maximum over the subset (Eq. 5):
+// s = (mx - mn) / L, or |mn| (1 if 0) for a constant channel; z = -rint(mn / s).
+static __device__ __forceinline__ void channel_params(float mn, float mx, float L, float* s_out, float* z_out) {
+  float s = __fdiv_rn(__fsub_rn(mx, mn), L);
+  if (mx == mn) s = mn != 0.f ? fabsf(mn) : 1.f;
+  *s_out = s;
+  *z_out = -rintf(__fdiv_rn(mn, s));
+}
+
 // One 16-byte vector v of a cache tile from byte codes and per-token (s, z), the arrays holding
 // the tile's tokens from token row0 on: K codes in canonical order, V codes in fragment order, then the parameters, per
 // 16-token sub-block.
-static __device__ __forceinline__ uint4 compose_vec(int bits, int v, int row0, const unsigned char (*codesK)[ZC_D],
+// kch: channelwise keys, the parameter block holds (sV, zV) per token only.
+static __device__ __forceinline__ uint4 compose_vec(int bits, int kch, int v, int row0,
+                                             const unsigned char (*codesK)[ZC_D],
                                              const unsigned char (*codesV)[ZC_D], const float (*parK)[2],
                                              const float (*parV)[2]) {
-  const int sub_words = zc_sub_bytes(bits) / 4;
+  const int sub_words = zc_sub_bytes(bits, kch) / 4;
   const int kw = 64 * bits;                           // K-code words per sub-block (= V-code words)
   const int per = 32 / bits;                          // codes per word
   unsigned out[4];
@@ -77,9 +101,13 @@ static __device__ __forceinline__ uint4 compose_vec(int bits, int v, int row0, c
         }
       }
     } else {
-      const int wp = wl - 2 * kw;  // params: (sK, zK, sV, zV) per token
-      const int tk = 16 * st - row0 + (wp >> 2), f = wp & 3;
-      word = __float_as_uint(f < 2 ? parK[tk][f] : parV[tk][f - 2]);
+      const int wp = wl - 2 * kw;  // params: (sK, zK, sV, zV) per token, or (sV, zV)
+      if (kch) {
+        word = __float_as_uint(parV[16 * st - row0 + (wp >> 1)][wp & 1]);
+      } else {
+        const int tk = 16 * st - row0 + (wp >> 2), f = wp & 3;
+        word = __float_as_uint(f < 2 ? parK[tk][f] : parV[tk][f - 2]);
+      }
     }
     out[q] = word;
   }

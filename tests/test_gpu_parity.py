@@ -379,3 +379,79 @@ def test_prefill_accepts_token_major_inputs(dtype):
     assert tl.compare_segment(results[1][2], oc, 0) == 0
     import paper_2405_14256_b200 as zc
     assert zc.zc_device_status() == 0
+
+
+# ------------------------------------------------------------------ channelwise keys (ZC_K_CHANNEL)
+@pytest.mark.parametrize("l", [1, 17, 100, 513])
+@pytest.mark.parametrize("ratio", [0.0, 0.4, 1.0])
+def test_channelwise_keys_codes_bit_exact(l, ratio):
+    """Keys by ChannelQuant (Sec. 4.1, Alg. 2), values by CSTQuant: K codes and the per-channel
+    (s, z), V codes, per-token (s, z) and channel factors equal the oracle's bit for bit."""
+    _staged_quant_case(tl.small_workload(context=l, saliency_ratio=ratio, n_q_heads=2, n_kv_heads=2,
+                                         rho_recent=0.2, rho_random=0.2, k_scheme="channel"))
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", [(4, 2), (4, 4), (2, 2)])
+def test_channelwise_keys_bit_pairs(dtype, bits):
+    _staged_quant_case(tl.small_workload(dtype=dtype, context=333, batch=2, n_q_heads=8, n_kv_heads=2,
+                                         bits_hi=bits[0], bits_lo=bits[1], outlier_fixed=0,
+                                         k_scheme="channel"))
+
+
+def test_channelwise_keys_with_an_offset_channel():
+    """A key channel that lies far from zero gets a large negative zero point: codes must
+    still be the oracle's and decode attention must stay within tolerance."""
+    w = tl.small_workload(context=300, n_q_heads=4, n_kv_heads=2, k_scheme="channel")
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    K[:, :, :, 5] += 9.0
+    K[:, :, :, 77] -= 6.5
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w, max_new=4)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    assert tl.compare_segment(cache, oc, 0) == 0
+    from workloads import make_decode_step
+    for step in range(3):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        cache.append(k, v)
+        out = tl.to64(cache.decode_attention(q, False))
+        oc.append(tl.to64(k), tl.to64(v))
+        ref = oc.decode_attention(tl.to64(q), False)
+        for (bi, kv), o in ref.items():
+            assert tl.output_excess(out[bi, kv * w.group:(kv + 1) * w.group], o, w.torch_dtype) <= 0.0
+
+
+@pytest.mark.parametrize("kw,steps", [
+    (dict(context=512, n_q_heads=4, n_kv_heads=4), 16),
+    (dict(context=300, batch=2, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0), 6),
+    (dict(context=129, n_q_heads=2, n_kv_heads=2, saliency_ratio=0.0), 3),
+    (dict(context=200, n_q_heads=4, n_kv_heads=1, bits_hi=4, bits_lo=4), 3),
+    (dict(context=150, n_q_heads=4, n_kv_heads=2, window=16, rho_recent=0.1, rho_random=0.1), 40),
+    (dict(context=150, n_q_heads=16, n_kv_heads=2, window=100, rho_recent=0.1, rho_random=0.1), 105),
+])
+@pytest.mark.parametrize("defer", [False, True])
+def test_channelwise_keys_decode_and_windows(kw, steps, defer):
+    """Decode attention over channelwise-key caches, across re-compressed windows, with the
+    separate append launch and with the deferred append."""
+    w = tl.small_workload(k_scheme="channel", **kw)
+    worst, cache, oc = tl.run_decode_parity(w, steps, defer_append=defer)
+    import paper_2405_14256_b200 as zc
+    for seg in range(1, zc.zc_num_segments(cache.handle)):
+        assert tl.compare_segment(cache, oc, seg) == 0
+    assert zc.zc_device_status() == 0
+
+
+@pytest.mark.parametrize("cfg_id,units,steps", [
+    (2, [(0, 0), (5, 3)], 105), (3, [(11, 5)], 3), (4, [(17, 13), (31, 31)], 3), (5, [(2, 6)], 2),
+])
+def test_channelwise_keys_full_size_in_the_benchmark_configuration(cfg_id, units, steps):
+    w = get_config(cfg_id).scaled(k_scheme="channel")
+    r = tl.run_benchmark_mode(w, units, steps, layers=2)
+    assert r["excess"] <= 0.0, r
+    tl.record("full size, benchmark configuration, channelwise keys", config=cfg_id, units=2 * len(units),
+              steps=steps, max_abs_out=r["worst"], max_abs_out_vs_rounded_oracle=r["worst_rounded"],
+              near_tie_swaps=r["near_tie_swaps"], units_code_exact=r["units_code_exact"],
+              window_set_swaps=r["window_set_mismatches"])

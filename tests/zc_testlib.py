@@ -29,12 +29,12 @@ def make_cache(w: Workload, max_new=None, defer_append: bool = False, overlap_ca
     return zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context,
                        w.decode_steps if max_new is None else max_new, w.saliency_ratio,
                        w.bits_hi, w.bits_lo, w.window, device=DEV, defer_append=defer_append,
-                       overlap_calls=overlap_calls)
+                       overlap_calls=overlap_calls, k_channel=w.k_scheme == "channel")
 
 
 def make_oracle(w: Workload, units=None) -> zo.ZipCacheOracle:
     return zo.ZipCacheOracle(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.saliency_ratio,
-                             w.bits_hi, w.bits_lo, w.window, units=units)
+                             w.bits_hi, w.bits_lo, w.window, units=units, k_scheme=w.k_scheme)
 
 
 def probes_for(w: Workload, layer: int = 0) -> np.ndarray:
@@ -57,9 +57,11 @@ def compare_segment(cache, oc: zo.ZipCacheOracle, seg: int, units=None):
                 want = zo.pack_codes(q["codes"], sub.bits)
                 mism += int((codes[bi, kv] != want).sum())
                 np.testing.assert_array_equal(codes[bi, kv], want)
+                # per token (CSTQuant) or per channel (channelwise keys): same export slots
                 np.testing.assert_array_equal(sz[bi, kv, :, 0], q["s"])
                 np.testing.assert_array_equal(sz[bi, kv, :, 1], q["z"])
-                np.testing.assert_array_equal(cf[bi, kv], q["c"])
+                if "c" in q:
+                    np.testing.assert_array_equal(cf[bi, kv], q["c"])
     return mism
 
 
@@ -233,7 +235,8 @@ def run_benchmark_mode(w: Workload, units, n_steps: int, layers: int = 2, graph:
         oc.prefill_compress(*oracle_inputs(w, Q, K, V, units), P)
         c = zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context, max(n_steps, 1),
                         w.saliency_ratio, w.bits_hi, w.bits_lo, w.window, device=DEV, workspace=ws,
-                        defer_append=defer_append, overlap_calls=overlap_calls)
+                        defer_append=defer_append, overlap_calls=overlap_calls,
+                        k_channel=w.k_scheme == "channel")
         ws = c.workspace
         c.prefill_compress(Q, K, V, P.tolist())
         torch.cuda.synchronize()

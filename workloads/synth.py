@@ -39,6 +39,7 @@ class Workload:
     decode_steps: int
     outlier_fixed: int    # >0: exactly this many outlier channels, x15
     band: int             # number of extra heavy columns (0 = none)
+    k_scheme: str = "cst"  # "cst": CSTQuant for keys and values; "channel": channelwise keys
 
     @property
     def torch_dtype(self) -> torch.dtype:
