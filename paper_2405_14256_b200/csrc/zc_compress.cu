@@ -161,6 +161,7 @@ __global__ void __launch_bounds__(256) k_channel_absmax(char* cache, ZcLayout la
   const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
   const int groups_c0 = zc_ceil_div(zc_ceil_div(seg.n_tok[0], ZC_TILE), kAbsTiles);
   const int cls = (int)blockIdx.x < groups_c0 ? 0 : 1;
+  if (lay.bits[cls] == 16) return;   // tokens kept as they are: no factors
   const int grp = cls == 0 ? blockIdx.x : blockIdx.x - groups_c0;
   char* ub = zc_unit_base(cache, lay, unit);
   const int32_t* idx = reinterpret_cast<const int32_t*>(ub + lay.off_idx) + seg.idx_off +
@@ -235,6 +236,24 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh;
   const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (bits == 16) {
+    // 16-bit "quantisation" (the 16/16 and 16/2 settings): the subset's rows are gathered into
+    // the tile as they are, [K rows][V rows] per 16-token sub-block; rows past the end are zero
+    char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
+    for (int i = 0; i < 8; ++i) {
+      const int tl = w * 8 + i, tt = tile * ZC_TILE + tl;
+      uint2 k = make_uint2(0, 0), v = make_uint2(0, 0);
+      if (tt < seg.n_tok[cls]) {
+        const long long row = (long long)idx[tt] * src.sl;
+        k = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
+        v = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
+      }
+      char* sub = tile_ptr + (tl / ZC_SUB) * zc_sub_bytes(16, 0) + (tl % ZC_SUB) * ZC_D * 2;
+      reinterpret_cast<uint2*>(sub)[lane] = k;
+      reinterpret_cast<uint2*>(sub + ZC_SUB * ZC_D * 2)[lane] = v;
+    }
+    return;
+  }
   const unsigned* cmax = reinterpret_cast<const unsigned*>(ub + lay.off_cmax) + cls * 3 * ZC_D;
   float* fac = reinterpret_cast<float*>(ub + lay.off_fac) + (seg.run0 + cls) * ZC_FAC_FLOATS;
   const bool kch = lay.kch != 0;

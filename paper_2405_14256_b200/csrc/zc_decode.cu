@@ -770,6 +770,151 @@ __device__ __forceinline__ void tail_tile(const T* tK, const T* tV, int n_tail, 
   }
 }
 
+// One item of a class kept at 16 bits (the "16/16" and "16/2" settings): its tokens sit in the
+// cache as rows of the input type, [K rows 16 x 128][V rows 16 x 128] per sub-tile, and are
+// attended like the tail -- on tensor cores in the input type, q exact, probabilities as
+// hi + lo -- but with one running (maximum, sum, accumulator) per warp over all its sub-tiles.
+// On return every warp has put its (m, l) and accumulators where compressed_item puts them;
+// the merge then takes them with unit scales.
+template <typename T>
+__device__ __noinline__ ItemScale raw_item(ItemDesc d, const char* class_base, const T* qbase, int Gl,
+                                           char* smem, int ring_bytes) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+  float* wm = reinterpret_cast<float*>(smem + kOffWm);
+  float* wl = reinterpret_cast<float*>(smem + kOffWl);
+  float* wz = reinterpret_cast<float*>(smem + kOffWz);
+  uint4 qv[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+    qv[c] = g < Gl ? *reinterpret_cast<const uint4*>(qbase + g * ZC_D + 32 * c + 8 * t) : make_uint4(0, 0, 0, 0);
+  const float scale = kLog2e * rsqrtf((float)ZC_D);
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+  float oacc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) oacc[i][0] = oacc[i][1] = oacc[i][2] = oacc[i][3] = 0.f;
+  const int hh = g & 3, srcA = 8 * t + (hh >> 1), srcB = srcA + 4;
+  const int corr_src = (lane & ~3) | (t & 1);   // the lane that holds the heads of this lane's columns
+  for (int s = d.sub_lo + warp; s < d.sub_hi; s += kWarps) {
+    const T* tK = reinterpret_cast<const T*>(class_base + (long long)s * (ZC_SUB * 2 * ZC_D * 2));
+    const T* tV = tK + ZC_SUB * ZC_D;
+    const int nv = min(ZC_SUB, d.n_tok - (s - d.run_sub0) * ZC_SUB);
+    const int last = nv - 1;
+    const int r0 = min(g, last), r1 = min(g + 8, last);
+    uint4 ka[4], kb[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      ka[c] = __ldcg(reinterpret_cast<const uint4*>(tK + r0 * ZC_D + 32 * c + 8 * t));
+      kb[c] = __ldcg(reinterpret_cast<const uint4*>(tK + r1 * ZC_D + 32 * c + 8 * t));
+    }
+    const T* vap = tV + min(2 * t, last) * ZC_D;
+    const T* vbp = tV + min(2 * t + 8, last) * ZC_D;
+    const T* vcp = tV + min(2 * t + 1, last) * ZC_D;
+    const T* vdp = tV + min(2 * t + 9, last) * ZC_D;
+    uint4 va[2], vb[2], vc[2], vd[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      va[u] = __ldcg(reinterpret_cast<const uint4*>(vap + 16 * g + 8 * u));
+      vb[u] = __ldcg(reinterpret_cast<const uint4*>(vbp + 16 * g + 8 * u));
+      vc[u] = __ldcg(reinterpret_cast<const uint4*>(vcp + 16 * g + 8 * u));
+      vd[u] = __ldcg(reinterpret_cast<const uint4*>(vdp + 16 * g + 8 * u));
+    }
+    float dacc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint32_t a0[4] = {ka[c].x, kb[c].x, ka[c].y, kb[c].y};
+      zc_mma16816<T>(dacc, a0, qv[c].x, qv[c].y);
+      const uint32_t a1[4] = {ka[c].z, kb[c].z, ka[c].w, kb[c].w};
+      zc_mma16816<T>(dacc, a1, qv[c].z, qv[c].w);
+    }
+    const bool v0 = g < nv, v1 = g + 8 < nv;
+    float lg[2][2];   // [token slot][head 2t + e]
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      lg[0][e] = v0 ? dacc[e] * scale : -INFINITY;
+      lg[1][e] = v1 ? dacc[2 + e] * scale : -INFINITY;
+    }
+    float mx[2] = {fmaxf(lg[0][0], lg[1][0]), fmaxf(lg[0][1], lg[1][1])};
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+      mx[0] = fmaxf(mx[0], __shfl_xor_sync(kFull, mx[0], o));
+      mx[1] = fmaxf(mx[1], __shfl_xor_sync(kFull, mx[1], o));
+    }
+    float corr[2];
+    uint32_t Xhi[2], Xlo[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const float mn = fmaxf(m[e], mx[e]);            // finite: token 0 of the sub-tile is valid
+      corr[e] = m[e] == -INFINITY ? 0.f : zc_exp2(m[e] - mn);
+      m[e] = mn;
+      const float pa = zc_exp2(lg[0][e] - mn), pb = zc_exp2(lg[1][e] - mn);
+      l[e] = l[e] * corr[e] + pa + pb;
+      const T ha = zc_from_float<T>(pa), hb = zc_from_float<T>(pb);
+      const T la = zc_from_float<T>(pa - zc_to_float<T>(ha)), lb = zc_from_float<T>(pb - zc_to_float<T>(hb));
+      Xhi[e] = (uint32_t)(*reinterpret_cast<const unsigned short*>(&ha)) |
+               ((uint32_t)(*reinterpret_cast<const unsigned short*>(&hb)) << 16);
+      Xlo[e] = (uint32_t)(*reinterpret_cast<const unsigned short*>(&la)) |
+               ((uint32_t)(*reinterpret_cast<const unsigned short*>(&lb)) << 16);
+    }
+    // this lane's accumulator columns 2t, 2t+1 belong to heads (2t) & 3, (2t+1) & 3
+    const float c0 = __shfl_sync(kFull, corr[0], corr_src), c1 = __shfl_sync(kFull, corr[1], corr_src);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      oacc[i][0] *= c0; oacc[i][1] *= c1; oacc[i][2] *= c0; oacc[i][3] *= c1;
+    }
+    uint32_t pb0, pb1;
+    {
+      const uint32_t a_h0 = __shfl_sync(kFull, Xhi[0], srcA), a_h1 = __shfl_sync(kFull, Xhi[1], srcA);
+      const uint32_t a_l0 = __shfl_sync(kFull, Xlo[0], srcA), a_l1 = __shfl_sync(kFull, Xlo[1], srcA);
+      const uint32_t b_h0 = __shfl_sync(kFull, Xhi[0], srcB), b_h1 = __shfl_sync(kFull, Xhi[1], srcB);
+      const uint32_t b_l0 = __shfl_sync(kFull, Xlo[0], srcB), b_l1 = __shfl_sync(kFull, Xlo[1], srcB);
+      const bool lo_part = g >= 4, second = hh & 1;
+      pb0 = lo_part ? (second ? a_l1 : a_l0) : (second ? a_h1 : a_h0);
+      pb1 = lo_part ? (second ? b_l1 : b_l0) : (second ? b_h1 : b_h0);
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t ra = (&va[i >> 2].x)[i & 3], rb = (&vb[i >> 2].x)[i & 3];
+      const uint32_t rc = (&vc[i >> 2].x)[i & 3], rd = (&vd[i >> 2].x)[i & 3];
+      const uint32_t a[4] = {prmt(ra, rb, 0x5410u), prmt(ra, rb, 0x7632u), prmt(rc, rd, 0x5410u),
+                             prmt(rc, rd, 0x7632u)};
+      zc_mma16816<T>(oacc[i], a, pb0, pb1);
+    }
+  }
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) {
+    l[0] += __shfl_xor_sync(kFull, l[0], o);
+    l[1] += __shfl_xor_sync(kFull, l[1], o);
+  }
+  // columns 4..7 (lanes t >= 2) hold the lo-part products of heads 0..3
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) oacc[i][e] += __shfl_xor_sync(kFull, oacc[i][e], 2);
+  if (g == 0 && t < 2) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      wm[warp * 4 + 2 * t + e] = m[e];
+      wl[warp * 4 + 2 * t + e] = l[e];
+      wz[warp * 4 + 2 * t + e] = 0.f;
+    }
+  }
+  float* mbuf = reinterpret_cast<float*>(smem + kOffRing + warp * ring_bytes);   // [4 heads][128]
+  if (t < 2) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e)
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        // M-tile i: rows g <-> channel 16g + 2i, g + 8 <-> channel 16g + 2i + 1
+        mbuf[(2 * t + e) * ZC_D + 16 * g + 2 * i] = oacc[i][e];
+        mbuf[(2 * t + e) * ZC_D + 16 * g + 2 * i + 1] = oacc[i][2 + e];
+      }
+  }
+  ItemScale r;
+  r.chan_factor = 1.f;
+  r.rowscale = 1.f;
+  return r;
+}
+
 // shared-memory map of the merge phase (it reuses the memory of the item phase, but not the
 // mbarriers': memory that holds mbarrier objects is never reused as data -- plain stores
 // over a used barrier were observed to be replaced by barrier state)
@@ -823,7 +968,7 @@ constexpr int kFlushSmem = kFlOffSmax + 16;
 static_assert(kFlushSmem <= decode_smem(kRingNarrow), "the re-compression must fit the item phase's memory");
 static_assert(ZC_MAX_WINDOW == 32 * kWarps, "one thread per window token");
 
-template <typename T, bool KCH>
+template <typename T, bool KCH, bool RAW>
 __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay, const ZcFlushArgs& fl, char* smem) {
   auto codesK = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesK);
   auto codesV = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesV);
@@ -889,8 +1034,25 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
   for (int cls = 0; cls < 2; ++cls) {
     const int n_c = fl.seg.n_tok[cls];
     if (n_c == 0) continue;
-    // ---- channel |x| maxima over the class (Eq. 6); channelwise keys: their signed min and max ----
     const int bits = lay.bits[cls];
+    if (RAW && bits == 16) {
+      // a class kept at 16 bits: its rows are gathered into the new tiles as they are
+      const int subs16 = (n_c + ZC_SUB - 1) / ZC_SUB;
+      for (int r = w; r < subs16 * ZC_SUB; r += kWarps) {
+        uint2 k = make_uint2(0, 0), v = make_uint2(0, 0);
+        if (r < n_c) {
+          const int row = s_tok[cls][r] * ZC_D;
+          k = *reinterpret_cast<const uint2*>(tK + row + 4 * lane);
+          v = *reinterpret_cast<const uint2*>(tV + row + 4 * lane);
+        }
+        char* sub = ub + lay.off_tiles[cls] + (long long)fl.seg.tile0[cls] * lay.tile_bytes[cls] +
+                    (long long)(r / ZC_SUB) * zc_sub_bytes(16, 0) + (r % ZC_SUB) * ZC_D * 2;
+        reinterpret_cast<uint2*>(sub)[lane] = k;
+        reinterpret_cast<uint2*>(sub + ZC_SUB * ZC_D * 2)[lane] = v;
+      }
+      continue;
+    }
+    // ---- channel |x| maxima over the class (Eq. 6); channelwise keys: their signed min and max ----
     const float L = (float)((1 << bits) - 1);
     {
       const float k0 = kch ? -INFINITY : 0.f;
@@ -1106,7 +1268,9 @@ __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_t
 // share is kept apart by the host: each call of an epoch (the launches between two launches
 // made without early start) gets its own `slot`, which selects its region of the workspace
 // and its arrival counter.
-template <typename T, int RING, int NCTA, bool KCH>
+// RAW: the build that also serves a class kept at 16 bits (kept apart so that the 4- and 2-bit
+// kernels are compiled exactly as they are without it).
+template <typename T, int RING, int NCTA, bool KCH, bool RAW>
 __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay, ZcDecodePlan plan,
                                                       const T* __restrict__ q, T* __restrict__ out,
                                                       float* part, float* stash_all, int slot,
@@ -1209,8 +1373,10 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
       const char* class_base = ub + lay.off_tiles[d.cls];
       if (lay.bits[d.cls] == 4)
         sc = compressed_item<T, 4, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
-      else
+      else if (!RAW || lay.bits[d.cls] == 2)
         sc = compressed_item<T, 2, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
+      else
+        sc = raw_item<T>(d, class_base, qbase, Gl, smem, RING);
     }
     __syncthreads();
     // ---- merge the warps: one thread per head fixes the weights, then thread = channel ----
@@ -1274,7 +1440,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
                   lay.out_f32 ? reinterpret_cast<float*>(out) + out_off : nullptr, mine, stash_g, collect, smem);
     if (fl.on) {
       __syncthreads();   // the merge is done with the shared arrays; its additions to the statistics are visible
-      window_flush_unit<T, KCH>(ub, lay, fl, smem);
+      window_flush_unit<T, KCH, RAW>(ub, lay, fl, smem);
     }
   }
 }
@@ -1416,7 +1582,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   const int groups = (plan.items + plan.cta_items - 1) / plan.cta_items;
   const dim3 grid((unsigned)(c->lay.units * (groups * zs + (plan.fold_tail ? 0 : 1)) + 1));
   cudaError_t e;
-#define ZC_LAUNCH_STEP(T, RING, NCTA, KCH)                                                         \
+#define ZC_LAUNCH_STEP(T, RING, NCTA, KCH, RAW)                                                        \
   do {                                                                                             \
     /* the opt-in to large shared memory is per device and per kernel: one bit per device */       \
     static std::atomic<unsigned long long> attr_done{0};                                           \
@@ -1424,23 +1590,28 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
     cudaGetDevice(&dev_now);                                                                       \
     const unsigned long long bit = 1ull << (dev_now & 63);                                         \
     if (!(attr_done.load(std::memory_order_acquire) & bit)) {                                      \
-      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA, KCH>,                                       \
+      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA, KCH, RAW>,                                  \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));    \
       if (e != cudaSuccess) return e;                                                              \
       attr_done.fetch_or(bit, std::memory_order_release);                                          \
     }                                                                                              \
-    e = launch_pdl(k_decode<T, RING, NCTA, KCH>, grid, dim3(128), decode_smem(RING), st, overlap,  \
+    e = launch_pdl(k_decode<T, RING, NCTA, KCH, RAW>, grid, dim3(128), decode_smem(RING), st,      \
+                   overlap,                                                                        \
                    c->base, c->lay, plan, (const T*)q, (T*)out, part, stash, slot, collect,        \
                    (const T*)k_new, (const T*)v_new, ord, fl);                                     \
   } while (0)
 #define ZC_LAUNCH_T(T)                                                                             \
   do {                                                                                             \
-    if (c->lay.kch) {                                                                              \
-      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true);                          \
-      else ZC_LAUNCH_STEP(T, kRingWide, 3, true);                                                  \
+    const bool raw = c->lay.bits[0] == 16 || c->lay.bits[1] == 16;                                 \
+    if (raw) { /* a class kept at 16 bits: one build (narrow rings, 4 CTAs per SM) */              \
+      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, true);                               \
+      else ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, true);                                         \
+    } else if (c->lay.kch) {                                                                       \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, false);                   \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, true, false);                                           \
     } else {                                                                                       \
-      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false);                         \
-      else ZC_LAUNCH_STEP(T, kRingWide, 3, false);                                                 \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, false);                  \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false);                                          \
     }                                                                                              \
   } while (0)
   if (c->cfg.dtype == ZC_F16) ZC_LAUNCH_T(__half);

@@ -29,6 +29,18 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
       idx_out[(long long)unit * n + t0 + i] = idx[t0 + i];
   }
   const int kch = lay.kch;
+  if (bits == 16) {
+    // rows kept at full precision: "codes" are the rows' bytes, there are no parameters
+    if (codes_out) {
+      for (int i = threadIdx.x; i < n_here * 64; i += blockDim.x) {
+        const int tl = i >> 6, wd = i & 63;
+        const char* sb = tp + (tl / ZC_SUB) * zc_sub_bytes(16, 0) + (tensor ? ZC_SUB * ZC_D * 2 : 0);
+        reinterpret_cast<unsigned*>(codes_out + ((long long)unit * n + t0 + tl) * row_bytes)[wd] =
+            reinterpret_cast<const unsigned*>(sb + (tl % ZC_SUB) * ZC_D * 2)[wd];
+      }
+    }
+    return;
+  }
   if (sz_out && kch && tensor == 0) {
     // channelwise keys: (scale, zero point) of every channel, from the run's factor block
     if (tile == 0) {

@@ -25,8 +25,8 @@ int check_config(const zc_config* cfg) {
   if (cfg->max_prefill < 1 || cfg->max_prefill > (1 << 20)) return ZC_EINVAL;
   if (cfg->max_new_tokens < 0) return ZC_EINVAL;
   if (cfg->window < 8 || cfg->window > ZC_MAX_WINDOW) return ZC_EINVAL;
-  if (cfg->bits_hi != 4 && cfg->bits_hi != 2) return ZC_EINVAL;
-  if (cfg->bits_lo != 4 && cfg->bits_lo != 2) return ZC_EINVAL;
+  if (cfg->bits_hi != 4 && cfg->bits_hi != 2 && cfg->bits_hi != 16) return ZC_EINVAL;
+  if (cfg->bits_lo != 4 && cfg->bits_lo != 2 && cfg->bits_lo != 16) return ZC_EINVAL;
   if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32)) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if (cfg->k_scheme != ZC_K_CST && cfg->k_scheme != ZC_K_CHANNEL) return ZC_EINVAL;
@@ -496,11 +496,12 @@ int64_t zc_decode_bytes(const zc_cache* c) {
   if (!c || c->l0 < 0) return 0;
   int64_t per_unit = 0;
   for (int k = 0; k < 2; ++k) {
-    const int64_t per_tok = 32 * c->lay.bits[k] + (c->lay.kch ? 8 : 16);  // K+V codes, (s,z) pairs
+    const bool raw = c->lay.bits[k] == 16;   // tokens kept at full precision: rows only
+    const int64_t per_tok = raw ? 2 * ZC_D * 2 : 32 * c->lay.bits[k] + (c->lay.kch ? 8 : 16);  // K+V codes, (s,z) pairs
     const int64_t toks = (int64_t)c->n0[k] + (int64_t)(c->n_seg - 1) * c->nw[k];
     per_unit += toks * per_tok;
     const int runs = (c->n0[k] > 0 ? 1 : 0) + (c->nw[k] > 0 ? c->n_seg - 1 : 0);
-    per_unit += (int64_t)runs * (c->lay.kch ? 3 : 2) * ZC_D * 4;   // channel factors of V; of K, or its (s, z) per channel
+    if (!raw) per_unit += (int64_t)runs * (c->lay.kch ? 3 : 2) * ZC_D * 4;   // channel factors of V; of K, or its (s, z) per channel
   }
   per_unit += (int64_t)c->n_tail * 2 * ZC_D * 2;     // full-precision tail
   per_unit += (int64_t)c->lay.G * ZC_D * 2 * 2;      // q in, out

@@ -18,7 +18,10 @@
 // everything a warp needs for one MMA sub-tile:
 //   [K codes 16 rows x 16*bits B][V codes, fragment order][(sK, zK, sV, zV) x 16]
 // kch: keys quantised channelwise, the parameter block is [(sV, zV) x 16].
-__host__ __device__ inline int zc_sub_bytes(int bits, int kch) { return ZC_SUB * (32 * bits + (kch ? 8 : 16)); }
+// bits = 16: the tokens are kept as they came (no codes, no parameters): [K rows 16 x 256 B][V rows 16 x 256 B].
+__host__ __device__ inline int zc_sub_bytes(int bits, int kch) {
+  return bits == 16 ? ZC_SUB * 2 * ZC_D * 2 : ZC_SUB * (32 * bits + (kch ? 8 : 16));
+}
 __host__ __device__ inline int zc_tile_bytes(int bits, int kch) { return (ZC_TILE / ZC_SUB) * zc_sub_bytes(bits, kch); }
 __host__ __device__ inline int zc_sub_off_vcodes(int bits) { return 256 * bits; }
 __host__ __device__ inline int zc_sub_off_par(int bits) { return 512 * bits; }

@@ -455,3 +455,63 @@ def test_channelwise_keys_full_size_in_the_benchmark_configuration(cfg_id, units
               steps=steps, max_abs_out=r["worst"], max_abs_out_vs_rounded_oracle=r["worst_rounded"],
               near_tie_swaps=r["near_tie_swaps"], units_code_exact=r["units_code_exact"],
               window_set_swaps=r["window_set_mismatches"])
+
+
+# ------------------------------------------------------------------ 16-bit classes ("16/16", "16/2")
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("kw", [
+    dict(context=300, n_q_heads=4, n_kv_heads=2),
+    dict(context=777, batch=2, n_q_heads=8, n_kv_heads=2, outlier_fixed=0),
+    dict(context=1, n_q_heads=1, n_kv_heads=1),
+    dict(context=50, n_q_heads=16, n_kv_heads=2),
+])
+def test_every_token_salient_at_16_bits_is_exact_attention(dtype, kw):
+    """The pin the method's statement gives for the CUDA path: with every token salient and
+    salient tokens kept at 16 bits, decode attention IS Eq. 4 -- compared with the oracle's
+    library-free exact attention over the raw keys and values (fp32 output, 1e-4)."""
+    import paper_2405_14256_b200 as zc
+    from workloads import make_decode_step
+    w = tl.small_workload(dtype=dtype, saliency_ratio=1.0, bits_hi=16, bits_lo=2, **kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    cache = zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context, 8, 1.0, 16, 2,
+                        w.window, device=tl.DEV, out_f32=True)
+    cache.prefill_compress(Q, K, V, tl.probes_for(w).tolist())
+    K_all, V_all = tl.to64(K), tl.to64(V)
+    G = w.group
+    for step in range(3):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        cache.append(k, v)
+        out = cache.decode_attention(q, False).double().cpu().numpy()
+        K_all = np.concatenate([K_all, tl.to64(k)[:, :, None, :]], axis=2)
+        V_all = np.concatenate([V_all, tl.to64(v)[:, :, None, :]], axis=2)
+        q64 = tl.to64(q)
+        for bi in range(w.batch):
+            for kv in range(w.n_kv_heads):
+                ref = zo.exact_attention(q64[bi, kv * G:(kv + 1) * G], K_all[bi, kv], V_all[bi, kv])
+                assert np.abs(out[bi, kv * G:(kv + 1) * G] - ref).max() <= 1e-4
+    assert zc.zc_device_status() == 0
+
+
+@pytest.mark.parametrize("bits,ratio", [((16, 2), 0.15), ((16, 4), 0.5), ((4, 16), 0.4), ((16, 16), 0.3)])
+@pytest.mark.parametrize("defer", [False, True])
+def test_mixed_16_bit_and_quantised_classes(bits, ratio, defer):
+    """One class kept at 16 bits beside a quantised one (Table 3's "16/2" setting): rows,
+    codes and parameters bit-exact, decode within tolerance, across two re-compressed windows."""
+    w = tl.small_workload(context=333, batch=2, n_q_heads=8, n_kv_heads=2, bits_hi=bits[0], bits_lo=bits[1],
+                          saliency_ratio=ratio, window=16, rho_recent=0.1, rho_random=0.1)
+    worst, cache, oc = tl.run_decode_parity(w, 36, defer_append=defer)
+    import paper_2405_14256_b200 as zc
+    assert zc.zc_num_segments(cache.handle) == 3
+    for seg in range(zc.zc_num_segments(cache.handle)):
+        assert tl.compare_segment(cache, oc, seg) == 0
+    assert zc.zc_device_status() == 0
+
+
+def test_16_2_full_size_in_the_benchmark_configuration():
+    w = get_config(2).scaled(bits_hi=16, bits_lo=2, saliency_ratio=0.152)
+    r = tl.run_benchmark_mode(w, [(0, 0), (5, 3)], 105, layers=2)
+    assert r["excess"] <= 0.0, r
+    tl.record("full size, benchmark configuration, 16/2 bits at 15.2 % salient", config=2, units=4, steps=105,
+              max_abs_out=r["worst"], max_abs_out_vs_rounded_oracle=r["worst_rounded"],
+              near_tie_swaps=r["near_tie_swaps"], units_code_exact=r["units_code_exact"],
+              window_set_swaps=r["window_set_mismatches"])
