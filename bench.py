@@ -145,14 +145,19 @@ def profiled_traffic(cfg_id: int):
 
 def algorithmic_decode_bytes(w, n_windows: int, n_tail: int) -> int:
     """Bytes one decode-attention call must read for ALL units of one layer: packed K and V
-    codes, one (scale, zero) fp32 pair per token per tensor, the full-precision tail, the
-    channel factors of every (segment, class), q and the output."""
+    codes, one (scale, zero) fp32 pair per token per tensor quantised tokenwise, the
+    full-precision tail, the channel factors of every (segment, class), q and the output."""
     per_unit = 0
     n_s0 = int(math.floor(w.saliency_ratio * w.context))
     n_sw = int(math.floor(w.saliency_ratio * w.window))
+    kch = w.k_scheme == "channel"
     for bits, n0, nw in ((w.bits_hi, n_s0, n_sw), (w.bits_lo, w.context - n_s0, w.window - n_sw)):
-        per_unit += (n0 + n_windows * nw) * (32 * bits + 16)
-        per_unit += ((1 if n0 > 0 else 0) + (n_windows if nw > 0 else 0)) * 2 * 128 * 4
+        runs = (1 if n0 > 0 else 0) + (n_windows if nw > 0 else 0)
+        if bits == 16:                       # rows kept at full precision
+            per_unit += (n0 + n_windows * nw) * 512
+            continue
+        per_unit += (n0 + n_windows * nw) * (32 * bits + (8 if kch else 16))
+        per_unit += runs * (3 if kch else 2) * 128 * 4
     per_unit += n_tail * 2 * 128 * 2
     per_unit += w.group * 128 * 2 * 2
     return per_unit * w.units_per_layer
@@ -290,14 +295,14 @@ def oracle_prefill(w, n_units: int, layer: int = 0):
     del Q, K, V
     P = zo.probe_positions(w.context, w.rho_recent, w.rho_random, w.seed(layer))
     oc = zo.ZipCacheOracle(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.saliency_ratio,
-                           w.bits_hi, w.bits_lo, w.window, units=units)
+                           w.bits_hi, w.bits_lo, w.window, units=units, k_scheme=w.k_scheme)
     t0 = time.perf_counter()
     oc.prefill_compress(Qh, Kh, Vh, P)
     return oc, units, time.perf_counter() - t0
 
 
 # units and decode steps of the oracle sample per workload: about 10 to 30 s of CPU work
-ORACLE_SAMPLE = {1: (4, 16), 2: (64, 96), 3: (16, 32), 4: (64, 32), 5: (1, 16)}
+ORACLE_SAMPLE = {1: (4, 16), 2: (64, 96), 3: (16, 32), 4: (64, 32), 5: (4, 32)}
 
 
 def rank_layers(rank: int, layers_per_rank: int):
@@ -399,6 +404,8 @@ class Workbench:
             kw = dict(MODES[mode])
             if append == "kernel":
                 kw["defer_append"] = False
+            if w.k_scheme == "channel":
+                kw["k_channel"] = True
             self.caches[mode] = [self.make_cache(**kw) for _ in range(R)]
         with torch.cuda.stream(self.stream):
             for mode in modes:
@@ -450,9 +457,9 @@ class Workbench:
             ev[2].record(self.stream)
 
 
-def measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, modes, headline):
+def measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, modes, headline, **override):
     from workloads import get_config
-    w = get_config(cfg_id)
+    w = get_config(cfg_id).scaled(**override)
     R = layers_for(w, args.layers)
     n_dec = args.decode_steps or w.decode_steps
     wb = Workbench(zc, w, R, rank, dev, n_dec, modes, args.append)
@@ -603,6 +610,8 @@ def main():
     ap.add_argument("--append", default="deferred", choices=["deferred", "kernel"],
                     help="deferred: zc_append hands the new row to the next zc_decode_attention "
                          "(ZC_FLAG_DEFER_APPEND); kernel: zc_append copies with its own launch")
+    ap.add_argument("--bits", default="", help="H/L bit pair instead of the workload's 4/2 (2, 4 or 16 each)")
+    ap.add_argument("--saliency", type=float, default=-1.0, help="saliency ratio instead of the workload's")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -631,12 +640,28 @@ def main():
     head_mode = modes[0]
     per_config, head = {}, None
     e2e = None
+    override = {}
+    if args.bits:
+        override.update(bits_hi=int(args.bits.split("/")[0]), bits_lo=int(args.bits.split("/")[1]))
+    if args.saliency >= 0:
+        override.update(saliency_ratio=args.saliency)
     for cfg_id in configs:
         r = measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, modes,
-                           headline=cfg_id == head_cfg)
+                           headline=cfg_id == head_cfg, **override)
         if rank == 0 and world == 1:
             r["per_config"]["parity"] = parity_counters(zc, get_config(cfg_id), dev)
         per_config[str(cfg_id)] = r["per_config"]
+        if cfg_id == 2 and args.mode == "both" and not args.config:
+            # the other bit pairs of the paper's comparison grid (Table 3), on workload 2
+            pairs = {}
+            for name, ov in (("4/4 all salient", dict(bits_hi=4, bits_lo=4, saliency_ratio=1.0)),
+                             ("16/2 15.2% salient", dict(bits_hi=16, bits_lo=2, saliency_ratio=0.152)),
+                             ("2/2", dict(bits_hi=2, bits_lo=2))):
+                rr = measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, ["overlap"],
+                                    headline=False, **ov)["per_config"]
+                pairs[name] = {"us_per_call": rr["overlap"]["us_per_call"], "frac": rr["overlap"]["frac"],
+                               "gbs": rr["overlap"]["gbs"], "prefill_tokens_per_s": rr["prefill_tokens_per_s"]}
+            per_config[str(cfg_id)]["bit_pairs_overlap_mode"] = pairs
         if cfg_id == head_cfg:
             head = r
             if not args.no_e2e:

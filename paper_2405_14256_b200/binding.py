@@ -246,7 +246,8 @@ class ZipCache:
     def __init__(self, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
                  workspace: Optional[torch.Tensor] = None, defer_append: bool = False,
-                 overlap_calls: bool = False, out_f32: bool = False, k_channel: bool = False):
+                 overlap_calls: bool = False, out_f32: bool = False, k_channel: bool = False,
+                 guard_bytes: int = 0):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
@@ -260,12 +261,35 @@ class ZipCache:
         self.dtype, self.device = dtype, torch.device(device)
         self.batch, self.n_q_heads, self.n_kv_heads = batch, n_q_heads, n_kv_heads
         self.cache_bytes, self.workspace_bytes = zc_cache_bytes(self.cfg)
-        self.mem = torch.empty(self.cache_bytes, dtype=torch.uint8, device=self.device)
-        self.workspace = workspace if workspace is not None else torch.empty(
-            self.workspace_bytes, dtype=torch.uint8, device=self.device)
+        # guard_bytes > 0 (a multiple of 256): the cache buffer and a workspace allocated here sit
+        # between two bands filled with 0xA5, which check_guards() verifies (a debugging aid:
+        # a kernel that writes outside its buffers shows up there)
+        self.guard_bytes = int(guard_bytes)
+        g = self.guard_bytes
+        self._mem_all = torch.full((self.cache_bytes + 2 * g,), 0xA5, dtype=torch.uint8, device=self.device) \
+            if g else torch.empty(self.cache_bytes, dtype=torch.uint8, device=self.device)
+        self.mem = self._mem_all[g:g + self.cache_bytes]
+        self._ws_all = None
+        if workspace is None:
+            self._ws_all = torch.full((self.workspace_bytes + 2 * g,), 0xA5, dtype=torch.uint8, device=self.device) \
+                if g else torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+            workspace = self._ws_all[g:g + self.workspace_bytes]
+        self.workspace = workspace
         if self.workspace.numel() * self.workspace.element_size() < self.workspace_bytes:
             raise ZipCacheError("shared workspace too small")
         self.handle = zc_cache_init(self.mem, self.cache_bytes, self.cfg)
+
+    def check_guards(self) -> bool:
+        """True when the guard bands around the cache buffer (and the workspace, if this object
+        allocated it) still hold their fill pattern."""
+        g = self.guard_bytes
+        if not g:
+            return True
+        ok = True
+        for buf in (self._mem_all, self._ws_all):
+            if buf is not None:
+                ok = ok and bool((buf[:g] == 0xA5).all()) and bool((buf[-g:] == 0xA5).all())
+        return ok
 
     def close(self):
         if getattr(self, "handle", None):

@@ -13,7 +13,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzipcache.so")
 SOURCES = ["zc_host.cu", "zc_scores.cu", "zc_compress.cu", "zc_decode.cu", "zc_order.cu",
            "zc_export.cu"]
-HEADERS = ["zc_internal.h", "zc_layout.cuh", "zc_mma.cuh", "zc_order.h"]
+HEADERS = ["zc_internal.h", "zc_layout.cuh", "zc_mma.cuh", "zc_order.h", "zc_quant.cuh"]
 
 
 def _nvcc() -> str:

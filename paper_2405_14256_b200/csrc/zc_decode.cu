@@ -1496,21 +1496,33 @@ size_t zc_decode_scratch_bytes(const zc_cache* c, int items) {
 // captured graph never disturbs the word of the calls issued directly.
 static __device__ unsigned g_zc_order_words[2 * kZcStreamRecs];
 
-int zc_order_words(unsigned** ptr) {
+// Per-device address of a symbol of the library image, looked up once per device; several
+// host threads may ask at the same time (the table is guarded by a mutex).
+template <typename Sym>
+static int symbol_address(const Sym& sym, void** table, std::mutex& guard, void** out) {
   constexpr int kMaxDev = 64;
-  static unsigned* addr[kMaxDev] = {nullptr};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return (int)e;
   if (dev < 0 || dev >= kMaxDev) return (int)cudaErrorInvalidDevice;
-  if (!addr[dev]) {
+  std::lock_guard<std::mutex> lock(guard);
+  if (!table[dev]) {
     void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_zc_order_words);
+    e = cudaGetSymbolAddress(&p, sym);
     if (e != cudaSuccess) return (int)e;
-    addr[dev] = (unsigned*)p;
+    table[dev] = p;
   }
-  if (ptr) *ptr = addr[dev];
+  if (out) *out = table[dev];
   return (int)cudaSuccess;
+}
+
+int zc_order_words(unsigned** ptr) {
+  static void* addr[64] = {nullptr};
+  static std::mutex guard;
+  void* p = nullptr;
+  const int rc = symbol_address(g_zc_order_words, addr, guard, &p);
+  if (rc == (int)cudaSuccess && ptr) *ptr = (unsigned*)p;
+  return rc;
 }
 
 int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void* out, int collect,
@@ -1628,20 +1640,9 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
 static __device__ __align__(256) unsigned char g_zc_noalloc_scratch[ZC_NOALLOC_SCRATCH_BYTES];
 
 int zc_static_scratch(void** ptr) {
-  constexpr int kMaxDev = 64;
-  static void* addr[kMaxDev] = {nullptr};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return (int)e;
-  if (dev < 0 || dev >= kMaxDev) return (int)cudaErrorInvalidDevice;
-  if (!addr[dev]) {
-    void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_zc_noalloc_scratch);
-    if (e != cudaSuccess) return (int)e;
-    addr[dev] = p;
-  }
-  *ptr = addr[dev];
-  return (int)cudaSuccess;
+  static void* addr[64] = {nullptr};
+  static std::mutex guard;
+  return symbol_address(g_zc_noalloc_scratch, addr, guard, ptr);
 }
 
 int zc_device_error_code(int* out) {

@@ -276,6 +276,7 @@ int zc_cache_init(void* dev_mem, size_t bytes, const zc_config* cfg, zc_cache** 
   c->n_sm = n_sm > 0 ? n_sm : 148;
   // the address look-ups the decode launches need are done here, outside any stream capture
   if (zc_order_words(nullptr) != (int)cudaSuccess) cudaGetLastError();
+  if (zc_static_scratch(nullptr) != (int)cudaSuccess) cudaGetLastError();
   *out = c;
   return ZC_OK;
 }
@@ -356,6 +357,7 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
   c->n_seg = 1;
   c->n_tail = 0;
   c->step_i = 0;
+  c->fresh = 0;
   c->n_new = 0;
   memset(c->tail_nnz, 0, sizeof(c->tail_nnz));
   c->last_scores_n = l;
@@ -396,6 +398,7 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
   }
   c->n_tail += 1;
   c->n_new += 1;
+  c->fresh = 1;
   return ZC_OK;
 }
 
@@ -413,14 +416,19 @@ static int decode_attention(zc_cache* c, const void* q, void* out, int is_probe_
     if (rc) return rc;
   }
   ZcDecodePlan plan = zc_make_plan(c);
+  // Alg. 3 counts one step per generated token: a call that follows an append takes the step
+  // (probe-row collection, the window's completion); a further call on the same tail (a
+  // re-query) attends the cache as it is and leaves the window's bookkeeping alone.
+  const bool fresh = c->fresh != 0;
+  c->fresh = 0;
   const int i_next = c->step_i + 1;
   const int collect =
-      (c->n_tail > 0) && (is_probe_step || i_next > c->cfg.window - 5) ? 1 : 0;
+      fresh && (c->n_tail > 0) && (is_probe_step || i_next > c->cfg.window - 5) ? 1 : 0;
   const void* pk = c->pend_k;
   const void* pv = c->pend_v;
   c->pend_k = c->pend_v = nullptr;
   // Alg. 3: the call that completes the window also re-compresses it (inside its kernel)
-  const bool completes = c->n_tail > 0 && i_next == c->cfg.window && c->n_tail == c->cfg.window;
+  const bool completes = fresh && c->n_tail == c->cfg.window;
   ZcFlushArgs fl;
   memset(&fl, 0, sizeof(fl));
   if (completes) {
@@ -431,7 +439,7 @@ static int decode_attention(zc_cache* c, const void* q, void* out, int is_probe_
   ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (char*)workspace, workspace_bytes, pk, pv,
                            completes ? &fl : nullptr, st));
   // Alg. 3 bookkeeping: the step counter follows the tokens of the current window
-  if (c->n_tail > 0) {
+  if (fresh && c->n_tail > 0) {
     c->step_i = i_next;
     if (collect)
       for (int j = 0; j < c->n_tail; ++j) c->tail_nnz[j] += 1;

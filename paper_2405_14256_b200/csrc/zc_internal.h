@@ -17,15 +17,9 @@
 #define ZC_MAX_SPLIT_HOST 32      // most items one class of segment 0 is split into
 #define ZC_MAX_ITEMS 128          // most items of one unit in one decode call
 #define ZC_EPOCH_CALLS 64          // most decode calls in flight together on a stream (arrival counters per unit)
-#ifndef ZC_ITEM_OVERHEAD
 #define ZC_ITEM_OVERHEAD 24       // fixed cost of one split-K item, in 16-token sub-tiles of streaming
-#endif
-#ifndef ZC_WAVE_SLACK
 #define ZC_WAVE_SLACK 0.0         // share of a wave that may spill over without counting as one more
-#endif
-#ifndef ZC_MANY_WAVES
-#define ZC_MANY_WAVES 1.2          // from this many waves of 4-per-SM CTAs on, the narrow build is used
-#endif    // CTAs the decode kernel keeps resident per SM
+#define ZC_MANY_WAVES 1.2         // from this many waves of 4-per-SM CTAs on, the narrow build is used
 
 // Device-side description of the cache buffer.  One "unit" = (batch, KV head).
 // Per unit, at byte offsets from base + unit * unit_stride:
@@ -117,6 +111,7 @@ struct zc_cache {
   int n_seg;       // 1 + number of re-compressed windows
   int n_tail;
   int step_i;      // decode steps taken in the current window
+  int fresh;       // a token was appended since the last decode call (that call takes a step of Alg. 3)
   int n_new;       // tokens appended since prefill
   int tail_nnz[ZC_MAX_WINDOW];
   int last_scores_n;

@@ -515,3 +515,102 @@ def test_16_2_full_size_in_the_benchmark_configuration():
               max_abs_out=r["worst"], max_abs_out_vs_rounded_oracle=r["worst_rounded"],
               near_tie_swaps=r["near_tie_swaps"], units_code_exact=r["units_code_exact"],
               window_set_swaps=r["window_set_mismatches"])
+
+
+# ------------------------------------------------------------------ properties that hold at any size
+def test_decode_is_invariant_under_a_permutation_of_the_cached_tokens():
+    """Attention is order-free: the prompt's tokens permuted (with the salient list mapped
+    along) give the same codes per token and the same decode output up to the kernel's own
+    arithmetic noise (fp32 output, 2e-4: the order decides where the running maximum is
+    refreshed and so how each weight is scaled before its hi + lo split)."""
+    import paper_2405_14256_b200 as zc
+    from workloads import make_decode_step
+    w = tl.small_workload(context=700, batch=2, n_q_heads=8, n_kv_heads=2, dtype="bf16")
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    n_s = zo.salient_count(w.saliency_ratio, w.context)
+    g = torch.Generator(device="cpu").manual_seed(5)
+    sal = torch.stack([torch.stack([torch.randperm(w.context, generator=g)[:n_s].sort().values
+                                    for _ in range(w.n_kv_heads)]) for _ in range(w.batch)]).to(torch.int32)
+    perm = torch.randperm(w.context, generator=g)
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(w.context)
+    outs = []
+    for permuted in (False, True):
+        c = tl.make_cache(w, max_new=4, out_f32=True)
+        if permuted:   # token j of the permuted prompt is token perm[j] of the original
+            Kp, Vp = K[:, :, perm.to(tl.DEV)].contiguous(), V[:, :, perm.to(tl.DEV)].contiguous()
+            salp = inv[sal.long()].sort(dim=2).values.to(torch.int32)
+            c.prefill_compress(None, Kp, Vp, None, salient_idx=salp.to(tl.DEV))
+        else:
+            c.prefill_compress(None, K, V, None, salient_idx=sal.to(tl.DEV))
+        q, k, v = make_decode_step(w, 0, 0, tl.DEV)
+        c.append(k, v)
+        outs.append(c.decode_attention(q, False).clone())
+        torch.cuda.synchronize()
+        assert c.check_guards()
+    assert float((outs[0] - outs[1]).abs().max()) <= 2e-4
+    assert zc.zc_device_status() == 0
+
+
+@pytest.mark.parametrize("cfg_id", [2, 3])
+def test_decode_is_invariant_under_the_split_count(cfg_id):
+    """The same cache attended with different split-K plans (one CTA per unit and large items;
+    items sized for one call at a time; separate and deferred append) gives the same output up
+    to the kernel's arithmetic noise (2e-4 on the fp32 output), at full size."""
+    import paper_2405_14256_b200 as zc
+    from workloads import make_decode_step
+    w = get_config(cfg_id)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w).tolist()
+    outs = []
+    for overlap, defer in ((False, False), (True, True), (False, True)):
+        c = tl.make_cache(w, max_new=4, defer_append=defer, overlap_calls=overlap, out_f32=True)
+        c.prefill_compress(Q, K, V, P)
+        for step in range(2):
+            q, k, v = make_decode_step(w, 0, step, tl.DEV)
+            c.append(k, v)
+            o = c.decode_attention(q, False)
+        outs.append(o.clone())
+        torch.cuda.synchronize()
+        assert c.check_guards()
+    assert float((outs[0] - outs[1]).abs().max()) <= 2e-4
+    assert float((outs[0] - outs[2]).abs().max()) <= 2e-4
+    assert zc.zc_device_status() == 0
+
+
+def test_a_second_decode_call_on_the_same_tail_leaves_the_window_bookkeeping_alone():
+    """Alg. 3 takes one step per generated token.  A re-query (a second decode call without an
+    append) must attend the same cache and change nothing: the window still completes after
+    `window` tokens and its re-compressed segment equals the oracle's, which never saw the
+    extra calls."""
+    import paper_2405_14256_b200 as zc
+    from workloads import make_decode_step
+    w = tl.small_workload(context=200, batch=2, n_q_heads=8, n_kv_heads=2, window=16,
+                          rho_recent=0.1, rho_random=0.1)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    for defer in (False, True):
+        cache = tl.make_cache(w, max_new=40, defer_append=defer)
+        cache.prefill_compress(Q, K, V, P.tolist())
+        oc2 = tl.make_oracle(w)
+        for u in oc.unit_ids:
+            oc2.units[u].segments = list(oc.units[u].segments)
+        for step in range(20):
+            q, k, v = make_decode_step(w, 0, step, tl.DEV)
+            cache.append(k, v)
+            first = cache.decode_attention(q, step % 3 == 0).clone()
+            if step % 4 == 1 or step == 15:            # also on the step that completes the window
+                again = cache.decode_attention(q, True)
+                if step != 15:                          # same cache, same query: same result
+                    assert torch.equal(first, again)
+            oc2.append(tl.to64(k), tl.to64(v))
+            ref = oc2.decode_attention(tl.to64(q), step % 3 == 0)
+            got = tl.to64(first)
+            for (bi, kv), o in ref.items():
+                assert tl.output_excess(got[bi, kv * w.group:(kv + 1) * w.group], o, w.torch_dtype) <= 0.0
+        torch.cuda.synchronize()
+        assert zc.zc_num_segments(cache.handle) == 2 and zc.zc_tail_tokens(cache.handle) == 4
+        assert tl.compare_segment(cache, oc2, 1) == 0
+        assert cache.check_guards()

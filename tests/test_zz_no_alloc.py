@@ -91,3 +91,40 @@ def test_noalloc_entry_rejects_shapes_beyond_its_buffer():
     big.decode_attention(q, False, out=out)
     torch.cuda.synchronize()
     assert torch.isfinite(out.float()).all()
+
+
+def test_noalloc_calls_back_to_back_without_synchronising():
+    """Several caches, call after call on one stream with no host synchronisation between
+    them: every call uses the one built-in buffer, the library gives calls that may be in
+    flight together separate parts of it (or orders them).  Results must equal those of the
+    same sequence through a caller workspace."""
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(context=260, batch=2, n_q_heads=8, n_kv_heads=2, window=8)
+    layers, steps = 3, 20
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w).tolist()
+    ins = [make_decode_step(w, 0, s, tl.DEV) for s in range(steps)]
+    results = []
+    for noalloc in (False, True):
+        caches = [tl.make_cache(w, max_new=32, defer_append=True, overlap_calls=True) for _ in range(layers)]
+        for c in caches:
+            c.mem.zero_()
+            c.prefill_compress(Q, K, V, P)
+        outs = [[torch.empty_like(ins[0][0]) for _ in range(layers)] for _ in range(steps)]
+        torch.cuda.synchronize()
+        for s in range(steps):
+            q, k, v = ins[s]
+            for ly, c in enumerate(caches):
+                c.append(k, v)
+                if noalloc:
+                    zc.zc_decode_attention_noalloc(c.handle, q, outs[s][ly], s % 3 == 0)
+                else:
+                    c.decode_attention(q, s % 3 == 0, out=outs[s][ly])
+        torch.cuda.synchronize()
+        assert zc.zc_device_status() == 0
+        results.append((outs, [c.mem.clone() for c in caches]))
+    for a, b in zip(results[0][0], results[1][0]):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
+    for x, y in zip(results[0][1], results[1][1]):
+        assert torch.equal(x, y)

@@ -24,12 +24,16 @@ def to64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu", torch.float64).numpy()
 
 
-def make_cache(w: Workload, max_new=None, defer_append: bool = False, overlap_calls: bool = False):
+GUARD = 4096   # bytes of canary on each side of every cache buffer and workspace the tests allocate
+
+
+def make_cache(w: Workload, max_new=None, defer_append: bool = False, overlap_calls: bool = False, **kw):
     import paper_2405_14256_b200 as zc
     return zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context,
                        w.decode_steps if max_new is None else max_new, w.saliency_ratio,
                        w.bits_hi, w.bits_lo, w.window, device=DEV, defer_append=defer_append,
-                       overlap_calls=overlap_calls, k_channel=w.k_scheme == "channel")
+                       overlap_calls=overlap_calls, k_channel=w.k_scheme == "channel", guard_bytes=GUARD,
+                       **kw)
 
 
 def make_oracle(w: Workload, units=None) -> zo.ZipCacheOracle:
@@ -192,6 +196,7 @@ def run_decode_parity(w: Workload, n_steps: int, units=None, layer: int = 0,
             worst = max(worst, output_error(g_, o))
             assert output_excess(g_, o, w.torch_dtype) <= 0.0, (step, worst)
     torch.cuda.synchronize()
+    assert cache.check_guards(), "a kernel wrote outside the cache buffer or the workspace"
     if check_segments:
         import paper_2405_14256_b200 as zc
         n_seg = zc.zc_num_segments(cache.handle)
@@ -242,7 +247,7 @@ def run_benchmark_mode(w: Workload, units, n_steps: int, layers: int = 2, graph:
         c = zc.ZipCache(w.torch_dtype, w.batch, w.n_q_heads, w.n_kv_heads, w.context, max(n_steps, 1),
                         w.saliency_ratio, w.bits_hi, w.bits_lo, w.window, device=DEV, workspace=ws,
                         defer_append=defer_append, overlap_calls=overlap_calls,
-                        k_channel=w.k_scheme == "channel")
+                        k_channel=w.k_scheme == "channel", guard_bytes=GUARD)
         ws = c.workspace
         c.prefill_compress(Q, K, V, P.tolist())
         torch.cuda.synchronize()
@@ -276,6 +281,7 @@ def run_benchmark_mode(w: Workload, units, n_steps: int, layers: int = 2, graph:
         issue()
     torch.cuda.synchronize()
     assert zc.zc_device_status() == 0
+    assert all(c.check_guards() for c in caches), "a kernel wrote outside its buffers"
     G = w.group
     worst = worst_r = 0.0
     excess = -1.0
