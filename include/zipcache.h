@@ -61,12 +61,17 @@ enum {
  * stay valid and unchanged until the stream has passed that zc_decode_attention call.  Any
  * other call on the cache first performs the pending append as its own launch. */
 #define ZC_FLAG_DEFER_APPEND 1
-/* With ZC_FLAG_OVERLAP_CALLS the caller tells the library that decode calls on independent
- * caches follow one another on the stream with nothing else between them (the layers of a
- * benchmark, caches of different requests).  Consecutive zc_decode_attention calls always run
- * side by side on the GPU where their buffers allow it; the flag only changes how a call is
- * cut into work items: few large ones, which is best when several calls share the GPU and
- * worst for a single call that has the GPU to itself. */
+/* With ZC_FLAG_OVERLAP_CALLS the caller PROMISES that, on the stream it passes, a decode call of
+ * this cache is preceded only by work that has completed or by other zc_decode_attention /
+ * zc_append calls of this library (the layers of a benchmark, caches of independent requests),
+ * with no kernel of another library between them.  The decode kernel then does not wait for the
+ * kernel before it: consecutive calls run side by side on the GPU, ordered among themselves only
+ * where their buffers require it (see zc_decode_attention), and a call is cut into few large
+ * work items, which is best when several calls share the GPU.
+ * Without the flag (the default) every decode kernel waits for everything that precedes it on
+ * the stream before it reads q, k_new, v_new or the cache -- also when the kernel before it is
+ * one that lets its successors start early (programmatic dependent launch), e.g. the projection
+ * that produces q -- and a call is cut into items sized for a call that has the GPU to itself. */
 #define ZC_FLAG_OVERLAP_CALLS 2
 /* With ZC_FLAG_OUT_F32 zc_decode_attention stores its result as fp32 (out [device]
  * b x h_q x d floats) instead of rounding it to cfg.dtype.  A 16-bit output cannot be closer
@@ -87,8 +92,9 @@ typedef struct {
   int32_t max_new_tokens; /* decode capacity (tokens appended after prefill) */
   int32_t window;         /* tokens kept at full precision before re-compression
                              (Alg. 3 uses 100); 8 <= window <= ZC_MAX_WINDOW */
-  int32_t bits_hi;        /* bit-width of salient tokens: 4 or 2 */
-  int32_t bits_lo;        /* bit-width of regular tokens: 4 or 2 */
+  int32_t bits_hi;        /* bit-width of salient tokens: 4, 2, or 16 (kept as they are: the
+                             "16/16" and "16/2" settings of Table 3) */
+  int32_t bits_lo;        /* bit-width of regular tokens: 4, 2 or 16 */
   int32_t flags;          /* 0 or an OR of the ZC_FLAG_* values above */
   double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
   int32_t k_scheme;       /* quantiser of the keys: ZC_K_CST (Alg. 1 on K and V) or ZC_K_CHANNEL
@@ -145,12 +151,17 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
  * tokens is added to the window statistics; the call that takes the window's last step
  * also re-compresses the tail into a new segment, inside the same kernel (no further launch,
  * no host synchronisation).
- * Ordering: consecutive calls on one stream may run at the same time on the GPU.  The library
- * orders a call after the earlier ones whenever it reads or overwrites one of their outputs,
- * overwrites one of their inputs, or updates the same cache's window statistics; it cannot see
- * other aliasing, so q, k_new, v_new and out of calls issued back to back must not overlap
- * buffers that an earlier call of the stream still uses in any other way.  Kernels of other
- * libraries on the stream are ordered as usual.  The workspace must not be used by calls on
+ * Only a call that follows a zc_append takes a step of Alg. 3; a further call on the same tail
+ * (the same token queried again) attends the cache as it is and leaves the window's counters,
+ * statistics and segments alone.
+ * Ordering.  Default: the call's kernel starts its work after everything issued before it on
+ * the stream has completed, whoever launched it.  With ZC_FLAG_OVERLAP_CALLS: consecutive calls
+ * on one stream may run at the same time on the GPU; the library orders a call after the
+ * earlier ones whenever it reads or overwrites one of their outputs, overwrites one of their
+ * inputs, or updates the same cache's window statistics; it cannot see other aliasing, so q,
+ * k_new, v_new and out of calls issued back to back must not overlap buffers that an earlier
+ * call of the stream still uses in any other way, and (the flag's promise) no kernel of another
+ * library may sit between the calls.  In both modes the workspace must not be used by calls on
  * another stream at the same time, and CUDA graphs captured from one stream must not be
  * replayed at the same time on several streams (the calls of a capture share one ordering
  * word per captured stream). */
@@ -170,6 +181,7 @@ int zc_tail_tokens(const zc_cache* c);
  * (4-bit: element 2m low nibble, 2m+1 high nibble of byte m; 2-bit: element 4m+j in
  * bits [2j,2j+1] of byte m); sz b x h_kv x n x 2 floats (scale, zero point);
  * cf b x h_kv x d floats (channel factors).  tensor 0 = K, 1 = V.  Any out may be NULL.
+ * A subset kept at 16 bits exports its rows' bytes as codes (256 per token) and nothing else.
  * Keys under ZC_K_CHANNEL have no per-token parameters and no channel factors: for tensor 0,
  * sz then receives b x h_kv x d x 2 floats, the (scale, zero point) of every channel, and cf
  * is left untouched. */
@@ -193,8 +205,9 @@ int zc_export_segment(zc_cache* c, int segment, int tensor, int subset, int32_t*
  *     built-in buffer (about batch * n_q_heads * (items + 8) * 528 bytes, items = split-K
  *     pieces per KV head, 8 = tiles of the full-precision tail; use zc_decode_attention with a
  *     caller workspace then).
- *   - The first call on each device looks up the buffer's device address (a synchronous
- *     runtime query): make that first call outside any stream capture.
+ *   - The buffer's device address is looked up once per device (a synchronous runtime
+ *     query), by zc_cache_init when a device is current there, else by the first call of
+ *     this entry point on the device: that first call then belongs outside any stream capture.
  *   - All calls share the one buffer, whatever cache they work on.  Calls that follow one
  *     another in ONE stream get separate parts of it or are ordered by the library; calls in
  *     different streams, or from several host threads, that may run at the same time on the
