@@ -13,6 +13,8 @@ compared bit for bit.
 Passages followed (paper section / equation / algorithm):
   probe selection ............ Sec. 4.3 "random+recent" strategy, Alg. 2 line 1
   probe attention ............ Eq. 9 (with the causal mask of Eq. 2 / Sec. 4.2)
+  prefill attention output ... Eq. 2, Alg. 2 "O = FlashAttention(Q, K, V)" (causal), with the
+                               row log-sum-exp a fast-attention kernel keeps beside it
   accumulated score .......... Eq. 7
   normalised score ........... Eq. 8
   split by saliency ratio .... Alg. 2 "Split"
@@ -104,6 +106,28 @@ def probe_attention(Qp: np.ndarray, K: np.ndarray, P: Sequence[int]) -> np.ndarr
         e = np.exp(row - row.max())
         A[r, : p + 1] = e / e.sum()
     return A
+
+
+def prefill_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 2 for one head under the causal mask: O = Softmax(Q K^T / sqrt(d_k)) V with row i
+    seeing columns j <= i (Alg. 2's attention-output line).  Also returns, per row, the
+    base-2 log-sum-exp of its scaled logits, log2(sum_j 2^(s_ij log2 e)) -- the one number per
+    row from which any entry of the row's softmax can be rebuilt (Eq. 9's rows included).
+    Q, K, V [l, d]."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    l, d = K.shape
+    S = (Q @ K.T) / math.sqrt(d)
+    O = np.zeros((l, V.shape[1]))
+    lse2 = np.zeros(l)
+    for i in range(l):
+        row = S[i, : i + 1]
+        mx = row.max()
+        e = np.exp(row - mx)
+        O[i] = (e / e.sum()) @ V[: i + 1]
+        lse2[i] = (mx + math.log(e.sum())) / math.log(2.0)
+    return O, lse2
 
 
 def accumulated_scores(A_list: Sequence[np.ndarray]) -> np.ndarray:

@@ -670,3 +670,39 @@ def test_token_scope_shares_one_split_across_heads():
     one.prefill_compress(Q[:1, :2], K[:1, :1], V[:1, :1], P)
     ref.prefill_compress(Q[:1, :2], K[:1, :1], V[:1, :1], P)
     np.testing.assert_array_equal(one.units[(0, 0)].segments[0].hi.idx, ref.units[(0, 0)].segments[0].hi.idx)
+
+
+# ---------------------------------------------------------------- Eq. 2: causal prefill attention
+@pytest.mark.parametrize("l,d", [(1, 8), (7, 8), (33, 16), (130, 32)])
+def test_prefill_attention_is_library_causal_attention(l, d):
+    """Eq. 2 with the causal mask against the library's scaled-dot-product attention
+    (is_causal=True, fp64 on the CPU), and its row log-sum-exp against the library's logsumexp
+    of the masked logits; the rows of Eq. 9's probe attention are rebuilt from that number."""
+    rs = _rng(3 + l)
+    Q, K, V = rs.standard_normal((l, d)), rs.standard_normal((l, d)) * 2, rs.standard_normal((l, d))
+    O, lse2 = zo.prefill_attention(Q, K, V)
+    want = torch.nn.functional.scaled_dot_product_attention(
+        torch.tensor(Q)[None, None], torch.tensor(K)[None, None], torch.tensor(V)[None, None], is_causal=True)
+    np.testing.assert_allclose(O, want[0, 0].numpy(), rtol=1e-10, atol=1e-12)
+    S = torch.tensor(Q @ K.T / math.sqrt(d))
+    S = S.masked_fill(torch.triu(torch.ones(l, l, dtype=torch.bool), diagonal=1), float("-inf"))
+    np.testing.assert_allclose(lse2, (torch.logsumexp(S, dim=1) / math.log(2.0)).numpy(), rtol=1e-12)
+    P = list(range(0, l, 3)) + ([l - 1] if (l - 1) % 3 else [])
+    A = zo.probe_attention(Q[P], K, P)
+    for r, p in enumerate(P):
+        rebuilt = np.exp2(S[p, : p + 1].numpy() / math.log(2.0) - lse2[p])
+        np.testing.assert_allclose(A[r, : p + 1], rebuilt, rtol=1e-10)
+
+
+def test_prefill_attention_brute_force_and_last_row_is_decode():
+    """Pure-Python loops on a tiny case; the last row of the causal output is Eq. 4 for the
+    last query over all keys."""
+    rs = _rng(9)
+    l, d = 9, 4
+    Q, K, V = rs.standard_normal((l, d)), rs.standard_normal((l, d)), rs.standard_normal((l, d))
+    A = _brute_force_causal_attention(Q, K)
+    O, _ = zo.prefill_attention(Q, K, V)
+    for i in range(l):
+        for c in range(d):
+            assert abs(O[i, c] - sum(A[i][j] * V[j, c] for j in range(i + 1))) < 1e-12
+    np.testing.assert_allclose(O[-1], zo.exact_attention(Q[-1:], K, V)[0], rtol=1e-12)
