@@ -69,6 +69,48 @@ def _peaks():
     return 6650.0, "fallback"
 
 
+def _tensor_peak():
+    """Dense bf16 / fp16 TFLOP/s for a kernel timed inside a loop (the sustained figure)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d.get("bf16_tflops_sustained", d.get("bf16_tflops", 1400.0))), "measured, sustained"
+    return 1400.0, "fallback, sustained"
+
+
+def measure_prefill_attention(zc, wb, w, R):
+    """The step beside the path in Alg. 2: causal attention output with row log-sum-exp
+    (zc_prefill_attention), and prefill compression that takes the probe rows' statistics from
+    it (zc_prefill_compress_lse) instead of running its first score pass."""
+    n = min(R, 4)
+    c0 = wb.caches[next(iter(wb.caches))]
+    O = torch.empty((w.batch, w.n_q_heads, w.context, 128), dtype=w.torch_dtype, device=wb.dev)
+    lse = [torch.empty((w.batch, w.n_q_heads, w.context), dtype=torch.float32, device=wb.dev) for _ in range(n)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    with torch.cuda.stream(wb.stream):
+        for rep in range(4):           # one warm-up pass, three timed
+            if rep == 1:
+                ev[0].record(wb.stream)
+            for i in range(n):
+                Q, K, V = wb.inputs[i]
+                zc.zc_prefill_attention(c0[i].handle, Q, K, V, w.context, O, lse[i])
+        ev[1].record(wb.stream)
+        for rep in range(3):
+            for i in range(n):
+                Q, K, V = wb.inputs[i]
+                c0[i].prefill_compress_lse(Q, K, V, wb.probes[i], lse[i])
+        ev[2].record(wb.stream)
+    torch.cuda.synchronize()
+    t_att = ev[0].elapsed_time(ev[1]) / (3 * n)
+    t_cmp = ev[1].elapsed_time(ev[2]) / (3 * n)
+    flops = 2.0 * w.context * w.context * 128 * w.batch * w.n_q_heads      # causal: half of 4 l^2 d per head
+    peak, kind = _tensor_peak()
+    return {"attention_ms_per_layer": t_att, "attention_tflops": flops / (t_att * 1e-3) / 1e12,
+            "attention_frac_of_tensor_peak": flops / (t_att * 1e-3) / 1e12 / peak, "tensor_peak": f"{peak} TFLOP/s ({kind})",
+            "compress_with_attention_lse_tokens_per_s": w.batch * w.context / (t_cmp * 1e-3)}
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -502,6 +544,8 @@ def measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, modes, 
                      "sm_mhz": clocks.get("sm_mhz"), "reasons": clocks.get("reasons")}
         res["prefill_tokens_per_s"] = pre_tps
         res["prefill_roofline_frac"] = (R * algorithmic_prefill_bytes(w) / (t_pre * 1e-3) / 1e9) / peak
+    if not override and world == 1:
+        res["prefill_attention"] = measure_prefill_attention(zc, wb, w, R)
     assert zc.zc_device_status() == 0, "a bounded wait inside a kernel ran out"
     out = {"per_config": res}
     if headline:

@@ -139,6 +139,25 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
                         const int32_t* probe_pos, int n_probe, const int32_t* salient_idx,
                         void* workspace, size_t workspace_bytes, zc_stream_t stream);
 
+/* Prefill attention output (Eq. 2 with the causal mask; Alg. 2's line "O = FlashAttention(Q, K,
+ * V)", Appendix B): O [device] b x h_q x l x d (contiguous, cfg.dtype) = Softmax(Q K^T /
+ * sqrt(d)) V, row i over keys j <= i, and row_lse [device] b x h_q x l floats, every row's
+ * base-2 log-sum-exp of its scaled logits (log2 sum_j 2^(q_i.k_j log2(e) / sqrt(d))).  Q, K, V and
+ * their strides as for zc_prefill_compress.  The cache is not touched (the handle supplies the
+ * shapes).  Needs the driver's tensor-map entry point (ZC_ECUDA "not supported" without it). */
+int zc_prefill_attention(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                         const int64_t q_strides[3], const int64_t kv_strides[3], void* O,
+                         float* row_lse, zc_stream_t stream);
+
+/* zc_prefill_compress for a caller that has just run zc_prefill_attention on the same Q and K:
+ * row_lse [device] (that call's output) stands in for the first of the two probe-score passes
+ * (Eq. 9's row statistics), which is then not run; everything else, and the resulting cache, is
+ * the same. */
+int zc_prefill_compress_lse(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                            const int64_t q_strides[3], const int64_t kv_strides[3],
+                            const int32_t* probe_pos, int n_probe, const float* row_lse,
+                            void* workspace, size_t workspace_bytes, zc_stream_t stream);
+
 /* Append (Eq. 3, Alg. 3): k_new, v_new [device] b x h_kv x d, contiguous, are copied
  * verbatim into the full-precision tail.  ZC_ECAPACITY beyond max_new_tokens.  With
  * ZC_FLAG_DEFER_APPEND the copy happens inside the next zc_decode_attention (see the flag). */
@@ -225,7 +244,7 @@ int64_t zc_launch_count(const zc_cache* c);
 /* Synchronises the device and reads the library's device-side error word into *code
  * [host]: 0 = none, 1 = a bounded wait on an asynchronous copy inside the decode kernel
  * ran out, 2 = a bounded wait for an earlier decode call of the stream ran out, 3 = a bounded wait
- * on the tensor cores inside a probe-score kernel ran out (outputs are then invalid).  Device code never traps or spins forever. */
+ * on the tensor cores inside a probe-score or prefill-attention kernel ran out (outputs are then invalid).  Device code never traps or spins forever. */
 int zc_device_status(int* code);
 
 /* Host-only model of the ordering the library applies to zc_decode_attention calls issued on

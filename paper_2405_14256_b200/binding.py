@@ -54,6 +54,13 @@ _SIGS = {
                                       C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                       C.POINTER(C.c_int32), C.c_int, C.c_void_p, C.c_void_p,
                                       C.c_size_t, C.c_void_p]),
+    "zc_prefill_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                       C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.c_void_p, C.c_void_p,
+                                       C.c_void_p]),
+    "zc_prefill_compress_lse": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                          C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                          C.POINTER(C.c_int32), C.c_int, C.c_void_p, C.c_void_p,
+                                          C.c_size_t, C.c_void_p]),
     "zc_append": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "zc_decode_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                       C.c_size_t, C.c_void_p]),
@@ -166,6 +173,28 @@ def zc_prefill_compress(handle, Q, K, V, l: int, probe_pos: Optional[Sequence[in
     _check(lib().zc_prefill_compress(handle, _ptr(Q), _ptr(K), _ptr(V), l, qs, ks, pp, n_probe,
                                      _ptr(salient_idx), _ptr(workspace), ws_bytes,
                                      _stream(stream)), "zc_prefill_compress")
+
+
+def zc_prefill_attention(handle, Q, K, V, l: int, O, row_lse, stream=None) -> None:
+    qs = (C.c_int64 * 3)(*Q.stride()[:3])
+    ks = (C.c_int64 * 3)(*K.stride()[:3])
+    if K.stride() != V.stride():
+        raise ZipCacheError("K and V must share strides")
+    _check(lib().zc_prefill_attention(handle, _ptr(Q), _ptr(K), _ptr(V), l, qs, ks, _ptr(O), _ptr(row_lse),
+                                      _stream(stream)), "zc_prefill_attention")
+
+
+def zc_prefill_compress_lse(handle, Q, K, V, l: int, probe_pos: Sequence[int], row_lse, workspace,
+                            stream=None) -> None:
+    qs = (C.c_int64 * 3)(*Q.stride()[:3])
+    ks = (C.c_int64 * 3)(*K.stride()[:3])
+    if K.stride() != V.stride():
+        raise ZipCacheError("K and V must share strides")
+    pp = (C.c_int32 * max(1, len(probe_pos)))(*probe_pos)
+    ws_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().zc_prefill_compress_lse(handle, _ptr(Q), _ptr(K), _ptr(V), l, qs, ks, pp, len(probe_pos),
+                                         _ptr(row_lse), _ptr(workspace), ws_bytes, _stream(stream)),
+           "zc_prefill_compress_lse")
 
 
 def zc_append(handle, k_new, v_new, stream=None) -> None:
@@ -305,6 +334,17 @@ class ZipCache:
     def prefill_compress(self, Q, K, V, probe_pos=None, salient_idx=None, stream=None):
         zc_prefill_compress(self.handle, Q, K, V, K.shape[2], probe_pos, salient_idx,
                             self.workspace, stream)
+
+    def prefill_attention(self, Q, K, V, stream=None):
+        """Causal attention output O and the rows' log-sum-exp (Alg. 2's attention-output line)."""
+        l = K.shape[2]
+        O = torch.empty((self.batch, self.n_q_heads, l, 128), dtype=self.dtype, device=self.device)
+        lse = torch.empty((self.batch, self.n_q_heads, l), dtype=torch.float32, device=self.device)
+        zc_prefill_attention(self.handle, Q, K, V, l, O, lse, stream)
+        return O, lse
+
+    def prefill_compress_lse(self, Q, K, V, probe_pos, row_lse, stream=None):
+        zc_prefill_compress_lse(self.handle, Q, K, V, K.shape[2], probe_pos, row_lse, self.workspace, stream)
 
     def append(self, k_new, v_new, stream=None):
         zc_append(self.handle, k_new, v_new, stream)

@@ -12,8 +12,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzipcache.so")
 SOURCES = ["zc_host.cu", "zc_scores.cu", "zc_compress.cu", "zc_decode.cu", "zc_order.cu",
-           "zc_export.cu"]
-HEADERS = ["zc_internal.h", "zc_layout.cuh", "zc_mma.cuh", "zc_order.h", "zc_quant.cuh"]
+           "zc_export.cu", "zc_attention.cu"]
+HEADERS = ["zc_internal.h", "zc_layout.cuh", "zc_mma.cuh", "zc_order.h", "zc_quant.cuh", "zc_tc.cuh"]
 
 
 def _nvcc() -> str:

@@ -318,10 +318,13 @@ int zc_default_probes(int l, double rho_recent, double rho_random, uint64_t seed
   return ZC_OK;
 }
 
-int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V, int l,
-                        const int64_t q_strides[3], const int64_t kv_strides[3],
-                        const int32_t* probe_pos, int n_probe, const int32_t* salient_idx,
-                        void* workspace, size_t workspace_bytes, zc_stream_t stream) {
+}  // extern "C"
+
+static int prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                            const int64_t q_strides[3], const int64_t kv_strides[3],
+                            const int32_t* probe_pos, int n_probe, const int32_t* salient_idx,
+                            const float* row_lse, void* workspace, size_t workspace_bytes,
+                            zc_stream_t stream) {
   if (!c || !K || !V || !kv_strides) return ZC_EINVAL;
   if (l < 1) return ZC_EINVAL;
   if (l > c->cfg.max_prefill) return ZC_ECAPACITY;
@@ -373,11 +376,45 @@ int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V
                         align_up((size_t)c->cfg.batch * c->cfg.n_q_heads * (size_t)n_probe * 4, 256);
     void* qp = used < workspace_bytes ? (char*)workspace + used : nullptr;
     ZC_CUDA(zc_launch_probe_scores(c, Q, K, l, q_strides, kv_strides, P_dev, n_probe, lse, qp,
-                                   qp ? workspace_bytes - used : 0, st));
+                                   qp ? workspace_bytes - used : 0, row_lse, st));
   }
   ZC_CUDA(zc_launch_topk(c, l, c->n0[0], 0, salient_idx, st));
   ZcSrc src{K, V, kv_strides[0], kv_strides[1], kv_strides[2]};
   ZC_CUDA(zc_launch_quantize(c, src, zc_segment(c, 0), st));
+  return ZC_OK;
+}
+
+extern "C" {
+
+int zc_prefill_compress(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                        const int64_t q_strides[3], const int64_t kv_strides[3],
+                        const int32_t* probe_pos, int n_probe, const int32_t* salient_idx,
+                        void* workspace, size_t workspace_bytes, zc_stream_t stream) {
+  return prefill_compress(c, Q, K, V, l, q_strides, kv_strides, probe_pos, n_probe, salient_idx, nullptr,
+                          workspace, workspace_bytes, stream);
+}
+
+int zc_prefill_compress_lse(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                            const int64_t q_strides[3], const int64_t kv_strides[3],
+                            const int32_t* probe_pos, int n_probe, const float* row_lse,
+                            void* workspace, size_t workspace_bytes, zc_stream_t stream) {
+  if (!row_lse) return ZC_EINVAL;
+  if (!aligned16(row_lse)) return ZC_EALIGN;
+  return prefill_compress(c, Q, K, V, l, q_strides, kv_strides, probe_pos, n_probe, nullptr, row_lse,
+                          workspace, workspace_bytes, stream);
+}
+
+int zc_prefill_attention(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                         const int64_t q_strides[3], const int64_t kv_strides[3], void* O, float* row_lse,
+                         zc_stream_t stream) {
+  if (!c || !Q || !K || !V || !O || !row_lse || !q_strides || !kv_strides) return ZC_EINVAL;
+  if (l < 1) return ZC_EINVAL;
+  if (l > c->cfg.max_prefill) return ZC_ECAPACITY;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(row_lse)) return ZC_EALIGN;
+  for (int i = 0; i < 3; ++i)
+    if (q_strides[i] < 0 || (q_strides[i] % 8) || kv_strides[i] < 0 || (kv_strides[i] % 8)) return ZC_EINVAL;
+  if (q_strides[2] < ZC_D || kv_strides[2] < ZC_D) return ZC_EINVAL;
+  ZC_CUDA(zc_launch_prefill_attention(c, Q, K, V, l, q_strides, kv_strides, O, row_lse, (cudaStream_t)stream));
   return ZC_OK;
 }
 
@@ -522,9 +559,10 @@ int zc_device_status(int* code) {
   if (!code) return ZC_EINVAL;
   ZC_CUDA(cudaDeviceSynchronize());
   ZC_CUDA(zc_device_error_code(code));
-  int probe = 0;
+  int probe = 0, att = 0;
   ZC_CUDA(zc_probe_error_code(&probe));
-  if (*code == 0 && probe) *code = 3;
+  ZC_CUDA(zc_attention_error_code(&att));
+  if (*code == 0 && (probe || att)) *code = 3;
   return ZC_OK;
 }
 

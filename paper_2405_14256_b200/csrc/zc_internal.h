@@ -133,9 +133,18 @@ ZcDecodePlan zc_make_plan(const zc_cache* c);
 // ---- launchers (each returns a cudaError_t as int) ----
 // qp_ws / qp_bytes: room for a dense copy of the probe rows (batch * n_q_heads * n_probe rows of
 // 256 bytes, 16-byte aligned); used when large enough.
+// lse_rows: non-null = every row's log-sum-exp [batch][n_q_heads][l] is known already (from
+// zc_launch_prefill_attention): pass 1 is replaced by a gather of the probe rows' values.
 int zc_launch_probe_scores(zc_cache* c, const void* Q, const void* K, int l,
                            const int64_t* qs, const int64_t* ks, const int32_t* P_dev,
-                           int n_probe, float* lse_ws, void* qp_ws, size_t qp_bytes, cudaStream_t st);
+                           int n_probe, float* lse_ws, void* qp_ws, size_t qp_bytes,
+                           const float* lse_rows, cudaStream_t st);
+// Causal attention output O [batch][n_q_heads][l][128] and row log-sum-exp lse [batch][n_q_heads][l].
+int zc_launch_prefill_attention(zc_cache* c, const void* Q, const void* K, const void* V, int l,
+                                const int64_t* qs, const int64_t* ks, void* O, float* lse, cudaStream_t st);
+int zc_launch_gather_probe_lse(zc_cache* c, const float* lse_rows, const int32_t* P_dev, int n_probe, int l,
+                               float* lse_probe, cudaStream_t st);
+int zc_attention_error_code(int* out);   // 0 or 1: a bounded wait in the prefill attention kernel ran out
 int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
                    cudaStream_t st);
 int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st);

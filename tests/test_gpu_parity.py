@@ -614,3 +614,78 @@ def test_a_second_decode_call_on_the_same_tail_leaves_the_window_bookkeeping_alo
         assert zc.zc_num_segments(cache.handle) == 2 and zc.zc_tail_tokens(cache.handle) == 4
         assert tl.compare_segment(cache, oc2, 1) == 0
         assert cache.check_guards()
+
+
+# ------------------------------------------------------------------ prefill attention (Eq. 2) with row log-sum-exp
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("kw", [
+    dict(context=1, n_q_heads=1, n_kv_heads=1),
+    dict(context=17, n_q_heads=2, n_kv_heads=2),
+    dict(context=128, n_q_heads=4, n_kv_heads=1),
+    dict(context=129, n_q_heads=2, n_kv_heads=1),
+    dict(context=300, batch=2, n_q_heads=8, n_kv_heads=2),
+    dict(context=1000, n_q_heads=4, n_kv_heads=4, outlier_fixed=0),
+])
+def test_prefill_attention_output_and_row_lse(dtype, kw):
+    """O = causal Softmax(Q K^T / sqrt(d)) V and every row's log-sum-exp against the oracle's
+    Eq. 2, head by head.  The weights reach the tensor cores in the input type, so O carries
+    their rounding (2^-9 relative for bf16, 2^-12 for fp16) on top of its own storage
+    rounding: 2e-2 / 4e-3 absolute on outputs of magnitude up to 4; the log-sum-exp is formed
+    in fp32 from unrounded values: 2e-4 (base-2 units)."""
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(dtype=dtype, **kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    cache = tl.make_cache(w)
+    O, lse = cache.prefill_attention(Q, K, V)
+    torch.cuda.synchronize()
+    assert zc.zc_device_status() == 0 and cache.check_guards()
+    Q64, K64, V64 = tl.to64(Q), tl.to64(K), tl.to64(V)
+    O_g, lse_g = tl.to64(O), lse.double().cpu().numpy()
+    tol = 2e-2 if dtype == "bf16" else 4e-3
+    for bi in range(w.batch):
+        for h in range(w.n_q_heads):
+            kv = h // w.group
+            O_ref, lse_ref = zo.prefill_attention(Q64[bi, h], K64[bi, kv], V64[bi, kv])
+            assert np.abs(O_g[bi, h] - O_ref).max() <= tol, (bi, h, np.abs(O_g[bi, h] - O_ref).max())
+            assert np.abs(lse_g[bi, h] - lse_ref).max() <= 2e-4, (bi, h, np.abs(lse_g[bi, h] - lse_ref).max())
+
+
+@pytest.mark.parametrize("kw", [
+    dict(context=777, batch=2, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0),
+    dict(context=1300, n_q_heads=2, n_kv_heads=2, band=20, saliency_ratio=0.3),
+])
+def test_prefill_compress_from_the_attention_kernels_lse(kw):
+    """zc_prefill_compress_lse: the probe rows' statistics come from zc_prefill_attention instead
+    of the first probe-score pass; scores, salient sets and codes must match the oracle as with
+    zc_prefill_compress."""
+    w = tl.small_workload(**kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w)
+    _, lse = cache.prefill_attention(Q, K, V)
+    cache.prefill_compress_lse(Q, K, V, P.tolist(), lse)
+    torch.cuda.synchronize()
+    swaps, clean, rel = tl.compare_prefill_segment(w, cache, oc, oc.unit_ids)
+    assert swaps == 0 and clean == len(oc.unit_ids)
+    assert cache.check_guards()
+
+
+def test_prefill_attention_full_size_config2():
+    """Workload 2 at full size on sampled heads."""
+    import paper_2405_14256_b200 as zc
+    w = get_config(2)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    cache = tl.make_cache(w, max_new=4)
+    O, lse = cache.prefill_attention(Q, K, V)
+    torch.cuda.synchronize()
+    assert zc.zc_device_status() == 0
+    worst_o = worst_l = 0.0
+    for (bi, h) in [(0, 0), (3, 17), (7, 31)]:
+        kv = h // w.group
+        O_ref, lse_ref = zo.prefill_attention(tl.to64(Q[bi, h]), tl.to64(K[bi, kv]), tl.to64(V[bi, kv]))
+        worst_o = max(worst_o, float(np.abs(tl.to64(O[bi, h]) - O_ref).max()))
+        worst_l = max(worst_l, float(np.abs(lse[bi, h].double().cpu().numpy() - lse_ref).max()))
+    assert worst_o <= 2e-2 and worst_l <= 2e-4, (worst_o, worst_l)
+    tl.record("prefill attention, full size (3 heads)", config=2, max_abs_out=worst_o, score_rel=worst_l)
