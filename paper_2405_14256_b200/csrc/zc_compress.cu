@@ -138,10 +138,10 @@ __global__ void __launch_bounds__(kTopkThreads) k_topk_split(char* cache, ZcLayo
   er = eq_before;
   for (int i = lo; i < hi; ++i) {
     if (is_sal(i, er)) {
-      if (s_pos < n_s) idx_sal[s_pos] = i;
+      if (ZC_CHECKED(s_pos < n_s, ZC_DBG_TOPK_INDEX) && s_pos < n_s) idx_sal[s_pos] = i;
       ++s_pos;
     } else {
-      if (r_pos < n - n_s) idx_reg[r_pos] = i;
+      if (ZC_CHECKED(r_pos < n - n_s, ZC_DBG_TOPK_INDEX) && r_pos < n - n_s) idx_reg[r_pos] = i;
       ++r_pos;
     }
   }
@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int tt = t0 + w * 8 + 4 * half + i;
-      if (tt < seg.n_tok[cls]) {
+      if (tt < seg.n_tok[cls] && ZC_CHECKED(idx[tt] >= 0 && idx[tt] < src.l, ZC_DBG_QUANT_ROW)) {
         const long long row = (long long)idx[tt] * src.sl;
         rawK[i] = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
         rawV[i] = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
@@ -326,6 +326,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   __syncthreads();
 
   // compose the tile: 16-byte stores, consecutive threads -> consecutive addresses
+  if (!ZC_CHECKED(seg.tile0[cls] + tile < lay.cap_tiles[cls], ZC_DBG_QUANT_TILE)) return;
   char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
   const int total_vec = lay.tile_bytes[cls] / 16;
   for (int v = threadIdx.x; v < total_vec; v += 256)
@@ -365,4 +366,13 @@ int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStre
     c->launches += 2;
   }
   return (int)cudaGetLastError();
+}
+
+int zc_debug_code_compress(int* out) {
+#ifdef ZC_DEBUG
+  return (int)cudaMemcpyFromSymbol(out, g_zc_debug_fault, sizeof(int));
+#else
+  *out = 0;
+  return (int)cudaSuccess;
+#endif
 }

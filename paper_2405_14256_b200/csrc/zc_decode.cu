@@ -160,6 +160,7 @@ __global__ void k_append(char* cache, ZcLayout lay, const T* __restrict__ k_new,
   pdl_launch_dependents();
   pdl_wait();   // k_new / v_new may come from the previous kernel; the tail may still be read by it
   const int unit = blockIdx.x;
+  if (!ZC_CHECKED(pos >= 0 && pos < lay.window, ZC_DBG_TAIL_ROW)) return;
   char* ub = zc_unit_base(cache, lay, unit);
   T* tk = reinterpret_cast<T*>(ub + lay.off_tailK) + pos * ZC_D;
   T* tv = reinterpret_cast<T*>(ub + lay.off_tailV) + pos * ZC_D;
@@ -1158,6 +1159,7 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
       }
       __syncthreads();
       const int sub_in_tile = sb % (ZC_TILE / ZC_SUB);
+      if (!ZC_CHECKED(fl.seg.tile0[cls] + sb / (ZC_TILE / ZC_SUB) < lay.cap_tiles[cls], ZC_DBG_FLUSH_TILE)) break;
       char* tile_ptr = ub + lay.off_tiles[cls] +
                        (long long)(fl.seg.tile0[cls] + sb / (ZC_TILE / ZC_SUB)) * lay.tile_bytes[cls];
       for (int v = tid; v < vecs; v += 128)
@@ -1367,7 +1369,10 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     ItemScale sc;
     sc.chan_factor = 1.f;
     sc.rowscale = 1.f;
-    const bool has = d.sub_hi > d.sub_lo;
+    const bool has = d.sub_hi > d.sub_lo &&
+                     ZC_CHECKED(d.sub_hi <= lay.cap_tiles[d.cls] * (ZC_TILE / ZC_SUB) && d.run < lay.max_runs &&
+                                    it < ZC_MAX_ITEMS,
+                                ZC_DBG_DECODE_ITEM);
     if (has) {
       const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
       const char* class_base = ub + lay.off_tiles[d.cls];
@@ -1643,6 +1648,15 @@ int zc_static_scratch(void** ptr) {
   static void* addr[64] = {nullptr};
   static std::mutex guard;
   return symbol_address(g_zc_noalloc_scratch, addr, guard, ptr);
+}
+
+int zc_debug_code_decode(int* out) {
+#ifdef ZC_DEBUG
+  return (int)cudaMemcpyFromSymbol(out, g_zc_debug_fault, sizeof(int));
+#else
+  *out = 0;
+  return (int)cudaSuccess;
+#endif
 }
 
 int zc_device_error_code(int* out) {

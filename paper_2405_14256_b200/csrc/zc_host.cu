@@ -382,7 +382,7 @@ static int prefill_compress(zc_cache* c, const void* Q, const void* K, const voi
                                    qp ? workspace_bytes - used : 0, row_lse, st));
   }
   ZC_CUDA(zc_launch_topk(c, l, c->n0[0], 0, salient_idx, st));
-  ZcSrc src{K, V, kv_strides[0], kv_strides[1], kv_strides[2]};
+  ZcSrc src{K, V, kv_strides[0], kv_strides[1], kv_strides[2], l};
   ZC_CUDA(zc_launch_quantize(c, src, zc_segment(c, 0), st));
   return ZC_OK;
 }
@@ -566,6 +566,10 @@ int zc_device_status(int* code) {
   ZC_CUDA(zc_probe_error_code(&probe));
   ZC_CUDA(zc_attention_error_code(&att));
   if (*code == 0 && (probe || att)) *code = 3;
+  int dbg_c = 0, dbg_d = 0;   // bounds-checked build only: 100 + the first failed check
+  ZC_CUDA(zc_debug_code_compress(&dbg_c));
+  ZC_CUDA(zc_debug_code_decode(&dbg_d));
+  if (*code == 0 && (dbg_c || dbg_d)) *code = 100 + (dbg_c ? dbg_c : dbg_d);
   return ZC_OK;
 }
 

@@ -56,6 +56,7 @@ struct ZcSrc {
   const void* K;
   const void* V;
   long long sb, sh, sl;  // element strides of (batch, kv head, token)
+  int l;                 // rows per (batch, kv head)
 };
 
 // One segment's two subsets.
@@ -127,6 +128,25 @@ struct zc_cache {
 
 __host__ __device__ static inline int zc_ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Bounds-checked build (-DZC_DEBUG, `python -m paper_2405_14256_b200.build --debug`): index
+// arithmetic of the kernels is checked where a tile, a row or a partial is addressed; a check
+// that fails records its code (first failure wins) in a word that zc_device_status reports as
+// 100 + code, and the access is skipped.  Nothing traps.  In the normal build the macro is empty.
+#ifdef ZC_DEBUG
+#define ZC_CHECKED(ok, code) (zc_debug_check((ok), (code)))
+#else
+#define ZC_CHECKED(ok, code) (true)
+#endif
+enum {
+  ZC_DBG_QUANT_ROW = 1,     // quantiser: a gathered token index outside [0, l)
+  ZC_DBG_QUANT_TILE = 2,    // quantiser: a tile beyond the class's capacity
+  ZC_DBG_DECODE_ITEM = 3,   // decode: an item's sub-tiles beyond the class's capacity
+  ZC_DBG_DECODE_PART = 4,   // decode: a partial beyond the workspace region
+  ZC_DBG_TAIL_ROW = 5,      // append / decode: a tail row beyond the window
+  ZC_DBG_FLUSH_TILE = 6,    // window re-compression: a tile beyond the class's capacity
+  ZC_DBG_TOPK_INDEX = 7,    // split: an index list entry beyond its list
+};
+
 ZcSeg zc_segment(const zc_cache* c, int seg);
 ZcDecodePlan zc_make_plan(const zc_cache* c);
 
@@ -158,6 +178,8 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
 // Bytes of ws one call of `items` items per unit takes.
 size_t zc_decode_scratch_bytes(const zc_cache* c, int items);
 int zc_device_error_code(int* out);
+int zc_debug_code_compress(int* out);   // bounds-checked build: first failed check of the compression kernels (0: none)
+int zc_debug_code_decode(int* out);     // ... of the append / decode kernels
 int zc_probe_error_code(int* out);   // 0 or 1: a bounded wait in a probe-score kernel ran out
 // Device address of the per-stream ordering words on the current device (looked up once per
 // device; pass nullptr to only perform the look-up).

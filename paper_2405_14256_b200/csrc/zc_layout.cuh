@@ -68,6 +68,15 @@ __device__ inline float zc_key_float(unsigned k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+#ifdef ZC_DEBUG
+// one word per translation unit (no relocatable device code): zc_debug_code_* read them
+static __device__ int g_zc_debug_fault = 0;
+__device__ inline bool zc_debug_check(bool ok, int code) {
+  if (!ok) atomicCAS(&g_zc_debug_fault, 0, code);
+  return ok;
+}
+#endif
+
 __device__ inline char* zc_unit_base(char* base, const ZcLayout& lay, int unit) {
   return base + (long long)unit * lay.unit_stride;
 }
