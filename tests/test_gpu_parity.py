@@ -297,13 +297,14 @@ def test_kernel_arithmetic_within_2e3_of_the_oracle_on_every_config(cfg_id, unit
 
 
 @pytest.mark.parametrize("cfg_id,units,steps", [(2, [(3, 1), (4, 6)], 4), (4, [(9, 30)], 3)])
-def test_full_size_single_call_plan_with_calls_in_flight(cfg_id, units, steps):
-    """The other plan the benchmark reports: items sized for one call at a time, deferred
-    append, calls still issued back to back."""
+def test_full_size_one_call_at_a_time(cfg_id, units, steps):
+    """The other launch mode the benchmark reports (no ZC_FLAG_OVERLAP_CALLS): every call waits
+    for the kernel before it, items sized for a call that has the GPU to itself (workload 4: one
+    CTA per unit), deferred append, calls issued back to back."""
     w = get_config(cfg_id)
     r = tl.run_benchmark_mode(w, units, steps, layers=2, overlap_calls=False)
     assert r["excess"] <= 0.0, r
-    tl.record("full size, single-call plan back to back", config=cfg_id, units=2 * len(units),
+    tl.record("full size, one call at a time (benchmark mode `dependent`)", config=cfg_id, units=2 * len(units),
               steps=steps, max_abs_out=r["worst"], max_abs_out_vs_rounded_oracle=r["worst_rounded"])
 
 
