@@ -451,22 +451,20 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
       }
     }
   };
+  // One loop body for every pair (the end-of-run handling costs two uniform compares per pair;
+  // a second copy of the unrolled step for the last pairs would double the loop's code, and the
+  // instruction cache is what this loop runs out of first).
   const int n_refill = my_np - NST;
-  for (int i = 0; i < n_refill; ++i) {
+  for (int i = 0; i < my_np; ++i) {
     uint64_t* bar = &my_bar[stage];
     wait_stage(bar);
     char* st = my_ring + stage * PB;
-    pair_step<BITS, false, KCH>(st, lane, 0, qb, qs, isc, logKs, tau_u, srcA, srcB, c0_src, c1_src, oacc, S);
+    pair_step<BITS, true, KCH>(st, lane, rem0 - i * (2 * ZC_SUB * kWarps), qb, qs, isc, logKs, tau_u, srcA, srcB,
+                               c0_src, c1_src, oacc, S);
     __syncwarp();
-    refill_if(lane == 0, bar, st, src_refill, rem_refill > ZC_SUB ? PB : SB);
+    refill_if(lane == 0 && i < n_refill, bar, st, src_refill, rem_refill > ZC_SUB ? PB : SB);
     src_refill += kWarps * PB;
     rem_refill -= 2 * ZC_SUB * kWarps;
-    if (++stage == NST) { stage = 0; parity ^= 1u; }
-  }
-  for (int i = max(n_refill, 0); i < my_np; ++i) {
-    wait_stage(&my_bar[stage]);
-    pair_step<BITS, true, KCH>(my_ring + stage * PB, lane, rem0 - i * (2 * ZC_SUB * kWarps), qb, qs, isc, logKs,
-                          tau_u, srcA, srcB, c0_src, c1_src, oacc, S);
     if (++stage == NST) { stage = 0; parity ^= 1u; }
   }
   // sums back to plain units: l' = sum p 2^logKs; zacc' = sum w z with w short by the odd-token 1/4
