@@ -297,13 +297,17 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
         rawV[i] = make_uint2(0, 0);
       }
     }
-#pragma unroll
+    // one copy of the quantiser's code for the batch's four rows (not unrolled: the kernel is
+    // straight-line code executed once per CTA, and what it waits for most is instruction fetch)
+#pragma unroll 1
     for (int i = 0; i < 4; ++i) {
       const int tl = w * 8 + 4 * half + i, tt = t0 + tl;
       const bool live = tt < seg.n_tok[cls];
+      const uint2 rk = i == 0 ? rawK[0] : i == 1 ? rawK[1] : i == 2 ? rawK[2] : rawK[3];
+      const uint2 rv = i == 0 ? rawV[0] : i == 1 ? rawV[1] : i == 2 ? rawV[2] : rawV[3];
       float x[4], s, z;
       unsigned pk;
-      const T* ek = reinterpret_cast<const T*>(&rawK[i]);
+      const T* ek = reinterpret_cast<const T*>(&rk);
 #pragma unroll
       for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
       if (kch) {
@@ -313,7 +317,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
         if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
       }
       *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live ? pk : 0u;
-      const T* ev = reinterpret_cast<const T*>(&rawV[i]);
+      const T* ev = reinterpret_cast<const T*>(&rv);
 #pragma unroll
       for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
       quant_token(x, cV, L, &s, &z, &pk);
