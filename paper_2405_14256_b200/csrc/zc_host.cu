@@ -211,7 +211,7 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   p.ctas_per_sm = 3;
   if (choose(4) >= ZC_MANY_WAVES * c->n_sm * 4) p.ctas_per_sm = 4;
   else choose(3);
-  // One CTA per unit and head group, items as large as they get: for calls that run side by
+  // One CTA per unit and head group, one item per class of the prompt's segment: for calls that run side by
   // side with their neighbours (wave fill is then no concern, only the fixed cost per CTA), and
   // for a call alone whose units by themselves fill every slot of the GPU (workload 4: 1024 units
   // on 592 slots; 115 us per call against 134 us with one CTA per item).
@@ -220,10 +220,9 @@ ZcDecodePlan zc_make_plan(const zc_cache* c) {
   if (unit_ctas) {
     p.ctas_per_sm = 4;
     p.fold_tail = 1;
-    for (int k = 0; k < 2; ++k) {
-      const int want = std::min(std::min(zc_ceil_div(subs[k], kCand[0]), std::min(ZC_MAX_SPLIT_HOST, cap)), subs[k]);
-      p.spi0[k] = (zc_ceil_div(subs[k], std::max(1, want)) + 1) & ~1;
-      p.split0[k] = zc_ceil_div(subs[k], p.spi0[k]);
+    for (int k = 0; k < 2; ++k) {   // one item per class, however long: every further item costs a set-up and a merge
+      p.spi0[k] = (subs[k] + 1) & ~1;
+      p.split0[k] = 1;
     }
   }
   p.chain_free = overlap_calls ? 1 : 0;

@@ -234,7 +234,7 @@ def test_full_size_staged_codes_bit_exact(cfg_id, units, steps):
     (2, [(1, 2), (6, 5)], 305, False),            # three re-compressed windows
     (3, [(0, 0), (11, 5)], 4, False),
     (4, [(0, 0), (17, 13), (31, 31)], 4, False),
-    (5, [(2, 6)], 3, False),                      # several 256-sub-tile items per CTA
+    (5, [(2, 6)], 3, False),                      # items of 820 and 1229 sub-tiles, one CTA per unit
     (5, [(1, 1)], 3, True),
 ])
 def test_full_size_in_the_benchmark_configuration(cfg_id, units, steps, graph):
