@@ -143,9 +143,19 @@ __global__ void __launch_bounds__(kFaThreads, 1) k_flash_prefill(
       mma_tile(tmem, q_addr, k_addr, idesc_s);
       mma_commit(&s_done[0]);
       for (int kt = 0; kt < n_kt; ++kt) {
-        const int buf = kt & 1;
+        const int buf = kt & 1, nb = buf ^ 1;
+        // the key buffer of tile kt is free as soon as S of tile kt has completed (it was issued an
+        // iteration ago): tile kt + 2 is sent for now, two iterations ahead of its use
+        if (kt + 2 < n_kt) {
+          bar_wait(&s_done[buf], (uint32_t)(kt >> 1) & 1u);
+          tma_key_tile(&kmap, k_addr + buf * kTile, &k_full[buf], (kt + 2) * kM, kv, b);
+        }
+        // the value buffer of tile kt - 1 is free once its P V has completed: tile kt + 1
+        if (kt >= 1 && kt + 1 < n_kt) {
+          bar_wait(pv_done, (uint32_t)(kt - 1) & 1u);
+          tma_key_tile(&vmap, v_addr + nb * kTile, &v_full[nb], (kt + 1) * kM, kv, b);
+        }
         if (kt + 1 < n_kt) {   // S of the next tile, while the workers turn this one into P
-          const int nb = (kt + 1) & 1;
           bar_wait(&k_full[nb], (uint32_t)((kt + 1) >> 1) & 1u);
           if (kt + 1 >= 2) bar_wait(&s_free[nb], (uint32_t)((kt - 1) >> 1) & 1u);
           async_proxy_fence();
@@ -159,14 +169,6 @@ __global__ void __launch_bounds__(kFaThreads, 1) k_flash_prefill(
         tc_fence_after();
         mma_pv(tmem_o, p_addr, v_addr + buf * kTile, idesc_pv, kt > 0);
         mma_commit(pv_done);
-        if (kt + 2 < n_kt) {
-          // the key buffer was read by S of tile kt (completed before its P could be written),
-          // the value buffer is being read by the MMA just issued
-          bar_wait(&s_done[buf], (uint32_t)(kt >> 1) & 1u);
-          tma_key_tile(&kmap, k_addr + buf * kTile, &k_full[buf], (kt + 2) * kM, kv, b);
-          bar_wait(pv_done, (uint32_t)kt & 1u);
-          tma_key_tile(&vmap, v_addr + buf * kTile, &v_full[buf], (kt + 2) * kM, kv, b);
-        }
       }
     }
   } else {
