@@ -270,6 +270,17 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     }
     cV[e] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
   }
+  // the divisors that stay for the whole tile: their correctly rounded reciprocals once
+  float rK[4], rV[4];
+  bool midK = true, midV = true;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    rK[e] = __frcp_rn(cK[e]);
+    rV[e] = __frcp_rn(cV[e]);
+    midK = midK && zc_mid(cK[e]);
+    midV = midV && zc_mid(cV[e]);
+  }
+  const float rL = __frcp_rn(L);
   if (tile == 0 && w == 0) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -311,16 +322,16 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
 #pragma unroll
       for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
       if (kch) {
-        pk = quant_channel4(x, cK, zK, L);
+        pk = quant_channel4_rc(x, cK, rK, midK, zK, L);
       } else {
-        quant_token(x, cK, L, &s, &z, &pk);
+        quant_token_rc(x, cK, rK, midK, L, rL, &s, &z, &pk);
         if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
       }
       *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live ? pk : 0u;
       const T* ev = reinterpret_cast<const T*>(&rv);
 #pragma unroll
       for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
-      quant_token(x, cV, L, &s, &z, &pk);
+      quant_token_rc(x, cV, rV, midV, L, rL, &s, &z, &pk);
       *reinterpret_cast<unsigned*>(&codesV[tl][4 * lane]) = live ? pk : 0u;
       if (lane == 0) { parV[tl][0] = live ? s : 0.f; parV[tl][1] = live ? z : 0.f; }
       if (live) smax = fmaxf(smax, s);
@@ -333,8 +344,14 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   if (!ZC_CHECKED(seg.tile0[cls] + tile < lay.cap_tiles[cls], ZC_DBG_QUANT_TILE)) return;
   char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
   const int total_vec = lay.tile_bytes[cls] / 16;
-  for (int v = threadIdx.x; v < total_vec; v += 256)
-    reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(bits, lay.kch, v, 0, codesK, codesV, parK, parV);
+  // one copy per code width, so that the word-building loops have constant trip counts
+  if (bits == 4) {
+    for (int v = threadIdx.x; v < total_vec; v += 256)
+      reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(4, lay.kch, v, 0, codesK, codesV, parK, parV);
+  } else {
+    for (int v = threadIdx.x; v < total_vec; v += 256)
+      reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(2, lay.kch, v, 0, codesK, codesV, parK, parV);
+  }
 }
 
 }  // namespace

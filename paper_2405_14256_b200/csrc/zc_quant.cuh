@@ -36,6 +36,75 @@ static __device__ __forceinline__ void quant_token(const float (&x)[4], const fl
   *codes4 = packed;
 }
 
+// a / b, correctly rounded, from b's correctly rounded reciprocal rb = __frcp_rn(b), for a
+// divisor that serves many dividends (a channel's c, a token's s, the level count L).  With
+// q0 = RN(a rb), each step q <- RN(q + (a - b q) rb) takes the residual by one FMA: the first
+// step leaves q within one unit in the last place of a / b, and from there the residual is exact
+// and the second step yields RN(a / b) (Markstein's theorem on division by a correctly rounded
+// reciprocal).  That needs every intermediate to stay a normal number, which the callers see to:
+// 2^-40 <= |a|, b <= 2^40 (zc_mid), or the bounds stated where it is called.  Anything else
+// (zeros, subnormals, infinities, NaN) takes __fdiv_rn.
+static __device__ __forceinline__ float zc_div_by(float a, float b, float rb) {
+  float q = __fmul_rn(a, rb);
+  q = __fmaf_rn(__fmaf_rn(-b, q, a), rb, q);
+  return __fmaf_rn(__fmaf_rn(-b, q, a), rb, q);
+}
+static __device__ __forceinline__ bool zc_mid(float a) {
+  const float m = fabsf(a);
+  return m >= 0x1p-40f && m <= 0x1p40f;   // false for NaN
+}
+
+// quant_token for a caller that keeps its channels over many tokens: rc[e] = __frcp_rn(c[e]),
+// c_mid = every c[e] passes zc_mid, rL = __frcp_rn(L).  Bit for bit quant_token's results: the
+// same sequence with the divisions taken by zc_div_by where the whole warp's operands allow it
+// (|y| = |x / c| then lies in [2^-80, 2^80], mx - mn is 0 or at least an ulp of 2^-80, and with
+// s in [2^-40, 2^40] the codes' quotients stay below 2^120), by quant_token otherwise.
+static __device__ __noinline__ float4 quant_token_ieee(float4 xv, float4 cv, float L) {   // (s, z, codes, -)
+  const float x[4] = {xv.x, xv.y, xv.z, xv.w}, c[4] = {cv.x, cv.y, cv.z, cv.w};
+  float s, z;
+  unsigned pk;
+  quant_token(x, c, L, &s, &z, &pk);
+  return make_float4(s, z, __uint_as_float(pk), 0.f);
+}
+static __device__ __forceinline__ void quant_token_rc(const float (&x)[4], const float (&c)[4], const float (&rc)[4],
+                                                      bool c_mid, float L, float rL, float* s_out, float* z_out,
+                                                      unsigned* codes4) {
+  const bool mine = c_mid && zc_mid(x[0]) && zc_mid(x[1]) && zc_mid(x[2]) && zc_mid(x[3]);
+  if (__all_sync(0xffffffffu, mine)) {
+    float y[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) y[e] = zc_div_by(x[e], c[e], rc[e]);
+    float mn = fminf(fminf(y[0], y[1]), fminf(y[2], y[3]));
+    float mx = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    float s = zc_div_by(__fsub_rn(mx, mn), L, rL);   // 0 when mx == mn, replaced below
+    if (mx == mn) s = fabsf(mn);                     // mn != 0 here
+    if (zc_mid(s)) {                                 // the same for every lane
+      const float rs = __frcp_rn(s);
+      const float z = -rintf(zc_div_by(mn, s, rs));
+      unsigned packed = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float q = __fadd_rn(rintf(zc_div_by(y[e], s, rs)), z);
+        q = fminf(fmaxf(q, 0.f), L);
+        packed |= ((unsigned)(int)q) << (8 * e);
+      }
+      *s_out = s;
+      *z_out = z;
+      *codes4 = packed;
+      return;
+    }
+  }
+  const float4 r = quant_token_ieee(make_float4(x[0], x[1], x[2], x[3]), make_float4(c[0], c[1], c[2], c[3]), L);
+  *s_out = r.x;
+  *z_out = r.y;
+  *codes4 = __float_as_uint(r.z);
+}
+
 // ChannelQuant (Eq. 5 per channel, Sec. 4.1) of one token's four channels, whose (s, z) the
 // caller holds: code = clamp(rint(x / s_i) + z_i, 0, L), each step one IEEE operation.
 static __device__ __forceinline__ unsigned quant_channel4(const float (&x)[4], const float (&s)[4],
@@ -44,6 +113,21 @@ static __device__ __forceinline__ unsigned quant_channel4(const float (&x)[4], c
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
     float q = __fadd_rn(rintf(__fdiv_rn(x[e], s[e])), z[e]);
+    q = fminf(fmaxf(q, 0.f), L);
+    packed |= ((unsigned)(int)q) << (8 * e);
+  }
+  return packed;
+}
+// quant_channel4 with rs[e] = __frcp_rn(s[e]) and s_mid = every s[e] passes zc_mid: the same
+// codes, the divisions by zc_div_by where this thread's operands allow it.
+static __device__ __forceinline__ unsigned quant_channel4_rc(const float (&x)[4], const float (&s)[4],
+                                                             const float (&rs)[4], bool s_mid,
+                                                             const float (&z)[4], float L) {
+  if (!(s_mid && zc_mid(x[0]) && zc_mid(x[1]) && zc_mid(x[2]) && zc_mid(x[3]))) return quant_channel4(x, s, z, L);
+  unsigned packed = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    float q = __fadd_rn(rintf(zc_div_by(x[e], s[e], rs[e])), z[e]);
     q = fminf(fmaxf(q, 0.f), L);
     packed |= ((unsigned)(int)q) << (8 * e);
   }

@@ -11,8 +11,10 @@ import zc_testlib as tl
 pytestmark = pytest.mark.gpu
 
 
-def _staged_quant_case(w):
+def _staged_quant_case(w, edit=None):
     Q, K, V = make_prefill(w, 0, tl.DEV)
+    if edit is not None:
+        edit(K, V)
     P = tl.probes_for(w)
     oc = tl.make_oracle(w)
     oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
@@ -63,6 +65,44 @@ def test_quantize_degenerate_rows():
     idx = cache.segment(0, 0, 0)[0].cpu().numpy()[0, 0]
     assert tl.salient_sets_match(p_gpu, u.segments[0].p_tilde, idx, u.segments[0].hi.idx, n_s) == 0
     assert tl.compare_segment(cache, oc, 0) == 0
+
+
+def test_quantize_operands_outside_the_kept_reciprocal_range():
+    """The prefill quantiser divides by kept reciprocals only while every operand of the warp
+    lies in 2^-40 .. 2^40 and takes the IEEE division otherwise: zeros, tiny and huge values in
+    single elements, whole tokens and whole channels must give the oracle's bits all the same."""
+    def edit(K, V):
+        K[0, 0, 3, 17] = 0.0                 # one zero element: the token's warp leaves the fast path
+        K[0, 0, 9, :] = 2.0 ** -50           # tiny constant token
+        K[0, 0, 12, 40] = 2.0 ** -60         # tiny element
+        V[0, 0, 20, 5] = 2.0 ** 50           # huge element (its channel's c = 2^25 stays inside)
+        V[0, 0, :, 64] *= 2.0 ** 90          # channel whose c = 2^45-ish lies outside
+        V[0, 1, 33, :] *= 2.0 ** -45         # token whose scale s lies outside
+        K[0, 1, :, 100] *= 2.0 ** -90        # channel with a tiny c
+    _staged_quant_case(tl.small_workload(dtype="bf16", context=300, n_q_heads=2, n_kv_heads=2,
+                                         saliency_ratio=0.5, outlier_fixed=0), edit)
+
+
+def test_division_by_a_kept_reciprocal_is_the_ieee_division():
+    """zc_div_by (the quantiser's a / b from RN(1 / b), two residual steps) against the
+    hardware's IEEE division on 4e9 pseudo-random pairs: operands over the whole admitted range,
+    operands of like magnitude, and quotients at and beside integers and halves, where a wrong
+    last bit would flip a code."""
+    import ctypes as C
+    import os
+    import sys
+    sys.path.insert(0, os.path.join(os.path.dirname(os.path.abspath(__file__)), "helpers"))
+    import build_helpers
+    helper = C.CDLL(build_helpers.build())
+    helper.zct_div_check.restype = C.c_int
+    helper.zct_div_check.argtypes = [C.c_longlong, C.c_ulonglong, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+    bad = torch.zeros(1, dtype=torch.int64, device=tl.DEV)
+    first = torch.zeros(2, dtype=torch.float32, device=tl.DEV)
+    st = torch.cuda.current_stream().cuda_stream
+    for seed, span in ((1, 40), (2, 20), (3, 3), (4, 0)):
+        assert helper.zct_div_check(1_000_000_000, seed, span, bad.data_ptr(), first.data_ptr(), st) == 0
+    torch.cuda.synchronize()
+    assert int(bad.item()) == 0, f"first differing pair: a={first[0].item()!r} b={first[1].item()!r}"
 
 
 @pytest.mark.parametrize("kw", [
