@@ -26,16 +26,20 @@
 namespace {
 
 // What both kernels share: shared memory carved at a 1024-byte boundary, TMEM, barriers.
-// 160 threads: lane 0 of warp 0 issues the MMAs, warps 1..4 are the row workers (they also
-// copy the tiles into shared memory, 16 bytes per thread and row); worker warp w may touch
-// TMEM lanes 32 (w mod 4) .. +31, so together they cover the 128 rows of a tile.
+// 288 threads: lane 0 of warp 0 issues the MMAs, warps 1..8 are the row workers; worker warp w
+// may touch TMEM lanes 32 (w mod 4) .. +31, so warps 1..4 cover the 128 rows of a tile and take
+// the first 64 of its columns, warps 5..8 the same rows and the other 64 (two threads per row:
+// neither pass needs a row's halves together before its end, and eight warps per CTA cover one
+// another's waits where four left the exp2 unit idle a third of the time).  The first 128
+// workers also copy the tiles that do not come by bulk copy (16 bytes per thread and row).
 //   a_full        the A tile has landed
 //   b_full[b]     B buffer b has been filled: by all 128 workers' copies
 //                 (cp.async.mbarrier.arrive) or by the bulk copies (complete_tx)
 //   mma_done[b]   the MMA into accumulator b has completed (tcgen05.commit): the workers may
 //                 read it, and the B buffer it read may be refilled
-//   tmem_free[b]  the four worker warps have read accumulator b: the next MMA may overwrite it
-constexpr int kThreads = 160;
+//   tmem_free[b]  the eight worker warps have read accumulator b: the next MMA may overwrite it
+constexpr int kThreads = 288;
+constexpr int kHalf = kM / 2;      // columns of a tile per worker thread
 struct TcCtx {
   char* As;
   char* Bs;          // two tiles
@@ -44,11 +48,11 @@ struct TcCtx {
   uint64_t* b_full;
   uint64_t* a_full;
   uint32_t* tmem_slot;
-  char* extra;       // pass 2: per worker warp, probe positions and lse of kSide B tiles
+  char* extra;       // pass 2: per worker warp, probe positions and lse of its columns of kSide B tiles
   uint32_t a_addr, b_addr, tmem;
 };
 constexpr int kSide = 3;           // per-column data of pass 2: three tiles per worker warp (see k_probe_colsum)
-constexpr int kTcSmem = 3 * kTile + 1024 /* alignment */ + 128 /* barriers, tmem slot */ + 4 * kSide * kM * 8;
+constexpr int kTcSmem = 3 * kTile + 1024 /* alignment */ + 128 /* barriers, tmem slot */ + 8 * kSide * kHalf * 8;
 
 __device__ __forceinline__ TcCtx tc_setup(char* raw, int a_count, int b_count) {
   TcCtx c;
@@ -68,7 +72,7 @@ __device__ __forceinline__ TcCtx tc_setup(char* raw, int a_count, int b_count) {
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       bar_init(&c.mma_done[i], 1);
-      bar_init(&c.tmem_free[i], 4);
+      bar_init(&c.tmem_free[i], 8);
       bar_init(&c.b_full[i], b_count);
     }
     bar_init(c.a_full, a_count);
@@ -116,16 +120,22 @@ __device__ __forceinline__ void issue_loop(const TcCtx& c, int n, uint32_t idesc
     }
   }
 }
-// Worker: waits for tile cb's accumulator and fetches this thread's row of it.
-__device__ __forceinline__ void worker_fetch(const TcCtx& c, int cb, int quarter, float (&v)[kM]) {
+// Worker: waits for tile cb's accumulator and fetches this thread's half of its row of it.
+__device__ __forceinline__ void worker_fetch(const TcCtx& c, int cb, int quarter, int half, float (&v)[kHalf]) {
   const int buf = cb & 1;
   bar_wait(&c.mma_done[buf], (uint32_t)(cb >> 1) & 1u);
   tc_fence_after();
-  tmem_ld128(v, c.tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * kM);
+  const uint32_t t = c.tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kM + half * kHalf);
+  tmem_ld32_nowait(v, t);
+  tmem_ld32_nowait(v + 32, t + 32);
+  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
   tc_fence_before();
   __syncwarp();
   if ((threadIdx.x & 31) == 0) bar_arrive(&c.tmem_free[buf]);
 }
+
+// The eight worker warps meet (warp 0 does not take part).
+__device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, 256;\n" ::: "memory"); }
 
 // ---- pass 1: row log-sum-exp (base 2) of the causal probe rows ----
 // grid.x: blocks of rph = 128 / Gt probe rows, longest first; grid.y: (batch, group of Gt query heads).
@@ -159,9 +169,11 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
     }
   } else {
     const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
-    const int quarter = warp & 3, row = quarter * 32 + lane;
-    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the 128 workers
+    const int quarter = warp & 3, row = quarter * 32 + lane, half = (warp - 1) >> 2;
+    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the first 128 workers
+    const bool copier = wt < kM;
     auto load_b = [&](int cb) {   // tile cb's keys into B buffer cb & 1
+      if (!copier) return;
 #pragma unroll 4
       for (int i = 0; i < 16; ++i) {
         const int rw = row_ld + 8 * i, j = cb * kM + rw;
@@ -170,14 +182,16 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
       copies_arrive(&c.b_full[cb & 1]);
     };
     // A: the block's probe rows of the Gt heads (it lands with tile 0)
+    if (copier) {
 #pragma unroll 4
-    for (int i = 0; i < 16; ++i) {
-      const int rw = row_ld + 8 * i, hl = rw / rph, r = r0 + rw % rph;
-      const char* src = nullptr;
-      if (r < n_probe) src = reinterpret_cast<const char*>(Q + b * qsb + (h0 + hl) * qsh) + (long long)P[r] * qsl * 2;
-      load_row(c.As, rw, chunk, src);
+      for (int i = 0; i < 16; ++i) {
+        const int rw = row_ld + 8 * i, hl = rw / rph, r = r0 + rw % rph;
+        const char* src = nullptr;
+        if (r < n_probe) src = reinterpret_cast<const char*>(Q + b * qsb + (h0 + hl) * qsh) + (long long)P[r] * qsl * 2;
+        load_row(c.As, rw, chunk, src);
+      }
+      copies_arrive(c.a_full);
     }
-    copies_arrive(c.a_full);
     if (!use_tma) {
       load_b(0);
       if (n_cb > 1) load_b(1);
@@ -187,17 +201,17 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
     const float scale = kLog2e * rsqrtf((float)ZC_D);
     float m_run = -INFINITY, s_run = 0.f;
     for (int cb = 0; cb < n_cb; ++cb) {
-      float v[kM];
-      worker_fetch(c, cb, quarter, v);
+      float v[kHalf];
+      worker_fetch(c, cb, quarter, half, v);
       if (!use_tma && cb + 2 < n_cb) load_b(cb + 2);   // its buffer was read by the MMA that has just completed
-      const int j_base = cb * kM;
+      const int j_base = cb * kM + half * kHalf;
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      if (j_base + kM - 1 <= my_p) {
+      if (j_base + kHalf - 1 <= my_p) {
 #pragma unroll
-        for (int e = 0; e < kM; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
+        for (int e = 0; e < kHalf; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
       } else {
 #pragma unroll
-        for (int e = 0; e < kM; ++e) {
+        for (int e = 0; e < kHalf; ++e) {
           if (j_base + e > my_p) v[e] = -INFINITY;
           mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
         }
@@ -207,12 +221,21 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
       if (mn != -INFINITY) {
         float add[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int e = 0; e < kM; ++e) add[e & 3] += zc_exp2(fmaf(v[e], scale, -mn));
+        for (int e = 0; e < kHalf; ++e) add[e & 3] += zc_exp2(fmaf(v[e], scale, -mn));
         s_run = s_run * zc_exp2(m_run - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
         m_run = mn;
       }
     }
-    if (my_r < n_probe) lse[((long long)b * h_q + h0 + row / rph) * n_probe + my_r] = m_run + log2f(s_run);
+    // the row's two halves (maximum and sum over the even and the odd half-tiles) meet here
+    float2* part = reinterpret_cast<float2*>(c.extra);
+    if (half == 1) part[row] = make_float2(m_run, s_run);
+    workers_sync();
+    if (half == 0 && my_r < n_probe) {
+      const float2 o = part[row];
+      const float mn = fmaxf(m_run, o.x);   // key 0 is in half 0 of tile 0 and every row sees it
+      const float tot = s_run * zc_exp2(m_run - mn) + (o.x == -INFINITY ? 0.f : o.y * zc_exp2(o.x - mn));
+      lse[((long long)b * h_q + h0 + row / rph) * n_probe + my_r] = mn + log2f(tot);
+    }
   }
   tc_teardown(c);
 }
@@ -231,12 +254,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
   // A (the key block): one bulk copy, or the workers; B (probe rows): bulk copies from the
   // gathered copy of the probe rows when there is one (qmap), else the workers gather them
   TcCtx c = tc_setup(smem_raw, use_tma ? 1 : kM, use_qp ? 1 : kM);
-  // Per-column data of a B tile (probe position and lse of each of its 128 rows): every worker
-  // warp keeps its own copy, slot = tile mod 3, written two tiles ahead of its use, so the
-  // warps need no barrier among themselves.
+  // Per-column data of a B tile (probe position and lse of the 64 of its rows that the warp
+  // sums over): every worker warp keeps its own copy, slot = tile mod 3, written two tiles ahead
+  // of its use, so the warps need no barrier among themselves.
   const int wq = (threadIdx.x >> 5) > 0 ? (threadIdx.x >> 5) - 1 : 0;
-  int* Pp = reinterpret_cast<int*>(c.extra + wq * (kSide * kM * 8));   // [kSide][128]
-  float* Ll = reinterpret_cast<float*>(Pp + kSide * kM);                // [kSide][128]
+  int* Pp = reinterpret_cast<int*>(c.extra + wq * (kSide * kHalf * 8));   // [kSide][64]
+  float* Ll = reinterpret_cast<float*>(Pp + kSide * kHalf);                // [kSide][64]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int j0 = blockIdx.x * kM;
   const int unit = blockIdx.y, b = unit / n_kv, kv = unit % n_kv;
@@ -263,11 +286,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     }
   } else {
     const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
-    const int quarter = warp & 3, row = quarter * 32 + lane;
-    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the 128 workers
+    const int quarter = warp & 3, row = quarter * 32 + lane, half = (warp - 1) >> 2;
+    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the first 128 workers
+    const bool copier = wt < kM;
     auto load_b = [&](int tile) {   // tile's probe rows into B buffer tile & 1, its per-column data into its slot
       const int gq = tile / n_rb, rb = tile % n_rb;
-      if (!use_qp) {
+      if (!use_qp && copier) {
         const char* Qb = reinterpret_cast<const char*>(Q + b * qsb + (kv * G + gq) * qsh);
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
@@ -278,13 +302,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
       }
       const int slot = tile % kSide;
 #pragma unroll
-      for (int k = 0; k < kM / 32; ++k) {
-        const int i = lane + 32 * k, r = r_start + rb * kM + i;
-        Pp[slot * kM + i] = r < n_probe ? P[r] : -1;
-        Ll[slot * kM + i] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
+      for (int k = 0; k < kHalf / 32; ++k) {
+        const int i = lane + 32 * k, r = r_start + rb * kM + half * kHalf + i;
+        Pp[slot * kHalf + i] = r < n_probe ? P[r] : -1;
+        Ll[slot * kHalf + i] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
       }
     };
-    if (!use_tma) {
+    if (!use_tma && copier) {
 #pragma unroll 4
       for (int i = 0; i < 16; ++i) {
         const int rw = row_ld + 8 * i, jj = j0 + rw;
@@ -300,28 +324,35 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     float sum4[4] = {0.f, 0.f, 0.f, 0.f};
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int slot = tile % kSide;
-      float v[kM];
-      worker_fetch(c, tile, quarter, v);
+      float v[kHalf];
+      worker_fetch(c, tile, quarter, half, v);
       if (tile + 2 < n_tiles) load_b(tile + 2);   // its buffer was read by the MMA that has just completed
       __syncwarp();   // per-column data written here is read two iterations on
-      const int* pp = Pp + slot * kM;
-      const float* ll = Ll + slot * kM;
-      if (j <= pp[0]) {   // probe rows ascend in position: every row of the tile sees column j
+      const int* pp = Pp + slot * kHalf;
+      const float* ll = Ll + slot * kHalf;
+      if (j <= pp[0]) {   // probe rows ascend in position: every row of the half-tile sees column j
 #pragma unroll
-        for (int e = 0; e < kM; ++e) sum4[e & 3] += zc_exp2(fmaf(v[e], scale, -ll[e]));
+        for (int e = 0; e < kHalf; ++e) sum4[e & 3] += zc_exp2(fmaf(v[e], scale, -ll[e]));
       } else {
 #pragma unroll
-        for (int e = 0; e < kM; ++e) sum4[e & 3] += j <= pp[e] ? zc_exp2(fmaf(v[e], scale, -ll[e])) : 0.f;
+        for (int e = 0; e < kHalf; ++e) sum4[e & 3] += j <= pp[e] ? zc_exp2(fmaf(v[e], scale, -ll[e])) : 0.f;
       }
     }
-    if (j < l) {
+    // the column's two partial sums (over the first and the second 64 rows of every tile) meet
+    float mine = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+    float* part = reinterpret_cast<float*>(c.extra);
+    workers_sync();   // every warp is done with its per-column data: the space is free
+    if (half == 1) part[row] = mine;
+    workers_sync();
+    if (half == 0) mine += part[row];
+    if (half == 0 && j < l) {
       int lo2 = r_start, hi2 = n_probe;   // rows with p_r >= j
       while (lo2 < hi2) {
         const int mid = (lo2 + hi2) >> 1;
         if (P[mid] < j) lo2 = mid + 1; else hi2 = mid;
       }
       float* scores = reinterpret_cast<float*>(cache + unit * unit_stride + off_scores);
-      scores[j] = __fdiv_rn((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]), (float)(G * (n_probe - lo2)));
+      scores[j] = __fdiv_rn(mine, (float)(G * (n_probe - lo2)));
     }
   }
   tc_teardown(c);
