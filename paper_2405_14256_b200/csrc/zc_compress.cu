@@ -218,16 +218,28 @@ __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
 }
 
 // ------------------------------------------------------------------ CSTQuant + pack (arithmetic in zc_quant.cuh)
+template <typename T> __device__ __forceinline__ void raw4(float (&x)[4], uint2 raw) {
+  const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) x[i] = zc_to_float<T>(e[i]);
+}
+
+// One warp = one 16-token sub-block of a tile at a time (a lane: four channels of every token),
+// `rounds` sub-blocks per warp.  K codes leave the registers as words of the canonical order
+// (a shuffle joins the lanes of a word); V codes pass through the warp's own 2 KB of shared
+// memory, from which each lane gathers its words of the fragment order; the tokens' (s, z) are
+// kept by the lane of the token's number.  No barrier of the CTA.
+// grid.x: CTAs of class 0 (8 * rounds sub-blocks each), then of class 1; grid.y: unit.
 template <typename T>
-__global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
-  __shared__ __align__(16) unsigned char codesK[ZC_TILE][ZC_D];
-  __shared__ __align__(16) unsigned char codesV[ZC_TILE][ZC_D];
-  __shared__ __align__(16) float parK[ZC_TILE][2];
-  __shared__ __align__(16) float parV[ZC_TILE][2];
+__global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg, int rounds) {
+  __shared__ __align__(16) unsigned char stageV[8][ZC_SUB][ZC_D];
   const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
-  const int tiles_c0 = zc_ceil_div(seg.n_tok[0], ZC_TILE);
-  const int cls = (int)blockIdx.x < tiles_c0 ? 0 : 1;
-  const int tile = cls == 0 ? blockIdx.x : blockIdx.x - tiles_c0;
+  const int per_tile = ZC_TILE / ZC_SUB;
+  const int subs0 = per_tile * zc_ceil_div(seg.n_tok[0], ZC_TILE);
+  const int ctas0 = zc_ceil_div(subs0, 8 * rounds);
+  const int cls = (int)blockIdx.x < ctas0 ? 0 : 1;
+  const int cta = cls == 0 ? blockIdx.x : blockIdx.x - ctas0;
+  const int subs = per_tile * zc_ceil_div(seg.n_tok[cls], ZC_TILE);   // whole tiles: rows past the end are zero
   const int bits = lay.bits[cls];
   const float L = (float)((1 << bits) - 1);
   char* ub = zc_unit_base(cache, lay, unit);
@@ -236,27 +248,32 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh;
   const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const bool kch = lay.kch != 0;
+  const int sub_bytes = zc_sub_bytes(bits, lay.kch);
+  char* tiles = ub + lay.off_tiles[cls] + (long long)seg.tile0[cls] * lay.tile_bytes[cls];
   if (bits == 16) {
     // 16-bit "quantisation" (the 16/16 and 16/2 settings): the subset's rows are gathered into
     // the tile as they are, [K rows][V rows] per 16-token sub-block; rows past the end are zero
-    char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
-    for (int i = 0; i < 8; ++i) {
-      const int tl = w * 8 + i, tt = tile * ZC_TILE + tl;
-      uint2 k = make_uint2(0, 0), v = make_uint2(0, 0);
-      if (tt < seg.n_tok[cls]) {
-        const long long row = (long long)idx[tt] * src.sl;
-        k = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
-        v = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
+    for (int r = 0; r < rounds; ++r) {
+      const int sb = (cta * rounds + r) * 8 + w;
+      if (sb >= subs) break;
+      char* sub = tiles + (long long)(sb / per_tile) * lay.tile_bytes[cls] + (sb % per_tile) * sub_bytes;
+      for (int i = 0; i < ZC_SUB; ++i) {
+        const int tt = sb * ZC_SUB + i;
+        uint2 k = make_uint2(0, 0), v = make_uint2(0, 0);
+        if (tt < seg.n_tok[cls]) {
+          const long long row = (long long)idx[tt] * src.sl;
+          k = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
+          v = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
+        }
+        reinterpret_cast<uint2*>(sub + i * ZC_D * 2)[lane] = k;
+        reinterpret_cast<uint2*>(sub + (ZC_SUB + i) * ZC_D * 2)[lane] = v;
       }
-      char* sub = tile_ptr + (tl / ZC_SUB) * zc_sub_bytes(16, 0) + (tl % ZC_SUB) * ZC_D * 2;
-      reinterpret_cast<uint2*>(sub)[lane] = k;
-      reinterpret_cast<uint2*>(sub + ZC_SUB * ZC_D * 2)[lane] = v;
     }
     return;
   }
   const unsigned* cmax = reinterpret_cast<const unsigned*>(ub + lay.off_cmax) + cls * 3 * ZC_D;
   float* fac = reinterpret_cast<float*>(ub + lay.off_fac) + (seg.run0 + cls) * ZC_FAC_FLOATS;
-  const bool kch = lay.kch != 0;
   float cK[4], cV[4], zK[4];   // channelwise keys: cK holds the channel scales, zK the zero points
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
@@ -270,7 +287,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     }
     cV[e] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
   }
-  // the divisors that stay for the whole tile: their correctly rounded reciprocals once
+  // the divisors that stay for all of the CTA's tokens: their correctly rounded reciprocals once
   float rK[4], rV[4];
   bool midK = true, midV = true;
 #pragma unroll
@@ -281,7 +298,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     midV = midV && zc_mid(cV[e]);
   }
   const float rL = __frcp_rn(L);
-  if (tile == 0 && w == 0) {
+  if (cta == 0 && w == 0) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       fac[4 * lane + e] = cK[e];
@@ -289,69 +306,115 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
       if (kch) fac[ZC_FAC_ZK + 4 * lane + e] = zK[e];
     }
   }
-  const int t0 = tile * ZC_TILE;
-  // the warp's 8 token rows in two batches of four: gather a batch (memory-level parallelism),
-  // then quantise it
+  const int k_row_bytes = 16 * bits;            // a token's K codes
+  const int v_off = ZC_SUB * k_row_bytes;       // the sub-block's V codes follow its K codes, then the parameters
   float smax = 0.f;
-#pragma unroll 1
-  for (int half = 0; half < 2; ++half) {
-    uint2 rawK[4], rawV[4];
+  for (int r = 0; r < rounds; ++r) {
+    const int sb = (cta * rounds + r) * 8 + w;
+    if (sb >= subs) break;   // the same for the whole warp
+    if (!ZC_CHECKED(seg.tile0[cls] + sb / per_tile < lay.cap_tiles[cls], ZC_DBG_QUANT_TILE)) break;
+    char* sub = tiles + (long long)(sb / per_tile) * lay.tile_bytes[cls] + (sb % per_tile) * sub_bytes;
+    float4 par = make_float4(0.f, 0.f, 0.f, 0.f);   // lane t < 16: (sK, zK, sV, zV) of the sub-block's token t
+    // lane t < 16: the source row of the sub-block's token t (-1 past the end of the subset)
+    int my_row = -1;
+    if (lane < ZC_SUB && sb * ZC_SUB + lane < seg.n_tok[cls]) {
+      my_row = idx[sb * ZC_SUB + lane];
+      if (!ZC_CHECKED(my_row >= 0 && my_row < src.l, ZC_DBG_QUANT_ROW)) my_row = -1;
+    }
+    auto prefetch_batch = [&](int bat) {   // the batch's rows on their way while the one before is quantised
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int tt = t0 + w * 8 + 4 * half + i;
-      if (tt < seg.n_tok[cls] && ZC_CHECKED(idx[tt] >= 0 && idx[tt] < src.l, ZC_DBG_QUANT_ROW)) {
-        const long long row = (long long)idx[tt] * src.sl;
-        rawK[i] = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
-        rawV[i] = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
-      } else {
-        rawK[i] = make_uint2(0, 0);
-        rawV[i] = make_uint2(0, 0);
+      for (int i = 0; i < 4; ++i) {
+        const int rowi = __shfl_sync(0xffffffffu, my_row, 4 * bat + i);
+        if (rowi >= 0) {
+          const long long row = (long long)rowi * src.sl;
+          asm volatile("prefetch.global.L1 [%0];\n" ::"l"(Kb + row + 4 * lane));
+          asm volatile("prefetch.global.L1 [%0];\n" ::"l"(Vb + row + 4 * lane));
+        }
+      }
+    };
+    prefetch_batch(0);
+    // the sub-block's 16 token rows in four batches of four: gather a batch (memory-level
+    // parallelism), then quantise it two rows at a time
+#pragma unroll 1
+    for (int bat = 0; bat < 4; ++bat) {
+      uint2 rawK[4], rawV[4];
+      if (bat + 1 < 4) prefetch_batch(bat + 1);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int rowi = __shfl_sync(0xffffffffu, my_row, 4 * bat + i);
+        if (rowi >= 0) {
+          const long long row = (long long)rowi * src.sl;
+          rawK[i] = *reinterpret_cast<const uint2*>(Kb + row + 4 * lane);
+          rawV[i] = *reinterpret_cast<const uint2*>(Vb + row + 4 * lane);
+        } else {
+          rawK[i] = make_uint2(0, 0);
+          rawV[i] = make_uint2(0, 0);
+        }
+      }
+      // one copy of the pair's code for the batch's two pairs (the kernel is straight-line code
+      // executed once per warp and waits for instruction fetch when it grows)
+#pragma unroll 1
+      for (int pr = 0; pr < 2; ++pr) {
+        const int ta = 4 * bat + 2 * pr;                       // the pair's tokens within the sub-block: ta, ta + 1
+        const bool live_a = sb * ZC_SUB + ta < seg.n_tok[cls], live_b = sb * ZC_SUB + ta + 1 < seg.n_tok[cls];
+        const uint2 rk_a = pr == 0 ? rawK[0] : rawK[2], rk_b = pr == 0 ? rawK[1] : rawK[3];
+        const uint2 rv_a = pr == 0 ? rawV[0] : rawV[2], rv_b = pr == 0 ? rawV[1] : rawV[3];
+        float x[4], sKa = 0.f, zKa = 0.f, sKb = 0.f, zKb = 0.f, sVa, zVa, sVb, zVb;
+        unsigned kA, kB, vA, vB;
+        raw4<T>(x, rk_a);
+        if (kch) kA = quant_channel4_rc(x, cK, rK, midK, zK, L);
+        else quant_token_rc(x, cK, rK, midK, L, rL, &sKa, &zKa, &kA);
+        raw4<T>(x, rk_b);
+        if (kch) kB = quant_channel4_rc(x, cK, rK, midK, zK, L);
+        else quant_token_rc(x, cK, rK, midK, L, rL, &sKb, &zKb, &kB);
+        raw4<T>(x, rv_a);
+        quant_token_rc(x, cV, rV, midV, L, rL, &sVa, &zVa, &vA);
+        raw4<T>(x, rv_b);
+        quant_token_rc(x, cV, rV, midV, L, rL, &sVb, &zVb, &vB);
+        if (!live_a) { kA = 0u; vA = 0u; sKa = zKa = sVa = zVa = 0.f; }
+        if (!live_b) { kB = 0u; vB = 0u; sKb = zKb = sVb = zVb = 0.f; }
+        smax = fmaxf(smax, fmaxf(sVa, sVb));
+        if (lane == ta) par = make_float4(sKa, zKa, sVa, zVa);
+        if (lane == ta + 1) par = make_float4(sKb, zKb, sVb, zVb);
+        // K: straight from the registers
+        bool tok_b, owner;
+        int wr;
+        const unsigned kw = bits == 4 ? zc_k_words(4, kA, kB, lane, &tok_b, &wr, &owner)
+                                      : zc_k_words(2, kA, kB, lane, &tok_b, &wr, &owner);
+        if (owner) *reinterpret_cast<unsigned*>(sub + (ta + (tok_b ? 1 : 0)) * k_row_bytes + 4 * wr) = kw;
+        // V: byte codes into the warp's staging rows
+        *reinterpret_cast<unsigned*>(&stageV[w][ta][4 * lane]) = vA;
+        *reinterpret_cast<unsigned*>(&stageV[w][ta + 1][4 * lane]) = vB;
       }
     }
-    // one copy of the quantiser's code for the batch's four rows (not unrolled: the kernel is
-    // straight-line code executed once per CTA, and what it waits for most is instruction fetch)
-#pragma unroll 1
-    for (int i = 0; i < 4; ++i) {
-      const int tl = w * 8 + 4 * half + i, tt = t0 + tl;
-      const bool live = tt < seg.n_tok[cls];
-      const uint2 rk = i == 0 ? rawK[0] : i == 1 ? rawK[1] : i == 2 ? rawK[2] : rawK[3];
-      const uint2 rv = i == 0 ? rawV[0] : i == 1 ? rawV[1] : i == 2 ? rawV[2] : rawV[3];
-      float x[4], s, z;
-      unsigned pk;
-      const T* ek = reinterpret_cast<const T*>(&rk);
+    __syncwarp();
+    // V: this lane's words of the fragment order, 16 bytes at a time
+    if (bits == 4) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ek[e]);
-      if (kch) {
-        pk = quant_channel4_rc(x, cK, rK, midK, zK, L);
-      } else {
-        quant_token_rc(x, cK, rK, midK, L, rL, &s, &z, &pk);
-        if (lane == 0) { parK[tl][0] = live ? s : 0.f; parK[tl][1] = live ? z : 0.f; }
+      for (int qd = 0; qd < 2; ++qd) {
+        uint4 o;
+        o.x = zc_v_word(4, stageV[w], qd * 128 + lane * 4 + 0);
+        o.y = zc_v_word(4, stageV[w], qd * 128 + lane * 4 + 1);
+        o.z = zc_v_word(4, stageV[w], qd * 128 + lane * 4 + 2);
+        o.w = zc_v_word(4, stageV[w], qd * 128 + lane * 4 + 3);
+        *reinterpret_cast<uint4*>(sub + v_off + (qd * 128 + lane * 4) * 4) = o;
       }
-      *reinterpret_cast<unsigned*>(&codesK[tl][4 * lane]) = live ? pk : 0u;
-      const T* ev = reinterpret_cast<const T*>(&rv);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) x[e] = zc_to_float<T>(ev[e]);
-      quant_token_rc(x, cV, rV, midV, L, rL, &s, &z, &pk);
-      *reinterpret_cast<unsigned*>(&codesV[tl][4 * lane]) = live ? pk : 0u;
-      if (lane == 0) { parV[tl][0] = live ? s : 0.f; parV[tl][1] = live ? z : 0.f; }
-      if (live) smax = fmaxf(smax, s);
+    } else {
+      uint4 o;
+      o.x = zc_v_word(2, stageV[w], lane * 4 + 0);
+      o.y = zc_v_word(2, stageV[w], lane * 4 + 1);
+      o.z = zc_v_word(2, stageV[w], lane * 4 + 2);
+      o.w = zc_v_word(2, stageV[w], lane * 4 + 3);
+      *reinterpret_cast<uint4*>(sub + v_off + lane * 16) = o;
     }
+    // the tokens' parameters: (sK, zK, sV, zV), or (sV, zV) with channelwise keys
+    if (lane < ZC_SUB) {
+      if (kch) *reinterpret_cast<float2*>(sub + 2 * v_off + lane * 8) = make_float2(par.z, par.w);
+      else *reinterpret_cast<float4*>(sub + 2 * v_off + lane * 16) = par;
+    }
+    __syncwarp();   // the staging rows are free for the next sub-block
   }
   if (lane == 0 && smax > 0.f) atomicMax(reinterpret_cast<unsigned*>(&fac[2 * ZC_D]), __float_as_uint(smax));
-  __syncthreads();
-
-  // compose the tile: 16-byte stores, consecutive threads -> consecutive addresses
-  if (!ZC_CHECKED(seg.tile0[cls] + tile < lay.cap_tiles[cls], ZC_DBG_QUANT_TILE)) return;
-  char* tile_ptr = ub + lay.off_tiles[cls] + (long long)(seg.tile0[cls] + tile) * lay.tile_bytes[cls];
-  const int total_vec = lay.tile_bytes[cls] / 16;
-  // one copy per code width, so that the word-building loops have constant trip counts
-  if (bits == 4) {
-    for (int v = threadIdx.x; v < total_vec; v += 256)
-      reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(4, lay.kch, v, 0, codesK, codesV, parK, parV);
-  } else {
-    for (int v = threadIdx.x; v < total_vec; v += 256)
-      reinterpret_cast<uint4*>(tile_ptr)[v] = compose_vec(2, lay.kch, v, 0, codesK, codesV, parK, parV);
-  }
 }
 
 }  // namespace
@@ -373,16 +436,24 @@ int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStre
   k_clear_cmax<<<c->lay.units, 128, 0, st>>>(c->base, c->lay, seg);
   c->launches += 1;
   if (tiles > 0) {
-    dim3 grid(tiles, c->lay.units);
+    // sub-blocks per warp of the quantiser: more than one once the grid is many waves deep (the
+    // set-up of a CTA, its channels' factors and their reciprocals, is then paid less often)
+    const int per_tile = ZC_TILE / ZC_SUB;
+    const long long ctas1 = (long long)zc_ceil_div(tiles * per_tile, 8) * c->lay.units;
+    const long long slots = (long long)c->n_sm * 4;
+    const int rounds = ctas1 >= 16 * slots ? 4 : ctas1 >= 8 * slots ? 2 : 1;
+    dim3 grid(zc_ceil_div(per_tile * zc_ceil_div(seg.n_tok[0], ZC_TILE), 8 * rounds) +
+                  zc_ceil_div(per_tile * zc_ceil_div(seg.n_tok[1], ZC_TILE), 8 * rounds),
+              c->lay.units);
     dim3 grid_max(zc_ceil_div(zc_ceil_div(seg.n_tok[0], ZC_TILE), kAbsTiles) +
                       zc_ceil_div(zc_ceil_div(seg.n_tok[1], ZC_TILE), kAbsTiles),
                   c->lay.units);
     if (c->cfg.dtype == ZC_F16) {
       k_channel_absmax<__half><<<grid_max, 256, 0, st>>>(c->base, c->lay, src, seg);
-      k_quantize_pack<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_quantize_pack<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds);
     } else {
       k_channel_absmax<__nv_bfloat16><<<grid_max, 256, 0, st>>>(c->base, c->lay, src, seg);
-      k_quantize_pack<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg);
+      k_quantize_pack<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds);
     }
     c->launches += 2;
   }

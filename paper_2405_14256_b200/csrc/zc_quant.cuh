@@ -198,3 +198,59 @@ static __device__ __forceinline__ uint4 compose_vec(int bits, int kch, int v, in
   return make_uint4(out[0], out[1], out[2], out[3]);
 }
 
+
+// Word wv of the V codes of one 16-token sub-block (fragment order, as compose_vec lays them
+// out) from the sub-block's byte codes cv[token][channel]; bits is a constant where it is called.
+static __device__ __forceinline__ unsigned zc_v_word(int bits, const unsigned char (*cv)[ZC_D], int wv) {
+  unsigned word = 0;
+  if (bits == 4) {
+    const int qd = wv >> 7, ln = (wv >> 2) & 31, jj = wv & 3;
+    const int j = 4 * qd + jj, g = ln >> 2, t = ln & 3;
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+      const int hi_row = p & 1, isB = (p >> 1) & 1, is1 = p >> 2;
+      word |= (unsigned)cv[2 * t + isB + 8 * is1][16 * j + g + 8 * hi_row] << (4 * p);
+    }
+  } else {
+    const int ln = wv >> 2, m = wv & 3, g = ln >> 2, t = ln & 3;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const int is1 = i >> 3, pp = i & 7, e2 = pp >> 2, hi_row = (pp >> 1) & 1, isB = pp & 1;
+      word |= (unsigned)cv[2 * t + isB + 8 * is1][16 * (2 * m + e2) + g + 8 * hi_row] << (2 * i);
+    }
+  }
+  return word;
+}
+
+// The K codes of two tokens a and b (each lane: its four channels' codes of either, a byte each)
+// as words of the canonical order (a token's row of 4 * bits words, codes ascending from bit 0).
+// Returns this lane's word; *tok_b says which token it belongs to and *wr which word of the
+// row; *owner is false in the lanes that hold no word (2-bit codes: half of them).
+static __device__ __forceinline__ unsigned zc_k_words(int bits, unsigned pk_a, unsigned pk_b, int lane, bool* tok_b,
+                                                      int* wr, bool* owner) {
+  if (bits == 4) {
+    // four codes -> 16 bits per token; the neighbour lane holds the other half of the word
+    const unsigned ta = pk_a | (pk_a >> 4), tb = pk_b | (pk_b >> 4);
+    const unsigned hh = __byte_perm(ta, tb, 0x6420);            // [a: 16 bits][b: 16 bits]
+    const unsigned other = __shfl_xor_sync(0xffffffffu, hh, 1);
+    const bool odd = lane & 1;
+    *tok_b = odd;
+    *wr = lane >> 1;
+    *owner = true;
+    // even lane: a's word = own low half | neighbour's low half << 16; odd lane: b's word =
+    // neighbour's high half | own high half << 16
+    return __byte_perm(hh, other, odd ? 0x3276 : 0x5410);
+  }
+  // four codes -> 8 bits per token; four lanes hold a word
+  const unsigned ta = pk_a | (pk_a >> 6), tb = pk_b | (pk_b >> 6);
+  const unsigned ua = ta | (ta >> 12), ub = tb | (tb >> 12);
+  const unsigned mine = __byte_perm(ua, ub, 0x0040);             // [a byte][b byte][unused][unused]
+  const unsigned nb = __shfl_xor_sync(0xffffffffu, mine, 1);
+  // both lanes of a pair: [a even lane][b even lane][a odd lane][b odd lane]
+  const unsigned v = (lane & 1) ? __byte_perm(nb, mine, 0x5410) : __byte_perm(mine, nb, 0x5410);
+  const unsigned v2 = __shfl_xor_sync(0xffffffffu, v, 2);
+  *tok_b = lane & 1;
+  *wr = lane >> 2;
+  *owner = (lane & 2) == 0;
+  return __byte_perm(v, v2, (lane & 1) ? 0x7531 : 0x6420);
+}
