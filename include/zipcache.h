@@ -40,6 +40,16 @@ enum { ZC_F16 = 0, ZC_BF16 = 1 };
  * taken over the tokens of a subset, one (s, z) pair per channel and none per token, which
  * saves 8 bytes per cached token. */
 enum { ZC_K_CST = 0, ZC_K_CHANNEL = 1 };
+/* Who shares a saliency decision (Sec. 4.2 speaks of the saliency "of each token"; the paper
+ * does not say how heads are combined).  ZC_SCOPE_KV_HEAD: one decision per (batch row, KV head)
+ * from that head's own normalised scores (Eq. 8 over its query heads).  ZC_SCOPE_TOKEN: one
+ * decision per token of a batch row, shared by all its KV heads: the token's score is the mean
+ * of its per-KV-head normalised scores, in the prompt and in every re-compressed window, so
+ * every head of the row keeps the same tokens at the higher precision.  With ZC_SCOPE_TOKEN the
+ * window is re-compressed by kernels of its own that follow the decode kernel of the call that
+ * completes it (the heads' statistics must meet first), so it cannot be combined with
+ * ZC_FLAG_OVERLAP_CALLS (zc_cache_bytes / zc_cache_init return ZC_EINVAL). */
+enum { ZC_SCOPE_KV_HEAD = 0, ZC_SCOPE_TOKEN = 1 };
 
 enum {
   ZC_OK = 0,
@@ -99,7 +109,7 @@ typedef struct {
   double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
   int32_t k_scheme;       /* quantiser of the keys: ZC_K_CST (Alg. 1 on K and V) or ZC_K_CHANNEL
                              (channelwise keys, Sec. 4.1 last paragraph / Alg. 2; values stay CST) */
-  int32_t reserved;       /* must be 0 */
+  int32_t scope;          /* ZC_SCOPE_KV_HEAD (0) or ZC_SCOPE_TOKEN: who shares a saliency decision */
 } zc_config;
 
 typedef struct zc_cache zc_cache; /* small host-side handle */

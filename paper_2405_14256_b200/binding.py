@@ -16,6 +16,7 @@ ZC_FLAG_DEFER_APPEND = 1
 ZC_FLAG_OVERLAP_CALLS = 2
 ZC_FLAG_OUT_F32 = 4
 ZC_K_CST, ZC_K_CHANNEL = 0, 1
+ZC_SCOPE_KV_HEAD, ZC_SCOPE_TOKEN = 0, 1
 
 
 class ZipCacheError(RuntimeError):
@@ -28,17 +29,17 @@ class ZcConfig(C.Structure):
         ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
         ("max_prefill", C.c_int32), ("max_new_tokens", C.c_int32), ("window", C.c_int32),
         ("bits_hi", C.c_int32), ("bits_lo", C.c_int32), ("flags", C.c_int32),
-        ("saliency_ratio", C.c_double), ("k_scheme", C.c_int32), ("reserved", C.c_int32),
+        ("saliency_ratio", C.c_double), ("k_scheme", C.c_int32), ("scope", C.c_int32),
     ]
 
     @classmethod
     def make(cls, dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
              saliency_ratio, bits_hi=4, bits_lo=2, window=100, head_dim=128,
-             flags=0, k_scheme=0) -> "ZcConfig":
+             flags=0, k_scheme=0, scope=0) -> "ZcConfig":
         code = {torch.float16: ZC_F16, torch.bfloat16: ZC_BF16}.get(dtype, dtype)
         return cls(C.sizeof(cls), code, batch, n_q_heads, n_kv_heads, head_dim, max_prefill,
                    max_new_tokens, window, bits_hi, bits_lo, flags, float(saliency_ratio),
-                   int(k_scheme), 0)
+                   int(k_scheme), int(scope))
 
 
 _lib = None
@@ -276,7 +277,7 @@ class ZipCache:
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
                  workspace: Optional[torch.Tensor] = None, defer_append: bool = False,
                  overlap_calls: bool = False, out_f32: bool = False, k_channel: bool = False,
-                 guard_bytes: int = 0):
+                 guard_bytes: int = 0, token_scope: bool = False):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
@@ -284,7 +285,8 @@ class ZipCache:
                                  flags=(ZC_FLAG_DEFER_APPEND if defer_append else 0) |
                                  (ZC_FLAG_OVERLAP_CALLS if overlap_calls else 0) |
                                  (ZC_FLAG_OUT_F32 if out_f32 else 0),
-                                 k_scheme=ZC_K_CHANNEL if k_channel else ZC_K_CST)
+                                 k_scheme=ZC_K_CHANNEL if k_channel else ZC_K_CST,
+                                 scope=ZC_SCOPE_TOKEN if token_scope else ZC_SCOPE_KV_HEAD)
         self.k_channel = bool(k_channel)
         self.out_dtype = torch.float32 if out_f32 else dtype
         self.dtype, self.device = dtype, torch.device(device)

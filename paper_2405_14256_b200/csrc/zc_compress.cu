@@ -217,6 +217,32 @@ __global__ void k_clear_cmax(char* cache, ZcLayout lay, ZcSeg seg) {
   if (threadIdx.x < 2) fac[(seg.run0 + threadIdx.x) * ZC_FAC_FLOATS + 2 * ZC_D] = 0.f;  // smaxV
 }
 
+// ------------------------------------------------------------------ token-level saliency (ZC_SCOPE_TOKEN)
+// scores[b][kv][j] <- mean over the KV heads of batch row b of scores[b][.][j], j < n: every head
+// of the row then makes the same split.  grid.x: blocks of 256 tokens; grid.y: batch row.
+__global__ void k_share_scores(char* cache, ZcLayout lay, int n) {
+  const int j = blockIdx.x * 256 + threadIdx.x, b = blockIdx.y;
+  if (j >= n) return;
+  float sum = 0.f;
+  for (int kv = 0; kv < lay.n_kv; ++kv)
+    sum = __fadd_rn(sum, reinterpret_cast<const float*>(zc_unit_base(cache, lay, b * lay.n_kv + kv) + lay.off_scores)[j]);
+  const float mean = __fdiv_rn(sum, (float)lay.n_kv);
+  for (int kv = 0; kv < lay.n_kv; ++kv)
+    reinterpret_cast<float*>(zc_unit_base(cache, lay, b * lay.n_kv + kv) + lay.off_scores)[j] = mean;
+}
+
+// The completed window's normalised scores of every unit (Eq. 8 on the collected probe rows:
+// column sum / (G * rows that saw the token)); the statistics start from zero for the next
+// window.  The same two steps open the re-compression inside the decode kernel.
+__global__ void k_window_scores(char* cache, ZcLayout lay, ZcFlushArgs fl) {
+  char* ub = zc_unit_base(cache, lay, blockIdx.x);
+  const int tid = threadIdx.x;
+  if (tid >= lay.window) return;
+  float* colsum = reinterpret_cast<float*>(ub + lay.off_colsum);
+  reinterpret_cast<float*>(ub + lay.off_scores)[tid] = __fdiv_rn(colsum[tid], (float)(lay.G * max(1, (int)fl.nnz[tid])));
+  colsum[tid] = 0.f;
+}
+
 // ------------------------------------------------------------------ CSTQuant + pack (arithmetic in zc_quant.cuh)
 template <typename T> __device__ __forceinline__ void raw4(float (&x)[4], uint2 raw) {
   const T* e = reinterpret_cast<const T*>(&raw);
@@ -427,6 +453,18 @@ int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* give
     if (e != cudaSuccess) return e;
   }
   k_topk_split<<<c->lay.units, kTopkThreads, (size_t)smem, st>>>(c->base, c->lay, n, n_s, idx_off, given_sal);
+  c->launches += 1;
+  return (int)cudaGetLastError();
+}
+
+int zc_launch_share_scores(zc_cache* c, int n, cudaStream_t st) {
+  k_share_scores<<<dim3(zc_ceil_div(n, 256), c->cfg.batch), 256, 0, st>>>(c->base, c->lay, n);
+  c->launches += 1;
+  return (int)cudaGetLastError();
+}
+
+int zc_launch_window_scores(zc_cache* c, const ZcFlushArgs& fl, cudaStream_t st) {
+  k_window_scores<<<c->lay.units, ZC_MAX_WINDOW, 0, st>>>(c->base, c->lay, fl);
   c->launches += 1;
   return (int)cudaGetLastError();
 }

@@ -30,7 +30,10 @@ int check_config(const zc_config* cfg) {
   if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32)) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if (cfg->k_scheme != ZC_K_CST && cfg->k_scheme != ZC_K_CHANNEL) return ZC_EINVAL;
-  if (cfg->reserved != 0) return ZC_EINVAL;
+  if (cfg->scope != ZC_SCOPE_KV_HEAD && cfg->scope != ZC_SCOPE_TOKEN) return ZC_EINVAL;
+  // token scope re-compresses a window by kernels that follow the decode kernel: every call must
+  // then wait for what precedes it on the stream
+  if (cfg->scope == ZC_SCOPE_TOKEN && (cfg->flags & ZC_FLAG_OVERLAP_CALLS)) return ZC_EINVAL;
   if ((long long)cfg->batch * cfg->n_kv_heads > 65535) return ZC_EINVAL;
   // every re-compressed window adds two items to a decode call
   if (2 * (cfg->max_new_tokens / cfg->window) + 2 + 2 > ZC_MAX_ITEMS) return ZC_EINVAL;
@@ -379,6 +382,8 @@ static int prefill_compress(zc_cache* c, const void* Q, const void* K, const voi
     void* qp = used < workspace_bytes ? (char*)workspace + used : nullptr;
     ZC_CUDA(zc_launch_probe_scores(c, Q, K, l, q_strides, kv_strides, P_dev, n_probe, lse, qp,
                                    qp ? workspace_bytes - used : 0, row_lse, st));
+    // one decision per token of a batch row: the mean of its KV heads' scores, for every head
+    if (c->cfg.scope == ZC_SCOPE_TOKEN) ZC_CUDA(zc_launch_share_scores(c, l, st));
   }
   ZC_CUDA(zc_launch_topk(c, l, c->n0[0], 0, salient_idx, st));
   ZcSrc src{K, V, kv_strides[0], kv_strides[1], kv_strides[2], l};
@@ -470,13 +475,25 @@ static int decode_attention(zc_cache* c, const void* q, void* out, int is_probe_
   const bool completes = fresh && c->n_tail == c->cfg.window;
   ZcFlushArgs fl;
   memset(&fl, 0, sizeof(fl));
+  const bool token_scope = c->cfg.scope == ZC_SCOPE_TOKEN;
   if (completes) {
-    fl.on = 1;
+    fl.on = token_scope ? 0 : 1;   // token scope: by kernels of their own, below
     fl.seg = zc_segment(c, c->n_seg);
     for (int j = 0; j < c->n_tail; ++j) fl.nnz[j] = (unsigned char)(c->tail_nnz[j] + (collect ? 1 : 0));
   }
   ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (char*)workspace, workspace_bytes, pk, pv,
                            completes ? &fl : nullptr, st));
+  if (completes && token_scope) {
+    // The window's scores of all KV heads of a batch row meet before the split: scores from
+    // the statistics the decode kernels collected, their mean over the row's heads, then the
+    // prompt's own split and quantise kernels with the tail as their source.
+    ZC_CUDA(zc_launch_window_scores(c, fl, st));
+    ZC_CUDA(zc_launch_share_scores(c, c->cfg.window, st));
+    ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], fl.seg.idx_off, nullptr, st));
+    const int64_t sh = (int64_t)(c->lay.unit_stride / 2);   // elements from one unit's tail to the next
+    ZcSrc src{c->base + c->lay.off_tailK, c->base + c->lay.off_tailV, sh * c->lay.n_kv, sh, ZC_D, c->cfg.window};
+    ZC_CUDA(zc_launch_quantize(c, src, fl.seg, st));
+  }
   // Alg. 3 bookkeeping: the step counter follows the tokens of the current window
   if (fresh && c->n_tail > 0) {
     c->step_i = i_next;

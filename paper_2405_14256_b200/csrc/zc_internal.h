@@ -168,6 +168,8 @@ int zc_attention_error_code(int* out);   // 0 or 1: a bounded wait in the prefil
 int zc_launch_topk(zc_cache* c, int n, int n_s, int idx_off, const int32_t* given_sal,
                    cudaStream_t st);
 int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStream_t st);
+int zc_launch_share_scores(zc_cache* c, int n, cudaStream_t st);
+int zc_launch_window_scores(zc_cache* c, const ZcFlushArgs& fl, cudaStream_t st);
 int zc_launch_append(zc_cache* c, const void* k_new, const void* v_new, int pos,
                      cudaStream_t st);
 // k_new / v_new non-null: the newest tail row is read from them and stored into the tail.

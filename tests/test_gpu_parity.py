@@ -730,3 +730,74 @@ def test_prefill_attention_full_size_config2():
         worst_l = max(worst_l, float(np.abs(lse[bi, h].double().cpu().numpy() - lse_ref).max()))
     assert worst_o <= 2e-2 and worst_l <= 2e-4, (worst_o, worst_l)
     tl.record("prefill attention, full size (3 heads)", config=2, max_abs_out=worst_o, score_rel=worst_l)
+
+
+# ---------------------------------------------------------------- token-level saliency (ZC_SCOPE_TOKEN)
+@pytest.mark.parametrize("kw", [
+    dict(context=300, batch=2, n_q_heads=8, n_kv_heads=4),
+    dict(context=515, batch=1, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0),
+    dict(context=130, batch=2, n_q_heads=4, n_kv_heads=4, k_scheme="channel"),
+])
+def test_token_scope_prefill_one_split_per_batch_row(kw):
+    """ZC_SCOPE_TOKEN: a token's score is the mean of its KV heads' normalised scores, every
+    head of a batch row makes the same split, and codes, parameters and factors are the
+    oracle's (scope="token") bit for bit."""
+    w = tl.small_workload(**kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w, scope="token")
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w, token_scope=True)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    p_gpu = cache.scores(w.context).cpu().numpy()
+    idx_hi = cache.segment(0, 0, 0)[0].cpu().numpy()
+    for bi in range(w.batch):
+        for kv in range(w.n_kv_heads):
+            s0 = oc.units[(bi, kv)].segments[0]
+            rel = np.abs(p_gpu[bi, kv] - s0.p_tilde) / np.maximum(np.abs(s0.p_tilde), 1e-30)
+            assert rel.max() <= 1e-4, rel.max()
+            np.testing.assert_array_equal(p_gpu[bi, kv], p_gpu[bi, 0])       # one score per token of the row
+            np.testing.assert_array_equal(idx_hi[bi, kv], idx_hi[bi, 0])     # one split per row
+            assert tl.salient_sets_match(p_gpu[bi, kv], s0.p_tilde, idx_hi[bi, kv], s0.hi.idx, s0.hi.n) == 0
+    assert tl.compare_segment(cache, oc, 0) == 0
+
+
+@pytest.mark.parametrize("defer", [False, True])
+def test_token_scope_decode_across_two_windows(defer):
+    """The window's re-compression under ZC_SCOPE_TOKEN (kernels of their own after the decode
+    kernel of the completing call): outputs within the bound at every step, the two new
+    segments' lists, codes and parameters equal to the oracle's, one split per batch row."""
+    w = tl.small_workload(context=200, batch=2, n_q_heads=8, n_kv_heads=4, window=16, decode_steps=40,
+                          rho_recent=0.2, rho_random=0.2)
+    from workloads import make_decode_step
+    import paper_2405_14256_b200 as zc
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w, scope="token")
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w, max_new=40, defer_append=defer, token_scope=True)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    worst = 0.0
+    for step in range(36):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        probe = step % 3 == 0
+        cache.append(k, v)
+        out = cache.decode_attention(q, probe)
+        oc.append(tl.to64(k), tl.to64(v))
+        ref = oc.decode_attention(tl.to64(q), probe)
+        torch.cuda.synchronize()
+        got = out.float().cpu().numpy()
+        for (bi, kv), r in ref.items():
+            g = got[bi, kv * oc.G:(kv + 1) * oc.G]
+            assert tl.output_excess(g, r, w.torch_dtype) <= 0.0
+            worst = max(worst, float(np.abs(g - r).max()))
+    assert zc.zc_num_segments(cache.handle) == 3 and zc.zc_tail_tokens(cache.handle) == 4
+    assert zc.zc_device_status() == 0
+    for seg in (1, 2):
+        idx_hi = cache.segment(seg, 0, 0)[0].cpu().numpy()
+        for bi in range(w.batch):
+            for kv in range(w.n_kv_heads):
+                np.testing.assert_array_equal(idx_hi[bi, kv], idx_hi[bi, 0])
+        assert tl.compare_segment(cache, oc, seg) == 0
+    cache.check_guards()
