@@ -217,6 +217,15 @@ def algorithmic_prefill_bytes(w) -> int:
     return per_unit * w.units_per_layer
 
 
+EXP2_PER_S_PEAK = 148 * 16 * 1.965e9   # the exp2 unit: 16 results per clock and SM, 148 SMs at the maximum SM clock
+
+
+def prefill_exponentials(w, probes) -> float:
+    """exp2 evaluations the probe scores of one layer need (Eq. 9): every probe row's causal
+    keys, for every query head, in both passes (row log-sum-exp, then the normalised columns)."""
+    return 2.0 * float(sum(p + 1 for p in probes)) * w.n_q_heads * w.batch
+
+
 def oracle_sample(w, n_units: int, n_steps: int, layer: int = 0, prefilled=None):
     """Times the oracle on `n_units` units of the workload: prefill compression and `n_steps`
     decode steps.  Returns a dict; `threads` is what the oracle really used (process CPU time
@@ -544,6 +553,10 @@ def measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, modes, 
                      "sm_mhz": clocks.get("sm_mhz"), "reasons": clocks.get("reasons")}
         res["prefill_tokens_per_s"] = pre_tps
         res["prefill_roofline_frac"] = (R * algorithmic_prefill_bytes(w) / (t_pre * 1e-3) / 1e9) / peak
+        # prefill compression is bound by the exponentials of the probe scores, not by bytes: the
+        # share of the exp2 unit's peak that the whole of prefill compression sustains
+        res["prefill_exp2_frac"] = (sum(prefill_exponentials(w, wb.probes[i]) for i in range(R)) /
+                                    (t_pre * 1e-3)) / EXP2_PER_S_PEAK
     if not override and world == 1:
         res["prefill_attention"] = measure_prefill_attention(zc, wb, w, R)
     assert zc.zc_device_status() == 0, "a bounded wait inside a kernel ran out"
