@@ -27,17 +27,20 @@ namespace {
 
 // What both kernels share: shared memory carved at a 1024-byte boundary, TMEM, barriers.
 // 288 threads: lane 0 of warp 0 issues the MMAs, warps 1..8 are the row workers; worker warp w
-// may touch TMEM lanes 32 (w mod 4) .. +31, so warps 1..4 cover the 128 rows of a tile and take
-// the first 64 of its columns, warps 5..8 the same rows and the other 64 (two threads per row:
-// neither pass needs a row's halves together before its end, and eight warps per CTA cover one
-// another's waits where four left the exp2 unit idle a third of the time).  The first 128
-// workers also copy the tiles that do not come by bulk copy (16 bytes per thread and row).
+// may touch TMEM lanes 32 (w mod 4) .. +31, so warps 1..4 cover the 128 rows of a tile and so do
+// warps 5..8: the first group works on the even tiles (accumulator 0), the second on the odd
+// ones (accumulator 1), a thread taking its row in two halves of 64 columns.  Two threads per
+// row: neither pass needs a row's tiles together before its end, where the groups meet once
+// through shared memory; and the groups are at different points of their tiles at any time, so
+// one group's exponentials run while the other waits or loads (with all eight warps on the same
+// tile the exp2 unit idled while they all waited).  A group's 128 threads also copy the tiles of
+// its accumulator that do not come by bulk copy (16 bytes per thread and row).
 //   a_full        the A tile has landed
 //   b_full[b]     B buffer b has been filled: by all 128 workers' copies
 //                 (cp.async.mbarrier.arrive) or by the bulk copies (complete_tx)
 //   mma_done[b]   the MMA into accumulator b has completed (tcgen05.commit): the workers may
 //                 read it, and the B buffer it read may be refilled
-//   tmem_free[b]  the eight worker warps have read accumulator b: the next MMA may overwrite it
+//   tmem_free[b]  the four worker warps of group b have read accumulator b: the next MMA may overwrite it
 constexpr int kThreads = 288;
 constexpr int kHalf = kM / 2;      // columns of a tile per worker thread
 struct TcCtx {
@@ -48,16 +51,24 @@ struct TcCtx {
   uint64_t* b_full;
   uint64_t* a_full;
   uint32_t* tmem_slot;
-  char* extra;       // pass 2: per worker warp, probe positions and lse of its columns of kSide B tiles
+  char* extra;       // pass 2: per worker warp, probe positions and lse of the rows of kSide B tiles
   uint32_t a_addr, b_addr, tmem;
+  bool bad;          // the tiles would not fit behind the alignment padding: nothing was set up
 };
-constexpr int kSide = 3;           // per-column data of pass 2: three tiles per worker warp (see k_probe_colsum)
-constexpr int kTcSmem = 3 * kTile + 1024 /* alignment */ + 128 /* barriers, tmem slot */ + 8 * kSide * kHalf * 8;
+constexpr int kSide = 2;           // per-column data of pass 2: two tiles per worker warp (see k_probe_colsum)
+constexpr int kTcSlack = 768;      // what aligning the tiles to 1 KB may take (the base is declared 1 KB aligned)
+constexpr int kTcSmem = 3 * kTile + kTcSlack + 128 /* barriers, tmem slot */ + 8 * kSide * kM * 8;
+static_assert(kTcSmem <= 115712, "two CTAs per SM");
 
 __device__ __forceinline__ TcCtx tc_setup(char* raw, int a_count, int b_count) {
   TcCtx c;
   const uint32_t raw_u = zc_smem_u32(raw);
   const uint32_t base_u = (raw_u + 1023u) & ~1023u;
+  c.bad = base_u - raw_u > (uint32_t)kTcSlack;
+  if (c.bad) {
+    if (threadIdx.x == 0) atomicExch(&g_zc_tc_error, 3);
+    return c;
+  }
   char* base = raw + (base_u - raw_u);
   c.As = base;
   c.Bs = base + kTile;
@@ -72,7 +83,7 @@ __device__ __forceinline__ TcCtx tc_setup(char* raw, int a_count, int b_count) {
   if (threadIdx.x == 0) {
     for (int i = 0; i < 2; ++i) {
       bar_init(&c.mma_done[i], 1);
-      bar_init(&c.tmem_free[i], 8);
+      bar_init(&c.tmem_free[i], 4);
       bar_init(&c.b_full[i], b_count);
     }
     bar_init(c.a_full, a_count);
@@ -120,18 +131,22 @@ __device__ __forceinline__ void issue_loop(const TcCtx& c, int n, uint32_t idesc
     }
   }
 }
-// Worker: waits for tile cb's accumulator and fetches this thread's half of its row of it.
-__device__ __forceinline__ void worker_fetch(const TcCtx& c, int cb, int quarter, int half, float (&v)[kHalf]) {
-  const int buf = cb & 1;
-  bar_wait(&c.mma_done[buf], (uint32_t)(cb >> 1) & 1u);
+// Worker: waits for tile cb's accumulator; fetches one half (64 columns) of this thread's row of
+// it; after the second half, gives the accumulator back.
+__device__ __forceinline__ void worker_wait(const TcCtx& c, int cb) {
+  bar_wait(&c.mma_done[cb & 1], (uint32_t)(cb >> 1) & 1u);
   tc_fence_after();
-  const uint32_t t = c.tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kM + half * kHalf);
+}
+__device__ __forceinline__ void worker_load(const TcCtx& c, int cb, int quarter, int half, float (&v)[kHalf]) {
+  const uint32_t t = c.tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((cb & 1) * kM + half * kHalf);
   tmem_ld32_nowait(v, t);
   tmem_ld32_nowait(v + 32, t + 32);
   asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void worker_release(const TcCtx& c, int cb) {
   tc_fence_before();
   __syncwarp();
-  if ((threadIdx.x & 31) == 0) bar_arrive(&c.tmem_free[buf]);
+  if ((threadIdx.x & 31) == 0) bar_arrive(&c.tmem_free[cb & 1]);
 }
 
 // The eight worker warps meet (warp 0 does not take part).
@@ -148,9 +163,10 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
                                                              float* __restrict__ lse,
                                                              const __grid_constant__ CUtensorMap kmap,
                                                              int use_tma) {
-  extern __shared__ char smem_raw[];
+  extern __shared__ __align__(1024) char smem_raw[];
   // A (gathered probe rows): the 128 workers' copies; B (key tiles): bulk copies, or the workers
   TcCtx c = tc_setup(smem_raw, kM, use_tma ? 1 : kM);
+  if (c.bad) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int rph = kM / Gt;
   const int r0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * rph;   // rows ascend in position: long blocks first
@@ -169,11 +185,10 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
     }
   } else {
     const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
-    const int quarter = warp & 3, row = quarter * 32 + lane, half = (warp - 1) >> 2;
-    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the first 128 workers
-    const bool copier = wt < kM;
-    auto load_b = [&](int cb) {   // tile cb's keys into B buffer cb & 1
-      if (!copier) return;
+    const int quarter = warp & 3, row = quarter * 32 + lane, grp = (warp - 1) >> 2;   // grp: tiles of this parity
+    const int wt = (tid - 32) & (kM - 1), row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of a group's 128 workers
+    const bool copier = grp == 0;                                              // of the A tile
+    auto load_b = [&](int cb) {   // tile cb's keys into B buffer cb & 1, by the group of that parity
 #pragma unroll 4
       for (int i = 0; i < 16; ++i) {
         const int rw = row_ld + 8 * i, j = cb * kM + rw;
@@ -192,18 +207,19 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
       }
       copies_arrive(c.a_full);
     }
-    if (!use_tma) {
-      load_b(0);
-      if (n_cb > 1) load_b(1);
-    }
+    if (!use_tma && grp < n_cb) load_b(grp);
     const int my_r = r0 + row % rph;
     const int my_p = my_r < n_probe ? P[my_r] : -1;
     const float scale = kLog2e * rsqrtf((float)ZC_D);
     float m_run = -INFINITY, s_run = 0.f;
-    for (int cb = 0; cb < n_cb; ++cb) {
-      float v[kHalf];
-      worker_fetch(c, cb, quarter, half, v);
+    for (int cb = grp; cb < n_cb; cb += 2) {
+      worker_wait(c, cb);
       if (!use_tma && cb + 2 < n_cb) load_b(cb + 2);   // its buffer was read by the MMA that has just completed
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+      float v[kHalf];
+      worker_load(c, cb, quarter, half, v);
+      if (half == 1) worker_release(c, cb);
       const int j_base = cb * kM + half * kHalf;
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       if (j_base + kHalf - 1 <= my_p) {
@@ -225,14 +241,15 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
         s_run = s_run * zc_exp2(m_run - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
         m_run = mn;
       }
+      }
     }
-    // the row's two halves (maximum and sum over the even and the odd half-tiles) meet here
+    // the row's two partial results (maximum and sum over the even and over the odd tiles) meet here
     float2* part = reinterpret_cast<float2*>(c.extra);
-    if (half == 1) part[row] = make_float2(m_run, s_run);
+    if (grp == 1) part[row] = make_float2(m_run, s_run);
     workers_sync();
-    if (half == 0 && my_r < n_probe) {
+    if (grp == 0 && my_r < n_probe) {
       const float2 o = part[row];
-      const float mn = fmaxf(m_run, o.x);   // key 0 is in half 0 of tile 0 and every row sees it
+      const float mn = fmaxf(m_run, o.x);   // key 0 is in tile 0 and every row sees it
       const float tot = s_run * zc_exp2(m_run - mn) + (o.x == -INFINITY ? 0.f : o.y * zc_exp2(o.x - mn));
       lse[((long long)b * h_q + h0 + row / rph) * n_probe + my_r] = mn + log2f(tot);
     }
@@ -250,16 +267,17 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     long long ksl, const float* __restrict__ lse, char* cache, long long unit_stride, long long off_scores,
     const __grid_constant__ CUtensorMap kmap, int use_tma, const __grid_constant__ CUtensorMap qmap,
     int use_qp) {
-  extern __shared__ char smem_raw[];
+  extern __shared__ __align__(1024) char smem_raw[];
   // A (the key block): one bulk copy, or the workers; B (probe rows): bulk copies from the
   // gathered copy of the probe rows when there is one (qmap), else the workers gather them
   TcCtx c = tc_setup(smem_raw, use_tma ? 1 : kM, use_qp ? 1 : kM);
-  // Per-column data of a B tile (probe position and lse of the 64 of its rows that the warp
-  // sums over): every worker warp keeps its own copy, slot = tile mod 3, written two tiles ahead
-  // of its use, so the warps need no barrier among themselves.
+  if (c.bad) return;
+  // Per-column data of a B tile (probe position and lse of its 128 rows): every worker warp
+  // keeps its own copy of its group's tiles, slot = (tile / 2) mod 2, written while the warp's
+  // tile before it is worked on, so the warps need no barrier among themselves.
   const int wq = (threadIdx.x >> 5) > 0 ? (threadIdx.x >> 5) - 1 : 0;
-  int* Pp = reinterpret_cast<int*>(c.extra + wq * (kSide * kHalf * 8));   // [kSide][64]
-  float* Ll = reinterpret_cast<float*>(Pp + kSide * kHalf);                // [kSide][64]
+  int* Pp = reinterpret_cast<int*>(c.extra + wq * (kSide * kM * 8));   // [kSide][128]
+  float* Ll = reinterpret_cast<float*>(Pp + kSide * kM);                // [kSide][128]
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int j0 = blockIdx.x * kM;
   const int unit = blockIdx.y, b = unit / n_kv, kv = unit % n_kv;
@@ -286,12 +304,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
     }
   } else {
     const char* Kb = reinterpret_cast<const char*>(K + b * ksb + kv * ksh);
-    const int quarter = warp & 3, row = quarter * 32 + lane, half = (warp - 1) >> 2;
-    const int wt = tid - 32, row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of the first 128 workers
-    const bool copier = wt < kM;
-    auto load_b = [&](int tile) {   // tile's probe rows into B buffer tile & 1, its per-column data into its slot
+    const int quarter = warp & 3, row = quarter * 32 + lane, grp = (warp - 1) >> 2;   // grp: tiles of this parity
+    const int wt = (tid - 32) & (kM - 1), row_ld = wt >> 4, chunk = wt & 15;   // 8 rows per pass of a group's 128 workers
+    const bool copier = grp == 0;                                              // of the A tile
+    auto load_b = [&](int tile) {   // tile's probe rows into B buffer tile & 1 (by the group of that parity), its per-column data into the warp's slot
       const int gq = tile / n_rb, rb = tile % n_rb;
-      if (!use_qp && copier) {
+      if (!use_qp) {
         const char* Qb = reinterpret_cast<const char*>(Q + b * qsb + (kv * G + gq) * qsh);
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
@@ -300,12 +318,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
         }
         copies_arrive(&c.b_full[tile & 1]);
       }
-      const int slot = tile % kSide;
+      const int slot = (tile >> 1) % kSide;
 #pragma unroll
-      for (int k = 0; k < kHalf / 32; ++k) {
-        const int i = lane + 32 * k, r = r_start + rb * kM + half * kHalf + i;
-        Pp[slot * kHalf + i] = r < n_probe ? P[r] : -1;
-        Ll[slot * kHalf + i] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
+      for (int k = 0; k < kM / 32; ++k) {
+        const int i = lane + 32 * k, r = r_start + rb * kM + i;
+        Pp[slot * kM + i] = r < n_probe ? P[r] : -1;
+        Ll[slot * kM + i] = r < n_probe ? lse[((long long)b * h_q + kv * G + gq) * n_probe + r] : INFINITY;
       }
     };
     if (!use_tma && copier) {
@@ -316,20 +334,23 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
       }
       copies_arrive(c.a_full);
     }
-    load_b(0);
-    if (n_tiles > 1) load_b(1);
-    __syncwarp();   // per-column data of tiles 0 and 1 is visible to the warp
+    if (grp < n_tiles) load_b(grp);
+    __syncwarp();   // per-column data of the warp's first tile is visible to the warp
     const int j = j0 + row;
     const float scale = kLog2e * rsqrtf((float)ZC_D);
     float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int tile = 0; tile < n_tiles; ++tile) {
-      const int slot = tile % kSide;
-      float v[kHalf];
-      worker_fetch(c, tile, quarter, half, v);
+    for (int tile = grp; tile < n_tiles; tile += 2) {
+      const int slot = (tile >> 1) % kSide;
+      worker_wait(c, tile);
       if (tile + 2 < n_tiles) load_b(tile + 2);   // its buffer was read by the MMA that has just completed
-      __syncwarp();   // per-column data written here is read two iterations on
-      const int* pp = Pp + slot * kHalf;
-      const float* ll = Ll + slot * kHalf;
+      __syncwarp();   // per-column data written here is read in the warp's next iteration
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+      float v[kHalf];
+      worker_load(c, tile, quarter, half, v);
+      if (half == 1) worker_release(c, tile);
+      const int* pp = Pp + slot * kM + half * kHalf;
+      const float* ll = Ll + slot * kM + half * kHalf;
       if (j <= pp[0]) {   // probe rows ascend in position: every row of the half-tile sees column j
 #pragma unroll
         for (int e = 0; e < kHalf; ++e) sum4[e & 3] += zc_exp2(fmaf(v[e], scale, -ll[e]));
@@ -337,15 +358,16 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
 #pragma unroll
         for (int e = 0; e < kHalf; ++e) sum4[e & 3] += j <= pp[e] ? zc_exp2(fmaf(v[e], scale, -ll[e])) : 0.f;
       }
+      }
     }
-    // the column's two partial sums (over the first and the second 64 rows of every tile) meet
+    // the column's two partial sums (over the even and over the odd tiles) meet
     float mine = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
     float* part = reinterpret_cast<float*>(c.extra);
     workers_sync();   // every warp is done with its per-column data: the space is free
-    if (half == 1) part[row] = mine;
+    if (grp == 1) part[row] = mine;
     workers_sync();
-    if (half == 0) mine += part[row];
-    if (half == 0 && j < l) {
+    if (grp == 0) mine += part[row];
+    if (grp == 0 && j < l) {
       int lo2 = r_start, hi2 = n_probe;   // rows with p_r >= j
       while (lo2 < hi2) {
         const int mid = (lo2 + hi2) >> 1;
