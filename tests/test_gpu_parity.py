@@ -666,6 +666,11 @@ def test_a_second_decode_call_on_the_same_tail_leaves_the_window_bookkeeping_alo
     dict(context=129, n_q_heads=2, n_kv_heads=1),
     dict(context=300, batch=2, n_q_heads=8, n_kv_heads=2),
     dict(context=1000, n_q_heads=4, n_kv_heads=4, outlier_fixed=0),
+    # around the kernel's blocks of 256 query rows (two groups of 128) and its 128-key tiles
+    dict(context=256, n_q_heads=2, n_kv_heads=1),
+    dict(context=257, n_q_heads=2, n_kv_heads=2),
+    dict(context=385, n_q_heads=4, n_kv_heads=2),
+    dict(context=640, n_q_heads=2, n_kv_heads=1),
 ])
 def test_prefill_attention_output_and_row_lse(dtype, kw):
     """O = causal Softmax(Q K^T / sqrt(d)) V and every row's log-sum-exp against the oracle's
