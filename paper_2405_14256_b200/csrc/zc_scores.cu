@@ -217,30 +217,30 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_lse(const T* __restrict__
       if (!use_tma && cb + 2 < n_cb) load_b(cb + 2);   // its buffer was read by the MMA that has just completed
 #pragma unroll 1
       for (int half = 0; half < 2; ++half) {
-      float v[kHalf];
-      worker_load(c, cb, quarter, half, v);
-      if (half == 1) worker_release(c, cb);
-      const int j_base = cb * kM + half * kHalf;
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      if (j_base + kHalf - 1 <= my_p) {
+        float v[kHalf];
+        worker_load(c, cb, quarter, half, v);
+        if (half == 1) worker_release(c, cb);
+        const int j_base = cb * kM + half * kHalf;
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (j_base + kHalf - 1 <= my_p) {
 #pragma unroll
-        for (int e = 0; e < kHalf; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
-      } else {
+          for (int e = 0; e < kHalf; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
+        } else {
 #pragma unroll
-        for (int e = 0; e < kHalf; ++e) {
-          if (j_base + e > my_p) v[e] = -INFINITY;
-          mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
+          for (int e = 0; e < kHalf; ++e) {
+            if (j_base + e > my_p) v[e] = -INFINITY;
+            mx4[e & 3] = fmaxf(mx4[e & 3], v[e]);
+          }
         }
-      }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      const float mn = fmaxf(m_run, mx * scale);
-      if (mn != -INFINITY) {
-        float add[4] = {0.f, 0.f, 0.f, 0.f};
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        const float mn = fmaxf(m_run, mx * scale);
+        if (mn != -INFINITY) {
+          float add[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int e = 0; e < kHalf; ++e) add[e & 3] += zc_exp2(fmaf(v[e], scale, -mn));
-        s_run = s_run * zc_exp2(m_run - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
-        m_run = mn;
-      }
+          for (int e = 0; e < kHalf; ++e) add[e & 3] += zc_exp2(fmaf(v[e], scale, -mn));
+          s_run = s_run * zc_exp2(m_run - mn) + ((add[0] + add[1]) + (add[2] + add[3]));
+          m_run = mn;
+        }
       }
     }
     // the row's two partial results (maximum and sum over the even and over the odd tiles) meet here
@@ -346,18 +346,18 @@ __global__ void __launch_bounds__(kThreads, 2) k_probe_colsum(
       __syncwarp();   // per-column data written here is read in the warp's next iteration
 #pragma unroll 1
       for (int half = 0; half < 2; ++half) {
-      float v[kHalf];
-      worker_load(c, tile, quarter, half, v);
-      if (half == 1) worker_release(c, tile);
-      const int* pp = Pp + slot * kM + half * kHalf;
-      const float* ll = Ll + slot * kM + half * kHalf;
-      if (j <= pp[0]) {   // probe rows ascend in position: every row of the half-tile sees column j
+        float v[kHalf];
+        worker_load(c, tile, quarter, half, v);
+        if (half == 1) worker_release(c, tile);
+        const int* pp = Pp + slot * kM + half * kHalf;
+        const float* ll = Ll + slot * kM + half * kHalf;
+        if (j <= pp[0]) {   // probe rows ascend in position: every row of the half-tile sees column j
 #pragma unroll
-        for (int e = 0; e < kHalf; ++e) sum4[e & 3] += zc_exp2(fmaf(v[e], scale, -ll[e]));
-      } else {
+          for (int e = 0; e < kHalf; ++e) sum4[e & 3] += zc_exp2(fmaf(v[e], scale, -ll[e]));
+        } else {
 #pragma unroll
-        for (int e = 0; e < kHalf; ++e) sum4[e & 3] += j <= pp[e] ? zc_exp2(fmaf(v[e], scale, -ll[e])) : 0.f;
-      }
+          for (int e = 0; e < kHalf; ++e) sum4[e & 3] += j <= pp[e] ? zc_exp2(fmaf(v[e], scale, -ll[e])) : 0.f;
+        }
       }
     }
     // the column's two partial sums (over the even and over the odd tiles) meet
