@@ -667,7 +667,7 @@ def main():
     ap.add_argument("--append", default="deferred", choices=["deferred", "kernel"],
                     help="deferred: zc_append hands the new row to the next zc_decode_attention "
                          "(ZC_FLAG_DEFER_APPEND); kernel: zc_append copies with its own launch")
-    ap.add_argument("--bits", default="", help="H/L bit pair instead of the workload's 4/2 (2, 4 or 16 each)")
+    ap.add_argument("--bits", default="", help="H/L bit pair instead of the workload's 4/2 (2, 4, 8 or 16 each; not 8 with 16)")
     ap.add_argument("--saliency", type=float, default=-1.0, help="saliency ratio instead of the workload's")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -713,7 +713,8 @@ def main():
             pairs = {}
             for name, ov in (("4/4 all salient", dict(bits_hi=4, bits_lo=4, saliency_ratio=1.0)),
                              ("16/2 15.2% salient", dict(bits_hi=16, bits_lo=2, saliency_ratio=0.152)),
-                             ("2/2", dict(bits_hi=2, bits_lo=2))):
+                             ("2/2", dict(bits_hi=2, bits_lo=2)),
+                             ("8/4", dict(bits_hi=8, bits_lo=4))):
                 rr = measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, ["overlap"],
                                     headline=False, **ov)["per_config"]
                 pairs[name] = {"us_per_call": rr["overlap"]["us_per_call"], "frac": rr["overlap"]["frac"],

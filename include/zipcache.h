@@ -102,9 +102,10 @@ typedef struct {
   int32_t max_new_tokens; /* decode capacity (tokens appended after prefill) */
   int32_t window;         /* tokens kept at full precision before re-compression
                              (Alg. 3 uses 100); 8 <= window <= ZC_MAX_WINDOW */
-  int32_t bits_hi;        /* bit-width of salient tokens: 4, 2, or 16 (kept as they are: the
+  int32_t bits_hi;        /* bit-width of salient tokens: 8, 4, 2, or 16 (kept as they are: the
                              "16/16" and "16/2" settings of Table 3) */
-  int32_t bits_lo;        /* bit-width of regular tokens: 4, 2 or 16 */
+  int32_t bits_lo;        /* bit-width of regular tokens: 8, 4, 2 or 16; a cache with an 8-bit
+                             class cannot also have a 16-bit one (ZC_EINVAL) */
   int32_t flags;          /* 0 or an OR of the ZC_FLAG_* values above */
   double saliency_ratio;  /* r in [0,1]; n_salient = floor(r * n) */
   int32_t k_scheme;       /* quantiser of the keys: ZC_K_CST (Alg. 1 on K and V) or ZC_K_CHANNEL

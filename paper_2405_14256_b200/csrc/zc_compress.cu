@@ -403,11 +403,16 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
         if (lane == ta) par = make_float4(sKa, zKa, sVa, zVa);
         if (lane == ta + 1) par = make_float4(sKb, zKb, sVb, zVb);
         // K: straight from the registers
-        bool tok_b, owner;
-        int wr;
-        const unsigned kw = bits == 4 ? zc_k_words(4, kA, kB, lane, &tok_b, &wr, &owner)
-                                      : zc_k_words(2, kA, kB, lane, &tok_b, &wr, &owner);
-        if (owner) *reinterpret_cast<unsigned*>(sub + (ta + (tok_b ? 1 : 0)) * k_row_bytes + 4 * wr) = kw;
+        if (bits == 8) {   // a lane's four codes are a word of the row
+          *reinterpret_cast<unsigned*>(sub + ta * k_row_bytes + 4 * lane) = kA;
+          *reinterpret_cast<unsigned*>(sub + (ta + 1) * k_row_bytes + 4 * lane) = kB;
+        } else {
+          bool tok_b, owner;
+          int wr;
+          const unsigned kw = bits == 4 ? zc_k_words(4, kA, kB, lane, &tok_b, &wr, &owner)
+                                        : zc_k_words(2, kA, kB, lane, &tok_b, &wr, &owner);
+          if (owner) *reinterpret_cast<unsigned*>(sub + (ta + (tok_b ? 1 : 0)) * k_row_bytes + 4 * wr) = kw;
+        }
         // V: byte codes into the warp's staging rows
         *reinterpret_cast<unsigned*>(&stageV[w][ta][4 * lane]) = vA;
         *reinterpret_cast<unsigned*>(&stageV[w][ta + 1][4 * lane]) = vB;
@@ -415,7 +420,17 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     }
     __syncwarp();
     // V: this lane's words of the fragment order, 16 bytes at a time
-    if (bits == 4) {
+    if (bits == 8) {
+#pragma unroll 1
+      for (int q = 0; q < 4; ++q) {
+        uint4 o;
+        o.x = zc_v_word(8, stageV[w], q * 128 + lane * 4 + 0);
+        o.y = zc_v_word(8, stageV[w], q * 128 + lane * 4 + 1);
+        o.z = zc_v_word(8, stageV[w], q * 128 + lane * 4 + 2);
+        o.w = zc_v_word(8, stageV[w], q * 128 + lane * 4 + 3);
+        *reinterpret_cast<uint4*>(sub + v_off + (q * 128 + lane * 4) * 4) = o;
+      }
+    } else if (bits == 4) {
 #pragma unroll
       for (int qd = 0; qd < 2; ++qd) {
         uint4 o;

@@ -211,7 +211,13 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 // B-fragment register (2 * k-step + {0: k = 2t,2t+1; 1: k = 2t+8,2t+9}), half e of it, and the
 // inverse of the power of two that the matching masked code carries.
 template <int BITS> __device__ __forceinline__ void chan_slot(int off, int* reg, int* e, float* inv_sigma) {
-  if (BITS == 4) {
+  if (BITS == 8) {
+    // a word = four channels = one k-step: bytes 0, 2 are k = 2t, 2t+1; bytes 1, 3 are k = 2t+8, 2t+9
+    const int jw = off >> 2, b = off & 3;
+    *reg = 2 * jw + (b & 1);
+    *e = b >> 1;
+    *inv_sigma = 1.f;
+  } else if (BITS == 4) {
     const int jw = off >> 3, hi = (off >> 2) & 1, hb = (off >> 1) & 1, odd = off & 1;
     *reg = 2 * (2 * jw + hb) + odd;
     *e = hi;
@@ -277,7 +283,20 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const char* sh = st + h * SB;
-    if (BITS == 4) {
+    if (BITS == 8) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const uint4 a = *reinterpret_cast<const uint4*>(sh + lane * 32 + 16 * q);
+        const uint4 b = *reinterpret_cast<const uint4*>(sh + 1024 + lane * 32 + 16 * q);
+        kw[h][0][4 * q] = a.x; kw[h][0][4 * q + 1] = a.y; kw[h][0][4 * q + 2] = a.z; kw[h][0][4 * q + 3] = a.w;
+        kw[h][1][4 * q] = b.x; kw[h][1][4 * q + 1] = b.y; kw[h][1][4 * q + 2] = b.z; kw[h][1][4 * q + 3] = b.w;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 c = *reinterpret_cast<const uint4*>(sh + 2048 + q * 512 + lane * 16);
+        vw[h][4 * q] = c.x; vw[h][4 * q + 1] = c.y; vw[h][4 * q + 2] = c.z; vw[h][4 * q + 3] = c.w;
+      }
+    } else if (BITS == 4) {
       const uint4 a = *reinterpret_cast<const uint4*>(sh + lane * 16);
       const uint4 b = *reinterpret_cast<const uint4*>(sh + 512 + lane * 16);
       kw[h][0][0] = a.x; kw[h][0][1] = a.y; kw[h][0][2] = a.z; kw[h][0][3] = a.w;
@@ -309,7 +328,15 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     float dacc[4];
-    if (BITS == 4) {
+    if (BITS == 8) {
+#pragma unroll
+      for (int jw = 0; jw < 8; ++jw) {   // one word per token = one k-step
+        const uint32_t w0 = kw[h][0][jw], w1 = kw[h][1][jw];
+        const uint32_t a0[4] = {w0 & 0x00FF00FFu, w1 & 0x00FF00FFu, shr8(w0) & 0x00FF00FFu, shr8(w1) & 0x00FF00FFu};
+        if (jw == 0) zc_mma16816_z(dacc, a0, qb[0], qb[1]);
+        else zc_mma16816<__half>(dacc, a0, qb[2 * jw], qb[2 * jw + 1]);
+      }
+    } else if (BITS == 4) {
 #pragma unroll
       for (int jw = 0; jw < 4; ++jw) {
         const uint32_t w0 = kw[h][0][jw], w1 = kw[h][1][jw];
@@ -394,7 +421,14 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
   // ---- O^T += V^T(128 channels x 16 tokens) . P^T per half: 8 M-tiles ----
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    if (BITS == 4) {
+    if (BITS == 8) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {   // channel rows g and g + 8 in a word each; bytes = tokens 2t, 2t+1, 2t+8, 2t+9
+        const uint32_t w0 = vw[h][2 * j], w1 = vw[h][2 * j + 1];
+        const uint32_t a[4] = {w0 & 0x00FF00FFu, w1 & 0x00FF00FFu, shr8(w0) & 0x00FF00FFu, shr8(w1) & 0x00FF00FFu};
+        zc_mma16816<__half>(oacc[j], a, pb[h][0], pb[h][1]);
+      }
+    } else if (BITS == 4) {
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const uint32_t w = vw[h][j], x = shr8(w);
@@ -573,7 +607,8 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
 #pragma unroll
   for (int ks = 0; ks < 8; ++ks) {
     uint32_t one_lo, one_hi;
-    if (BITS == 4) { one_lo = 0x00010001u; one_hi = 0x00100010u; }
+    if (BITS == 8) { one_lo = 0x00010001u; one_hi = 0x00010001u; }
+    else if (BITS == 4) { one_lo = 0x00010001u; one_hi = 0x00100010u; }
     else if ((ks & 1) == 0) { one_lo = 0x00010001u; one_hi = 0x00040004u; }
     else { one_lo = 0x00100010u; one_hi = 0x00400040u; }
     const uint32_t a[4] = {one_lo, one_lo, one_hi, one_hi};
@@ -627,7 +662,7 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
   // o[ch] = c^V[ch] 2^-logK (acc 2^24 / sigma(row) - z sum); rows g+8 of a tile carry sigma = 16
   ItemScale r;
   r.chan_factor = cV * zc_exp2(-logK);
-  r.rowscale = (tid & 8) ? 1048576.f : 16777216.f;
+  r.rowscale = (BITS != 8 && (tid & 8)) ? 1048576.f : 16777216.f;   // 8-bit codes carry no power of two
   return r;
 }
 
@@ -967,7 +1002,7 @@ constexpr int kFlushSmem = kFlOffSmax + 16;
 static_assert(kFlushSmem <= decode_smem(kRingNarrow), "the re-compression must fit the item phase's memory");
 static_assert(ZC_MAX_WINDOW == 32 * kWarps, "one thread per window token");
 
-template <typename T, bool KCH, bool RAW>
+template <typename T, bool KCH, bool RAW, bool B8>
 __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay, const ZcFlushArgs& fl, char* smem) {
   auto codesK = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesK);
   auto codesV = reinterpret_cast<unsigned char (*)[ZC_D]>(smem + kFlOffCodesV);
@@ -1162,7 +1197,9 @@ __device__ __forceinline__ void window_flush_unit(char* ub, const ZcLayout& lay,
                        (long long)(fl.seg.tile0[cls] + sb / (ZC_TILE / ZC_SUB)) * lay.tile_bytes[cls];
       for (int v = tid; v < vecs; v += 128)
         reinterpret_cast<uint4*>(tile_ptr)[sub_in_tile * vecs + v] =
-            compose_vec(bits, kch, sub_in_tile * vecs + v, ZC_SUB * sub_in_tile, codesK, codesV, parK, parV);
+            (B8 && bits == 8)
+                ? compose_vec8(kch, sub_in_tile * vecs + v, ZC_SUB * sub_in_tile, codesK, codesV, parK, parV)
+                : compose_vec(bits, kch, sub_in_tile * vecs + v, ZC_SUB * sub_in_tile, codesK, codesV, parK, parV);
       __syncthreads();   // the next sub-block reuses the code arrays
     }
     if (lane == 0 && smax > 0.f) atomicMax(&s_smax[cls], __float_as_uint(smax));
@@ -1270,7 +1307,7 @@ __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_t
 // and its arrival counter.
 // RAW: the build that also serves a class kept at 16 bits (kept apart so that the 4- and 2-bit
 // kernels are compiled exactly as they are without it).
-template <typename T, int RING, int NCTA, bool KCH, bool RAW>
+template <typename T, int RING, int NCTA, bool KCH, bool RAW, bool B8 = false>
 __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay, ZcDecodePlan plan,
                                                       const T* __restrict__ q, T* __restrict__ out,
                                                       float* part, float* stash_all, int slot,
@@ -1374,7 +1411,9 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     if (has) {
       const float* fac = reinterpret_cast<const float*>(ub + lay.off_fac) + d.run * ZC_FAC_FLOATS;
       const char* class_base = ub + lay.off_tiles[d.cls];
-      if (lay.bits[d.cls] == 4)
+      if (B8 && lay.bits[d.cls] == 8)
+        sc = compressed_item<T, 8, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
+      else if (lay.bits[d.cls] == 4)
         sc = compressed_item<T, 4, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
       else if (!RAW || lay.bits[d.cls] == 2)
         sc = compressed_item<T, 2, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
@@ -1443,7 +1482,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
                   lay.out_f32 ? reinterpret_cast<float*>(out) + out_off : nullptr, mine, stash_g, collect, smem);
     if (fl.on) {
       __syncthreads();   // the merge is done with the shared arrays; its additions to the statistics are visible
-      window_flush_unit<T, KCH, RAW>(ub, lay, fl, smem);
+      window_flush_unit<T, KCH, RAW, B8>(ub, lay, fl, smem);
     }
   }
 }
@@ -1597,7 +1636,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   const int groups = (plan.items + plan.cta_items - 1) / plan.cta_items;
   const dim3 grid((unsigned)(c->lay.units * (groups * zs + (plan.fold_tail ? 0 : 1)) + 1));
   cudaError_t e;
-#define ZC_LAUNCH_STEP(T, RING, NCTA, KCH, RAW)                                                        \
+#define ZC_LAUNCH_STEP(T, RING, NCTA, KCH, RAW, B8)                                                    \
   do {                                                                                             \
     /* the opt-in to large shared memory is per device and per kernel: one bit per device */       \
     static std::atomic<unsigned long long> attr_done{0};                                           \
@@ -1605,12 +1644,12 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
     cudaGetDevice(&dev_now);                                                                       \
     const unsigned long long bit = 1ull << (dev_now & 63);                                         \
     if (!(attr_done.load(std::memory_order_acquire) & bit)) {                                      \
-      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA, KCH, RAW>,                                  \
+      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA, KCH, RAW, B8>,                              \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));    \
       if (e != cudaSuccess) return e;                                                              \
       attr_done.fetch_or(bit, std::memory_order_release);                                          \
     }                                                                                              \
-    e = launch_pdl(k_decode<T, RING, NCTA, KCH, RAW>, grid, dim3(128), decode_smem(RING), st,      \
+    e = launch_pdl(k_decode<T, RING, NCTA, KCH, RAW, B8>, grid, dim3(128), decode_smem(RING), st,  \
                    overlap,                                                                        \
                    c->base, c->lay, plan, (const T*)q, (T*)out, part, stash, slot, collect,        \
                    (const T*)k_new, (const T*)v_new, ord, fl);                                     \
@@ -1618,15 +1657,19 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
 #define ZC_LAUNCH_T(T)                                                                             \
   do {                                                                                             \
     const bool raw = c->lay.bits[0] == 16 || c->lay.bits[1] == 16;                                 \
-    if (raw) { /* a class kept at 16 bits: one build (narrow rings, 4 CTAs per SM) */              \
-      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, true);                               \
-      else ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, true);                                         \
+    const bool b8 = c->lay.bits[0] == 8 || c->lay.bits[1] == 8;                                    \
+    if (b8) { /* an 8-bit class: one build (wide rings hold one pair of its sub-tiles, 3 CTAs per SM) */ \
+      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingWide, 3, true, false, true);                          \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false, true);                                    \
+    } else if (raw) { /* a class kept at 16 bits: one build (narrow rings, 4 CTAs per SM) */       \
+      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, true, false);                        \
+      else ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, true, false);                                  \
     } else if (c->lay.kch) {                                                                       \
-      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, false);                   \
-      else ZC_LAUNCH_STEP(T, kRingWide, 3, true, false);                                           \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, false, false);            \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, true, false, false);                                    \
     } else {                                                                                       \
-      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, false);                  \
-      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false);                                          \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, false, false);           \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false, false);                                   \
     }                                                                                              \
   } while (0)
   if (c->cfg.dtype == ZC_F16) ZC_LAUNCH_T(__half);

@@ -25,8 +25,10 @@ int check_config(const zc_config* cfg) {
   if (cfg->max_prefill < 1 || cfg->max_prefill > (1 << 20)) return ZC_EINVAL;
   if (cfg->max_new_tokens < 0) return ZC_EINVAL;
   if (cfg->window < 8 || cfg->window > ZC_MAX_WINDOW) return ZC_EINVAL;
-  if (cfg->bits_hi != 4 && cfg->bits_hi != 2 && cfg->bits_hi != 16) return ZC_EINVAL;
-  if (cfg->bits_lo != 4 && cfg->bits_lo != 2 && cfg->bits_lo != 16) return ZC_EINVAL;
+  if (cfg->bits_hi != 4 && cfg->bits_hi != 2 && cfg->bits_hi != 8 && cfg->bits_hi != 16) return ZC_EINVAL;
+  if (cfg->bits_lo != 4 && cfg->bits_lo != 2 && cfg->bits_lo != 8 && cfg->bits_lo != 16) return ZC_EINVAL;
+  // an 8-bit class and a class kept at 16 bits have separate builds of the decode kernel
+  if ((cfg->bits_hi == 8 || cfg->bits_lo == 8) && (cfg->bits_hi == 16 || cfg->bits_lo == 16)) return ZC_EINVAL;
   if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32)) return ZC_EINVAL;
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if (cfg->k_scheme != ZC_K_CST && cfg->k_scheme != ZC_K_CHANNEL) return ZC_EINVAL;

@@ -32,7 +32,11 @@ __host__ __device__ inline void zc_vcode_pos(int bits, int tau, int ch, int* wor
   int j = ch >> 4, rho = ch & 15, g = rho & 7, hi_row = rho >> 3;
   int is1 = tau >> 3, tp = tau & 7, t = tp >> 1, isB = tp & 1;
   int lane = g * 4 + t;
-  if (bits == 4) {
+  if (bits == 8) {
+    // two words per lane and 16-channel group: channel row g, then g + 8; bytes = tokens 2t, 2t+1, 2t+8, 2t+9
+    *word = (j >> 1) * 128 + lane * 4 + 2 * (j & 1) + hi_row;
+    *shift = 8 * (isB + 2 * is1);
+  } else if (bits == 4) {
     int p = hi_row + 2 * isB + 4 * is1;
     *word = (j >> 2) * 128 + lane * 4 + (j & 3);
     *shift = 4 * p;

@@ -203,7 +203,12 @@ static __device__ __forceinline__ uint4 compose_vec(int bits, int kch, int v, in
 // out) from the sub-block's byte codes cv[token][channel]; bits is a constant where it is called.
 static __device__ __forceinline__ unsigned zc_v_word(int bits, const unsigned char (*cv)[ZC_D], int wv) {
   unsigned word = 0;
-  if (bits == 4) {
+  if (bits == 8) {
+    const int q = wv >> 7, ln = (wv >> 2) & 31, i = wv & 3;
+    const int ch = 16 * (2 * q + (i >> 1)) + (ln >> 2) + 8 * (i & 1), t = ln & 3;
+    word = (unsigned)cv[2 * t][ch] | (unsigned)cv[2 * t + 1][ch] << 8 | (unsigned)cv[2 * t + 8][ch] << 16 |
+           (unsigned)cv[2 * t + 9][ch] << 24;
+  } else if (bits == 4) {
     const int qd = wv >> 7, ln = (wv >> 2) & 31, jj = wv & 3;
     const int j = 4 * qd + jj, g = ln >> 2, t = ln & 3;
 #pragma unroll
@@ -253,4 +258,36 @@ static __device__ __forceinline__ unsigned zc_k_words(int bits, unsigned pk_a, u
   *wr = lane >> 2;
   *owner = (lane & 2) == 0;
   return __byte_perm(v, v2, (lane & 1) ? 0x7531 : 0x6420);
+}
+
+// compose_vec for 8-bit codes (a K row is the codes themselves, four to a word; V words as
+// zc_vcode_pos lays them out).  Kept apart so that the builds without an 8-bit class stay as
+// they are.
+static __device__ __forceinline__ uint4 compose_vec8(int kch, int v, int row0, const unsigned char (*codesK)[ZC_D],
+                                                     const unsigned char (*codesV)[ZC_D], const float (*parK)[2],
+                                                     const float (*parV)[2]) {
+  const int sub_words = zc_sub_bytes(8, kch) / 4;
+  unsigned out[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int wi = 4 * v + q;
+    const int st = wi / sub_words, wl = wi % sub_words;
+    unsigned word;
+    if (wl < 512) {
+      const int tok = 16 * st - row0 + (wl >> 5);
+      word = *reinterpret_cast<const unsigned*>(&codesK[tok][4 * (wl & 31)]);
+    } else if (wl < 1024) {
+      word = zc_v_word(8, codesV + (16 * st - row0), wl - 512);
+    } else {
+      const int wp = wl - 1024;
+      if (kch) {
+        word = __float_as_uint(parV[16 * st - row0 + (wp >> 1)][wp & 1]);
+      } else {
+        const int tk = 16 * st - row0 + (wp >> 2), f = wp & 3;
+        word = __float_as_uint(f < 2 ? parK[tk][f] : parV[tk][f - 2]);
+      }
+    }
+    out[q] = word;
+  }
+  return make_uint4(out[0], out[1], out[2], out[3]);
 }

@@ -56,7 +56,7 @@ def test_cache_bytes_cover_the_algorithmic_bytes(zc):
 
 
 @pytest.mark.parametrize("bad", [
-    dict(head_dim=64), dict(bits_hi=8), dict(bits_lo=3), dict(k_scheme=2), dict(window=4), dict(window=129),
+    dict(head_dim=64), dict(bits_hi=5), dict(bits_lo=3), dict(bits_hi=16, bits_lo=8), dict(k_scheme=2), dict(window=4), dict(window=129),
     dict(saliency_ratio=1.5), dict(n_q_heads=6), dict(batch=0), dict(n_q_heads=72, n_kv_heads=8),
     dict(scope=2), dict(scope=1, flags=2),   # token scope cannot be combined with ZC_FLAG_OVERLAP_CALLS (2)
 ])

@@ -36,7 +36,7 @@ def test_quantize_pack_bit_exact_edge_lengths(l, ratio):
 
 
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
-@pytest.mark.parametrize("bits", [(4, 2), (4, 4), (2, 2), (2, 4)])
+@pytest.mark.parametrize("bits", [(4, 2), (4, 4), (2, 2), (2, 4), (8, 8), (8, 4), (8, 2), (4, 8)])
 def test_quantize_pack_bit_exact_bit_pairs(dtype, bits):
     _staged_quant_case(tl.small_workload(dtype=dtype, context=333, batch=2, n_q_heads=8,
                                          n_kv_heads=2, bits_hi=bits[0], bits_lo=bits[1],
@@ -167,6 +167,12 @@ def test_topk_ties_prefer_lower_index():
     (dict(context=1, n_q_heads=1, n_kv_heads=1), 2),
     (dict(context=200, n_q_heads=4, n_kv_heads=1, bits_hi=4, bits_lo=4), 3),
     (dict(context=200, n_q_heads=4, n_kv_heads=1, bits_hi=2, bits_lo=2), 3),
+    # 8-bit codes (a build of the decode kernel of their own), with each of the other widths
+    (dict(context=200, n_q_heads=4, n_kv_heads=1, bits_hi=8, bits_lo=8), 3),
+    (dict(context=333, batch=2, n_q_heads=8, n_kv_heads=2, bits_hi=8, bits_lo=4, dtype="bf16", outlier_fixed=0), 4),
+    (dict(context=515, n_q_heads=4, n_kv_heads=4, bits_hi=8, bits_lo=2), 5),
+    (dict(context=70, n_q_heads=2, n_kv_heads=2, bits_hi=4, bits_lo=8, saliency_ratio=0.5), 3),
+    (dict(context=300, n_q_heads=4, n_kv_heads=2, bits_hi=8, bits_lo=2, k_scheme="channel"), 4),
 ])
 def test_decode_attention_parity(kw, steps):
     w = tl.small_workload(**kw)
@@ -806,3 +812,49 @@ def test_token_scope_decode_across_two_windows(defer):
                 np.testing.assert_array_equal(idx_hi[bi, kv], idx_hi[bi, 0])
         assert tl.compare_segment(cache, oc, seg) == 0
     cache.check_guards()
+
+
+# ---------------------------------------------------------------- 8-bit codes
+@pytest.mark.parametrize("bits,kch", [((8, 4), False), ((8, 8), False), ((2, 8), False), ((8, 2), True)])
+@pytest.mark.parametrize("defer", [False, True])
+def test_8_bit_classes_across_two_windows(bits, kch, defer):
+    """8-bit codes in the prompt and in two re-compressed windows (the in-kernel re-compression
+    composes 8-bit tiles too): outputs within the bound at every step, every segment's lists,
+    codes and parameters equal to the oracle's."""
+    from workloads import make_decode_step
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(context=260, batch=2, n_q_heads=8, n_kv_heads=2, window=16, decode_steps=40,
+                          rho_recent=0.2, rho_random=0.2, bits_hi=bits[0], bits_lo=bits[1],
+                          k_scheme="channel" if kch else "cst")
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w, max_new=40, defer_append=defer)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    for step in range(35):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        probe = step % 3 == 0
+        cache.append(k, v)
+        out = cache.decode_attention(q, probe)
+        oc.append(tl.to64(k), tl.to64(v))
+        ref = oc.decode_attention(tl.to64(q), probe)
+        torch.cuda.synchronize()
+        got = out.float().cpu().numpy()
+        for (bi, kv), r in ref.items():
+            assert tl.output_excess(got[bi, kv * oc.G:(kv + 1) * oc.G], r, w.torch_dtype) <= 0.0
+    assert zc.zc_num_segments(cache.handle) == 3 and zc.zc_device_status() == 0
+    for seg in range(3):
+        assert tl.compare_segment(cache, oc, seg) == 0
+    cache.check_guards()
+
+
+def test_8_bit_full_size_in_the_benchmark_configuration():
+    """Workload 2 at 8/4 bits: calls side by side with the append deferred, through one window."""
+    w = get_config(2).scaled(bits_hi=8, bits_lo=4)
+    r = tl.run_benchmark_mode(w, [(0, 0), (5, 3)], 105, layers=2)
+    assert r["excess"] <= 0.0, r
+    tl.record("full size, benchmark configuration, 8/4 bits", config=2, units=4, steps=105,
+              max_abs_out=r["worst"], max_abs_out_vs_rounded_oracle=r["worst_rounded"],
+              near_tie_swaps=r["near_tie_swaps"], units_code_exact=r["units_code_exact"],
+              window_set_swaps=r["window_set_mismatches"])
