@@ -89,6 +89,14 @@ enum {
  * this is the form in which the kernel's own arithmetic (Eq. 4 over the dequantised cache)
  * can be compared with a reference at a tolerance below that. */
 #define ZC_FLAG_OUT_F32 4
+/* With ZC_FLAG_PARAMS_F16 the quantisation parameters are stored in 16 bits each, as Appendix A
+ * counts them: the channel factors and the token scales as fp16 values, ROUNDED UP before the
+ * codes are formed (a scale rounded down would no longer cover its token's range), the zero
+ * points as 16-bit integers; a cached token then takes 8 bytes of parameters instead of 16.
+ * For CSTQuant on keys and values (ZC_K_CST) at 2 or 4 bits; the window is re-compressed by
+ * kernels of their own behind the decode kernel of the call that completes it, so the flag
+ * cannot be combined with ZC_FLAG_OVERLAP_CALLS (ZC_EINVAL for either violation). */
+#define ZC_FLAG_PARAMS_F16 8
 
 /* Plain-data configuration; set struct_size = sizeof(zc_config). */
 typedef struct {

@@ -15,6 +15,7 @@ ZC_F16, ZC_BF16 = 0, 1
 ZC_FLAG_DEFER_APPEND = 1
 ZC_FLAG_OVERLAP_CALLS = 2
 ZC_FLAG_OUT_F32 = 4
+ZC_FLAG_PARAMS_F16 = 8
 ZC_K_CST, ZC_K_CHANNEL = 0, 1
 ZC_SCOPE_KV_HEAD, ZC_SCOPE_TOKEN = 0, 1
 
@@ -277,14 +278,15 @@ class ZipCache:
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
                  workspace: Optional[torch.Tensor] = None, defer_append: bool = False,
                  overlap_calls: bool = False, out_f32: bool = False, k_channel: bool = False,
-                 guard_bytes: int = 0, token_scope: bool = False):
+                 guard_bytes: int = 0, token_scope: bool = False, params_f16: bool = False):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
                                  saliency_ratio, bits_hi, bits_lo, window,
                                  flags=(ZC_FLAG_DEFER_APPEND if defer_append else 0) |
                                  (ZC_FLAG_OVERLAP_CALLS if overlap_calls else 0) |
-                                 (ZC_FLAG_OUT_F32 if out_f32 else 0),
+                                 (ZC_FLAG_OUT_F32 if out_f32 else 0) |
+                                 (ZC_FLAG_PARAMS_F16 if params_f16 else 0),
                                  k_scheme=ZC_K_CHANNEL if k_channel else ZC_K_CST,
                                  scope=ZC_SCOPE_TOKEN if token_scope else ZC_SCOPE_KV_HEAD)
         self.k_channel = bool(k_channel)

@@ -275,7 +275,8 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const bool kch = lay.kch != 0;
-  const int sub_bytes = zc_sub_bytes(bits, lay.kch);
+  const bool p16 = lay.p16 != 0;
+  const int sub_bytes = zc_sub_bytes(bits, lay.kch, lay.p16);
   char* tiles = ub + lay.off_tiles[cls] + (long long)seg.tile0[cls] * lay.tile_bytes[cls];
   if (bits == 16) {
     // 16-bit "quantisation" (the 16/16 and 16/2 settings): the subset's rows are gathered into
@@ -312,6 +313,10 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
       zK[e] = 0.f;
     }
     cV[e] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
+    if (p16) {   // stored as fp16 values, rounded up
+      cK[e] = __half2float(__float2half_ru(cK[e]));
+      cV[e] = __half2float(__float2half_ru(cV[e]));
+    }
   }
   // the divisors that stay for all of the CTA's tokens: their correctly rounded reciprocals once
   float rK[4], rV[4];
@@ -389,14 +394,14 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
         unsigned kA, kB, vA, vB;
         raw4<T>(x, rk_a);
         if (kch) kA = quant_channel4_rc(x, cK, rK, midK, zK, L);
-        else quant_token_rc(x, cK, rK, midK, L, rL, &sKa, &zKa, &kA);
+        else quant_token_rc(x, cK, rK, midK, L, rL, &sKa, &zKa, &kA, p16);
         raw4<T>(x, rk_b);
         if (kch) kB = quant_channel4_rc(x, cK, rK, midK, zK, L);
-        else quant_token_rc(x, cK, rK, midK, L, rL, &sKb, &zKb, &kB);
+        else quant_token_rc(x, cK, rK, midK, L, rL, &sKb, &zKb, &kB, p16);
         raw4<T>(x, rv_a);
-        quant_token_rc(x, cV, rV, midV, L, rL, &sVa, &zVa, &vA);
+        quant_token_rc(x, cV, rV, midV, L, rL, &sVa, &zVa, &vA, p16);
         raw4<T>(x, rv_b);
-        quant_token_rc(x, cV, rV, midV, L, rL, &sVb, &zVb, &vB);
+        quant_token_rc(x, cV, rV, midV, L, rL, &sVb, &zVb, &vB, p16);
         if (!live_a) { kA = 0u; vA = 0u; sKa = zKa = sVa = zVa = 0.f; }
         if (!live_b) { kB = 0u; vB = 0u; sKb = zKb = sVb = zVb = 0.f; }
         smax = fmaxf(smax, fmaxf(sVa, sVb));
@@ -450,8 +455,15 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     }
     // the tokens' parameters: (sK, zK, sV, zV), or (sV, zV) with channelwise keys
     if (lane < ZC_SUB) {
-      if (kch) *reinterpret_cast<float2*>(sub + 2 * v_off + lane * 8) = make_float2(par.z, par.w);
-      else *reinterpret_cast<float4*>(sub + 2 * v_off + lane * 16) = par;
+      if (p16) {   // (fp16 scale, int16 zero point) per tensor
+        const unsigned k2 = (unsigned)__half_as_ushort(__float2half_rn(par.x)) | (unsigned)(unsigned short)(short)par.y << 16;
+        const unsigned v2 = (unsigned)__half_as_ushort(__float2half_rn(par.z)) | (unsigned)(unsigned short)(short)par.w << 16;
+        *reinterpret_cast<uint2*>(sub + 2 * v_off + lane * 8) = make_uint2(k2, v2);
+      } else if (kch) {
+        *reinterpret_cast<float2*>(sub + 2 * v_off + lane * 8) = make_float2(par.z, par.w);
+      } else {
+        *reinterpret_cast<float4*>(sub + 2 * v_off + lane * 16) = par;
+      }
     }
     __syncwarp();   // the staging rows are free for the next sub-block
   }

@@ -258,18 +258,19 @@ struct PairState {
 // of the run (`rem` tokens left from its first token); otherwise it is complete.
 // KCH: channelwise keys -- a token has no key parameters (the channel scales are folded into
 // q', qs is then sum_i q'_i z_i), its parameter slot holds (sV, zV) only.
-template <int BITS, bool LAST, bool KCH>
+// P16: a token's parameters are (fp16 scale, int16 zero point) pairs, 8 bytes (ZC_FLAG_PARAMS_F16).
+template <int BITS, bool LAST, bool KCH, bool P16 = false>
 __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uint32_t (&qb)[16],
                                           float qs, float isc, float logKs, float tau_u, int srcA,
                                           int srcB, int c0_src, int c1_src, float (&oacc)[8][4],
                                           PairState& S) {
-  constexpr int PARB = KCH ? 8 : 16;
+  constexpr int PARB = (KCH || P16) ? 8 : 16;
   constexpr int SB = ZC_SUB * (32 * BITS + PARB);
   const int g = lane >> 2;
   if (LAST && rem <= ZC_SUB) {
     // the run ends inside the first half: the second half was not copied; its tokens are
     // masked below, its parameters must not hold stale bits
-    if (KCH) {
+    if (KCH || P16) {
       if (lane < ZC_SUB) *reinterpret_cast<float2*>(st + SB + 512 * BITS + lane * 8) = make_float2(0.f, 0.f);
     } else {
       if (lane < ZC_SUB) *reinterpret_cast<float4*>(st + SB + 512 * BITS + lane * 16) = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -313,7 +314,14 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
       const uint4 c = *reinterpret_cast<const uint4*>(sh + 512 + lane * 16);
       vw[h][0] = c.x; vw[h][1] = c.y; vw[h][2] = c.z; vw[h][3] = c.w;
     }
-    if (KCH) {
+    if (P16) {
+      const uint2 a = *reinterpret_cast<const uint2*>(sh + 512 * BITS + g * 8);
+      const uint2 b = *reinterpret_cast<const uint2*>(sh + 512 * BITS + (g + 8) * 8);
+      pp[h][0] = make_float4(__half2float(__ushort_as_half((unsigned short)a.x)), (float)(short)(a.x >> 16),
+                             __half2float(__ushort_as_half((unsigned short)a.y)), (float)(short)(a.y >> 16));
+      pp[h][1] = make_float4(__half2float(__ushort_as_half((unsigned short)b.x)), (float)(short)(b.x >> 16),
+                             __half2float(__ushort_as_half((unsigned short)b.y)), (float)(short)(b.y >> 16));
+    } else if (KCH) {
       const float2 a = *reinterpret_cast<const float2*>(sh + 512 * BITS + g * 8);
       const float2 b = *reinterpret_cast<const float2*>(sh + 512 * BITS + (g + 8) * 8);
       pp[h][0] = make_float4(1.f, 1.f, a.x, a.y);
@@ -452,13 +460,13 @@ __device__ __forceinline__ void pair_step(char* st, int lane, int rem, const uin
 // Compressed-run part of one item, one warp: prologue done by the CTA, stages primed.  The
 // first my_np - NST iterations refill their stage and need no end-of-run handling; the last
 // NST do not refill and the very last pair may be cut short by the end of the run.
-template <int BITS, int RING, bool KCH>
+template <int BITS, int RING, bool KCH, bool P16 = false>
 __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_base, char* my_ring,
                                           uint64_t* my_bar, const uint32_t (&qb)[16], float qs,
                                           float isc, float logK, int my_np, int warp, int lane,
                                           float (&oacc)[8][4], float& m_out, float& l_out,
                                           float& z_out, int* err) {
-  constexpr int SB = ZC_SUB * (32 * BITS + (KCH ? 8 : 16));
+  constexpr int SB = ZC_SUB * (32 * BITS + ((KCH || P16) ? 8 : 16));
   constexpr int PB = 2 * SB;
   constexpr int NST = (RING / PB) < kMaxStages ? (RING / PB) : kMaxStages;
   const int g = lane >> 2, t = lane & 3;
@@ -493,7 +501,7 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
     uint64_t* bar = &my_bar[stage];
     wait_stage(bar);
     char* st = my_ring + stage * PB;
-    pair_step<BITS, true, KCH>(st, lane, rem0 - i * (2 * ZC_SUB * kWarps), qb, qs, isc, logKs, tau_u, srcA, srcB,
+    pair_step<BITS, true, KCH, P16>(st, lane, rem0 - i * (2 * ZC_SUB * kWarps), qb, qs, isc, logKs, tau_u, srcA, srcB,
                                c0_src, c1_src, oacc, S);
     __syncwarp();
     refill_if(lane == 0 && i < n_refill, bar, st, src_refill, rem_refill > ZC_SUB ? PB : SB);
@@ -514,10 +522,10 @@ __device__ __forceinline__ void run_pairs(const ItemDesc& d, const char* class_b
 // Not inlined: the loop inside gets the whole register budget to itself, whatever the caller
 // keeps alive around the call.
 struct ItemScale { float chan_factor, rowscale; };
-template <typename T, int BITS, int RING, bool KCH>
+template <typename T, int BITS, int RING, bool KCH, bool P16 = false>
 __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_base, const float* fac,
                                                   const T* qbase, int Gl, char* smem, int* err) {
-  constexpr int SB = ZC_SUB * (32 * BITS + (KCH ? 8 : 16));
+  constexpr int SB = ZC_SUB * (32 * BITS + ((KCH || P16) ? 8 : 16));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   constexpr int PB = 2 * SB;
   constexpr int NST = (RING / PB) < kMaxStages ? (RING / PB) : kMaxStages;
@@ -631,7 +639,7 @@ __device__ __noinline__ ItemScale compressed_item(ItemDesc d, const char* class_
 #pragma unroll
     for (int e = 0; e < 4; ++e) oacc[j][e] = 0.f;
   float m, l, z;
-  run_pairs<BITS, RING, KCH>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
+  run_pairs<BITS, RING, KCH, P16>(d, class_base, my_ring, my_bar, qb, qs, isc, logK, my_np, warp, lane, oacc, m, l, z, err);
   __syncwarp();
   if (lane == 0)   // every copy has landed and been consumed: retire the barriers
     for (int s = 0; s < NST; ++s) mbar_inval(&my_bar[s]);
@@ -1307,7 +1315,7 @@ __device__ __noinline__ void merge_unit(float* colsum, int G, int items, int n_t
 // and its arrival counter.
 // RAW: the build that also serves a class kept at 16 bits (kept apart so that the 4- and 2-bit
 // kernels are compiled exactly as they are without it).
-template <typename T, int RING, int NCTA, bool KCH, bool RAW, bool B8 = false>
+template <typename T, int RING, int NCTA, bool KCH, bool RAW, bool B8 = false, bool P16 = false>
 __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay, ZcDecodePlan plan,
                                                       const T* __restrict__ q, T* __restrict__ out,
                                                       float* part, float* stash_all, int slot,
@@ -1414,9 +1422,9 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
       if (B8 && lay.bits[d.cls] == 8)
         sc = compressed_item<T, 8, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
       else if (lay.bits[d.cls] == 4)
-        sc = compressed_item<T, 4, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
+        sc = compressed_item<T, 4, RING, KCH, P16>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
       else if (!RAW || lay.bits[d.cls] == 2)
-        sc = compressed_item<T, 2, RING, KCH>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
+        sc = compressed_item<T, 2, RING, KCH, P16>(d, class_base, fac, qbase, Gl, smem, &g_zc_error);
       else
         sc = raw_item<T>(d, class_base, qbase, Gl, smem, RING);
     }
@@ -1480,7 +1488,7 @@ __global__ void __launch_bounds__(128, NCTA) k_decode(char* cache, ZcLayout lay,
     const long long out_off = ((long long)b * lay.n_kv * G + kv * G) * ZC_D;
     merge_unit<T>(reinterpret_cast<float*>(ub + lay.off_colsum), G, plan.items, plan.n_tail, out + out_off,
                   lay.out_f32 ? reinterpret_cast<float*>(out) + out_off : nullptr, mine, stash_g, collect, smem);
-    if (fl.on) {
+    if (!P16 && fl.on) {   // (16-bit parameters: the host re-compresses by kernels of their own)
       __syncthreads();   // the merge is done with the shared arrays; its additions to the statistics are visible
       window_flush_unit<T, KCH, RAW, B8>(ub, lay, fl, smem);
     }
@@ -1636,7 +1644,7 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   const int groups = (plan.items + plan.cta_items - 1) / plan.cta_items;
   const dim3 grid((unsigned)(c->lay.units * (groups * zs + (plan.fold_tail ? 0 : 1)) + 1));
   cudaError_t e;
-#define ZC_LAUNCH_STEP(T, RING, NCTA, KCH, RAW, B8)                                                    \
+#define ZC_LAUNCH_STEP(T, RING, NCTA, KCH, RAW, B8, P16)                                               \
   do {                                                                                             \
     /* the opt-in to large shared memory is per device and per kernel: one bit per device */       \
     static std::atomic<unsigned long long> attr_done{0};                                           \
@@ -1644,12 +1652,12 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
     cudaGetDevice(&dev_now);                                                                       \
     const unsigned long long bit = 1ull << (dev_now & 63);                                         \
     if (!(attr_done.load(std::memory_order_acquire) & bit)) {                                      \
-      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA, KCH, RAW, B8>,                              \
+      e = cudaFuncSetAttribute(k_decode<T, RING, NCTA, KCH, RAW, B8, P16>,                         \
                                cudaFuncAttributeMaxDynamicSharedMemorySize, decode_smem(RING));    \
       if (e != cudaSuccess) return e;                                                              \
       attr_done.fetch_or(bit, std::memory_order_release);                                          \
     }                                                                                              \
-    e = launch_pdl(k_decode<T, RING, NCTA, KCH, RAW, B8>, grid, dim3(128), decode_smem(RING), st,  \
+    e = launch_pdl(k_decode<T, RING, NCTA, KCH, RAW, B8, P16>, grid, dim3(128), decode_smem(RING), st, \
                    overlap,                                                                        \
                    c->base, c->lay, plan, (const T*)q, (T*)out, part, stash, slot, collect,        \
                    (const T*)k_new, (const T*)v_new, ord, fl);                                     \
@@ -1658,18 +1666,21 @@ int zc_launch_decode(zc_cache* c, const ZcDecodePlan& plan, const void* q, void*
   do {                                                                                             \
     const bool raw = c->lay.bits[0] == 16 || c->lay.bits[1] == 16;                                 \
     const bool b8 = c->lay.bits[0] == 8 || c->lay.bits[1] == 8;                                    \
-    if (b8) { /* an 8-bit class: one build (wide rings hold one pair of its sub-tiles, 3 CTAs per SM) */ \
-      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingWide, 3, true, false, true);                          \
-      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false, true);                                    \
+    if (c->lay.p16) { /* 16-bit parameters: CSTQuant at 2 or 4 bits only */                        \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, false, false, true);     \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false, false, true);                             \
+    } else if (b8) { /* an 8-bit class: one build (wide rings hold one pair of its sub-tiles, 3 CTAs per SM) */ \
+      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingWide, 3, true, false, true, false);                   \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false, true, false);                             \
     } else if (raw) { /* a class kept at 16 bits: one build (narrow rings, 4 CTAs per SM) */       \
-      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, true, false);                        \
-      else ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, true, false);                                  \
+      if (c->lay.kch) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, true, false, false);                 \
+      else ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, true, false, false);                           \
     } else if (c->lay.kch) {                                                                       \
-      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, false, false);            \
-      else ZC_LAUNCH_STEP(T, kRingWide, 3, true, false, false);                                    \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, true, false, false, false);     \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, true, false, false, false);                             \
     } else {                                                                                       \
-      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, false, false);           \
-      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false, false);                                   \
+      if (plan.ctas_per_sm == 4) ZC_LAUNCH_STEP(T, kRingNarrow, 4, false, false, false, false);    \
+      else ZC_LAUNCH_STEP(T, kRingWide, 3, false, false, false, false);                            \
     }                                                                                              \
   } while (0)
   if (c->cfg.dtype == ZC_F16) ZC_LAUNCH_T(__half);

@@ -52,9 +52,16 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
     const int poff = zc_sub_off_par(bits);
     for (int i = threadIdx.x; i < 2 * n_here; i += blockDim.x) {
       const int tl = i >> 1;
-      const float* par = reinterpret_cast<const float*>(tp + (tl / ZC_SUB) * zc_sub_bytes(bits, kch) + poff);
-      sz_out[((long long)unit * n + t0) * 2 + i] =
-          kch ? par[2 * (tl % ZC_SUB) + (i & 1)] : par[4 * (tl % ZC_SUB) + 2 * tensor + (i & 1)];
+      const char* blk = tp + (tl / ZC_SUB) * zc_sub_bytes(bits, kch, lay.p16) + poff;
+      float val;
+      if (lay.p16) {   // (fp16 scale, int16 zero point) per tensor
+        const unsigned short raw = reinterpret_cast<const unsigned short*>(blk)[4 * (tl % ZC_SUB) + 2 * tensor + (i & 1)];
+        val = (i & 1) ? (float)(short)raw : __half2float(__ushort_as_half(raw));
+      } else {
+        const float* par = reinterpret_cast<const float*>(blk);
+        val = kch ? par[2 * (tl % ZC_SUB) + (i & 1)] : par[4 * (tl % ZC_SUB) + 2 * tensor + (i & 1)];
+      }
+      sz_out[((long long)unit * n + t0) * 2 + i] = val;
     }
   }
   if (cf_out && tile == 0 && !(kch && tensor == 0)) {
@@ -67,7 +74,7 @@ __global__ void k_export_segment(const char* cache, ZcLayout lay, ZcSeg seg, int
     for (int i = threadIdx.x; i < n_here * row_bytes; i += blockDim.x) {
       const int tl = i / row_bytes, m = i % row_bytes;
       unsigned byte = 0;
-      const char* sb = tp + (tl / ZC_SUB) * zc_sub_bytes(bits, kch);
+      const char* sb = tp + (tl / ZC_SUB) * zc_sub_bytes(bits, kch, lay.p16);
       if (tensor == 0) {
         byte = reinterpret_cast<const unsigned char*>(sb)[(tl % ZC_SUB) * row_bytes + m];
       } else {

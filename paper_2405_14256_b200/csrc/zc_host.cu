@@ -29,7 +29,12 @@ int check_config(const zc_config* cfg) {
   if (cfg->bits_lo != 4 && cfg->bits_lo != 2 && cfg->bits_lo != 8 && cfg->bits_lo != 16) return ZC_EINVAL;
   // an 8-bit class and a class kept at 16 bits have separate builds of the decode kernel
   if ((cfg->bits_hi == 8 || cfg->bits_lo == 8) && (cfg->bits_hi == 16 || cfg->bits_lo == 16)) return ZC_EINVAL;
-  if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32)) return ZC_EINVAL;
+  if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32 | ZC_FLAG_PARAMS_F16)) return ZC_EINVAL;
+  if (cfg->flags & ZC_FLAG_PARAMS_F16) {   // 16-bit parameters: CSTQuant at 2 or 4 bits, every call waits for what precedes it
+    if (cfg->flags & ZC_FLAG_OVERLAP_CALLS) return ZC_EINVAL;
+    if (cfg->k_scheme != ZC_K_CST) return ZC_EINVAL;
+    if ((cfg->bits_hi != 2 && cfg->bits_hi != 4) || (cfg->bits_lo != 2 && cfg->bits_lo != 4)) return ZC_EINVAL;
+  }
   if (!(cfg->saliency_ratio >= 0.0 && cfg->saliency_ratio <= 1.0)) return ZC_EINVAL;
   if (cfg->k_scheme != ZC_K_CST && cfg->k_scheme != ZC_K_CHANNEL) return ZC_EINVAL;
   if (cfg->scope != ZC_SCOPE_KV_HEAD && cfg->scope != ZC_SCOPE_TOKEN) return ZC_EINVAL;
@@ -51,6 +56,7 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   lay->dtype = cfg->dtype;
   lay->out_f32 = (cfg->flags & ZC_FLAG_OUT_F32) ? 1 : 0;
   lay->kch = cfg->k_scheme == ZC_K_CHANNEL ? 1 : 0;
+  lay->p16 = (cfg->flags & ZC_FLAG_PARAMS_F16) ? 1 : 0;
   lay->bits[0] = cfg->bits_hi;
   lay->bits[1] = cfg->bits_lo;
   const int max_flush = cfg->max_new_tokens / cfg->window;
@@ -65,7 +71,7 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   lay->idx_cap0 = cfg->max_prefill;
   size_t off = 0;
   for (int c = 0; c < 2; ++c) {
-    lay->tile_bytes[c] = zc_tile_bytes(lay->bits[c], lay->kch);
+    lay->tile_bytes[c] = zc_tile_bytes(lay->bits[c], lay->kch, lay->p16);
     lay->off_tiles[c] = (long long)off;
     off = align_up(off + (size_t)lay->cap_tiles[c] * lay->tile_bytes[c], 256);
   }
@@ -478,19 +484,22 @@ static int decode_attention(zc_cache* c, const void* q, void* out, int is_probe_
   ZcFlushArgs fl;
   memset(&fl, 0, sizeof(fl));
   const bool token_scope = c->cfg.scope == ZC_SCOPE_TOKEN;
+  // the heads' statistics must meet first (token scope), or the tiles carry 16-bit parameters,
+  // which only the prefill quantiser writes: the window is re-compressed by kernels of their own
+  const bool host_flush = token_scope || c->lay.p16 != 0;
   if (completes) {
-    fl.on = token_scope ? 0 : 1;   // token scope: by kernels of their own, below
+    fl.on = host_flush ? 0 : 1;
     fl.seg = zc_segment(c, c->n_seg);
     for (int j = 0; j < c->n_tail; ++j) fl.nnz[j] = (unsigned char)(c->tail_nnz[j] + (collect ? 1 : 0));
   }
   ZC_CUDA(zc_launch_decode(c, plan, q, out, collect, (char*)workspace, workspace_bytes, pk, pv,
                            completes ? &fl : nullptr, st));
-  if (completes && token_scope) {
+  if (completes && host_flush) {
     // The window's scores of all KV heads of a batch row meet before the split: scores from
     // the statistics the decode kernels collected, their mean over the row's heads, then the
     // prompt's own split and quantise kernels with the tail as their source.
     ZC_CUDA(zc_launch_window_scores(c, fl, st));
-    ZC_CUDA(zc_launch_share_scores(c, c->cfg.window, st));
+    if (token_scope) ZC_CUDA(zc_launch_share_scores(c, c->cfg.window, st));
     ZC_CUDA(zc_launch_topk(c, c->cfg.window, c->nw[0], fl.seg.idx_off, nullptr, st));
     const int64_t sh = (int64_t)(c->lay.unit_stride / 2);   // elements from one unit's tail to the next
     ZcSrc src{c->base + c->lay.off_tailK, c->base + c->lay.off_tailV, sh * c->lay.n_kv, sh, ZC_D, c->cfg.window};
@@ -563,7 +572,7 @@ int64_t zc_decode_bytes(const zc_cache* c) {
   int64_t per_unit = 0;
   for (int k = 0; k < 2; ++k) {
     const bool raw = c->lay.bits[k] == 16;   // tokens kept at full precision: rows only
-    const int64_t per_tok = raw ? 2 * ZC_D * 2 : 32 * c->lay.bits[k] + (c->lay.kch ? 8 : 16);  // K+V codes, (s,z) pairs
+    const int64_t per_tok = raw ? 2 * ZC_D * 2 : 32 * c->lay.bits[k] + ((c->lay.kch ? 8 : 16) >> c->lay.p16);  // K+V codes, (s,z) pairs
     const int64_t toks = (int64_t)c->n0[k] + (int64_t)(c->n_seg - 1) * c->nw[k];
     per_unit += toks * per_tok;
     const int runs = (c->n0[k] > 0 ? 1 : 0) + (c->nw[k] > 0 ? c->n_seg - 1 : 0);

@@ -41,6 +41,7 @@ struct ZcLayout {
   int units, G, n_kv, window, dtype;
   int out_f32;            // decode outputs are stored as fp32 (ZC_FLAG_OUT_F32)
   int kch;                // keys are quantised channelwise (ZC_K_CHANNEL): no per-token key parameters
+  int p16;                // ZC_FLAG_PARAMS_F16: per-token parameters as (fp16 scale, int16 zero) pairs
   int bits[2];
   int tile_bytes[2];
   int cap_tiles[2];

@@ -19,10 +19,13 @@
 //   [K codes 16 rows x 16*bits B][V codes, fragment order][(sK, zK, sV, zV) x 16]
 // kch: keys quantised channelwise, the parameter block is [(sV, zV) x 16].
 // bits = 16: the tokens are kept as they came (no codes, no parameters): [K rows 16 x 256 B][V rows 16 x 256 B].
-__host__ __device__ inline int zc_sub_bytes(int bits, int kch) {
-  return bits == 16 ? ZC_SUB * 2 * ZC_D * 2 : ZC_SUB * (32 * bits + (kch ? 8 : 16));
+// p16: the parameters are 16 bits each (fp16 scale, int16 zero point): half the block.
+__host__ __device__ inline int zc_sub_bytes(int bits, int kch, int p16 = 0) {
+  return bits == 16 ? ZC_SUB * 2 * ZC_D * 2 : ZC_SUB * (32 * bits + ((kch ? 8 : 16) >> (p16 ? 1 : 0)));
 }
-__host__ __device__ inline int zc_tile_bytes(int bits, int kch) { return (ZC_TILE / ZC_SUB) * zc_sub_bytes(bits, kch); }
+__host__ __device__ inline int zc_tile_bytes(int bits, int kch, int p16 = 0) {
+  return (ZC_TILE / ZC_SUB) * zc_sub_bytes(bits, kch, p16);
+}
 __host__ __device__ inline int zc_sub_off_vcodes(int bits) { return 256 * bits; }
 __host__ __device__ inline int zc_sub_off_par(int bits) { return 512 * bits; }
 

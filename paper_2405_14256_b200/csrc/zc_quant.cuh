@@ -9,6 +9,9 @@
 // fused): c = sqrt(max|x|) (1 if the channel is all zero); y = x / c; per token mn, mx over
 // the 128 channels; s = (mx - mn) / L, or |mn| (1 if mn == 0) when mx == mn;
 // z = -rint(mn / s); code = clamp(rint(y / s) + z, 0, L).
+// P16 (ZC_FLAG_PARAMS_F16): the scale is rounded UP to the next fp16 value before z and the codes
+// are formed (the caller has done the same to c).
+template <bool P16 = false>
 static __device__ __forceinline__ void quant_token(const float (&x)[4], const float (&c)[4], float L,
                                             float* s_out, float* z_out, unsigned* codes4) {
   float y[4];
@@ -23,6 +26,7 @@ static __device__ __forceinline__ void quant_token(const float (&x)[4], const fl
   }
   float s = __fdiv_rn(__fsub_rn(mx, mn), L);
   if (mx == mn) s = mn != 0.f ? fabsf(mn) : 1.f;
+  if (P16) s = __half2float(__float2half_ru(s));
   const float z = -rintf(__fdiv_rn(mn, s));
   unsigned packed = 0;
 #pragma unroll
@@ -59,16 +63,17 @@ static __device__ __forceinline__ bool zc_mid(float a) {
 // same sequence with the divisions taken by zc_div_by where the whole warp's operands allow it
 // (|y| = |x / c| then lies in [2^-80, 2^80], mx - mn is 0 or at least an ulp of 2^-80, and with
 // s in [2^-40, 2^40] the codes' quotients stay below 2^120), by quant_token otherwise.
-static __device__ __noinline__ float4 quant_token_ieee(float4 xv, float4 cv, float L) {   // (s, z, codes, -)
+static __device__ __noinline__ float4 quant_token_ieee(float4 xv, float4 cv, float L, bool p16) {   // (s, z, codes, -)
   const float x[4] = {xv.x, xv.y, xv.z, xv.w}, c[4] = {cv.x, cv.y, cv.z, cv.w};
   float s, z;
   unsigned pk;
-  quant_token(x, c, L, &s, &z, &pk);
+  if (p16) quant_token<true>(x, c, L, &s, &z, &pk);
+  else quant_token<false>(x, c, L, &s, &z, &pk);
   return make_float4(s, z, __uint_as_float(pk), 0.f);
 }
 static __device__ __forceinline__ void quant_token_rc(const float (&x)[4], const float (&c)[4], const float (&rc)[4],
                                                       bool c_mid, float L, float rL, float* s_out, float* z_out,
-                                                      unsigned* codes4) {
+                                                      unsigned* codes4, bool p16 = false) {
   const bool mine = c_mid && zc_mid(x[0]) && zc_mid(x[1]) && zc_mid(x[2]) && zc_mid(x[3]);
   if (__all_sync(0xffffffffu, mine)) {
     float y[4];
@@ -83,6 +88,7 @@ static __device__ __forceinline__ void quant_token_rc(const float (&x)[4], const
     }
     float s = zc_div_by(__fsub_rn(mx, mn), L, rL);   // 0 when mx == mn, replaced below
     if (mx == mn) s = fabsf(mn);                     // mn != 0 here
+    if (p16) s = __half2float(__float2half_ru(s));   // stored as fp16: never below the exact scale
     if (zc_mid(s)) {                                 // the same for every lane
       const float rs = __frcp_rn(s);
       const float z = -rintf(zc_div_by(mn, s, rs));
@@ -99,7 +105,7 @@ static __device__ __forceinline__ void quant_token_rc(const float (&x)[4], const
       return;
     }
   }
-  const float4 r = quant_token_ieee(make_float4(x[0], x[1], x[2], x[3]), make_float4(c[0], c[1], c[2], c[3]), L);
+  const float4 r = quant_token_ieee(make_float4(x[0], x[1], x[2], x[3]), make_float4(c[0], c[1], c[2], c[3]), L, p16);
   *s_out = r.x;
   *z_out = r.y;
   *codes4 = __float_as_uint(r.z);

@@ -858,3 +858,102 @@ def test_8_bit_full_size_in_the_benchmark_configuration():
               max_abs_out=r["worst"], max_abs_out_vs_rounded_oracle=r["worst_rounded"],
               near_tie_swaps=r["near_tie_swaps"], units_code_exact=r["units_code_exact"],
               window_set_swaps=r["window_set_mismatches"])
+
+
+# ---------------------------------------------------------------- 16-bit parameters (ZC_FLAG_PARAMS_F16)
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+@pytest.mark.parametrize("kw", [
+    dict(context=333, batch=2, n_q_heads=8, n_kv_heads=2),
+    dict(context=64, n_q_heads=2, n_kv_heads=2, saliency_ratio=1.0, bits_hi=4, bits_lo=4),
+    dict(context=513, n_q_heads=4, n_kv_heads=4, bits_hi=2, bits_lo=2, outlier_fixed=0),
+    dict(context=17, n_q_heads=1, n_kv_heads=1),
+])
+def test_params_f16_codes_and_parameters_bit_exact(dtype, kw):
+    """Scales and channel factors rounded up to fp16 before the codes are formed, zero points as
+    16-bit integers: lists, codes, parameters and factors equal to the oracle's
+    (param_dtype="f16") bit for bit."""
+    w = tl.small_workload(dtype=dtype, **kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w, param_dtype="f16")
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    n_s = zo.salient_count(w.saliency_ratio, w.context)
+    sal = np.zeros((w.batch, w.n_kv_heads, max(n_s, 1)), dtype=np.int32)
+    for (bi, kv), u in oc.units.items():
+        sal[bi, kv, :n_s] = u.segments[0].hi.idx
+    cache = tl.make_cache(w, params_f16=True)
+    cache.prefill_compress(None, K, V, None, salient_idx=torch.tensor(sal, device=tl.DEV))
+    torch.cuda.synchronize()
+    assert tl.compare_segment(cache, oc, 0) == 0
+    cache.check_guards()
+
+
+@pytest.mark.parametrize("kw", [
+    dict(context=260, batch=2, n_q_heads=8, n_kv_heads=2),
+    dict(context=150, n_q_heads=4, n_kv_heads=4, dtype="bf16", outlier_fixed=0, bits_hi=4, bits_lo=4),
+    dict(context=97, n_q_heads=2, n_kv_heads=1, bits_hi=2, bits_lo=2, saliency_ratio=0.5),
+])
+@pytest.mark.parametrize("defer", [False, True])
+def test_params_f16_decode_across_two_windows(kw, defer):
+    """16-bit parameters in the decode loop (fp16 scale and int16 zero point per token and tensor)
+    and in two re-compressed windows (by kernels of their own behind the completing call): outputs
+    within the bound at every step, every segment equal to the oracle's (param_dtype="f16")."""
+    from workloads import make_decode_step
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(window=16, decode_steps=40, rho_recent=0.2, rho_random=0.2, **kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w, param_dtype="f16")
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w, max_new=40, defer_append=defer, params_f16=True)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    for step in range(35):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        probe = step % 3 == 0
+        cache.append(k, v)
+        out = cache.decode_attention(q, probe)
+        oc.append(tl.to64(k), tl.to64(v))
+        ref = oc.decode_attention(tl.to64(q), probe)
+        torch.cuda.synchronize()
+        got = out.float().cpu().numpy()
+        for (bi, kv), r in ref.items():
+            assert tl.output_excess(got[bi, kv * oc.G:(kv + 1) * oc.G], r, w.torch_dtype) <= 0.0
+    assert zc.zc_num_segments(cache.handle) == 3 and zc.zc_device_status() == 0
+    for seg in range(3):
+        assert tl.compare_segment(cache, oc, seg) == 0
+    cache.check_guards()
+
+
+def test_params_f16_full_size_one_call_at_a_time():
+    """Workload 2 with 16-bit parameters, the launch mode they admit (every call waits for what
+    precedes it), sampled units, through one window."""
+    w = get_config(2)
+    units = [(0, 0), (5, 3)]
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w, units, param_dtype="f16")
+    oc.prefill_compress(*tl.oracle_inputs(w, Q, K, V, units), P)
+    cache = tl.make_cache(w, max_new=104, defer_append=True, params_f16=True)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    from workloads import make_decode_step, decode_probe_flags
+    flags = decode_probe_flags(w, 0, 103)
+    worst = 0.0
+    for step in range(103):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        probe = bool(flags[step])
+        cache.append(k, v)
+        out = cache.decode_attention(q, probe)
+        qq, kk, vv = tl.oracle_step_inputs(w, q, k, v, units)
+        oc.append(kk, vv)
+        ref = oc.decode_attention(qq, probe)
+        got = out.float().cpu().numpy()
+        for (bi, kv), r in ref.items():
+            g = got[bi, kv * oc.G:(kv + 1) * oc.G]
+            assert tl.output_excess(g, r, w.torch_dtype) <= 0.0
+            worst = max(worst, float(np.abs(g - r).max()))
+    import paper_2405_14256_b200 as zc
+    assert zc.zc_num_segments(cache.handle) == 2 and zc.zc_device_status() == 0
+    for seg in range(2):
+        assert tl.compare_segment(cache, oc, seg, units) == 0
+    tl.record("full size, 16-bit parameters, one call at a time", config=2, units=len(units), steps=103,
+              max_abs_out=worst)
