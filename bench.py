@@ -439,6 +439,8 @@ MODES = {
     "dependent": dict(overlap_calls=False, defer_append=True),
     # the paper's own key quantiser (channelwise keys: 8 bytes per token less to read)
     "overlap_channelwise_keys": dict(overlap_calls=True, defer_append=True, k_channel=True),
+    # 16-bit quantisation parameters (8 bytes per token less); every call waits for what precedes it
+    "dependent_params_f16": dict(overlap_calls=False, defer_append=True, params_f16=True),
 }
 
 
@@ -672,7 +674,7 @@ def main():
     ap.add_argument("--config", type=int, default=0, help="one workload only (default: 2, 3, 4 and 5)")
     ap.add_argument("--decode-steps", type=int, default=0,
                     help="profiling only: fewer decode steps than the workload's own")
-    ap.add_argument("--mode", default="both", choices=["both", "overlap", "dependent", "overlap_channelwise_keys"],
+    ap.add_argument("--mode", default="both", choices=["both", "overlap", "dependent", "overlap_channelwise_keys", "dependent_params_f16"],
                     help="overlap: ZC_FLAG_OVERLAP_CALLS (independent caches, calls side by side); "
                          "dependent: every call waits for the kernel before it")
     ap.add_argument("--append", default="deferred", choices=["deferred", "kernel"],
@@ -731,6 +733,10 @@ def main():
                 pairs[name] = {"us_per_call": rr["overlap"]["us_per_call"], "frac": rr["overlap"]["frac"],
                                "gbs": rr["overlap"]["gbs"], "prefill_tokens_per_s": rr["prefill_tokens_per_s"]}
             per_config[str(cfg_id)]["bit_pairs_overlap_mode"] = pairs
+            rr = measure_config(zc, cfg_id, args, rank, local_rank, world, dist, dev, ["dependent_params_f16"],
+                                headline=False)["per_config"]["dependent_params_f16"]
+            per_config[str(cfg_id)]["params_f16_one_call_at_a_time"] = {
+                "us_per_call": rr["us_per_call"], "frac": rr["frac"], "gbs": rr["gbs"]}
         if cfg_id == head_cfg:
             head = r
             if not args.no_e2e:
