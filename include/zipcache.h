@@ -188,7 +188,7 @@ int zc_append(zc_cache* c, const void* k_new, const void* v_new, zc_stream_t str
  * or one of the last five steps of a window) this step's attention over the tail's
  * tokens is added to the window statistics; the call that takes the window's last step
  * also re-compresses the tail into a new segment, inside the same kernel (no further launch,
- * no host synchronisation); with ZC_SCOPE_TOKEN or ZC_FLAG_PARAMS_F16 by five small kernels
+ * no host synchronisation); with ZC_SCOPE_TOKEN or ZC_FLAG_PARAMS_F16 by five or six small kernels
  * launched behind it on the same stream (still no host synchronisation).
  * Only a call that follows a zc_append takes a step of Alg. 3; a further call on the same tail
  * (the same token queried again) attends the cache as it is and leaves the window's counters,
