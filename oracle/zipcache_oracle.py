@@ -547,14 +547,23 @@ class ZipCacheOracle:
     def __init__(self, batch: int, n_q_heads: int, n_kv_heads: int, head_dim: int, ratio: float,
                  bits_hi: int = 4, bits_lo: int = 2, window: int = 100,
                  units: Optional[Sequence[Tuple[int, int]]] = None, k_scheme: str = "cst",
-                 param_dtype: str = "f32", scope: str = "kv_head"):
+                 param_dtype: str = "f32", scope: str = "kv_head", group: str = "head"):
         """scope "kv_head": one saliency decision per (batch, KV head).  scope "token": the
         paper's literal reading, one decision per token of a batch row shared by all heads --
         the score of a token is the mean of its per-KV-head normalised scores (all units of the
-        batch row are then needed).  parity unpinned (how heads are combined is a convention)."""
+        batch row are then needed).  parity unpinned (how heads are combined is a convention).
+        group "head": a token's (s, z) are taken over the d channels of one KV head (2 b h l
+        parameters per tensor).  group "all_heads": Alg. 1 as printed, X in R^{l x hd}: one (s, z)
+        per token over the channels of ALL KV heads of its batch row (Sec. 4.1's 2 b l parameters);
+        the heads must then agree on the subsets, so it needs scope "token"."""
+        if group not in ("head", "all_heads"):
+            raise ValueError("group must be 'head' or 'all_heads'")
+        if group == "all_heads" and scope != "token":
+            raise ValueError("token groups over all heads need one split per token (scope='token')")
         self.b, self.hq, self.hkv, self.d = batch, n_q_heads, n_kv_heads, head_dim
         self.G = n_q_heads // n_kv_heads
         self.scope = scope
+        self.group = group
         self.unit_ids = list(units) if units is not None else [
             (bi, kv) for bi in range(batch) for kv in range(n_kv_heads)]
         self.units = {u: UnitCache(self.G, head_dim, ratio, bits_hi, bits_lo, window, k_scheme,
@@ -575,6 +584,40 @@ class ZipCacheOracle:
             self.units[(bi, kv)].prefill_compress(
                 Q[bi, kv * self.G:(kv + 1) * self.G], K[bi, kv], V[bi, kv], P, sal,
                 p_tilde=shared.get(bi))
+        if self.group == "all_heads":
+            for bi in sorted({u[0] for u in self.unit_ids}):
+                self._quantise_row_jointly(bi, [K[bi, kv] for kv in range(self.hkv)],
+                                           [V[bi, kv] for kv in range(self.hkv)])
+
+    def _quantise_row_jointly(self, bi: int, Ks, Vs) -> None:
+        """Alg. 1 on X in R^{n x (h d)}: the newest segment's subsets of every KV head of batch row
+        bi are quantised again as ONE matrix per tensor whose columns are the channels of all the
+        heads, so a token has one (s, z) for all of them; every head keeps its own columns of the
+        codes and of the channel factors.  (Channelwise keys have no token parameters: their K
+        stays as it is.)"""
+        row = [self.units[(bi, kv)] for kv in range(self.hkv)]
+        d = self.d
+        for name in ("hi", "lo"):
+            subs = [getattr(u.segments[-1], name) for u in row]
+            if subs[0].bits == 16 or subs[0].n == 0:
+                continue
+            idx = subs[0].idx
+            for sub in subs:
+                assert np.array_equal(sub.idx, idx), "token groups need the same subsets in every head"
+            cst = cst_quant_f16_params if row[0].param_dtype == "f16" else cst_quant
+            for tensor, Xs in (("V", Vs), ("K", Ks)):
+                if tensor == "K" and row[0].k_scheme == "channel":
+                    continue
+                X = np.concatenate([np.asarray(x, dtype=np.float32)[idx] for x in Xs], axis=1)
+                q = cst(X, subs[0].bits)
+                for kv, sub in enumerate(subs):
+                    part = {"c": q["c"][kv * d:(kv + 1) * d], "s": q["s"], "z": q["z"],
+                            "codes": q["codes"][:, kv * d:(kv + 1) * d], "bits": q["bits"],
+                            "pre_round": q["pre_round"][:, kv * d:(kv + 1) * d]}
+                    if tensor == "V":
+                        sub.qV, sub.V_hat = part, cst_dequant(part)
+                    else:
+                        sub.qK, sub.K_hat = part, cst_dequant(part)
 
     def append(self, k, v) -> None:
         for (bi, kv) in self.unit_ids:
@@ -591,6 +634,9 @@ class ZipCacheOracle:
                 row = [self.units[(bi, kv)] for kv in range(self.hkv)]
                 if row[0].i == row[0].window:
                     shared = sum(u.window_scores() for u in row) / self.hkv
+                    tails = [(u.tail_K.copy(), u.tail_V.copy()) for u in row]
                     for u in row:
                         u._flush(shared)
+                    if self.group == "all_heads":
+                        self._quantise_row_jointly(bi, [t[0] for t in tails], [t[1] for t in tails])
         return out

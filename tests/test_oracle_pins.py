@@ -672,6 +672,73 @@ def test_token_scope_shares_one_split_across_heads():
     np.testing.assert_array_equal(one.units[(0, 0)].segments[0].hi.idx, ref.units[(0, 0)].segments[0].hi.idx)
 
 
+# ---------------------------------------------------------------- token groups over all heads (Alg. 1, X in R^{l x hd})
+def test_token_groups_over_all_heads():
+    """group="all_heads": one (s, z) per token for the channels of every KV head of its batch row
+    (Sec. 4.1: 2bl parameters per tensor beside the hd channel factors).  Pinned by pure-Python
+    loops for the token statistics, the half-step bound under the shared scale, the parameter
+    count, and the reduction to the per-head grouping when there is one KV head."""
+    rs = _rng(21)
+    b, hq, hkv, l, d = 2, 4, 2, 40, 8
+    Q = rs.standard_normal((b, hq, l, d)); K = rs.standard_normal((b, hkv, l, d)) * 3; V = rs.standard_normal((b, hkv, l, d))
+    K[:, 1] *= 7.0                                    # heads of unlike range: the shared scale is the wider head's
+    P = zo.probe_positions(l, 0.1, 0.1, 1)
+    oc = zo.ZipCacheOracle(b, hq, hkv, d, 0.4, window=8, scope="token", group="all_heads")
+    oc.prefill_compress(Q, K, V, P)
+    f32 = np.float32
+    n_params = 0
+    for bi in range(b):
+        subs = [oc.units[(bi, kv)].segments[0].hi for kv in range(hkv)]
+        idx = subs[0].idx
+        for tensor, X in (("qK", K), ("qV", V)):
+            qs = [getattr(sub, tensor) for sub in subs]
+            for kv in range(1, hkv):
+                np.testing.assert_array_equal(qs[kv]["s"], qs[0]["s"])      # one (s, z) per token for all heads
+                np.testing.assert_array_equal(qs[kv]["z"], qs[0]["z"])
+            n_params += 2 * len(idx) + hkv * d
+            # the token statistics by loops: minimum and maximum of x / c over every head's channels
+            for r, j in enumerate(idx):
+                ys = []
+                for kv in range(hkv):
+                    Xs = X[bi, kv].astype(f32)[idx]
+                    for ch in range(d):
+                        c = f32(np.sqrt(f32(np.abs(Xs[:, ch]).max())))
+                        assert c == qs[kv]["c"][ch]
+                        ys.append(f32(Xs[r, ch] / c))
+                mn, mx = min(ys), max(ys)
+                assert qs[0]["s"][r] == f32(f32(mx - mn) / f32(15))
+                assert qs[0]["z"][r] == -np.rint(f32(mn / qs[0]["s"][r]))
+                # half-step bound of every head's codes under the shared scale
+                k = 0
+                for kv in range(hkv):
+                    for ch in range(d):
+                        y = ys[k]; k += 1
+                        code = float(qs[kv]["codes"][r, ch])
+                        assert abs(float(y) - (code - float(qs[0]["z"][r])) * float(qs[0]["s"][r])) <= 0.5 * float(qs[0]["s"][r]) * (1 + 1e-5)
+    # Sec. 4.1's count for the salient subsets: (2 n_s + h d) per tensor and batch row
+    n_s = zo.salient_count(0.4, l)
+    assert n_params == b * 2 * (2 * n_s + hkv * d)
+    # a re-compressed window is grouped the same way
+    for s in range(8):
+        oc.append(rs.standard_normal((b, hkv, d)), rs.standard_normal((b, hkv, d)))
+        oc.decode_attention(rs.standard_normal((b, hq, d)), s % 2 == 0)
+    for bi in range(b):
+        a, c = oc.units[(bi, 0)].segments[1].lo, oc.units[(bi, 1)].segments[1].lo
+        np.testing.assert_array_equal(a.qV["s"], c.qV["s"]); np.testing.assert_array_equal(a.qK["z"], c.qK["z"])
+    # one KV head: the same as the grouping per head
+    one = zo.ZipCacheOracle(1, 2, 1, d, 0.4, scope="token", group="all_heads")
+    ref = zo.ZipCacheOracle(1, 2, 1, d, 0.4, scope="token")
+    for o in (one, ref):
+        o.prefill_compress(Q[:1, :2], K[:1, :1], V[:1, :1], P)
+    for name in ("hi", "lo"):
+        for t in ("qK", "qV"):
+            x, y = getattr(getattr(one.units[(0, 0)].segments[0], name), t), getattr(getattr(ref.units[(0, 0)].segments[0], name), t)
+            for key in ("c", "s", "z", "codes"):
+                np.testing.assert_array_equal(x[key], y[key])
+    with pytest.raises(ValueError):
+        zo.ZipCacheOracle(1, 2, 1, d, 0.4, group="all_heads")          # needs one split per token
+
+
 # ---------------------------------------------------------------- Eq. 2: causal prefill attention
 @pytest.mark.parametrize("l,d", [(1, 8), (7, 8), (33, 16), (130, 32)])
 def test_prefill_attention_is_library_causal_attention(l, d):
