@@ -97,6 +97,13 @@ enum {
  * kernels of their own behind the decode kernel of the call that completes it, so the flag
  * cannot be combined with ZC_FLAG_OVERLAP_CALLS (ZC_EINVAL for either violation). */
 #define ZC_FLAG_PARAMS_F16 8
+/* With ZC_FLAG_GROUP_ALL_HEADS a token's scale and zero point are taken over the channels of ALL
+ * KV heads of its batch row (Alg. 1 as printed: X in R^{l x hd}; Sec. 4.1 counts 2bl token
+ * parameters per tensor), not over one head's head_dim channels; every head's tiles carry the
+ * row's shared pair.  The heads must agree on the subsets, so it needs ZC_SCOPE_TOKEN (and with
+ * it no ZC_FLAG_OVERLAP_CALLS); 16-bit classes are not admitted (ZC_EINVAL otherwise).
+ * Channelwise keys have no token parameters: with ZC_K_CHANNEL only the values are grouped. */
+#define ZC_FLAG_GROUP_ALL_HEADS 16
 
 /* Plain-data configuration; set struct_size = sizeof(zc_config). */
 typedef struct {

@@ -16,6 +16,7 @@ ZC_FLAG_DEFER_APPEND = 1
 ZC_FLAG_OVERLAP_CALLS = 2
 ZC_FLAG_OUT_F32 = 4
 ZC_FLAG_PARAMS_F16 = 8
+ZC_FLAG_GROUP_ALL_HEADS = 16
 ZC_K_CST, ZC_K_CHANNEL = 0, 1
 ZC_SCOPE_KV_HEAD, ZC_SCOPE_TOKEN = 0, 1
 
@@ -278,7 +279,8 @@ class ZipCache:
                  saliency_ratio, bits_hi=4, bits_lo=2, window=100, device="cuda:0",
                  workspace: Optional[torch.Tensor] = None, defer_append: bool = False,
                  overlap_calls: bool = False, out_f32: bool = False, k_channel: bool = False,
-                 guard_bytes: int = 0, token_scope: bool = False, params_f16: bool = False):
+                 guard_bytes: int = 0, token_scope: bool = False, params_f16: bool = False,
+                 group_all_heads: bool = False):
         if not torch.cuda.is_available():
             raise ZipCacheError("a CUDA device is required (no CPU fallback)")
         self.cfg = ZcConfig.make(dtype, batch, n_q_heads, n_kv_heads, max_prefill, max_new_tokens,
@@ -286,7 +288,8 @@ class ZipCache:
                                  flags=(ZC_FLAG_DEFER_APPEND if defer_append else 0) |
                                  (ZC_FLAG_OVERLAP_CALLS if overlap_calls else 0) |
                                  (ZC_FLAG_OUT_F32 if out_f32 else 0) |
-                                 (ZC_FLAG_PARAMS_F16 if params_f16 else 0),
+                                 (ZC_FLAG_PARAMS_F16 if params_f16 else 0) |
+                                 (ZC_FLAG_GROUP_ALL_HEADS if group_all_heads else 0),
                                  k_scheme=ZC_K_CHANNEL if k_channel else ZC_K_CST,
                                  scope=ZC_SCOPE_TOKEN if token_scope else ZC_SCOPE_KV_HEAD)
         self.k_channel = bool(k_channel)

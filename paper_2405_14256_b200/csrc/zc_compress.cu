@@ -243,6 +243,66 @@ __global__ void k_window_scores(char* cache, ZcLayout lay, ZcFlushArgs fl) {
   colsum[tid] = 0.f;
 }
 
+// ------------------------------------------------------------------ token groups over all heads (ZC_FLAG_GROUP_ALL_HEADS)
+// Channel factor of Alg. 1 from the subset's channel maximum: c = sqrt(max |x|), 1 for an all-zero
+// channel; with 16-bit parameters the fp16 value at or above it.
+__device__ __forceinline__ float channel_factor(unsigned key, bool p16) {
+  const float m = zc_key_float(key);
+  float c = m == 0.f ? 1.f : __fsqrt_rn(m);
+  if (p16) c = __half2float(__float2half_ru(c));
+  return c;
+}
+
+template <typename T> __device__ __forceinline__ void raw4_load(float (&x)[4], const T* p) {
+  const uint2 raw = *reinterpret_cast<const uint2*>(p);
+  const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) x[i] = zc_to_float<T>(e[i]);
+}
+
+// Per token of a subset: minimum and maximum of y = x / c over the channels of ALL KV heads of
+// its batch row, for K and for V (Alg. 1 on X in R^{n x hd}).  One warp per token; the row's
+// first unit keeps the results.  grid: (tokens / 8, batch, class).
+template <typename T>
+__global__ void k_token_minmax(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg) {
+  const int cls = blockIdx.z, n_c = seg.n_tok[cls];
+  const int lane = threadIdx.x & 31, t = blockIdx.x * 8 + (threadIdx.x >> 5), b = blockIdx.y;
+  if (t >= n_c || lay.bits[cls] == 16) return;
+  char* ub0 = zc_unit_base(cache, lay, b * lay.n_kv);
+  const int32_t* idx = reinterpret_cast<const int32_t*>(ub0 + lay.off_idx) + seg.idx_off + (cls == 0 ? 0 : seg.n_tok[0]);
+  const long long row = (long long)idx[t] * src.sl;
+  float mnK = INFINITY, mxK = -INFINITY, mnV = INFINITY, mxV = -INFINITY;
+  for (int kv = 0; kv < lay.n_kv; ++kv) {
+    const char* ub = zc_unit_base(cache, lay, b * lay.n_kv + kv);
+    const unsigned* cmax = reinterpret_cast<const unsigned*>(ub + lay.off_cmax) + cls * 3 * ZC_D;
+    const T* Kb = reinterpret_cast<const T*>(src.K) + b * src.sb + kv * src.sh + row + 4 * lane;
+    const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh + row + 4 * lane;
+    float xk[4], xv[4];
+    raw4_load<T>(xk, Kb);
+    raw4_load<T>(xv, Vb);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (!lay.kch) {   // channelwise keys have no token parameters
+        const float y = __fdiv_rn(xk[e], channel_factor(cmax[4 * lane + e], lay.p16 != 0));
+        mnK = fminf(mnK, y);
+        mxK = fmaxf(mxK, y);
+      }
+      const float y = __fdiv_rn(xv[e], channel_factor(cmax[ZC_D + 4 * lane + e], lay.p16 != 0));
+      mnV = fminf(mnV, y);
+      mxV = fmaxf(mxV, y);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mnK = fminf(mnK, __shfl_xor_sync(0xffffffffu, mnK, o));
+    mxK = fmaxf(mxK, __shfl_xor_sync(0xffffffffu, mxK, o));
+    mnV = fminf(mnV, __shfl_xor_sync(0xffffffffu, mnV, o));
+    mxV = fmaxf(mxV, __shfl_xor_sync(0xffffffffu, mxV, o));
+  }
+  if (lane == 0)
+    reinterpret_cast<float4*>(ub0 + lay.off_tokmm)[(cls == 0 ? 0 : seg.n_tok[0]) + t] = make_float4(mnK, mxK, mnV, mxV);
+}
+
 // ------------------------------------------------------------------ CSTQuant + pack (arithmetic in zc_quant.cuh)
 template <typename T> __device__ __forceinline__ void raw4(float (&x)[4], uint2 raw) {
   const T* e = reinterpret_cast<const T*>(&raw);
@@ -256,7 +316,9 @@ template <typename T> __device__ __forceinline__ void raw4(float (&x)[4], uint2 
 // memory, from which each lane gathers its words of the fragment order; the tokens' (s, z) are
 // kept by the lane of the token's number.  No barrier of the CTA.
 // grid.x: CTAs of class 0 (8 * rounds sub-blocks each), then of class 1; grid.y: unit.
-template <typename T>
+// GA: token groups over all heads (the row's statistics come from k_token_minmax); P16: 16-bit
+// parameters; B8: a class of 8-bit codes.  Template parameters, so that the plain build carries none of them.
+template <typename T, bool GA, bool P16, bool B8>
 __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout lay, ZcSrc src, ZcSeg seg, int rounds) {
   __shared__ __align__(16) unsigned char stageV[8][ZC_SUB][ZC_D];
   const int unit = blockIdx.y, b = unit / lay.n_kv, kv = unit % lay.n_kv;
@@ -275,8 +337,8 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
   const T* Vb = reinterpret_cast<const T*>(src.V) + b * src.sb + kv * src.sh;
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const bool kch = lay.kch != 0;
-  const bool p16 = lay.p16 != 0;
-  const int sub_bytes = zc_sub_bytes(bits, lay.kch, lay.p16);
+  constexpr bool p16 = P16;
+  const int sub_bytes = zc_sub_bytes(bits, lay.kch, P16 ? 1 : 0);
   char* tiles = ub + lay.off_tiles[cls] + (long long)seg.tile0[cls] * lay.tile_bytes[cls];
   if (bits == 16) {
     // 16-bit "quantisation" (the 16/16 and 16/2 settings): the subset's rows are gathered into
@@ -309,14 +371,10 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     if (kch) {
       channel_params(zc_key_float(cmax[2 * ZC_D + 4 * lane + e]), mk, L, &cK[e], &zK[e]);
     } else {
-      cK[e] = mk == 0.f ? 1.f : __fsqrt_rn(mk);
+      cK[e] = channel_factor(cmax[4 * lane + e], p16);
       zK[e] = 0.f;
     }
-    cV[e] = mv == 0.f ? 1.f : __fsqrt_rn(mv);
-    if (p16) {   // stored as fp16 values, rounded up
-      cK[e] = __half2float(__float2half_ru(cK[e]));
-      cV[e] = __half2float(__float2half_ru(cV[e]));
-    }
+    cV[e] = channel_factor(cmax[ZC_D + 4 * lane + e], p16);
   }
   // the divisors that stay for all of the CTA's tokens: their correctly rounded reciprocals once
   float rK[4], rV[4];
@@ -337,6 +395,10 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
       if (kch) fac[ZC_FAC_ZK + 4 * lane + e] = zK[e];
     }
   }
+  // token groups over all heads: the row's statistics, kept by its first unit
+  const float4* tokmm = GA ? reinterpret_cast<const float4*>(zc_unit_base(cache, lay, b * lay.n_kv) + lay.off_tokmm) +
+                                 (cls == 0 ? 0 : seg.n_tok[0])
+                           : nullptr;
   const int k_row_bytes = 16 * bits;            // a token's K codes
   const int v_off = ZC_SUB * k_row_bytes;       // the sub-block's V codes follow its K codes, then the parameters
   float smax = 0.f;
@@ -392,23 +454,30 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
         const uint2 rv_a = pr == 0 ? rawV[0] : rawV[2], rv_b = pr == 0 ? rawV[1] : rawV[3];
         float x[4], sKa = 0.f, zKa = 0.f, sKb = 0.f, zKb = 0.f, sVa, zVa, sVb, zVb;
         unsigned kA, kB, vA, vB;
+        // token groups over all heads: the row's (min, max) of y for the pair's tokens
+        constexpr bool shared = GA;
+        float4 mmA = make_float4(0.f, 0.f, 0.f, 0.f), mmB = mmA;
+        if (shared) {
+          if (live_a) mmA = tokmm[sb * ZC_SUB + ta];
+          if (live_b) mmB = tokmm[sb * ZC_SUB + ta + 1];
+        }
         raw4<T>(x, rk_a);
         if (kch) kA = quant_channel4_rc(x, cK, rK, midK, zK, L);
-        else quant_token_rc(x, cK, rK, midK, L, rL, &sKa, &zKa, &kA, p16);
+        else quant_token_rc(x, cK, rK, midK, L, rL, &sKa, &zKa, &kA, p16, shared, mmA.x, mmA.y);
         raw4<T>(x, rk_b);
         if (kch) kB = quant_channel4_rc(x, cK, rK, midK, zK, L);
-        else quant_token_rc(x, cK, rK, midK, L, rL, &sKb, &zKb, &kB, p16);
+        else quant_token_rc(x, cK, rK, midK, L, rL, &sKb, &zKb, &kB, p16, shared, mmB.x, mmB.y);
         raw4<T>(x, rv_a);
-        quant_token_rc(x, cV, rV, midV, L, rL, &sVa, &zVa, &vA, p16);
+        quant_token_rc(x, cV, rV, midV, L, rL, &sVa, &zVa, &vA, p16, shared, mmA.z, mmA.w);
         raw4<T>(x, rv_b);
-        quant_token_rc(x, cV, rV, midV, L, rL, &sVb, &zVb, &vB, p16);
+        quant_token_rc(x, cV, rV, midV, L, rL, &sVb, &zVb, &vB, p16, shared, mmB.z, mmB.w);
         if (!live_a) { kA = 0u; vA = 0u; sKa = zKa = sVa = zVa = 0.f; }
         if (!live_b) { kB = 0u; vB = 0u; sKb = zKb = sVb = zVb = 0.f; }
         smax = fmaxf(smax, fmaxf(sVa, sVb));
         if (lane == ta) par = make_float4(sKa, zKa, sVa, zVa);
         if (lane == ta + 1) par = make_float4(sKb, zKb, sVb, zVb);
         // K: straight from the registers
-        if (bits == 8) {   // a lane's four codes are a word of the row
+        if (B8 && bits == 8) {   // a lane's four codes are a word of the row
           *reinterpret_cast<unsigned*>(sub + ta * k_row_bytes + 4 * lane) = kA;
           *reinterpret_cast<unsigned*>(sub + (ta + 1) * k_row_bytes + 4 * lane) = kB;
         } else {
@@ -425,7 +494,7 @@ __global__ void __launch_bounds__(256, 4) k_quantize_pack(char* cache, ZcLayout 
     }
     __syncwarp();
     // V: this lane's words of the fragment order, 16 bytes at a time
-    if (bits == 8) {
+    if (B8 && bits == 8) {
 #pragma unroll 1
       for (int q = 0; q < 4; ++q) {
         uint4 o;
@@ -513,14 +582,29 @@ int zc_launch_quantize(zc_cache* c, const ZcSrc& src, const ZcSeg& seg, cudaStre
     dim3 grid_max(zc_ceil_div(zc_ceil_div(seg.n_tok[0], ZC_TILE), kAbsTiles) +
                       zc_ceil_div(zc_ceil_div(seg.n_tok[1], ZC_TILE), kAbsTiles),
                   c->lay.units);
-    if (c->cfg.dtype == ZC_F16) {
-      k_channel_absmax<__half><<<grid_max, 256, 0, st>>>(c->base, c->lay, src, seg);
-      k_quantize_pack<__half><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds);
-    } else {
-      k_channel_absmax<__nv_bfloat16><<<grid_max, 256, 0, st>>>(c->base, c->lay, src, seg);
-      k_quantize_pack<__nv_bfloat16><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds);
-    }
-    c->launches += 2;
+    const dim3 grid_mm(zc_ceil_div(std::max(seg.n_tok[0], seg.n_tok[1]), 8), c->cfg.batch, 2);
+#define ZC_QUANT_GO(T)                                                                                   \
+  do {                                                                                                 \
+    const bool b8 = c->lay.bits[0] == 8 || c->lay.bits[1] == 8;   /* never together with 16-bit parameters */ \
+    k_channel_absmax<T><<<grid_max, 256, 0, st>>>(c->base, c->lay, src, seg);                          \
+    if (c->lay.grp_all) k_token_minmax<T><<<grid_mm, 256, 0, st>>>(c->base, c->lay, src, seg);         \
+    if (c->lay.grp_all && c->lay.p16)                                                                  \
+      k_quantize_pack<T, true, true, false><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds);  \
+    else if (c->lay.grp_all && b8)                                                                     \
+      k_quantize_pack<T, true, false, true><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds);  \
+    else if (c->lay.grp_all)                                                                           \
+      k_quantize_pack<T, true, false, false><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds); \
+    else if (c->lay.p16)                                                                               \
+      k_quantize_pack<T, false, true, false><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds); \
+    else if (b8)                                                                                       \
+      k_quantize_pack<T, false, false, true><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds); \
+    else                                                                                               \
+      k_quantize_pack<T, false, false, false><<<grid, 256, 0, st>>>(c->base, c->lay, src, seg, rounds); \
+  } while (0)
+    if (c->cfg.dtype == ZC_F16) ZC_QUANT_GO(__half);
+    else ZC_QUANT_GO(__nv_bfloat16);
+#undef ZC_QUANT_GO
+    c->launches += c->lay.grp_all ? 3 : 2;
   }
   return (int)cudaGetLastError();
 }

@@ -29,7 +29,13 @@ int check_config(const zc_config* cfg) {
   if (cfg->bits_lo != 4 && cfg->bits_lo != 2 && cfg->bits_lo != 8 && cfg->bits_lo != 16) return ZC_EINVAL;
   // an 8-bit class and a class kept at 16 bits have separate builds of the decode kernel
   if ((cfg->bits_hi == 8 || cfg->bits_lo == 8) && (cfg->bits_hi == 16 || cfg->bits_lo == 16)) return ZC_EINVAL;
-  if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32 | ZC_FLAG_PARAMS_F16)) return ZC_EINVAL;
+  if (cfg->flags & ~(ZC_FLAG_DEFER_APPEND | ZC_FLAG_OVERLAP_CALLS | ZC_FLAG_OUT_F32 | ZC_FLAG_PARAMS_F16 |
+                     ZC_FLAG_GROUP_ALL_HEADS))
+    return ZC_EINVAL;
+  if (cfg->flags & ZC_FLAG_GROUP_ALL_HEADS) {   // one (s, z) per token for all heads: one split per token, quantised classes
+    if (cfg->scope != ZC_SCOPE_TOKEN) return ZC_EINVAL;
+    if (cfg->bits_hi == 16 || cfg->bits_lo == 16) return ZC_EINVAL;
+  }
   if (cfg->flags & ZC_FLAG_PARAMS_F16) {   // 16-bit parameters: CSTQuant at 2 or 4 bits, every call waits for what precedes it
     if (cfg->flags & ZC_FLAG_OVERLAP_CALLS) return ZC_EINVAL;
     if (cfg->k_scheme != ZC_K_CST) return ZC_EINVAL;
@@ -57,6 +63,7 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   lay->out_f32 = (cfg->flags & ZC_FLAG_OUT_F32) ? 1 : 0;
   lay->kch = cfg->k_scheme == ZC_K_CHANNEL ? 1 : 0;
   lay->p16 = (cfg->flags & ZC_FLAG_PARAMS_F16) ? 1 : 0;
+  lay->grp_all = (cfg->flags & ZC_FLAG_GROUP_ALL_HEADS) ? 1 : 0;
   lay->bits[0] = cfg->bits_hi;
   lay->bits[1] = cfg->bits_lo;
   const int max_flush = cfg->max_new_tokens / cfg->window;
@@ -91,6 +98,8 @@ void make_layout(const zc_config* cfg, ZcLayout* lay, size_t* cache_bytes, size_
   off = align_up(off + (size_t)std::max(cfg->max_prefill, cfg->window) * 4, 256);
   lay->off_idx = (long long)off;
   off = align_up(off + ((size_t)cfg->max_prefill + (size_t)max_flush * cfg->window) * 4, 256);
+  lay->off_tokmm = (long long)off;   // only with token groups over all heads (the other layouts stay as they were)
+  if (lay->grp_all) off = align_up(off + (size_t)std::max(cfg->max_prefill, cfg->window) * 16, 256);
   lay->unit_stride = (long long)off;
   if (cache_bytes) *cache_bytes = off * (size_t)lay->units;
   if (ws_bytes) {

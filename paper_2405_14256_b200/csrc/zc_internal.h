@@ -42,6 +42,7 @@ struct ZcLayout {
   int out_f32;            // decode outputs are stored as fp32 (ZC_FLAG_OUT_F32)
   int kch;                // keys are quantised channelwise (ZC_K_CHANNEL): no per-token key parameters
   int p16;                // ZC_FLAG_PARAMS_F16: per-token parameters as (fp16 scale, int16 zero) pairs
+  int grp_all;            // ZC_FLAG_GROUP_ALL_HEADS: a token's (s, z) over the channels of all KV heads of its batch row
   int bits[2];
   int tile_bytes[2];
   int cap_tiles[2];
@@ -49,7 +50,7 @@ struct ZcLayout {
   int idx_cap0;
   long long unit_stride;
   long long off_tiles[2], off_fac, off_cmax, off_tailK, off_tailV, off_colsum, off_sync, off_scores,
-      off_idx;
+      off_idx, off_tokmm;   // off_tokmm: [tokens of a subset] x (min K, max K, min V, max V) of y = x / c over all heads (grp_all; kept by the row's first unit)
 };
 
 // Where the rows to compress come from (caller tensors at prefill, the tail at a flush).

@@ -11,18 +11,26 @@
 // z = -rint(mn / s); code = clamp(rint(y / s) + z, 0, L).
 // P16 (ZC_FLAG_PARAMS_F16): the scale is rounded UP to the next fp16 value before z and the codes
 // are formed (the caller has done the same to c).
+// mm (ZC_FLAG_GROUP_ALL_HEADS): the token's minimum and maximum of y over the channels of all KV
+// heads of its batch row, taken beforehand, in place of this head's own.
 template <bool P16 = false>
 static __device__ __forceinline__ void quant_token(const float (&x)[4], const float (&c)[4], float L,
-                                            float* s_out, float* z_out, unsigned* codes4) {
+                                            float* s_out, float* z_out, unsigned* codes4,
+                                            const float* mm = nullptr) {
   float y[4];
 #pragma unroll
   for (int e = 0; e < 4; ++e) y[e] = __fdiv_rn(x[e], c[e]);
   float mn = fminf(fminf(y[0], y[1]), fminf(y[2], y[3]));
   float mx = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
+  if (mm) {
+    mn = mm[0];
+    mx = mm[1];
+  } else {
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int o = 16; o > 0; o >>= 1) {
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
   }
   float s = __fdiv_rn(__fsub_rn(mx, mn), L);
   if (mx == mn) s = mn != 0.f ? fabsf(mn) : 1.f;
@@ -71,9 +79,20 @@ static __device__ __noinline__ float4 quant_token_ieee(float4 xv, float4 cv, flo
   else quant_token<false>(x, c, L, &s, &z, &pk);
   return make_float4(s, z, __uint_as_float(pk), 0.f);
 }
+static __device__ __noinline__ float4 quant_token_ieee_shared(float4 xv, float4 cv, float L, bool p16, float mn_sh,
+                                                              float mx_sh) {
+  const float x[4] = {xv.x, xv.y, xv.z, xv.w}, c[4] = {cv.x, cv.y, cv.z, cv.w};
+  const float mm[2] = {mn_sh, mx_sh};
+  float s, z;
+  unsigned pk;
+  if (p16) quant_token<true>(x, c, L, &s, &z, &pk, mm);
+  else quant_token<false>(x, c, L, &s, &z, &pk, mm);
+  return make_float4(s, z, __uint_as_float(pk), 0.f);
+}
 static __device__ __forceinline__ void quant_token_rc(const float (&x)[4], const float (&c)[4], const float (&rc)[4],
                                                       bool c_mid, float L, float rL, float* s_out, float* z_out,
-                                                      unsigned* codes4, bool p16 = false) {
+                                                      unsigned* codes4, bool p16 = false, bool shared = false,
+                                                      float mn_sh = 0.f, float mx_sh = 0.f) {
   const bool mine = c_mid && zc_mid(x[0]) && zc_mid(x[1]) && zc_mid(x[2]) && zc_mid(x[3]);
   if (__all_sync(0xffffffffu, mine)) {
     float y[4];
@@ -81,15 +100,22 @@ static __device__ __forceinline__ void quant_token_rc(const float (&x)[4], const
     for (int e = 0; e < 4; ++e) y[e] = zc_div_by(x[e], c[e], rc[e]);
     float mn = fminf(fminf(y[0], y[1]), fminf(y[2], y[3]));
     float mx = fmaxf(fmaxf(y[0], y[1]), fmaxf(y[2], y[3]));
+    bool range_ok = true;
+    if (shared) {   // the row's statistics over all heads: other heads' values must be in range as well
+      mn = mn_sh;
+      mx = mx_sh;
+      range_ok = zc_mid(mn) && zc_mid(mx);
+    } else {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      for (int o = 16; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      }
     }
     float s = zc_div_by(__fsub_rn(mx, mn), L, rL);   // 0 when mx == mn, replaced below
     if (mx == mn) s = fabsf(mn);                     // mn != 0 here
     if (p16) s = __half2float(__float2half_ru(s));   // stored as fp16: never below the exact scale
-    if (zc_mid(s)) {                                 // the same for every lane
+    if (range_ok && zc_mid(s)) {                     // the same for every lane
       const float rs = __frcp_rn(s);
       const float z = -rintf(zc_div_by(mn, s, rs));
       unsigned packed = 0;
@@ -105,7 +131,8 @@ static __device__ __forceinline__ void quant_token_rc(const float (&x)[4], const
       return;
     }
   }
-  const float4 r = quant_token_ieee(make_float4(x[0], x[1], x[2], x[3]), make_float4(c[0], c[1], c[2], c[3]), L, p16);
+  const float4 xv = make_float4(x[0], x[1], x[2], x[3]), cv = make_float4(c[0], c[1], c[2], c[3]);
+  const float4 r = shared ? quant_token_ieee_shared(xv, cv, L, p16, mn_sh, mx_sh) : quant_token_ieee(xv, cv, L, p16);
   *s_out = r.x;
   *z_out = r.y;
   *codes4 = __float_as_uint(r.z);

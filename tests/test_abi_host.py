@@ -60,7 +60,9 @@ def test_cache_bytes_cover_the_algorithmic_bytes(zc):
     dict(saliency_ratio=1.5), dict(n_q_heads=6), dict(batch=0), dict(n_q_heads=72, n_kv_heads=8),
     dict(scope=2), dict(scope=1, flags=2),   # token scope cannot be combined with ZC_FLAG_OVERLAP_CALLS (2)
     # ZC_FLAG_PARAMS_F16 (8): not with overlapping calls, channelwise keys, or classes other than 2 / 4 bits
-    dict(flags=8 | 2), dict(flags=8, k_scheme=1), dict(flags=8, bits_hi=16), dict(flags=8, bits_lo=8), dict(flags=16),
+    dict(flags=8 | 2), dict(flags=8, k_scheme=1), dict(flags=8, bits_hi=16), dict(flags=8, bits_lo=8), dict(flags=32),
+    # ZC_FLAG_GROUP_ALL_HEADS (16): needs token scope, no 16-bit class
+    dict(flags=16), dict(flags=16, scope=1, bits_hi=16),
 ])
 def test_invalid_configurations_are_rejected(zc, bad):
     kw = dict(dtype=torch.float16, batch=2, n_q_heads=8, n_kv_heads=8, max_prefill=256,

@@ -957,3 +957,49 @@ def test_params_f16_full_size_one_call_at_a_time():
         assert tl.compare_segment(cache, oc, seg, units) == 0
     tl.record("full size, 16-bit parameters, one call at a time", config=2, units=len(units), steps=103,
               max_abs_out=worst)
+
+
+# ---------------------------------------------------------------- token groups over all heads (ZC_FLAG_GROUP_ALL_HEADS)
+@pytest.mark.parametrize("kw,p16", [
+    (dict(context=260, batch=2, n_q_heads=8, n_kv_heads=4), False),
+    (dict(context=150, n_q_heads=8, n_kv_heads=2, dtype="bf16", outlier_fixed=0, bits_hi=4, bits_lo=4), False),
+    (dict(context=97, n_q_heads=4, n_kv_heads=4, bits_hi=8, bits_lo=2, saliency_ratio=0.5), False),
+    (dict(context=200, batch=2, n_q_heads=8, n_kv_heads=2, k_scheme="channel"), False),
+    (dict(context=130, n_q_heads=8, n_kv_heads=4), True),
+])
+def test_token_groups_over_all_heads_across_two_windows(kw, p16):
+    """Alg. 1 on X in R^{l x hd}: one (s, z) per token over the channels of all KV heads of its
+    batch row, in the prompt and in two re-compressed windows: every head's tiles carry the
+    row's pair, codes, parameters and factors equal to the oracle's (scope="token",
+    group="all_heads"), decode within the bound at every step."""
+    from workloads import make_decode_step
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(window=16, decode_steps=40, rho_recent=0.2, rho_random=0.2, **kw)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    K[:, -1] *= 5.0            # heads of unlike range: the shared scale is the widest head's
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w, scope="token", group="all_heads", param_dtype="f16" if p16 else "f32")
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w, max_new=40, token_scope=True, group_all_heads=True, params_f16=p16)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    assert tl.compare_segment(cache, oc, 0) == 0
+    sz = cache.segment(0, 1, 0)[2].cpu().numpy()          # V parameters of the salient subset
+    for bi in range(w.batch):
+        for kv in range(1, w.n_kv_heads):
+            np.testing.assert_array_equal(sz[bi, kv], sz[bi, 0])      # one pair per token for every head
+    for step in range(35):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        probe = step % 3 == 0
+        cache.append(k, v)
+        out = cache.decode_attention(q, probe)
+        oc.append(tl.to64(k), tl.to64(v))
+        ref = oc.decode_attention(tl.to64(q), probe)
+        torch.cuda.synchronize()
+        got = out.float().cpu().numpy()
+        for (bi, kv), r in ref.items():
+            assert tl.output_excess(got[bi, kv * oc.G:(kv + 1) * oc.G], r, w.torch_dtype) <= 0.0
+    assert zc.zc_num_segments(cache.handle) == 3 and zc.zc_device_status() == 0
+    for seg in (1, 2):
+        assert tl.compare_segment(cache, oc, seg) == 0
+    cache.check_guards()

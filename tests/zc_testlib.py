@@ -36,10 +36,11 @@ def make_cache(w: Workload, max_new=None, defer_append: bool = False, overlap_ca
                        **kw)
 
 
-def make_oracle(w: Workload, units=None, scope: str = "kv_head", param_dtype: str = "f32") -> zo.ZipCacheOracle:
+def make_oracle(w: Workload, units=None, scope: str = "kv_head", param_dtype: str = "f32",
+                group: str = "head") -> zo.ZipCacheOracle:
     return zo.ZipCacheOracle(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.saliency_ratio,
                              w.bits_hi, w.bits_lo, w.window, units=units, k_scheme=w.k_scheme, scope=scope,
-                             param_dtype=param_dtype)
+                             param_dtype=param_dtype, group=group)
 
 
 def probes_for(w: Workload, layer: int = 0) -> np.ndarray:
