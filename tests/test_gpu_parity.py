@@ -1003,3 +1003,53 @@ def test_token_groups_over_all_heads_across_two_windows(kw, p16):
     for seg in (1, 2):
         assert tl.compare_segment(cache, oc, seg) == 0
     cache.check_guards()
+
+
+def test_token_scope_all_heads_full_size_one_call_at_a_time():
+    """Workload 2 with one split per token and one (s, z) per token over all KV heads, in the
+    launch mode they admit, on every head of one batch row (the oracle needs the whole row),
+    through one re-compressed window."""
+    from workloads import make_decode_step, decode_probe_flags
+    import paper_2405_14256_b200 as zc
+    w = get_config(2)
+    units = [(5, kv) for kv in range(w.n_kv_heads)]
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w, units, scope="token", group="all_heads")
+    oc.prefill_compress(*tl.oracle_inputs(w, Q, K, V, units), P)
+    cache = tl.make_cache(w, max_new=104, defer_append=True, token_scope=True, group_all_heads=True)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    p_gpu = cache.scores(w.context).cpu().numpy()
+    idx_hi = cache.segment(0, 0, 0)[0].cpu().numpy()
+    s0 = oc.units[units[0]].segments[0]
+    assert (np.abs(p_gpu[5, 0] - s0.p_tilde) / np.maximum(np.abs(s0.p_tilde), 1e-30)).max() <= 1e-4
+    swaps = tl.salient_sets_match(p_gpu[5, 0], s0.p_tilde, idx_hi[5, 0], s0.hi.idx, s0.hi.n)
+    flags = decode_probe_flags(w, 0, 103)
+    worst = 0.0
+    for step in range(103):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        probe = bool(flags[step])
+        cache.append(k, v)
+        out = cache.decode_attention(q, probe)
+        qq, kk, vv = tl.oracle_step_inputs(w, q, k, v, units)
+        oc.append(kk, vv)
+        ref = oc.decode_attention(qq, probe)
+        if swaps:
+            continue
+        got = out.float().cpu().numpy()
+        for (bi, kv), r in ref.items():
+            g = got[bi, kv * oc.G:(kv + 1) * oc.G]
+            assert tl.output_excess(g, r, w.torch_dtype) <= 0.0
+            worst = max(worst, float(np.abs(g - r).max()))
+    assert zc.zc_num_segments(cache.handle) == 2 and zc.zc_device_status() == 0
+    exact = 0
+    if swaps == 0:
+        assert tl.compare_segment(cache, oc, 0, units) == 0
+        exact = len(units)
+        sg = oc.units[units[0]].segments[1]
+        ihi = cache.segment(1, 0, 0)[0].cpu().numpy()
+        if set(ihi[5, 0].tolist()) == set(sg.hi.idx.tolist()):
+            assert tl.compare_segment(cache, oc, 1, units) == 0
+    tl.record("full size, token scope and token groups over all heads, one call at a time", config=2,
+              units=len(units), steps=103, max_abs_out=worst, near_tie_swaps=swaps, units_code_exact=exact)
