@@ -128,3 +128,35 @@ def test_noalloc_calls_back_to_back_without_synchronising():
             assert torch.equal(x, y)
     for x, y in zip(results[0][1], results[1][1]):
         assert torch.equal(x, y)
+
+
+def test_noalloc_entry_against_the_oracle():
+    """The no-allocation call compared with the oracle itself (not only with the workspace
+    call): every output within the decode bound over two re-compressed windows, and the
+    windows' lists, codes and parameters equal to the oracle's."""
+    import numpy as np
+    import paper_2405_14256_b200 as zc
+    w = tl.small_workload(context=260, batch=2, n_q_heads=8, n_kv_heads=2, window=16, rho_recent=0.2,
+                          rho_random=0.2)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    cache = tl.make_cache(w, max_new=40)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    for step in range(35):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        probe = step % 3 == 0
+        cache.append(k, v)
+        got = torch.empty_like(q)
+        zc.zc_decode_attention_noalloc(cache.handle, q, got, probe)
+        oc.append(tl.to64(k), tl.to64(v))
+        ref = oc.decode_attention(tl.to64(q), probe)
+        torch.cuda.synchronize()
+        g = got.float().cpu().numpy()
+        for (bi, kv), r in ref.items():
+            assert tl.output_excess(g[bi, kv * oc.G:(kv + 1) * oc.G], r, w.torch_dtype) <= 0.0, step
+    assert zc.zc_num_segments(cache.handle) == 3 and zc.zc_device_status() == 0
+    for seg in range(3):
+        assert tl.compare_segment(cache, oc, seg) == 0
+    assert cache.check_guards()
