@@ -185,6 +185,7 @@ def test_decode_attention_parity(kw, steps):
     (100, 105, 0.8),                  # 80 salient tokens: more than one tile in a class
     (16, 20, 0.0), (16, 20, 1.0),     # an empty class
     (128, 130, 0.5),                  # the largest window, both tiles full
+    (8, 323, 0.4),                    # forty windows: 82 items per unit and call at the end
 ])
 def test_decode_across_window_recompression(window, steps, ratio):
     """The tail is re-compressed after `window` steps: new segment codes must be bit-exact
@@ -1053,3 +1054,65 @@ def test_token_scope_all_heads_full_size_one_call_at_a_time():
             assert tl.compare_segment(cache, oc, 1, units) == 0
     tl.record("full size, token scope and token groups over all heads, one call at a time", config=2,
               units=len(units), steps=103, max_abs_out=worst, near_tie_swaps=swaps, units_code_exact=exact)
+
+
+@pytest.mark.parametrize("opts", [
+    dict(token_scope=True), dict(params_f16=True),
+    dict(token_scope=True, group_all_heads=True, params_f16=True),
+])
+def test_window_recompression_by_kernels_behind_the_call_inside_a_cuda_graph(opts):
+    """Token scope and 16-bit parameters re-compress a window by kernels launched behind the
+    decode kernel of the completing call.  36 steps (two windows) captured into one CUDA graph
+    and replayed must leave the same outputs and the same cache, byte for byte, as the same calls
+    issued directly (which the tests above compare with the oracle)."""
+    import paper_2405_14256_b200 as zc
+    from workloads import make_decode_step
+    w = tl.small_workload(context=260, batch=2, n_q_heads=8, n_kv_heads=2, window=16, rho_recent=0.2,
+                          rho_random=0.2)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w).tolist()
+    n = 36
+    ins = [make_decode_step(w, 0, s, tl.DEV) for s in range(n)]
+    res = {}
+    for mode in ("direct", "graph"):
+        c = tl.make_cache(w, max_new=40, defer_append=True, **opts)
+        c.mem.zero_()
+        c.prefill_compress(Q, K, V, P)
+        outs = [torch.empty_like(ins[0][0]) for _ in range(n)]
+
+        def issue():
+            for s in range(n):
+                q, k, v = ins[s]
+                c.append(k, v)
+                c.decode_attention(q, s % 3 == 0, out=outs[s])
+
+        torch.cuda.synchronize()
+        if mode == "graph":
+            st = torch.cuda.Stream()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(st):
+                with torch.cuda.graph(g, stream=st):
+                    issue()
+                g.replay()
+        else:
+            issue()
+        torch.cuda.synchronize()
+        assert zc.zc_num_segments(c.handle) == 3 and zc.zc_device_status() == 0
+        assert c.check_guards()
+        res[mode] = (torch.stack(outs).clone(), c.mem.clone())
+    assert torch.equal(res["direct"][0], res["graph"][0])
+    assert torch.equal(res["direct"][1], res["graph"][1])
+
+
+@pytest.mark.parametrize("graph", [False, True])
+def test_forty_windows_with_calls_side_by_side(graph):
+    """A long generation in the benchmark's launch mode: window 8, 323 steps, so every unit's
+    one CTA ends up working through 82 items per call; outputs within the bound at every step,
+    all 41 segments equal to the oracle's (up to near-tie splits, which are counted)."""
+    w = tl.small_workload(context=150, batch=2, n_q_heads=4, n_kv_heads=2, window=8, rho_recent=0.1,
+                          rho_random=0.1)
+    units = [(bi, kv) for bi in range(w.batch) for kv in range(w.n_kv_heads)]
+    r = tl.run_benchmark_mode(w, units, 323, layers=2, graph=graph)
+    assert r["excess"] <= 0.0, r["excess"]
+    import paper_2405_14256_b200 as zc
+    assert all(zc.zc_num_segments(c.handle) == 41 for c in r["caches"])
