@@ -1116,3 +1116,50 @@ def test_forty_windows_with_calls_side_by_side(graph):
     assert r["excess"] <= 0.0, r["excess"]
     import paper_2405_14256_b200 as zc
     assert all(zc.zc_num_segments(c.handle) == 41 for c in r["caches"])
+
+
+@pytest.mark.parametrize("l,G,rho", [(262144, 2, 0.002), (1 << 20, 1, 0.0005)])
+def test_longest_prompts(l, G, rho):
+    """One unit at 2^18 tokens and at 2^20, the largest max_prefill the library accepts (about a
+    thousand probe rows, so that the oracle finishes in seconds): scores, the split, every packed
+    code and parameter, and three decode steps over the whole cache."""
+    import paper_2405_14256_b200 as zc
+    from workloads import make_decode_step
+    w = tl.small_workload(context=l, batch=1, n_q_heads=G, n_kv_heads=1, dtype="bf16", rho_recent=rho,
+                          rho_random=rho, decode_steps=4)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    cache = tl.make_cache(w, max_new=4, defer_append=True)
+    cache.prefill_compress(Q, K, V, P.tolist())
+    torch.cuda.synchronize()
+    assert zc.zc_device_status() == 0
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    swaps, clean, rel = tl.compare_prefill_segment(w, cache, oc, [(0, 0)])
+    worst = 0.0
+    for step in range(3):
+        q, k, v = make_decode_step(w, 0, step, tl.DEV)
+        cache.append(k, v)
+        out = cache.decode_attention(q, step == 1)
+        oc.append(tl.to64(k), tl.to64(v))
+        ref = oc.decode_attention(tl.to64(q), step == 1)
+        torch.cuda.synchronize()
+        if swaps == 0:
+            g = out.float().cpu().numpy()[0]
+            worst = max(worst, tl.output_error(g, ref[(0, 0)]))
+            assert worst <= tl.TOL_OUT, (step, worst)
+    assert zc.zc_device_status() == 0 and cache.check_guards()
+    tl.record(f"one unit, {l} tokens", units=1, steps=3, max_abs_out=worst, near_tie_swaps=swaps,
+              units_code_exact=clean, score_rel=rel)
+
+
+def test_many_units():
+    """4096 units (batch 512 x 8 KV heads, 32 query heads) of 300 tokens through one re-compressed
+    window: several times more units than CTA slots on the GPU; sampled units against the oracle."""
+    w = tl.small_workload(context=300, batch=512, n_q_heads=32, n_kv_heads=8, window=16, rho_recent=0.1,
+                          rho_random=0.1, dtype="bf16")
+    units = [(0, 0), (1, 7), (255, 3), (256, 4), (511, 0), (511, 7)]
+    worst, cache, oc = tl.run_decode_parity(w, 20, units=units, staged=False, defer_append=True)
+    import paper_2405_14256_b200 as zc
+    assert zc.zc_num_segments(cache.handle) == 2 and zc.zc_device_status() == 0
+    assert tl.compare_segment(cache, oc, 0, units) == 0
