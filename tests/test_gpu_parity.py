@@ -1163,3 +1163,31 @@ def test_many_units():
     import paper_2405_14256_b200 as zc
     assert zc.zc_num_segments(cache.handle) == 2 and zc.zc_device_status() == 0
     assert tl.compare_segment(cache, oc, 0, units) == 0
+
+
+def test_prefill_attention_statistics_at_2_18_tokens():
+    """zc_prefill_attention over 2^18 tokens: its row statistics, given to
+    zc_prefill_compress_lse, must lead to the oracle's scores, split and codes (every probe row's
+    log-sum-exp is then right to the score tolerance), and O's first 300 rows must be the
+    oracle's attention over the same prefix (causal: later tokens do not touch them)."""
+    import paper_2405_14256_b200 as zc
+    l = 262144
+    w = tl.small_workload(context=l, batch=1, n_q_heads=2, n_kv_heads=1, dtype="bf16", rho_recent=0.002,
+                          rho_random=0.002)
+    Q, K, V = make_prefill(w, 0, tl.DEV)
+    P = tl.probes_for(w)
+    cache = tl.make_cache(w, max_new=4)
+    O, lse = cache.prefill_attention(Q, K, V)
+    cache.prefill_compress_lse(Q, K, V, P.tolist(), lse)
+    torch.cuda.synchronize()
+    assert zc.zc_device_status() == 0 and cache.check_guards()
+    oc = tl.make_oracle(w)
+    oc.prefill_compress(tl.to64(Q), tl.to64(K), tl.to64(V), P)
+    swaps, clean, rel = tl.compare_prefill_segment(w, cache, oc, [(0, 0)])
+    n = 300
+    for h in range(2):
+        O_ref, lse_ref = zo.prefill_attention(tl.to64(Q[0, h, :n]), tl.to64(K[0, 0, :n]), tl.to64(V[0, 0, :n]))
+        assert np.abs(tl.to64(O[0, h, :n]) - O_ref).max() <= 2e-2
+        assert np.abs(lse[0, h, :n].double().cpu().numpy() - lse_ref).max() <= 2e-4
+    tl.record("prefill attention statistics, 262144 tokens", units=1, near_tie_swaps=swaps, units_code_exact=clean,
+              score_rel=rel)
